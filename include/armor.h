@@ -1,0 +1,162 @@
+/*
+ * armor.h -- C ABI of the B200 (sm_100a) implementation of ARMOR's per-layer
+ * block coordinate descent (arXiv 2510.05528).
+ *
+ * One linear layer W [d_out, d_in] is factorised as  W ~ A * S * B  with
+ * block-diagonal wrappers A, B (blocks of d_block x d_block) around an N:M
+ * sparse core S = W' (.) M  (Section 3.1 of the paper).  The library minimises
+ * the layer-wise proxy loss  L = tr(E H_w E^T),  E = W - A S B,  where
+ * H_w = diag(X^T X) is the paper's weighting (Eq. proxy_loss, Section 3.2) and
+ * H_w = X^T X is the full-Gram generalisation this build is timed on.
+ *
+ * Conventions for every call
+ *   - All d_* pointers are DEVICE pointers owned by the caller; tensors are
+ *     row-major and contiguous unless a leading dimension is given.
+ *   - The library allocates no device memory.  Scratch comes from the
+ *     workspace handed to armor_create (size from armor_workspace_bytes).
+ *   - Work is enqueued on the given stream; no call synchronises the device.
+ *     Calls on one context must be issued in stream order (they share the
+ *     workspace).
+ *   - Argument errors are returned immediately.  Conditions found on the
+ *     device (a block that is not positive definite, a bounded wait that ran
+ *     out) are recorded in a device status buffer; read it with
+ *     armor_get_device_status after synchronising the stream yourself.
+ *   - A, B: [d/d_block, d_block, d_block] fp32.  S: [d_out, d_in] fp32 with
+ *     zeros outside the mask.  M: one byte per group of m_group consecutive
+ *     columns, uint8 [d_out, d_in/m_group]; bit p set <=> column m*c+p kept.
+ */
+#ifndef ARMOR_H
+#define ARMOR_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct armor_ctx armor_ctx;
+typedef struct CUstream_st* armor_stream_t; /* == cudaStream_t */
+
+typedef enum {
+  ARMOR_OK = 0,
+  ARMOR_ERR_INVALID_ARG = 1,
+  ARMOR_ERR_SHAPE = 2,
+  ARMOR_ERR_WORKSPACE = 3,
+  ARMOR_ERR_CUDA = 4,
+  ARMOR_ERR_NOT_SPD = 5,
+  ARMOR_ERR_TIMEOUT = 6,
+  ARMOR_ERR_UNSUPPORTED = 7
+} armor_status;
+
+enum { ARMOR_H_FULL = 0, ARMOR_H_DIAG = 1 };
+enum { ARMOR_SELECT_L1_RANDOM = 0, ARMOR_SELECT_L1_GREEDY = 1 };
+enum { ARMOR_S_EXACT = 0, ARMOR_S_BETA = 1 };
+/* How the dense contractions (Gram, .H) are evaluated on the tensor cores:
+ *   FP32X3 : operands split into tf32 high and low parts, three tcgen05 passes
+ *            accumulated in fp32 -- fp32-grade results (the parity mode);
+ *   TF32   : one pass, operands rounded to tf32 (10-bit mantissa);
+ *   SIMT   : fp32 CUDA-core reference path (slow; for debugging and checks). */
+enum { ARMOR_PREC_FP32X3 = 0, ARMOR_PREC_TF32 = 1, ARMOR_PREC_SIMT = 2 };
+enum { ARMOR_PHASE_A = 1, ARMOR_PHASE_B = 2, ARMOR_PHASE_S = 4, ARMOR_PHASE_MASK = 8 };
+enum { ARMOR_DTYPE_F32 = 0, ARMOR_DTYPE_BF16 = 1 };
+
+typedef struct {
+  int64_t d_out, d_in;
+  int32_t d_block;     /* divides d_out and d_in; multiple of m_group */
+  int32_t n_keep;      /* N of N:M (2) */
+  int32_t m_group;     /* M of N:M (4) */
+  int32_t h_mode;      /* ARMOR_H_* */
+  int32_t select_mode; /* ARMOR_SELECT_* (Section 3.3.2 / Appendix E.1) */
+  int32_t s_step;      /* ARMOR_S_* */
+  int32_t precision;   /* ARMOR_PREC_* */
+  int32_t normalize;   /* 1: armor_init applies the NoWag normalisation */
+  int32_t phases;      /* bitmask of ARMOR_PHASE_*; 0 means all four */
+  float ridge;         /* relative proximal ridge of the block solves (1e-6) */
+  uint64_t seed;       /* seed of the counter-based group selection */
+} armor_config;
+
+/* One record per BCD iteration, written on the device.  The losses after the
+ * sub-steps follow from loss_start by the exact decrease of each quadratic
+ * step; loss_start itself is evaluated from the residual. */
+typedef struct {
+  double loss_start, loss_A, loss_B, loss_S, loss_mask;
+  double delta_L_mask;   /* exact loss change of the iteration's group updates */
+  float tau_B, tau_S;    /* exact step lengths of the B-step and S-step */
+  int32_t groups_changed;/* groups whose mask changed (0 if rejected) */
+  int32_t mask_accepted; /* 1 if the group updates were kept */
+  int32_t chol_failed;   /* blocks skipped because a Cholesky pivot was <= 0 */
+  int32_t reserved;
+} armor_iter_stats;
+
+/* Scratch size for a configuration.  Error: INVALID_ARG (null), SHAPE
+ * (d_block does not divide the dims, m_group does not divide d_block),
+ * UNSUPPORTED (N:M other than 2:4, d_block > 128 or not a multiple of 32). */
+armor_status armor_workspace_bytes(const armor_config* cfg, size_t* bytes);
+
+/* Creates a context over caller-owned device scratch (256-byte aligned, at
+ * least armor_workspace_bytes).  The context holds the configuration and the
+ * carve-up of the workspace only.  Must be called with the device current. */
+armor_status armor_create(armor_ctx** ctx, const armor_config* cfg, void* d_workspace, size_t bytes);
+armor_status armor_destroy(armor_ctx* ctx);
+
+/* Calibration Gram (Section 2 / Eq. proxy_loss: its diagonal is ||X_j||^2).
+ * d_H [d_in, d_in] fp32 += X^T X for a chunk X [n_rows, d_in] with leading
+ * dimension ldx (elements).  The caller zeroes d_H before the first chunk.
+ * x_dtype: ARMOR_DTYPE_F32.  n_rows == 0 is a no-op. */
+armor_status armor_gram(armor_ctx* ctx, const void* d_X, int32_t x_dtype, int64_t n_rows, int64_t ldx,
+                        float* d_H, armor_stream_t stream);
+
+/* Normalisation and initialisation (Section 3.2 display after Eq. proxy_loss;
+ * Eq. init): optionally W_bar = W / r1 / r2 (zero norms read as 1), then
+ * A = B = I, M = top-n_keep of every group by W_bar^2 * H_jj (ties keep the
+ * lower column), S = W_bar (.) M.  d_Wbar receives the matrix the later calls
+ * take as W (a copy of d_W when cfg.normalize == 0; may alias d_W).  d_r1
+ * [d_in], d_r2 [d_out] are written only when cfg.normalize == 1 (else may be
+ * NULL). */
+armor_status armor_init(armor_ctx* ctx, const float* d_W, const float* d_H, float* d_Wbar, float* d_r1,
+                        float* d_r2, float* d_A, float* d_B, float* d_S, uint8_t* d_M,
+                        armor_stream_t stream);
+
+/* n_iters iterations of Algorithm 1's loop, numbered t_first .. t_first +
+ * n_iters - 1: A-step, B-step, S-step (the continuous update of Algorithm 2,
+ * with exact block solves / exact line searches in place of the 1/beta
+ * gradient steps) and the greedy sparse-core update of Algorithm 3 (one group
+ * per block, closed-form solve over all masks, Eq. mask_loss_opt and
+ * mask_loss_opt_sol).  A, B, S, M are updated in place.  d_stats may be NULL,
+ * else [n_iters].  Each iteration is a function of (state, W, H, t) only, so
+ * splitting a run into several calls gives the same bits. */
+armor_status armor_bcd_step(armor_ctx* ctx, const float* d_Wbar, const float* d_H, float* d_A, float* d_B,
+                            float* d_S, uint8_t* d_M, int64_t t_first, int32_t n_iters,
+                            armor_iter_stats* d_stats, armor_stream_t stream);
+
+/* Proxy loss L = tr(E H_w E^T), E = W - A S B (Eq. proxy_loss; full-Gram form
+ * when h_mode == FULL), written to *d_loss (device, double). */
+armor_status armor_proxy_loss(armor_ctx* ctx, const float* d_Wbar, const float* d_H, const float* d_A,
+                              const float* d_B, const float* d_S, double* d_loss, armor_stream_t stream);
+
+/* Deployment form (Section 3.1): y_t = A (S (B x_t)) for the rows of
+ * x [n_tokens, d_in] -> y [n_tokens, d_out].  With d_r1, d_r2 non-NULL the
+ * normalisation is undone: y_t = r2 (.) A S B (r1 (.) x_t).  xy_dtype:
+ * ARMOR_DTYPE_F32.  d_M is accepted for symmetry and may be NULL (S already
+ * carries the zeros). */
+armor_status armor_apply(armor_ctx* ctx, const float* d_A, const float* d_B, const float* d_S,
+                         const uint8_t* d_M, const float* d_r1, const float* d_r2, const void* d_x,
+                         void* d_y, int32_t xy_dtype, int64_t n_tokens, armor_stream_t stream);
+
+/* Copies up to n device status words to h_codes (host).  Word 0: number of
+ * Cholesky failures since the context was created; word 1: first failing
+ * block id + 1; word 2: bounded waits that gave up; word 3: last
+ * armor_status recorded by a kernel.  The caller must have synchronised the
+ * stream the context's work ran on.  (This call itself copies synchronously.) */
+armor_status armor_get_device_status(armor_ctx* ctx, int32_t* h_codes, int32_t n);
+
+const char* armor_status_string(armor_status s);
+
+/* Number of kernel launches the context has enqueued so far (host counter). */
+int64_t armor_launch_count(const armor_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ARMOR_H */

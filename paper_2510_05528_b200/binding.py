@@ -1,0 +1,264 @@
+"""ctypes binding of libarmor (see include/armor.h).  Argument marshalling only: every step of the
+method runs in the library's CUDA kernels.  PyTorch supplies device memory and streams.
+
+The module-level functions carry the names of the C entry points and take torch CUDA tensors.
+``ArmorContext`` bundles a configuration with its workspace.  There is no CPU path: if the shared
+library is missing, or a tensor is not on a CUDA device, the call raises."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libarmor.so")
+
+H_FULL, H_DIAG = 0, 1
+SELECT_L1_RANDOM, SELECT_L1_GREEDY = 0, 1
+S_EXACT, S_BETA = 0, 1
+PREC_FP32X3, PREC_TF32, PREC_SIMT = 0, 1, 2
+PHASE_A, PHASE_B, PHASE_S, PHASE_MASK = 1, 2, 4, 8
+DTYPE_F32, DTYPE_BF16 = 0, 1
+
+EXPORTS = ["armor_workspace_bytes", "armor_create", "armor_destroy", "armor_gram", "armor_init",
+           "armor_bcd_step", "armor_proxy_loss", "armor_apply", "armor_get_device_status",
+           "armor_status_string", "armor_launch_count"]
+
+
+class ArmorError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+class armor_config(C.Structure):
+    _fields_ = [("d_out", C.c_int64), ("d_in", C.c_int64), ("d_block", C.c_int32), ("n_keep", C.c_int32),
+                ("m_group", C.c_int32), ("h_mode", C.c_int32), ("select_mode", C.c_int32),
+                ("s_step", C.c_int32), ("precision", C.c_int32), ("normalize", C.c_int32),
+                ("phases", C.c_int32), ("ridge", C.c_float), ("seed", C.c_uint64)]
+
+
+STATS_DTYPE = np.dtype([("loss_start", "<f8"), ("loss_A", "<f8"), ("loss_B", "<f8"), ("loss_S", "<f8"),
+                        ("loss_mask", "<f8"), ("delta_L_mask", "<f8"), ("tau_B", "<f4"), ("tau_S", "<f4"),
+                        ("groups_changed", "<i4"), ("mask_accepted", "<i4"), ("chol_failed", "<i4"),
+                        ("reserved", "<i4")])
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libarmor.so on first use; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(f"{LIB_PATH} not found: build it with `python -m paper_2510_05528_b200.build`")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
+        L.armor_workspace_bytes.argtypes = [C.POINTER(armor_config), C.POINTER(C.c_size_t)]
+        L.armor_create.argtypes = [C.POINTER(vp), C.POINTER(armor_config), vp, C.c_size_t]
+        L.armor_destroy.argtypes = [vp]
+        L.armor_gram.argtypes = [vp, vp, i32, i64, i64, vp, vp]
+        L.armor_init.argtypes = [vp] + [vp] * 9 + [vp]
+        L.armor_bcd_step.argtypes = [vp] + [vp] * 6 + [i64, i32, vp, vp]
+        L.armor_proxy_loss.argtypes = [vp] + [vp] * 6 + [vp]
+        L.armor_apply.argtypes = [vp] + [vp] * 8 + [i32, i64, vp]
+        L.armor_get_device_status.argtypes = [vp, C.POINTER(i32), i32]
+        L.armor_status_string.argtypes = [C.c_int]
+        L.armor_status_string.restype = C.c_char_p
+        L.armor_launch_count.argtypes = [vp]
+        L.armor_launch_count.restype = i64
+        for name in EXPORTS:
+            if name not in ("armor_status_string", "armor_launch_count"):
+                getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().armor_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != 0:
+        raise ArmorError(code, where)
+
+
+def _ptr(t: torch.Tensor | None, dtype=None, name: str = "tensor") -> C.c_void_p:
+    if t is None:
+        return C.c_void_p(0)
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (this library has no CPU path)")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"{name} must have dtype {dtype}, got {t.dtype}")
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream() -> C.c_void_p:
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def make_config(d_out, d_in, d_block, *, n_keep=2, m_group=4, h_mode=H_FULL, select_mode=SELECT_L1_RANDOM,
+                s_step=S_EXACT, precision=PREC_FP32X3, normalize=0, phases=0, ridge=1e-6, seed=0) -> armor_config:
+    return armor_config(d_out, d_in, d_block, n_keep, m_group, h_mode, select_mode, s_step, precision,
+                        int(normalize), phases, ridge, seed)
+
+
+# ---------------------------------------------------------------- C entry points, same names
+def armor_workspace_bytes(cfg: armor_config) -> int:
+    n = C.c_size_t(0)
+    _check(lib().armor_workspace_bytes(C.byref(cfg), C.byref(n)), "armor_workspace_bytes")
+    return int(n.value)
+
+
+def armor_create(cfg: armor_config, workspace: torch.Tensor) -> C.c_void_p:
+    ctx = C.c_void_p(0)
+    _check(lib().armor_create(C.byref(ctx), C.byref(cfg), _ptr(workspace, name="workspace"),
+                              workspace.numel() * workspace.element_size()), "armor_create")
+    return ctx
+
+
+def armor_destroy(ctx) -> None:
+    _check(lib().armor_destroy(ctx), "armor_destroy")
+
+
+def armor_gram(ctx, X: torch.Tensor, H: torch.Tensor) -> None:
+    if X.dim() != 2 or X.stride(1) != 1:
+        raise ValueError("X must be [n_rows, d_in] with unit column stride")
+    if not X.is_cuda or X.dtype != torch.float32:
+        raise ValueError("X must be a float32 CUDA tensor (this library has no CPU path)")
+    ldx = X.stride(0) if X.shape[0] > 1 else X.shape[1]
+    _check(lib().armor_gram(ctx, C.c_void_p(X.data_ptr()), DTYPE_F32, X.shape[0], ldx,
+                            _ptr(H, torch.float32, "H"), _stream()), "armor_gram")
+
+
+def armor_init(ctx, W, H, Wbar, r1, r2, A, B, S, M) -> None:
+    f = torch.float32
+    _check(lib().armor_init(ctx, _ptr(W, f, "W"), _ptr(H, f, "H"), _ptr(Wbar, f, "Wbar"), _ptr(r1, f, "r1"),
+                            _ptr(r2, f, "r2"), _ptr(A, f, "A"), _ptr(B, f, "B"), _ptr(S, f, "S"),
+                            _ptr(M, torch.uint8, "M"), _stream()), "armor_init")
+
+
+def armor_bcd_step(ctx, Wbar, H, A, B, S, M, t_first: int, n_iters: int, stats: torch.Tensor | None) -> None:
+    f = torch.float32
+    _check(lib().armor_bcd_step(ctx, _ptr(Wbar, f, "Wbar"), _ptr(H, f, "H"), _ptr(A, f, "A"), _ptr(B, f, "B"),
+                                _ptr(S, f, "S"), _ptr(M, torch.uint8, "M"), int(t_first), int(n_iters),
+                                _ptr(stats, torch.uint8, "stats"), _stream()), "armor_bcd_step")
+
+
+def armor_proxy_loss(ctx, Wbar, H, A, B, S, loss: torch.Tensor) -> None:
+    f = torch.float32
+    _check(lib().armor_proxy_loss(ctx, _ptr(Wbar, f, "Wbar"), _ptr(H, f, "H"), _ptr(A, f, "A"), _ptr(B, f, "B"),
+                                  _ptr(S, f, "S"), _ptr(loss, torch.float64, "loss"), _stream()), "armor_proxy_loss")
+
+
+def armor_apply(ctx, A, B, S, M, r1, r2, x, y) -> None:
+    f = torch.float32
+    _check(lib().armor_apply(ctx, _ptr(A, f, "A"), _ptr(B, f, "B"), _ptr(S, f, "S"), _ptr(M, torch.uint8, "M"),
+                             _ptr(r1, f, "r1"), _ptr(r2, f, "r2"), _ptr(x, f, "x"), _ptr(y, f, "y"), DTYPE_F32,
+                             x.shape[0], _stream()), "armor_apply")
+
+
+def armor_get_device_status(ctx, n: int = 8) -> list[int]:
+    buf = (C.c_int32 * n)()
+    _check(lib().armor_get_device_status(ctx, buf, n), "armor_get_device_status")
+    return list(buf)
+
+
+def armor_launch_count(ctx) -> int:
+    return int(lib().armor_launch_count(ctx))
+
+
+# ---------------------------------------------------------------- convenience wrapper
+@dataclass
+class LayerState:
+    Wbar: torch.Tensor
+    A: torch.Tensor
+    B: torch.Tensor
+    S: torch.Tensor
+    M: torch.Tensor
+    r1: torch.Tensor | None = None
+    r2: torch.Tensor | None = None
+
+
+class ArmorContext:
+    """A configuration plus its device workspace.  All methods enqueue on torch's current stream."""
+
+    def __init__(self, d_out, d_in, d_block, device="cuda:0", **kw):
+        self.device = torch.device(device)
+        if self.device.type != "cuda":
+            raise ValueError("ArmorContext needs a CUDA device")
+        self.cfg = make_config(d_out, d_in, d_block, **kw)
+        self.d_out, self.d_in, self.d_block = d_out, d_in, d_block
+        nbytes = armor_workspace_bytes(self.cfg)
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+            off = (-self.workspace.data_ptr()) % 256
+            self._ws_view = self.workspace[off: off + nbytes]
+            self.ctx = armor_create(self.cfg, self._ws_view)
+
+    def close(self):
+        if getattr(self, "ctx", None) is not None:
+            armor_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- calls
+    def new_gram(self) -> torch.Tensor:
+        return torch.zeros(self.d_in, self.d_in, dtype=torch.float32, device=self.device)
+
+    def gram(self, X: torch.Tensor, H: torch.Tensor) -> torch.Tensor:
+        armor_gram(self.ctx, X, H)
+        return H
+
+    def init(self, W: torch.Tensor, H: torch.Tensor) -> LayerState:
+        dev, f = self.device, torch.float32
+        nbo, nbi, db = self.d_out // self.d_block, self.d_in // self.d_block, self.d_block
+        st = LayerState(
+            Wbar=torch.empty_like(W),
+            A=torch.empty(nbo, db, db, dtype=f, device=dev), B=torch.empty(nbi, db, db, dtype=f, device=dev),
+            S=torch.empty_like(W), M=torch.empty(self.d_out, self.d_in // self.cfg.m_group, dtype=torch.uint8, device=dev))
+        if self.cfg.normalize:
+            st.r1 = torch.empty(self.d_in, dtype=f, device=dev)
+            st.r2 = torch.empty(self.d_out, dtype=f, device=dev)
+        armor_init(self.ctx, W, H, st.Wbar, st.r1, st.r2, st.A, st.B, st.S, st.M)
+        return st
+
+    def bcd_step(self, st: LayerState, H: torch.Tensor, t_first: int, n_iters: int, want_stats: bool = True):
+        stats = None
+        if want_stats:
+            stats = torch.zeros(max(n_iters, 1) * STATS_DTYPE.itemsize, dtype=torch.uint8, device=self.device)
+        armor_bcd_step(self.ctx, st.Wbar, H, st.A, st.B, st.S, st.M, t_first, n_iters, stats)
+        return stats
+
+    @staticmethod
+    def read_stats(stats: torch.Tensor) -> np.ndarray:
+        """Device->host copy of the per-iteration records (synchronises)."""
+        return stats.cpu().numpy().view(STATS_DTYPE)
+
+    def proxy_loss(self, st: LayerState, H: torch.Tensor) -> torch.Tensor:
+        out = torch.zeros(1, dtype=torch.float64, device=self.device)
+        armor_proxy_loss(self.ctx, st.Wbar, H, st.A, st.B, st.S, out)
+        return out
+
+    def apply(self, st: LayerState, x: torch.Tensor, denormalize: bool = False) -> torch.Tensor:
+        y = torch.empty(x.shape[0], self.d_out, dtype=torch.float32, device=self.device)
+        r1, r2 = (st.r1, st.r2) if denormalize else (None, None)
+        armor_apply(self.ctx, st.A, st.B, st.S, st.M, r1, r2, x, y)
+        return y
+
+    def device_status(self) -> list[int]:
+        torch.cuda.current_stream().synchronize()
+        return armor_get_device_status(self.ctx)
+
+    def launch_count(self) -> int:
+        return armor_launch_count(self.ctx)

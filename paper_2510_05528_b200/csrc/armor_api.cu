@@ -1,0 +1,361 @@
+// C ABI entry points and the host-side orchestration of one ARMOR layer optimisation.
+#include <new>
+
+#include "armor_internal.cuh"
+
+namespace {
+
+constexpr int64_t GRAM_ROWS = 16384;  // rows of X staged (transposed, split) per tensor-core Gram pass
+
+struct Layout {
+  size_t total = 0;
+  size_t take(size_t bytes) {
+    size_t off = total;
+    total += (bytes + 255) / 256 * 256;
+    return off;
+  }
+};
+
+armor_status check_config(const armor_config* cfg) {
+  if (!cfg) return ARMOR_ERR_INVALID_ARG;
+  if (cfg->d_out <= 0 || cfg->d_in <= 0 || cfg->d_block <= 0) return ARMOR_ERR_SHAPE;
+  if (cfg->m_group <= 0 || cfg->n_keep <= 0 || cfg->n_keep > cfg->m_group) return ARMOR_ERR_SHAPE;
+  if (cfg->d_out % cfg->d_block || cfg->d_in % cfg->d_block || cfg->d_block % cfg->m_group) return ARMOR_ERR_SHAPE;
+  if (cfg->n_keep != 2 || cfg->m_group != 4) return ARMOR_ERR_UNSUPPORTED;
+  if (cfg->d_block > 128 || cfg->d_block % 4) return ARMOR_ERR_UNSUPPORTED;
+  if (cfg->h_mode != ARMOR_H_FULL && cfg->h_mode != ARMOR_H_DIAG) return ARMOR_ERR_INVALID_ARG;
+  if (cfg->select_mode != ARMOR_SELECT_L1_RANDOM && cfg->select_mode != ARMOR_SELECT_L1_GREEDY)
+    return ARMOR_ERR_INVALID_ARG;
+  if (cfg->s_step != ARMOR_S_EXACT && cfg->s_step != ARMOR_S_BETA) return ARMOR_ERR_INVALID_ARG;
+  if (cfg->s_step == ARMOR_S_BETA) return ARMOR_ERR_UNSUPPORTED;
+  if (cfg->precision < ARMOR_PREC_FP32X3 || cfg->precision > ARMOR_PREC_SIMT) return ARMOR_ERR_INVALID_ARG;
+  if (cfg->precision != ARMOR_PREC_SIMT) {
+    // the tensor-core GEMM works on whole 128 x 128 tiles with K in steps of 32
+    if (cfg->h_mode == ARMOR_H_FULL && (cfg->d_out % 128 || cfg->d_in % 128)) return ARMOR_ERR_UNSUPPORTED;
+  }
+  if (!(cfg->ridge >= 0.f)) return ARMOR_ERR_INVALID_ARG;
+  if (cfg->phases < 0 || cfg->phases > 15) return ARMOR_ERR_INVALID_ARG;
+  return ARMOR_OK;
+}
+
+// Carves the workspace; with ctx == nullptr only the size is computed.
+size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
+  Layout L;
+  const int64_t wn = cfg.d_out * cfg.d_in;
+  const int db = cfg.d_block;
+  const int64_t nbo = cfg.d_out / db, nbi = cfg.d_in / db;
+  const size_t wbytes = (size_t)wn * sizeof(float);
+  const size_t hbytes = (size_t)cfg.d_in * cfg.d_in * sizeof(float);
+  const bool tc = cfg.precision != ARMOR_PREC_SIMT;
+  const bool x3 = cfg.precision == ARMOR_PREC_FP32X3;
+#define TAKE(field, type, bytes)                         \
+  do {                                                   \
+    size_t off_ = L.take(bytes);                         \
+    if (c) c->field = reinterpret_cast<type>(base + off_); \
+  } while (0)
+  TAKE(T, float*, wbytes);
+  TAKE(E, float*, wbytes);
+  TAKE(EH, float*, wbytes);
+  TAKE(P, float*, wbytes);
+  TAKE(U, float*, wbytes);
+  TAKE(V, float*, wbytes);
+  TAKE(VH, float*, wbytes);
+  TAKE(Gam, float*, wbytes);
+  TAKE(Tmp, float*, wbytes);
+  if (x3) { TAKE(LoHi, float*, wbytes); TAKE(Lo, float*, wbytes); } else if (c) { c->LoHi = nullptr; c->Lo = nullptr; }
+  if (x3) { TAKE(Hhi, float*, hbytes); TAKE(Hlo, float*, hbytes); } else if (c) { c->Hhi = nullptr; c->Hlo = nullptr; }
+  const size_t ao = (size_t)nbo * db * db * sizeof(float), bo = (size_t)nbi * db * db * sizeof(float);
+  TAKE(G, float*, ao);
+  TAKE(GamA, float*, ao);
+  TAKE(dA, float*, ao);
+  TAKE(At, float*, ao);
+  TAKE(C, float*, bo);
+  TAKE(GamB, float*, bo);
+  TAKE(Delta, float*, bo);
+  TAKE(Hjj, float*, bo);
+  TAKE(Kfull, float*, bo);
+  TAKE(Ktmp, float*, bo);
+  TAKE(Bt, float*, bo);
+  TAKE(alpha, float*, (size_t)cfg.d_out * sizeof(float));
+  TAKE(hdiag, float*, (size_t)cfg.d_in * sizeof(float));
+  TAKE(colpart, double*, (size_t)64 * cfg.d_in * sizeof(double));
+  if (tc) {
+    TAKE(Xt_hi, float*, (size_t)cfg.d_in * GRAM_ROWS * sizeof(float));
+    if (x3) TAKE(Xt_lo, float*, (size_t)cfg.d_in * GRAM_ROWS * sizeof(float)); else if (c) c->Xt_lo = nullptr;
+  } else if (c) { c->Xt_hi = nullptr; c->Xt_lo = nullptr; }
+  const int64_t tiles = ((cfg.d_out + 127) / 128) * ((cfg.d_in + 127) / 128) + ((cfg.d_in + 127) / 128) * ((cfg.d_in + 127) / 128);
+  const int64_t npart = tiles > ARMOR_DOT_BLOCKS ? tiles : ARMOR_DOT_BLOCKS;
+  TAKE(sc, double*, SC_COUNT * sizeof(double));
+  TAKE(partials, double*, (size_t)8 * npart * sizeof(double));
+  const int64_t nbmax = nbo > nbi ? nbo : nbi;
+  TAKE(partblk, double*, (size_t)(nbmax > nbo * nbi ? nbmax : nbo * nbi) * sizeof(double));
+  TAKE(failflag, int32_t*, (size_t)nbmax * sizeof(int32_t));
+  TAKE(sel, SelRec*, (size_t)nbo * nbi * sizeof(SelRec));
+  TAKE(status, int32_t*, ST_COUNT * sizeof(int32_t));
+#undef TAKE
+  if (c) {
+    c->npart = npart;
+    c->gram_rows = GRAM_ROWS;
+  }
+  return L.total;
+}
+
+inline cudaStream_t cs(armor_stream_t s) { return reinterpret_cast<cudaStream_t>(s); }
+
+// per-block Gram-type products over a long contraction
+void rowblock_gram(armor_ctx* c, const float* P, const float* T, float* G, cudaStream_t s) {
+  // G_i = P_i T_i^T  (contraction over d_in), batch over row-blocks i
+  const int db = c->db;
+  BGemm g{};
+  g.A = P; g.sAb = (int64_t)db * c->d_in; g.sAm = c->d_in; g.sAk = 1;
+  g.B = T; g.sBb = (int64_t)db * c->d_in; g.sBk = 1; g.sBn = c->d_in;
+  g.C = G; g.sCb = (int64_t)db * db; g.sCm = db; g.sCn = 1;
+  g.M = db; g.N = db; g.K = (int)c->d_in; g.batch = c->nbo; g.alpha = 1.f;
+  launch_bgemm(c, g, s);
+}
+void colblock_gram(armor_ctx* c, const float* U, const float* Y, float* Cm, cudaStream_t s) {
+  // C_j = U_j^T Y_j  (contraction over d_out), batch over column-blocks j
+  const int db = c->db;
+  BGemm g{};
+  g.A = U; g.sAb = db; g.sAm = 1; g.sAk = c->d_in;
+  g.B = Y; g.sBb = db; g.sBk = c->d_in; g.sBn = 1;
+  g.C = Cm; g.sCb = (int64_t)db * db; g.sCm = db; g.sCn = 1;
+  g.M = db; g.N = db; g.K = (int)c->d_out; g.batch = c->nbi; g.alpha = 1.f;
+  launch_bgemm(c, g, s);
+}
+void block_mm(armor_ctx* c, const float* X, bool tX, const float* Y, bool tY, float* Z, int nb, cudaStream_t s) {
+  const int db = c->db;
+  BGemm g{};
+  g.A = X; g.sAb = (int64_t)db * db; g.sAm = tX ? 1 : db; g.sAk = tX ? db : 1;
+  g.B = Y; g.sBb = (int64_t)db * db; g.sBk = tY ? 1 : db; g.sBn = tY ? db : 1;
+  g.C = Z; g.sCb = (int64_t)db * db; g.sCm = db; g.sCn = 1;
+  g.M = db; g.N = db; g.K = db; g.batch = nb; g.alpha = 1.f;
+  launch_bgemm(c, g, s);
+}
+
+armor_status core_gradient(armor_ctx* c, const float* A, const float* B, cudaStream_t s) {
+  // Gamma = A^T (E H_w) B^T  (minus half of the gradient display of Appendix D.3)
+  bd_left(c, A, true, c->EH, c->Tmp, c->d_out, c->d_in, 1.f, nullptr, 0.f, s);
+  bd_right(c, c->Tmp, B, true, c->Gam, c->d_out, c->d_in, 1.f, nullptr, 0.f, s);
+  return ARMOR_OK;
+}
+
+armor_status residual_and_loss(armor_ctx* c, const float* W, const float* H, const float* A, const float* B,
+                               const float* S, double* out, cudaStream_t s) {
+  bd_right(c, S, B, false, c->T, c->d_out, c->d_in, 1.f, nullptr, 0.f, s);      // T = S B
+  bd_left(c, A, false, c->T, c->E, c->d_out, c->d_in, -1.f, W, 1.f, s);         // E = W - A T
+  return rmul_H(c, c->E, H, c->EH, c->d_out, c->E, out, nullptr, nullptr, s);   // EH = E H_w, L = <EH, E>
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* armor_status_string(armor_status st) {
+  switch (st) {
+    case ARMOR_OK: return "ok";
+    case ARMOR_ERR_INVALID_ARG: return "invalid argument";
+    case ARMOR_ERR_SHAPE: return "shape error: d_block must divide d_out and d_in, m_group must divide d_block";
+    case ARMOR_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case ARMOR_ERR_CUDA: return "CUDA runtime error";
+    case ARMOR_ERR_NOT_SPD: return "block not positive definite";
+    case ARMOR_ERR_TIMEOUT: return "bounded device wait ran out";
+    case ARMOR_ERR_UNSUPPORTED: return "configuration not supported";
+  }
+  return "unknown status";
+}
+
+armor_status armor_workspace_bytes(const armor_config* cfg, size_t* bytes) {
+  if (!bytes) return ARMOR_ERR_INVALID_ARG;
+  armor_status st = check_config(cfg);
+  if (st != ARMOR_OK) return st;
+  *bytes = carve(*cfg, nullptr, nullptr);
+  return ARMOR_OK;
+}
+
+armor_status armor_create(armor_ctx** out, const armor_config* cfg, void* d_workspace, size_t bytes) {
+  if (!out) return ARMOR_ERR_INVALID_ARG;
+  *out = nullptr;
+  armor_status st = check_config(cfg);
+  if (st != ARMOR_OK) return st;
+  if (!d_workspace) return ARMOR_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(d_workspace) % 256) return ARMOR_ERR_WORKSPACE;
+  if (bytes < carve(*cfg, nullptr, nullptr)) return ARMOR_ERR_WORKSPACE;
+  armor_ctx* c = new (std::nothrow) armor_ctx();
+  if (!c) return ARMOR_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  if (c->cfg.phases == 0) c->cfg.phases = 15;
+  c->d_out = cfg->d_out; c->d_in = cfg->d_in; c->wn = cfg->d_out * cfg->d_in;
+  c->db = cfg->d_block; c->nbo = (int)(cfg->d_out / cfg->d_block); c->nbi = (int)(cfg->d_in / cfg->d_block);
+  c->ws = static_cast<char*>(d_workspace); c->ws_bytes = bytes;
+  c->launches = 0;
+  c->h_cached = nullptr;
+  carve(*cfg, c, c->ws);
+  if (cudaMemset(c->status, 0, ST_COUNT * sizeof(int32_t)) != cudaSuccess) { delete c; return ARMOR_ERR_CUDA; }
+  if (cudaMemset(c->sc, 0, SC_COUNT * sizeof(double)) != cudaSuccess) { delete c; return ARMOR_ERR_CUDA; }
+  *out = c;
+  return ARMOR_OK;
+}
+
+armor_status armor_destroy(armor_ctx* c) {
+  if (!c) return ARMOR_ERR_INVALID_ARG;
+  delete c;
+  return ARMOR_OK;
+}
+
+int64_t armor_launch_count(const armor_ctx* c) { return c ? c->launches : -1; }
+
+armor_status armor_get_device_status(armor_ctx* c, int32_t* h_codes, int32_t n) {
+  if (!c || !h_codes || n < 0) return ARMOR_ERR_INVALID_ARG;
+  if (n > ST_COUNT) n = ST_COUNT;
+  ARMOR_CUDA_OK(cudaMemcpy(h_codes, c->status, (size_t)n * sizeof(int32_t), cudaMemcpyDeviceToHost));
+  return ARMOR_OK;
+}
+
+armor_status armor_gram(armor_ctx* c, const void* d_X, int32_t x_dtype, int64_t n_rows, int64_t ldx, float* d_H,
+                        armor_stream_t stream) {
+  if (!c || !d_H || n_rows < 0) return ARMOR_ERR_INVALID_ARG;
+  if (n_rows == 0) return ARMOR_OK;
+  if (!d_X || ldx < c->d_in) return ARMOR_ERR_INVALID_ARG;
+  if (x_dtype != ARMOR_DTYPE_F32) return ARMOR_ERR_UNSUPPORTED;
+  cudaStream_t s = cs(stream);
+  const float* X = static_cast<const float*>(d_X);
+  return gram_accumulate(c, X, n_rows, ldx, d_H, s);
+}
+
+armor_status armor_init(armor_ctx* c, const float* d_W, const float* d_H, float* d_Wbar, float* d_r1, float* d_r2,
+                        float* d_A, float* d_B, float* d_S, uint8_t* d_M, armor_stream_t stream) {
+  if (!c || !d_W || !d_H || !d_Wbar || !d_A || !d_B || !d_S || !d_M) return ARMOR_ERR_INVALID_ARG;
+  if (c->cfg.normalize && (!d_r1 || !d_r2)) return ARMOR_ERR_INVALID_ARG;
+  launch_init(c, d_W, d_H, d_Wbar, d_r1, d_r2, d_A, d_B, d_S, d_M, cs(stream));
+  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+}
+
+armor_status armor_proxy_loss(armor_ctx* c, const float* W, const float* H, const float* A, const float* B,
+                              const float* S, double* d_loss, armor_stream_t stream) {
+  if (!c || !W || !H || !A || !B || !S || !d_loss) return ARMOR_ERR_INVALID_ARG;
+  cudaStream_t s = cs(stream);
+  armor_status st = prepare_H(c, H, s);
+  if (st != ARMOR_OK) return st;
+  st = residual_and_loss(c, W, H, A, B, S, d_loss, s);
+  if (st != ARMOR_OK) return st;
+  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+}
+
+armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float* A, float* B, float* S, uint8_t* M,
+                            int64_t t_first, int32_t n_iters, armor_iter_stats* d_stats, armor_stream_t stream) {
+  if (!c || !W || !H || !A || !B || !S || !M || n_iters < 0 || t_first < 0) return ARMOR_ERR_INVALID_ARG;
+  cudaStream_t s = cs(stream);
+  const int db = c->db, nbo = c->nbo, nbi = c->nbi;
+  const int64_t d_out = c->d_out, d_in = c->d_in;
+  const int ph = c->cfg.phases;
+  armor_status st = prepare_H(c, H, s);
+  if (st != ARMOR_OK) return st;
+  for (int it = 0; it < n_iters; ++it) {
+    armor_iter_stats* is = d_stats ? d_stats + it : nullptr;
+    const int64_t t = t_first + it;
+    launch_zero_scalars(c, s);
+    st = residual_and_loss(c, W, H, A, B, S, c->sc + SC_L0, s);
+    if (st != ARMOR_OK) return st;
+    launch_stage(c, is, 0, nullptr, 0, 0, s);
+
+    // ---- A-step: A_i += Gamma_i (G_i + lam I)^-1 -------------------------------------------
+    if (ph & ARMOR_PHASE_A) {
+      st = rmul_H(c, c->T, H, c->P, d_out, nullptr, nullptr, nullptr, nullptr, s);   // P = T H_w
+      if (st != ARMOR_OK) return st;
+      rowblock_gram(c, c->P, c->T, c->G, s);        // G_i = T_i H_w T_i^T
+      rowblock_gram(c, c->EH, c->T, c->GamA, s);    // Gamma_i = E_i H_w T_i^T
+      st = launch_chol(c, 0, c->G, c->GamA, c->dA, nullptr, A, c->At, nbo, c->partblk, s);
+      if (st != ARMOR_OK) return st;
+      launch_stage(c, is, 1, c->partblk, nbo, nbo, s);
+      bd_left(c, c->dA, false, c->P, c->EH, d_out, d_in, -1.f, c->EH, 1.f, s);       // EH -= dA P
+    } else {
+      launch_stage(c, is, 1, nullptr, 0, 0, s);
+    }
+
+    // ---- B-step: block-Newton directions, one exact step --------------------------------------
+    if (ph & ARMOR_PHASE_B) {
+      launch_zero_flags(c, s);
+      bd_left(c, A, false, S, c->U, d_out, d_in, 1.f, nullptr, 0.f, s);              // U = A S
+      colblock_gram(c, c->U, c->U, c->C, s);        // C_j = U_j^T U_j
+      colblock_gram(c, c->U, c->EH, c->GamB, s);    // Gamma_j = U_j^T (E H_w)_j
+      st = launch_chol(c, 1, c->C, c->GamB, c->Delta, nullptr, nullptr, nullptr, nbi, nullptr, s);
+      if (st != ARMOR_OK) return st;
+      st = launch_chol(c, 2, c->Hjj, c->Delta, c->Delta, c->GamB, nullptr, nullptr, nbi, c->partblk, s);
+      if (st != ARMOR_OK) return st;
+      bd_right(c, c->U, c->Delta, false, c->V, d_out, d_in, 1.f, nullptr, 0.f, s);   // V = U Delta
+      st = rmul_H(c, c->V, H, c->VH, d_out, c->V, c->sc + SC_Q_B, nullptr, nullptr, s);
+      if (st != ARMOR_OK) return st;
+      launch_stage(c, is, 2, c->partblk, nbi, nbi, s);
+      launch_axpy_slot(c, B, c->Delta, (int64_t)nbi * db * db, SC_TAU_B, 1.f, s);    // B += tau Delta
+      launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_B, -1.f, s);                   // EH -= tau V H_w
+    } else {
+      launch_stage(c, is, 2, nullptr, 0, 0, s);
+    }
+
+    // ---- S-step: exact line search along Gamma (.) M ------------------------------------------
+    if (ph & ARMOR_PHASE_S) {
+      core_gradient(c, A, B, s);
+      launch_masked_copy(c, c->Gam, M, c->U, SC_NRM_S, s);                           // U = Gamma (.) M
+      bd_left(c, A, false, c->U, c->Tmp, d_out, d_in, 1.f, nullptr, 0.f, s);
+      bd_right(c, c->Tmp, B, false, c->V, d_out, d_in, 1.f, nullptr, 0.f, s);        // V = A Gamma_M B
+      st = rmul_H(c, c->V, H, c->VH, d_out, c->V, c->sc + SC_Q_S, nullptr, nullptr, s);
+      if (st != ARMOR_OK) return st;
+      launch_stage(c, is, 3, nullptr, 0, 0, s);
+      launch_axpy_slot(c, S, c->U, c->wn, SC_TAU_S, 1.f, s);                         // S += tau Gamma_M
+      launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_S, -1.f, s);                   // EH -= tau V H_w
+    } else {
+      launch_stage(c, is, 3, nullptr, 0, 0, s);
+    }
+
+    // ---- sparse-core update (Algorithm 3) -----------------------------------------------------
+    if (ph & ARMOR_PHASE_MASK) {
+      core_gradient(c, A, B, s);
+      launch_alpha(c, A, s);
+      block_mm(c, B, false, c->Hjj, false, c->Ktmp, nbi, s);                         // B_j H_jj
+      block_mm(c, c->Ktmp, false, B, true, c->Kfull, nbi, s);                        // K_j = B_j H_jj B_j^T
+      launch_mask_select(c, c->Gam, S, M, t, s);
+      launch_mask_build_v(c, A, B, c->V, s);
+      st = rmul_H(c, c->V, H, c->VH, d_out, c->V, c->sc + SC_Q_M, nullptr, nullptr, s);
+      if (st != ARMOR_OK) return st;
+      launch_stage(c, is, 4, c->partblk, nbo * nbi, 0, s);
+      launch_mask_commit(c, S, M, is, s);
+    } else {
+      launch_stage(c, is, 4, nullptr, 0, 0, s);
+    }
+  }
+  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+}
+
+armor_status armor_apply(armor_ctx* c, const float* A, const float* B, const float* S, const uint8_t* M,
+                         const float* r1, const float* r2, const void* d_x, void* d_y, int32_t xy_dtype,
+                         int64_t n_tokens, armor_stream_t stream) {
+  (void)M;
+  if (!c || !A || !B || !S || n_tokens < 0) return ARMOR_ERR_INVALID_ARG;
+  if (n_tokens == 0) return ARMOR_OK;
+  if (!d_x || !d_y) return ARMOR_ERR_INVALID_ARG;
+  if (xy_dtype != ARMOR_DTYPE_F32) return ARMOR_ERR_UNSUPPORTED;
+  if ((r1 == nullptr) != (r2 == nullptr)) return ARMOR_ERR_INVALID_ARG;
+  cudaStream_t s = cs(stream);
+  const float* x = static_cast<const float*>(d_x);
+  float* y = static_cast<float*>(d_y);
+  const int64_t d_out = c->d_out, d_in = c->d_in;
+  const int64_t chunk = d_out < d_in ? d_out : d_in;   // z1 [chunk, d_in] and z2 [chunk, d_out] fit W-shaped scratch
+  for (int64_t t0 = 0; t0 < n_tokens; t0 += chunk) {
+    const int64_t n = (n_tokens - t0 < chunk) ? n_tokens - t0 : chunk;
+    const float* xc = x + t0 * d_in;
+    float* yc = y + t0 * d_out;
+    if (r1) {
+      launch_scale_rows_cols(c, xc, r1, nullptr, c->Tmp, n, d_in, s);
+      xc = c->Tmp;
+    }
+    bd_right(c, xc, B, true, c->T, n, d_in, 1.f, nullptr, 0.f, s);                   // z1 = x B^T
+    armor_status st = apply_core(c, c->T, S, c->E, n, s);                            // z2 = z1 S^T
+    if (st != ARMOR_OK) return st;
+    bd_right(c, c->E, A, true, yc, n, d_out, 1.f, nullptr, 0.f, s);                  // y = z2 A^T
+    if (r2) launch_scale_rows_cols(c, yc, r2, nullptr, yc, n, d_out, s);
+  }
+  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+}
+
+}  // extern "C"

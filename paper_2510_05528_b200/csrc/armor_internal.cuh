@@ -1,0 +1,170 @@
+// Internal declarations shared by the translation units of libarmor.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "armor.h"
+
+// ---------------------------------------------------------------- scalars
+// Device-resident double scalars (one set per context).  Kernels read step
+// lengths and accept flags from here so that no sub-step needs the host.
+enum {
+  SC_L0 = 0,     // <E H_w, E> at the start of the iteration
+  SC_DEC_A,      // exact decrease of the A-step
+  SC_GD_B,       // <Gamma^B, Delta>
+  SC_Q_B,        // tr(V H_w V^T) of the B direction
+  SC_NRM_S,      // ||Gamma (.) M||_F^2
+  SC_Q_S,        // tr(V H_w V^T) of the S direction
+  SC_EHV_M,      // <E H_w, V> of the group updates
+  SC_Q_M,        // tr(V H_w V^T) of the group updates
+  SC_TAU_B,
+  SC_TAU_S,
+  SC_ACCEPT,     // 1.0 if the group updates are kept
+  SC_DL_M,       // exact loss change of the group updates
+  SC_LOSS,       // running loss inside an iteration
+  SC_BETA_A,     // ||A^T A||_F^2 (BETA step)
+  SC_BETA_K,     // ||B H_w B^T||_F^2 (BETA step)
+  SC_TMP0,
+  SC_TMP1,
+  SC_COUNT = 32
+};
+
+// status words in the device status buffer
+enum { ST_CHOL_FAILS = 0, ST_FIRST_FAIL = 1, ST_WAIT_TIMEOUTS = 2, ST_LAST_ERR = 3, ST_COUNT = 8 };
+
+// One selected group per (i, j) block of the sparse core (Algorithm 3).
+struct SelRec {
+  int32_t valid;      // 0: nothing selected in this block
+  int32_t row;        // global row r
+  int32_t cgrp;       // group index inside the row (columns m*cgrp ..)
+  int32_t new_mask;   // bit p <=> position p kept
+  int32_t old_mask;
+  float new_val[4];
+  float old_val[4];
+};
+
+static const int ARMOR_DOT_BLOCKS = 592;  // 4 x 148 partial sums per reduction
+
+struct armor_ctx {
+  armor_config cfg;
+  int64_t d_out, d_in, wn;  // wn = d_out * d_in
+  int db, nbo, nbi;
+  char* ws;
+  size_t ws_bytes;
+  // W-shaped fp32 scratch
+  float *T, *E, *EH, *P, *U, *V, *VH, *Gam, *Tmp;
+  // low parts of the left operands / of H for the three-pass tensor-core mode
+  float *LoHi, *Lo, *Hhi, *Hlo;
+  // [nb, db, db] scratch
+  float *G, *GamA, *dA, *At, *C, *GamB, *Delta, *Hjj, *Kfull, *Ktmp, *Bt;
+  float *alpha, *hdiag;
+  // Gram staging (transposed, split chunk of X)
+  float *Xt_hi, *Xt_lo;
+  int64_t gram_rows;  // rows of X staged per pass
+  double* sc;         // [SC_COUNT]
+  double* partials;   // [2][4 * npart] partial sums of the fused / streaming reductions
+  int64_t npart;
+  double* partblk;    // [max(nbo, nbi, nbo * nbi)] per-block partial sums
+  double* colpart;    // [64][d_in] column partial sums of the normalisation
+  int32_t* failflag;  // [max(nbo, nbi)]
+  SelRec* sel;        // [nbo * nbi]
+  int32_t* status;    // [ST_COUNT]
+  int64_t launches;
+  // identity of the H whose split copy is cached in Hhi/Hlo
+  const float* h_cached;
+};
+
+#define ARMOR_CUDA_OK(expr)                                  \
+  do {                                                       \
+    cudaError_t _e = (expr);                                 \
+    if (_e != cudaSuccess) return ARMOR_ERR_CUDA;            \
+  } while (0)
+
+// ---------------------------------------------------------------- launchers
+// Generic strided batched fp32 GEMM on CUDA cores:
+//   C_b[m][n] = alpha * sum_k A_b[m][k] B_b[k][n] + beta * D_b[m][n]
+// element (m,k) of A_b lives at A + b*sAb + m*sAm + k*sAk (likewise B, C, D).
+struct BGemm {
+  const float* A; int64_t sAb, sAm, sAk;
+  const float* B; int64_t sBb, sBk, sBn;
+  float* C; int64_t sCb, sCm, sCn;
+  const float* D; int64_t sDb, sDm, sDn;
+  int M, N, K, batch;
+  float alpha, beta;
+};
+void launch_bgemm(armor_ctx* c, const BGemm& g, cudaStream_t s);
+
+// block-diagonal products on row-major [rows, cols] matrices
+//  right: out[:, jblk] = alpha * in[:, jblk] * Bblk[j] (+ beta * add[:, jblk]); transB uses Bblk[j]^T
+//  left : out[iblk, :] = alpha * Ablk[i] * in[iblk, :] (+ beta * add[iblk, :]); transA uses Ablk[i]^T
+void bd_right(armor_ctx* c, const float* in, const float* Bblk, bool transB, float* out, int64_t rows,
+              int64_t cols, float alpha, const float* add, float beta, cudaStream_t s);
+void bd_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, float* out, int64_t rows,
+             int64_t cols, float alpha, const float* add, float beta, cudaStream_t s);
+
+// out = in * H_w (FULL: dense GEMM by cfg.precision; DIAG: column scale) with up to two
+// fused dot products <out, d1> -> sc[slot1], <out, d2> -> sc[slot2] (slot < 0: none).
+armor_status rmul_H(armor_ctx* c, const float* in, const float* H, float* out, int64_t rows,
+                    const float* d1, double* out1, const float* d2, double* out2, cudaStream_t s);
+// per-call preparation of everything derived from H (diagonal, diagonal blocks, split copy)
+armor_status prepare_H(armor_ctx* c, const float* H, cudaStream_t s);
+armor_status gram_accumulate(armor_ctx* c, const float* X, int64_t n_rows, int64_t ldx, float* H, cudaStream_t s);
+// z2 [n, d_out] = z1 [n, d_in] * S^T
+armor_status apply_core(armor_ctx* c, const float* z1, const float* S, float* z2, int64_t n, cudaStream_t s);
+
+// deterministic reductions (two stages, fixed order)
+void dot_to_ptr(armor_ctx* c, const float* x, const float* y, int64_t n, double* out, cudaStream_t s);
+void reduce_partials_to(armor_ctx* c, const double* part, int n, double* out, cudaStream_t s);
+
+// streaming kernels (kernels_stream.cu)
+void launch_colscale(armor_ctx* c, const float* in, const float* h, float* out, int64_t rows, int64_t cols,
+                     cudaStream_t s);
+void launch_extract_hblocks(armor_ctx* c, const float* H, cudaStream_t s);   // hdiag, Hjj (per h_mode)
+void launch_transpose_blocks(armor_ctx* c, const float* in, float* out, int nb, cudaStream_t s);
+void launch_masked_copy(armor_ctx* c, const float* Gam, const uint8_t* M, float* out, int slot_norm,
+                        cudaStream_t s);                                     // out = Gam (.) M, sc[slot] = ||out||^2
+void launch_axpy_slot(armor_ctx* c, float* y, const float* x, int64_t n, int slot, float sign,
+                      cudaStream_t s);                                       // y += sign * sc[slot] * x
+void launch_init(armor_ctx* c, const float* W, const float* H, float* Wbar, float* r1, float* r2,
+                 float* A, float* B, float* S, uint8_t* M, cudaStream_t s);
+void launch_zero_scalars(armor_ctx* c, cudaStream_t s);
+void launch_zero_flags(armor_ctx* c, cudaStream_t s);
+// per-iteration bookkeeping on the device: stage 0 start, 1 after A, 2 after B, 3 after S, 4 mask accept
+void launch_stage(armor_ctx* c, armor_iter_stats* st, int stage, const double* part, int npart, int nflag,
+                  cudaStream_t s);
+void launch_scale_rows_cols(armor_ctx* c, const float* in, const float* colscale, const float* rowscale,
+                            float* out, int64_t rows, int64_t cols, cudaStream_t s);
+void launch_split_hilo(armor_ctx* c, const float* in, float* hi, float* lo, int64_t n, cudaStream_t s);
+void launch_transpose_split(armor_ctx* c, const float* X, int64_t ldx, int64_t rows, int64_t cols,
+                            float* Thi, float* Tlo, int64_t ldt, cudaStream_t s);
+
+// block solves (kernels_chol.cu)
+// mode 0: X = rhs (G + lam I)^-1, A += X, At = A^T, out = X, part[b] = exact decrease of block b
+// mode 1: out = (G + lam I)^-1 rhs
+// mode 2: out = rhs (G + lam I)^-1, part[b] = <dotw, out>
+armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float* rhs, float* out, const float* dotw,
+                         float* A, float* At, int nb, double* part, cudaStream_t s);
+
+// sparse-core update (kernels_mask.cu)
+void launch_alpha(armor_ctx* c, const float* A, cudaStream_t s);
+void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const uint8_t* M, int64_t t,
+                        cudaStream_t s);
+void launch_mask_build_v(armor_ctx* c, const float* A, const float* B, float* V, cudaStream_t s);
+void launch_mask_commit(armor_ctx* c, float* S, uint8_t* M, armor_iter_stats* st, cudaStream_t s);
+
+// tensor-core GEMM (gemm_tcgen05.cu):  C[M][N] (+)= sum_k A[m][k] * B[n][k]  (both K-major, fp32 storage).
+// passes == 3 uses the split operands (A, Alo, B, Blo).  Partial dot products of the output tile with up
+// to two W-shaped tensors go to dot partial buffers.
+struct TcGemm {
+  const float* A; const float* Alo; int64_t lda;
+  const float* B; const float* Blo; int64_t ldb;
+  float* C; int64_t ldc;
+  int64_t M, N, K;
+  int passes;            // 1 or 3
+  int accumulate;        // C += (read-modify-write) instead of C =
+  int symmetric_lower;   // only tiles with n0 <= m0 are computed; mirrored into the upper triangle (M == N)
+  const float* d1; const float* d2;  // optional dot operands (ld = ldc)
+  double* part1; double* part2;      // [tiles] partial sums
+};
+armor_status launch_tc_gemm(armor_ctx* c, const TcGemm& g, int* n_tiles, cudaStream_t s);
+bool tc_gemm_shape_ok(int64_t M, int64_t N, int64_t K);

@@ -1,0 +1,111 @@
+// Dense contractions of the ARMOR iteration, dispatched by the configured precision:
+// right-multiplication by the weighting H_w, the calibration Gram, and the core product of the
+// deployment form.  SIMT = fp32 CUDA cores; TF32 / FP32X3 = tcgen05 tensor cores (1 or 3 passes).
+#include "armor_internal.cuh"
+
+armor_status prepare_H(armor_ctx* c, const float* H, cudaStream_t s) {
+  launch_extract_hblocks(c, H, s);
+  if (c->cfg.h_mode == ARMOR_H_FULL && c->cfg.precision == ARMOR_PREC_FP32X3)
+    launch_split_hilo(c, H, c->Hhi, c->Hlo, c->d_in * c->d_in, s);
+  return ARMOR_OK;
+}
+
+armor_status rmul_H(armor_ctx* c, const float* in, const float* H, float* out, int64_t rows, const float* d1,
+                    double* out1, const float* d2, double* out2, cudaStream_t s) {
+  const int64_t d_in = c->d_in;
+  if (c->cfg.h_mode == ARMOR_H_DIAG) {
+    launch_colscale(c, in, c->hdiag, out, rows, d_in, s);
+  } else if (c->cfg.precision == ARMOR_PREC_SIMT) {
+    BGemm g{};
+    g.A = in; g.sAm = d_in; g.sAk = 1;
+    g.B = H; g.sBk = d_in; g.sBn = 1;
+    g.C = out; g.sCm = d_in; g.sCn = 1;
+    g.M = (int)rows; g.N = (int)d_in; g.K = (int)d_in; g.batch = 1; g.alpha = 1.f;
+    launch_bgemm(c, g, s);
+  } else {
+    TcGemm g{};
+    g.lda = d_in; g.ldb = d_in; g.ldc = d_in;
+    g.M = rows; g.N = d_in; g.K = d_in;
+    g.C = out;
+    if (c->cfg.precision == ARMOR_PREC_FP32X3) {
+      // left operand as a tf32-exact high part plus the fp32 remainder
+      launch_split_hilo(c, in, c->LoHi, c->Lo, rows * d_in, s);
+      g.A = c->LoHi; g.Alo = c->Lo; g.B = c->Hhi; g.Blo = c->Hlo; g.passes = 3;
+    } else {
+      g.A = in; g.B = H; g.passes = 1;
+    }
+    g.d1 = d1; g.d2 = d2;
+    g.part1 = d1 ? c->partials : nullptr;
+    g.part2 = d2 ? c->partials + 4 * c->npart : nullptr;
+    int tiles = 0;
+    armor_status st = launch_tc_gemm(c, g, &tiles, s);
+    if (st != ARMOR_OK) return st;
+    if (d1) reduce_partials_to(c, c->partials, 4 * tiles, out1, s);
+    if (d2) reduce_partials_to(c, c->partials + 4 * c->npart, 4 * tiles, out2, s);
+    return ARMOR_OK;
+  }
+  if (d1) dot_to_ptr(c, out, d1, rows * d_in, out1, s);
+  if (d2) dot_to_ptr(c, out, d2, rows * d_in, out2, s);
+  return ARMOR_OK;
+}
+
+armor_status gram_accumulate(armor_ctx* c, const float* X, int64_t n_rows, int64_t ldx, float* H, cudaStream_t s) {
+  const int64_t d_in = c->d_in;
+  if (c->cfg.precision == ARMOR_PREC_SIMT) {
+    // H += X^T X, element (m, k) of the left operand is X[k][m]
+    const int64_t step = 1 << 20;
+    for (int64_t r0 = 0; r0 < n_rows; r0 += step) {
+      const int64_t n = n_rows - r0 < step ? n_rows - r0 : step;
+      BGemm g{};
+      g.A = X + r0 * ldx; g.sAm = 1; g.sAk = ldx;
+      g.B = X + r0 * ldx; g.sBk = ldx; g.sBn = 1;
+      g.C = H; g.sCm = d_in; g.sCn = 1;
+      g.D = H; g.sDm = d_in; g.sDn = 1;
+      g.M = (int)d_in; g.N = (int)d_in; g.K = (int)n; g.batch = 1; g.alpha = 1.f; g.beta = 1.f;
+      launch_bgemm(c, g, s);
+    }
+    return ARMOR_OK;
+  }
+  const bool x3 = c->cfg.precision == ARMOR_PREC_FP32X3;
+  for (int64_t r0 = 0; r0 < n_rows; r0 += c->gram_rows) {
+    const int64_t n = n_rows - r0 < c->gram_rows ? n_rows - r0 : c->gram_rows;
+    const int64_t kpad = (n + 31) / 32 * 32;     // staged row length (zero padded)
+    launch_transpose_split(c, X + r0 * ldx, ldx, n, d_in, c->Xt_hi, x3 ? c->Xt_lo : nullptr, kpad, s);
+    TcGemm g{};
+    g.A = c->Xt_hi; g.Alo = c->Xt_lo; g.lda = kpad;
+    g.B = c->Xt_hi; g.Blo = c->Xt_lo; g.ldb = kpad;
+    g.C = H; g.ldc = d_in;
+    g.M = d_in; g.N = d_in; g.K = kpad;
+    g.passes = x3 ? 3 : 1;
+    g.accumulate = 1;
+    g.symmetric_lower = 1;
+    armor_status st = launch_tc_gemm(c, g, nullptr, s);
+    if (st != ARMOR_OK) return st;
+  }
+  return ARMOR_OK;
+}
+
+armor_status apply_core(armor_ctx* c, const float* z1, const float* S, float* z2, int64_t n, cudaStream_t s) {
+  const int64_t d_in = c->d_in, d_out = c->d_out;
+  if (c->cfg.precision == ARMOR_PREC_SIMT || (d_out % 32) || (d_in % 4)) {
+    BGemm g{};
+    g.A = z1; g.sAm = d_in; g.sAk = 1;
+    g.B = S; g.sBk = 1; g.sBn = d_in;
+    g.C = z2; g.sCm = d_out; g.sCn = 1;
+    g.M = (int)n; g.N = (int)d_out; g.K = (int)d_in; g.batch = 1; g.alpha = 1.f;
+    launch_bgemm(c, g, s);
+    return ARMOR_OK;
+  }
+  TcGemm g{};
+  g.lda = d_in; g.ldb = d_in; g.ldc = d_out;
+  g.M = n; g.N = d_out; g.K = d_in;
+  g.C = z2;
+  if (c->cfg.precision == ARMOR_PREC_FP32X3) {
+    launch_split_hilo(c, z1, c->LoHi, c->Lo, n * d_in, s);
+    launch_split_hilo(c, S, c->P, c->U, c->wn, s);
+    g.A = c->LoHi; g.Alo = c->Lo; g.B = c->P; g.Blo = c->U; g.passes = 3;
+  } else {
+    g.A = z1; g.B = S; g.passes = 1;
+  }
+  return launch_tc_gemm(c, g, nullptr, s);
+}

@@ -1,0 +1,435 @@
+// Tensor-core GEMM for sm_100a:  C[M][N] (+)= sum_k A[m][k] * B[n][k]   (fp32 storage, both operands K-major)
+//
+// Used for the dense contractions of the ARMOR iteration: the calibration Gram X^T X (Section 2 of the
+// paper; both operands are the transposed, staged chunk of X) and the right-multiplications by the
+// symmetric Gram, E.H, T.H and V.H (H[n][k] = H[k][n], so H itself is the K-major B operand).
+//
+// Design: persistent kernel, one CTA per SM, 192 threads:
+//   warp 0   : TMA producer  (cp.async.bulk.tensor.2d, 128-byte swizzle, mbarrier complete_tx)
+//   warp 1   : MMA issuer    (one thread issues tcgen05.mma kind::tf32, 128 x 256 x 8 per instruction,
+//                             accumulators in tensor memory, two accumulator buffers of 256 columns)
+//   warps 2-5: epilogue      (tcgen05.ld 32 lanes x 32 columns, fused C-update / mirror / dot products)
+// passes == 3: every operand is given as a tf32-exact high part and an fp32 low part; the three products
+// hi*hi, lo*hi, hi*lo are accumulated into the same fp32 accumulator (error-compensated tf32, fp32-grade).
+// Every wait is bounded: a wait that runs out raises a status word and the CTA leaves through the common
+// exit that frees its tensor memory.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include "armor_internal.cuh"
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 32;          // BK fp32 = 128 bytes = one swizzle row
+constexpr int NTHREADS = 192;
+constexpr uint32_t TMEM_COLS = 512;                 // two accumulator buffers of BN columns
+constexpr int A_BYTES = BM * BK * 4;                // 16 KiB
+constexpr int B_BYTES = BN * BK * 4;                // 32 KiB
+constexpr long long WAIT_CYCLES = 4000000000ll;     // ~2 s at 2 GHz
+
+struct Params {
+  float* C; int64_t ldc;
+  int64_t M, N, K;
+  int m_tiles, n_tiles, n_tiles_total;
+  int accumulate, symmetric_lower;
+  const float* d1; const float* d2;
+  double* part1; double* part2;
+  int32_t* status;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the CTA is aborting (this wait or another one ran out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > WAIT_CYCLES) {
+      *abort_flag = 1;
+      atomicAdd(&status[ST_WAIT_TIMEOUTS], 1);
+      status[ST_LAST_ERR] = ARMOR_ERR_TIMEOUT;
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// K-major operand tile, rows of 128 bytes, 128-byte swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);          // start address
+  d |= (uint64_t)1 << 16;                           // leading byte offset (unused with swizzle)
+  d |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset
+  d |= (uint64_t)1 << 46;                           // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                           // 128-byte swizzle
+  return d;
+}
+
+// kind::tf32, fp32 accumulate, both operands K-major, M = 128, N = 256.
+__device__ __forceinline__ uint32_t instr_desc_tf32() {
+  uint32_t d = 0;
+  d |= 1u << 4;                   // D format: F32
+  d |= 2u << 7;                   // A format: TF32
+  d |= 2u << 10;                  // B format: TF32
+  d |= (uint32_t)(BN >> 3) << 17; // N
+  d |= (uint32_t)(BM >> 4) << 24; // M
+  return d;
+}
+
+// tile index -> (m tile, n tile).  m runs fastest so that concurrently running CTAs share a B tile.
+__device__ __forceinline__ void tile_coords(const Params& p, int tile, int& mt, int& nt) {
+  if (!p.symmetric_lower) {
+    mt = tile % p.m_tiles;
+    nt = tile / p.m_tiles;
+    return;
+  }
+  // only tiles that hold an element with column <= row: m tile >= 2 * n tile
+  int rem = tile;
+  for (nt = 0; nt < p.n_tiles; ++nt) {
+    const int cnt = p.m_tiles - 2 * nt;
+    if (rem < cnt) break;
+    rem -= cnt;
+  }
+  mt = 2 * nt + rem;
+}
+
+template <int PASSES>
+__global__ void __launch_bounds__(NTHREADS, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapAlo,
+               const __grid_constant__ CUtensorMap mapB, const __grid_constant__ CUtensorMap mapBlo, const Params p) {
+  constexpr int STAGE_BYTES = (PASSES == 3 ? 2 : 1) * (A_BYTES + B_BYTES);
+  constexpr int STAGES = (PASSES == 3) ? 2 : 4;
+  extern __shared__ uint8_t smem_raw[];
+  // 1024-byte alignment for the swizzled tiles
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 4];
+  __shared__ uint32_t tmem_base_holder;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]);
+  const uint32_t tfull0 = smem_u32(&bars[2 * STAGES]), tempty0 = smem_u32(&bars[2 * STAGES + 2]);
+  const int kt_total = (int)((p.K + BK - 1) / BK);
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(tfull0 + 8 * s, 1); mbar_init(tempty0 + 8 * s, 4); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_holder;
+  volatile int* abortp = &abort_flag;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0; long long issued = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.n_tiles_total && ok; tile += gridDim.x) {
+        int mt, nt;
+        tile_coords(p, tile, mt, nt);
+        for (int kt = 0; kt < kt_total; ++kt) {
+          if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abortp, p.status)) { ok = false; break; }
+          const uint32_t fb = full0 + 8 * stage;
+          mbar_expect_tx(fb, STAGE_BYTES);
+          uint32_t dst = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+          tma_load_2d(dst, &mapA, kt * BK, mt * BM, fb);
+          dst += A_BYTES;
+          if (PASSES == 3) { tma_load_2d(dst, &mapAlo, kt * BK, mt * BM, fb); dst += A_BYTES; }
+          tma_load_2d(dst, &mapB, kt * BK, nt * BN, fb);
+          dst += B_BYTES;
+          if (PASSES == 3) tma_load_2d(dst, &mapBlo, kt * BK, nt * BN, fb);
+          ++issued;
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) {
+        // leave no bulk copy in flight: wait (bounded) for the stages armed most recently
+        for (int back = 1; back <= STAGES && back <= issued; ++back) {
+          int s = stage - back; uint32_t ph = phase;
+          if (s < 0) { s += STAGES; ph ^= 1; }
+          const long long t0 = clock64();
+          while (!mbar_try(full0 + 8 * s, ph) && clock64() - t0 < 20000000ll) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc_tf32();
+      int stage = 0; uint32_t phase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.n_tiles_total && ok; tile += gridDim.x, ++local) {
+        const int as = local & 1;
+        const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
+        if (!mbar_wait(tempty0 + 8 * as, aphase ^ 1, abortp, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tacc = tmem_base + (uint32_t)(as * BN);
+        for (int kt = 0; kt < kt_total; ++kt) {
+          if (!mbar_wait(full0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+          const uint32_t sa_lo = sa + A_BYTES;
+          const uint32_t sb = sa + (PASSES == 3 ? 2 : 1) * A_BYTES;
+          const uint32_t sb_lo = sb + B_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 8; ++k) {
+            const uint64_t da = smem_desc_k_sw128(sa + k * 32), dbm = smem_desc_k_sw128(sb + k * 32);
+            if (PASSES == 3) {
+              const uint64_t dal = smem_desc_k_sw128(sa_lo + k * 32), dbl = smem_desc_k_sw128(sb_lo + k * 32);
+              umma_tf32(tacc, dal, dbm, idesc, (kt | k) != 0);
+              umma_tf32(tacc, da, dbl, idesc, 1);
+              umma_tf32(tacc, da, dbm, idesc, 1);
+            } else {
+              umma_tf32(tacc, da, dbm, idesc, (kt | k) != 0);
+            }
+          }
+          umma_commit(empty0 + 8 * stage);   // frees the stage once these MMAs have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (ok) umma_commit(tfull0 + 8 * as);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue warps
+    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    int local = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < p.n_tiles_total && ok; tile += gridDim.x, ++local) {
+      int mt, nt;
+      tile_coords(p, tile, mt, nt);
+      const int as = local & 1;
+      const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
+      if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
+      tc_fence_after();
+      const int64_t row = (int64_t)mt * BM + q * 32 + lane;
+      const bool row_ok = row < p.M;
+      double dot1 = 0.0, dot2 = 0.0;
+#pragma unroll 1
+      for (int ch = 0; ch < BN / 32; ++ch) {
+        const int64_t col0 = (int64_t)nt * BN + ch * 32;
+        uint32_t r[32];
+        tmem_ld32(tmem_base + (uint32_t)(as * BN + ch * 32) + ((uint32_t)(q * 32) << 16), r);
+        if (col0 >= p.N || !row_ok) continue;
+        float* crow = p.C + row * p.ldc + col0;
+        if (!p.symmetric_lower) {
+          float f1 = 0.f, f2 = 0.f;
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) {
+            float4 v = make_float4(__uint_as_float(r[i]), __uint_as_float(r[i + 1]), __uint_as_float(r[i + 2]),
+                                   __uint_as_float(r[i + 3]));
+            if (p.accumulate) {
+              const float4 o = *reinterpret_cast<const float4*>(crow + i);
+              v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+            }
+            if (p.d1) {
+              const float4 d = *reinterpret_cast<const float4*>(p.d1 + row * p.ldc + col0 + i);
+              f1 = fmaf(v.x, d.x, f1); f1 = fmaf(v.y, d.y, f1); f1 = fmaf(v.z, d.z, f1); f1 = fmaf(v.w, d.w, f1);
+            }
+            if (p.d2) {
+              const float4 d = *reinterpret_cast<const float4*>(p.d2 + row * p.ldc + col0 + i);
+              f2 = fmaf(v.x, d.x, f2); f2 = fmaf(v.y, d.y, f2); f2 = fmaf(v.z, d.z, f2); f2 = fmaf(v.w, d.w, f2);
+            }
+            *reinterpret_cast<float4*>(crow + i) = v;
+          }
+          dot1 += (double)f1;
+          dot2 += (double)f2;
+        } else {
+          // lower triangle (+ diagonal) is owned by this tile; each kept element is mirrored once
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int64_t cc = col0 + i;
+            if (cc <= row) {
+              const float v = __uint_as_float(r[i]);
+              crow[i] = p.accumulate ? crow[i] + v : v;
+              if (cc < row) {
+                float* mp = p.C + cc * p.ldc + row;
+                *mp = p.accumulate ? *mp + v : v;
+              }
+            }
+          }
+        }
+      }
+      // accumulator buffer is free again
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty0 + 8 * as);
+      if (p.part1 || p.part2) {
+        for (int o = 16; o > 0; o >>= 1) {
+          dot1 += __shfl_down_sync(0xffffffffu, dot1, o);
+          dot2 += __shfl_down_sync(0xffffffffu, dot2, o);
+        }
+        if (lane == 0) {
+          if (p.part1) p.part1[(int64_t)tile * 4 + q] = dot1;
+          if (p.part2) p.part2[(int64_t)tile * 4 + q] = dot2;
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------ host side
+PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(ptr);
+  }
+  return fn;
+}
+
+// [rows][K] fp32, leading dimension ld: box = BK x box_rows, 128-byte swizzle, zero fill out of bounds.
+bool make_map(CUtensorMap* map, const float* base, int64_t rows, int64_t K, int64_t ld, int box_rows) {
+  PFN_cuTensorMapEncodeTiled_v12000 enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(float)};
+  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+template <int PASSES>
+armor_status launch_impl(armor_ctx* c, const TcGemm& g, const Params& p, cudaStream_t s) {
+  CUtensorMap mA, mAlo, mB, mBlo;
+  if (!make_map(&mA, g.A, g.M, g.K, g.lda, BM)) return ARMOR_ERR_CUDA;
+  if (!make_map(&mB, g.B, g.N, g.K, g.ldb, BN)) return ARMOR_ERR_CUDA;
+  if (PASSES == 3) {
+    if (!make_map(&mAlo, g.Alo, g.M, g.K, g.lda, BM)) return ARMOR_ERR_CUDA;
+    if (!make_map(&mBlo, g.Blo, g.N, g.K, g.ldb, BN)) return ARMOR_ERR_CUDA;
+  } else {
+    mAlo = mA;
+    mBlo = mB;
+  }
+  constexpr int STAGE_BYTES = (PASSES == 3 ? 2 : 1) * (A_BYTES + B_BYTES);
+  constexpr int STAGES = (PASSES == 3) ? 2 : 4;
+  constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024;
+  static bool attr = false;
+  if (!attr) {
+    if (cudaFuncSetAttribute(tc_gemm_kernel<PASSES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess)
+      return ARMOR_ERR_CUDA;
+    attr = true;
+  }
+  static int n_sm = 0;
+  if (!n_sm) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ARMOR_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ARMOR_ERR_CUDA;
+  }
+  const int grid = p.n_tiles_total < n_sm ? p.n_tiles_total : n_sm;
+  tc_gemm_kernel<PASSES><<<grid, NTHREADS, SMEM, s>>>(mA, mAlo, mB, mBlo, p);
+  c->launches++;
+  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+}
+
+}  // namespace
+
+bool tc_gemm_shape_ok(int64_t M, int64_t N, int64_t K) {
+  return M > 0 && N > 0 && K > 0 && (N % 32 == 0) && (K % 4 == 0);
+}
+
+armor_status launch_tc_gemm(armor_ctx* c, const TcGemm& g, int* n_tiles, cudaStream_t s) {
+  if (!tc_gemm_shape_ok(g.M, g.N, g.K)) return ARMOR_ERR_UNSUPPORTED;
+  if ((g.lda % 4) || (g.ldb % 4) || (g.ldc % 4)) return ARMOR_ERR_UNSUPPORTED;
+  if (g.symmetric_lower && g.M != g.N) return ARMOR_ERR_INVALID_ARG;
+  Params p{};
+  p.C = g.C; p.ldc = g.ldc; p.M = g.M; p.N = g.N; p.K = g.K;
+  p.m_tiles = (int)((g.M + BM - 1) / BM);
+  p.n_tiles = (int)((g.N + BN - 1) / BN);
+  if (g.symmetric_lower) {
+    int tot = 0;
+    for (int nt = 0; nt < p.n_tiles; ++nt) {
+      const int cnt = p.m_tiles - 2 * nt;
+      if (cnt > 0) tot += cnt;
+    }
+    p.n_tiles_total = tot;
+  } else {
+    p.n_tiles_total = p.m_tiles * p.n_tiles;
+  }
+  p.accumulate = g.accumulate; p.symmetric_lower = g.symmetric_lower;
+  p.d1 = g.d1; p.d2 = g.d2; p.part1 = g.part1; p.part2 = g.part2;
+  p.status = c->status;
+  if (n_tiles) *n_tiles = p.n_tiles_total;
+  if (g.passes == 3) return launch_impl<3>(c, g, p, s);
+  return launch_impl<1>(c, g, p, s);
+}

@@ -1,0 +1,235 @@
+// Greedy sparse-core update (Algorithm 3 and Appendix B.1 of the paper): every 2:4 group of every
+// (i, j) block is scored by the L1 norm of the core gradient, one group per block is drawn with
+// probability proportional to its score, and that group is re-solved in closed form over all six
+// masks (Eq. mask_loss_opt / mask_loss_opt_sol).
+#include "armor_internal.cuh"
+
+namespace {
+
+constexpr int NT = 256;
+
+__device__ __forceinline__ uint64_t splitmix64(uint64_t x) {
+  uint64_t z = x + 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+// -ln(u) for u = (k + 1/2) / 2^24, k the top 24 bits of the hash.  Both branches feed the logarithm an
+// argument that is exact in fp32, so the result is good to a few ulp even for u next to 1, where the
+// winners of the exponential race live.
+__device__ __forceinline__ float neg_log_uniform(uint32_t k24) {
+  if (k24 < (1u << 23)) return -logf((float)(2u * k24 + 1u) * 2.98023223876953125e-8f);        // * 2^-25
+  return -log1pf(-(float)(2u * ((1u << 24) - k24) - 1u) * 2.98023223876953125e-8f);
+}
+
+__global__ void alpha_kernel(const float* __restrict__ A, float* __restrict__ alpha, int db) {
+  // alpha[r] = || A[:, r] ||^2 : column r of the block that owns row r of the core
+  const int i = blockIdx.x;
+  const float* Ai = A + (int64_t)i * db * db;
+  for (int r = threadIdx.x; r < db; r += blockDim.x) {
+    double acc = 0.0;
+    for (int o = 0; o < db; ++o) {
+      double v = Ai[o * db + r];
+      acc += v * v;
+    }
+    alpha[i * db + r] = (float)acc;
+  }
+}
+
+// 2x2 PSD solve with the pseudo-inverse rule: w = K^+ z, red = z^T K^+ z.
+__device__ __forceinline__ void pinv2(double k11, double k12, double k22, double z1, double z2, double& w1,
+                                      double& w2, double& red) {
+  const double det = k11 * k22 - k12 * k12;
+  if (det <= 1e-12 * k11 * k22) {
+    const double tr = k11 + k22;
+    if (tr <= 0.0) { w1 = w2 = 0.0; red = 0.0; return; }
+    const double inv = 1.0 / (tr * tr);
+    w1 = (k11 * z1 + k12 * z2) * inv;
+    w2 = (k12 * z1 + k22 * z2) * inv;
+  } else {
+    w1 = (k22 * z1 - k12 * z2) / det;
+    w2 = (k11 * z2 - k12 * z1) / det;
+  }
+  red = z1 * w1 + z2 * w2;
+}
+
+// One CTA per (i, j) block.  Pass 1: float4 per group, score, key, arg-min by warp shuffles.
+// Pass 2 (thread 0): the six-mask sweep for the winner.
+__global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict__ Gam, const float* __restrict__ S,
+                                                         const uint8_t* __restrict__ M, const float* __restrict__ alpha,
+                                                         const float* __restrict__ Kfull, SelRec* __restrict__ sel,
+                                                         double* __restrict__ part, int64_t d_in, int db, int nbi,
+                                                         int select_mode, uint64_t seed, uint64_t t,
+                                                         uint64_t n_groups_total) {
+  const int blk = blockIdx.x;
+  const int bi = blk / nbi, bj = blk % nbi;
+  const int gpb = db / 4;                 // groups per block row
+  const int64_t ng_row = d_in / 4;        // groups per matrix row
+  const int n_in_block = db * gpb;
+  float best_key = INFINITY;
+  uint64_t best_g = ~0ull;
+  for (int idx = threadIdx.x; idx < n_in_block; idx += NT) {
+    const int rl = idx / gpb, cl = idx % gpb;
+    const int64_t row = (int64_t)bi * db + rl;
+    const int64_t cg = (int64_t)bj * gpb + cl;
+    const float4 g4 = *reinterpret_cast<const float4*>(Gam + row * d_in + cg * 4);
+    float score = fabsf(g4.x) + fabsf(g4.y) + fabsf(g4.z) + fabsf(g4.w);
+    if (!(alpha[row] > 0.f)) score = 0.f;
+    const uint64_t g = (uint64_t)row * (uint64_t)ng_row + (uint64_t)cg;
+    float key = INFINITY;
+    if (score > 0.f) {
+      if (select_mode == ARMOR_SELECT_L1_RANDOM) {
+        const uint64_t bits = splitmix64(seed ^ splitmix64(t * n_groups_total + g));
+        key = neg_log_uniform((uint32_t)(bits >> 40)) / score;
+      } else {
+        key = -score;
+      }
+    }
+    if (key < best_key || (key == best_key && g < best_g)) { best_key = key; best_g = g; }
+  }
+  // arg-min over the CTA; ties go to the lower group index
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ok = __shfl_down_sync(0xffffffffu, best_key, o);
+    const uint64_t og = __shfl_down_sync(0xffffffffu, best_g, o);
+    if (ok < best_key || (ok == best_key && og < best_g)) { best_key = ok; best_g = og; }
+  }
+  __shared__ float skey[NT / 32];
+  __shared__ uint64_t sg[NT / 32];
+  if ((threadIdx.x & 31) == 0) { skey[threadIdx.x >> 5] = best_key; sg[threadIdx.x >> 5] = best_g; }
+  __syncthreads();
+  if (threadIdx.x != 0) return;
+  for (int w = 1; w < NT / 32; ++w)
+    if (skey[w] < best_key || (skey[w] == best_key && sg[w] < best_g)) { best_key = skey[w]; best_g = sg[w]; }
+
+  SelRec rec;
+  double ehv = 0.0;
+  rec.valid = 0; rec.row = 0; rec.cgrp = 0; rec.new_mask = 0; rec.old_mask = 0;
+  for (int p = 0; p < 4; ++p) { rec.new_val[p] = 0.f; rec.old_val[p] = 0.f; }
+  if (best_key < INFINITY) {
+    const int64_t row = (int64_t)(best_g / (uint64_t)ng_row);
+    const int64_t cg = (int64_t)(best_g % (uint64_t)ng_row);
+    const int lc = (int)(cg % gpb) * 4;   // first row of the group inside B_j
+    const float* Kj = Kfull + (int64_t)bj * db * db;
+    double K[4][4], z[4], sg4[4];
+    const double a_r = (double)alpha[row];
+    const unsigned om = M[row * ng_row + cg];
+    for (int p = 0; p < 4; ++p) {
+      sg4[p] = (double)S[row * d_in + cg * 4 + p];
+      for (int q = 0; q < 4; ++q) K[p][q] = (double)Kj[(int64_t)(lc + p) * db + (lc + q)];
+    }
+    for (int p = 0; p < 4; ++p) {
+      double kz = 0.0;
+      for (int q = 0; q < 4; ++q) kz += K[p][q] * sg4[q];
+      z[p] = (double)Gam[row * d_in + cg * 4 + p] + a_r * kz;
+    }
+    // incumbent first, then lexicographic order; strict improvement only
+    const int pa[6] = {0, 0, 0, 1, 1, 2}, pb[6] = {1, 2, 3, 2, 3, 3};
+    int inc = -1;
+    for (int m = 0; m < 6; ++m)
+      if (om == ((1u << pa[m]) | (1u << pb[m]))) inc = m;
+    double best_red = -INFINITY, bw1 = 0.0, bw2 = 0.0;
+    int best_m = -1;
+    for (int step = (inc >= 0 ? -1 : 0); step < 6; ++step) {
+      const int m = (step < 0) ? inc : step;
+      if (step >= 0 && m == inc) continue;
+      double w1, w2, red;
+      pinv2(K[pa[m]][pa[m]], K[pa[m]][pb[m]], K[pb[m]][pb[m]], z[pa[m]], z[pb[m]], w1, w2, red);
+      red /= a_r;
+      if (best_m < 0 || red > best_red) { best_red = red; best_m = m; bw1 = w1 / a_r; bw2 = w2 / a_r; }
+    }
+    rec.valid = 1;
+    rec.row = (int32_t)row;
+    rec.cgrp = (int32_t)cg;
+    rec.old_mask = (int32_t)om;
+    rec.new_mask = (int32_t)((1u << pa[best_m]) | (1u << pb[best_m]));
+    for (int p = 0; p < 4; ++p) rec.old_val[p] = (float)sg4[p];
+    rec.new_val[pa[best_m]] = (float)bw1;
+    rec.new_val[pb[best_m]] = (float)bw2;
+    // <Gamma, dS> restricted to this group: this block's share of <E H_w, V>
+    for (int p = 0; p < 4; ++p)
+      ehv += (double)Gam[row * d_in + cg * 4 + p] * ((double)rec.new_val[p] - (double)rec.old_val[p]);
+  }
+  part[blk] = ehv;
+  sel[blk] = rec;
+}
+
+// V = A dS B for the iteration's group updates: block (i, j) of V is the rank-one matrix
+// A_i[:, r] (x) (delta^T B_j[rows of the group, :]).
+__global__ void __launch_bounds__(NT) mask_build_v_kernel(const float* __restrict__ A, const float* __restrict__ B,
+                                                          const SelRec* __restrict__ sel, float* __restrict__ V,
+                                                          int64_t d_in, int db, int nbi) {
+  const int blk = blockIdx.x;
+  const int bi = blk / nbi, bj = blk % nbi;
+  __shared__ float av[128], bv[128];
+  const SelRec rec = sel[blk];
+  if (threadIdx.x < db) {
+    float a = 0.f, bsum = 0.f;
+    if (rec.valid) {
+      const int rl = rec.row - bi * db;
+      const int lc = (rec.cgrp % (db / 4)) * 4;
+      a = A[(int64_t)bi * db * db + (int64_t)threadIdx.x * db + rl];
+      const float* Bj = B + (int64_t)bj * db * db;
+      for (int p = 0; p < 4; ++p)
+        bsum = fmaf(rec.new_val[p] - rec.old_val[p], Bj[(int64_t)(lc + p) * db + threadIdx.x], bsum);
+    }
+    av[threadIdx.x] = a;
+    bv[threadIdx.x] = bsum;
+  }
+  __syncthreads();
+  const int q = db / 4;
+  for (int e = threadIdx.x; e < db * q; e += NT) {
+    const int o = e / q, n4 = (e % q) * 4;
+    const float a = av[o];
+    float4 v = make_float4(a * bv[n4], a * bv[n4 + 1], a * bv[n4 + 2], a * bv[n4 + 3]);
+    *reinterpret_cast<float4*>(V + ((int64_t)bi * db + o) * d_in + (int64_t)bj * db + n4) = v;
+  }
+}
+
+__global__ void mask_commit_kernel(const SelRec* __restrict__ sel, int nblocks, float* __restrict__ S,
+                                   uint8_t* __restrict__ M, int64_t d_in, const double* __restrict__ sc,
+                                   armor_iter_stats* st) {
+  __shared__ int changed;
+  if (threadIdx.x == 0) changed = 0;
+  __syncthreads();
+  const bool accept = sc[SC_ACCEPT] != 0.0;
+  int mine = 0;
+  if (accept) {
+    for (int b = threadIdx.x; b < nblocks; b += blockDim.x) {
+      const SelRec rec = sel[b];
+      if (!rec.valid) continue;
+      float* sp = S + (int64_t)rec.row * d_in + (int64_t)rec.cgrp * 4;
+      *reinterpret_cast<float4*>(sp) = make_float4(rec.new_val[0], rec.new_val[1], rec.new_val[2], rec.new_val[3]);
+      M[(int64_t)rec.row * (d_in / 4) + rec.cgrp] = (uint8_t)rec.new_mask;
+      mine += (rec.new_mask != rec.old_mask) ? 1 : 0;
+    }
+  }
+  atomicAdd(&changed, mine);
+  __syncthreads();
+  if (threadIdx.x == 0 && st) st->groups_changed = changed;
+}
+
+}  // namespace
+
+void launch_alpha(armor_ctx* c, const float* A, cudaStream_t s) {
+  alpha_kernel<<<c->nbo, 128, 0, s>>>(A, c->alpha, c->db);
+  c->launches++;
+}
+
+void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const uint8_t* M, int64_t t, cudaStream_t s) {
+  mask_select_kernel<<<c->nbo * c->nbi, NT, 0, s>>>(Gam, S, M, c->alpha, c->Kfull, c->sel, c->partblk, c->d_in, c->db,
+                                                   c->nbi,
+                                                   c->cfg.select_mode, c->cfg.seed, (uint64_t)t,
+                                                   (uint64_t)(c->d_out * (c->d_in / 4)));
+  c->launches++;
+}
+
+void launch_mask_build_v(armor_ctx* c, const float* A, const float* B, float* V, cudaStream_t s) {
+  mask_build_v_kernel<<<c->nbo * c->nbi, NT, 0, s>>>(A, B, c->sel, V, c->d_in, c->db, c->nbi);
+  c->launches++;
+}
+
+void launch_mask_commit(armor_ctx* c, float* S, uint8_t* M, armor_iter_stats* st, cudaStream_t s) {
+  mask_commit_kernel<<<1, 256, 0, s>>>(c->sel, c->nbo * c->nbi, S, M, c->d_in, c->sc, st);
+  c->launches++;
+}

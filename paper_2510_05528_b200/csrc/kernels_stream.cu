@@ -1,0 +1,408 @@
+// Streaming (HBM-bound) kernels over W-shaped tensors, reductions and small bookkeeping kernels.
+#include "armor_internal.cuh"
+
+namespace {
+
+constexpr int NT = 256;
+
+__device__ __forceinline__ double block_reduce_sum(double v) {
+  __shared__ double sm[32];
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  if (lane == 0) sm[w] = v;
+  __syncthreads();
+  const int nw = (blockDim.x + 31) >> 5;
+  v = (threadIdx.x < nw) ? sm[threadIdx.x] : 0.0;
+  if (w == 0) {
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+  }
+  __syncthreads();
+  return v;  // valid in thread 0
+}
+
+// ---- deterministic two-stage dot product: fixed grid, fixed order --------------------------------
+__global__ void __launch_bounds__(NT) dot_partial_kernel(const float4* __restrict__ x,
+                                                         const float4* __restrict__ y, int64_t n4,
+                                                         double* __restrict__ part) {
+  double acc = 0.0;
+  for (int64_t i = (int64_t)blockIdx.x * NT + threadIdx.x; i < n4; i += (int64_t)gridDim.x * NT) {
+    float4 a = x[i], b = y[i];
+    float s = a.x * b.x;
+    s = fmaf(a.y, b.y, s);
+    s = fmaf(a.z, b.z, s);
+    s = fmaf(a.w, b.w, s);
+    acc += (double)s;
+  }
+  acc = block_reduce_sum(acc);
+  if (threadIdx.x == 0) part[blockIdx.x] = acc;
+}
+
+__global__ void __launch_bounds__(NT) reduce_final_kernel(const double* __restrict__ part, int n,
+                                                          double* __restrict__ out) {
+  double acc = 0.0;
+  for (int i = threadIdx.x; i < n; i += NT) acc += part[i];
+  acc = block_reduce_sum(acc);
+  if (threadIdx.x == 0) *out = acc;
+}
+
+// ---- column scale: out = in * diag(h) -----------------------------------------------------------
+__global__ void __launch_bounds__(NT) colscale_kernel(const float4* __restrict__ in, const float4* __restrict__ h,
+                                                      float4* __restrict__ out, int64_t n4, int cols4) {
+  for (int64_t i = (int64_t)blockIdx.x * NT + threadIdx.x; i < n4; i += (int64_t)gridDim.x * NT) {
+    float4 a = in[i], s = h[i % cols4];
+    out[i] = make_float4(a.x * s.x, a.y * s.y, a.z * s.z, a.w * s.w);
+  }
+}
+
+__global__ void __launch_bounds__(NT) rowcolscale_kernel(const float* __restrict__ in, const float* __restrict__ cs,
+                                                         const float* __restrict__ rs, float* __restrict__ out,
+                                                         int64_t rows, int64_t cols) {
+  const int64_t n = rows * cols;
+  for (int64_t i = (int64_t)blockIdx.x * NT + threadIdx.x; i < n; i += (int64_t)gridDim.x * NT) {
+    float v = in[i];
+    if (cs) v *= cs[i % cols];
+    if (rs) v *= rs[i / cols];
+    out[i] = v;
+  }
+}
+
+// ---- H diagonal and diagonal blocks -------------------------------------------------------------
+__global__ void extract_hblocks_kernel(const float* __restrict__ H, float* __restrict__ hdiag,
+                                       float* __restrict__ Hjj, int64_t d_in, int db, int diag_only) {
+  const int j = blockIdx.x;
+  for (int e = threadIdx.x; e < db * db; e += blockDim.x) {
+    int a = e / db, b = e % db;
+    float v = H[(int64_t)(j * db + a) * d_in + (j * db + b)];
+    if (diag_only && a != b) v = 0.f;
+    Hjj[(int64_t)j * db * db + e] = v;
+    if (a == b) hdiag[j * db + a] = v;
+  }
+}
+
+__global__ void transpose_blocks_kernel(const float* __restrict__ in, float* __restrict__ out, int db) {
+  const int64_t off = (int64_t)blockIdx.x * db * db;
+  for (int e = threadIdx.x; e < db * db; e += blockDim.x) {
+    int r = e / db, cc = e % db;
+    out[off + (int64_t)cc * db + r] = in[off + e];
+  }
+}
+
+// ---- Gamma_M = Gamma (.) M and its squared norm -------------------------------------------------
+__global__ void __launch_bounds__(NT) masked_copy_kernel(const float4* __restrict__ gam, const uint8_t* __restrict__ M,
+                                                         float4* __restrict__ out, int64_t ngroups,
+                                                         double* __restrict__ part) {
+  double acc = 0.0;
+  for (int64_t g = (int64_t)blockIdx.x * NT + threadIdx.x; g < ngroups; g += (int64_t)gridDim.x * NT) {
+    float4 v = gam[g];
+    const unsigned m = M[g];
+    v.x = (m & 1u) ? v.x : 0.f;
+    v.y = (m & 2u) ? v.y : 0.f;
+    v.z = (m & 4u) ? v.z : 0.f;
+    v.w = (m & 8u) ? v.w : 0.f;
+    out[g] = v;
+    float s = v.x * v.x;
+    s = fmaf(v.y, v.y, s);
+    s = fmaf(v.z, v.z, s);
+    s = fmaf(v.w, v.w, s);
+    acc += (double)s;
+  }
+  acc = block_reduce_sum(acc);
+  if (threadIdx.x == 0) part[blockIdx.x] = acc;
+}
+
+// ---- y += sign * sc[slot] * x -------------------------------------------------------------------
+__global__ void __launch_bounds__(NT) axpy_slot_kernel(float4* __restrict__ y, const float4* __restrict__ x,
+                                                       int64_t n4, const double* __restrict__ sc, int slot,
+                                                       float sign) {
+  const float a = sign * (float)sc[slot];
+  for (int64_t i = (int64_t)blockIdx.x * NT + threadIdx.x; i < n4; i += (int64_t)gridDim.x * NT) {
+    float4 u = y[i], v = x[i];
+    y[i] = make_float4(fmaf(a, v.x, u.x), fmaf(a, v.y, u.y), fmaf(a, v.z, u.z), fmaf(a, v.w, u.w));
+  }
+}
+
+// ---- normalisation (Section 3.2): r1 = column norms, r2 = row norms of W / r1 -------------------
+constexpr int COLSUM_CHUNKS = 64;
+__global__ void __launch_bounds__(NT) colsumsq_partial_kernel(const float* __restrict__ W, int64_t rows, int64_t cols,
+                                                              double* __restrict__ part) {
+  const int64_t col = (int64_t)blockIdx.x * NT + threadIdx.x;
+  if (col >= cols) return;
+  const int64_t per = (rows + COLSUM_CHUNKS - 1) / COLSUM_CHUNKS;
+  const int64_t r0 = blockIdx.y * per, r1 = min(rows, r0 + per);
+  double acc = 0.0;
+  for (int64_t r = r0; r < r1; ++r) {
+    double w = W[r * cols + col];
+    acc += w * w;
+  }
+  part[(int64_t)blockIdx.y * cols + col] = acc;
+}
+__global__ void __launch_bounds__(NT) colnorm_final_kernel(const double* __restrict__ part, int64_t cols,
+                                                           float* __restrict__ r1) {
+  const int64_t col = (int64_t)blockIdx.x * NT + threadIdx.x;
+  if (col >= cols) return;
+  double acc = 0.0;
+  for (int ch = 0; ch < COLSUM_CHUNKS; ++ch) acc += part[(int64_t)ch * cols + col];
+  float r = (float)sqrt(acc);
+  r1[col] = (r == 0.f) ? 1.f : r;
+}
+__global__ void __launch_bounds__(NT) rownorm_scale_kernel(const float* __restrict__ W, const float* __restrict__ r1,
+                                                           float* __restrict__ r2, float* __restrict__ Wbar,
+                                                           int64_t cols) {
+  const int64_t row = blockIdx.x;
+  const float* w = W + row * cols;
+  double acc = 0.0;
+  for (int64_t c = threadIdx.x; c < cols; c += NT) {
+    double v = (double)w[c] / (double)r1[c];
+    acc += v * v;
+  }
+  __shared__ float r2s;
+  acc = block_reduce_sum(acc);
+  if (threadIdx.x == 0) {
+    float r = (float)sqrt(acc);
+    r = (r == 0.f) ? 1.f : r;
+    r2[row] = r;
+    r2s = r;
+  }
+  __syncthreads();
+  const float rr = r2s;
+  for (int64_t c = threadIdx.x; c < cols; c += NT) Wbar[row * cols + c] = (w[c] / r1[c]) / rr;
+}
+
+// ---- initialisation (Eq. init): top-2 of each group of 4 by W^2 * H_jj --------------------------
+__global__ void __launch_bounds__(NT) init_core_kernel(const float4* __restrict__ W, const float* __restrict__ H,
+                                                       int64_t d_in, float4* __restrict__ S, uint8_t* __restrict__ M,
+                                                       int64_t ngroups, int groups_per_row) {
+  for (int64_t g = (int64_t)blockIdx.x * NT + threadIdx.x; g < ngroups; g += (int64_t)gridDim.x * NT) {
+    const int64_t c0 = (g % groups_per_row) * 4;
+    float4 w = W[g];
+    const float wv[4] = {w.x, w.y, w.z, w.w};
+    double sc[4];
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+      double h = (double)H[(c0 + p) * d_in + (c0 + p)];
+      sc[p] = (double)wv[p] * (double)wv[p] * h;
+    }
+    int i1 = 0;
+#pragma unroll
+    for (int p = 1; p < 4; ++p)
+      if (sc[p] > sc[i1]) i1 = p;  // strict: ties keep the lower column
+    int i2 = (i1 == 0) ? 1 : 0;
+#pragma unroll
+    for (int p = 0; p < 4; ++p)
+      if (p != i1 && p != i2 && sc[p] > sc[i2]) i2 = p;
+    const unsigned m = (1u << i1) | (1u << i2);
+    M[g] = (uint8_t)m;
+    S[g] = make_float4((m & 1u) ? w.x : 0.f, (m & 2u) ? w.y : 0.f, (m & 4u) ? w.z : 0.f, (m & 8u) ? w.w : 0.f);
+  }
+}
+
+__global__ void identity_blocks_kernel(float* __restrict__ A, int db) {
+  const int64_t off = (int64_t)blockIdx.x * db * db;
+  for (int e = threadIdx.x; e < db * db; e += blockDim.x) A[off + e] = (e / db == e % db) ? 1.f : 0.f;
+}
+
+__global__ void copy_kernel(const float4* __restrict__ in, float4* __restrict__ out, int64_t n4) {
+  for (int64_t i = (int64_t)blockIdx.x * NT + threadIdx.x; i < n4; i += (int64_t)gridDim.x * NT) out[i] = in[i];
+}
+
+// ---- scalars and per-iteration bookkeeping ------------------------------------------------------
+__global__ void zero_scalars_kernel(double* sc, int32_t* failflag, int nflag) {
+  for (int i = threadIdx.x; i < SC_COUNT; i += blockDim.x) sc[i] = 0.0;
+  for (int i = threadIdx.x; i < nflag; i += blockDim.x) failflag[i] = 0;
+}
+
+// stage 0: start, 1: after A, 2: after B, 3: after S, 4: mask accept
+__global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const int32_t* failflag, int nflag,
+                             const double* partA, int nA, int32_t* status) {
+  if (threadIdx.x != 0) return;
+  if (stage == 0) {
+    sc[SC_LOSS] = sc[SC_L0];
+    if (st) {
+      st->loss_start = sc[SC_L0];
+      st->chol_failed = 0;
+      st->groups_changed = 0;
+      st->mask_accepted = 0;
+      st->delta_L_mask = 0.0;
+      st->tau_B = 0.f;
+      st->tau_S = 0.f;
+      st->reserved = 0;
+    }
+  } else if (stage == 1) {
+    double dec = 0.0;
+    for (int i = 0; i < nA; ++i) dec += partA[i];
+    sc[SC_DEC_A] = dec;
+    sc[SC_LOSS] -= dec;
+    int nf = 0;
+    for (int i = 0; i < nflag; ++i) nf += failflag[i] ? 1 : 0;
+    if (st) { st->loss_A = sc[SC_LOSS]; st->chol_failed += nf; }
+    if (nf) atomicAdd(&status[ST_CHOL_FAILS], nf);
+  } else if (stage == 2) {
+    double gd = 0.0;
+    for (int i = 0; i < nA; ++i) gd += partA[i];
+    sc[SC_GD_B] = gd;
+    const double q = sc[SC_Q_B];
+    const double tau = (q > 0.0) ? gd / q : 0.0;
+    sc[SC_TAU_B] = tau;
+    sc[SC_LOSS] -= 2.0 * tau * gd - tau * tau * q;
+    int nf = 0;
+    for (int i = 0; i < nflag; ++i) nf += failflag[i] ? 1 : 0;
+    if (st) { st->loss_B = sc[SC_LOSS]; st->tau_B = (float)tau; st->chol_failed += nf; }
+    if (nf) atomicAdd(&status[ST_CHOL_FAILS], nf);
+  } else if (stage == 3) {
+    const double nrm = sc[SC_NRM_S], q = sc[SC_Q_S];
+    const double tau = (q > 0.0) ? nrm / q : 0.0;
+    sc[SC_TAU_S] = tau;
+    sc[SC_LOSS] -= 2.0 * tau * nrm - tau * tau * q;
+    if (st) { st->loss_S = sc[SC_LOSS]; st->tau_S = (float)tau; }
+  } else if (stage == 4) {
+    double ehv = 0.0;
+    for (int i = 0; i < nA; ++i) ehv += partA[i];   // <Gamma, dS> = <E H_w, V>, one term per block
+    sc[SC_EHV_M] = ehv;
+    const double dl = -2.0 * sc[SC_EHV_M] + sc[SC_Q_M];
+    const bool acc = (dl <= 0.0);
+    sc[SC_DL_M] = dl;
+    sc[SC_ACCEPT] = acc ? 1.0 : 0.0;
+    if (acc) sc[SC_LOSS] += dl;
+    if (st) { st->delta_L_mask = dl; st->mask_accepted = acc ? 1 : 0; st->loss_mask = sc[SC_LOSS]; }
+  } else if (stage == 5) {  // phases skipped: carry the loss forward
+    if (st) { st->loss_A = st->loss_B = st->loss_S = st->loss_mask = sc[SC_LOSS]; }
+  }
+}
+
+// ---- operand split for the three-pass tensor-core mode ------------------------------------------
+__global__ void __launch_bounds__(NT) split_hilo_kernel(const float4* __restrict__ in, float4* __restrict__ hi,
+                                                        float4* __restrict__ lo, int64_t n4) {
+  for (int64_t i = (int64_t)blockIdx.x * NT + threadIdx.x; i < n4; i += (int64_t)gridDim.x * NT) {
+    float4 v = in[i];
+    float4 h;
+    h.x = __uint_as_float(__float_as_uint(v.x) & 0xffffe000u);
+    h.y = __uint_as_float(__float_as_uint(v.y) & 0xffffe000u);
+    h.z = __uint_as_float(__float_as_uint(v.z) & 0xffffe000u);
+    h.w = __uint_as_float(__float_as_uint(v.w) & 0xffffe000u);
+    if (hi) hi[i] = h;
+    lo[i] = make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w);
+  }
+}
+
+// X [rows, cols] (ld ldx) -> Thi/Tlo [cols, rows] (ld ldt): transposed and split.
+__global__ void transpose_split_kernel(const float* __restrict__ X, int64_t ldx, int64_t rows, int64_t cols,
+                                       float* __restrict__ Thi, float* __restrict__ Tlo, int64_t ldt) {
+  __shared__ float tile[32][33];
+  const int64_t c0 = (int64_t)blockIdx.x * 32, r0 = (int64_t)blockIdx.y * 32;
+  for (int j = threadIdx.y; j < 32; j += blockDim.y) {
+    int64_t r = r0 + j, cidx = c0 + threadIdx.x;
+    tile[j][threadIdx.x] = (r < rows && cidx < cols) ? X[r * ldx + cidx] : 0.f;
+  }
+  __syncthreads();
+  for (int j = threadIdx.y; j < 32; j += blockDim.y) {
+    int64_t cidx = c0 + j, r = r0 + threadIdx.x;
+    if (cidx < cols && r < ldt) {
+      float v = tile[threadIdx.x][j];
+      float h = __uint_as_float(__float_as_uint(v) & 0xffffe000u);
+      Thi[cidx * ldt + r] = h;
+      if (Tlo) Tlo[cidx * ldt + r] = v - h;
+    }
+  }
+}
+
+inline int grid_for(int64_t n) {
+  int64_t b = (n + NT - 1) / NT;
+  return (int)(b < 1 ? 1 : (b > 148 * 16 ? 148 * 16 : b));
+}
+
+}  // namespace
+
+void dot_to_ptr(armor_ctx* c, const float* x, const float* y, int64_t n, double* out, cudaStream_t s) {
+  dot_partial_kernel<<<ARMOR_DOT_BLOCKS, NT, 0, s>>>((const float4*)x, (const float4*)y, n / 4, c->partials);
+  reduce_final_kernel<<<1, NT, 0, s>>>(c->partials, ARMOR_DOT_BLOCKS, out);
+  c->launches += 2;
+}
+
+void reduce_partials_to(armor_ctx* c, const double* part, int n, double* out, cudaStream_t s) {
+  reduce_final_kernel<<<1, NT, 0, s>>>(part, n, out);
+  c->launches++;
+}
+
+void launch_zero_flags(armor_ctx* c, cudaStream_t s) {
+  const int nflag = c->nbo > c->nbi ? c->nbo : c->nbi;
+  cudaMemsetAsync(c->failflag, 0, (size_t)nflag * sizeof(int32_t), s);
+}
+
+void launch_colscale(armor_ctx* c, const float* in, const float* h, float* out, int64_t rows, int64_t cols,
+                     cudaStream_t s) {
+  colscale_kernel<<<grid_for(rows * cols / 4), NT, 0, s>>>((const float4*)in, (const float4*)h, (float4*)out,
+                                                          rows * cols / 4, (int)(cols / 4));
+  c->launches++;
+}
+
+void launch_scale_rows_cols(armor_ctx* c, const float* in, const float* colscale, const float* rowscale, float* out,
+                            int64_t rows, int64_t cols, cudaStream_t s) {
+  rowcolscale_kernel<<<grid_for(rows * cols), NT, 0, s>>>(in, colscale, rowscale, out, rows, cols);
+  c->launches++;
+}
+
+void launch_extract_hblocks(armor_ctx* c, const float* H, cudaStream_t s) {
+  extract_hblocks_kernel<<<c->nbi, NT, 0, s>>>(H, c->hdiag, c->Hjj, c->d_in, c->db, c->cfg.h_mode == ARMOR_H_DIAG);
+  c->launches++;
+}
+
+void launch_transpose_blocks(armor_ctx* c, const float* in, float* out, int nb, cudaStream_t s) {
+  transpose_blocks_kernel<<<nb, NT, 0, s>>>(in, out, c->db);
+  c->launches++;
+}
+
+void launch_masked_copy(armor_ctx* c, const float* Gam, const uint8_t* M, float* out, int slot_norm, cudaStream_t s) {
+  masked_copy_kernel<<<ARMOR_DOT_BLOCKS, NT, 0, s>>>((const float4*)Gam, M, (float4*)out, c->wn / 4, c->partials);
+  reduce_final_kernel<<<1, NT, 0, s>>>(c->partials, ARMOR_DOT_BLOCKS, c->sc + slot_norm);
+  c->launches += 2;
+}
+
+void launch_axpy_slot(armor_ctx* c, float* y, const float* x, int64_t n, int slot, float sign, cudaStream_t s) {
+  axpy_slot_kernel<<<grid_for(n / 4), NT, 0, s>>>((float4*)y, (const float4*)x, n / 4, c->sc, slot, sign);
+  c->launches++;
+}
+
+void launch_init(armor_ctx* c, const float* W, const float* H, float* Wbar, float* r1, float* r2, float* A, float* B,
+                 float* S, uint8_t* M, cudaStream_t s) {
+  const int64_t rows = c->d_out, cols = c->d_in;
+  if (c->cfg.normalize) {
+    double* part = c->colpart;
+    dim3 g1((unsigned)((cols + NT - 1) / NT), COLSUM_CHUNKS);
+    colsumsq_partial_kernel<<<g1, NT, 0, s>>>(W, rows, cols, part);
+    colnorm_final_kernel<<<(unsigned)((cols + NT - 1) / NT), NT, 0, s>>>(part, cols, r1);
+    rownorm_scale_kernel<<<(unsigned)rows, NT, 0, s>>>(W, r1, r2, Wbar, cols);
+    c->launches += 3;
+  } else if (Wbar != W) {
+    copy_kernel<<<grid_for(c->wn / 4), NT, 0, s>>>((const float4*)W, (float4*)Wbar, c->wn / 4);
+    c->launches++;
+  }
+  init_core_kernel<<<grid_for(c->wn / 4), NT, 0, s>>>((const float4*)Wbar, H, cols, (float4*)S, M, c->wn / 4,
+                                                     (int)(cols / 4));
+  identity_blocks_kernel<<<c->nbo, NT, 0, s>>>(A, c->db);
+  identity_blocks_kernel<<<c->nbi, NT, 0, s>>>(B, c->db);
+  c->launches += 3;
+}
+
+void launch_zero_scalars(armor_ctx* c, cudaStream_t s) {
+  const int nflag = c->nbo > c->nbi ? c->nbo : c->nbi;
+  zero_scalars_kernel<<<1, NT, 0, s>>>(c->sc, c->failflag, nflag);
+  c->launches++;
+}
+
+void launch_stage(armor_ctx* c, armor_iter_stats* st, int stage, const double* part, int npart, int nflag,
+                  cudaStream_t s) {
+  stage_kernel<<<1, 32, 0, s>>>(c->sc, st, stage, c->failflag, nflag, part, npart, c->status);
+  c->launches++;
+}
+
+void launch_split_hilo(armor_ctx* c, const float* in, float* hi, float* lo, int64_t n, cudaStream_t s) {
+  split_hilo_kernel<<<grid_for(n / 4), NT, 0, s>>>((const float4*)in, (float4*)hi, (float4*)lo, n / 4);
+  c->launches++;
+}
+
+void launch_transpose_split(armor_ctx* c, const float* X, int64_t ldx, int64_t rows, int64_t cols, float* Thi,
+                            float* Tlo, int64_t ldt, cudaStream_t s) {
+  dim3 grid((unsigned)((cols + 31) / 32), (unsigned)((ldt + 31) / 32));
+  transpose_split_kernel<<<grid, dim3(32, 8), 0, s>>>(X, ldx, rows, cols, Thi, Tlo, ldt);
+  c->launches++;
+}
