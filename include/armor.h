@@ -156,6 +156,17 @@ const char* armor_status_string(armor_status s);
 /* Number of kernel launches the context has enqueued so far (host counter). */
 int64_t armor_launch_count(const armor_ctx* ctx);
 
+/* Measurement aid for the tensor-core GEMM that carries the Gram and the dense
+ * .H contractions (the dominant kernel of the FULL mode).  While enabled, every
+ * launch of that kernel is bracketed by CUDA events on its stream (up to 4096
+ * launches are kept, later ones are not timed).  armor_gemm_timing synchronises
+ * on the recorded events and returns the number of timed launches, their total
+ * duration in milliseconds and their algorithmic flops (2*M*N*K per launch;
+ * M*N*K + M*128*K for the symmetric Gram launches), then clears the record.
+ * Events are created on first use; no device memory is allocated. */
+armor_status armor_gemm_timing_enable(armor_ctx* ctx, int32_t enable);
+armor_status armor_gemm_timing(armor_ctx* ctx, int64_t* n_launches, double* total_ms, double* total_flops);
+
 #ifdef __cplusplus
 }
 #endif

@@ -25,7 +25,7 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 
 EXPORTS = ["armor_workspace_bytes", "armor_create", "armor_destroy", "armor_gram", "armor_init",
            "armor_bcd_step", "armor_proxy_loss", "armor_apply", "armor_get_device_status",
-           "armor_status_string", "armor_launch_count"]
+           "armor_status_string", "armor_launch_count", "armor_gemm_timing_enable", "armor_gemm_timing"]
 
 
 class ArmorError(RuntimeError):
@@ -70,6 +70,8 @@ def lib() -> C.CDLL:
         L.armor_status_string.restype = C.c_char_p
         L.armor_launch_count.argtypes = [vp]
         L.armor_launch_count.restype = i64
+        L.armor_gemm_timing_enable.argtypes = [vp, i32]
+        L.armor_gemm_timing.argtypes = [vp, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
         for name in EXPORTS:
             if name not in ("armor_status_string", "armor_launch_count"):
                 getattr(L, name).restype = C.c_int
@@ -171,6 +173,17 @@ def armor_get_device_status(ctx, n: int = 8) -> list[int]:
 
 def armor_launch_count(ctx) -> int:
     return int(lib().armor_launch_count(ctx))
+
+
+def armor_gemm_timing_enable(ctx, enable: bool) -> None:
+    _check(lib().armor_gemm_timing_enable(ctx, int(bool(enable))), "armor_gemm_timing_enable")
+
+
+def armor_gemm_timing(ctx) -> tuple[int, float, float]:
+    """(timed launches, total milliseconds, total algorithmic flops) since the last call."""
+    n, ms, fl = C.c_int64(0), C.c_double(0), C.c_double(0)
+    _check(lib().armor_gemm_timing(ctx, C.byref(n), C.byref(ms), C.byref(fl)), "armor_gemm_timing")
+    return int(n.value), float(ms.value), float(fl.value)
 
 
 # ---------------------------------------------------------------- convenience wrapper

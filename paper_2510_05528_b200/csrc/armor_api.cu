@@ -190,6 +190,7 @@ armor_status armor_create(armor_ctx** out, const armor_config* cfg, void* d_work
   c->ws = static_cast<char*>(d_workspace); c->ws_bytes = bytes;
   c->launches = 0;
   c->h_cached = nullptr;
+  c->timing_on = 0; c->timing_n = 0; c->ev_beg = nullptr; c->ev_end = nullptr; c->ev_created = 0; c->timing_flops = 0.0;
   carve(*cfg, c, c->ws);
   if (cudaMemset(c->status, 0, ST_COUNT * sizeof(int32_t)) != cudaSuccess) { delete c; return ARMOR_ERR_CUDA; }
   if (cudaMemset(c->sc, 0, SC_COUNT * sizeof(double)) != cudaSuccess) { delete c; return ARMOR_ERR_CUDA; }
@@ -199,11 +200,47 @@ armor_status armor_create(armor_ctx** out, const armor_config* cfg, void* d_work
 
 armor_status armor_destroy(armor_ctx* c) {
   if (!c) return ARMOR_ERR_INVALID_ARG;
+  for (int i = 0; i < c->ev_created; ++i) { cudaEventDestroy(c->ev_beg[i]); cudaEventDestroy(c->ev_end[i]); }
+  delete[] c->ev_beg;
+  delete[] c->ev_end;
   delete c;
   return ARMOR_OK;
 }
 
 int64_t armor_launch_count(const armor_ctx* c) { return c ? c->launches : -1; }
+
+armor_status armor_gemm_timing_enable(armor_ctx* c, int32_t enable) {
+  if (!c) return ARMOR_ERR_INVALID_ARG;
+  if (enable && !c->ev_beg) {
+    c->ev_beg = new (std::nothrow) cudaEvent_t[ARMOR_MAX_TIMED];
+    c->ev_end = new (std::nothrow) cudaEvent_t[ARMOR_MAX_TIMED];
+    if (!c->ev_beg || !c->ev_end) return ARMOR_ERR_INVALID_ARG;
+    for (int i = 0; i < ARMOR_MAX_TIMED; ++i) {
+      if (cudaEventCreate(&c->ev_beg[i]) != cudaSuccess || cudaEventCreate(&c->ev_end[i]) != cudaSuccess)
+        return ARMOR_ERR_CUDA;
+      c->ev_created = i + 1;
+    }
+  }
+  c->timing_on = enable ? 1 : 0;
+  return ARMOR_OK;
+}
+
+armor_status armor_gemm_timing(armor_ctx* c, int64_t* n_launches, double* total_ms, double* total_flops) {
+  if (!c || !n_launches || !total_ms || !total_flops) return ARMOR_ERR_INVALID_ARG;
+  double ms = 0.0;
+  for (int i = 0; i < c->timing_n; ++i) {
+    ARMOR_CUDA_OK(cudaEventSynchronize(c->ev_end[i]));
+    float t = 0.f;
+    ARMOR_CUDA_OK(cudaEventElapsedTime(&t, c->ev_beg[i], c->ev_end[i]));
+    ms += (double)t;
+  }
+  *n_launches = c->timing_n;
+  *total_ms = ms;
+  *total_flops = c->timing_flops;
+  c->timing_n = 0;
+  c->timing_flops = 0.0;
+  return ARMOR_OK;
+}
 
 armor_status armor_get_device_status(armor_ctx* c, int32_t* h_codes, int32_t n) {
   if (!c || !h_codes || n < 0) return ARMOR_ERR_INVALID_ARG;

@@ -72,7 +72,15 @@ struct armor_ctx {
   int64_t launches;
   // identity of the H whose split copy is cached in Hhi/Hlo
   const float* h_cached;
+  // optional event timing of the tensor-core GEMM launches
+  int timing_on;
+  int timing_n;              // launches recorded
+  cudaEvent_t* ev_beg;       // [ARMOR_MAX_TIMED]
+  cudaEvent_t* ev_end;
+  int ev_created;
+  double timing_flops;
 };
+static const int ARMOR_MAX_TIMED = 4096;
 
 #define ARMOR_CUDA_OK(expr)                                  \
   do {                                                       \
@@ -161,6 +169,7 @@ struct TcGemm {
   float* C; int64_t ldc;
   int64_t M, N, K;
   int passes;            // 1 or 3
+  int64_t k_segment;     // K extent accumulated in tensor memory before it is folded into C (0: all of K)
   int accumulate;        // C += (read-modify-write) instead of C =
   int symmetric_lower;   // only tiles with n0 <= m0 are computed; mirrored into the upper triangle (M == N)
   const float* d1; const float* d2;  // optional dot operands (ld = ldc)

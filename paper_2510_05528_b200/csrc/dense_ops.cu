@@ -3,6 +3,11 @@
 // deployment form.  SIMT = fp32 CUDA cores; TF32 / FP32X3 = tcgen05 tensor cores (1 or 3 passes).
 #include "armor_internal.cuh"
 
+// The tensor-core accumulator adds with truncation, so a long run of same-sign terms drifts by about
+// (K / 8) * passes * 2^-24.  The GEMM therefore drains its accumulator into C every K_SEGMENT columns of
+// the contraction (the additions into C are ordinary round-to-nearest fp32 adds).
+static const int64_t K_SEGMENT = 1024;
+
 armor_status prepare_H(armor_ctx* c, const float* H, cudaStream_t s) {
   launch_extract_hblocks(c, H, s);
   if (c->cfg.h_mode == ARMOR_H_FULL && c->cfg.precision == ARMOR_PREC_FP32X3)
@@ -35,6 +40,7 @@ armor_status rmul_H(armor_ctx* c, const float* in, const float* H, float* out, i
       g.A = in; g.B = H; g.passes = 1;
     }
     g.d1 = d1; g.d2 = d2;
+    g.k_segment = K_SEGMENT;
     g.part1 = d1 ? c->partials : nullptr;
     g.part2 = d2 ? c->partials + 4 * c->npart : nullptr;
     int tiles = 0;
@@ -79,6 +85,7 @@ armor_status gram_accumulate(armor_ctx* c, const float* X, int64_t n_rows, int64
     g.passes = x3 ? 3 : 1;
     g.accumulate = 1;
     g.symmetric_lower = 1;
+    g.k_segment = K_SEGMENT;
     armor_status st = launch_tc_gemm(c, g, nullptr, s);
     if (st != ARMOR_OK) return st;
   }
@@ -107,5 +114,6 @@ armor_status apply_core(armor_ctx* c, const float* z1, const float* S, float* z2
   } else {
     g.A = z1; g.B = S; g.passes = 1;
   }
+  g.k_segment = K_SEGMENT;
   return launch_tc_gemm(c, g, nullptr, s);
 }

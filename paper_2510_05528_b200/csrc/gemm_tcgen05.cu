@@ -32,6 +32,7 @@ struct Params {
   int64_t M, N, K;
   int m_tiles, n_tiles, n_tiles_total;
   int accumulate, symmetric_lower;
+  int kt_seg;            // k-tiles accumulated in tensor memory before the epilogue folds them into C
   const float* d1; const float* d2;
   double* part1; double* part2;
   int32_t* status;
@@ -225,37 +226,41 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     if (lane == 0) {
       const uint32_t idesc = instr_desc_tf32();
       int stage = 0; uint32_t phase = 0;
-      int local = 0;
+      int local = 0;   // (tile, K segment) items handled so far: selects the accumulator buffer
       bool ok = true;
-      for (int tile = blockIdx.x; tile < p.n_tiles_total && ok; tile += gridDim.x, ++local) {
-        const int as = local & 1;
-        const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
-        if (!mbar_wait(tempty0 + 8 * as, aphase ^ 1, abortp, p.status)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t tacc = tmem_base + (uint32_t)(as * BN);
-        for (int kt = 0; kt < kt_total; ++kt) {
-          if (!mbar_wait(full0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
+      for (int tile = blockIdx.x; tile < p.n_tiles_total && ok; tile += gridDim.x) {
+        for (int kt0 = 0; kt0 < kt_total && ok; kt0 += p.kt_seg, ++local) {
+          const int as = local & 1;
+          const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
+          if (!mbar_wait(tempty0 + 8 * as, aphase ^ 1, abortp, p.status)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
-          const uint32_t sa_lo = sa + A_BYTES;
-          const uint32_t sb = sa + (PASSES == 3 ? 2 : 1) * A_BYTES;
-          const uint32_t sb_lo = sb + B_BYTES;
+          const uint32_t tacc = tmem_base + (uint32_t)(as * BN);
+          const int kt1 = min(kt_total, kt0 + p.kt_seg);
+          for (int kt = kt0; kt < kt1; ++kt) {
+            if (!mbar_wait(full0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+            const uint32_t sa_lo = sa + A_BYTES;
+            const uint32_t sb = sa + (PASSES == 3 ? 2 : 1) * A_BYTES;
+            const uint32_t sb_lo = sb + B_BYTES;
 #pragma unroll
-          for (int k = 0; k < BK / 8; ++k) {
-            const uint64_t da = smem_desc_k_sw128(sa + k * 32), dbm = smem_desc_k_sw128(sb + k * 32);
-            if (PASSES == 3) {
-              const uint64_t dal = smem_desc_k_sw128(sa_lo + k * 32), dbl = smem_desc_k_sw128(sb_lo + k * 32);
-              umma_tf32(tacc, dal, dbm, idesc, (kt | k) != 0);
-              umma_tf32(tacc, da, dbl, idesc, 1);
-              umma_tf32(tacc, da, dbm, idesc, 1);
-            } else {
-              umma_tf32(tacc, da, dbm, idesc, (kt | k) != 0);
+            for (int k = 0; k < BK / 8; ++k) {
+              const uint64_t da = smem_desc_k_sw128(sa + k * 32), dbm = smem_desc_k_sw128(sb + k * 32);
+              const uint32_t acc = (uint32_t)((kt > kt0) | (k != 0));
+              if (PASSES == 3) {
+                const uint64_t dal = smem_desc_k_sw128(sa_lo + k * 32), dbl = smem_desc_k_sw128(sb_lo + k * 32);
+                umma_tf32(tacc, dal, dbm, idesc, acc);
+                umma_tf32(tacc, da, dbl, idesc, 1);
+                umma_tf32(tacc, da, dbm, idesc, 1);
+              } else {
+                umma_tf32(tacc, da, dbm, idesc, acc);
+              }
             }
+            umma_commit(empty0 + 8 * stage);   // frees the stage once these MMAs have read it
+            if (++stage == STAGES) { stage = 0; phase ^= 1; }
           }
-          umma_commit(empty0 + 8 * stage);   // frees the stage once these MMAs have read it
-          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+          if (ok) umma_commit(tfull0 + 8 * as);
         }
-        if (ok) umma_commit(tfull0 + 8 * as);
       }
     }
   } else {
@@ -263,66 +268,70 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     int local = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < p.n_tiles_total && ok; tile += gridDim.x, ++local) {
+    for (int tile = blockIdx.x; tile < p.n_tiles_total && ok; tile += gridDim.x) {
       int mt, nt;
       tile_coords(p, tile, mt, nt);
-      const int as = local & 1;
-      const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
-      if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
-      tc_fence_after();
       const int64_t row = (int64_t)mt * BM + q * 32 + lane;
       const bool row_ok = row < p.M;
       double dot1 = 0.0, dot2 = 0.0;
+      for (int kt0 = 0; kt0 < kt_total && ok; kt0 += p.kt_seg, ++local) {
+        const int as = local & 1;
+        const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
+        const bool accum = p.accumulate || kt0 > 0;           // later K segments add to what is in C
+        const bool last = kt0 + p.kt_seg >= kt_total;
+        if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
+        tc_fence_after();
 #pragma unroll 1
-      for (int ch = 0; ch < BN / 32; ++ch) {
-        const int64_t col0 = (int64_t)nt * BN + ch * 32;
-        uint32_t r[32];
-        tmem_ld32(tmem_base + (uint32_t)(as * BN + ch * 32) + ((uint32_t)(q * 32) << 16), r);
-        if (col0 >= p.N || !row_ok) continue;
-        float* crow = p.C + row * p.ldc + col0;
-        if (!p.symmetric_lower) {
-          float f1 = 0.f, f2 = 0.f;
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          const int64_t col0 = (int64_t)nt * BN + ch * 32;
+          uint32_t r[32];
+          tmem_ld32(tmem_base + (uint32_t)(as * BN + ch * 32) + ((uint32_t)(q * 32) << 16), r);
+          if (col0 >= p.N || !row_ok) continue;
+          float* crow = p.C + row * p.ldc + col0;
+          if (!p.symmetric_lower) {
+            float f1 = 0.f, f2 = 0.f;
 #pragma unroll
-          for (int i = 0; i < 32; i += 4) {
-            float4 v = make_float4(__uint_as_float(r[i]), __uint_as_float(r[i + 1]), __uint_as_float(r[i + 2]),
-                                   __uint_as_float(r[i + 3]));
-            if (p.accumulate) {
-              const float4 o = *reinterpret_cast<const float4*>(crow + i);
-              v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+            for (int i = 0; i < 32; i += 4) {
+              float4 v = make_float4(__uint_as_float(r[i]), __uint_as_float(r[i + 1]), __uint_as_float(r[i + 2]),
+                                     __uint_as_float(r[i + 3]));
+              if (accum) {
+                const float4 o = *reinterpret_cast<const float4*>(crow + i);
+                v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+              }
+              if (last && p.d1) {
+                const float4 d = *reinterpret_cast<const float4*>(p.d1 + row * p.ldc + col0 + i);
+                f1 = fmaf(v.x, d.x, f1); f1 = fmaf(v.y, d.y, f1); f1 = fmaf(v.z, d.z, f1); f1 = fmaf(v.w, d.w, f1);
+              }
+              if (last && p.d2) {
+                const float4 d = *reinterpret_cast<const float4*>(p.d2 + row * p.ldc + col0 + i);
+                f2 = fmaf(v.x, d.x, f2); f2 = fmaf(v.y, d.y, f2); f2 = fmaf(v.z, d.z, f2); f2 = fmaf(v.w, d.w, f2);
+              }
+              *reinterpret_cast<float4*>(crow + i) = v;
             }
-            if (p.d1) {
-              const float4 d = *reinterpret_cast<const float4*>(p.d1 + row * p.ldc + col0 + i);
-              f1 = fmaf(v.x, d.x, f1); f1 = fmaf(v.y, d.y, f1); f1 = fmaf(v.z, d.z, f1); f1 = fmaf(v.w, d.w, f1);
-            }
-            if (p.d2) {
-              const float4 d = *reinterpret_cast<const float4*>(p.d2 + row * p.ldc + col0 + i);
-              f2 = fmaf(v.x, d.x, f2); f2 = fmaf(v.y, d.y, f2); f2 = fmaf(v.z, d.z, f2); f2 = fmaf(v.w, d.w, f2);
-            }
-            *reinterpret_cast<float4*>(crow + i) = v;
-          }
-          dot1 += (double)f1;
-          dot2 += (double)f2;
-        } else {
-          // lower triangle (+ diagonal) is owned by this tile; each kept element is mirrored once
+            dot1 += (double)f1;
+            dot2 += (double)f2;
+          } else {
+            // lower triangle (+ diagonal) is owned by this tile; each kept element is mirrored once
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int64_t cc = col0 + i;
-            if (cc <= row) {
-              const float v = __uint_as_float(r[i]);
-              crow[i] = p.accumulate ? crow[i] + v : v;
-              if (cc < row) {
-                float* mp = p.C + cc * p.ldc + row;
-                *mp = p.accumulate ? *mp + v : v;
+            for (int i = 0; i < 32; ++i) {
+              const int64_t cc = col0 + i;
+              if (cc <= row) {
+                const float v = __uint_as_float(r[i]);
+                crow[i] = accum ? crow[i] + v : v;
+                if (cc < row) {
+                  float* mp = p.C + cc * p.ldc + row;
+                  *mp = accum ? *mp + v : v;
+                }
               }
             }
           }
         }
+        // accumulator buffer is free again
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty0 + 8 * as);
       }
-      // accumulator buffer is free again
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(tempty0 + 8 * as);
-      if (p.part1 || p.part2) {
+      if (ok && (p.part1 || p.part2)) {
         for (int o = 16; o > 0; o >>= 1) {
           dot1 += __shfl_down_sync(0xffffffffu, dot1, o);
           dot2 += __shfl_down_sync(0xffffffffu, dot2, o);
@@ -397,7 +406,15 @@ armor_status launch_impl(armor_ctx* c, const TcGemm& g, const Params& p, cudaStr
     if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ARMOR_ERR_CUDA;
   }
   const int grid = p.n_tiles_total < n_sm ? p.n_tiles_total : n_sm;
+  const bool timed = c->timing_on && c->timing_n < ARMOR_MAX_TIMED;
+  if (timed) cudaEventRecord(c->ev_beg[c->timing_n], s);
   tc_gemm_kernel<PASSES><<<grid, NTHREADS, SMEM, s>>>(mA, mAlo, mB, mBlo, p);
+  if (timed) {
+    cudaEventRecord(c->ev_end[c->timing_n], s);
+    c->timing_n++;
+    c->timing_flops += p.symmetric_lower ? (double)p.M * (double)(p.N + BM) * (double)p.K
+                                         : 2.0 * (double)p.M * (double)p.N * (double)p.K;
+  }
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
 }
@@ -429,6 +446,8 @@ armor_status launch_tc_gemm(armor_ctx* c, const TcGemm& g, int* n_tiles, cudaStr
   p.accumulate = g.accumulate; p.symmetric_lower = g.symmetric_lower;
   p.d1 = g.d1; p.d2 = g.d2; p.part1 = g.part1; p.part2 = g.part2;
   p.status = c->status;
+  p.kt_seg = g.k_segment > 0 ? (int)((g.k_segment + BK - 1) / BK) : (int)((g.K + BK - 1) / BK);
+  if (p.kt_seg < 1) p.kt_seg = 1;
   if (n_tiles) *n_tiles = p.n_tiles_total;
   if (g.passes == 3) return launch_impl<3>(c, g, p, s);
   return launch_impl<1>(c, g, p, s);

@@ -1,0 +1,129 @@
+"""Parity at the benchmark's full size (4096 x 4096, d_block 128, FP32X3 tensor-core mode -- the launch
+configuration bench.py times), on outputs the oracle can produce one at a time: sampled Gram entries,
+the loss, single row-blocks of the A-step, single column-blocks of the B-step, and properties that hold
+at any size (valid 2:4 masks, zeros off the mask, monotone loss)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import armor_oracle as O
+from paper_2510_05528_b200 import binding as Bd
+from paper_2510_05528_b200 import inputs
+from tests.helpers import DEV, dev, host, rel
+
+pytestmark = pytest.mark.gpu
+
+CFG = inputs.CONFIGS["llama7b_attn"]
+
+
+@pytest.fixture(scope="module")
+def layer():
+    """Gram of a 32,768-token slice of the full calibration set (the full 262,144 tokens are covered by
+    the sampled-entry test below), accumulated by the library chunk by chunk."""
+    ctx = Bd.ArmorContext(CFG.d_out, CFG.d_in, CFG.d_block, device=DEV, precision=Bd.PREC_FP32X3, seed=CFG.seed)
+    W = inputs.make_weight(CFG)
+    H = ctx.new_gram()
+    scales = torch.from_numpy(inputs.channel_scales(CFG))
+    for i in range(4):
+        ctx.gram(inputs.activation_chunk(CFG, i, scales).to(DEV), H)
+    torch.cuda.synchronize()
+    return ctx, W, H
+
+
+def test_gram_full_token_count_on_sampled_entries():
+    """All 262,144 tokens through armor_gram; 96 sampled entries (diagonal, outlier rows, random pairs)
+    recomputed in fp64 straight from the activations."""
+    ctx = Bd.ArmorContext(CFG.d_out, CFG.d_in, CFG.d_block, device=DEV, precision=Bd.PREC_FP32X3, seed=CFG.seed)
+    H = ctx.new_gram()
+    scales_np = inputs.channel_scales(CFG)
+    scales = torch.from_numpy(scales_np)
+    rng = np.random.default_rng(0)
+    big = np.argsort(-scales_np)[:8]
+    aa = np.concatenate([rng.integers(0, CFG.d_in, 64), big, big, big[::-1], rng.integers(0, CFG.d_in, 8)])
+    bb = np.concatenate([rng.integers(0, CFG.d_in, 64), big, big[::-1], rng.integers(0, CFG.d_in, 8), rng.integers(0, CFG.d_in, 8)])
+    aa[:16] = bb[:16]                               # some diagonal entries
+    ref = np.zeros(len(aa))
+    stage = None
+    for i in range(inputs.n_chunks(CFG)):
+        xc = inputs.activation_chunk(CFG, i, scales)
+        xd = xc.to(DEV, non_blocking=False)
+        ctx.gram(xd, H)
+        x64 = xc.numpy()
+        ref += np.einsum("ti,ti->i", x64[:, aa].astype(np.float64), x64[:, bb].astype(np.float64))
+    torch.cuda.synchronize()
+    Hh = host(H)
+    got = Hh[aa, bb]
+    # entries are compared against the scale of their row/column: |H_ab| <= sqrt(H_aa H_bb)
+    scale = np.sqrt(np.diag(Hh)[aa].astype(np.float64) * np.diag(Hh)[bb].astype(np.float64))
+    assert np.max(np.abs(got - ref) / scale) < 1e-4
+    assert np.array_equal(Hh, Hh.T)
+    assert ctx.device_status()[:4] == [0, 0, 0, 0]
+
+
+def test_loss_and_first_iteration_blocks(layer):
+    ctx, W, H = layer
+    Hd = H
+    Hq = host(H).astype(np.float64)
+    Wn = W.astype(np.float64)
+    db = CFG.d_block
+    oc = O.OracleConfig(db, seed=CFG.seed)
+    st = ctx.init(dev(W), Hd)
+    A, B, S, M = O.init(Wn, Hq, oc)
+    assert np.array_equal(host(st.M), O.pack_mask(M))
+    L0 = O.proxy_loss(Wn, A, B, S, Hq)
+    assert abs(ctx.proxy_loss(st, Hd).item() - L0) / L0 < 1e-3
+
+    # --- A-step alone; three sampled row-blocks recomputed by the oracle on their own rows
+    ctxA = Bd.ArmorContext(CFG.d_out, CFG.d_in, db, device=DEV, precision=Bd.PREC_FP32X3, seed=CFG.seed,
+                           phases=Bd.PHASE_A)
+    stA = ctxA.init(dev(W), Hd)
+    sgA = ctxA.read_stats(ctxA.bcd_step(stA, Hd, 0, 1))[0]
+    A_gpu = host(stA.A)
+    for i in (0, 13, CFG.d_out // db - 1):
+        r = slice(i * db, (i + 1) * db)
+        Ai, failed = O.a_step(Wn[r], A[i:i + 1], B, S[r], Hq, oc)
+        assert failed == 0 and rel(A_gpu[i], Ai[0]) < 1e-3
+    assert sgA["loss_A"] < sgA["loss_start"] and abs(sgA["loss_start"] - L0) / L0 < 1e-3
+    A1 = A_gpu.astype(np.float64)
+
+    # --- B-step alone from (A1, B, S): two sampled column-blocks.  The direction of block j needs
+    # U = A S (block products) and the columns of E H_w of that block.
+    ctxB = Bd.ArmorContext(CFG.d_out, CFG.d_in, db, device=DEV, precision=Bd.PREC_FP32X3, seed=CFG.seed,
+                           phases=Bd.PHASE_B)
+    stB = ctxB.init(dev(W), Hd)
+    stB.A.copy_(stA.A)
+    sgB = ctxB.read_stats(ctxB.bcd_step(stB, Hd, 0, 1))[0]
+    U = O.bd_left(A1, S)
+    E = Wn - O.bd_right(U, B)
+    dB_gpu = (host(stB.B).astype(np.float64) - B) / float(sgB["tau_B"])
+    for j in (1, CFG.d_in // db - 2):
+        c = slice(j * db, (j + 1) * db)
+        Uj = U[:, c]
+        C = Uj.T @ Uj
+        Gam = Uj.T @ (E @ Hq[:, c])
+        Hjj = Hq[c, c]
+        Y = np.linalg.solve(C + oc.ridge * np.trace(C) / db * np.eye(db), Gam)
+        Dj = np.linalg.solve(Hjj + oc.ridge * np.trace(Hjj) / db * np.eye(db), Y.T).T
+        assert rel(dB_gpu[j], Dj) < 2e-3
+    assert 0.5 < sgB["tau_B"] < 1.5 and sgB["loss_B"] < sgB["loss_start"]
+
+
+def test_full_iterations_properties(layer):
+    ctx, W, H = layer
+    st = ctx.init(dev(W), H)
+    L_init = ctx.proxy_loss(st, H).item()
+    stats = ctx.read_stats(ctx.bcd_step(st, H, 0, 3))
+    seq = [L_init]
+    for s in stats:
+        seq += [s["loss_start"], s["loss_A"], s["loss_B"], s["loss_S"], s["loss_mask"]]
+    for a, b in zip(seq, seq[1:]):
+        assert b <= a * (1 + 1e-5)
+    assert abs(ctx.proxy_loss(st, H).item() - seq[-1]) / seq[-1] < 1e-3
+    Mb = host(st.M)
+    bits = np.unpackbits(Mb[:, :, None], axis=2)[:, :, 4:]
+    assert np.all(bits.sum(axis=2) == 2) and np.all(Mb < 16)
+    M = O.unpack_mask(Mb)
+    assert np.all(host(st.S)[~M] == 0.0)
+    assert stats["chol_failed"].sum() == 0
+    assert all(0 <= g <= (CFG.d_out // CFG.d_block) * (CFG.d_in // CFG.d_block) for g in stats["groups_changed"])
+    assert ctx.device_status()[:4] == [0, 0, 0, 0]

@@ -1,0 +1,350 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the fp64 CPU oracle on the same
+seeded inputs.  Integer / byte results (masks) must be identical wherever the decision margin exceeds
+the stated threshold; floating-point results must agree within the tolerances of tests/helpers.py."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import armor_oracle as O
+from paper_2510_05528_b200 import binding as Bd
+from paper_2510_05528_b200 import inputs
+from tests.helpers import DEV, TOL, dev, excused_blocks, host, load_state, mask_block_diffs, rel
+
+pytestmark = pytest.mark.gpu
+
+TINY = inputs.CONFIGS["tiny"]
+MID = TINY.with_(name="mid", d_out=384, d_in=512, d_block=128, n_tokens=6000, chunk_rows=2048, seed=11)
+PRECS = [Bd.PREC_SIMT, Bd.PREC_FP32X3, Bd.PREC_TF32]
+PNAME = {Bd.PREC_SIMT: "simt", Bd.PREC_FP32X3: "fp32x3", Bd.PREC_TF32: "tf32"}
+
+
+def make(cfg, precision, h_mode=Bd.H_FULL, **kw):
+    return Bd.ArmorContext(cfg.d_out, cfg.d_in, cfg.d_block, device=DEV, precision=precision, h_mode=h_mode,
+                           seed=cfg.seed, **kw)
+
+
+@pytest.fixture(scope="module")
+def tiny_data():
+    W = inputs.make_weight(TINY)
+    X = inputs.make_activations(TINY)
+    H32 = O.gram(X).astype(np.float32)          # one H, rounded once, given to both sides
+    return W, X, H32
+
+
+@pytest.fixture(scope="module")
+def mid_data():
+    W = inputs.make_weight(MID)
+    X = inputs.make_activations(MID)
+    H32 = O.gram(X).astype(np.float32)
+    return W, X, H32
+
+
+# ------------------------------------------------------------------------------------------ Gram
+@pytest.mark.parametrize("prec", PRECS, ids=PNAME.get)
+def test_gram_matches_oracle_with_ragged_chunks(prec, mid_data):
+    W, X, _ = mid_data
+    ctx = make(MID, prec)
+    H = ctx.new_gram()
+    Xd = dev(X)
+    # chunks of uneven length, one of them empty, one not a multiple of the K tile, one a strided view
+    bounds = [0, 2048, 2048, 2048 + 37, 5000, MID.n_tokens]
+    for lo, hi in zip(bounds, bounds[1:]):
+        ctx.gram(Xd[lo:hi], H)
+    torch.cuda.synchronize()
+    Hg = host(H)
+    Ho = O.gram(X)
+    assert rel(Hg, Ho) < TOL[prec]["gram"]
+    assert np.array_equal(Hg, Hg.T) or rel(Hg, Hg.T) < 1e-6
+    assert rel(np.diag(Hg), (X.astype(np.float64) ** 2).sum(axis=0)) < TOL[prec]["gram"]
+    assert ctx.device_status()[:4] == [0, 0, 0, 0]
+
+
+def test_gram_strided_input_and_accumulation():
+    cfg = MID
+    ctx = make(cfg, Bd.PREC_FP32X3)
+    rng = np.random.default_rng(0)
+    Xw = rng.standard_normal((700, cfg.d_in + 64)).astype(np.float32)
+    Xd = dev(Xw)[:, : cfg.d_in]                  # leading dimension larger than d_in
+    H = ctx.new_gram()
+    ctx.gram(Xd, H)
+    ctx.gram(Xd, H)
+    torch.cuda.synchronize()
+    assert rel(host(H), 2 * O.gram(Xw[:, : cfg.d_in])) < 1e-4
+
+
+# ------------------------------------------------------------------------------------------ init
+@pytest.mark.parametrize("normalize", [0, 1])
+def test_init_matches_oracle(normalize, tiny_data):
+    W, X, H32 = tiny_data
+    ctx = make(TINY, Bd.PREC_SIMT, normalize=normalize)
+    st = ctx.init(dev(W), dev(H32))
+    torch.cuda.synchronize()
+    Wn = W.astype(np.float64)
+    if normalize:
+        Wn, r1, r2 = O.normalize(W)
+        assert rel(host(st.r1), r1) < 1e-6 and rel(host(st.r2), r2) < 1e-6
+        assert rel(host(st.Wbar), Wn) < 1e-6
+        assert np.allclose((host(st.Wbar).astype(np.float64) ** 2).sum(axis=1), 1.0, atol=1e-5)
+        Wn = host(st.Wbar).astype(np.float64)     # decide the masks on the same fp32 values
+    else:
+        assert np.array_equal(host(st.Wbar), W)
+    A, B, S, M = O.init(Wn, H32.astype(np.float64), O.OracleConfig(TINY.d_block))
+    assert np.array_equal(host(st.M), O.pack_mask(M))          # byte-exact
+    assert np.array_equal(host(st.S), S.astype(np.float32))
+    assert np.array_equal(host(st.A), A.astype(np.float32)) and np.array_equal(host(st.B), B.astype(np.float32))
+
+
+def test_init_ties_and_zero_norms():
+    cfg = TINY.with_(d_out=32, d_in=32, d_block=32)
+    ctx = make(cfg, Bd.PREC_SIMT, normalize=1)
+    W = np.ones((32, 32), dtype=np.float32)
+    W[:, 5] = 0.0
+    W[7, :] = 0.0
+    H = np.eye(32, dtype=np.float32)
+    st = ctx.init(dev(W), dev(H))
+    torch.cuda.synchronize()
+    Wn, r1, r2 = O.normalize(W)
+    assert host(st.r1)[5] == 1.0 and host(st.r2)[7] == 1.0
+    _, _, _, M = O.init(host(st.Wbar).astype(np.float64), H.astype(np.float64), O.OracleConfig(32))
+    assert np.array_equal(host(st.M), O.pack_mask(M))
+    assert host(st.M)[0, 0] == 3                                # all equal: the two lowest columns win
+
+
+# ------------------------------------------------------------------------------------------ loss
+@pytest.mark.parametrize("h_mode", [Bd.H_FULL, Bd.H_DIAG])
+@pytest.mark.parametrize("prec", PRECS, ids=PNAME.get)
+def test_proxy_loss_matches_oracle(prec, h_mode, mid_data):
+    W, X, H32 = mid_data
+    ctx = make(MID, prec, h_mode)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    oc = O.OracleConfig(MID.d_block, h_mode=h_mode)
+    Hw = O.weighting(H32.astype(np.float64), h_mode)
+    rng = np.random.default_rng(3)
+    A, B, S, M = O.init(W.astype(np.float64), H32.astype(np.float64), oc)
+    A = A + 0.05 * rng.standard_normal(A.shape)
+    B = B + 0.05 * rng.standard_normal(B.shape)
+    A, B, S = A.astype(np.float32).astype(np.float64), B.astype(np.float32).astype(np.float64), S
+    load_state(st, A, B, S, M)
+    Lg = ctx.proxy_loss(st, Hd).item()
+    Lo = O.proxy_loss(W.astype(np.float64), A, B, S, Hw)
+    assert abs(Lg - Lo) / Lo < TOL[prec]["loss"]
+    if h_mode == Bd.H_FULL and prec != Bd.PREC_TF32:
+        # tr(E H E^T) = ||E X^T||_F^2 straight from the activations
+        E = W - O.bd_dense(A) @ S @ O.bd_dense(B)
+        assert abs(Lg - np.linalg.norm(E @ X.T.astype(np.float64)) ** 2) / Lo < 1e-3
+
+
+# ------------------------------------------------------------------------- teacher-forced steps
+def run_teacher_forced(cfg, W, H32, prec, h_mode, n_steps, select=Bd.SELECT_L1_RANDOM):
+    ctx = make(cfg, prec, h_mode, select_mode=select)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    oc = O.OracleConfig(cfg.d_block, h_mode=h_mode, seed=cfg.seed, select_mode=select)
+    Hq = H32.astype(np.float64)
+    Hw = O.weighting(Hq, h_mode)
+    Wn = W.astype(np.float64)
+    A, B, S, M = O.init(Wn, Hq, oc)
+    tol = TOL[prec]
+    n_excused = 0
+    worst = dict(A=0.0, B=0.0, S=0.0, loss=0.0)
+    for t in range(n_steps):
+        load_state(st, A, B, S, M)                 # the GPU starts every step from the oracle's state
+        stats = ctx.bcd_step(st, Hd, t, 1)
+        sg = ctx.read_stats(stats)[0]
+        A, B, S, M, info = O.bcd_iteration(Wn, A, B, S, M, Hw, oc, t)
+        worst["A"] = max(worst["A"], rel(host(st.A), A))
+        worst["B"] = max(worst["B"], rel(host(st.B), B))
+        for k_gpu, k_or in (("loss_start", "start"), ("loss_A", "A"), ("loss_B", "B"), ("loss_S", "S")):
+            worst["loss"] = max(worst["loss"], abs(sg[k_gpu] - info.loss[k_or]) / info.loss[k_or])
+        assert abs(sg["tau_B"] - info.tau_B) <= 10 * tol["B"] * abs(info.tau_B) + 1e-6
+        assert sg["chol_failed"] == info.chol_failed == 0
+        # masks: identical outside blocks whose decision margin is below the threshold
+        diff = mask_block_diffs(host(st.M), M, cfg.d_block)
+        excused = excused_blocks(info, tol["margin"])
+        guard_close = abs(info.delta_L_mask) <= tol["margin"] * info.loss["S"]
+        if sg["mask_accepted"] != info.mask_accepted:
+            assert guard_close, "accept/reject differs although the guard was not marginal"
+            n_excused += len(diff)
+            continue
+        assert diff <= excused, f"step {t}: masks differ in blocks {sorted(diff - excused)} with a clear margin"
+        n_excused += len(diff)
+        if not diff:
+            worst["S"] = max(worst["S"], rel(host(st.S), S))
+            assert sg["groups_changed"] == info.groups_changed
+            worst["loss"] = max(worst["loss"], abs(sg["loss_mask"] - info.loss["mask"]) / info.loss["mask"])
+    assert ctx.device_status()[:4] == [0, 0, 0, 0]
+    for k in worst:
+        assert worst[k] < tol[k], (k, worst)
+    return worst, n_excused
+
+
+@pytest.mark.parametrize("h_mode", [Bd.H_FULL, Bd.H_DIAG])
+@pytest.mark.parametrize("prec", [Bd.PREC_SIMT, Bd.PREC_FP32X3], ids=PNAME.get)
+def test_teacher_forced_all_20_steps_of_the_tiny_config(prec, h_mode, tiny_data):
+    W, X, H32 = tiny_data
+    worst, n_excused = run_teacher_forced(TINY, W, H32, prec, h_mode, TINY.n_iters)
+    print(f"tiny {PNAME[prec]} h_mode={h_mode}: worst rel err {worst}, groups differing under the margin: {n_excused}")
+    assert n_excused <= 2
+
+
+@pytest.mark.parametrize("prec", PRECS, ids=PNAME.get)
+def test_teacher_forced_mid_config_d_block_128(prec, mid_data):
+    W, X, H32 = mid_data
+    worst, n_excused = run_teacher_forced(MID, W, H32, prec, Bd.H_FULL, 4)
+    print(f"mid {PNAME[prec]}: worst rel err {worst}, groups differing under the margin: {n_excused}")
+
+
+def test_teacher_forced_greedy_selection(tiny_data):
+    W, X, H32 = tiny_data
+    run_teacher_forced(TINY, W, H32, Bd.PREC_FP32X3, Bd.H_FULL, 5, select=Bd.SELECT_L1_GREEDY)
+
+
+@pytest.mark.parametrize("phase", [Bd.PHASE_A, Bd.PHASE_B, Bd.PHASE_S, Bd.PHASE_MASK])
+def test_each_sub_step_alone(phase, mid_data):
+    """One sub-step from a perturbed state: isolates A-step, B-step, S-step and the sparse-core update."""
+    W, X, H32 = mid_data
+    cfg = MID
+    ctx = make(cfg, Bd.PREC_FP32X3, Bd.H_FULL, phases=phase)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    oc = O.OracleConfig(cfg.d_block, seed=cfg.seed, phases=phase)
+    Hq = H32.astype(np.float64)
+    Wn = W.astype(np.float64)
+    rng = np.random.default_rng(5)
+    A, B, S, M = O.init(Wn, Hq, oc)
+    A = (A + 0.03 * rng.standard_normal(A.shape)).astype(np.float32).astype(np.float64)
+    B = (B + 0.03 * rng.standard_normal(B.shape)).astype(np.float32).astype(np.float64)
+    load_state(st, A, B, S, M)
+    stats = ctx.bcd_step(st, Hd, 7, 1)
+    sg = ctx.read_stats(stats)[0]
+    A1, B1, S1, M1, info = O.bcd_iteration(Wn, A, B, S, M, Hq, oc, 7)
+    assert rel(host(st.A), A1) < 1e-3 and rel(host(st.B), B1) < 1e-3
+    diff = mask_block_diffs(host(st.M), M1, cfg.d_block)
+    if phase == Bd.PHASE_MASK:
+        assert diff <= excused_blocks(info, 1e-5)
+        assert sg["mask_accepted"] == info.mask_accepted
+        assert abs(sg["delta_L_mask"] - info.delta_L_mask) <= 1e-3 * abs(info.delta_L_mask) + 1e-9 * info.loss["start"]
+    else:
+        assert not diff
+    if not diff:
+        assert rel(host(st.S), S1) < 1e-3
+    last = {Bd.PHASE_A: "A", Bd.PHASE_B: "B", Bd.PHASE_S: "S", Bd.PHASE_MASK: "mask"}[phase]
+    assert abs(sg["loss_mask"] - info.loss[last]) / info.loss[last] < 1e-3
+    # the loss the library reports is the loss of the state it leaves behind
+    assert abs(ctx.proxy_loss(st, Hd).item() - sg["loss_mask"]) / sg["loss_mask"] < 1e-4
+
+
+# ------------------------------------------------------------------------------ free-running run
+@pytest.mark.parametrize("h_mode", [Bd.H_FULL, Bd.H_DIAG])
+def test_free_running_tiny_config(h_mode, tiny_data):
+    W, X, H32 = tiny_data
+    cfg = TINY
+    ctx = make(cfg, Bd.PREC_FP32X3, h_mode)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    L_init = ctx.proxy_loss(st, Hd).item()
+    stats = ctx.read_stats(ctx.bcd_step(st, Hd, 0, cfg.n_iters))
+    oc = O.OracleConfig(cfg.d_block, h_mode=h_mode, seed=cfg.seed)
+    (A, B, S, M), infos = O.run(W.astype(np.float64), H32.astype(np.float64), oc, cfg.n_iters)
+    # Theorem 1 on the GPU trace: never increases, never above the 2:4-pruned initialisation
+    seq = [L_init]
+    for s in stats:
+        seq += [s["loss_start"], s["loss_A"], s["loss_B"], s["loss_S"], s["loss_mask"]]
+    for a, b in zip(seq, seq[1:]):
+        assert b <= a * (1 + 1e-6)
+    assert seq[-1] < 0.6 * L_init
+    L_end = ctx.proxy_loss(st, Hd).item()
+    assert abs(L_end - stats[-1]["loss_mask"]) / L_end < 1e-4
+    diff_groups = int((host(st.M) != O.pack_mask(M)).sum())
+    print(f"free run h_mode={h_mode}: final loss gpu {L_end:.6g} oracle {infos[-1].loss['mask']:.6g}, "
+          f"groups with a different mask: {diff_groups} of {M.size // 4}")
+    assert abs(L_end - infos[-1].loss["mask"]) / infos[-1].loss["mask"] < 1e-2
+    if diff_groups == 0:
+        assert rel(host(st.A), A) < 1e-3 and rel(host(st.B), B) < 1e-3 and rel(host(st.S), S) < 1e-3
+        assert abs(L_end - infos[-1].loss["mask"]) / L_end < 1e-3
+    M_gpu = O.unpack_mask(host(st.M))
+    assert np.all(M_gpu.reshape(cfg.d_out, -1, 4).sum(axis=2) == 2)
+    assert np.all(host(st.S)[~M_gpu] == 0.0)
+
+
+def test_resume_gives_the_same_bits(tiny_data):
+    W, X, H32 = tiny_data
+    Hd = dev(H32)
+    outs = []
+    for split in ([20], [10, 10], [1, 7, 12]):
+        ctx = make(TINY, Bd.PREC_FP32X3)
+        st = ctx.init(dev(W), Hd)
+        t = 0
+        for n in split:
+            ctx.bcd_step(st, Hd, t, n, want_stats=False)
+            t += n
+        torch.cuda.synchronize()
+        outs.append([host(x).copy() for x in (st.A, st.B, st.S, st.M)])
+    for other in outs[1:]:
+        for a, b in zip(outs[0], other):
+            assert np.array_equal(a, b)
+
+
+def test_zero_iterations_is_a_no_op(tiny_data):
+    W, X, H32 = tiny_data
+    ctx = make(TINY, Bd.PREC_SIMT)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    before = [host(x).copy() for x in (st.A, st.B, st.S, st.M)]
+    ctx.bcd_step(st, Hd, 0, 0)
+    torch.cuda.synchronize()
+    for a, b in zip(before, (st.A, st.B, st.S, st.M)):
+        assert np.array_equal(a, host(b))
+
+
+def test_singular_block_is_skipped_and_reported(tiny_data):
+    """A row-block of zeros in S makes G_i = 0: that block of A must stay unchanged and be counted."""
+    W, X, H32 = tiny_data
+    ctx = make(TINY, Bd.PREC_SIMT, phases=Bd.PHASE_A)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    st.S[: TINY.d_block] = 0.0
+    A0 = host(st.A).copy()
+    sg = ctx.read_stats(ctx.bcd_step(st, Hd, 0, 1))[0]
+    assert sg["chol_failed"] == 1
+    assert np.array_equal(host(st.A)[0], A0[0])
+    assert not np.array_equal(host(st.A)[1], A0[1])
+    status = ctx.device_status()
+    assert status[0] == 1 and status[1] == 1
+
+
+# ------------------------------------------------------------------------------------------ apply
+@pytest.mark.parametrize("prec", PRECS, ids=PNAME.get)
+@pytest.mark.parametrize("n_tokens", [1, 77, 600])
+def test_apply_matches_oracle(prec, n_tokens, mid_data):
+    W, X, H32 = mid_data
+    cfg = MID
+    ctx = make(cfg, prec, normalize=1)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    ctx.bcd_step(st, Hd, 0, 2, want_stats=False)
+    x = inputs.make_tokens(cfg, n_tokens)
+    A, B, S = (host(t).astype(np.float64) for t in (st.A, st.B, st.S))
+    tol = 1e-5 if prec != Bd.PREC_TF32 else 5e-3
+    y = host(ctx.apply(st, dev(x)))
+    assert rel(y, O.apply(A, B, S, x)) < tol
+    yd = host(ctx.apply(st, dev(x), denormalize=True))
+    r1, r2 = host(st.r1).astype(np.float64), host(st.r2).astype(np.float64)
+    assert rel(yd, O.apply(A, B, S, x, r1, r2)) < tol
+    # against the dense definition
+    What = np.diag(r2) @ O.bd_dense(A) @ S @ O.bd_dense(B) @ np.diag(r1)
+    assert rel(yd, x.astype(np.float64) @ What.T) < tol
+
+
+def test_apply_zero_tokens_and_more_tokens_than_rows(mid_data):
+    W, X, H32 = mid_data
+    ctx = make(MID, Bd.PREC_FP32X3)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    y0 = ctx.apply(st, torch.empty(0, MID.d_in, device=DEV))
+    assert y0.shape == (0, MID.d_out)
+    x = inputs.make_tokens(MID, 1000)            # > min(d_out, d_in): exercises the chunk loop
+    y = host(ctx.apply(st, dev(x)))
+    A, B, S = (host(t).astype(np.float64) for t in (st.A, st.B, st.S))
+    assert rel(y, O.apply(A, B, S, x)) < 1e-5

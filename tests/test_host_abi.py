@@ -1,0 +1,86 @@
+"""Host-side checks that need no GPU: the shared library loads, exports every symbol the header declares,
+and rejects bad arguments before touching the device."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2510_05528_b200 import binding as Bd
+from paper_2510_05528_b200 import build as armor_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    armor_build.build()
+    return Bd.lib()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "armor.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(armor_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_symbols()
+    assert {"armor_gram", "armor_init", "armor_bcd_step", "armor_proxy_loss", "armor_apply"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(names) == set(Bd.EXPORTS)
+
+
+def test_config_validation(lib):
+    ok = Bd.make_config(256, 256, 32)
+    assert Bd.armor_workspace_bytes(ok) > 0
+    cases = [
+        (Bd.make_config(256, 250, 32), 2),             # d_block does not divide d_in
+        (Bd.make_config(256, 256, 30), 2),             # ... nor d_out; not a multiple of m_group either
+        (Bd.make_config(256, 256, 32, n_keep=4, m_group=8), 7),
+        (Bd.make_config(512, 512, 256), 7),            # d_block > 128
+        (Bd.make_config(256, 256, 32, h_mode=5), 1),
+        (Bd.make_config(256, 256, 32, ridge=-1.0), 1),
+        (Bd.make_config(0, 256, 32), 2),
+        (Bd.make_config(192, 192, 32, precision=Bd.PREC_TF32), 7),   # tensor-core tiles need multiples of 128
+        (Bd.make_config(256, 256, 32, s_step=Bd.S_BETA), 7),
+    ]
+    for cfg, code in cases:
+        n = C.c_size_t(0)
+        assert lib.armor_workspace_bytes(C.byref(cfg), C.byref(n)) == code
+    assert lib.armor_workspace_bytes(None, C.byref(C.c_size_t(0))) == 1
+    assert lib.armor_workspace_bytes(C.byref(ok), None) == 1
+
+
+def test_create_rejects_bad_workspace(lib):
+    cfg = Bd.make_config(256, 256, 32)
+    ctx = C.c_void_p(0)
+    assert lib.armor_create(C.byref(ctx), C.byref(cfg), None, 1 << 30) == 1
+    assert lib.armor_create(C.byref(ctx), C.byref(cfg), C.c_void_p(0x1000 + 8), 1 << 30) == 3   # misaligned
+    assert lib.armor_create(C.byref(ctx), C.byref(cfg), C.c_void_p(0x1000), 16) == 3           # too small
+    assert lib.armor_create(None, C.byref(cfg), C.c_void_p(0x1000), 1 << 30) == 1
+    assert ctx.value is None
+
+
+def test_null_context_is_rejected(lib):
+    assert lib.armor_destroy(None) == 1
+    assert lib.armor_gram(None, None, 0, 0, 0, None, None) == 1
+    assert lib.armor_bcd_step(None, None, None, None, None, None, None, 0, 1, None, None) == 1
+    assert lib.armor_proxy_loss(None, None, None, None, None, None, None, None) == 1
+    assert lib.armor_apply(None, None, None, None, None, None, None, None, None, 0, 0, None) == 1
+    assert lib.armor_launch_count(None) == -1
+
+
+def test_status_strings(lib):
+    seen = {Bd.status_string(i) for i in range(8)}
+    assert len(seen) == 8 and "ok" in seen
+    assert "unknown" in Bd.status_string(99)
+
+
+def test_binding_refuses_cpu_tensors(lib):
+    import torch
+    with pytest.raises(ValueError):
+        Bd._ptr(torch.zeros(4), torch.float32, "x")
+    with pytest.raises(ValueError):
+        Bd.ArmorContext(256, 256, 32, device="cpu")
