@@ -1,0 +1,372 @@
+#!/usr/bin/env python
+"""Benchmark of the ARMOR per-layer optimisation on B200.
+
+One "step" is one pass of the whole hot path over one synthetic layer: calibration Gram of all tokens,
+initialisation, n_iters BCD iterations, proxy loss, and the factorised forward y = A S B x on a token batch.
+Default workload: the Llama-7B-shaped attention projection (4096 x 4096, d_block 128, 262,144 calibration
+tokens, 50 iterations).  Prints ONE JSON line (rank 0).
+
+  python bench.py --gpus 1 --steps 3 --warmup 3
+  python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N     (N independent replicas)
+  python bench.py --impl reference      (the CPU oracle, timed on a bounded sample of the same workload)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2510_05528_b200 import inputs  # noqa: E402
+
+METRIC = "bcd_iterations_per_s"
+UNIT = "iterations/s"
+APPLY_TOKENS = 8192
+# nominal dense tensor ratio tf32 : bf16 (1.1 : 2.25 PFLOP/s) applied to the measured bf16 peak
+TF32_OVER_BF16 = 1.1 / 2.25
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM bytes (read + write) of one dense 4096^3 launch of the tensor-core GEMM in FP32X3 mode, from the ncu
+# capture summarised in profiles/ (None until a capture exists for the current kernel)
+GEMM_DRAM_TRAFFIC_BYTES = None
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.samples, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for s in self.samples:
+            f = [x.strip() for x in s.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+# ------------------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample(cfg, gram_tokens=8192):
+    """Times the oracle, as it stands, on a bounded sample: the Gram of `gram_tokens` tokens and ONE full BCD
+    iteration at the layer's full size, and extrapolates the whole layer linearly."""
+    from oracle import armor_oracle as O
+    W = inputs.make_weight(cfg).astype(np.float64)
+    scales = torch.from_numpy(inputs.channel_scales(cfg))
+    nchunk = max(1, min(inputs.n_chunks(cfg), (gram_tokens + cfg.chunk_rows - 1) // cfg.chunk_rows))
+    X = np.concatenate([inputs.activation_chunk(cfg, i, scales).numpy() for i in range(nchunk)])[:gram_tokens]
+    t0 = time.perf_counter()
+    H = O.gram(X)
+    t_gram = time.perf_counter() - t0
+    H *= cfg.n_tokens / X.shape[0]
+    oc = O.OracleConfig(cfg.d_block, seed=cfg.seed)
+    t0 = time.perf_counter()
+    A, B, S, M = O.init(W, H, oc)
+    t_init = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    O.bcd_iteration(W, A, B, S, M, H, oc, 0, want_loss=False)
+    t_iter = time.perf_counter() - t0
+    t_layer = t_gram * cfg.n_tokens / X.shape[0] + t_init + cfg.n_iters * t_iter
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count()])
+    except Exception:
+        cores = os.cpu_count()
+    return {"value": cfg.n_iters / t_layer, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+            "sample": f"Gram of {X.shape[0]} of {cfg.n_tokens} tokens ({t_gram:.2f} s) + init ({t_init:.2f} s) + 1 of "
+                      f"{cfg.n_iters} BCD iterations at full {cfg.d_out}x{cfg.d_in} ({t_iter:.2f} s), extrapolated linearly",
+            "sec_per_layer_extrapolated": t_layer, "sec_per_iteration": t_iter}
+
+
+def run_reference(args, cfg):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    vals = []
+    last = None
+    for i in range(args.warmup + args.steps):
+        last = oracle_sample(cfg, gram_tokens=4096)
+        if i >= args.warmup:
+            vals.append(last)
+    t_layer = float(np.mean([v["sec_per_layer_extrapolated"] for v in vals]))
+    value = cfg.n_iters / t_layer
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_layer * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(cfg, "oracle"),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["cores"], "kind": "oracle", "sample": last["sample"]},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(cfg, precision):
+    return {"workload": f"{cfg.name}: W {cfg.d_out}x{cfg.d_in} fp32, d_block {cfg.d_block}, 2:4, {cfg.n_tokens} calibration "
+                        f"tokens, {cfg.n_iters} BCD iterations, h_mode FULL, apply on {APPLY_TOKENS} tokens",
+            "precision": precision, "l2": "inputs larger than L2 (X is %.2f GB, streamed every step)" % (cfg.n_tokens * cfg.d_in * 4 / 1e9),
+            "step": "gram + init + bcd iterations + proxy loss + apply"}
+
+
+# ------------------------------------------------------------------------------------- GPU arm
+def run_ours(args, cfg):
+    from paper_2510_05528_b200 import binding as Bd
+    from paper_2510_05528_b200 import build as armor_build
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    armor_build.build()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    use_dist = world > 1
+    if use_dist:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    prec = {"fp32x3": Bd.PREC_FP32X3, "tf32": Bd.PREC_TF32}[args.precision]
+    lcfg = cfg.with_(seed=cfg.seed + 1000 * rank)          # every rank optimises its own layer
+    ctx = Bd.ArmorContext(lcfg.d_out, lcfg.d_in, lcfg.d_block, device=dev, precision=prec, seed=lcfg.seed)
+
+    # ---- synthetic inputs, generated on the host and staged in pinned memory
+    W_h = torch.from_numpy(inputs.make_weight(lcfg)).pin_memory()
+    X_h = torch.empty(lcfg.n_tokens, lcfg.d_in, dtype=torch.float32, pin_memory=True)
+    scales = torch.from_numpy(inputs.channel_scales(lcfg))
+    for i in range(inputs.n_chunks(lcfg)):
+        lo = i * lcfg.chunk_rows
+        inputs.activation_chunk(lcfg, i, scales, out=X_h[lo: lo + lcfg.chunk_rows])
+    xt_h = torch.from_numpy(inputs.make_tokens(lcfg, APPLY_TOKENS)).pin_memory()
+    X_d, W_d, xt_d = X_h.to(dev), W_h.to(dev), xt_h.to(dev)
+    H = ctx.new_gram()
+    loss_h = torch.zeros(1, dtype=torch.float64).pin_memory()
+
+    def step_resident():
+        H.zero_()
+        ctx.gram(X_d, H)
+        st = ctx.init(W_d, H)
+        ctx.bcd_step(st, H, 0, lcfg.n_iters, want_stats=False)
+        loss = ctx.proxy_loss(st, H)
+        y = ctx.apply(st, xt_d)
+        return st, loss, y
+
+    e2e_chunk = 32768
+    xbuf = [torch.empty(e2e_chunk, lcfg.d_in, dtype=torch.float32, device=dev) for _ in range(2)]
+    copy_stream = torch.cuda.Stream(device=dev)
+    out_h = {"A": torch.empty(lcfg.d_out // lcfg.d_block, lcfg.d_block, lcfg.d_block).pin_memory(),
+             "B": torch.empty(lcfg.d_in // lcfg.d_block, lcfg.d_block, lcfg.d_block).pin_memory(),
+             "S": torch.empty(lcfg.d_out, lcfg.d_in).pin_memory(),
+             "M": torch.empty(lcfg.d_out, lcfg.d_in // 4, dtype=torch.uint8).pin_memory(),
+             "y": torch.empty(APPLY_TOKENS, lcfg.d_out).pin_memory()}
+    h2d = X_h.numel() * 4 + W_h.numel() * 4 + xt_h.numel() * 4
+    d2h = sum(t.numel() * t.element_size() for t in out_h.values()) + 8
+
+    def step_e2e():
+        """Host buffers in, host buffers out: every copy is inside the timed region.  The token chunks are
+        double-buffered so that the next host->device copy overlaps the Gram of the current chunk."""
+        main = torch.cuda.current_stream()
+        H.zero_()
+        Wd = W_h.to(dev, non_blocking=True)
+        n = lcfg.n_tokens
+        evs = [None, None]
+        for k, lo in enumerate(range(0, n, e2e_chunk)):
+            b = k & 1
+            rows = min(e2e_chunk, n - lo)
+            with torch.cuda.stream(copy_stream):
+                if evs[b] is not None:
+                    copy_stream.wait_event(evs[b])          # the Gram that read this buffer has finished
+                xbuf[b][:rows].copy_(X_h[lo: lo + rows], non_blocking=True)
+                ready = torch.cuda.Event()
+                ready.record(copy_stream)
+            main.wait_event(ready)
+            ctx.gram(xbuf[b][:rows], H)
+            evs[b] = torch.cuda.Event()
+            evs[b].record(main)
+        st = ctx.init(Wd, H)
+        ctx.bcd_step(st, H, 0, lcfg.n_iters, want_stats=False)
+        loss = ctx.proxy_loss(st, H)
+        y = ctx.apply(st, xt_h.to(dev, non_blocking=True))
+        out_h["A"].copy_(st.A, non_blocking=True); out_h["B"].copy_(st.B, non_blocking=True)
+        out_h["S"].copy_(st.S, non_blocking=True); out_h["M"].copy_(st.M, non_blocking=True)
+        out_h["y"].copy_(y, non_blocking=True); loss_h.copy_(loss, non_blocking=True)
+        return st
+
+    def barrier():
+        if use_dist:
+            import torch.distributed as dist
+            dist.barrier(device_ids=[local_rank])
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if use_dist:
+            import torch.distributed as dist
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for _ in range(args.warmup):
+        step_resident()
+    torch.cuda.synchronize()
+
+    # ---- timed region (device-resident inputs)
+    Bd.armor_gemm_timing_enable(ctx.ctx, True)
+    Bd.armor_gemm_timing(ctx.ctx)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    l0 = ctx.launch_count()
+    ms_total = timed(step_resident, args.steps)
+    launches = ctx.launch_count() - l0
+    clocks = sampler.stop() if rank == 0 else None
+    n_gemm, gemm_ms, gemm_flops = Bd.armor_gemm_timing(ctx.ctx)
+    Bd.armor_gemm_timing_enable(ctx.ctx, False)
+    status = ctx.device_status()
+
+    # ---- per-phase breakdown (one extra step, not part of the headline)
+    def t_phase(fn):
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); r = fn(); b.record(); torch.cuda.synchronize()
+        return a.elapsed_time(b), r
+    H.zero_()
+    ms_gram, _ = t_phase(lambda: ctx.gram(X_d, H))
+    ms_init, st = t_phase(lambda: ctx.init(W_d, H))
+    ms_bcd, stats = t_phase(lambda: ctx.bcd_step(st, H, 0, lcfg.n_iters))
+    ms_loss, loss = t_phase(lambda: ctx.proxy_loss(st, H))
+    ms_apply, _ = t_phase(lambda: ctx.apply(st, xt_d))
+    srec = ctx.read_stats(stats)
+
+    # ---- end to end (host buffers)
+    for _ in range(min(args.warmup, 2)):
+        step_e2e()
+    ms_e2e = timed(step_e2e, args.steps)
+    del X_d
+
+    if rank != 0:
+        if use_dist:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return
+    peaks, peak_kind = load_peaks()
+    ms_step = ms_total / args.steps
+    value = world * lcfg.n_iters / (ms_step / 1e3)
+    e2e_value = world * lcfg.n_iters / (ms_e2e / args.steps / 1e3)
+    tf32_peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * TF32_OVER_BF16
+    achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic", "config": workload_config(lcfg, args.precision),
+        "sec_per_layer": ms_step / 1e3,
+        "bcd_only_iterations_per_s": lcfg.n_iters / (ms_bcd / 1e3),
+        "phases_ms": {"gram": ms_gram, "init": ms_init, "bcd": ms_bcd, "bcd_per_iteration": ms_bcd / lcfg.n_iters,
+                      "proxy_loss": ms_loss, "apply": ms_apply},
+        "loss": {"init": float(srec["loss_start"][0]), "final": float(loss.item()),
+                 "mask_steps_accepted": int(srec["mask_accepted"].sum()), "chol_failed": int(srec["chol_failed"].sum())},
+        "device_status": status[:4],
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                "ms_per_step": ms_e2e / args.steps},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": {"bound": "tensor", "kernel": "tc_gemm_kernel (tcgen05 tf32, Gram + dense .H contractions)",
+                     "achieved": achieved, "peak": tf32_peak, "unit": "TFLOP/s", "frac": achieved / tf32_peak,
+                     "traffic": GEMM_DRAM_TRAFFIC_BYTES,
+                     "note": f"achieved = algorithmic (single-pass) flops of {n_gemm} launches / their CUDA-event time "
+                             f"({gemm_ms:.1f} ms of {ms_total:.1f} ms); the {args.precision} mode issues "
+                             f"{3 if args.precision == 'fp32x3' else 1} tensor-core pass(es) per product; peak = {peak_kind} "
+                             f"sustained bf16 x nominal tf32/bf16 ratio",
+                     "tensor_pipe_rate": achieved * (3 if args.precision == "fp32x3" else 1),
+                     "share_of_step": gemm_ms / ms_total},
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = {k: v for k, v in oracle_sample(lcfg).items()
+                                if k in ("value", "unit", "cores", "kind", "sample")}
+    print(json.dumps(line), flush=True)
+    if use_dist:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="llama7b_attn", choices=sorted(inputs.CONFIGS))
+    ap.add_argument("--precision", default="fp32x3", choices=["fp32x3", "tf32"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    cfg = inputs.CONFIGS[args.config]
+    _, _, world = dist_env()
+    if args.gpus > 1 and world == 1 and args.impl == "ours":
+        # not launched by torchrun: start one process per GPU ourselves
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", "29511", os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()
