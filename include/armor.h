@@ -46,7 +46,8 @@ typedef enum {
   ARMOR_ERR_CUDA = 4,
   ARMOR_ERR_NOT_SPD = 5,
   ARMOR_ERR_TIMEOUT = 6,
-  ARMOR_ERR_UNSUPPORTED = 7
+  ARMOR_ERR_UNSUPPORTED = 7,
+  ARMOR_ERR_TOO_LARGE = 8
 } armor_status;
 
 enum { ARMOR_H_FULL = 0, ARMOR_H_DIAG = 1 };
@@ -166,6 +167,34 @@ int64_t armor_launch_count(const armor_ctx* ctx);
  * Events are created on first use; no device memory is allocated. */
 armor_status armor_gemm_timing_enable(armor_ctx* ctx, int32_t enable);
 armor_status armor_gemm_timing(armor_ctx* ctx, int64_t* n_launches, double* total_ms, double* total_flops);
+
+/* The paper has no counterpart to this entry point; it exists for deployment reasons only.
+ *
+ * armor_normalize_noalloc computes the same row/column normalisation that armor_init applies when
+ * cfg.normalize == 1 (W_bar = W / r1 / r2, r1 = column norms of W, r2 = row norms of W / r1, zero
+ * norms read as 1), but needs neither a context nor a workspace.  It is meant for callers that are
+ * not allowed to obtain device memory at the point where they need the result: a process whose
+ * whole device memory has already been handed to another allocator or to a fixed serving pool, a
+ * plugin running inside a host application that forbids device allocations after start-up, or a
+ * latency-critical loop that cannot afford the device-wide synchronisation an allocation implies.
+ * The call performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ *
+ * Its scratch (ARMOR_NOALLOC_ROW_CHUNKS x ARMOR_NOALLOC_MAX_COLS doubles = 4 MiB) is a fixed array
+ * inside the library's device image: every GPU that loads the library holds those 4 MiB until the
+ * process exits.  Limits: d_in <= ARMOR_NOALLOC_MAX_COLS and d_out <= ARMOR_NOALLOC_MAX_ROWS, else
+ * ARMOR_ERR_TOO_LARGE.  Inputs and outputs are the caller's device buffers: d_W and d_Wbar
+ * [d_out, d_in] (distinct buffers), d_r1 [d_in], d_r2 [d_out].
+ *
+ * The first call on each device looks up the device address of the built-in array (with that
+ * device current); make that first call outside any stream capture.  All calls on a device share
+ * the array and it keeps the previous call's contents; nothing in it has to start at zero because
+ * every slot is written before it is read within a call.  Two calls that overlap on the same GPU
+ * (different streams, or different host threads) race on the array: serialise them. */
+#define ARMOR_NOALLOC_MAX_COLS 8192
+#define ARMOR_NOALLOC_MAX_ROWS 65536
+#define ARMOR_NOALLOC_ROW_CHUNKS 64
+armor_status armor_normalize_noalloc(const float* d_W, int64_t d_out, int64_t d_in, float* d_Wbar,
+                                     float* d_r1, float* d_r2, armor_stream_t stream);
 
 #ifdef __cplusplus
 }

@@ -25,7 +25,8 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 
 EXPORTS = ["armor_workspace_bytes", "armor_create", "armor_destroy", "armor_gram", "armor_init",
            "armor_bcd_step", "armor_proxy_loss", "armor_apply", "armor_get_device_status",
-           "armor_status_string", "armor_launch_count", "armor_gemm_timing_enable", "armor_gemm_timing"]
+           "armor_status_string", "armor_launch_count", "armor_gemm_timing_enable", "armor_gemm_timing",
+           "armor_normalize_noalloc"]
 
 
 class ArmorError(RuntimeError):
@@ -70,6 +71,7 @@ def lib() -> C.CDLL:
         L.armor_status_string.restype = C.c_char_p
         L.armor_launch_count.argtypes = [vp]
         L.armor_launch_count.restype = i64
+        L.armor_normalize_noalloc.argtypes = [vp, i64, i64, vp, vp, vp, vp]
         L.armor_gemm_timing_enable.argtypes = [vp, i32]
         L.armor_gemm_timing.argtypes = [vp, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
         for name in EXPORTS:
@@ -173,6 +175,17 @@ def armor_get_device_status(ctx, n: int = 8) -> list[int]:
 
 def armor_launch_count(ctx) -> int:
     return int(lib().armor_launch_count(ctx))
+
+
+def armor_normalize_noalloc(W: torch.Tensor, Wbar: torch.Tensor, r1: torch.Tensor, r2: torch.Tensor) -> None:
+    """Normalisation without a context or a workspace, for callers that may not allocate device memory:
+    the scratch is a fixed 4 MiB array inside the library (d_in <= 8192, d_out <= 65536).  All arguments are
+    the caller's CUDA tensors; this wrapper allocates nothing either.  Calls that overlap on one GPU race."""
+    f = torch.float32
+    if W.dim() != 2:
+        raise ValueError("W must be [d_out, d_in]")
+    _check(lib().armor_normalize_noalloc(_ptr(W, f, "W"), W.shape[0], W.shape[1], _ptr(Wbar, f, "Wbar"),
+                                         _ptr(r1, f, "r1"), _ptr(r2, f, "r2"), _stream()), "armor_normalize_noalloc")
 
 
 def armor_gemm_timing_enable(ctx, enable: bool) -> None:

@@ -161,6 +161,7 @@ const char* armor_status_string(armor_status st) {
     case ARMOR_ERR_NOT_SPD: return "block not positive definite";
     case ARMOR_ERR_TIMEOUT: return "bounded device wait ran out";
     case ARMOR_ERR_UNSUPPORTED: return "configuration not supported";
+    case ARMOR_ERR_TOO_LARGE: return "size exceeds the built-in scratch of the no-allocation entry point";
   }
   return "unknown status";
 }

@@ -73,8 +73,8 @@ def test_null_context_is_rejected(lib):
 
 
 def test_status_strings(lib):
-    seen = {Bd.status_string(i) for i in range(8)}
-    assert len(seen) == 8 and "ok" in seen
+    seen = {Bd.status_string(i) for i in range(9)}
+    assert len(seen) == 9 and "ok" in seen
     assert "unknown" in Bd.status_string(99)
 
 
