@@ -6,7 +6,8 @@
 // The tensor-core accumulator adds with truncation, so a long run of same-sign terms drifts by about
 // (K / 8) * passes * 2^-24.  The GEMM therefore drains its accumulator into C every K_SEGMENT columns of
 // the contraction (the additions into C are ordinary round-to-nearest fp32 adds).
-static const int64_t K_SEGMENT = 1024;
+static int64_t K_SEGMENT = 1024;
+extern "C" void armor_debug_set_k_segment(int64_t k) { K_SEGMENT = k; }
 
 armor_status prepare_H(armor_ctx* c, const float* H, cudaStream_t s) {
   launch_extract_hblocks(c, H, s);
@@ -40,7 +41,7 @@ armor_status rmul_H(armor_ctx* c, const float* in, const float* H, float* out, i
       g.A = in; g.B = H; g.passes = 1;
     }
     g.d1 = d1; g.d2 = d2;
-    g.k_segment = K_SEGMENT;
+    g.k_segment = (g.passes == 3) ? K_SEGMENT : 0;   // one-pass tf32 rounding (2^-11) dwarfs the accumulator drift
     g.part1 = d1 ? c->partials : nullptr;
     g.part2 = d2 ? c->partials + 4 * c->npart : nullptr;
     int tiles = 0;
@@ -85,7 +86,7 @@ armor_status gram_accumulate(armor_ctx* c, const float* X, int64_t n_rows, int64
     g.passes = x3 ? 3 : 1;
     g.accumulate = 1;
     g.symmetric_lower = 1;
-    g.k_segment = K_SEGMENT;
+    g.k_segment = x3 ? K_SEGMENT : 4 * K_SEGMENT;
     armor_status st = launch_tc_gemm(c, g, nullptr, s);
     if (st != ARMOR_OK) return st;
   }
@@ -114,6 +115,6 @@ armor_status apply_core(armor_ctx* c, const float* z1, const float* S, float* z2
   } else {
     g.A = z1; g.B = S; g.passes = 1;
   }
-  g.k_segment = K_SEGMENT;
+  g.k_segment = (g.passes == 3) ? K_SEGMENT : 0;
   return launch_tc_gemm(c, g, nullptr, s);
 }

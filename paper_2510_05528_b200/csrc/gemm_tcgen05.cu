@@ -281,47 +281,65 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         const bool last = kt0 + p.kt_seg >= kt_total;
         if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
         tc_fence_after();
+        // Each lane holds one row of a 32 x 32 chunk.  The chunk is turned through shared memory so that
+        // global memory sees whole 128-byte row segments (lanes = consecutive columns).
+        float* tilebuf = reinterpret_cast<float*>(smem + (size_t)STAGES * STAGE_BYTES) + q * (32 * 33);
+        const int64_t row_base = (int64_t)mt * BM + q * 32;
 #pragma unroll 1
         for (int ch = 0; ch < BN / 32; ++ch) {
           const int64_t col0 = (int64_t)nt * BN + ch * 32;
           uint32_t r[32];
           tmem_ld32(tmem_base + (uint32_t)(as * BN + ch * 32) + ((uint32_t)(q * 32) << 16), r);
-          if (col0 >= p.N || !row_ok) continue;
-          float* crow = p.C + row * p.ldc + col0;
-          if (!p.symmetric_lower) {
-            float f1 = 0.f, f2 = 0.f;
+          if (col0 >= p.N || row_base >= p.M) continue;                       // warp-uniform
+          if (p.symmetric_lower && col0 > row_base + 31) continue;           // chunk lies above the diagonal
 #pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-              float4 v = make_float4(__uint_as_float(r[i]), __uint_as_float(r[i + 1]), __uint_as_float(r[i + 2]),
-                                     __uint_as_float(r[i + 3]));
-              if (accum) {
-                const float4 o = *reinterpret_cast<const float4*>(crow + i);
-                v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-              }
-              if (last && p.d1) {
-                const float4 d = *reinterpret_cast<const float4*>(p.d1 + row * p.ldc + col0 + i);
-                f1 = fmaf(v.x, d.x, f1); f1 = fmaf(v.y, d.y, f1); f1 = fmaf(v.z, d.z, f1); f1 = fmaf(v.w, d.w, f1);
-              }
-              if (last && p.d2) {
-                const float4 d = *reinterpret_cast<const float4*>(p.d2 + row * p.ldc + col0 + i);
-                f2 = fmaf(v.x, d.x, f2); f2 = fmaf(v.y, d.y, f2); f2 = fmaf(v.z, d.z, f2); f2 = fmaf(v.w, d.w, f2);
-              }
-              *reinterpret_cast<float4*>(crow + i) = v;
+          for (int cidx = 0; cidx < 32; ++cidx) tilebuf[lane * 33 + cidx] = __uint_as_float(r[cidx]);
+          __syncwarp();
+          const int64_t col = col0 + lane;
+          float f1 = 0.f, f2 = 0.f;
+#pragma unroll 1
+          for (int r0 = 0; r0 < 32; r0 += 8) {
+            float x[8], o[8];
+            bool keep[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const int64_t grow = row_base + r0 + j;
+              keep[j] = grow < p.M && (!p.symmetric_lower || col <= grow);
+              x[j] = tilebuf[(r0 + j) * 33 + lane];
+              o[j] = (accum && keep[j]) ? p.C[grow * p.ldc + col] : 0.f;
             }
-            dot1 += (double)f1;
-            dot2 += (double)f2;
-          } else {
-            // lower triangle (+ diagonal) is owned by this tile; each kept element is mirrored once
+            if (last && p.d1) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const int64_t cc = col0 + i;
-              if (cc <= row) {
-                const float v = __uint_as_float(r[i]);
-                crow[i] = accum ? crow[i] + v : v;
-                if (cc < row) {
-                  float* mp = p.C + cc * p.ldc + row;
-                  *mp = accum ? *mp + v : v;
-                }
+              for (int j = 0; j < 8; ++j)
+                if (keep[j]) f1 = fmaf(x[j] + o[j], p.d1[(row_base + r0 + j) * p.ldc + col], f1);
+            }
+            if (last && p.d2) {
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                if (keep[j]) f2 = fmaf(x[j] + o[j], p.d2[(row_base + r0 + j) * p.ldc + col], f2);
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              if (keep[j]) p.C[(row_base + r0 + j) * p.ldc + col] = x[j] + o[j];
+          }
+          dot1 += (double)f1;
+          dot2 += (double)f2;
+          __syncwarp();
+          if (p.symmetric_lower && row_ok) {
+            // mirror of the strictly lower part, straight from the registers: for a fixed column the lanes
+            // hold consecutive rows, so C[col][row ..] is one contiguous segment
+#pragma unroll
+            for (int c0 = 0; c0 < 32; c0 += 8) {
+              float o[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const int64_t gcol = col0 + c0 + j;
+                o[j] = (accum && gcol < row) ? p.C[gcol * p.ldc + row] : 0.f;
+              }
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const int64_t gcol = col0 + c0 + j;
+                if (gcol < row) p.C[gcol * p.ldc + row] = __uint_as_float(r[c0 + j]) + o[j];
               }
             }
           }
@@ -392,7 +410,7 @@ armor_status launch_impl(armor_ctx* c, const TcGemm& g, const Params& p, cudaStr
   }
   constexpr int STAGE_BYTES = (PASSES == 3 ? 2 : 1) * (A_BYTES + B_BYTES);
   constexpr int STAGES = (PASSES == 3) ? 2 : 4;
-  constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024;
+  constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024 + 4 * 32 * 33 * sizeof(float);
   static bool attr = false;
   if (!attr) {
     if (cudaFuncSetAttribute(tc_gemm_kernel<PASSES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess)
