@@ -35,8 +35,8 @@ APPLY_TOKENS = 8192
 TF32_OVER_BF16 = 1.1 / 2.25
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes (read + write) of one dense 4096^3 launch of the tensor-core GEMM in FP32X3 mode, from the ncu
-# capture summarised in profiles/ (None until a capture exists for the current kernel)
-GEMM_DRAM_TRAFFIC_BYTES = None
+# capture summarised in profiles/ncu_tc_gemm_4096x4096x4096_fp32x3.md (read 768.3 MB + write 158.2 MB)
+GEMM_DRAM_TRAFFIC_BYTES = 926.5e6
 
 
 def load_peaks():
@@ -293,9 +293,12 @@ def run_ours(args, cfg):
     srec = ctx.read_stats(stats)
 
     # ---- end to end (host buffers)
-    for _ in range(min(args.warmup, 2)):
-        step_e2e()
-    ms_e2e = timed(step_e2e, args.steps)
+    if args.no_e2e:
+        ms_e2e = None
+    else:
+        for _ in range(min(args.warmup, 2)):
+            step_e2e()
+        ms_e2e = timed(step_e2e, args.steps)
     del X_d
 
     if rank != 0:
@@ -306,7 +309,7 @@ def run_ours(args, cfg):
     peaks, peak_kind = load_peaks()
     ms_step = ms_total / args.steps
     value = world * lcfg.n_iters / (ms_step / 1e3)
-    e2e_value = world * lcfg.n_iters / (ms_e2e / args.steps / 1e3)
+    e2e_value = world * lcfg.n_iters / (ms_e2e / args.steps / 1e3) if ms_e2e else None
     tf32_peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * TF32_OVER_BF16
     achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
     line = {
@@ -321,7 +324,7 @@ def run_ours(args, cfg):
                  "mask_steps_accepted": int(srec["mask_accepted"].sum()), "chol_failed": int(srec["chol_failed"].sum())},
         "device_status": status[:4],
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-                "ms_per_step": ms_e2e / args.steps},
+                "ms_per_step": ms_e2e / args.steps if ms_e2e else None},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": {"bound": "tensor", "kernel": "tc_gemm_kernel (tcgen05 tf32, Gram + dense .H contractions)",
@@ -352,10 +355,18 @@ def main():
     ap.add_argument("--config", default="llama7b_attn", choices=sorted(inputs.CONFIGS))
     ap.add_argument("--precision", default="fp32x3", choices=["fp32x3", "tf32"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tokens", type=int, default=0,
+                    help="profiling aid: calibration tokens instead of the workload's (the line then says 'reduced')")
+    ap.add_argument("--iters", type=int, default=0,
+                    help="profiling aid: BCD iterations per step instead of the workload's")
+    ap.add_argument("--no-e2e", action="store_true", help="profiling aid: skip the host-buffer leg")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     cfg = inputs.CONFIGS[args.config]
+    if args.tokens > 0 or args.iters > 0:
+        cfg = cfg.with_(name=cfg.name + " (reduced for profiling)", n_tokens=args.tokens or cfg.n_tokens,
+                        n_iters=args.iters or cfg.n_iters)
     _, _, world = dist_env()
     if args.gpus > 1 and world == 1 and args.impl == "ours":
         # not launched by torchrun: start one process per GPU ourselves
