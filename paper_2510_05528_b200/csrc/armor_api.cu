@@ -62,6 +62,7 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   TAKE(VH, float*, wbytes);
   TAKE(Gam, float*, wbytes);
   TAKE(Tmp, float*, wbytes);
+  TAKE(WH, float*, wbytes);
   if (x3) { TAKE(LoHi, float*, wbytes); TAKE(Lo, float*, wbytes); } else if (c) { c->LoHi = nullptr; c->Lo = nullptr; }
   if (x3) { TAKE(Hhi, float*, hbytes); TAKE(Hlo, float*, hbytes); } else if (c) { c->Hhi = nullptr; c->Hlo = nullptr; }
   const size_t ao = (size_t)nbo * db * db * sizeof(float), bo = (size_t)nbi * db * db * sizeof(float);
@@ -78,6 +79,9 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   TAKE(Bt, float*, bo);
   TAKE(alpha, float*, (size_t)cfg.d_out * sizeof(float));
   TAKE(hdiag, float*, (size_t)cfg.d_in * sizeof(float));
+  TAKE(Zsel, float*, (size_t)nbo * nbi * db * sizeof(float));
+  TAKE(Acol, float*, (size_t)nbo * nbi * db * sizeof(float));
+  TAKE(Ysel, float*, (size_t)nbo * nbi * cfg.d_in * sizeof(float));
   TAKE(colpart, double*, (size_t)64 * cfg.d_in * sizeof(double));
   if (tc) {
     TAKE(Xt_hi, float*, (size_t)cfg.d_in * GRAM_ROWS * sizeof(float));
@@ -289,18 +293,23 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
   const int ph = c->cfg.phases;
   armor_status st = prepare_H(c, H, s);
   if (st != ARMOR_OK) return st;
+  // W H_w is the same for every iteration of the call: E H_w = W H_w - A (T H_w)
+  st = rmul_H(c, W, H, c->WH, d_out, nullptr, nullptr, nullptr, nullptr, s);
+  if (st != ARMOR_OK) return st;
   for (int it = 0; it < n_iters; ++it) {
     armor_iter_stats* is = d_stats ? d_stats + it : nullptr;
     const int64_t t = t_first + it;
     launch_zero_scalars(c, s);
-    st = residual_and_loss(c, W, H, A, B, S, c->sc + SC_L0, s);
+    bd_right(c, S, B, false, c->T, d_out, d_in, 1.f, nullptr, 0.f, s);              // T = S B
+    st = rmul_H(c, c->T, H, c->P, d_out, nullptr, nullptr, nullptr, nullptr, s);     // P = T H_w
     if (st != ARMOR_OK) return st;
+    bd_left(c, A, false, c->P, c->EH, d_out, d_in, -1.f, c->WH, 1.f, s);             // E H_w = W H_w - A P
+    bd_left(c, A, false, c->T, c->E, d_out, d_in, -1.f, W, 1.f, s);                  // E = W - A T
+    dot_to_ptr(c, c->EH, c->E, c->wn, c->sc + SC_L0, s);                             // L = <E H_w, E>
     launch_stage(c, is, 0, nullptr, 0, 0, s);
 
     // ---- A-step: A_i += Gamma_i (G_i + lam I)^-1 -------------------------------------------
     if (ph & ARMOR_PHASE_A) {
-      st = rmul_H(c, c->T, H, c->P, d_out, nullptr, nullptr, nullptr, nullptr, s);   // P = T H_w
-      if (st != ARMOR_OK) return st;
       rowblock_gram(c, c->P, c->T, c->G, s);        // G_i = T_i H_w T_i^T
       rowblock_gram(c, c->EH, c->T, c->GamA, s);    // Gamma_i = E_i H_w T_i^T
       st = launch_chol(c, 0, c->G, c->GamA, c->dA, nullptr, A, c->At, nbo, c->partblk, s);
@@ -353,9 +362,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       block_mm(c, B, false, c->Hjj, false, c->Ktmp, nbi, s);                         // B_j H_jj
       block_mm(c, c->Ktmp, false, B, true, c->Kfull, nbi, s);                        // K_j = B_j H_jj B_j^T
       launch_mask_select(c, c->Gam, S, M, t, s);
-      launch_mask_build_v(c, A, B, c->V, s);
-      st = rmul_H(c, c->V, H, c->VH, d_out, c->V, c->sc + SC_Q_M, nullptr, nullptr, s);
-      if (st != ARMOR_OK) return st;
+      launch_mask_quadratic(c, A, B, H, s);
       launch_stage(c, is, 4, c->partblk, nbo * nbi, 0, s);
       launch_mask_commit(c, S, M, is, s);
     } else {

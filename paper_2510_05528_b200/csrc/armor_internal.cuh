@@ -52,12 +52,14 @@ struct armor_ctx {
   char* ws;
   size_t ws_bytes;
   // W-shaped fp32 scratch
-  float *T, *E, *EH, *P, *U, *V, *VH, *Gam, *Tmp;
+  float *T, *E, *EH, *P, *U, *V, *VH, *Gam, *Tmp, *WH;
   // low parts of the left operands / of H for the three-pass tensor-core mode
   float *LoHi, *Lo, *Hhi, *Hlo;
   // [nb, db, db] scratch
   float *G, *GamA, *dA, *At, *C, *GamB, *Delta, *Hjj, *Kfull, *Ktmp, *Bt;
   float *alpha, *hdiag;
+  // sparse-core update: per selected group z = delta^T B_j[rows of the group, :] and a = A_i[:, r]
+  float *Zsel, *Acol, *Ysel;  // [nbi][nbo][db], [nbo][nbi][db], [nbi][nbo][d_in]
   // Gram staging (transposed, split chunk of X)
   float *Xt_hi, *Xt_lo;
   int64_t gram_rows;  // rows of X staged per pass
@@ -157,7 +159,9 @@ armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float*
 void launch_alpha(armor_ctx* c, const float* A, cudaStream_t s);
 void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const uint8_t* M, int64_t t,
                         cudaStream_t s);
-void launch_mask_build_v(armor_ctx* c, const float* A, const float* B, float* V, cudaStream_t s);
+// exact loss change of the iteration's group updates without a dense product: fills sc[SC_Q_M] = tr(V H_w V^T)
+// for V = A dS B from the selection records
+void launch_mask_quadratic(armor_ctx* c, const float* A, const float* B, const float* H, cudaStream_t s);
 void launch_mask_commit(armor_ctx* c, float* S, uint8_t* M, armor_iter_stats* st, cudaStream_t s);
 
 // tensor-core GEMM (gemm_tcgen05.cu):  C[M][N] (+)= sum_k A[m][k] * B[n][k]  (both K-major, fp32 storage).

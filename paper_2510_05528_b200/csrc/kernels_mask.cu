@@ -154,35 +154,68 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
   sel[blk] = rec;
 }
 
-// V = A dS B for the iteration's group updates: block (i, j) of V is the rank-one matrix
-// A_i[:, r] (x) (delta^T B_j[rows of the group, :]).
-__global__ void __launch_bounds__(NT) mask_build_v_kernel(const float* __restrict__ A, const float* __restrict__ B,
-                                                          const SelRec* __restrict__ sel, float* __restrict__ V,
-                                                          int64_t d_in, int db, int nbi) {
+// The group updates of one iteration change the core by dS (one group per (i, j) block) and the
+// reconstruction by V = A dS B.  Block (i, j) of dS has a single non-zero row r, so
+//   tr(V H_w V^T) = sum_i sum_{j, j'} (a_ij . a_ij') * (z_ij H_w[j, j'] z_ij'^T)
+// with a_ij = A_i[:, r_ij] and z_ij = delta_ij^T B_j[rows of the group, :]: row-blocks decouple because A is
+// block diagonal.  mask_vectors_kernel gathers a and z, a batched product forms y_ij = z_ij H_w[j-th block
+// row, :], and mask_quad_kernel sums the pairs in a fixed order.
+__global__ void __launch_bounds__(NT) mask_vectors_kernel(const float* __restrict__ A, const float* __restrict__ B,
+                                                          const SelRec* __restrict__ sel, float* __restrict__ Zsel,
+                                                          float* __restrict__ Acol, int db, int nbo, int nbi, int mg) {
   const int blk = blockIdx.x;
   const int bi = blk / nbi, bj = blk % nbi;
-  __shared__ float av[128], bv[128];
   const SelRec rec = sel[blk];
-  if (threadIdx.x < db) {
-    float a = 0.f, bsum = 0.f;
+  for (int k = threadIdx.x; k < db; k += NT) {
+    float a = 0.f, z = 0.f;
     if (rec.valid) {
       const int rl = rec.row - bi * db;
-      const int lc = (rec.cgrp % (db / 4)) * 4;
-      a = A[(int64_t)bi * db * db + (int64_t)threadIdx.x * db + rl];
+      const int lc = (rec.cgrp % (db / mg)) * mg;
+      a = A[(int64_t)bi * db * db + (int64_t)k * db + rl];
       const float* Bj = B + (int64_t)bj * db * db;
-      for (int p = 0; p < 4; ++p)
-        bsum = fmaf(rec.new_val[p] - rec.old_val[p], Bj[(int64_t)(lc + p) * db + threadIdx.x], bsum);
+      for (int p = 0; p < mg; ++p) z = fmaf(rec.new_val[p] - rec.old_val[p], Bj[(int64_t)(lc + p) * db + k], z);
     }
-    av[threadIdx.x] = a;
-    bv[threadIdx.x] = bsum;
+    Acol[((int64_t)bi * nbi + bj) * db + k] = a;
+    Zsel[((int64_t)bj * nbo + bi) * db + k] = z;
   }
+}
+
+// One CTA per row-block i, one warp per (j, j') pair at a time.  Y == nullptr: diagonal weighting, only the
+// j == j' pairs contribute and y = z (.) hdiag.
+__global__ void __launch_bounds__(NT) mask_quad_kernel(const float* __restrict__ Zsel, const float* __restrict__ Acol,
+                                                       const float* __restrict__ Y, const float* __restrict__ hdiag,
+                                                       double* __restrict__ part, int64_t d_in, int db, int nbo,
+                                                       int nbi) {
+  const int bi = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = NT / 32;
+  double acc = 0.0;
+  const int npairs = Y ? nbi * nbi : nbi;
+  for (int pr = warp; pr < npairs; pr += nw) {
+    const int j = Y ? pr / nbi : pr, j2 = Y ? pr % nbi : pr;
+    const float* a1 = Acol + ((int64_t)bi * nbi + j) * db;
+    const float* a2 = Acol + ((int64_t)bi * nbi + j2) * db;
+    const float* z2 = Zsel + ((int64_t)j2 * nbo + bi) * db;
+    float w = 0.f, m = 0.f;
+    if (Y) {
+      const float* y = Y + ((int64_t)j * nbo + bi) * d_in + (int64_t)j2 * db;
+      for (int k = lane; k < db; k += 32) { w = fmaf(a1[k], a2[k], w); m = fmaf(y[k], z2[k], m); }
+    } else {
+      const float* h = hdiag + (int64_t)j * db;
+      for (int k = lane; k < db; k += 32) { w = fmaf(a1[k], a2[k], w); m = fmaf(z2[k] * h[k], z2[k], m); }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+      w += __shfl_xor_sync(0xffffffffu, w, o);
+      m += __shfl_xor_sync(0xffffffffu, m, o);
+    }
+    acc += (double)w * (double)m;
+  }
+  __shared__ double red[NT / 32];
+  if (lane == 0) red[warp] = acc;
   __syncthreads();
-  const int q = db / 4;
-  for (int e = threadIdx.x; e < db * q; e += NT) {
-    const int o = e / q, n4 = (e % q) * 4;
-    const float a = av[o];
-    float4 v = make_float4(a * bv[n4], a * bv[n4 + 1], a * bv[n4 + 2], a * bv[n4 + 3]);
-    *reinterpret_cast<float4*>(V + ((int64_t)bi * db + o) * d_in + (int64_t)bj * db + n4) = v;
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    for (int w2 = 0; w2 < nw; ++w2) t += red[w2];
+    part[bi] = t;
   }
 }
 
@@ -224,9 +257,25 @@ void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const ui
   c->launches++;
 }
 
-void launch_mask_build_v(armor_ctx* c, const float* A, const float* B, float* V, cudaStream_t s) {
-  mask_build_v_kernel<<<c->nbo * c->nbi, NT, 0, s>>>(A, B, c->sel, V, c->d_in, c->db, c->nbi);
+void launch_mask_quadratic(armor_ctx* c, const float* A, const float* B, const float* H, cudaStream_t s) {
+  const int db = c->db, nbo = c->nbo, nbi = c->nbi;
+  mask_vectors_kernel<<<nbo * nbi, NT, 0, s>>>(A, B, c->sel, c->Zsel, c->Acol, db, nbo, nbi, c->cfg.m_group);
   c->launches++;
+  const float* Y = nullptr;
+  if (c->cfg.h_mode == ARMOR_H_FULL) {
+    // y_ij = z_ij H[j-th block row, :], batched over j:  [nbo, db] x [db, d_in]
+    BGemm g{};
+    g.A = c->Zsel; g.sAb = (int64_t)nbo * db; g.sAm = db; g.sAk = 1;
+    g.B = H; g.sBb = (int64_t)db * c->d_in; g.sBk = c->d_in; g.sBn = 1;
+    g.C = c->Ysel; g.sCb = (int64_t)nbo * c->d_in; g.sCm = c->d_in; g.sCn = 1;
+    g.M = nbo; g.N = (int)c->d_in; g.K = db; g.batch = nbi; g.alpha = 1.f;
+    launch_bgemm(c, g, s);
+    Y = c->Ysel;
+  }
+  double* part = c->partials + 4 * c->npart;
+  mask_quad_kernel<<<nbo, NT, 0, s>>>(c->Zsel, c->Acol, Y, c->hdiag, part, c->d_in, db, nbo, nbi);
+  c->launches++;
+  reduce_partials_to(c, part, nbo, c->sc + SC_Q_M, s);
 }
 
 void launch_mask_commit(armor_ctx* c, float* S, uint8_t* M, armor_iter_stats* st, cudaStream_t s) {
