@@ -92,7 +92,7 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   TAKE(sc, double*, SC_COUNT * sizeof(double));
   TAKE(partials, double*, (size_t)8 * npart * sizeof(double));
   const int64_t nbmax = nbo > nbi ? nbo : nbi;
-  TAKE(partblk, double*, (size_t)(nbmax > nbo * nbi ? nbmax : nbo * nbi) * sizeof(double));
+  TAKE(partblk, double*, (size_t)(4 * nbmax > nbo * nbi ? 4 * nbmax : nbo * nbi) * sizeof(double));
   TAKE(failflag, int32_t*, (size_t)nbmax * sizeof(int32_t));
   TAKE(sel, SelRec*, (size_t)nbo * nbi * sizeof(SelRec));
   TAKE(status, int32_t*, ST_COUNT * sizeof(int32_t));
@@ -314,7 +314,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       rowblock_gram(c, c->EH, c->T, c->GamA, s);    // Gamma_i = E_i H_w T_i^T
       st = launch_chol(c, 0, c->G, c->GamA, c->dA, nullptr, A, c->At, nbo, c->partblk, s);
       if (st != ARMOR_OK) return st;
-      launch_stage(c, is, 1, c->partblk, nbo, nbo, s);
+      launch_stage(c, is, 1, c->partblk, nbo * chol_parts_per_block(db), nbo, s);
       bd_left(c, c->dA, false, c->P, c->EH, d_out, d_in, -1.f, c->EH, 1.f, s);       // EH -= dA P
     } else {
       launch_stage(c, is, 1, nullptr, 0, 0, s);
@@ -333,7 +333,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       bd_right(c, c->U, c->Delta, false, c->V, d_out, d_in, 1.f, nullptr, 0.f, s);   // V = U Delta
       st = rmul_H(c, c->V, H, c->VH, d_out, c->V, c->sc + SC_Q_B, nullptr, nullptr, s);
       if (st != ARMOR_OK) return st;
-      launch_stage(c, is, 2, c->partblk, nbi, nbi, s);
+      launch_stage(c, is, 2, c->partblk, nbi * chol_parts_per_block(db), nbi, s);
       launch_axpy_slot(c, B, c->Delta, (int64_t)nbi * db * db, SC_TAU_B, 1.f, s);    // B += tau Delta
       launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_B, -1.f, s);                   // EH -= tau V H_w
     } else {

@@ -152,6 +152,8 @@ void launch_transpose_split(armor_ctx* c, const float* X, int64_t ldx, int64_t r
 // mode 0: X = rhs (G + lam I)^-1, A += X, At = A^T, out = X, part[b] = exact decrease of block b
 // mode 1: out = (G + lam I)^-1 rhs
 // mode 2: out = rhs (G + lam I)^-1, part[b] = <dotw, out>
+// partial sums written per block by launch_chol (modes 0 and 2)
+int chol_parts_per_block(int db);
 armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float* rhs, float* out, const float* dotw,
                          float* A, float* At, int nb, double* part, cudaStream_t s);
 
