@@ -89,6 +89,14 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   } else if (c) { c->Xt_hi = nullptr; c->Xt_lo = nullptr; }
   const int64_t tiles = ((cfg.d_out + 127) / 128) * ((cfg.d_in + 127) / 128) + ((cfg.d_in + 127) / 128) * ((cfg.d_in + 127) / 128);
   const int64_t npart = tiles > ARMOR_DOT_BLOCKS ? tiles : ARMOR_DOT_BLOCKS;
+  {
+    const int64_t tiles = (int64_t)((db + 127) / 128) * ((db + 127) / 128);
+    const int64_t g1 = 2 * nbo * pick_ksplit(2 * nbo, tiles, cfg.d_in) * (int64_t)db * db;
+    const int64_t g2 = 2 * nbi * pick_ksplit(2 * nbi, tiles, cfg.d_out) * (int64_t)db * db;
+    const int64_t gp = g1 > g2 ? g1 : g2;
+    TAKE(gpart, float*, (size_t)gp * sizeof(float));
+    if (c) c->gpart_floats = gp;
+  }
   TAKE(sc, double*, SC_COUNT * sizeof(double));
   TAKE(partials, double*, (size_t)8 * npart * sizeof(double));
   const int64_t nbmax = nbo > nbi ? nbo : nbi;
@@ -106,25 +114,30 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
 
 inline cudaStream_t cs(armor_stream_t s) { return reinterpret_cast<cudaStream_t>(s); }
 
-// per-block Gram-type products over a long contraction
-void rowblock_gram(armor_ctx* c, const float* P, const float* T, float* G, cudaStream_t s) {
-  // G_i = P_i T_i^T  (contraction over d_in), batch over row-blocks i
+// per-block Gram-type products over a long contraction, two at a time (the second pair of operands is
+// addressed through the distance between workspace buffers)
+void rowblock_grams(armor_ctx* c, const float* P, const float* P2, const float* T, float* G, float* G2, cudaStream_t s) {
+  // G_i = P_i T_i^T, G2_i = P2_i T_i^T  (contraction over d_in), batch over row-blocks i
   const int db = c->db;
   BGemm g{};
   g.A = P; g.sAb = (int64_t)db * c->d_in; g.sAm = c->d_in; g.sAk = 1;
   g.B = T; g.sBb = (int64_t)db * c->d_in; g.sBk = 1; g.sBn = c->d_in;
   g.C = G; g.sCb = (int64_t)db * db; g.sCm = db; g.sCn = 1;
-  g.M = db; g.N = db; g.K = (int)c->d_in; g.batch = c->nbo; g.alpha = 1.f;
+  g.M = db; g.N = db; g.K = (int)c->d_in; g.batch = 2 * c->nbo; g.alpha = 1.f;
+  g.batch_inner = c->nbo; g.sAb2 = P2 - P; g.sBb2 = 0; g.sCb2 = G2 - G;
+  g.ksplit = pick_ksplit(g.batch, (int64_t)((db + 127) / 128) * ((db + 127) / 128), g.K);
   launch_bgemm(c, g, s);
 }
-void colblock_gram(armor_ctx* c, const float* U, const float* Y, float* Cm, cudaStream_t s) {
-  // C_j = U_j^T Y_j  (contraction over d_out), batch over column-blocks j
+void colblock_grams(armor_ctx* c, const float* U, const float* Y, const float* Y2, float* Cm, float* Cm2, cudaStream_t s) {
+  // C_j = U_j^T Y_j, C2_j = U_j^T Y2_j  (contraction over d_out), batch over column-blocks j
   const int db = c->db;
   BGemm g{};
   g.A = U; g.sAb = db; g.sAm = 1; g.sAk = c->d_in;
   g.B = Y; g.sBb = db; g.sBk = c->d_in; g.sBn = 1;
   g.C = Cm; g.sCb = (int64_t)db * db; g.sCm = db; g.sCn = 1;
-  g.M = db; g.N = db; g.K = (int)c->d_out; g.batch = c->nbi; g.alpha = 1.f;
+  g.M = db; g.N = db; g.K = (int)c->d_out; g.batch = 2 * c->nbi; g.alpha = 1.f;
+  g.batch_inner = c->nbi; g.sAb2 = 0; g.sBb2 = Y2 - Y; g.sCb2 = Cm2 - Cm;
+  g.ksplit = pick_ksplit(g.batch, (int64_t)((db + 127) / 128) * ((db + 127) / 128), g.K);
   launch_bgemm(c, g, s);
 }
 void block_mm(armor_ctx* c, const float* X, bool tX, const float* Y, bool tY, float* Z, int nb, cudaStream_t s) {
@@ -310,8 +323,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
 
     // ---- A-step: A_i += Gamma_i (G_i + lam I)^-1 -------------------------------------------
     if (ph & ARMOR_PHASE_A) {
-      rowblock_gram(c, c->P, c->T, c->G, s);        // G_i = T_i H_w T_i^T
-      rowblock_gram(c, c->EH, c->T, c->GamA, s);    // Gamma_i = E_i H_w T_i^T
+      rowblock_grams(c, c->P, c->EH, c->T, c->G, c->GamA, s);   // G_i = T_i H_w T_i^T, Gamma_i = E_i H_w T_i^T
       st = launch_chol(c, 0, c->G, c->GamA, c->dA, nullptr, A, c->At, nbo, c->partblk, s);
       if (st != ARMOR_OK) return st;
       launch_stage(c, is, 1, c->partblk, nbo * chol_parts_per_block(db), nbo, s);
@@ -324,8 +336,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
     if (ph & ARMOR_PHASE_B) {
       launch_zero_flags(c, s);
       bd_left(c, A, false, S, c->U, d_out, d_in, 1.f, nullptr, 0.f, s);              // U = A S
-      colblock_gram(c, c->U, c->U, c->C, s);        // C_j = U_j^T U_j
-      colblock_gram(c, c->U, c->EH, c->GamB, s);    // Gamma_j = U_j^T (E H_w)_j
+      colblock_grams(c, c->U, c->U, c->EH, c->C, c->GamB, s);   // C_j = U_j^T U_j, Gamma_j = U_j^T (E H_w)_j
       st = launch_chol(c, 1, c->C, c->GamB, c->Delta, nullptr, nullptr, nullptr, nbi, nullptr, s);
       if (st != ARMOR_OK) return st;
       st = launch_chol(c, 2, c->Hjj, c->Delta, c->Delta, c->GamB, nullptr, nullptr, nbi, c->partblk, s);

@@ -58,6 +58,8 @@ struct armor_ctx {
   // [nb, db, db] scratch
   float *G, *GamA, *dA, *At, *C, *GamB, *Delta, *Hjj, *Kfull, *Ktmp, *Bt;
   float *alpha, *hdiag;
+  float* gpart;          // partial products of split contractions
+  int64_t gpart_floats;
   // sparse-core update: per selected group z = delta^T B_j[rows of the group, :] and a = A_i[:, r]
   float *Zsel, *Acol, *Ysel;  // [nbi][nbo][db], [nbo][nbi][db], [nbi][nbo][d_in]
   // Gram staging (transposed, split chunk of X)
@@ -101,8 +103,22 @@ struct BGemm {
   const float* D; int64_t sDb, sDm, sDn;
   int M, N, K, batch;
   float alpha, beta;
+  // two-level batch: batch index b = bo * batch_inner + bi, operand offset bo * s?b2 + bi * s?b
+  // (batch_inner == 0: one level)
+  int batch_inner;
+  int64_t sAb2, sBb2, sCb2, sDb2;
+  // split of the contraction into ksplit equal chunks whose partial products are summed in a fixed order
+  // (needs c->gpart; only without D)
+  int ksplit;
 };
 void launch_bgemm(armor_ctx* c, const BGemm& g, cudaStream_t s);
+// number of chunks a long contraction is cut into so that batch * tiles * chunks fills the GPU about twice
+inline int pick_ksplit(int64_t batch, int64_t tiles, int64_t K) {
+  int64_t ks = (296 + batch * tiles - 1) / (batch * tiles);
+  if (ks > K / 256) ks = K / 256;
+  while (ks > 1 && K % (16 * ks)) --ks;
+  return ks < 1 ? 1 : (int)ks;
+}
 
 // block-diagonal products on row-major [rows, cols] matrices
 //  right: out[:, jblk] = alpha * in[:, jblk] * Bblk[j] (+ beta * add[:, jblk]); transB uses Bblk[j]^T
