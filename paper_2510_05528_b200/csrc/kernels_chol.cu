@@ -1,6 +1,6 @@
 // Per-block SPD solves for the wrapper updates.  The block systems are the zeros of the paper's
 // gradients with respect to A and B (Appendix D.1 and D.2) made proximal by a relative ridge:
-//   mode 0 (A update): X = Gamma (G + lam I)^-1;  A += X;  At = A^T;  dA = X;  part = <Gamma, X> + lam |X|^2
+//   mode 0 (A update): X = Gamma (G + lam I)^-1;  A += X;  dA = X;  part = <Gamma, X> + lam |X|^2
 //   mode 1 (left)    : out = (G + lam I)^-1 rhs
 //   mode 2 (right+gd): out = rhs (G + lam I)^-1;  part = <dotw, out>
 // A failed factorisation leaves A unchanged / writes zeros and raises failflag[block].
@@ -38,6 +38,11 @@ __host__ __device__ inline size_t panel_floats(int db) {
   return (size_t)LDP * ((size_t)np * db - (size_t)NB * np * (np - 1) / 2);
 }
 
+// y -= sum over the 32 columns of one earlier panel, fp32 products; the caller adds the chunk to an fp64 sum
+#define ARMOR_TILE_ZERO(acc)                                   \
+  _Pragma("unroll") for (int a_ = 0; a_ < 4; ++a_)             \
+  _Pragma("unroll") for (int b_ = 0; b_ < 4; ++b_) acc[a_][b_] = 0.f;
+
 __global__ void __launch_bounds__(NT, 1)
 chol_blocked_kernel(int mode, const float* __restrict__ Gmat, const float* __restrict__ rhs, float* __restrict__ out,
                     const float* __restrict__ dotw, float* __restrict__ A, float* __restrict__ At, float ridge, int db,
@@ -48,31 +53,71 @@ chol_blocked_kernel(int mode, const float* __restrict__ Gmat, const float* __res
   const int ldr = w + 1;
   float* Lp = smem;
   float* Rs = smem + panel_floats(db);                  // [db][w + 1]: row = unknown index, column = right-hand side
-  double* invd = reinterpret_cast<double*>(smem + ((panel_floats(db) + (size_t)db * ldr + 1) & ~(size_t)1));  // [db]
+  __shared__ float Df[NB][NB + 1];                      // diagonal block of the current panel
+  __shared__ float invd[NB];                            // reciprocals of its diagonal
   __shared__ double red[NT / 32];
-  __shared__ float s_diag;
   __shared__ int s_fail;
   __shared__ double s_lam;
-  const int b = blockIdx.x, q = blockIdx.y, tid = threadIdx.x;
+  const int b = blockIdx.x, q = blockIdx.y, tid = threadIdx.x, lane = threadIdx.x & 31;
   const int64_t off = (int64_t)b * db * db;
   const bool right = (mode != 1);
   const int v0 = q * w;  // first right-hand side of this CTA
 
-  // ---- load: lower triangle of G, the slice of right-hand sides
-  for (int e = tid; e < db * db; e += NT) {
-    const int r = e / db, cidx = e % db;
-    if (cidx <= r) Lp[pm.at(r, cidx)] = Gmat[off + e];
-  }
-  if (right) {
-    // right-hand side v is row v0 + v of rhs; unknown index r runs along the row
-    for (int e = tid; e < w * db; e += NT) {
-      const int v = e / db, r = e % db;
-      Rs[r * ldr + v] = rhs[off + (int64_t)(v0 + v) * db + r];
+  // ---- load: lower triangle of G, the slice of right-hand sides.  float4 loads, eight in flight per
+  // thread, so that the global-memory latency is paid a few times and not once per element.
+  {
+    const int q4 = db / 4;                      // float4 per row
+    const int n4 = db * q4;
+    for (int e0 = tid; e0 < n4; e0 += 8 * NT) {
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int e = e0 + u * NT;
+        v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (e < n4 && (e % q4) * 4 <= e / q4) v[u] = reinterpret_cast<const float4*>(Gmat + off)[e];
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int e = e0 + u * NT;
+        if (e >= n4) continue;
+        const int r = e / q4, c4 = (e % q4) * 4;
+        if (c4 > r) continue;
+        float* dst = Lp + pm.at(r, c4);         // c4 .. c4 + 3 lie in one panel
+        const float vv[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (c4 + j <= r) dst[j] = vv[j];
+      }
     }
-  } else {
-    for (int e = tid; e < db * w; e += NT) {
-      const int r = e / w, v = e % w;
-      Rs[r * ldr + v] = rhs[off + (int64_t)r * db + v0 + v];
+    // right-hand sides: vector id x unknown index
+    const int m4 = right ? w * q4 : db * (w / 4);
+    for (int e0 = tid; e0 < m4; e0 += 8 * NT) {
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int e = e0 + u * NT;
+        v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (e < m4) {
+          if (right) v[u] = *reinterpret_cast<const float4*>(rhs + off + (int64_t)(v0 + e / q4) * db + (e % q4) * 4);
+          else v[u] = *reinterpret_cast<const float4*>(rhs + off + (int64_t)(e / (w / 4)) * db + v0 + (e % (w / 4)) * 4);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int e = e0 + u * NT;
+        if (e >= m4) continue;
+        const float vv[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+        if (right) {
+          // right-hand side vid is row v0 + vid of rhs; the unknown index runs along the row
+          const int vid = e / q4, r4 = (e % q4) * 4;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) Rs[(r4 + j) * ldr + vid] = vv[j];
+        } else {
+          const int r = e / (w / 4), vid4 = (e % (w / 4)) * 4;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) Rs[r * ldr + vid4 + j] = vv[j];
+        }
+      }
     }
   }
   if (tid == 0) s_fail = 0;
@@ -91,6 +136,7 @@ chol_blocked_kernel(int mode, const float* __restrict__ Gmat, const float* __res
   // ---- blocked Cholesky
   for (int kb = 0; kb < np; ++kb) {
     const int c0 = NB * kb;
+    float* P = Lp + pm.off(kb);
     if (kb > 0) {
       // panel(i, k) -= sum_{p < c0} L(i, p) L(k, p): 4 x 4 tiles, rows c0 + 4*tr.., columns c0 + 4*tc..
       const int ntiles = ((db - c0) / 4) * (NB / 4);
@@ -104,18 +150,24 @@ chol_blocked_kernel(int mode, const float* __restrict__ Gmat, const float* __res
         for (int pb = 0; pb < kb; ++pb) {
           const float* Li = Lp + pm.off(pb) + (c0 + 4 * tr - NB * pb) * LDP;   // rows i of panel pb
           const float* Lk = Lp + pm.off(pb) + (c0 + 4 * tc - NB * pb) * LDP;   // rows k of panel pb
-#pragma unroll 4
+          float a32[4][4];
+          ARMOR_TILE_ZERO(a32)
+#pragma unroll 8
           for (int p = 0; p < NB; ++p) {
-            double li[4], lk[4];
+            float li[4], lk[4];
 #pragma unroll
-            for (int a = 0; a < 4; ++a) { li[a] = (double)Li[a * LDP + p]; lk[a] = (double)Lk[a * LDP + p]; }
+            for (int a = 0; a < 4; ++a) { li[a] = Li[a * LDP + p]; lk[a] = Lk[a * LDP + p]; }
 #pragma unroll
             for (int a = 0; a < 4; ++a)
 #pragma unroll
-              for (int bb = 0; bb < 4; ++bb) acc[a][bb] = fma(li[a], lk[bb], acc[a][bb]);
+              for (int bb = 0; bb < 4; ++bb) a32[a][bb] = fmaf(li[a], lk[bb], a32[a][bb]);
           }
+#pragma unroll
+          for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int bb = 0; bb < 4; ++bb) acc[a][bb] += (double)a32[a][bb];
         }
-        float* dst = Lp + pm.off(kb) + (4 * tr) * LDP + 4 * tc;
+        float* dst = P + (4 * tr) * LDP + 4 * tc;
 #pragma unroll
         for (int a = 0; a < 4; ++a)
 #pragma unroll
@@ -123,160 +175,217 @@ chol_blocked_kernel(int mode, const float* __restrict__ Gmat, const float* __res
       }
       __syncthreads();
     }
-    // eliminate the 32 columns of the panel; thread i owns row c0 + i of the panel
-    float* P = Lp + pm.off(kb);
-    const int nrow = db - c0;
-    for (int k = 0; k < NB; ++k) {
-      double s = 0.0;
-      if (tid >= k && tid < nrow) {
-        s = (double)P[tid * LDP + k];
-        double s1 = 0.0;
-        int p = 0;
-        for (; p + 1 < k; p += 2) {
-          s = fma(-(double)P[tid * LDP + p], (double)P[k * LDP + p], s);
-          s1 = fma(-(double)P[tid * LDP + p + 1], (double)P[k * LDP + p + 1], s1);
+    // diagonal block: warp 0, lane i owns row i of the copy in shared memory and the warp eliminates column
+    // by column (right-looking), so that every dependent chain is one multiply-add long
+    if (tid < 32) {
+#pragma unroll 4
+      for (int j = 0; j < NB; ++j) Df[lane][j] = (j <= lane) ? P[lane * LDP + j] : 0.f;
+      __syncwarp();
+      bool bad = false;
+      for (int k = 0; k < NB; ++k) {
+        const float akk = Df[k][k];
+        bad |= !(akk > 0.f) | !isfinite(akk);
+        // 1 / sqrt(a): hardware estimate refined by one Newton step
+        float inv = rsqrtf(akk);
+        inv = inv * fmaf(-0.5f * akk * inv, inv, 1.5f);
+        const float lik = (lane == k) ? akk * inv : Df[lane][k] * inv;
+        __syncwarp();
+        if (lane >= k) Df[lane][k] = lik;
+        if (lane == k) invd[k] = inv;
+        __syncwarp();
+#pragma unroll 4
+        for (int j = k + 1; j < NB; ++j) {
+          const float ljk = Df[j][k];
+          if (lane >= j) Df[lane][j] = fmaf(-lik, ljk, Df[lane][j]);
         }
-        if (p < k) s = fma(-(double)P[tid * LDP + p], (double)P[k * LDP + p], s);
-        s += s1;
-        if (tid == k) {
-          if (!(s > 0.0) || !isfinite(s)) s_fail = 1; else s_diag = (float)sqrt(s);
-        }
+        __syncwarp();
       }
-      __syncthreads();
-      if (s_fail) break;
-      if (tid >= k && tid < nrow) P[tid * LDP + k] = (tid == k) ? s_diag : (float)(s / (double)s_diag);
-      __syncthreads();
+      if (bad) {
+        if (lane == 0) s_fail = 1;
+      } else {
+#pragma unroll 4
+        for (int j = 0; j <= lane; ++j) P[lane * LDP + j] = Df[lane][j];
+      }
     }
+    __syncthreads();
     if (s_fail) break;
+    // rows below the diagonal block: l_ik = (a_ik - sum_{p<k} l_ip l_kp) / l_kk, row i in registers
+    const int nrow = db - c0;
+    if (tid >= NB && tid < nrow) {   // nrow <= d_block <= 256 = NT
+      const int i = tid;
+      // column-oriented elimination: once l_ik is final it leaves the later entries of the row at once, so the
+      // dependent chain is one multiply-add per column
+      float arow[NB];
+#pragma unroll
+      for (int j = 0; j < NB; ++j) arow[j] = P[i * LDP + j];
+#pragma unroll
+      for (int k = 0; k < NB; ++k) {
+        const float lik = arow[k] * invd[k];
+        arow[k] = lik;
+#pragma unroll
+        for (int j = k + 1; j < NB; ++j) arow[j] = fmaf(-lik, Df[j][k], arow[j]);
+      }
+#pragma unroll
+      for (int j = 0; j < NB; ++j) P[i * LDP + j] = arow[j];
+    }
+    __syncthreads();
   }
   __syncthreads();
   const bool fail = (s_fail != 0);
 
   if (!fail) {
-    for (int i = tid; i < db; i += NT) invd[i] = 1.0 / (double)Lp[pm.at(i, i)];
-    __syncthreads();
     const int wq = w / 4;          // column c of tile column tc: tc + wq * j  (conflict-free shared-memory rows)
-    // ---- forward substitution  L y = r
-    for (int kb = 0; kb < np; ++kb) {
-      const int c0 = NB * kb;
-      if (kb > 0) {
-        const int ntiles = (NB / 4) * wq;
-        for (int tix = tid; tix < ntiles; tix += NT) {
-          const int ta = tix / wq, tc = tix % wq;
-          double acc[4][4];
-#pragma unroll
-          for (int a = 0; a < 4; ++a)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) acc[a][j] = 0.0;
-          for (int pb = 0; pb < kb; ++pb) {
-            const float* Li = Lp + pm.off(pb) + (c0 + 4 * ta - NB * pb) * LDP;
-            const float* Xp = Rs + (NB * pb) * ldr + tc;
-#pragma unroll 4
-            for (int p = 0; p < NB; ++p) {
-              double li[4], x[4];
-#pragma unroll
-              for (int a = 0; a < 4; ++a) { li[a] = (double)Li[a * LDP + p]; x[a] = (double)Xp[p * ldr + wq * a]; }
-#pragma unroll
-              for (int a = 0; a < 4; ++a)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) acc[a][j] = fma(li[a], x[j], acc[a][j]);
-            }
-          }
-          float* dst = Rs + (c0 + 4 * ta) * ldr + tc;
-#pragma unroll
-          for (int a = 0; a < 4; ++a)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) dst[a * ldr + wq * j] = (float)((double)dst[a * ldr + wq * j] - acc[a][j]);
+    // ---- forward substitution  L y = r, then backward substitution  L^T x = y
+    for (int pass = 0; pass < 2; ++pass) {
+      for (int step = 0; step < np; ++step) {
+        const int kb = pass == 0 ? step : np - 1 - step;
+        const int c0 = NB * kb;
+        const float* P = Lp + pm.off(kb);
+        // the diagonal block and the reciprocals of its diagonal
+        for (int e = tid; e < NB * NB; e += NT) {
+          const int r = e / NB, cc = e % NB;
+          const float v = (cc <= r) ? P[r * LDP + cc] : 0.f;
+          Df[r][cc] = v;
+          if (r == cc) invd[r] = 1.f / v;
         }
-        __syncthreads();
-      }
-      if (tid < w) {
-        const float* D = Lp + pm.off(kb);   // diagonal block: rows 0..31 of the panel
-        double sreg[NB];
-#pragma unroll
-        for (int r = 0; r < NB; ++r) sreg[r] = (double)Rs[(c0 + r) * ldr + tid];
-#pragma unroll
-        for (int r = 0; r < NB; ++r) {
-          const double x = sreg[r] * invd[c0 + r];
-          sreg[r] = x;
-#pragma unroll
-          for (int r2 = r + 1; r2 < NB; ++r2) sreg[r2] = fma(-(double)D[r2 * LDP + r], x, sreg[r2]);
-        }
-#pragma unroll
-        for (int r = 0; r < NB; ++r) Rs[(c0 + r) * ldr + tid] = (float)sreg[r];
-      }
-      __syncthreads();
-    }
-    // ---- backward substitution  L^T x = y
-    for (int kb = np - 1; kb >= 0; --kb) {
-      const int c0 = NB * kb;
-      if (kb < np - 1) {
-        const int ntiles = (NB / 4) * wq;
-        for (int tix = tid; tix < ntiles; tix += NT) {
-          const int ta = tix / wq, tc = tix % wq;
-          double acc[4][4];
-#pragma unroll
-          for (int a = 0; a < 4; ++a)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) acc[a][j] = 0.0;
-          // sum over p >= c0 + NB of L(p, c0 + 4 ta + a) x[p]: column c0 + 4 ta + a lives in panel kb
-          const float* Lcol = Lp + pm.off(kb) + 4 * ta;
-          const float* Xp = Rs + tc;
-#pragma unroll 4
-          for (int p = c0 + NB; p < db; ++p) {
-            double lc[4], x[4];
-#pragma unroll
-            for (int a = 0; a < 4; ++a) { lc[a] = (double)Lcol[(p - c0) * LDP + a]; x[a] = (double)Xp[p * ldr + wq * a]; }
+        if (step > 0) {
+          const int ntiles = (NB / 4) * wq;
+          for (int tix = tid; tix < ntiles; tix += NT) {
+            const int ta = tix / wq, tc = tix % wq;
+            double acc[4][4];
 #pragma unroll
             for (int a = 0; a < 4; ++a)
 #pragma unroll
-              for (int j = 0; j < 4; ++j) acc[a][j] = fma(lc[a], x[j], acc[a][j]);
+              for (int j = 0; j < 4; ++j) acc[a][j] = 0.0;
+            if (pass == 0) {
+              for (int pb = 0; pb < kb; ++pb) {
+                const float* Li = Lp + pm.off(pb) + (c0 + 4 * ta - NB * pb) * LDP;
+                const float* Xp = Rs + (NB * pb) * ldr + tc;
+                float a32[4][4];
+                ARMOR_TILE_ZERO(a32)
+#pragma unroll 8
+                for (int p = 0; p < NB; ++p) {
+                  float li[4], x[4];
+#pragma unroll
+                  for (int a = 0; a < 4; ++a) { li[a] = Li[a * LDP + p]; x[a] = Xp[p * ldr + wq * a]; }
+#pragma unroll
+                  for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) a32[a][j] = fmaf(li[a], x[j], a32[a][j]);
+                }
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) acc[a][j] += (double)a32[a][j];
+              }
+            } else {
+              // sum over p >= c0 + NB of L(p, c0 + 4 ta + a) x[p]: column c0 + 4 ta + a lives in panel kb
+              const float* Lcol = P + 4 * ta;
+              const float* Xp = Rs + tc;
+              for (int p0 = c0 + NB; p0 < db; p0 += NB) {
+                float a32[4][4];
+                ARMOR_TILE_ZERO(a32)
+#pragma unroll 8
+                for (int p = p0; p < p0 + NB; ++p) {
+                  float lc[4], x[4];
+#pragma unroll
+                  for (int a = 0; a < 4; ++a) { lc[a] = Lcol[(p - c0) * LDP + a]; x[a] = Xp[p * ldr + wq * a]; }
+#pragma unroll
+                  for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) a32[a][j] = fmaf(lc[a], x[j], a32[a][j]);
+                }
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) acc[a][j] += (double)a32[a][j];
+              }
+            }
+            float* dst = Rs + (c0 + 4 * ta) * ldr + tc;
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+              for (int j = 0; j < 4; ++j) dst[a * ldr + wq * j] = (float)((double)dst[a * ldr + wq * j] - acc[a][j]);
           }
-          float* dst = Rs + (c0 + 4 * ta) * ldr + tc;
+        }
+        __syncthreads();
+        if (tid < w) {
+          float sreg[NB];
 #pragma unroll
-          for (int a = 0; a < 4; ++a)
+          for (int r = 0; r < NB; ++r) sreg[r] = Rs[(c0 + r) * ldr + tid];
+          if (pass == 0) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) dst[a * ldr + wq * j] = (float)((double)dst[a * ldr + wq * j] - acc[a][j]);
+            for (int r = 0; r < NB; ++r) {
+              const float x = sreg[r] * invd[r];
+              sreg[r] = x;
+#pragma unroll
+              for (int r2 = r + 1; r2 < NB; ++r2) sreg[r2] = fmaf(-Df[r2][r], x, sreg[r2]);
+            }
+          } else {
+#pragma unroll
+            for (int r = NB - 1; r >= 0; --r) {
+              const float x = sreg[r] * invd[r];
+              sreg[r] = x;
+#pragma unroll
+              for (int r2 = 0; r2 < r; ++r2) sreg[r2] = fmaf(-Df[r][r2], x, sreg[r2]);
+            }
+          }
+#pragma unroll
+          for (int r = 0; r < NB; ++r) Rs[(c0 + r) * ldr + tid] = sreg[r];
         }
         __syncthreads();
       }
-      if (tid < w) {
-        const float* D = Lp + pm.off(kb);
-        double sreg[NB];
-#pragma unroll
-        for (int r = 0; r < NB; ++r) sreg[r] = (double)Rs[(c0 + r) * ldr + tid];
-#pragma unroll
-        for (int r = NB - 1; r >= 0; --r) {
-          const double x = sreg[r] * invd[c0 + r];
-          sreg[r] = x;
-#pragma unroll
-          for (int r2 = 0; r2 < r; ++r2) sreg[r2] = fma(-(double)D[r * LDP + r2], x, sreg[r2]);
-        }
-#pragma unroll
-        for (int r = 0; r < NB; ++r) Rs[(c0 + r) * ldr + tid] = (float)sreg[r];
-      }
-      __syncthreads();
     }
   }
 
-  // ---- write back.  Right solves: solution v is row v0 + v of the result; left solves: column v0 + v.
+  // ---- write back.  Right solves: solution vid is row v0 + vid of the result; left solves: column v0 + vid.
   double acc = 0.0;
-  const int n_el = db * w;
-  for (int e = tid; e < n_el; e += NT) {
-    int r, v;
-    int64_t g;     // element of the [db][db] result
-    if (right) { v = e / db; r = e % db; g = (int64_t)(v0 + v) * db + r; }
-    else       { r = e / w;  v = e % w;  g = (int64_t)r * db + v0 + v; }
-    const float x = fail ? 0.f : Rs[r * ldr + v];
-    if (mode == 0) {
-      const float a = A[off + g] + x;
-      A[off + g] = a;
-      At[off + (int64_t)r * db + (v0 + v)] = a;
-      out[off + g] = x;
-      acc += (double)rhs[off + g] * (double)x + lam * (double)x * (double)x;
-    } else {
-      out[off + g] = x;
-      if (mode == 2) acc += (double)dotw[off + g] * (double)x;
+  {
+    const int q4 = db / 4;
+    const int m4 = right ? w * q4 : db * (w / 4);
+    for (int e0 = tid; e0 < m4; e0 += 4 * NT) {
+      float4 x[4], aold[4], gin[4];
+      int64_t gidx[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int e = e0 + u * NT;
+        x[u] = aold[u] = gin[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        gidx[u] = -1;
+        if (e >= m4) continue;
+        if (right) {
+          const int vid = e / q4, r4 = (e % q4) * 4;
+          gidx[u] = (int64_t)(v0 + vid) * db + r4;
+          if (!fail) x[u] = make_float4(Rs[r4 * ldr + vid], Rs[(r4 + 1) * ldr + vid], Rs[(r4 + 2) * ldr + vid],
+                                        Rs[(r4 + 3) * ldr + vid]);
+        } else {
+          const int r = e / (w / 4), vid4 = (e % (w / 4)) * 4;
+          gidx[u] = (int64_t)r * db + v0 + vid4;
+          if (!fail) x[u] = make_float4(Rs[r * ldr + vid4], Rs[r * ldr + vid4 + 1], Rs[r * ldr + vid4 + 2],
+                                        Rs[r * ldr + vid4 + 3]);
+        }
+        if (mode == 0) {
+          aold[u] = *reinterpret_cast<const float4*>(A + off + gidx[u]);
+          gin[u] = *reinterpret_cast<const float4*>(rhs + off + gidx[u]);
+        } else if (mode == 2) {
+          gin[u] = *reinterpret_cast<const float4*>(dotw + off + gidx[u]);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (gidx[u] < 0) continue;
+        *reinterpret_cast<float4*>(out + off + gidx[u]) = x[u];
+        if (mode == 0) {
+          *reinterpret_cast<float4*>(A + off + gidx[u]) =
+              make_float4(aold[u].x + x[u].x, aold[u].y + x[u].y, aold[u].z + x[u].z, aold[u].w + x[u].w);
+          acc += (double)gin[u].x * (double)x[u].x + lam * (double)x[u].x * (double)x[u].x;
+          acc += (double)gin[u].y * (double)x[u].y + lam * (double)x[u].y * (double)x[u].y;
+          acc += (double)gin[u].z * (double)x[u].z + lam * (double)x[u].z * (double)x[u].z;
+          acc += (double)gin[u].w * (double)x[u].w + lam * (double)x[u].w * (double)x[u].w;
+        } else if (mode == 2) {
+          acc += (double)gin[u].x * (double)x[u].x + (double)gin[u].y * (double)x[u].y +
+                 (double)gin[u].z * (double)x[u].z + (double)gin[u].w * (double)x[u].w;
+        }
+      }
     }
   }
   if (mode != 1) {
@@ -404,8 +513,7 @@ armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float*
   if (db % NB == 0) {
     const int slices = chol_parts_per_block(db);
     const int w = db / slices;
-    const size_t smem = ((panel_floats(db) + (size_t)db * (w + 1) + 1) & ~(size_t)1) * sizeof(float) +
-                        (size_t)db * sizeof(double);
+    const size_t smem = (panel_floats(db) + (size_t)db * (w + 1)) * sizeof(float);
     static size_t attr_bytes = 0;
     if (smem > attr_bytes) {
       if (cudaFuncSetAttribute(chol_blocked_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
