@@ -24,6 +24,7 @@
  *   - A, B: [d/d_block, d_block, d_block] fp32.  S: [d_out, d_in] fp32 with
  *     zeros outside the mask.  M: one byte per group of m_group consecutive
  *     columns, uint8 [d_out, d_in/m_group]; bit p set <=> column m*c+p kept.
+ *   - N:M patterns: 2:4 and 4:8 (Section 4.4 of the paper names both).
  */
 #ifndef ARMOR_H
 #define ARMOR_H
@@ -64,12 +65,13 @@ enum { ARMOR_DTYPE_F32 = 0, ARMOR_DTYPE_BF16 = 1 };
 
 typedef struct {
   int64_t d_out, d_in;
-  int32_t d_block;     /* divides d_out and d_in; multiple of m_group */
-  int32_t n_keep;      /* N of N:M (2) */
-  int32_t m_group;     /* M of N:M (4) */
+  int32_t d_block;     /* divides d_out and d_in; multiple of m_group; at most 256 */
+  int32_t n_keep;      /* N of N:M: 2 (with m_group 4) or 4 (with m_group 8) */
+  int32_t m_group;     /* M of N:M: 4 or 8 */
   int32_t h_mode;      /* ARMOR_H_* */
   int32_t select_mode; /* ARMOR_SELECT_* (Section 3.3.2 / Appendix E.1) */
-  int32_t s_step;      /* ARMOR_S_* */
+  int32_t s_step;      /* ARMOR_S_EXACT: exact line search along Gamma (.) M; ARMOR_S_BETA: the paper's
+                          step 1/beta_W' (Eq. lrWprime) */
   int32_t precision;   /* ARMOR_PREC_* */
   int32_t normalize;   /* 1: armor_init applies the NoWag normalisation */
   int32_t phases;      /* bitmask of ARMOR_PHASE_*; 0 means all four */
@@ -92,7 +94,8 @@ typedef struct {
 
 /* Scratch size for a configuration.  Error: INVALID_ARG (null), SHAPE
  * (d_block does not divide the dims, m_group does not divide d_block),
- * UNSUPPORTED (N:M other than 2:4, d_block > 128 or not a multiple of 32). */
+ * UNSUPPORTED (N:M other than 2:4 and 4:8; d_block > 256, not a multiple of 4, or above 128 and not a
+ * multiple of 32; tensor-core precisions with full weighting need d_out and d_in multiples of 128). */
 armor_status armor_workspace_bytes(const armor_config* cfg, size_t* bytes);
 
 /* Creates a context over caller-owned device scratch (256-byte aligned, at
@@ -104,7 +107,9 @@ armor_status armor_destroy(armor_ctx* ctx);
 /* Calibration Gram (Section 2 / Eq. proxy_loss: its diagonal is ||X_j||^2).
  * d_H [d_in, d_in] fp32 += X^T X for a chunk X [n_rows, d_in] with leading
  * dimension ldx (elements).  The caller zeroes d_H before the first chunk.
- * x_dtype: ARMOR_DTYPE_F32.  n_rows == 0 is a no-op. */
+ * x_dtype: ARMOR_DTYPE_F32 or ARMOR_DTYPE_BF16 (bf16 values are exact tensor-core
+ * operands, so their Gram needs one pass in every tensor-core precision; not
+ * available with ARMOR_PREC_SIMT).  n_rows == 0 is a no-op. */
 armor_status armor_gram(armor_ctx* ctx, const void* d_X, int32_t x_dtype, int64_t n_rows, int64_t ldx,
                         float* d_H, armor_stream_t stream);
 
@@ -126,7 +131,7 @@ armor_status armor_init(armor_ctx* ctx, const float* d_W, const float* d_H, floa
  * per block, closed-form solve over all masks, Eq. mask_loss_opt and
  * mask_loss_opt_sol).  A, B, S, M are updated in place.  d_stats may be NULL,
  * else [n_iters].  Each iteration is a function of (state, W, H, t) only, so
- * splitting a run into several calls gives the same bits. */
+ * splitting a run into several calls gives the same bits in A, B, S and M. */
 armor_status armor_bcd_step(armor_ctx* ctx, const float* d_Wbar, const float* d_H, float* d_A, float* d_B,
                             float* d_S, uint8_t* d_M, int64_t t_first, int32_t n_iters,
                             armor_iter_stats* d_stats, armor_stream_t stream);
@@ -139,8 +144,9 @@ armor_status armor_proxy_loss(armor_ctx* ctx, const float* d_Wbar, const float* 
 /* Deployment form (Section 3.1): y_t = A (S (B x_t)) for the rows of
  * x [n_tokens, d_in] -> y [n_tokens, d_out].  With d_r1, d_r2 non-NULL the
  * normalisation is undone: y_t = r2 (.) A S B (r1 (.) x_t).  xy_dtype:
- * ARMOR_DTYPE_F32.  d_M is accepted for symmetry and may be NULL (S already
- * carries the zeros). */
+ * ARMOR_DTYPE_F32, or ARMOR_DTYPE_BF16 for bf16 x and y (widened on the way in,
+ * rounded once on the way out; the products run in the context's precision).
+ * d_M is accepted for symmetry and may be NULL (S already carries the zeros). */
 armor_status armor_apply(armor_ctx* ctx, const float* d_A, const float* d_B, const float* d_S,
                          const uint8_t* d_M, const float* d_r1, const float* d_r2, const void* d_x,
                          void* d_y, int32_t xy_dtype, int64_t n_tokens, armor_stream_t stream);

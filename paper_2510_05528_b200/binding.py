@@ -133,10 +133,11 @@ def armor_destroy(ctx) -> None:
 def armor_gram(ctx, X: torch.Tensor, H: torch.Tensor) -> None:
     if X.dim() != 2 or X.stride(1) != 1:
         raise ValueError("X must be [n_rows, d_in] with unit column stride")
-    if not X.is_cuda or X.dtype != torch.float32:
-        raise ValueError("X must be a float32 CUDA tensor (this library has no CPU path)")
+    if not X.is_cuda or X.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError("X must be a float32 or bfloat16 CUDA tensor (this library has no CPU path)")
     ldx = X.stride(0) if X.shape[0] > 1 else X.shape[1]
-    _check(lib().armor_gram(ctx, C.c_void_p(X.data_ptr()), DTYPE_F32, X.shape[0], ldx,
+    _check(lib().armor_gram(ctx, C.c_void_p(X.data_ptr()), DTYPE_BF16 if X.dtype == torch.bfloat16 else DTYPE_F32,
+                            X.shape[0], ldx,
                             _ptr(H, torch.float32, "H"), _stream()), "armor_gram")
 
 
@@ -162,8 +163,11 @@ def armor_proxy_loss(ctx, Wbar, H, A, B, S, loss: torch.Tensor) -> None:
 
 def armor_apply(ctx, A, B, S, M, r1, r2, x, y) -> None:
     f = torch.float32
+    if x.dtype != y.dtype or x.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError("x and y must both be float32 or both be bfloat16")
+    dt = DTYPE_BF16 if x.dtype == torch.bfloat16 else DTYPE_F32
     _check(lib().armor_apply(ctx, _ptr(A, f, "A"), _ptr(B, f, "B"), _ptr(S, f, "S"), _ptr(M, torch.uint8, "M"),
-                             _ptr(r1, f, "r1"), _ptr(r2, f, "r2"), _ptr(x, f, "x"), _ptr(y, f, "y"), DTYPE_F32,
+                             _ptr(r1, f, "r1"), _ptr(r2, f, "r2"), _ptr(x, x.dtype, "x"), _ptr(y, y.dtype, "y"), dt,
                              x.shape[0], _stream()), "armor_apply")
 
 
@@ -277,7 +281,7 @@ class ArmorContext:
         return out
 
     def apply(self, st: LayerState, x: torch.Tensor, denormalize: bool = False) -> torch.Tensor:
-        y = torch.empty(x.shape[0], self.d_out, dtype=torch.float32, device=self.device)
+        y = torch.empty(x.shape[0], self.d_out, dtype=x.dtype, device=self.device)
         r1, r2 = (st.r1, st.r2) if denormalize else (None, None)
         armor_apply(self.ctx, st.A, st.B, st.S, st.M, r1, r2, x, y)
         return y

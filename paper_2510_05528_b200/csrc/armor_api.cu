@@ -21,13 +21,13 @@ armor_status check_config(const armor_config* cfg) {
   if (cfg->d_out <= 0 || cfg->d_in <= 0 || cfg->d_block <= 0) return ARMOR_ERR_SHAPE;
   if (cfg->m_group <= 0 || cfg->n_keep <= 0 || cfg->n_keep > cfg->m_group) return ARMOR_ERR_SHAPE;
   if (cfg->d_out % cfg->d_block || cfg->d_in % cfg->d_block || cfg->d_block % cfg->m_group) return ARMOR_ERR_SHAPE;
-  if (cfg->n_keep != 2 || cfg->m_group != 4) return ARMOR_ERR_UNSUPPORTED;
-  if (cfg->d_block > 128 || cfg->d_block % 4) return ARMOR_ERR_UNSUPPORTED;
+  if (!((cfg->n_keep == 2 && cfg->m_group == 4) || (cfg->n_keep == 4 && cfg->m_group == 8))) return ARMOR_ERR_UNSUPPORTED;
+  if (cfg->d_block > 256 || cfg->d_block % 4) return ARMOR_ERR_UNSUPPORTED;
+  if (cfg->d_block > 128 && cfg->d_block % 32) return ARMOR_ERR_UNSUPPORTED;   // large blocks use the panel solver
   if (cfg->h_mode != ARMOR_H_FULL && cfg->h_mode != ARMOR_H_DIAG) return ARMOR_ERR_INVALID_ARG;
   if (cfg->select_mode != ARMOR_SELECT_L1_RANDOM && cfg->select_mode != ARMOR_SELECT_L1_GREEDY)
     return ARMOR_ERR_INVALID_ARG;
   if (cfg->s_step != ARMOR_S_EXACT && cfg->s_step != ARMOR_S_BETA) return ARMOR_ERR_INVALID_ARG;
-  if (cfg->s_step == ARMOR_S_BETA) return ARMOR_ERR_UNSUPPORTED;
   if (cfg->precision < ARMOR_PREC_FP32X3 || cfg->precision > ARMOR_PREC_SIMT) return ARMOR_ERR_INVALID_ARG;
   if (cfg->precision != ARMOR_PREC_SIMT) {
     // the tensor-core GEMM works on whole 128 x 128 tiles with K in steps of 32
@@ -97,6 +97,10 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
     TAKE(gpart, float*, (size_t)gp * sizeof(float));
     if (c) c->gpart_floats = gp;
   }
+  if (cfg.s_step == ARMOR_S_BETA && cfg.h_mode == ARMOR_H_FULL) {
+    TAKE(Hq1, float*, hbytes);
+    TAKE(Hq2, float*, hbytes);
+  } else if (c) { c->Hq1 = nullptr; c->Hq2 = nullptr; }
   TAKE(sc, double*, SC_COUNT * sizeof(double));
   TAKE(partials, double*, (size_t)8 * npart * sizeof(double));
   const int64_t nbmax = nbo > nbi ? nbo : nbi;
@@ -272,10 +276,8 @@ armor_status armor_gram(armor_ctx* c, const void* d_X, int32_t x_dtype, int64_t 
   if (!c || !d_H || n_rows < 0) return ARMOR_ERR_INVALID_ARG;
   if (n_rows == 0) return ARMOR_OK;
   if (!d_X || ldx < c->d_in) return ARMOR_ERR_INVALID_ARG;
-  if (x_dtype != ARMOR_DTYPE_F32) return ARMOR_ERR_UNSUPPORTED;
-  cudaStream_t s = cs(stream);
-  const float* X = static_cast<const float*>(d_X);
-  return gram_accumulate(c, X, n_rows, ldx, d_H, s);
+  if (x_dtype != ARMOR_DTYPE_F32 && x_dtype != ARMOR_DTYPE_BF16) return ARMOR_ERR_UNSUPPORTED;
+  return gram_accumulate(c, d_X, x_dtype, n_rows, ldx, d_H, cs(stream));
 }
 
 armor_status armor_init(armor_ctx* c, const float* d_W, const float* d_H, float* d_Wbar, float* d_r1, float* d_r2,
@@ -359,7 +361,21 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       bd_right(c, c->Tmp, B, false, c->V, d_out, d_in, 1.f, nullptr, 0.f, s);        // V = A Gamma_M B
       st = rmul_H(c, c->V, H, c->VH, d_out, c->V, c->sc + SC_Q_S, nullptr, nullptr, s);
       if (st != ARMOR_OK) return st;
-      launch_stage(c, is, 3, nullptr, 0, 0, s);
+      if (c->cfg.s_step == ARMOR_S_BETA) {
+        // the paper's step size (Eq. lrWprime): |A^T A|_F and |B H_w B^T|_F
+        block_mm(c, A, true, A, false, c->G, nbo, s);
+        dot_to_ptr(c, c->G, c->G, (int64_t)nbo * db * db, c->sc + SC_BETA_A, s);
+        if (c->cfg.h_mode == ARMOR_H_FULL) {
+          bd_left(c, B, false, H, c->Hq1, d_in, d_in, 1.f, nullptr, 0.f, s);
+          bd_right(c, c->Hq1, B, true, c->Hq2, d_in, d_in, 1.f, nullptr, 0.f, s);
+          dot_to_ptr(c, c->Hq2, c->Hq2, d_in * d_in, c->sc + SC_BETA_K, s);
+        } else {
+          block_mm(c, B, false, c->Hjj, false, c->Ktmp, nbi, s);
+          block_mm(c, c->Ktmp, false, B, true, c->Kfull, nbi, s);
+          dot_to_ptr(c, c->Kfull, c->Kfull, (int64_t)nbi * db * db, c->sc + SC_BETA_K, s);
+        }
+      }
+      launch_stage(c, is, c->cfg.s_step == ARMOR_S_BETA ? 6 : 3, nullptr, 0, 0, s);
       launch_axpy_slot(c, S, c->U, c->wn, SC_TAU_S, 1.f, s);                         // S += tau Gamma_M
       launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_S, -1.f, s);                   // EH -= tau V H_w
     } else {
@@ -390,26 +406,37 @@ armor_status armor_apply(armor_ctx* c, const float* A, const float* B, const flo
   if (!c || !A || !B || !S || n_tokens < 0) return ARMOR_ERR_INVALID_ARG;
   if (n_tokens == 0) return ARMOR_OK;
   if (!d_x || !d_y) return ARMOR_ERR_INVALID_ARG;
-  if (xy_dtype != ARMOR_DTYPE_F32) return ARMOR_ERR_UNSUPPORTED;
+  if (xy_dtype != ARMOR_DTYPE_F32 && xy_dtype != ARMOR_DTYPE_BF16) return ARMOR_ERR_UNSUPPORTED;
   if ((r1 == nullptr) != (r2 == nullptr)) return ARMOR_ERR_INVALID_ARG;
   cudaStream_t s = cs(stream);
-  const float* x = static_cast<const float*>(d_x);
-  float* y = static_cast<float*>(d_y);
+  const bool bf16 = (xy_dtype == ARMOR_DTYPE_BF16);
+  const size_t esz = bf16 ? 2 : 4;
   const int64_t d_out = c->d_out, d_in = c->d_in;
   const int64_t chunk = d_out < d_in ? d_out : d_in;   // z1 [chunk, d_in] and z2 [chunk, d_out] fit W-shaped scratch
   for (int64_t t0 = 0; t0 < n_tokens; t0 += chunk) {
     const int64_t n = (n_tokens - t0 < chunk) ? n_tokens - t0 : chunk;
-    const float* xc = x + t0 * d_in;
-    float* yc = y + t0 * d_out;
-    if (r1) {
-      launch_scale_rows_cols(c, xc, r1, nullptr, c->Tmp, n, d_in, s);
+    const float* xc;
+    float* yc;
+    if (bf16) {
+      // bf16 activations are widened on the way in and rounded once on the way out; the three products run in
+      // the context's precision
+      launch_bf16_to_f32(c, static_cast<const char*>(d_x) + (size_t)(t0 * d_in) * esz, r1, c->Tmp, n, d_in, s);
       xc = c->Tmp;
+      yc = c->V;
+    } else {
+      xc = static_cast<const float*>(d_x) + t0 * d_in;
+      yc = static_cast<float*>(d_y) + t0 * d_out;
+      if (r1) {
+        launch_scale_rows_cols(c, xc, r1, nullptr, c->Tmp, n, d_in, s);
+        xc = c->Tmp;
+      }
     }
     bd_right(c, xc, B, true, c->T, n, d_in, 1.f, nullptr, 0.f, s);                   // z1 = x B^T
     armor_status st = apply_core(c, c->T, S, c->E, n, s);                            // z2 = z1 S^T
     if (st != ARMOR_OK) return st;
     bd_right(c, c->E, A, true, yc, n, d_out, 1.f, nullptr, 0.f, s);                  // y = z2 A^T
-    if (r2) launch_scale_rows_cols(c, yc, r2, nullptr, yc, n, d_out, s);
+    if (bf16) launch_f32_to_bf16(c, yc, r2, static_cast<char*>(d_y) + (size_t)(t0 * d_out) * esz, n, d_out, s);
+    else if (r2) launch_scale_rows_cols(c, yc, r2, nullptr, yc, n, d_out, s);
   }
   return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
 }

@@ -39,8 +39,8 @@ struct SelRec {
   int32_t cgrp;       // group index inside the row (columns m*cgrp ..)
   int32_t new_mask;   // bit p <=> position p kept
   int32_t old_mask;
-  float new_val[4];
-  float old_val[4];
+  float new_val[8];
+  float old_val[8];
 };
 
 static const int ARMOR_DOT_BLOCKS = 592;  // 4 x 148 partial sums per reduction
@@ -58,6 +58,7 @@ struct armor_ctx {
   // [nb, db, db] scratch
   float *G, *GamA, *dA, *At, *C, *GamB, *Delta, *Hjj, *Kfull, *Ktmp, *Bt;
   float *alpha, *hdiag;
+  float *Hq1, *Hq2;      // [d_in, d_in] scratch of the paper's step size (s_step BETA, full weighting)
   float* gpart;          // partial products of split contractions
   int64_t gpart_floats;
   // sparse-core update: per selected group z = delta^T B_j[rows of the group, :] and a = A_i[:, r]
@@ -134,7 +135,8 @@ armor_status rmul_H(armor_ctx* c, const float* in, const float* H, float* out, i
                     const float* d1, double* out1, const float* d2, double* out2, cudaStream_t s);
 // per-call preparation of everything derived from H (diagonal, diagonal blocks, split copy)
 armor_status prepare_H(armor_ctx* c, const float* H, cudaStream_t s);
-armor_status gram_accumulate(armor_ctx* c, const float* X, int64_t n_rows, int64_t ldx, float* H, cudaStream_t s);
+armor_status gram_accumulate(armor_ctx* c, const void* X, int x_dtype, int64_t n_rows, int64_t ldx, float* H,
+                             cudaStream_t s);
 // z2 [n, d_out] = z1 [n, d_in] * S^T
 armor_status apply_core(armor_ctx* c, const float* z1, const float* S, float* z2, int64_t n, cudaStream_t s);
 
@@ -161,8 +163,12 @@ void launch_stage(armor_ctx* c, armor_iter_stats* st, int stage, const double* p
 void launch_scale_rows_cols(armor_ctx* c, const float* in, const float* colscale, const float* rowscale,
                             float* out, int64_t rows, int64_t cols, cudaStream_t s);
 void launch_split_hilo(armor_ctx* c, const float* in, float* hi, float* lo, int64_t n, cudaStream_t s);
-void launch_transpose_split(armor_ctx* c, const float* X, int64_t ldx, int64_t rows, int64_t cols,
+void launch_transpose_split(armor_ctx* c, const void* X, int x_dtype, int64_t ldx, int64_t rows, int64_t cols,
                             float* Thi, float* Tlo, int64_t ldt, cudaStream_t s);
+void launch_bf16_to_f32(armor_ctx* c, const void* in, const float* colscale, float* out, int64_t rows, int64_t cols,
+                        cudaStream_t s);
+void launch_f32_to_bf16(armor_ctx* c, const float* in, const float* colscale, void* out, int64_t rows, int64_t cols,
+                        cudaStream_t s);
 
 // block solves (kernels_chol.cu)
 // mode 0: X = rhs (G + lam I)^-1, A += X, At = A^T, out = X, part[b] = exact decrease of block b

@@ -56,9 +56,13 @@ armor_status rmul_H(armor_ctx* c, const float* in, const float* H, float* out, i
   return ARMOR_OK;
 }
 
-armor_status gram_accumulate(armor_ctx* c, const float* X, int64_t n_rows, int64_t ldx, float* H, cudaStream_t s) {
+armor_status gram_accumulate(armor_ctx* c, const void* Xv, int x_dtype, int64_t n_rows, int64_t ldx, float* H,
+                             cudaStream_t s) {
   const int64_t d_in = c->d_in;
+  const float* X = static_cast<const float*>(Xv);
+  const bool bf16 = (x_dtype == ARMOR_DTYPE_BF16);
   if (c->cfg.precision == ARMOR_PREC_SIMT) {
+    if (bf16) return ARMOR_ERR_UNSUPPORTED;
     // H += X^T X, element (m, k) of the left operand is X[k][m]
     const int64_t step = 1 << 20;
     for (int64_t r0 = 0; r0 < n_rows; r0 += step) {
@@ -73,11 +77,14 @@ armor_status gram_accumulate(armor_ctx* c, const float* X, int64_t n_rows, int64
     }
     return ARMOR_OK;
   }
-  const bool x3 = c->cfg.precision == ARMOR_PREC_FP32X3;
+  // bf16 values are exact in tf32: one tensor-core pass gives exact products
+  const bool x3 = c->cfg.precision == ARMOR_PREC_FP32X3 && !bf16;
+  const size_t esz = bf16 ? 2 : 4;
   for (int64_t r0 = 0; r0 < n_rows; r0 += c->gram_rows) {
     const int64_t n = n_rows - r0 < c->gram_rows ? n_rows - r0 : c->gram_rows;
     const int64_t kpad = (n + 31) / 32 * 32;     // staged row length (zero padded)
-    launch_transpose_split(c, X + r0 * ldx, ldx, n, d_in, c->Xt_hi, x3 ? c->Xt_lo : nullptr, kpad, s);
+    launch_transpose_split(c, static_cast<const char*>(Xv) + (size_t)(r0 * ldx) * esz, x_dtype, ldx, n, d_in, c->Xt_hi,
+                           x3 ? c->Xt_lo : nullptr, kpad, s);
     TcGemm g{};
     g.A = c->Xt_hi; g.Alo = c->Xt_lo; g.lda = kpad;
     g.B = c->Xt_hi; g.Blo = c->Xt_lo; g.ldb = kpad;
@@ -86,7 +93,7 @@ armor_status gram_accumulate(armor_ctx* c, const float* X, int64_t n_rows, int64
     g.passes = x3 ? 3 : 1;
     g.accumulate = 1;
     g.symmetric_lower = 1;
-    g.k_segment = x3 ? K_SEGMENT : 4 * K_SEGMENT;
+    g.k_segment = (c->cfg.precision == ARMOR_PREC_FP32X3) ? K_SEGMENT : 4 * K_SEGMENT;
     armor_status st = launch_tc_gemm(c, g, nullptr, s);
     if (st != ARMOR_OK) return st;
   }

@@ -54,18 +54,69 @@ __device__ __forceinline__ void pinv2(double k11, double k12, double k22, double
   red = z1 * w1 + z2 * w2;
 }
 
-// One CTA per (i, j) block.  Pass 1: float4 per group, score, key, arg-min by warp shuffles.
-// Pass 2 (thread 0): the six-mask sweep for the winner.
+// n x n SPD solve (n <= 4) by unpivoted Cholesky; false if a pivot is not positive (that mask is skipped).
+__device__ __forceinline__ bool chol_small(int n, const double (&Kin)[4][4], const double (&z)[4], double (&w)[4],
+                                           double& red) {
+  double L[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (i >= n || j > i) continue;
+      double sacc = Kin[i][j];
+#pragma unroll
+      for (int p = 0; p < 4; ++p)
+        if (p < j) sacc -= L[i][p] * L[j][p];
+      if (i == j) {
+        if (!(sacc > 0.0) || !isfinite(sacc)) return false;
+        L[i][i] = sqrt(sacc);
+      } else {
+        L[i][j] = sacc / L[j][j];
+      }
+    }
+  }
+  double y[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    if (i >= n) continue;
+    double sacc = z[i];
+#pragma unroll
+    for (int p = 0; p < 4; ++p)
+      if (p < i) sacc -= L[i][p] * y[p];
+    y[i] = sacc / L[i][i];
+  }
+#pragma unroll
+  for (int i = 3; i >= 0; --i) {
+    if (i >= n) continue;
+    double sacc = y[i];
+#pragma unroll
+    for (int p = 0; p < 4; ++p)
+      if (p > i && p < n) sacc -= L[p][i] * w[p];
+    w[i] = sacc / L[i][i];
+  }
+  red = 0.0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    if (i < n) red += z[i] * w[i];
+  return true;
+}
+
+// One CTA per (i, j) block of the core, N:M groups with M = MG (4 or 8) and N = n_keep (<= 4).
+// Pass 1: every group of the block is scored, keyed and the arg-min found by warp shuffles.
+// Pass 2: thread b < 2^MG evaluates the mask with bit pattern b (if it keeps exactly n_keep positions);
+// the best one is found with the oracle's order: larger reduction first; among equal reductions the
+// incumbent, then the lexicographically first index tuple.
+template <int MG>
 __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict__ Gam, const float* __restrict__ S,
                                                          const uint8_t* __restrict__ M, const float* __restrict__ alpha,
                                                          const float* __restrict__ Kfull, SelRec* __restrict__ sel,
                                                          double* __restrict__ part, int64_t d_in, int db, int nbi,
-                                                         int select_mode, uint64_t seed, uint64_t t,
+                                                         int n_keep, int select_mode, uint64_t seed, uint64_t t,
                                                          uint64_t n_groups_total) {
   const int blk = blockIdx.x;
   const int bi = blk / nbi, bj = blk % nbi;
-  const int gpb = db / 4;                 // groups per block row
-  const int64_t ng_row = d_in / 4;        // groups per matrix row
+  const int gpb = db / MG;                // groups per block row
+  const int64_t ng_row = d_in / MG;       // groups per matrix row
   const int n_in_block = db * gpb;
   float best_key = INFINITY;
   uint64_t best_g = ~0ull;
@@ -73,8 +124,15 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
     const int rl = idx / gpb, cl = idx % gpb;
     const int64_t row = (int64_t)bi * db + rl;
     const int64_t cg = (int64_t)bj * gpb + cl;
-    const float4 g4 = *reinterpret_cast<const float4*>(Gam + row * d_in + cg * 4);
-    float score = fabsf(g4.x) + fabsf(g4.y) + fabsf(g4.z) + fabsf(g4.w);
+    float score = 0.f;
+#pragma unroll
+    for (int h = 0; h < MG / 4; ++h) {
+      const float4 g4 = *reinterpret_cast<const float4*>(Gam + row * d_in + cg * MG + 4 * h);
+      score += fabsf(g4.x);
+      score += fabsf(g4.y);
+      score += fabsf(g4.z);
+      score += fabsf(g4.w);
+    }
     if (!(alpha[row] > 0.f)) score = 0.f;
     const uint64_t g = (uint64_t)row * (uint64_t)ng_row + (uint64_t)cg;
     float key = INFINITY;
@@ -96,60 +154,135 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
   }
   __shared__ float skey[NT / 32];
   __shared__ uint64_t sg[NT / 32];
+  __shared__ float s_key;
+  __shared__ uint64_t s_g;
   if ((threadIdx.x & 31) == 0) { skey[threadIdx.x >> 5] = best_key; sg[threadIdx.x >> 5] = best_g; }
   __syncthreads();
-  if (threadIdx.x != 0) return;
-  for (int w = 1; w < NT / 32; ++w)
-    if (skey[w] < best_key || (skey[w] == best_key && sg[w] < best_g)) { best_key = skey[w]; best_g = sg[w]; }
-
-  SelRec rec;
-  double ehv = 0.0;
-  rec.valid = 0; rec.row = 0; rec.cgrp = 0; rec.new_mask = 0; rec.old_mask = 0;
-  for (int p = 0; p < 4; ++p) { rec.new_val[p] = 0.f; rec.old_val[p] = 0.f; }
-  if (best_key < INFINITY) {
-    const int64_t row = (int64_t)(best_g / (uint64_t)ng_row);
-    const int64_t cg = (int64_t)(best_g % (uint64_t)ng_row);
-    const int lc = (int)(cg % gpb) * 4;   // first row of the group inside B_j
-    const float* Kj = Kfull + (int64_t)bj * db * db;
-    double K[4][4], z[4], sg4[4];
-    const double a_r = (double)alpha[row];
-    const unsigned om = M[row * ng_row + cg];
-    for (int p = 0; p < 4; ++p) {
-      sg4[p] = (double)S[row * d_in + cg * 4 + p];
-      for (int q = 0; q < 4; ++q) K[p][q] = (double)Kj[(int64_t)(lc + p) * db + (lc + q)];
-    }
-    for (int p = 0; p < 4; ++p) {
-      double kz = 0.0;
-      for (int q = 0; q < 4; ++q) kz += K[p][q] * sg4[q];
-      z[p] = (double)Gam[row * d_in + cg * 4 + p] + a_r * kz;
-    }
-    // incumbent first, then lexicographic order; strict improvement only
-    const int pa[6] = {0, 0, 0, 1, 1, 2}, pb[6] = {1, 2, 3, 2, 3, 3};
-    int inc = -1;
-    for (int m = 0; m < 6; ++m)
-      if (om == ((1u << pa[m]) | (1u << pb[m]))) inc = m;
-    double best_red = -INFINITY, bw1 = 0.0, bw2 = 0.0;
-    int best_m = -1;
-    for (int step = (inc >= 0 ? -1 : 0); step < 6; ++step) {
-      const int m = (step < 0) ? inc : step;
-      if (step >= 0 && m == inc) continue;
-      double w1, w2, red;
-      pinv2(K[pa[m]][pa[m]], K[pa[m]][pb[m]], K[pb[m]][pb[m]], z[pa[m]], z[pb[m]], w1, w2, red);
-      red /= a_r;
-      if (best_m < 0 || red > best_red) { best_red = red; best_m = m; bw1 = w1 / a_r; bw2 = w2 / a_r; }
-    }
-    rec.valid = 1;
-    rec.row = (int32_t)row;
-    rec.cgrp = (int32_t)cg;
-    rec.old_mask = (int32_t)om;
-    rec.new_mask = (int32_t)((1u << pa[best_m]) | (1u << pb[best_m]));
-    for (int p = 0; p < 4; ++p) rec.old_val[p] = (float)sg4[p];
-    rec.new_val[pa[best_m]] = (float)bw1;
-    rec.new_val[pb[best_m]] = (float)bw2;
-    // <Gamma, dS> restricted to this group: this block's share of <E H_w, V>
-    for (int p = 0; p < 4; ++p)
-      ehv += (double)Gam[row * d_in + cg * 4 + p] * ((double)rec.new_val[p] - (double)rec.old_val[p]);
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < NT / 32; ++w)
+      if (skey[w] < best_key || (skey[w] == best_key && sg[w] < best_g)) { best_key = skey[w]; best_g = sg[w]; }
+    s_key = best_key;
+    s_g = best_g;
   }
+  __syncthreads();
+  best_key = s_key;
+  best_g = s_g;
+  if (!(best_key < INFINITY)) {
+    if (threadIdx.x == 0) {
+      SelRec rec;
+      rec.valid = 0; rec.row = 0; rec.cgrp = 0; rec.new_mask = 0; rec.old_mask = 0;
+      for (int p = 0; p < 8; ++p) { rec.new_val[p] = 0.f; rec.old_val[p] = 0.f; }
+      sel[blk] = rec;
+      part[blk] = 0.0;
+    }
+    return;
+  }
+
+  // ---- the selected group: z = Gamma_g + alpha K_c s_g, one candidate mask per thread
+  const int64_t row = (int64_t)(best_g / (uint64_t)ng_row);
+  const int64_t cg = (int64_t)(best_g % (uint64_t)ng_row);
+  const int lc = (int)(cg % gpb) * MG;   // first row of the group inside B_j
+  const float* Kj = Kfull + (int64_t)bj * db * db;
+  const double a_r = (double)alpha[row];
+  const unsigned om = M[row * ng_row + cg];
+  double z[MG], sg_old[MG];
+#pragma unroll
+  for (int p = 0; p < MG; ++p) sg_old[p] = (double)S[row * d_in + cg * MG + p];
+#pragma unroll
+  for (int p = 0; p < MG; ++p) {
+    double kz = 0.0;
+#pragma unroll
+    for (int q = 0; q < MG; ++q) kz += (double)Kj[(int64_t)(lc + p) * db + (lc + q)] * sg_old[q];
+    z[p] = (double)Gam[row * d_in + cg * MG + p] + a_r * kz;
+  }
+  const unsigned cand = threadIdx.x;
+  bool ok = cand < (1u << MG) && __popc(cand) == n_keep;
+  double red = 0.0, wv[4] = {0.0, 0.0, 0.0, 0.0};
+  int pos[4] = {0, 0, 0, 0};
+  if (ok) {
+    int cnt = 0;
+#pragma unroll
+    for (int p = 0; p < MG; ++p)
+      if ((cand >> p) & 1u) { if (cnt < 4) pos[cnt] = p; ++cnt; }
+    if (n_keep == 2) {
+      pinv2((double)Kj[(int64_t)(lc + pos[0]) * db + lc + pos[0]], (double)Kj[(int64_t)(lc + pos[0]) * db + lc + pos[1]],
+            (double)Kj[(int64_t)(lc + pos[1]) * db + lc + pos[1]], z[pos[0]], z[pos[1]], wv[0], wv[1], red);
+    } else {
+      double Ks[4][4], zs[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        zs[i] = 0.0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) Ks[i][j] = 0.0;
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (i >= n_keep) continue;
+#pragma unroll
+        for (int p = 0; p < MG; ++p)
+          if (p == pos[i]) zs[i] = z[p];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (j < n_keep) Ks[i][j] = (double)Kj[(int64_t)(lc + pos[i]) * db + lc + pos[j]];
+      }
+      ok = chol_small(n_keep, Ks, zs, wv, red);
+    }
+    red /= a_r;
+  }
+  // order: larger reduction; then the incumbent; then the lexicographically first tuple (= larger
+  // bit-reversed pattern)
+  const unsigned rev = __brev(cand) >> (32 - MG);
+  double b_red = ok ? red : -INFINITY;
+  unsigned b_tie = ok ? (((cand == om) ? (1u << MG) : 0u) | rev) : 0u;
+  unsigned b_cand = ok ? cand : 0xffffffffu;
+  for (int o = 16; o > 0; o >>= 1) {
+    const double o_red = __shfl_down_sync(0xffffffffu, b_red, o);
+    const unsigned o_tie = __shfl_down_sync(0xffffffffu, b_tie, o);
+    const unsigned o_cand = __shfl_down_sync(0xffffffffu, b_cand, o);
+    const bool take = (o_cand != 0xffffffffu) &&
+                      (b_cand == 0xffffffffu || o_red > b_red || (o_red == b_red && o_tie > b_tie));
+    if (take) { b_red = o_red; b_tie = o_tie; b_cand = o_cand; }
+  }
+  __shared__ double sred[NT / 32];
+  __shared__ unsigned stie[NT / 32], scand[NT / 32];
+  __shared__ unsigned s_win;
+  if ((threadIdx.x & 31) == 0) { sred[threadIdx.x >> 5] = b_red; stie[threadIdx.x >> 5] = b_tie; scand[threadIdx.x >> 5] = b_cand; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < NT / 32; ++w) {
+      const bool take = (scand[w] != 0xffffffffu) &&
+                        (b_cand == 0xffffffffu || sred[w] > b_red || (sred[w] == b_red && stie[w] > b_tie));
+      if (take) { b_red = sred[w]; b_tie = stie[w]; b_cand = scand[w]; }
+    }
+    s_win = b_cand;
+    if (b_cand == 0xffffffffu) {   // every mask failed its factorisation: nothing happens in this block
+      SelRec rec;
+      rec.valid = 0; rec.row = 0; rec.cgrp = 0; rec.new_mask = 0; rec.old_mask = 0;
+      for (int p = 0; p < 8; ++p) { rec.new_val[p] = 0.f; rec.old_val[p] = 0.f; }
+      sel[blk] = rec;
+      part[blk] = 0.0;
+    }
+  }
+  __syncthreads();
+  if (s_win == 0xffffffffu || cand != s_win) return;
+  // the winning thread writes the record
+  SelRec rec;
+  rec.valid = 1;
+  rec.row = (int32_t)row;
+  rec.cgrp = (int32_t)cg;
+  rec.old_mask = (int32_t)om;
+  rec.new_mask = (int32_t)cand;
+  for (int p = 0; p < 8; ++p) { rec.new_val[p] = 0.f; rec.old_val[p] = 0.f; }
+#pragma unroll
+  for (int p = 0; p < MG; ++p) rec.old_val[p] = (float)sg_old[p];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    if (i < n_keep) rec.new_val[pos[i]] = (float)(wv[i] / a_r);
+  // <Gamma, dS> restricted to this group: this block's share of <E H_w, V>
+  double ehv = 0.0;
+#pragma unroll
+  for (int p = 0; p < MG; ++p)
+    ehv += (double)Gam[row * d_in + cg * MG + p] * ((double)rec.new_val[p] - (double)rec.old_val[p]);
   part[blk] = ehv;
   sel[blk] = rec;
 }
@@ -220,7 +353,7 @@ __global__ void __launch_bounds__(NT) mask_quad_kernel(const float* __restrict__
 }
 
 __global__ void mask_commit_kernel(const SelRec* __restrict__ sel, int nblocks, float* __restrict__ S,
-                                   uint8_t* __restrict__ M, int64_t d_in, const double* __restrict__ sc,
+                                   uint8_t* __restrict__ M, int64_t d_in, int mg, const double* __restrict__ sc,
                                    armor_iter_stats* st) {
   __shared__ int changed;
   if (threadIdx.x == 0) changed = 0;
@@ -231,9 +364,11 @@ __global__ void mask_commit_kernel(const SelRec* __restrict__ sel, int nblocks, 
     for (int b = threadIdx.x; b < nblocks; b += blockDim.x) {
       const SelRec rec = sel[b];
       if (!rec.valid) continue;
-      float* sp = S + (int64_t)rec.row * d_in + (int64_t)rec.cgrp * 4;
-      *reinterpret_cast<float4*>(sp) = make_float4(rec.new_val[0], rec.new_val[1], rec.new_val[2], rec.new_val[3]);
-      M[(int64_t)rec.row * (d_in / 4) + rec.cgrp] = (uint8_t)rec.new_mask;
+      float* sp = S + (int64_t)rec.row * d_in + (int64_t)rec.cgrp * mg;
+      for (int h = 0; h < mg / 4; ++h)
+        *reinterpret_cast<float4*>(sp + 4 * h) =
+            make_float4(rec.new_val[4 * h], rec.new_val[4 * h + 1], rec.new_val[4 * h + 2], rec.new_val[4 * h + 3]);
+      M[(int64_t)rec.row * (d_in / mg) + rec.cgrp] = (uint8_t)rec.new_mask;
       mine += (rec.new_mask != rec.old_mask) ? 1 : 0;
     }
   }
@@ -250,10 +385,16 @@ void launch_alpha(armor_ctx* c, const float* A, cudaStream_t s) {
 }
 
 void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const uint8_t* M, int64_t t, cudaStream_t s) {
-  mask_select_kernel<<<c->nbo * c->nbi, NT, 0, s>>>(Gam, S, M, c->alpha, c->Kfull, c->sel, c->partblk, c->d_in, c->db,
-                                                   c->nbi,
-                                                   c->cfg.select_mode, c->cfg.seed, (uint64_t)t,
-                                                   (uint64_t)(c->d_out * (c->d_in / 4)));
+  const int mg = c->cfg.m_group;
+  const uint64_t n_groups = (uint64_t)(c->d_out * (c->d_in / mg));
+  if (mg == 8)
+    mask_select_kernel<8><<<c->nbo * c->nbi, NT, 0, s>>>(Gam, S, M, c->alpha, c->Kfull, c->sel, c->partblk, c->d_in,
+                                                        c->db, c->nbi, c->cfg.n_keep, c->cfg.select_mode, c->cfg.seed,
+                                                        (uint64_t)t, n_groups);
+  else
+    mask_select_kernel<4><<<c->nbo * c->nbi, NT, 0, s>>>(Gam, S, M, c->alpha, c->Kfull, c->sel, c->partblk, c->d_in,
+                                                        c->db, c->nbi, c->cfg.n_keep, c->cfg.select_mode, c->cfg.seed,
+                                                        (uint64_t)t, n_groups);
   c->launches++;
 }
 
@@ -279,6 +420,6 @@ void launch_mask_quadratic(armor_ctx* c, const float* A, const float* B, const f
 }
 
 void launch_mask_commit(armor_ctx* c, float* S, uint8_t* M, armor_iter_stats* st, cudaStream_t s) {
-  mask_commit_kernel<<<1, 256, 0, s>>>(c->sel, c->nbo * c->nbi, S, M, c->d_in, c->sc, st);
+  mask_commit_kernel<<<1, 256, 0, s>>>(c->sel, c->nbo * c->nbi, S, M, c->d_in, c->cfg.m_group, c->sc, st);
   c->launches++;
 }

@@ -1,4 +1,6 @@
 // Streaming (HBM-bound) kernels over W-shaped tensors, reductions and small bookkeeping kernels.
+#include <cuda_bf16.h>
+
 #include "armor_internal.cuh"
 
 namespace {
@@ -88,13 +90,14 @@ __global__ void transpose_blocks_kernel(const float* __restrict__ in, float* __r
 }
 
 // ---- Gamma_M = Gamma (.) M and its squared norm -------------------------------------------------
+// One float4 per thread step; a mask byte covers m_group / 4 consecutive float4 (q4 = 1 or 2).
 __global__ void __launch_bounds__(NT) masked_copy_kernel(const float4* __restrict__ gam, const uint8_t* __restrict__ M,
-                                                         float4* __restrict__ out, int64_t ngroups,
+                                                         float4* __restrict__ out, int64_t n4, int q4,
                                                          double* __restrict__ part) {
   double acc = 0.0;
-  for (int64_t g = (int64_t)blockIdx.x * NT + threadIdx.x; g < ngroups; g += (int64_t)gridDim.x * NT) {
+  for (int64_t g = (int64_t)blockIdx.x * NT + threadIdx.x; g < n4; g += (int64_t)gridDim.x * NT) {
     float4 v = gam[g];
-    const unsigned m = M[g];
+    const unsigned m = (q4 == 1) ? M[g] : ((unsigned)M[g >> 1] >> (4 * (int)(g & 1)));
     v.x = (m & 1u) ? v.x : 0.f;
     v.y = (m & 2u) ? v.y : 0.f;
     v.z = (m & 4u) ? v.z : 0.f;
@@ -168,31 +171,41 @@ __global__ void __launch_bounds__(NT) rownorm_scale_kernel(const float* __restri
   for (int64_t c = threadIdx.x; c < cols; c += NT) Wbar[row * cols + c] = (w[c] / r1[c]) / rr;
 }
 
-// ---- initialisation (Eq. init): top-2 of each group of 4 by W^2 * H_jj --------------------------
-__global__ void __launch_bounds__(NT) init_core_kernel(const float4* __restrict__ W, const float* __restrict__ H,
-                                                       int64_t d_in, float4* __restrict__ S, uint8_t* __restrict__ M,
-                                                       int64_t ngroups, int groups_per_row) {
+// ---- initialisation (Eq. init): top-n_keep of each group of MG by W^2 * H_jj ---------------------
+// Position p is kept iff fewer than n_keep positions beat it; q beats p if its score is larger, or equal
+// with q < p (ties keep the lower column).
+template <int MG>
+__global__ void __launch_bounds__(NT) init_core_kernel(const float* __restrict__ W, const float* __restrict__ H,
+                                                       int64_t d_in, float* __restrict__ S, uint8_t* __restrict__ M,
+                                                       int64_t ngroups, int groups_per_row, int n_keep) {
   for (int64_t g = (int64_t)blockIdx.x * NT + threadIdx.x; g < ngroups; g += (int64_t)gridDim.x * NT) {
-    const int64_t c0 = (g % groups_per_row) * 4;
-    float4 w = W[g];
-    const float wv[4] = {w.x, w.y, w.z, w.w};
-    double sc[4];
+    const int64_t c0 = (g % groups_per_row) * MG;
+    float wv[MG];
 #pragma unroll
-    for (int p = 0; p < 4; ++p) {
-      double h = (double)H[(c0 + p) * d_in + (c0 + p)];
+    for (int h = 0; h < MG / 4; ++h) {
+      const float4 w = *reinterpret_cast<const float4*>(W + g * MG + 4 * h);
+      wv[4 * h] = w.x; wv[4 * h + 1] = w.y; wv[4 * h + 2] = w.z; wv[4 * h + 3] = w.w;
+    }
+    double sc[MG];
+#pragma unroll
+    for (int p = 0; p < MG; ++p) {
+      const double h = (double)H[(c0 + p) * d_in + (c0 + p)];
       sc[p] = (double)wv[p] * (double)wv[p] * h;
     }
-    int i1 = 0;
+    unsigned m = 0;
 #pragma unroll
-    for (int p = 1; p < 4; ++p)
-      if (sc[p] > sc[i1]) i1 = p;  // strict: ties keep the lower column
-    int i2 = (i1 == 0) ? 1 : 0;
+    for (int p = 0; p < MG; ++p) {
+      int beaten = 0;
 #pragma unroll
-    for (int p = 0; p < 4; ++p)
-      if (p != i1 && p != i2 && sc[p] > sc[i2]) i2 = p;
-    const unsigned m = (1u << i1) | (1u << i2);
+      for (int q = 0; q < MG; ++q) beaten += (q != p) && (sc[q] > sc[p] || (sc[q] == sc[p] && q < p));
+      if (beaten < n_keep) m |= 1u << p;
+    }
     M[g] = (uint8_t)m;
-    S[g] = make_float4((m & 1u) ? w.x : 0.f, (m & 2u) ? w.y : 0.f, (m & 4u) ? w.z : 0.f, (m & 8u) ? w.w : 0.f);
+#pragma unroll
+    for (int h = 0; h < MG / 4; ++h)
+      *reinterpret_cast<float4*>(S + g * MG + 4 * h) =
+          make_float4((m >> (4 * h) & 1u) ? wv[4 * h] : 0.f, (m >> (4 * h + 1) & 1u) ? wv[4 * h + 1] : 0.f,
+                      (m >> (4 * h + 2) & 1u) ? wv[4 * h + 2] : 0.f, (m >> (4 * h + 3) & 1u) ? wv[4 * h + 3] : 0.f);
   }
 }
 
@@ -248,9 +261,13 @@ __global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const 
     for (int i = 0; i < nflag; ++i) nf += failflag[i] ? 1 : 0;
     if (st) { st->loss_B = sc[SC_LOSS]; st->tau_B = (float)tau; st->chol_failed += nf; }
     if (nf) atomicAdd(&status[ST_CHOL_FAILS], nf);
-  } else if (stage == 3) {
+  } else if (stage == 3 || stage == 6) {
     const double nrm = sc[SC_NRM_S], q = sc[SC_Q_S];
-    const double tau = (q > 0.0) ? nrm / q : 0.0;
+    double tau = (q > 0.0) ? nrm / q : 0.0;
+    if (stage == 6) {  // the paper's step 1 / beta_W' (Eq. lrWprime): the move is Gamma_M / (|A^T A|_F |B H_w B^T|_F)
+      const double bh = sqrt(sc[SC_BETA_A]) * sqrt(sc[SC_BETA_K]);
+      tau = (bh > 0.0) ? 1.0 / bh : 0.0;
+    }
     sc[SC_TAU_S] = tau;
     sc[SC_LOSS] -= 2.0 * tau * nrm - tau * tau * q;
     if (st) { st->loss_S = sc[SC_LOSS]; st->tau_S = (float)tau; }
@@ -284,14 +301,19 @@ __global__ void __launch_bounds__(NT) split_hilo_kernel(const float4* __restrict
   }
 }
 
-// X [rows, cols] (ld ldx) -> Thi/Tlo [cols, rows] (ld ldt): transposed and split.
-__global__ void transpose_split_kernel(const float* __restrict__ X, int64_t ldx, int64_t rows, int64_t cols,
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// X [rows, cols] (ld ldx) -> Thi/Tlo [cols, rows] (ld ldt): transposed and split.  bf16 input is exact in
+// tf32, so its low part is zero and Tlo is not needed.
+template <typename TIn>
+__global__ void transpose_split_kernel(const TIn* __restrict__ X, int64_t ldx, int64_t rows, int64_t cols,
                                        float* __restrict__ Thi, float* __restrict__ Tlo, int64_t ldt) {
   __shared__ float tile[32][33];
   const int64_t c0 = (int64_t)blockIdx.x * 32, r0 = (int64_t)blockIdx.y * 32;
   for (int j = threadIdx.y; j < 32; j += blockDim.y) {
     int64_t r = r0 + j, cidx = c0 + threadIdx.x;
-    tile[j][threadIdx.x] = (r < rows && cidx < cols) ? X[r * ldx + cidx] : 0.f;
+    tile[j][threadIdx.x] = (r < rows && cidx < cols) ? to_f32(X[r * ldx + cidx]) : 0.f;
   }
   __syncthreads();
   for (int j = threadIdx.y; j < 32; j += blockDim.y) {
@@ -302,6 +324,25 @@ __global__ void transpose_split_kernel(const float* __restrict__ X, int64_t ldx,
       Thi[cidx * ldt + r] = h;
       if (Tlo) Tlo[cidx * ldt + r] = v - h;
     }
+  }
+}
+
+// bf16 <-> fp32 with an optional per-column scale (the denormalisation of the deployment form)
+__global__ void __launch_bounds__(NT) bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ in,
+                                                         const float* __restrict__ cs, float* __restrict__ out,
+                                                         int64_t n, int64_t cols) {
+  for (int64_t i = (int64_t)blockIdx.x * NT + threadIdx.x; i < n; i += (int64_t)gridDim.x * NT) {
+    float v = __bfloat162float(in[i]);
+    if (cs) v *= cs[i % cols];
+    out[i] = v;
+  }
+}
+__global__ void __launch_bounds__(NT) f32_to_bf16_kernel(const float* __restrict__ in, const float* __restrict__ cs,
+                                                         __nv_bfloat16* __restrict__ out, int64_t n, int64_t cols) {
+  for (int64_t i = (int64_t)blockIdx.x * NT + threadIdx.x; i < n; i += (int64_t)gridDim.x * NT) {
+    float v = in[i];
+    if (cs) v *= cs[i % cols];
+    out[i] = __float2bfloat16_rn(v);
   }
 }
 
@@ -352,7 +393,8 @@ void launch_transpose_blocks(armor_ctx* c, const float* in, float* out, int nb, 
 }
 
 void launch_masked_copy(armor_ctx* c, const float* Gam, const uint8_t* M, float* out, int slot_norm, cudaStream_t s) {
-  masked_copy_kernel<<<ARMOR_DOT_BLOCKS, NT, 0, s>>>((const float4*)Gam, M, (float4*)out, c->wn / 4, c->partials);
+  masked_copy_kernel<<<ARMOR_DOT_BLOCKS, NT, 0, s>>>((const float4*)Gam, M, (float4*)out, c->wn / 4,
+                                                    c->cfg.m_group / 4, c->partials);
   reduce_final_kernel<<<1, NT, 0, s>>>(c->partials, ARMOR_DOT_BLOCKS, c->sc + slot_norm);
   c->launches += 2;
 }
@@ -376,8 +418,13 @@ void launch_init(armor_ctx* c, const float* W, const float* H, float* Wbar, floa
     copy_kernel<<<grid_for(c->wn / 4), NT, 0, s>>>((const float4*)W, (float4*)Wbar, c->wn / 4);
     c->launches++;
   }
-  init_core_kernel<<<grid_for(c->wn / 4), NT, 0, s>>>((const float4*)Wbar, H, cols, (float4*)S, M, c->wn / 4,
-                                                     (int)(cols / 4));
+  const int mg = c->cfg.m_group;
+  if (mg == 8)
+    init_core_kernel<8><<<grid_for(c->wn / 8), NT, 0, s>>>(Wbar, H, cols, S, M, c->wn / 8, (int)(cols / 8),
+                                                          c->cfg.n_keep);
+  else
+    init_core_kernel<4><<<grid_for(c->wn / 4), NT, 0, s>>>(Wbar, H, cols, S, M, c->wn / 4, (int)(cols / 4),
+                                                          c->cfg.n_keep);
   identity_blocks_kernel<<<c->nbo, NT, 0, s>>>(A, c->db);
   identity_blocks_kernel<<<c->nbi, NT, 0, s>>>(B, c->db);
   c->launches += 3;
@@ -400,9 +447,27 @@ void launch_split_hilo(armor_ctx* c, const float* in, float* hi, float* lo, int6
   c->launches++;
 }
 
-void launch_transpose_split(armor_ctx* c, const float* X, int64_t ldx, int64_t rows, int64_t cols, float* Thi,
-                            float* Tlo, int64_t ldt, cudaStream_t s) {
+void launch_transpose_split(armor_ctx* c, const void* X, int x_dtype, int64_t ldx, int64_t rows, int64_t cols,
+                            float* Thi, float* Tlo, int64_t ldt, cudaStream_t s) {
   dim3 grid((unsigned)((cols + 31) / 32), (unsigned)((ldt + 31) / 32));
-  transpose_split_kernel<<<grid, dim3(32, 8), 0, s>>>(X, ldx, rows, cols, Thi, Tlo, ldt);
+  if (x_dtype == ARMOR_DTYPE_BF16)
+    transpose_split_kernel<<<grid, dim3(32, 8), 0, s>>>(static_cast<const __nv_bfloat16*>(X), ldx, rows, cols, Thi,
+                                                       (float*)nullptr, ldt);
+  else
+    transpose_split_kernel<<<grid, dim3(32, 8), 0, s>>>(static_cast<const float*>(X), ldx, rows, cols, Thi, Tlo, ldt);
+  c->launches++;
+}
+
+void launch_bf16_to_f32(armor_ctx* c, const void* in, const float* colscale, float* out, int64_t rows, int64_t cols,
+                        cudaStream_t s) {
+  bf16_to_f32_kernel<<<grid_for(rows * cols), NT, 0, s>>>(static_cast<const __nv_bfloat16*>(in), colscale, out,
+                                                         rows * cols, cols);
+  c->launches++;
+}
+
+void launch_f32_to_bf16(armor_ctx* c, const float* in, const float* colscale, void* out, int64_t rows, int64_t cols,
+                        cudaStream_t s) {
+  f32_to_bf16_kernel<<<grid_for(rows * cols), NT, 0, s>>>(in, colscale, static_cast<__nv_bfloat16*>(out), rows * cols,
+                                                         cols);
   c->launches++;
 }

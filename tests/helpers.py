@@ -33,19 +33,19 @@ def host(t):
     return t.detach().cpu().numpy()
 
 
-def load_state(st, A, B, S, M):
+def load_state(st, A, B, S, M, m_group=4):
     """Copies an oracle state (fp64 arrays, boolean mask) into the GPU state tensors."""
     st.A.copy_(dev(A))
     st.B.copy_(dev(B))
     st.S.copy_(dev(S))
-    st.M.copy_(torch.from_numpy(O.pack_mask(M)).to(DEV))
+    st.M.copy_(torch.from_numpy(O.pack_mask(M, m_group)).to(DEV))
 
 
-def mask_block_diffs(Mg_packed, M_oracle, d_block):
+def mask_block_diffs(Mg_packed, M_oracle, d_block, m_group=4):
     """Set of (i, j) blocks in which the GPU mask differs from the oracle's."""
-    diff = Mg_packed != O.pack_mask(M_oracle)
+    diff = Mg_packed != O.pack_mask(M_oracle, m_group)
     rows, cgs = np.nonzero(diff)
-    return {(int(r) // d_block, int(c) * 4 // d_block) for r, c in zip(rows, cgs)}
+    return {(int(r) // d_block, int(c) * m_group // d_block) for r, c in zip(rows, cgs)}
 
 
 def excused_blocks(info, margin):

@@ -136,20 +136,22 @@ def test_proxy_loss_matches_oracle(prec, h_mode, mid_data):
 
 
 # ------------------------------------------------------------------------- teacher-forced steps
-def run_teacher_forced(cfg, W, H32, prec, h_mode, n_steps, select=Bd.SELECT_L1_RANDOM):
-    ctx = make(cfg, prec, h_mode, select_mode=select)
+def run_teacher_forced(cfg, W, H32, prec, h_mode, n_steps, select=Bd.SELECT_L1_RANDOM, n_keep=2, m_group=4,
+                       s_step=Bd.S_EXACT, tol_scale=1.0):
+    ctx = make(cfg, prec, h_mode, select_mode=select, n_keep=n_keep, m_group=m_group, s_step=s_step)
     Hd = dev(H32)
     st = ctx.init(dev(W), Hd)
-    oc = O.OracleConfig(cfg.d_block, h_mode=h_mode, seed=cfg.seed, select_mode=select)
+    oc = O.OracleConfig(cfg.d_block, h_mode=h_mode, seed=cfg.seed, select_mode=select, n_keep=n_keep,
+                        m_group=m_group, s_step=s_step)
     Hq = H32.astype(np.float64)
     Hw = O.weighting(Hq, h_mode)
     Wn = W.astype(np.float64)
     A, B, S, M = O.init(Wn, Hq, oc)
-    tol = TOL[prec]
+    tol = {k: v * tol_scale for k, v in TOL[prec].items()}
     n_excused = 0
     worst = dict(A=0.0, B=0.0, S=0.0, loss=0.0)
     for t in range(n_steps):
-        load_state(st, A, B, S, M)                 # the GPU starts every step from the oracle's state
+        load_state(st, A, B, S, M, m_group)        # the GPU starts every step from the oracle's state
         stats = ctx.bcd_step(st, Hd, t, 1)
         sg = ctx.read_stats(stats)[0]
         A, B, S, M, info = O.bcd_iteration(Wn, A, B, S, M, Hw, oc, t)
@@ -158,9 +160,10 @@ def run_teacher_forced(cfg, W, H32, prec, h_mode, n_steps, select=Bd.SELECT_L1_R
         for k_gpu, k_or in (("loss_start", "start"), ("loss_A", "A"), ("loss_B", "B"), ("loss_S", "S")):
             worst["loss"] = max(worst["loss"], abs(sg[k_gpu] - info.loss[k_or]) / info.loss[k_or])
         assert abs(sg["tau_B"] - info.tau_B) <= 10 * tol["B"] * abs(info.tau_B) + 1e-6
+        assert abs(sg["tau_S"] - info.tau_S) <= 10 * tol["S"] * abs(info.tau_S) + 1e-12
         assert sg["chol_failed"] == info.chol_failed == 0
         # masks: identical outside blocks whose decision margin is below the threshold
-        diff = mask_block_diffs(host(st.M), M, cfg.d_block)
+        diff = mask_block_diffs(host(st.M), M, cfg.d_block, m_group)
         excused = excused_blocks(info, tol["margin"])
         guard_close = abs(info.delta_L_mask) <= tol["margin"] * info.loss["S"]
         if sg["mask_accepted"] != info.mask_accepted:
@@ -198,6 +201,42 @@ def test_teacher_forced_mid_config_d_block_128(prec, mid_data):
 def test_teacher_forced_greedy_selection(tiny_data):
     W, X, H32 = tiny_data
     run_teacher_forced(TINY, W, H32, Bd.PREC_FP32X3, Bd.H_FULL, 5, select=Bd.SELECT_L1_GREEDY)
+
+
+@pytest.mark.parametrize("h_mode", [Bd.H_FULL, Bd.H_DIAG])
+def test_teacher_forced_4_of_8_groups(h_mode, tiny_data):
+    """The 4:8 pattern: top-4 of 8 at the initialisation, 70 masks with 4 x 4 solves per selected group."""
+    W, X, H32 = tiny_data
+    ctx = make(TINY, Bd.PREC_SIMT, h_mode, n_keep=4, m_group=8)
+    st = ctx.init(dev(W), dev(H32))
+    _, _, S0, M0 = O.init(W.astype(np.float64), H32.astype(np.float64), O.OracleConfig(TINY.d_block, n_keep=4, m_group=8))
+    assert np.array_equal(host(st.M), O.pack_mask(M0, 8)) and np.array_equal(host(st.S), S0.astype(np.float32))
+    worst, n_excused = run_teacher_forced(TINY, W, H32, Bd.PREC_FP32X3, h_mode, 8, n_keep=4, m_group=8)
+    print(f"4:8 h_mode={h_mode}: worst rel err {worst}, groups differing under the margin: {n_excused}")
+    assert n_excused <= 2
+
+
+def test_teacher_forced_paper_step_size_for_the_core(tiny_data):
+    """s_step = BETA: the paper's 1/beta_W' step (Eq. lrWprime) instead of the exact line search."""
+    W, X, H32 = tiny_data
+    for h_mode in (Bd.H_FULL, Bd.H_DIAG):
+        run_teacher_forced(TINY, W, H32, Bd.PREC_FP32X3, h_mode, 4, s_step=Bd.S_BETA)
+
+
+BIG_BLOCK = TINY.with_(name="db256", d_out=512, d_in=768, d_block=256, n_tokens=5000, chunk_rows=2048, seed=21)
+
+
+@pytest.mark.parametrize("prec", [Bd.PREC_FP32X3, Bd.PREC_TF32], ids=PNAME.get)
+def test_teacher_forced_d_block_256(prec):
+    """d_block = 256: block solves split over four CTAs, wrapper blocks of two tiles per side."""
+    W = inputs.make_weight(BIG_BLOCK)
+    X = inputs.make_activations(BIG_BLOCK)
+    H32 = O.gram(X).astype(np.float32)
+    # one-pass tf32: the 256 x 256 block systems are worse conditioned than the 128 x 128 ones the tf32
+    # tolerance was stated for and pass more of the operand rounding on to A and B (measured 4e-2)
+    worst, n_excused = run_teacher_forced(BIG_BLOCK, W, H32, prec, Bd.H_FULL, 3,
+                                          tol_scale=4.0 if prec == Bd.PREC_TF32 else 1.0)
+    print(f"d_block 256 {PNAME[prec]}: worst rel err {worst}, groups differing under the margin: {n_excused}")
 
 
 @pytest.mark.parametrize("phase", [Bd.PHASE_A, Bd.PHASE_B, Bd.PHASE_S, Bd.PHASE_MASK])
@@ -348,3 +387,37 @@ def test_apply_zero_tokens_and_more_tokens_than_rows(mid_data):
     y = host(ctx.apply(st, dev(x)))
     A, B, S = (host(t).astype(np.float64) for t in (st.A, st.B, st.S))
     assert rel(y, O.apply(A, B, S, x)) < 1e-5
+
+
+# ------------------------------------------------------------------------------------------ bf16 inputs
+@pytest.mark.parametrize("prec", [Bd.PREC_FP32X3, Bd.PREC_TF32], ids=PNAME.get)
+def test_gram_of_bf16_activations_is_exact_up_to_accumulation(prec, mid_data):
+    W, X, _ = mid_data
+    ctx = make(MID, prec)
+    Xb = dev(X).to(torch.bfloat16)
+    H = ctx.new_gram()
+    for lo, hi in ((0, 2048), (2048, 2048 + 37), (2048 + 37, MID.n_tokens)):
+        ctx.gram(Xb[lo:hi], H)
+    torch.cuda.synchronize()
+    Ho = O.gram(Xb.float().cpu().numpy())          # the same bf16-rounded values, fp64 products
+    # exact products; what remains is the fp32 accumulation of the tensor-core pipe
+    assert rel(host(H), Ho) < (2e-5 if prec == Bd.PREC_FP32X3 else 1e-4)
+    assert ctx.device_status()[:4] == [0, 0, 0, 0]
+
+
+def test_apply_with_bf16_activations(mid_data):
+    W, X, H32 = mid_data
+    ctx = make(MID, Bd.PREC_FP32X3, normalize=1)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    ctx.bcd_step(st, Hd, 0, 1, want_stats=False)
+    xb = dev(inputs.make_tokens(MID, 300)).to(torch.bfloat16)
+    A, B, S = (host(t).astype(np.float64) for t in (st.A, st.B, st.S))
+    xr = xb.float().cpu().numpy()
+    for den in (False, True):
+        y = ctx.apply(st, xb, denormalize=den)
+        assert y.dtype == torch.bfloat16
+        r1, r2 = (host(st.r1).astype(np.float64), host(st.r2).astype(np.float64)) if den else (None, None)
+        yo = O.apply(A, B, S, xr, r1, r2)
+        # one rounding to bf16 (2^-9 relative per element) on the way out
+        assert rel(y.float().cpu().numpy(), yo) < 3e-3

@@ -38,14 +38,18 @@ def test_config_validation(lib):
     cases = [
         (Bd.make_config(256, 250, 32), 2),             # d_block does not divide d_in
         (Bd.make_config(256, 256, 30), 2),             # ... nor d_out; not a multiple of m_group either
-        (Bd.make_config(256, 256, 32, n_keep=4, m_group=8), 7),
-        (Bd.make_config(512, 512, 256), 7),            # d_block > 128
+        (Bd.make_config(256, 256, 32, n_keep=3, m_group=8), 7),      # only 2:4 and 4:8
+        (Bd.make_config(256, 256, 32, n_keep=2, m_group=8), 7),
+        (Bd.make_config(1024, 1024, 512), 7),          # d_block > 256
+        (Bd.make_config(576, 576, 144), 7),            # above 128 the block size must be a multiple of 32
         (Bd.make_config(256, 256, 32, h_mode=5), 1),
         (Bd.make_config(256, 256, 32, ridge=-1.0), 1),
         (Bd.make_config(0, 256, 32), 2),
         (Bd.make_config(192, 192, 32, precision=Bd.PREC_TF32), 7),   # tensor-core tiles need multiples of 128
-        (Bd.make_config(256, 256, 32, s_step=Bd.S_BETA), 7),
     ]
+    for good in (Bd.make_config(256, 256, 32, n_keep=4, m_group=8), Bd.make_config(512, 512, 256),
+                 Bd.make_config(256, 256, 32, s_step=Bd.S_BETA)):
+        assert Bd.armor_workspace_bytes(good) > 0
     for cfg, code in cases:
         n = C.c_size_t(0)
         assert lib.armor_workspace_bytes(C.byref(cfg), C.byref(n)) == code

@@ -347,6 +347,63 @@ def test_group_solve_matches_brute_force_least_squares(h_mode):
             assert np.isclose(Lfrozen - red / alpha, Lbest, rtol=1e-9, atol=1e-12 * L0)
 
 
+@pytest.mark.parametrize("h_mode", [O.FULL, O.DIAG])
+def test_group_solve_4_of_8_matches_brute_force_least_squares(h_mode):
+    """The 4:8 pattern: for a group and each of the 70 masks the four free values fitted by generic least
+    squares on the full loss agree with the closed form, and the mask step's choice is the best of the 70."""
+    cfg, W, X = tiny(d_out=8, d_in=16, db=8, n=60)
+    H = O.gram(X)
+    Hw = O.weighting(H, h_mode)
+    R = X.T if h_mode == O.FULL else np.diag(np.sqrt(np.diag(H)))
+    oc = O.OracleConfig(8, n_keep=4, m_group=8, h_mode=h_mode, select_mode=O.L1_GREEDY, phases=O.PH_MASK)
+    A, B, S, M = rand_state(W, H, oc, np.random.default_rng(12), scale=0.3)
+    assert np.all(M.reshape(8, -1, 8).sum(axis=2) == 4)
+    Ad, Bd = O.bd_dense(A), O.bd_dense(B)
+    Gamma = O.core_gradient(W, A, B, S, Hw)
+    r, c = 5, 1
+    cols = np.arange(8 * c, 8 * c + 8)
+    S0 = S.copy()
+    S0[r, cols] = 0.0
+    dW = W - Ad @ S0 @ Bd
+    Lfrozen = np.linalg.norm(dW @ R) ** 2
+    a = Ad[:, r]
+    alpha = a @ a
+    Kc = Bd[cols] @ Hw @ Bd[cols].T
+    z = Gamma[r, cols] + alpha * Kc @ S[r, cols]
+    combos = list(itertools.combinations(range(8), 4))
+    assert len(combos) == 70
+    for keep in combos[::7] + [combos[-1]]:
+        ix = np.array(keep)
+        Dm = np.stack([(np.outer(a, Bd[cols[p]]) @ R).reshape(-1) for p in keep], axis=1)
+        sol, *_ = np.linalg.lstsq(Dm, (dW @ R).reshape(-1), rcond=None)
+        Lbest = np.linalg.norm((dW @ R).reshape(-1) - Dm @ sol) ** 2
+        w, red = O.pinv_solve(Kc[np.ix_(ix, ix)], z[ix])
+        assert np.allclose(w / alpha, sol, rtol=1e-6, atol=1e-10)
+        assert np.isclose(Lfrozen - red / alpha, Lbest, rtol=1e-8)
+    # the whole mask step with one block: greedy selection, best of the 70 masks, loss cannot rise
+    info = O.IterInfo()
+    L0 = O.proxy_loss(W, A, B, S, Hw)
+    S1, M1 = O.mask_step(W, A, B, S, M, Hw, oc, 0, info)
+    assert np.all(M1.reshape(8, -1, 8).sum(axis=2) == 4) and np.all(S1[~M1] == 0.0)
+    assert O.proxy_loss(W, A, B, S1, Hw) <= L0 * (1 + 1e-12)
+    for j in range(2):
+        g = int(info.selected[0, j])
+        rr, cc = divmod(g, 2)
+        cs = np.arange(8 * cc, 8 * cc + 8)
+        S0 = S.copy()
+        S0[rr, cs] = 0.0
+        dWj = (W - Ad @ S0 @ Bd) @ R
+        best = (np.inf, None)
+        for keep in combos:
+            Dm = np.stack([(np.outer(Ad[:, rr], Bd[cs[p]]) @ R).reshape(-1) for p in keep], axis=1)
+            sol, *_ = np.linalg.lstsq(Dm, dWj.reshape(-1), rcond=None)
+            Lm = np.linalg.norm(dWj.reshape(-1) - Dm @ sol) ** 2
+            if Lm < best[0] * (1 - 1e-12):
+                best = (Lm, keep)
+        if info.mask_accepted and info.mask_margin[0, j] > 1e-9:
+            assert tuple(np.nonzero(M1[rr, cs])[0]) == best[1]
+
+
 def test_pinv_solve_singular_cases():
     v = np.array([1.0, 2.0])
     K = np.outer(v, v)
@@ -523,6 +580,23 @@ def test_theorem_1_monotone_and_below_init(h_mode, select):
         prev = seq[-1]
     assert prev < L0            # wrappers strictly help on this input
     assert np.all(M.reshape(32, -1, 4).sum(axis=2) == 2) and np.all(S[~M] == 0)
+
+
+def test_theorem_1_with_4_of_8_groups():
+    cfg, W, X = tiny(d_out=32, d_in=32, db=8, n=128)
+    H = O.gram(X)
+    oc = O.OracleConfig(8, n_keep=4, m_group=8, seed=3)
+    L0 = O.proxy_loss(W, *O.init(W, H, oc)[:3], H)
+    (A, B, S, M), infos = O.run(W, H, oc, 6)
+    prev = L0
+    for info in infos:
+        seq = [info.loss[k] for k in ("start", "A", "B", "S", "mask")]
+        assert np.isclose(seq[0], prev, rtol=1e-12)
+        for a, b in zip(seq, seq[1:]):
+            assert b <= a * (1 + 1e-10)
+        prev = seq[-1]
+    assert prev < L0
+    assert np.all(M.reshape(32, -1, 8).sum(axis=2) == 4) and np.all(S[~M] == 0)
 
 
 def test_resume_is_bitwise():
