@@ -129,6 +129,13 @@ void bd_right(armor_ctx* c, const float* in, const float* Bblk, bool transB, flo
 void bd_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, float* out, int64_t rows,
              int64_t cols, float alpha, const float* add, float beta, cudaStream_t s);
 
+// the same two products on the tensor cores (block_tcgen05.cu); d_block must be a multiple of 128
+bool tc_block_ok(const armor_ctx* c, int64_t rows, int64_t cols);
+armor_status tc_bd_right(armor_ctx* c, const float* in, const float* Bblk, bool transB, float* out, int64_t rows,
+                         int64_t cols, float alpha, const float* add, float beta, cudaStream_t s);
+armor_status tc_bd_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, float* out, int64_t rows,
+                        int64_t cols, float alpha, const float* add, float beta, cudaStream_t s);
+
 // out = in * H_w (FULL: dense GEMM by cfg.precision; DIAG: column scale) with up to two
 // fused dot products <out, d1> -> sc[slot1], <out, d2> -> sc[slot2] (slot < 0: none).
 armor_status rmul_H(armor_ctx* c, const float* in, const float* H, float* out, int64_t rows,

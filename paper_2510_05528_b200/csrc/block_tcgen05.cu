@@ -1,0 +1,326 @@
+// Batched 128 x 128 x K products on the tensor cores for the block-diagonal wrappers (Section 3.1 of the
+// paper: A and B are block diagonal, so A.Y and Y.B are one small dense product per d_block x d_block tile
+// of the W-shaped operand).  Per tile the product has only 2*d_block flops per element moved, so these passes
+// are bound by HBM once the arithmetic runs on the tensor cores.
+//
+//   C_tile = alpha * sum_k Aop[m][k] * Bop[n][k] (+ beta * D_tile)
+//
+// Both operands are plain fp32 in global memory.  Either may be K-major (k contiguous) or MN-major (m or n
+// contiguous); tcgen05 reads both from swizzled shared memory (MN-major 32-bit operands in the 128-byte swizzle
+// with 32-byte atoms, which TMA writes directly), so no transposed copies are made.
+// fp32-grade accuracy comes from splitting every operand chunk, in shared memory, into a tf32-exact high part
+// and an fp32 low part and issuing three MMAs (lo*hi + hi*lo + hi*hi) into one fp32 accumulator.
+//
+// Persistent kernel, 320 threads:
+//   warp 0    : TMA producer (raw fp32 chunks of 32 along K; MN-major chunks as four 32 x 32 boxes)
+//   warp 1    : MMA issuer   (tcgen05.mma kind::tf32, 128 x 128 x 8, two accumulators of 128 TMEM columns)
+//   warps 2-5 : splitter     (raw chunk -> high part in place, low part next to it, proxy fence)
+//   warps 6-9 : epilogue     (tcgen05.ld, 32 x 32 chunks turned through shared memory, alpha / beta, stores)
+// Every wait is bounded; a wait that runs out raises a status word and the CTA leaves through the common
+// exit that frees its tensor memory.
+#include "tc_common.cuh"
+
+namespace {
+
+using namespace tc;
+
+constexpr int TILE = 128, BK = 32;
+constexpr int NTHREADS = 320;
+constexpr int STAGES = 3;
+constexpr int OP_BYTES = TILE * BK * 4;           // 16 KiB: one operand chunk
+constexpr int STAGE_BYTES = 4 * OP_BYTES;         // A hi, A lo, B hi, B lo
+constexpr uint32_t TMEM_COLS = 256;               // two accumulators of 128 columns
+constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 4 * 32 * 33 * sizeof(float) + 1024;
+
+struct OpCoord {
+  int mn_major;                     // 0: K-major, 1: MN-major
+  int x_b, x_t, x_k;                // TMA x (inner) coordinate = x_b * batch + x_t * tile + x_k * chunk
+  int y_b, y_t, y_k;                // TMA y (outer) coordinate likewise
+};
+
+struct BParams {
+  OpCoord a, b;
+  float* C; const float* D;
+  int64_t ldc, ldd;
+  int64_t c_rows, c_cols;           // extent of C (stores are guarded)
+  int64_t r_b, c_b;                 // tile origin: row = r_b * batch + 128 * tm, column = c_b * batch + 128 * tn
+  int m_tiles, n_tiles, batch, k_chunks;
+  float alpha, beta;
+  int32_t* status;
+};
+
+__device__ __forceinline__ void load_operand(uint32_t dst, const CUtensorMap* map, const OpCoord& o, int b, int t, int kc,
+                                             uint32_t bar) {
+  const int x = o.x_b * b + o.x_t * t + o.x_k * kc;
+  const int y = o.y_b * b + o.y_t * t + o.y_k * kc;
+  if (o.mn_major) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) tma_load_2d(dst + q * 4096, map, x + 32 * q, y, bar);
+  } else {
+    tma_load_2d(dst, map, x, y, bar);
+  }
+}
+
+__device__ __forceinline__ uint64_t operand_desc(uint32_t base, int mn_major, int kstep) {
+  // K-major: 8 columns of K are 32 bytes further along the 128-byte row.
+  // MN-major: 8 k-rows are two groups of 4 k-rows (512 bytes each); 32 more elements along M / N are the next
+  // 4 KiB box.
+  return mn_major ? smem_desc_mn_sw128_32b(base + kstep * 1024, 4096, 512) : smem_desc_sw128(base + kstep * 32, 16, 1024);
+}
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const BParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ __align__(8) uint64_t bars[3 * STAGES + 4];
+  __shared__ uint32_t tmem_base_holder;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t full0 = smem_u32(&bars[0]), split0 = smem_u32(&bars[STAGES]), empty0 = smem_u32(&bars[2 * STAGES]);
+  const uint32_t tfull0 = smem_u32(&bars[3 * STAGES]), tempty0 = smem_u32(&bars[3 * STAGES + 2]);
+  const int n_items = p.batch * p.m_tiles * p.n_tiles;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full0 + 8 * s, 1);
+      mbar_init(split0 + 8 * s, 4);
+      mbar_init(empty0 + 8 * s, 1);
+    }
+    for (int s = 0; s < 2; ++s) { mbar_init(tfull0 + 8 * s, 1); mbar_init(tempty0 + 8 * s, 4); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_holder;
+  volatile int* abortp = &abort_flag;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0; long long issued = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        const int tn = item % p.n_tiles, tm = (item / p.n_tiles) % p.m_tiles, b = item / (p.n_tiles * p.m_tiles);
+        for (int kc = 0; kc < p.k_chunks; ++kc) {
+          if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abortp, p.status)) { ok = false; break; }
+          const uint32_t fb = full0 + 8 * stage;
+          mbar_expect_tx(fb, 2 * OP_BYTES);
+          const uint32_t dst = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+          load_operand(dst, &mapA, p.a, b, tm, kc, fb);
+          load_operand(dst + 2 * OP_BYTES, &mapB, p.b, b, tn, kc, fb);
+          ++issued;
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) {
+        // leave no bulk copy in flight: wait (bounded) for the stages armed most recently
+        for (int back = 1; back <= STAGES && back <= issued; ++back) {
+          int s = stage - back; uint32_t ph = phase;
+          if (s < 0) { s += STAGES; ph ^= 1; }
+          const long long t0 = clock64();
+          while (!mbar_try(full0 + 8 * s, ph) && clock64() - t0 < 20000000ll) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc_tf32_mn(TILE, TILE, p.a.mn_major, p.b.mn_major);
+      int stage = 0; uint32_t phase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++local) {
+        const int as = local & 1;
+        const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
+        if (!mbar_wait(tempty0 + 8 * as, aphase ^ 1, abortp, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tacc = tmem_base + (uint32_t)(as * TILE);
+        for (int kc = 0; kc < p.k_chunks; ++kc) {
+          if (!mbar_wait(split0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+          const uint32_t sa_lo = sa + OP_BYTES, sb = sa + 2 * OP_BYTES, sb_lo = sa + 3 * OP_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 8; ++k) {
+            const uint64_t da = operand_desc(sa, p.a.mn_major, k), dal = operand_desc(sa_lo, p.a.mn_major, k);
+            const uint64_t dbm = operand_desc(sb, p.b.mn_major, k), dbl = operand_desc(sb_lo, p.b.mn_major, k);
+            umma_tf32(tacc, dal, dbm, idesc, (uint32_t)((kc > 0) | (k != 0)));
+            umma_tf32(tacc, da, dbl, idesc, 1);
+            umma_tf32(tacc, da, dbm, idesc, 1);
+          }
+          umma_commit(empty0 + 8 * stage);   // frees the stage once these MMAs have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (ok) umma_commit(tfull0 + 8 * as);
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------------------ splitter warps
+    const int t = threadIdx.x - 64;   // 0..127
+    int stage = 0; uint32_t phase = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+      for (int kc = 0; kc < p.k_chunks; ++kc) {
+        if (!mbar_wait(full0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
+        float4* base = reinterpret_cast<float4*>(smem + (size_t)stage * STAGE_BYTES);
+#pragma unroll
+        for (int op = 0; op < 2; ++op) {
+          float4* hi = base + op * (2 * OP_BYTES / 16);
+          float4* lo = hi + OP_BYTES / 16;
+#pragma unroll
+          for (int e = 0; e < OP_BYTES / 16 / 128; ++e) {
+            const int idx = t + e * 128;
+            const float4 v = hi[idx];
+            float4 h;
+            h.x = __uint_as_float(__float_as_uint(v.x) & 0xffffe000u);
+            h.y = __uint_as_float(__float_as_uint(v.y) & 0xffffe000u);
+            h.z = __uint_as_float(__float_as_uint(v.z) & 0xffffe000u);
+            h.w = __uint_as_float(__float_as_uint(v.w) & 0xffffe000u);
+            hi[idx] = h;
+            lo[idx] = make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w);
+          }
+        }
+        // make the generic-proxy writes visible to the tensor-core (async proxy) reads
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(split0 + 8 * stage);
+        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue warps
+    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    int local = 0;
+    bool ok = true;
+    float* tilebuf = reinterpret_cast<float*>(smem + (size_t)STAGES * STAGE_BYTES) + q * (32 * 33);
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++local) {
+      const int tn = item % p.n_tiles, tm = (item / p.n_tiles) % p.m_tiles, b = item / (p.n_tiles * p.m_tiles);
+      const int as = local & 1;
+      const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
+      if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
+      tc_fence_after();
+      const int64_t row_base = p.r_b * b + (int64_t)tm * TILE + q * 32;
+      const int64_t col_tile = p.c_b * b + (int64_t)tn * TILE;
+#pragma unroll 1
+      for (int ch = 0; ch < TILE / 32; ++ch) {
+        uint32_t r[32];
+        tmem_ld32(tmem_base + (uint32_t)(as * TILE + ch * 32) + ((uint32_t)(q * 32) << 16), r);
+        const int64_t col0 = col_tile + ch * 32;
+        if (col0 >= p.c_cols || row_base >= p.c_rows) continue;   // warp-uniform
+#pragma unroll
+        for (int cidx = 0; cidx < 32; ++cidx) tilebuf[lane * 33 + cidx] = __uint_as_float(r[cidx]);
+        __syncwarp();
+        const int64_t col = col0 + lane;
+        const bool col_ok = col < p.c_cols;
+#pragma unroll 1
+        for (int r0 = 0; r0 < 32; r0 += 8) {
+          float x[8], d[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int64_t grow = row_base + r0 + j;
+            x[j] = tilebuf[(r0 + j) * 33 + lane];
+            d[j] = (p.D && col_ok && grow < p.c_rows) ? p.D[grow * p.ldd + col] : 0.f;
+          }
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int64_t grow = row_base + r0 + j;
+            if (col_ok && grow < p.c_rows) p.C[grow * p.ldc + col] = fmaf(p.beta, d[j], p.alpha * x[j]);
+          }
+        }
+        __syncwarp();
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty0 + 8 * as);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+struct HostOp {
+  const float* base; int64_t inner, outer, ld;   // global 2-D view [outer][inner]
+  OpCoord c;
+};
+
+armor_status launch(armor_ctx* c, const HostOp& A, const HostOp& B, BParams p, cudaStream_t s) {
+  CUtensorMap mA, mB;
+  if (!make_map_2d(&mA, A.base, A.inner, A.outer, A.ld, 32, A.c.mn_major ? 32 : TILE, A.c.mn_major != 0)) return ARMOR_ERR_CUDA;
+  if (!make_map_2d(&mB, B.base, B.inner, B.outer, B.ld, 32, B.c.mn_major ? 32 : TILE, B.c.mn_major != 0)) return ARMOR_ERR_CUDA;
+  p.a = A.c; p.b = B.c;
+  p.status = c->status;
+  static bool attr = false;
+  if (!attr) {
+    if (cudaFuncSetAttribute(tc_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)
+      return ARMOR_ERR_CUDA;
+    attr = true;
+  }
+  static int n_sm = 0;
+  if (!n_sm) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ARMOR_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ARMOR_ERR_CUDA;
+  }
+  const int n_items = p.batch * p.m_tiles * p.n_tiles;
+  const int grid = n_items < n_sm ? n_items : n_sm;
+  tc_block_kernel<<<grid, NTHREADS, SMEM_BYTES, s>>>(mA, mB, p);
+  c->launches++;
+  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+}
+
+inline bool ptr_ok(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15) == 0; }
+
+}  // namespace
+
+bool tc_block_ok(const armor_ctx* c, int64_t rows, int64_t cols) {
+  return c->cfg.precision != ARMOR_PREC_SIMT && c->db % TILE == 0 && rows > 0 && cols % 4 == 0;
+}
+
+// out[:, j-th block] = alpha * in[:, j-th block] * Q_j (+ beta * add[:, j-th block]),  Q_j = Bblk[j] or its transpose
+armor_status tc_bd_right(armor_ctx* c, const float* in, const float* Bblk, bool transB, float* out, int64_t rows,
+                         int64_t cols, float alpha, const float* add, float beta, cudaStream_t s) {
+  const int db = c->db;
+  const int nb = (int)(cols / db);
+  if (!ptr_ok(in) || !ptr_ok(Bblk) || !ptr_ok(out)) return ARMOR_ERR_UNSUPPORTED;
+  HostOp A{in, cols, rows, cols, {0, db, 0, BK, 0, TILE, 0}};
+  HostOp B{Bblk, db, (int64_t)nb * db, db, {}};
+  if (transB) B.c = {0, 0, 0, BK, db, TILE, 0};         // Bop[n][k] = B_j[n][k]: K-major
+  else        B.c = {1, 0, TILE, 0, db, 0, BK};         // Bop[n][k] = B_j[k][n]: N-major
+  BParams p{};
+  p.C = out; p.D = add; p.ldc = cols; p.ldd = cols; p.c_rows = rows; p.c_cols = cols;
+  p.r_b = 0; p.c_b = db;
+  p.m_tiles = (int)((rows + TILE - 1) / TILE); p.n_tiles = db / TILE; p.batch = nb; p.k_chunks = db / BK;
+  p.alpha = alpha; p.beta = add ? beta : 0.f;
+  return launch(c, A, B, p, s);
+}
+
+// out[i-th block, :] = alpha * P_i * in[i-th block, :] (+ beta * add[i-th block, :]),  P_i = Ablk[i] or its transpose
+armor_status tc_bd_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, float* out, int64_t rows,
+                        int64_t cols, float alpha, const float* add, float beta, cudaStream_t s) {
+  const int db = c->db;
+  const int nb = (int)(rows / db);
+  if (!ptr_ok(in) || !ptr_ok(Ablk) || !ptr_ok(out)) return ARMOR_ERR_UNSUPPORTED;
+  HostOp A{Ablk, db, (int64_t)nb * db, db, {}};
+  if (transA) A.c = {1, 0, TILE, 0, db, 0, BK};         // Aop[m][k] = A_i[k][m]: M-major
+  else        A.c = {0, 0, 0, BK, db, TILE, 0};         // Aop[m][k] = A_i[m][k]: K-major
+  HostOp B{in, cols, rows, cols, {1, 0, TILE, 0, db, 0, BK}};   // Bop[n][k] = in[i*db + k][n]: N-major
+  BParams p{};
+  p.C = out; p.D = add; p.ldc = cols; p.ldd = cols; p.c_rows = rows; p.c_cols = cols;
+  p.r_b = db; p.c_b = 0;
+  p.m_tiles = db / TILE; p.n_tiles = (int)((cols + TILE - 1) / TILE); p.batch = nb; p.k_chunks = db / BK;
+  p.alpha = alpha; p.beta = add ? beta : 0.f;
+  return launch(c, A, B, p, s);
+}

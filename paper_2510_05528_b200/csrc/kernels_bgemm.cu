@@ -301,8 +301,15 @@ void launch_bgemm(armor_ctx* c, const BGemm& g_in, cudaStream_t s) {
   c->launches++;
 }
 
+// 1: block-diagonal products on the tensor cores where the shape allows; 0: always the fp32 CUDA-core kernels
+static int g_tc_blocks = 0;
+extern "C" void armor_debug_set_tc_blocks(int on) { g_tc_blocks = on; }
+
 void bd_right(armor_ctx* c, const float* in, const float* Bblk, bool transB, float* out, int64_t rows,
               int64_t cols, float alpha, const float* add, float beta, cudaStream_t s) {
+  if (g_tc_blocks && tc_block_ok(c, rows, cols) &&
+      tc_bd_right(c, in, Bblk, transB, out, rows, cols, alpha, add, beta, s) == ARMOR_OK)
+    return;
   const int db = c->db;
   BGemm g{};
   g.A = in; g.sAb = db; g.sAm = cols; g.sAk = 1;
@@ -317,6 +324,9 @@ void bd_right(armor_ctx* c, const float* in, const float* Bblk, bool transB, flo
 
 void bd_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, float* out, int64_t rows,
              int64_t cols, float alpha, const float* add, float beta, cudaStream_t s) {
+  if (g_tc_blocks && tc_block_ok(c, rows, cols) &&
+      tc_bd_left(c, Ablk, transA, in, out, rows, cols, alpha, add, beta, s) == ARMOR_OK)
+    return;
   const int db = c->db;
   BGemm g{};
   g.A = Ablk; g.sAb = (int64_t)db * db;
@@ -327,4 +337,15 @@ void bd_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, floa
   g.M = db; g.N = (int)cols; g.K = db; g.batch = (int)(rows / db);
   g.alpha = alpha; g.beta = beta;
   launch_bgemm(c, g, s);
+}
+
+// Test hook: one block-diagonal product through whichever path is switched on.
+extern "C" int armor_debug_block_product(armor_ctx* c, int left, int trans, const float* blk, const float* in,
+                                         float* out, int64_t rows, int64_t cols, float alpha, const float* add,
+                                         float beta, void* stream) {
+  if (!c) return ARMOR_ERR_INVALID_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (left) bd_left(c, blk, trans != 0, in, out, rows, cols, alpha, add, beta, s);
+  else bd_right(c, in, blk, trans != 0, out, rows, cols, alpha, add, beta, s);
+  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
 }
