@@ -15,7 +15,8 @@
 //   warp 0    : TMA producer (raw fp32 chunks of 32 along K; MN-major chunks as four 32 x 32 boxes)
 //   warp 1    : MMA issuer   (tcgen05.mma kind::tf32, 128 x 128 x 8, two accumulators of 128 TMEM columns)
 //   warps 2-5 : splitter     (raw chunk -> high part in place, low part next to it, proxy fence)
-//   warps 6-9 : epilogue     (tcgen05.ld, 32 x 32 chunks turned through shared memory, alpha / beta, stores)
+//   warps 6-9 : epilogue     (D tile prefetched by TMA into swizzled shared memory, tcgen05.ld, alpha / beta
+//                             in place, TMA store: no strided global access)
 // Every wait is bounded; a wait that runs out raises a status word and the CTA leaves through the common
 // exit that frees its tensor memory.
 #include "tc_common.cuh"
@@ -26,11 +27,12 @@ using namespace tc;
 
 constexpr int TILE = 128, BK = 32;
 constexpr int NTHREADS = 320;
-constexpr int STAGES = 3;
+constexpr int STAGES = 2;
 constexpr int OP_BYTES = TILE * BK * 4;           // 16 KiB: one operand chunk
 constexpr int STAGE_BYTES = 4 * OP_BYTES;         // A hi, A lo, B hi, B lo
 constexpr uint32_t TMEM_COLS = 256;               // two accumulators of 128 columns
-constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 4 * 32 * 33 * sizeof(float) + 1024;
+constexpr int EPI_BYTES = 32 * TILE * 4;          // per epilogue warp: 32 rows x 128 columns as four swizzled boxes
+constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 4 * EPI_BYTES + 1024;
 
 struct OpCoord {
   int mn_major;                     // 0: K-major, 1: MN-major
@@ -69,16 +71,18 @@ __device__ __forceinline__ uint64_t operand_desc(uint32_t base, int mn_major, in
 }
 
 __global__ void __launch_bounds__(NTHREADS, 1)
-tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const BParams p) {
+tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                const __grid_constant__ CUtensorMap mapC, const __grid_constant__ CUtensorMap mapD, const BParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  __shared__ __align__(8) uint64_t bars[3 * STAGES + 4];
+  __shared__ __align__(8) uint64_t bars[3 * STAGES + 8];
   __shared__ uint32_t tmem_base_holder;
   __shared__ int abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t full0 = smem_u32(&bars[0]), split0 = smem_u32(&bars[STAGES]), empty0 = smem_u32(&bars[2 * STAGES]);
   const uint32_t tfull0 = smem_u32(&bars[3 * STAGES]), tempty0 = smem_u32(&bars[3 * STAGES + 2]);
+  const uint32_t dfull0 = smem_u32(&bars[3 * STAGES + 4]);
   const int n_items = p.batch * p.m_tiles * p.n_tiles;
 
   if (threadIdx.x == 0) {
@@ -89,6 +93,7 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       mbar_init(empty0 + 8 * s, 1);
     }
     for (int s = 0; s < 2; ++s) { mbar_init(tfull0 + 8 * s, 1); mbar_init(tempty0 + 8 * s, 4); }
+    for (int s = 0; s < 4; ++s) mbar_init(dfull0 + 8 * s, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -200,48 +205,68 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     // ------------------------------------------------------------ epilogue warps
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     int local = 0;
+    uint32_t d_loads = 0;   // D slabs requested so far: parity of their barrier
     bool ok = true;
-    float* tilebuf = reinterpret_cast<float*>(smem + (size_t)STAGES * STAGE_BYTES) + q * (32 * 33);
+    uint8_t* buf = smem + (size_t)STAGES * STAGE_BYTES + (size_t)q * EPI_BYTES;   // four 4 KiB boxes of 32 x 32
+    const uint32_t buf_u32 = smem_u32(buf);
+    const uint32_t dbar = dfull0 + 8 * q;
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++local) {
       const int tn = item % p.n_tiles, tm = (item / p.n_tiles) % p.m_tiles, b = item / (p.n_tiles * p.m_tiles);
       const int as = local & 1;
       const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
-      if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
-      tc_fence_after();
       const int64_t row_base = p.r_b * b + (int64_t)tm * TILE + q * 32;
       const int64_t col_tile = p.c_b * b + (int64_t)tn * TILE;
+      // boxes of this warp's slab that lie inside C (warp-uniform)
+      int n_box = 0;
+      if (row_base < p.c_rows)
+        for (int ch = 0; ch < 4; ++ch) n_box += (col_tile + 32 * ch < p.c_cols) ? 1 : 0;
+      if (lane == 0) {
+        tma_store_wait_read();                      // the previous item's stores have read the slab
+        if (p.D && n_box > 0) {
+          mbar_expect_tx(dbar, (uint32_t)n_box * 4096u);
+          for (int ch = 0; ch < n_box; ++ch)
+            tma_load_2d(buf_u32 + ch * 4096, &mapD, (int)(col_tile + 32 * ch), (int)row_base, dbar);
+        }
+      }
+      __syncwarp();
+      if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
+      tc_fence_after();
+      if (p.D && n_box > 0) {
+        if (!mbar_wait(dbar, d_loads & 1u, abortp, p.status)) { ok = false; break; }
+        ++d_loads;
+      }
 #pragma unroll 1
       for (int ch = 0; ch < TILE / 32; ++ch) {
         uint32_t r[32];
         tmem_ld32(tmem_base + (uint32_t)(as * TILE + ch * 32) + ((uint32_t)(q * 32) << 16), r);
-        const int64_t col0 = col_tile + ch * 32;
-        if (col0 >= p.c_cols || row_base >= p.c_rows) continue;   // warp-uniform
+        if (ch >= n_box) continue;                  // warp-uniform
+        // lane = row of the box; 16-byte chunk c of the row sits at chunk c ^ (row % 8)  (128-byte swizzle)
+        uint8_t* rowp = buf + ch * 4096 + lane * 128;
 #pragma unroll
-        for (int cidx = 0; cidx < 32; ++cidx) tilebuf[lane * 33 + cidx] = __uint_as_float(r[cidx]);
-        __syncwarp();
-        const int64_t col = col0 + lane;
-        const bool col_ok = col < p.c_cols;
-#pragma unroll 1
-        for (int r0 = 0; r0 < 32; r0 += 8) {
-          float x[8], d[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const int64_t grow = row_base + r0 + j;
-            x[j] = tilebuf[(r0 + j) * 33 + lane];
-            d[j] = (p.D && col_ok && grow < p.c_rows) ? p.D[grow * p.ldd + col] : 0.f;
+        for (int cq = 0; cq < 8; ++cq) {
+          float4* cell = reinterpret_cast<float4*>(rowp + ((cq ^ (lane & 7)) << 4));
+          float4 v = make_float4(p.alpha * __uint_as_float(r[4 * cq]), p.alpha * __uint_as_float(r[4 * cq + 1]),
+                                 p.alpha * __uint_as_float(r[4 * cq + 2]), p.alpha * __uint_as_float(r[4 * cq + 3]));
+          if (p.D) {
+            const float4 d = *cell;
+            v.x = fmaf(p.beta, d.x, v.x); v.y = fmaf(p.beta, d.y, v.y);
+            v.z = fmaf(p.beta, d.z, v.z); v.w = fmaf(p.beta, d.w, v.w);
           }
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const int64_t grow = row_base + r0 + j;
-            if (col_ok && grow < p.c_rows) p.C[grow * p.ldc + col] = fmaf(p.beta, d[j], p.alpha * x[j]);
-          }
+          *cell = v;
         }
-        __syncwarp();
       }
+      // accumulator buffer is free again
       tc_fence_before();
+      fence_proxy_async();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty0 + 8 * as);
+      if (lane == 0) {
+        mbar_arrive(tempty0 + 8 * as);
+        for (int ch = 0; ch < n_box; ++ch)
+          tma_store_2d(&mapC, (int)(col_tile + 32 * ch), (int)row_base, buf_u32 + ch * 4096);
+        tma_store_commit();
+      }
     }
+    if (lane == 0) tma_store_wait_read();           // shared memory stays valid until the stores have read it
   }
   tc_fence_before();
   __syncthreads();
@@ -257,7 +282,13 @@ struct HostOp {
 };
 
 armor_status launch(armor_ctx* c, const HostOp& A, const HostOp& B, BParams p, cudaStream_t s) {
-  CUtensorMap mA, mB;
+  CUtensorMap mA, mB, mC, mD;
+  if (!make_map_2d(&mC, p.C, p.c_cols, p.c_rows, p.ldc, 32, 32)) return ARMOR_ERR_CUDA;
+  if (p.D) {
+    if (!make_map_2d(&mD, p.D, p.c_cols, p.c_rows, p.ldd, 32, 32)) return ARMOR_ERR_CUDA;
+  } else {
+    mD = mC;
+  }
   if (!make_map_2d(&mA, A.base, A.inner, A.outer, A.ld, 32, A.c.mn_major ? 32 : TILE, A.c.mn_major != 0)) return ARMOR_ERR_CUDA;
   if (!make_map_2d(&mB, B.base, B.inner, B.outer, B.ld, 32, B.c.mn_major ? 32 : TILE, B.c.mn_major != 0)) return ARMOR_ERR_CUDA;
   p.a = A.c; p.b = B.c;
@@ -276,7 +307,7 @@ armor_status launch(armor_ctx* c, const HostOp& A, const HostOp& B, BParams p, c
   }
   const int n_items = p.batch * p.m_tiles * p.n_tiles;
   const int grid = n_items < n_sm ? n_items : n_sm;
-  tc_block_kernel<<<grid, NTHREADS, SMEM_BYTES, s>>>(mA, mB, p);
+  tc_block_kernel<<<grid, NTHREADS, SMEM_BYTES, s>>>(mA, mB, mC, mD, p);
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
 }
