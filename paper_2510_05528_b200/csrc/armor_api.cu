@@ -93,7 +93,9 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
     const int64_t tiles = (int64_t)((db + 127) / 128) * ((db + 127) / 128);
     const int64_t g1 = 2 * nbo * pick_ksplit(2 * nbo, tiles, cfg.d_in) * (int64_t)db * db;
     const int64_t g2 = 2 * nbi * pick_ksplit(2 * nbi, tiles, cfg.d_out) * (int64_t)db * db;
-    const int64_t gp = g1 > g2 ? g1 : g2;
+    int64_t gp = g1 > g2 ? g1 : g2;
+    const int64_t nbm = nbo > nbi ? nbo : nbi;
+    if (gp < 16 * nbm * (int64_t)db * db) gp = 16 * nbm * (int64_t)db * db;   // up to 16 slabs of one Gram
     TAKE(gpart, float*, (size_t)gp * sizeof(float));
     if (c) c->gpart_floats = gp;
   }
@@ -105,6 +107,7 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   TAKE(partials, double*, (size_t)8 * npart * sizeof(double));
   const int64_t nbmax = nbo > nbi ? nbo : nbi;
   TAKE(partblk, double*, (size_t)(4 * nbmax > nbo * nbi ? 4 * nbmax : nbo * nbi) * sizeof(double));
+  TAKE(quadpart, double*, (size_t)nbo * nbi * sizeof(double));
   TAKE(failflag, int32_t*, (size_t)nbmax * sizeof(int32_t));
   TAKE(sel, SelRec*, (size_t)nbo * nbi * sizeof(SelRec));
   TAKE(status, int32_t*, ST_COUNT * sizeof(int32_t));
@@ -123,6 +126,9 @@ inline cudaStream_t cs(armor_stream_t s) { return reinterpret_cast<cudaStream_t>
 void rowblock_grams(armor_ctx* c, const float* P, const float* P2, const float* T, float* G, float* G2, cudaStream_t s) {
   // G_i = P_i T_i^T, G2_i = P2_i T_i^T  (contraction over d_in), batch over row-blocks i
   const int db = c->db;
+  if (g_tc_blocks && tc_gram_ok(c) && tc_rowblock_gram(c, P, T, G, s) == ARMOR_OK &&
+      tc_rowblock_gram(c, P2, T, G2, s) == ARMOR_OK)
+    return;
   BGemm g{};
   g.A = P; g.sAb = (int64_t)db * c->d_in; g.sAm = c->d_in; g.sAk = 1;
   g.B = T; g.sBb = (int64_t)db * c->d_in; g.sBk = 1; g.sBn = c->d_in;
@@ -135,6 +141,9 @@ void rowblock_grams(armor_ctx* c, const float* P, const float* P2, const float* 
 void colblock_grams(armor_ctx* c, const float* U, const float* Y, const float* Y2, float* Cm, float* Cm2, cudaStream_t s) {
   // C_j = U_j^T Y_j, C2_j = U_j^T Y2_j  (contraction over d_out), batch over column-blocks j
   const int db = c->db;
+  if (g_tc_blocks && tc_gram_ok(c) && tc_colblock_gram(c, U, Y, Cm, s) == ARMOR_OK &&
+      tc_colblock_gram(c, U, Y2, Cm2, s) == ARMOR_OK)
+    return;
   BGemm g{};
   g.A = U; g.sAb = db; g.sAm = 1; g.sAk = c->d_in;
   g.B = Y; g.sBb = db; g.sBk = c->d_in; g.sBn = 1;

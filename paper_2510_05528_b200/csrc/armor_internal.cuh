@@ -69,7 +69,8 @@ struct armor_ctx {
   double* sc;         // [SC_COUNT]
   double* partials;   // [2][4 * npart] partial sums of the fused / streaming reductions
   int64_t npart;
-  double* partblk;    // [max(nbo, nbi, nbo * nbi)] per-block partial sums
+  double* partblk;    // [max(4 * nbo, 4 * nbi, nbo * nbi)] per-block partial sums
+  double* quadpart;   // [nbo * nbi] per-block terms of the group updates' quadratic form
   double* colpart;    // [64][d_in] column partial sums of the normalisation
   int32_t* failflag;  // [max(nbo, nbi)]
   SelRec* sel;        // [nbo * nbi]
@@ -135,6 +136,12 @@ armor_status tc_bd_right(armor_ctx* c, const float* in, const float* Bblk, bool 
                          int64_t cols, float alpha, const float* add, float beta, cudaStream_t s);
 armor_status tc_bd_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, float* out, int64_t rows,
                         int64_t cols, float alpha, const float* add, float beta, cudaStream_t s);
+
+// per-block Grams over a long contraction on the tensor cores
+bool tc_gram_ok(const armor_ctx* c);
+armor_status tc_rowblock_gram(armor_ctx* c, const float* P, const float* T, float* G, cudaStream_t s);
+armor_status tc_colblock_gram(armor_ctx* c, const float* U, const float* Y, float* Cm, cudaStream_t s);
+extern int g_tc_blocks;   // 1: block products and per-block Grams on the tensor cores where the shape allows
 
 // out = in * H_w (FULL: dense GEMM by cfg.precision; DIAG: column scale) with up to two
 // fused dot products <out, d1> -> sc[slot1], <out, d2> -> sc[slot2] (slot < 0: none).

@@ -45,8 +45,10 @@ struct BParams {
   float* C; const float* D;
   int64_t ldc, ldd;
   int64_t c_rows, c_cols;           // extent of C (stores are guarded)
-  int64_t r_b, c_b;                 // tile origin: row = r_b * batch + 128 * tm, column = c_b * batch + 128 * tn
-  int m_tiles, n_tiles, batch, k_chunks;
+  int64_t r_b, c_b;                 // tile origin: row = r_b * batch + 128 * tm (+ r_s * split), column = c_b * batch + 128 * tn
+  int64_t r_s;
+  int m_tiles, n_tiles, batch, k_chunks;   // k_chunks: chunks of 32 along K per work item
+  int n_split;                      // the contraction is cut into n_split items of k_chunks chunks each
   float alpha, beta;
   int32_t* status;
 };
@@ -83,7 +85,7 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
   const uint32_t full0 = smem_u32(&bars[0]), split0 = smem_u32(&bars[STAGES]), empty0 = smem_u32(&bars[2 * STAGES]);
   const uint32_t tfull0 = smem_u32(&bars[3 * STAGES]), tempty0 = smem_u32(&bars[3 * STAGES + 2]);
   const uint32_t dfull0 = smem_u32(&bars[3 * STAGES + 4]);
-  const int n_items = p.batch * p.m_tiles * p.n_tiles;
+  const int n_items = p.batch * p.m_tiles * p.n_tiles * p.n_split;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -114,14 +116,15 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       int stage = 0; uint32_t phase = 0; long long issued = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-        const int tn = item % p.n_tiles, tm = (item / p.n_tiles) % p.m_tiles, b = item / (p.n_tiles * p.m_tiles);
+        const int tn = item % p.n_tiles, tm = (item / p.n_tiles) % p.m_tiles;
+        const int b = (item / (p.n_tiles * p.m_tiles)) % p.batch, ks = item / (p.n_tiles * p.m_tiles * p.batch);
         for (int kc = 0; kc < p.k_chunks; ++kc) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abortp, p.status)) { ok = false; break; }
           const uint32_t fb = full0 + 8 * stage;
           mbar_expect_tx(fb, 2 * OP_BYTES);
           const uint32_t dst = smem_u32(smem + (size_t)stage * STAGE_BYTES);
-          load_operand(dst, &mapA, p.a, b, tm, kc, fb);
-          load_operand(dst + 2 * OP_BYTES, &mapB, p.b, b, tn, kc, fb);
+          load_operand(dst, &mapA, p.a, b, tm, ks * p.k_chunks + kc, fb);
+          load_operand(dst + 2 * OP_BYTES, &mapB, p.b, b, tn, ks * p.k_chunks + kc, fb);
           ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -211,10 +214,11 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     const uint32_t buf_u32 = smem_u32(buf);
     const uint32_t dbar = dfull0 + 8 * q;
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++local) {
-      const int tn = item % p.n_tiles, tm = (item / p.n_tiles) % p.m_tiles, b = item / (p.n_tiles * p.m_tiles);
+      const int tn = item % p.n_tiles, tm = (item / p.n_tiles) % p.m_tiles;
+      const int b = (item / (p.n_tiles * p.m_tiles)) % p.batch, ks = item / (p.n_tiles * p.m_tiles * p.batch);
       const int as = local & 1;
       const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
-      const int64_t row_base = p.r_b * b + (int64_t)tm * TILE + q * 32;
+      const int64_t row_base = p.r_b * b + p.r_s * ks + (int64_t)tm * TILE + q * 32;
       const int64_t col_tile = p.c_b * b + (int64_t)tn * TILE;
       // boxes of this warp's slab that lie inside C (warp-uniform)
       int n_box = 0;
@@ -305,7 +309,7 @@ armor_status launch(armor_ctx* c, const HostOp& A, const HostOp& B, BParams p, c
     if (cudaGetDevice(&dev) != cudaSuccess) return ARMOR_ERR_CUDA;
     if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ARMOR_ERR_CUDA;
   }
-  const int n_items = p.batch * p.m_tiles * p.n_tiles;
+  const int n_items = p.batch * p.m_tiles * p.n_tiles * p.n_split;
   const int grid = n_items < n_sm ? n_items : n_sm;
   tc_block_kernel<<<grid, NTHREADS, SMEM_BYTES, s>>>(mA, mB, mC, mD, p);
   c->launches++;
@@ -335,6 +339,7 @@ armor_status tc_bd_right(armor_ctx* c, const float* in, const float* Bblk, bool 
   p.r_b = 0; p.c_b = db;
   p.m_tiles = (int)((rows + TILE - 1) / TILE); p.n_tiles = db / TILE; p.batch = nb; p.k_chunks = db / BK;
   p.alpha = alpha; p.beta = add ? beta : 0.f;
+  p.n_split = 1; p.r_s = 0;
   return launch(c, A, B, p, s);
 }
 
@@ -353,5 +358,76 @@ armor_status tc_bd_left(armor_ctx* c, const float* Ablk, bool transA, const floa
   p.r_b = db; p.c_b = 0;
   p.m_tiles = db / TILE; p.n_tiles = (int)((cols + TILE - 1) / TILE); p.batch = nb; p.k_chunks = db / BK;
   p.alpha = alpha; p.beta = add ? beta : 0.f;
+  p.n_split = 1; p.r_s = 0;
   return launch(c, A, B, p, s);
+}
+
+namespace {
+
+// out[e] = sum over the slabs, in slab order
+__global__ void __launch_bounds__(256) sum_slabs_kernel(const float4* __restrict__ part, int64_t n4, int n_slab,
+                                                        float4* __restrict__ out) {
+  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n4; i += (int64_t)gridDim.x * 256) {
+    float4 acc = part[i];
+    for (int k = 1; k < n_slab; ++k) {
+      const float4 v = part[(int64_t)k * n4 + i];
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    out[i] = acc;
+  }
+}
+
+// chunks of the contraction per work item so that about one CTA per SM has work
+int pick_split(int64_t items, int64_t chunks) {
+  int64_t ks = (148 + items - 1) / items;
+  if (ks > chunks / 8) ks = chunks / 8;
+  while (ks > 1 && chunks % ks) --ks;
+  return ks < 1 ? 1 : (int)ks;
+}
+
+armor_status gram_launch(armor_ctx* c, const HostOp& A, const HostOp& B, float* G, int nb, int64_t K, cudaStream_t s) {
+  const int db = c->db;
+  const int64_t chunks = K / BK;
+  const int tiles = (db / TILE) * (db / TILE);
+  int ks = pick_split((int64_t)nb * tiles, chunks);
+  const int64_t slab = (int64_t)nb * db * db;
+  if (ks > 1 && (!c->gpart || ks * slab > c->gpart_floats)) ks = 1;
+  BParams p{};
+  p.C = ks > 1 ? c->gpart : G; p.D = nullptr; p.ldc = db; p.ldd = db;
+  p.c_rows = (int64_t)ks * nb * db; p.c_cols = db;
+  p.r_b = db; p.c_b = 0; p.r_s = (int64_t)nb * db;
+  p.m_tiles = db / TILE; p.n_tiles = db / TILE; p.batch = nb; p.k_chunks = (int)(chunks / ks); p.n_split = ks;
+  p.alpha = 1.f; p.beta = 0.f;
+  armor_status st = launch(c, A, B, p, s);
+  if (st != ARMOR_OK || ks == 1) return st;
+  int64_t blocks = (slab / 4 + 255) / 256;
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  sum_slabs_kernel<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(c->gpart), slab / 4, ks,
+                                                   reinterpret_cast<float4*>(G));
+  c->launches++;
+  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+}
+
+}  // namespace
+
+bool tc_gram_ok(const armor_ctx* c) {
+  return c->cfg.precision != ARMOR_PREC_SIMT && c->db % TILE == 0 && c->d_in % BK == 0 && c->d_out % BK == 0;
+}
+
+// G_i = P_i T_i^T over the row-blocks i (contraction over d_in)
+armor_status tc_rowblock_gram(armor_ctx* c, const float* P, const float* T, float* G, cudaStream_t s) {
+  const int db = c->db;
+  if (!ptr_ok(P) || !ptr_ok(T) || !ptr_ok(G)) return ARMOR_ERR_UNSUPPORTED;
+  HostOp A{P, c->d_in, c->d_out, c->d_in, {0, 0, 0, BK, db, TILE, 0}};   // Aop[m][k] = P[i*db + m][k]: K-major
+  HostOp B{T, c->d_in, c->d_out, c->d_in, {0, 0, 0, BK, db, TILE, 0}};
+  return gram_launch(c, A, B, G, c->nbo, c->d_in, s);
+}
+
+// C_j = U_j^T Y_j over the column-blocks j (contraction over d_out)
+armor_status tc_colblock_gram(armor_ctx* c, const float* U, const float* Y, float* Cm, cudaStream_t s) {
+  const int db = c->db;
+  if (!ptr_ok(U) || !ptr_ok(Y) || !ptr_ok(Cm)) return ARMOR_ERR_UNSUPPORTED;
+  HostOp A{U, c->d_in, c->d_out, c->d_in, {1, db, TILE, 0, 0, 0, BK}};   // Aop[m][k] = U[k][j*db + m]: M-major
+  HostOp B{Y, c->d_in, c->d_out, c->d_in, {1, db, TILE, 0, 0, 0, BK}};
+  return gram_launch(c, A, B, Cm, c->nbi, c->d_out, s);
 }

@@ -302,7 +302,7 @@ void launch_bgemm(armor_ctx* c, const BGemm& g_in, cudaStream_t s) {
 }
 
 // 1: block-diagonal products on the tensor cores where the shape allows; 0: always the fp32 CUDA-core kernels
-static int g_tc_blocks = 1;
+int g_tc_blocks = 1;
 extern "C" void armor_debug_set_tc_blocks(int on) { g_tc_blocks = on; }
 
 void bd_right(armor_ctx* c, const float* in, const float* Bblk, bool transB, float* out, int64_t rows,

@@ -23,17 +23,25 @@ __device__ __forceinline__ float neg_log_uniform(uint32_t k24) {
   return -log1pf(-(float)(2u * ((1u << 24) - k24) - 1u) * 2.98023223876953125e-8f);
 }
 
+// alpha[r] = || A[:, r] ||^2 : column r of the block that owns row r of the core.
+// blockDim = (32 columns, 8 row slices); grid = (nbo, db / 32).
 __global__ void alpha_kernel(const float* __restrict__ A, float* __restrict__ alpha, int db) {
-  // alpha[r] = || A[:, r] ||^2 : column r of the block that owns row r of the core
   const int i = blockIdx.x;
+  const int r = blockIdx.y * 32 + threadIdx.x;
   const float* Ai = A + (int64_t)i * db * db;
-  for (int r = threadIdx.x; r < db; r += blockDim.x) {
-    double acc = 0.0;
-    for (int o = 0; o < db; ++o) {
-      double v = Ai[o * db + r];
+  double acc = 0.0;
+  if (r < db)
+    for (int o = threadIdx.y; o < db; o += 8) {
+      const double v = Ai[(int64_t)o * db + r];
       acc += v * v;
     }
-    alpha[i * db + r] = (float)acc;
+  __shared__ double part[8][33];
+  part[threadIdx.y][threadIdx.x] = acc;
+  __syncthreads();
+  if (threadIdx.y == 0 && r < db) {
+    double t = 0.0;
+    for (int k = 0; k < 8; ++k) t += part[k][threadIdx.x];
+    alpha[i * db + r] = (float)t;
   }
 }
 
@@ -313,19 +321,17 @@ __global__ void __launch_bounds__(NT) mask_vectors_kernel(const float* __restric
   }
 }
 
-// One CTA per row-block i, one warp per (j, j') pair at a time.  Y == nullptr: diagonal weighting, only the
-// j == j' pairs contribute and y = z (.) hdiag.
+// One CTA per block (i, j), one warp per pair (j, j') at a time.  Y == nullptr: diagonal weighting, only the
+// j == j' pair contributes and y = z (.) hdiag.
 __global__ void __launch_bounds__(NT) mask_quad_kernel(const float* __restrict__ Zsel, const float* __restrict__ Acol,
                                                        const float* __restrict__ Y, const float* __restrict__ hdiag,
                                                        double* __restrict__ part, int64_t d_in, int db, int nbo,
                                                        int nbi) {
-  const int bi = blockIdx.x;
+  const int bi = blockIdx.x / nbi, j = blockIdx.x % nbi;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = NT / 32;
   double acc = 0.0;
-  const int npairs = Y ? nbi * nbi : nbi;
-  for (int pr = warp; pr < npairs; pr += nw) {
-    const int j = Y ? pr / nbi : pr, j2 = Y ? pr % nbi : pr;
-    const float* a1 = Acol + ((int64_t)bi * nbi + j) * db;
+  const float* a1 = Acol + ((int64_t)bi * nbi + j) * db;
+  for (int j2 = Y ? warp : j + warp; j2 < (Y ? nbi : j + 1); j2 += nw) {
     const float* a2 = Acol + ((int64_t)bi * nbi + j2) * db;
     const float* z2 = Zsel + ((int64_t)j2 * nbo + bi) * db;
     float w = 0.f, m = 0.f;
@@ -348,7 +354,7 @@ __global__ void __launch_bounds__(NT) mask_quad_kernel(const float* __restrict__
   if (threadIdx.x == 0) {
     double t = 0.0;
     for (int w2 = 0; w2 < nw; ++w2) t += red[w2];
-    part[bi] = t;
+    part[blockIdx.x] = t;
   }
 }
 
@@ -380,7 +386,7 @@ __global__ void mask_commit_kernel(const SelRec* __restrict__ sel, int nblocks, 
 }  // namespace
 
 void launch_alpha(armor_ctx* c, const float* A, cudaStream_t s) {
-  alpha_kernel<<<c->nbo, 128, 0, s>>>(A, c->alpha, c->db);
+  alpha_kernel<<<dim3(c->nbo, (c->db + 31) / 32), dim3(32, 8), 0, s>>>(A, c->alpha, c->db);
   c->launches++;
 }
 
@@ -413,10 +419,10 @@ void launch_mask_quadratic(armor_ctx* c, const float* A, const float* B, const f
     launch_bgemm(c, g, s);
     Y = c->Ysel;
   }
-  double* part = c->partials + 4 * c->npart;
-  mask_quad_kernel<<<nbo, NT, 0, s>>>(c->Zsel, c->Acol, Y, c->hdiag, part, c->d_in, db, nbo, nbi);
+  double* part = c->quadpart;
+  mask_quad_kernel<<<nbo * nbi, NT, 0, s>>>(c->Zsel, c->Acol, Y, c->hdiag, part, c->d_in, db, nbo, nbi);
   c->launches++;
-  reduce_partials_to(c, part, nbo, c->sc + SC_Q_M, s);
+  reduce_partials_to(c, part, nbo * nbi, c->sc + SC_Q_M, s);
 }
 
 void launch_mask_commit(armor_ctx* c, float* S, uint8_t* M, armor_iter_stats* st, cudaStream_t s) {

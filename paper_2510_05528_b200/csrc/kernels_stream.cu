@@ -224,9 +224,27 @@ __global__ void zero_scalars_kernel(double* sc, int32_t* failflag, int nflag) {
   for (int i = threadIdx.x; i < nflag; i += blockDim.x) failflag[i] = 0;
 }
 
-// stage 0: start, 1: after A, 2: after B, 3: after S, 4: mask accept
+// Fixed-order sums by one warp: lane l adds entries l, l + 32, ...; then a shuffle tree.  All lanes get the sum.
+__device__ __forceinline__ double warp_sum_f64(const double* __restrict__ p, int n) {
+  double v = 0.0;
+  for (int i = threadIdx.x; i < n; i += 32) v += p[i];
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ int warp_count_flags(const int32_t* __restrict__ f, int n) {
+  int v = 0;
+  for (int i = threadIdx.x; i < n; i += 32) v += f[i] ? 1 : 0;
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// stage 0: start, 1: after A, 2: after B, 3 / 6: after S, 4: mask accept.  One warp.
 __global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const int32_t* failflag, int nflag,
                              const double* partA, int nA, int32_t* status) {
+  double psum = 0.0;
+  int nf = 0;
+  if (stage == 1 || stage == 2 || stage == 4) psum = warp_sum_f64(partA, nA);
+  if (stage == 1 || stage == 2) nf = warp_count_flags(failflag, nflag);
   if (threadIdx.x != 0) return;
   if (stage == 0) {
     sc[SC_LOSS] = sc[SC_L0];
@@ -241,24 +259,17 @@ __global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const 
       st->reserved = 0;
     }
   } else if (stage == 1) {
-    double dec = 0.0;
-    for (int i = 0; i < nA; ++i) dec += partA[i];
-    sc[SC_DEC_A] = dec;
-    sc[SC_LOSS] -= dec;
-    int nf = 0;
-    for (int i = 0; i < nflag; ++i) nf += failflag[i] ? 1 : 0;
+    sc[SC_DEC_A] = psum;
+    sc[SC_LOSS] -= psum;
     if (st) { st->loss_A = sc[SC_LOSS]; st->chol_failed += nf; }
     if (nf) atomicAdd(&status[ST_CHOL_FAILS], nf);
   } else if (stage == 2) {
-    double gd = 0.0;
-    for (int i = 0; i < nA; ++i) gd += partA[i];
+    const double gd = psum;
     sc[SC_GD_B] = gd;
     const double q = sc[SC_Q_B];
     const double tau = (q > 0.0) ? gd / q : 0.0;
     sc[SC_TAU_B] = tau;
     sc[SC_LOSS] -= 2.0 * tau * gd - tau * tau * q;
-    int nf = 0;
-    for (int i = 0; i < nflag; ++i) nf += failflag[i] ? 1 : 0;
     if (st) { st->loss_B = sc[SC_LOSS]; st->tau_B = (float)tau; st->chol_failed += nf; }
     if (nf) atomicAdd(&status[ST_CHOL_FAILS], nf);
   } else if (stage == 3 || stage == 6) {
@@ -272,9 +283,7 @@ __global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const 
     sc[SC_LOSS] -= 2.0 * tau * nrm - tau * tau * q;
     if (st) { st->loss_S = sc[SC_LOSS]; st->tau_S = (float)tau; }
   } else if (stage == 4) {
-    double ehv = 0.0;
-    for (int i = 0; i < nA; ++i) ehv += partA[i];   // <Gamma, dS> = <E H_w, V>, one term per block
-    sc[SC_EHV_M] = ehv;
+    sc[SC_EHV_M] = psum;   // <Gamma, dS> = <E H_w, V>, one term per block
     const double dl = -2.0 * sc[SC_EHV_M] + sc[SC_Q_M];
     const bool acc = (dl <= 0.0);
     sc[SC_DL_M] = dl;
