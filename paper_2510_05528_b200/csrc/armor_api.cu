@@ -79,9 +79,11 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   TAKE(Bt, float*, bo);
   TAKE(alpha, float*, (size_t)cfg.d_out * sizeof(float));
   TAKE(hdiag, float*, (size_t)cfg.d_in * sizeof(float));
-  TAKE(Zsel, float*, (size_t)nbo * nbi * db * sizeof(float));
+  const int64_t nbo_pad = (nbo + 31) / 32 * 32;
+  TAKE(Zsel, float*, (size_t)nbo_pad * nbi * db * sizeof(float));
   TAKE(Acol, float*, (size_t)nbo * nbi * db * sizeof(float));
-  TAKE(Ysel, float*, (size_t)nbo * nbi * cfg.d_in * sizeof(float));
+  TAKE(Ysel, float*, (size_t)nbo_pad * nbi * cfg.d_in * sizeof(float));
+  if (c) c->nbo_pad = (int)nbo_pad;
   TAKE(colpart, double*, (size_t)64 * cfg.d_in * sizeof(double));
   if (tc) {
     TAKE(Xt_hi, float*, (size_t)cfg.d_in * GRAM_ROWS * sizeof(float));

@@ -62,7 +62,8 @@ struct armor_ctx {
   float* gpart;          // partial products of split contractions
   int64_t gpart_floats;
   // sparse-core update: per selected group z = delta^T B_j[rows of the group, :] and a = A_i[:, r]
-  float *Zsel, *Acol, *Ysel;  // [nbi][nbo][db], [nbo][nbi][db], [nbi][nbo][d_in]
+  float *Zsel, *Acol, *Ysel;  // [nbi][nbo_pad][db], [nbo][nbi][db], [nbi][nbo_pad][d_in]
+  int nbo_pad;                // nbo rounded up to a multiple of 32
   // Gram staging (transposed, split chunk of X)
   float *Xt_hi, *Xt_lo;
   int64_t gram_rows;  // rows of X staged per pass
@@ -141,6 +142,7 @@ armor_status tc_bd_left(armor_ctx* c, const float* Ablk, bool transA, const floa
 bool tc_gram_ok(const armor_ctx* c);
 armor_status tc_rowblock_gram(armor_ctx* c, const float* P, const float* T, float* G, cudaStream_t s);
 armor_status tc_colblock_gram(armor_ctx* c, const float* U, const float* Y, float* Cm, cudaStream_t s);
+armor_status tc_select_rows_times_H(armor_ctx* c, const float* Z, const float* H, float* Y, int nbo_pad, cudaStream_t s);
 extern int g_tc_blocks;   // 1: block products and per-block Grams on the tensor cores where the shape allows
 
 // out = in * H_w (FULL: dense GEMM by cfg.precision; DIAG: column scale) with up to two

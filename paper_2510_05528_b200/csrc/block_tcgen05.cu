@@ -47,6 +47,7 @@ struct BParams {
   int64_t c_rows, c_cols;           // extent of C (stores are guarded)
   int64_t r_b, c_b;                 // tile origin: row = r_b * batch + 128 * tm (+ r_s * split), column = c_b * batch + 128 * tn
   int64_t r_s;
+  int m_valid;                      // rows of a batch's tile range that exist (boxes of 32 rows beyond it are not stored)
   int m_tiles, n_tiles, batch, k_chunks;   // k_chunks: chunks of 32 along K per work item
   int n_split;                      // the contraction is cut into n_split items of k_chunks chunks each
   float alpha, beta;
@@ -222,7 +223,7 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       const int64_t col_tile = p.c_b * b + (int64_t)tn * TILE;
       // boxes of this warp's slab that lie inside C (warp-uniform)
       int n_box = 0;
-      if (row_base < p.c_rows)
+      if (row_base < p.c_rows && tm * TILE + q * 32 < p.m_valid)
         for (int ch = 0; ch < 4; ++ch) n_box += (col_tile + 32 * ch < p.c_cols) ? 1 : 0;
       if (lane == 0) {
         tma_store_wait_read();                      // the previous item's stores have read the slab
@@ -339,7 +340,7 @@ armor_status tc_bd_right(armor_ctx* c, const float* in, const float* Bblk, bool 
   p.r_b = 0; p.c_b = db;
   p.m_tiles = (int)((rows + TILE - 1) / TILE); p.n_tiles = db / TILE; p.batch = nb; p.k_chunks = db / BK;
   p.alpha = alpha; p.beta = add ? beta : 0.f;
-  p.n_split = 1; p.r_s = 0;
+  p.n_split = 1; p.r_s = 0; p.m_valid = 1 << 30;
   return launch(c, A, B, p, s);
 }
 
@@ -358,7 +359,7 @@ armor_status tc_bd_left(armor_ctx* c, const float* Ablk, bool transA, const floa
   p.r_b = db; p.c_b = 0;
   p.m_tiles = db / TILE; p.n_tiles = (int)((cols + TILE - 1) / TILE); p.batch = nb; p.k_chunks = db / BK;
   p.alpha = alpha; p.beta = add ? beta : 0.f;
-  p.n_split = 1; p.r_s = 0;
+  p.n_split = 1; p.r_s = 0; p.m_valid = 1 << 30;
   return launch(c, A, B, p, s);
 }
 
@@ -397,7 +398,7 @@ armor_status gram_launch(armor_ctx* c, const HostOp& A, const HostOp& B, float* 
   p.c_rows = (int64_t)ks * nb * db; p.c_cols = db;
   p.r_b = db; p.c_b = 0; p.r_s = (int64_t)nb * db;
   p.m_tiles = db / TILE; p.n_tiles = db / TILE; p.batch = nb; p.k_chunks = (int)(chunks / ks); p.n_split = ks;
-  p.alpha = 1.f; p.beta = 0.f;
+  p.alpha = 1.f; p.beta = 0.f; p.m_valid = 1 << 30;
   armor_status st = launch(c, A, B, p, s);
   if (st != ARMOR_OK || ks == 1) return st;
   int64_t blocks = (slab / 4 + 255) / 256;
@@ -430,4 +431,21 @@ armor_status tc_colblock_gram(armor_ctx* c, const float* U, const float* Y, floa
   HostOp A{U, c->d_in, c->d_out, c->d_in, {1, db, TILE, 0, 0, 0, BK}};   // Aop[m][k] = U[k][j*db + m]: M-major
   HostOp B{Y, c->d_in, c->d_out, c->d_in, {1, db, TILE, 0, 0, 0, BK}};
   return gram_launch(c, A, B, Cm, c->nbi, c->d_out, s);
+}
+
+// Y[j][i][:] = Z[j][i][:] * H[j-th block row, :]  for i < nbo: per column-block j a thin [nbo, d_block] x
+// [d_block, d_in] product (the group-update guard).  Z and Y are stored with nbo_pad rows per j.
+armor_status tc_select_rows_times_H(armor_ctx* c, const float* Z, const float* H, float* Y, int nbo_pad, cudaStream_t s) {
+  const int db = c->db;
+  if (!ptr_ok(Z) || !ptr_ok(H) || !ptr_ok(Y)) return ARMOR_ERR_UNSUPPORTED;
+  HostOp A{Z, db, (int64_t)c->nbi * nbo_pad, db, {0, 0, 0, BK, nbo_pad, TILE, 0}};            // Aop[m][k] = Z[j][m][k]
+  HostOp B{H, c->d_in, c->d_in, c->d_in, {1, 0, TILE, 0, db, 0, BK}};                         // Bop[n][k] = H[j*db + k][n]
+  BParams p{};
+  p.C = Y; p.D = nullptr; p.ldc = c->d_in; p.ldd = c->d_in;
+  p.c_rows = (int64_t)c->nbi * nbo_pad; p.c_cols = c->d_in;
+  p.r_b = nbo_pad; p.c_b = 0; p.r_s = 0;
+  p.m_tiles = (c->nbo + TILE - 1) / TILE; p.n_tiles = (int)((c->d_in + TILE - 1) / TILE); p.batch = c->nbi;
+  p.k_chunks = db / BK; p.n_split = 1; p.m_valid = c->nbo;
+  p.alpha = 1.f; p.beta = 0.f;
+  return launch(c, A, B, p, s);
 }

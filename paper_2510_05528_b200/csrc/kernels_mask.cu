@@ -303,7 +303,7 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
 // row, :], and mask_quad_kernel sums the pairs in a fixed order.
 __global__ void __launch_bounds__(NT) mask_vectors_kernel(const float* __restrict__ A, const float* __restrict__ B,
                                                           const SelRec* __restrict__ sel, float* __restrict__ Zsel,
-                                                          float* __restrict__ Acol, int db, int nbo, int nbi, int mg) {
+                                                          float* __restrict__ Acol, int db, int nbo_pad, int nbi, int mg) {
   const int blk = blockIdx.x;
   const int bi = blk / nbi, bj = blk % nbi;
   const SelRec rec = sel[blk];
@@ -317,7 +317,7 @@ __global__ void __launch_bounds__(NT) mask_vectors_kernel(const float* __restric
       for (int p = 0; p < mg; ++p) z = fmaf(rec.new_val[p] - rec.old_val[p], Bj[(int64_t)(lc + p) * db + k], z);
     }
     Acol[((int64_t)bi * nbi + bj) * db + k] = a;
-    Zsel[((int64_t)bj * nbo + bi) * db + k] = z;
+    Zsel[((int64_t)bj * nbo_pad + bi) * db + k] = z;
   }
 }
 
@@ -325,7 +325,7 @@ __global__ void __launch_bounds__(NT) mask_vectors_kernel(const float* __restric
 // j == j' pair contributes and y = z (.) hdiag.
 __global__ void __launch_bounds__(NT) mask_quad_kernel(const float* __restrict__ Zsel, const float* __restrict__ Acol,
                                                        const float* __restrict__ Y, const float* __restrict__ hdiag,
-                                                       double* __restrict__ part, int64_t d_in, int db, int nbo,
+                                                       double* __restrict__ part, int64_t d_in, int db, int nbo_pad,
                                                        int nbi) {
   const int bi = blockIdx.x / nbi, j = blockIdx.x % nbi;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = NT / 32;
@@ -333,10 +333,10 @@ __global__ void __launch_bounds__(NT) mask_quad_kernel(const float* __restrict__
   const float* a1 = Acol + ((int64_t)bi * nbi + j) * db;
   for (int j2 = Y ? warp : j + warp; j2 < (Y ? nbi : j + 1); j2 += nw) {
     const float* a2 = Acol + ((int64_t)bi * nbi + j2) * db;
-    const float* z2 = Zsel + ((int64_t)j2 * nbo + bi) * db;
+    const float* z2 = Zsel + ((int64_t)j2 * nbo_pad + bi) * db;
     float w = 0.f, m = 0.f;
     if (Y) {
-      const float* y = Y + ((int64_t)j * nbo + bi) * d_in + (int64_t)j2 * db;
+      const float* y = Y + ((int64_t)j * nbo_pad + bi) * d_in + (int64_t)j2 * db;
       for (int k = lane; k < db; k += 32) { w = fmaf(a1[k], a2[k], w); m = fmaf(y[k], z2[k], m); }
     } else {
       const float* h = hdiag + (int64_t)j * db;
@@ -405,22 +405,24 @@ void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const ui
 }
 
 void launch_mask_quadratic(armor_ctx* c, const float* A, const float* B, const float* H, cudaStream_t s) {
-  const int db = c->db, nbo = c->nbo, nbi = c->nbi;
-  mask_vectors_kernel<<<nbo * nbi, NT, 0, s>>>(A, B, c->sel, c->Zsel, c->Acol, db, nbo, nbi, c->cfg.m_group);
+  const int db = c->db, nbo = c->nbo, nbi = c->nbi, nbo_pad = c->nbo_pad;
+  mask_vectors_kernel<<<nbo * nbi, NT, 0, s>>>(A, B, c->sel, c->Zsel, c->Acol, db, nbo_pad, nbi, c->cfg.m_group);
   c->launches++;
   const float* Y = nullptr;
   if (c->cfg.h_mode == ARMOR_H_FULL) {
     // y_ij = z_ij H[j-th block row, :], batched over j:  [nbo, db] x [db, d_in]
-    BGemm g{};
-    g.A = c->Zsel; g.sAb = (int64_t)nbo * db; g.sAm = db; g.sAk = 1;
-    g.B = H; g.sBb = (int64_t)db * c->d_in; g.sBk = c->d_in; g.sBn = 1;
-    g.C = c->Ysel; g.sCb = (int64_t)nbo * c->d_in; g.sCm = c->d_in; g.sCn = 1;
-    g.M = nbo; g.N = (int)c->d_in; g.K = db; g.batch = nbi; g.alpha = 1.f;
-    launch_bgemm(c, g, s);
+    if (!(g_tc_blocks && tc_gram_ok(c) && tc_select_rows_times_H(c, c->Zsel, H, c->Ysel, nbo_pad, s) == ARMOR_OK)) {
+      BGemm g{};
+      g.A = c->Zsel; g.sAb = (int64_t)nbo_pad * db; g.sAm = db; g.sAk = 1;
+      g.B = H; g.sBb = (int64_t)db * c->d_in; g.sBk = c->d_in; g.sBn = 1;
+      g.C = c->Ysel; g.sCb = (int64_t)nbo_pad * c->d_in; g.sCm = c->d_in; g.sCn = 1;
+      g.M = nbo; g.N = (int)c->d_in; g.K = db; g.batch = nbi; g.alpha = 1.f;
+      launch_bgemm(c, g, s);
+    }
     Y = c->Ysel;
   }
   double* part = c->quadpart;
-  mask_quad_kernel<<<nbo * nbi, NT, 0, s>>>(c->Zsel, c->Acol, Y, c->hdiag, part, c->d_in, db, nbo, nbi);
+  mask_quad_kernel<<<nbo * nbi, NT, 0, s>>>(c->Zsel, c->Acol, Y, c->hdiag, part, c->d_in, db, nbo_pad, nbi);
   c->launches++;
   reduce_partials_to(c, part, nbo * nbi, c->sc + SC_Q_M, s);
 }
