@@ -63,8 +63,8 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   TAKE(Gam, float*, wbytes);
   TAKE(Tmp, float*, wbytes);
   TAKE(WH, float*, wbytes);
-  if (x3) { TAKE(LoHi, float*, wbytes); TAKE(Lo, float*, wbytes); } else if (c) { c->LoHi = nullptr; c->Lo = nullptr; }
-  if (x3) { TAKE(Hhi, float*, hbytes); TAKE(Hlo, float*, hbytes); } else if (c) { c->Hhi = nullptr; c->Hlo = nullptr; }
+  if (x3) { TAKE(Lo, float*, wbytes); } else if (c) { c->Lo = nullptr; }
+  if (x3) { TAKE(Hlo, float*, hbytes); } else if (c) { c->Hlo = nullptr; }
   const size_t ao = (size_t)nbo * db * db * sizeof(float), bo = (size_t)nbi * db * db * sizeof(float);
   TAKE(G, float*, ao);
   TAKE(GamA, float*, ao);

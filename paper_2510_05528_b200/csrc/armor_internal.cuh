@@ -54,7 +54,7 @@ struct armor_ctx {
   // W-shaped fp32 scratch
   float *T, *E, *EH, *P, *U, *V, *VH, *Gam, *Tmp, *WH;
   // low parts of the left operands / of H for the three-pass tensor-core mode
-  float *LoHi, *Lo, *Hhi, *Hlo;
+  float *Lo, *Hlo;
   // [nb, db, db] scratch
   float *G, *GamA, *dA, *At, *C, *GamB, *Delta, *Hjj, *Kfull, *Ktmp, *Bt;
   float *alpha, *hdiag;
@@ -77,7 +77,7 @@ struct armor_ctx {
   SelRec* sel;        // [nbo * nbi]
   int32_t* status;    // [ST_COUNT]
   int64_t launches;
-  // identity of the H whose split copy is cached in Hhi/Hlo
+  // identity of the H whose low part is cached in Hlo
   const float* h_cached;
   // optional event timing of the tensor-core GEMM launches
   int timing_on;

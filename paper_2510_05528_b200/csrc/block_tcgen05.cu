@@ -21,6 +21,11 @@
 // exit that frees its tensor memory.
 #include "tc_common.cuh"
 
+// The tensor core reads the top 19 bits of a 32-bit tf32 operand and ignores the rest, so the raw fp32 word
+// serves as the high part and only the low part has to be written (checked against the masked form: same bits).
+int g_tc_raw_hi = 1;
+extern "C" void armor_debug_set_tc_raw_hi(int on) { g_tc_raw_hi = on; }
+
 namespace {
 
 using namespace tc;
@@ -52,6 +57,8 @@ struct BParams {
   int n_split;                      // the contraction is cut into n_split items of k_chunks chunks each
   float alpha, beta;
   int32_t* status;
+  int batch_fastest;                // 1: consecutive work items are consecutive batches (neighbouring column blocks)
+  int raw_hi;                       // 1: the high part is the raw fp32 word (the tensor core reads its top 19 bits)
 };
 
 __device__ __forceinline__ void load_operand(uint32_t dst, const CUtensorMap* map, const OpCoord& o, int b, int t, int kc,
@@ -63,6 +70,21 @@ __device__ __forceinline__ void load_operand(uint32_t dst, const CUtensorMap* ma
     for (int q = 0; q < 4; ++q) tma_load_2d(dst + q * 4096, map, x + 32 * q, y, bar);
   } else {
     tma_load_2d(dst, map, x, y, bar);
+  }
+}
+
+__device__ __forceinline__ void item_decode(const BParams& p, int item, int& tn, int& tm, int& b, int& ks) {
+  if (p.batch_fastest) {
+    b = item % p.batch;
+    const int rest = item / p.batch;
+    tn = rest % p.n_tiles;
+    tm = (rest / p.n_tiles) % p.m_tiles;
+    ks = rest / (p.n_tiles * p.m_tiles);
+  } else {
+    tn = item % p.n_tiles;
+    tm = (item / p.n_tiles) % p.m_tiles;
+    b = (item / (p.n_tiles * p.m_tiles)) % p.batch;
+    ks = item / (p.n_tiles * p.m_tiles * p.batch);
   }
 }
 
@@ -117,8 +139,8 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       int stage = 0; uint32_t phase = 0; long long issued = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-        const int tn = item % p.n_tiles, tm = (item / p.n_tiles) % p.m_tiles;
-        const int b = (item / (p.n_tiles * p.m_tiles)) % p.batch, ks = item / (p.n_tiles * p.m_tiles * p.batch);
+        int tn, tm, b, ks;
+        item_decode(p, item, tn, tm, b, ks);
         for (int kc = 0; kc < p.k_chunks; ++kc) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abortp, p.status)) { ok = false; break; }
           const uint32_t fb = full0 + 8 * stage;
@@ -194,7 +216,7 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             h.y = __uint_as_float(__float_as_uint(v.y) & 0xffffe000u);
             h.z = __uint_as_float(__float_as_uint(v.z) & 0xffffe000u);
             h.w = __uint_as_float(__float_as_uint(v.w) & 0xffffe000u);
-            hi[idx] = h;
+            if (!p.raw_hi) hi[idx] = h;
             lo[idx] = make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w);
           }
         }
@@ -215,8 +237,8 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     const uint32_t buf_u32 = smem_u32(buf);
     const uint32_t dbar = dfull0 + 8 * q;
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++local) {
-      const int tn = item % p.n_tiles, tm = (item / p.n_tiles) % p.m_tiles;
-      const int b = (item / (p.n_tiles * p.m_tiles)) % p.batch, ks = item / (p.n_tiles * p.m_tiles * p.batch);
+      int tn, tm, b, ks;
+      item_decode(p, item, tn, tm, b, ks);
       const int as = local & 1;
       const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
       const int64_t row_base = p.r_b * b + p.r_s * ks + (int64_t)tm * TILE + q * 32;
@@ -298,6 +320,7 @@ armor_status launch(armor_ctx* c, const HostOp& A, const HostOp& B, BParams p, c
   if (!make_map_2d(&mB, B.base, B.inner, B.outer, B.ld, 32, B.c.mn_major ? 32 : TILE, B.c.mn_major != 0)) return ARMOR_ERR_CUDA;
   p.a = A.c; p.b = B.c;
   p.status = c->status;
+  p.raw_hi = g_tc_raw_hi;
   static bool attr = false;
   if (!attr) {
     if (cudaFuncSetAttribute(tc_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)
@@ -341,6 +364,7 @@ armor_status tc_bd_right(armor_ctx* c, const float* in, const float* Bblk, bool 
   p.m_tiles = (int)((rows + TILE - 1) / TILE); p.n_tiles = db / TILE; p.batch = nb; p.k_chunks = db / BK;
   p.alpha = alpha; p.beta = add ? beta : 0.f;
   p.n_split = 1; p.r_s = 0; p.m_valid = 1 << 30;
+  p.batch_fastest = 1;   // neighbouring CTAs read neighbouring column blocks of the same rows
   return launch(c, A, B, p, s);
 }
 

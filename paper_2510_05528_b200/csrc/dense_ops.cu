@@ -12,7 +12,7 @@ extern "C" void armor_debug_set_k_segment(int64_t k) { K_SEGMENT = k; }
 armor_status prepare_H(armor_ctx* c, const float* H, cudaStream_t s) {
   launch_extract_hblocks(c, H, s);
   if (c->cfg.h_mode == ARMOR_H_FULL && c->cfg.precision == ARMOR_PREC_FP32X3)
-    launch_split_hilo(c, H, c->Hhi, c->Hlo, c->d_in * c->d_in, s);
+    launch_split_hilo(c, H, nullptr, c->Hlo, c->d_in * c->d_in, s);
   return ARMOR_OK;
 }
 
@@ -34,9 +34,10 @@ armor_status rmul_H(armor_ctx* c, const float* in, const float* H, float* out, i
     g.M = rows; g.N = d_in; g.K = d_in;
     g.C = out;
     if (c->cfg.precision == ARMOR_PREC_FP32X3) {
-      // left operand as a tf32-exact high part plus the fp32 remainder
-      launch_split_hilo(c, in, c->LoHi, c->Lo, rows * d_in, s);
-      g.A = c->LoHi; g.Alo = c->Lo; g.B = c->Hhi; g.Blo = c->Hlo; g.passes = 3;
+      // left operand as a high part plus the fp32 remainder.  The tensor core ignores the low 13 bits of a
+      // 32-bit operand, so the operand itself serves as its high part and only the remainder is written.
+      launch_split_hilo(c, in, nullptr, c->Lo, rows * d_in, s);
+      g.A = in; g.Alo = c->Lo; g.B = H; g.Blo = c->Hlo; g.passes = 3;
     } else {
       g.A = in; g.B = H; g.passes = 1;
     }
@@ -116,9 +117,9 @@ armor_status apply_core(armor_ctx* c, const float* z1, const float* S, float* z2
   g.M = n; g.N = d_out; g.K = d_in;
   g.C = z2;
   if (c->cfg.precision == ARMOR_PREC_FP32X3) {
-    launch_split_hilo(c, z1, c->LoHi, c->Lo, n * d_in, s);
-    launch_split_hilo(c, S, c->P, c->U, c->wn, s);
-    g.A = c->LoHi; g.Alo = c->Lo; g.B = c->P; g.Blo = c->U; g.passes = 3;
+    launch_split_hilo(c, z1, nullptr, c->Lo, n * d_in, s);
+    launch_split_hilo(c, S, nullptr, c->U, c->wn, s);
+    g.A = z1; g.Alo = c->Lo; g.B = S; g.Blo = c->U; g.passes = 3;
   } else {
     g.A = z1; g.B = S; g.passes = 1;
   }
