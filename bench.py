@@ -35,8 +35,8 @@ APPLY_TOKENS = 8192
 TF32_OVER_BF16 = 1.1 / 2.25
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes (read + write) of one dense 4096^3 launch of the tensor-core GEMM in FP32X3 mode, from the ncu
-# capture summarised in profiles/ncu_tc_gemm_4096x4096x4096_fp32x3.md (read 768.3 MB + write 158.2 MB)
-GEMM_DRAM_TRAFFIC_BYTES = 926.5e6
+# capture summarised in profiles/ncu_tc_gemm_4096x4096x4096_fp32x3.md (read 772.0 MB + write 162.3 MB)
+GEMM_DRAM_TRAFFIC_BYTES = 934.3e6
 
 
 def load_peaks():
@@ -292,6 +292,34 @@ def run_ours(args, cfg):
     ms_apply, _ = t_phase(lambda: ctx.apply(st, xt_d))
     srec = ctx.read_stats(stats)
 
+    # ---- the one-pass tf32 mode on the same workload (context only; not the headline: its parity tolerance
+    # is looser, see tests/helpers.py)
+    tf32_mode = None
+    if args.precision == "fp32x3" and not args.no_tf32:
+        ctx32 = Bd.ArmorContext(lcfg.d_out, lcfg.d_in, lcfg.d_block, device=dev, precision=Bd.PREC_TF32, seed=lcfg.seed)
+
+        def step32():
+            H.zero_()
+            ctx32.gram(X_d, H)
+            s32 = ctx32.init(W_d, H)
+            ctx32.bcd_step(s32, H, 0, lcfg.n_iters, want_stats=False)
+            l32 = ctx32.proxy_loss(s32, H)
+            ctx32.apply(s32, xt_d)
+            return l32
+        for _ in range(3):
+            step32()
+        Bd.armor_gemm_timing_enable(ctx32.ctx, True)
+        Bd.armor_gemm_timing(ctx32.ctx)
+        ms32 = timed(step32, args.steps)
+        n32, gms32, gfl32 = Bd.armor_gemm_timing(ctx32.ctx)
+        Bd.armor_gemm_timing_enable(ctx32.ctx, False)
+        l32 = step32()
+        tf32_mode = {"ms_per_step": ms32 / args.steps, "iterations_per_s": world * lcfg.n_iters / (ms32 / args.steps / 1e3),
+                     "final_loss": float(l32.item()),
+                     "gemm_tflops": gfl32 / (gms32 * 1e-3) / 1e12 if gms32 > 0 else None,
+                     "gemm_share_of_step": gms32 / ms32 if ms32 > 0 else None}
+        del ctx32
+
     # ---- end to end (host buffers)
     if args.no_e2e:
         ms_e2e = None
@@ -326,6 +354,7 @@ def run_ours(args, cfg):
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                 "ms_per_step": ms_e2e / args.steps if ms_e2e else None},
         "gpu_launches": int(launches),
+        "tf32_mode": tf32_mode,
         "clocks": clocks,
         "roofline": {"bound": "tensor", "kernel": "tc_gemm_kernel (tcgen05 tf32, Gram + dense .H contractions)",
                      "achieved": achieved, "peak": tf32_peak, "unit": "TFLOP/s", "frac": achieved / tf32_peak,
@@ -360,6 +389,7 @@ def main():
     ap.add_argument("--iters", type=int, default=0,
                     help="profiling aid: BCD iterations per step instead of the workload's")
     ap.add_argument("--no-e2e", action="store_true", help="profiling aid: skip the host-buffer leg")
+    ap.add_argument("--no-tf32", action="store_true", help="skip the extra measurement of the one-pass tf32 mode")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

@@ -174,6 +174,20 @@ int64_t armor_launch_count(const armor_ctx* ctx);
 armor_status armor_gemm_timing_enable(armor_ctx* ctx, int32_t enable);
 armor_status armor_gemm_timing(armor_ctx* ctx, int64_t* n_launches, double* total_ms, double* total_flops);
 
+/* One product with a block-diagonal wrapper (Section 3.1: A and B are applied as batched d_block x d_block
+ * products), exposed for tests and measurements; armor_bcd_step and armor_apply are built from it.
+ *   side 0: d_out[:, j-th block] = alpha * d_in[:, j-th block] * Q_j (+ beta * d_add[:, j-th block])
+ *   side 1: d_out[i-th block, :] = alpha * Q_i * d_in[i-th block, :] (+ beta * d_add[i-th block, :])
+ * with Q = d_blocks [n_blocks, d_block, d_block] or, if transpose != 0, its blocks transposed.  d_in, d_out,
+ * d_add (may be NULL; may equal d_out) are [rows, cols] fp32; d_in must not overlap d_out.  path 0: fp32
+ * CUDA-core kernel; path 1: tensor-core kernel (tcgen05, operands split in shared memory into tf32 high and
+ * low parts, three passes; needs d_block a multiple of 128 and a tensor-core precision, else UNSUPPORTED);
+ * any other value: what the library itself would use.  Errors: INVALID_ARG, SHAPE (the blocked dimension is
+ * not a multiple of d_block, or cols is not a multiple of 4). */
+armor_status armor_block_product(armor_ctx* ctx, int32_t side, int32_t transpose, const float* d_blocks,
+                                 const float* d_in, float* d_out, int64_t rows, int64_t cols, float alpha,
+                                 const float* d_add, float beta, int32_t path, armor_stream_t stream);
+
 /* The paper has no counterpart to this entry point; it exists for deployment reasons only.
  *
  * armor_normalize_noalloc computes the same row/column normalisation that armor_init applies when

@@ -26,7 +26,7 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 EXPORTS = ["armor_workspace_bytes", "armor_create", "armor_destroy", "armor_gram", "armor_init",
            "armor_bcd_step", "armor_proxy_loss", "armor_apply", "armor_get_device_status",
            "armor_status_string", "armor_launch_count", "armor_gemm_timing_enable", "armor_gemm_timing",
-           "armor_normalize_noalloc"]
+           "armor_normalize_noalloc", "armor_block_product"]
 
 
 class ArmorError(RuntimeError):
@@ -72,6 +72,7 @@ def lib() -> C.CDLL:
         L.armor_launch_count.argtypes = [vp]
         L.armor_launch_count.restype = i64
         L.armor_normalize_noalloc.argtypes = [vp, i64, i64, vp, vp, vp, vp]
+        L.armor_block_product.argtypes = [vp, i32, i32, vp, vp, vp, i64, i64, C.c_float, vp, C.c_float, i32, vp]
         L.armor_gemm_timing_enable.argtypes = [vp, i32]
         L.armor_gemm_timing.argtypes = [vp, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
         for name in EXPORTS:
@@ -190,6 +191,14 @@ def armor_normalize_noalloc(W: torch.Tensor, Wbar: torch.Tensor, r1: torch.Tenso
         raise ValueError("W must be [d_out, d_in]")
     _check(lib().armor_normalize_noalloc(_ptr(W, f, "W"), W.shape[0], W.shape[1], _ptr(Wbar, f, "Wbar"),
                                          _ptr(r1, f, "r1"), _ptr(r2, f, "r2"), _stream()), "armor_normalize_noalloc")
+
+
+def armor_block_product(ctx, side: int, transpose: bool, blocks, x, out, alpha=1.0, add=None, beta=0.0, path=-1) -> None:
+    """out = alpha * (x . Q or Q . x) + beta * add with the block-diagonal Q (see armor.h)."""
+    f = torch.float32
+    _check(lib().armor_block_product(ctx, int(side), int(bool(transpose)), _ptr(blocks, f, "blocks"), _ptr(x, f, "x"),
+                                     _ptr(out, f, "out"), x.shape[0], x.shape[1], float(alpha), _ptr(add, f, "add"),
+                                     float(beta), int(path), _stream()), "armor_block_product")
 
 
 def armor_gemm_timing_enable(ctx, enable: bool) -> None:

@@ -24,7 +24,6 @@
 // The tensor core reads the top 19 bits of a 32-bit tf32 operand and ignores the rest, so the raw fp32 word
 // serves as the high part and only the low part has to be written (checked against the masked form: same bits).
 int g_tc_raw_hi = 1;
-extern "C" void armor_debug_set_tc_raw_hi(int on) { g_tc_raw_hi = on; }
 
 namespace {
 

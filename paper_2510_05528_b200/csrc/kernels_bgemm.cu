@@ -303,7 +303,6 @@ void launch_bgemm(armor_ctx* c, const BGemm& g_in, cudaStream_t s) {
 
 // 1: block-diagonal products on the tensor cores where the shape allows; 0: always the fp32 CUDA-core kernels
 int g_tc_blocks = 1;
-extern "C" void armor_debug_set_tc_blocks(int on) { g_tc_blocks = on; }
 
 void bd_right(armor_ctx* c, const float* in, const float* Bblk, bool transB, float* out, int64_t rows,
               int64_t cols, float alpha, const float* add, float beta, cudaStream_t s) {
@@ -339,13 +338,18 @@ void bd_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, floa
   launch_bgemm(c, g, s);
 }
 
-// Test hook: one block-diagonal product through whichever path is switched on.
-extern "C" int armor_debug_block_product(armor_ctx* c, int left, int trans, const float* blk, const float* in,
-                                         float* out, int64_t rows, int64_t cols, float alpha, const float* add,
-                                         float beta, void* stream) {
-  if (!c) return ARMOR_ERR_INVALID_ARG;
+extern "C" armor_status armor_block_product(armor_ctx* c, int32_t side, int32_t transpose, const float* d_blocks,
+                                            const float* d_in, float* d_out, int64_t rows, int64_t cols, float alpha,
+                                            const float* d_add, float beta, int32_t path, armor_stream_t stream) {
+  if (!c || !d_blocks || !d_in || !d_out || rows <= 0 || cols <= 0) return ARMOR_ERR_INVALID_ARG;
+  if (side != 0 && side != 1) return ARMOR_ERR_INVALID_ARG;
+  if (cols % 4 || (side == 0 ? cols : rows) % c->db) return ARMOR_ERR_SHAPE;
+  if (path == 1 && !tc_block_ok(c, rows, cols)) return ARMOR_ERR_UNSUPPORTED;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-  if (left) bd_left(c, blk, trans != 0, in, out, rows, cols, alpha, add, beta, s);
-  else bd_right(c, in, blk, trans != 0, out, rows, cols, alpha, add, beta, s);
+  const int saved = g_tc_blocks;
+  g_tc_blocks = (path != 0);
+  if (side == 1) bd_left(c, d_blocks, transpose != 0, d_in, d_out, rows, cols, alpha, d_add, beta, s);
+  else bd_right(c, d_in, d_blocks, transpose != 0, d_out, rows, cols, alpha, d_add, beta, s);
+  g_tc_blocks = saved;
   return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
 }

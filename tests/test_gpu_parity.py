@@ -421,3 +421,30 @@ def test_apply_with_bf16_activations(mid_data):
         yo = O.apply(A, B, S, xr, r1, r2)
         # one rounding to bf16 (2^-9 relative per element) on the way out
         assert rel(y.float().cpu().numpy(), yo) < 3e-3
+
+
+# ------------------------------------------------------------------------------------------ block products
+@pytest.mark.parametrize("db", [128, 256])
+@pytest.mark.parametrize("side,transpose", [(0, False), (0, True), (1, False), (1, True)])
+def test_block_products_on_both_paths(db, side, transpose):
+    """The products with a block-diagonal wrapper, CUDA-core and tensor-core kernels, against the oracle's
+    definition: all four operand layouts, with and without the fused addend, in place, and a ragged row count
+    on the right product (token batches of the forward)."""
+    rng = np.random.default_rng(db + 2 * side + int(transpose))
+    rows, cols = (512, 768) if side == 1 else (200, 768)
+    ctx = Bd.ArmorContext(512, 768, db, device=DEV, precision=Bd.PREC_FP32X3)
+    nb = (rows if side == 1 else cols) // db
+    Q = rng.standard_normal((nb, db, db))
+    X = rng.standard_normal((rows, cols))
+    D = rng.standard_normal((rows, cols))
+    Qe = np.ascontiguousarray(np.transpose(Q, (0, 2, 1))) if transpose else Q
+    ref = O.bd_left(Qe, X) if side == 1 else O.bd_right(X, Qe)
+    Qd, Xd = dev(Q), dev(X)
+    for path, tol in ((0, 2e-6), (1, 1e-5)):
+        out = torch.full((rows, cols), 7.0, device=DEV)
+        Bd.armor_block_product(ctx.ctx, side, transpose, Qd, Xd, out, path=path)
+        assert rel(host(out), ref) < tol
+        out = dev(D)                                   # addend in place: out = 1.5 * product - 0.5 * out
+        Bd.armor_block_product(ctx.ctx, side, transpose, Qd, Xd, out, alpha=1.5, add=out, beta=-0.5, path=path)
+        assert rel(host(out), 1.5 * ref - 0.5 * D) < tol
+    assert ctx.device_status()[:4] == [0, 0, 0, 0]
