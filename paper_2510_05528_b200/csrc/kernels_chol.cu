@@ -175,36 +175,38 @@ chol_blocked_kernel(int mode, const float* __restrict__ Gmat, const float* __res
       }
       __syncthreads();
     }
-    // diagonal block: warp 0, lane i owns row i of the copy in shared memory and the warp eliminates column
-    // by column (right-looking), so that every dependent chain is one multiply-add long
+    // diagonal block: warp 0, lane i keeps row i in registers and the warp eliminates column by column
+    // (right-looking); the entries of the pivot column come from the other lanes by shuffle, so nothing in the
+    // chain goes through memory
     if (tid < 32) {
-#pragma unroll 4
-      for (int j = 0; j < NB; ++j) Df[lane][j] = (j <= lane) ? P[lane * LDP + j] : 0.f;
-      __syncwarp();
+      float arow[NB];
+#pragma unroll
+      for (int j = 0; j < NB; ++j) arow[j] = (j <= lane) ? P[lane * LDP + j] : 0.f;
       bool bad = false;
+#pragma unroll
       for (int k = 0; k < NB; ++k) {
-        const float akk = Df[k][k];
+        const float akk = __shfl_sync(0xffffffffu, arow[k], k);
         bad |= !(akk > 0.f) | !isfinite(akk);
         // 1 / sqrt(a): hardware estimate refined by one Newton step
         float inv = rsqrtf(akk);
         inv = inv * fmaf(-0.5f * akk * inv, inv, 1.5f);
-        const float lik = (lane == k) ? akk * inv : Df[lane][k] * inv;
-        __syncwarp();
-        if (lane >= k) Df[lane][k] = lik;
+        const float lik = (lane == k) ? akk * inv : arow[k] * inv;
+        arow[k] = lik;
         if (lane == k) invd[k] = inv;
-        __syncwarp();
-#pragma unroll 4
+#pragma unroll
         for (int j = k + 1; j < NB; ++j) {
-          const float ljk = Df[j][k];
-          if (lane >= j) Df[lane][j] = fmaf(-lik, ljk, Df[lane][j]);
+          const float ljk = __shfl_sync(0xffffffffu, lik, j);
+          arow[j] = fmaf(-lik, ljk, arow[j]);      // entries above the diagonal (j > lane) are never used
         }
-        __syncwarp();
       }
       if (bad) {
         if (lane == 0) s_fail = 1;
       } else {
-#pragma unroll 4
-        for (int j = 0; j <= lane; ++j) P[lane * LDP + j] = Df[lane][j];
+#pragma unroll
+        for (int j = 0; j < NB; ++j) {
+          Df[lane][j] = (j <= lane) ? arow[j] : 0.f;
+          if (j <= lane) P[lane * LDP + j] = arow[j];
+        }
       }
     }
     __syncthreads();
