@@ -339,7 +339,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       rowblock_grams(c, c->P, c->EH, c->T, c->G, c->GamA, s);   // G_i = T_i H_w T_i^T, Gamma_i = E_i H_w T_i^T
       st = launch_chol(c, 0, c->G, c->GamA, c->dA, nullptr, A, c->At, nbo, c->partblk, s);
       if (st != ARMOR_OK) return st;
-      launch_stage(c, is, 1, c->partblk, nbo * chol_parts_per_block(db), nbo, s);
+      launch_stage(c, is, 1, c->partblk, nbo * chol_parts_per_block(db, nbo), nbo, s);
       bd_left(c, c->dA, false, c->P, c->EH, d_out, d_in, -1.f, c->EH, 1.f, s);       // EH -= dA P
     } else {
       launch_stage(c, is, 1, nullptr, 0, 0, s);
@@ -357,7 +357,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       bd_right(c, c->U, c->Delta, false, c->V, d_out, d_in, 1.f, nullptr, 0.f, s);   // V = U Delta
       st = rmul_H(c, c->V, H, c->VH, d_out, c->V, c->sc + SC_Q_B, nullptr, nullptr, s);
       if (st != ARMOR_OK) return st;
-      launch_stage(c, is, 2, c->partblk, nbi * chol_parts_per_block(db), nbi, s);
+      launch_stage(c, is, 2, c->partblk, nbi * chol_parts_per_block(db, nbi), nbi, s);
       launch_axpy_slot(c, B, c->Delta, (int64_t)nbi * db * db, SC_TAU_B, 1.f, s);    // B += tau Delta
       launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_B, -1.f, s);                   // EH -= tau V H_w
     } else {

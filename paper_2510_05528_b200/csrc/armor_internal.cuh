@@ -191,7 +191,7 @@ void launch_f32_to_bf16(armor_ctx* c, const float* in, const float* colscale, vo
 // mode 1: out = (G + lam I)^-1 rhs
 // mode 2: out = rhs (G + lam I)^-1, part[b] = <dotw, out>
 // partial sums written per block by launch_chol (modes 0 and 2)
-int chol_parts_per_block(int db);
+int chol_parts_per_block(int db, int nb);
 armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float* rhs, float* out, const float* dotw,
                          float* A, float* At, int nb, double* part, cudaStream_t s);
 

@@ -507,13 +507,21 @@ __global__ void chol_kernel(int mode, const float* __restrict__ Gmat, const floa
 
 }  // namespace
 
-int chol_parts_per_block(int db) { return (db % NB == 0 && db > 128) ? db / 64 : 1; }
+// Right-hand sides of one block are split over this many CTAs (each repeats the factorisation).  d_block 256
+// needs 4 for its shared memory; smaller blocks are split while that still fits one wave of CTAs.
+int chol_parts_per_block(int db, int nb) {
+  if (db % NB) return 1;
+  if (db > 128) return db / 64;
+  int parts = 1;
+  while (parts < 4 && 2 * parts * nb <= 148 && db / (2 * parts) >= 32) parts *= 2;
+  return parts;
+}
 
 armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float* rhs, float* out, const float* dotw,
                          float* A, float* At, int nb, double* part, cudaStream_t s) {
   const int db = c->db;
   if (db % NB == 0) {
-    const int slices = chol_parts_per_block(db);
+    const int slices = chol_parts_per_block(db, nb);
     const int w = db / slices;
     const size_t smem = (panel_floats(db) + (size_t)db * (w + 1)) * sizeof(float);
     static size_t attr_bytes = 0;
