@@ -181,6 +181,7 @@ void launch_scale_rows_cols(armor_ctx* c, const float* in, const float* colscale
 void launch_split_hilo(armor_ctx* c, const float* in, float* hi, float* lo, int64_t n, cudaStream_t s);
 void launch_transpose_split(armor_ctx* c, const void* X, int x_dtype, int64_t ldx, int64_t rows, int64_t cols,
                             float* Thi, float* Tlo, int64_t ldt, cudaStream_t s);
+void launch_mirror_lower(armor_ctx* c, float* H, int64_t n, cudaStream_t s);
 void launch_bf16_to_f32(armor_ctx* c, const void* in, const float* colscale, float* out, int64_t rows, int64_t cols,
                         cudaStream_t s);
 void launch_f32_to_bf16(armor_ctx* c, const float* in, const float* colscale, void* out, int64_t rows, int64_t cols,
@@ -215,7 +216,7 @@ struct TcGemm {
   int passes;            // 1 or 3
   int64_t k_segment;     // K extent accumulated in tensor memory before it is folded into C (0: all of K)
   int accumulate;        // C += (read-modify-write) instead of C =
-  int symmetric_lower;   // only tiles with n0 <= m0 are computed; mirrored into the upper triangle (M == N)
+  int symmetric_lower;   // only the lower triangle (tiles with n0 <= m0, elements with column <= row) is computed (M == N)
   const float* d1; const float* d2;  // optional dot operands (ld = ldc)
   double* part1; double* part2;      // [tiles] partial sums
 };

@@ -98,6 +98,7 @@ armor_status gram_accumulate(armor_ctx* c, const void* Xv, int x_dtype, int64_t 
     armor_status st = launch_tc_gemm(c, g, nullptr, s);
     if (st != ARMOR_OK) return st;
   }
+  launch_mirror_lower(c, H, d_in, s);   // the product accumulates the lower triangle only
   return ARMOR_OK;
 }
 

@@ -8,7 +8,8 @@
 //   warp 0   : TMA producer  (cp.async.bulk.tensor.2d, 128-byte swizzle, mbarrier complete_tx)
 //   warp 1   : MMA issuer    (one thread issues tcgen05.mma kind::tf32, 128 x 256 x 8 per instruction,
 //                             accumulators in tensor memory, two accumulator buffers of 256 columns)
-//   warps 2-5: epilogue      (tcgen05.ld 32 lanes x 32 columns, fused C-update / mirror / dot products)
+//   warps 2-5: epilogue      (tcgen05.ld 32 lanes x 32 columns, fused C-update / dot products; a symmetric
+//                             product writes its lower triangle only, the caller mirrors it once at the end)
 // passes == 3: every operand is given as a tf32-exact high part and an fp32 low part; the three products
 // hi*hi, lo*hi, hi*lo are accumulated into the same fp32 accumulator (error-compensated tf32, fp32-grade).
 // Every wait is bounded: a wait that runs out raises a status word and the CTA leaves through the common
@@ -21,6 +22,7 @@ using namespace tc;
 
 constexpr int BM = 128, BN = 256, BK = 32;          // BK fp32 = 128 bytes = one swizzle row
 constexpr int NTHREADS = 192;
+constexpr int RB = 16;                              // rows of C an epilogue lane keeps in flight
 constexpr uint32_t TMEM_COLS = 512;                 // two accumulator buffers of BN columns
 constexpr int A_BYTES = BM * BK * 4;                // 16 KiB
 constexpr int B_BYTES = BN * BK * 4;                // 32 KiB
@@ -194,8 +196,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     for (int tile = blockIdx.x; tile < p.n_tiles_total && ok; tile += gridDim.x) {
       int mt, nt;
       tile_coords(p, tile, mt, nt);
-      const int64_t row = (int64_t)mt * BM + q * 32 + lane;
-      const bool row_ok = row < p.M;
       double dot1 = 0.0, dot2 = 0.0;
       for (int kt0 = 0; kt0 < kt_total && ok; kt0 += p.kt_seg, ++local) {
         const int as = local & 1;
@@ -221,11 +221,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
           const int64_t col = col0 + lane;
           float f1 = 0.f, f2 = 0.f;
 #pragma unroll 1
-          for (int r0 = 0; r0 < 32; r0 += 8) {
-            float x[8], o[8];
-            bool keep[8];
+          for (int r0 = 0; r0 < 32; r0 += RB) {
+            float x[RB], o[RB];
+            bool keep[RB];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
+            for (int j = 0; j < RB; ++j) {
               const int64_t grow = row_base + r0 + j;
               keep[j] = grow < p.M && (!p.symmetric_lower || col <= grow);
               x[j] = tilebuf[(r0 + j) * 33 + lane];
@@ -233,39 +233,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
             }
             if (last && p.d1) {
 #pragma unroll
-              for (int j = 0; j < 8; ++j)
+              for (int j = 0; j < RB; ++j)
                 if (keep[j]) f1 = fmaf(x[j] + o[j], p.d1[(row_base + r0 + j) * p.ldc + col], f1);
             }
             if (last && p.d2) {
 #pragma unroll
-              for (int j = 0; j < 8; ++j)
+              for (int j = 0; j < RB; ++j)
                 if (keep[j]) f2 = fmaf(x[j] + o[j], p.d2[(row_base + r0 + j) * p.ldc + col], f2);
             }
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
+            for (int j = 0; j < RB; ++j)
               if (keep[j]) p.C[(row_base + r0 + j) * p.ldc + col] = x[j] + o[j];
           }
           dot1 += (double)f1;
           dot2 += (double)f2;
           __syncwarp();
-          if (p.symmetric_lower && row_ok) {
-            // mirror of the strictly lower part, straight from the registers: for a fixed column the lanes
-            // hold consecutive rows, so C[col][row ..] is one contiguous segment
-#pragma unroll
-            for (int c0 = 0; c0 < 32; c0 += 8) {
-              float o[8];
-#pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                const int64_t gcol = col0 + c0 + j;
-                o[j] = (accum && gcol < row) ? p.C[gcol * p.ldc + row] : 0.f;
-              }
-#pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                const int64_t gcol = col0 + c0 + j;
-                if (gcol < row) p.C[gcol * p.ldc + row] = __uint_as_float(r[c0 + j]) + o[j];
-              }
-            }
-          }
         }
         // accumulator buffer is free again
         tc_fence_before();

@@ -355,6 +355,23 @@ __global__ void __launch_bounds__(NT) f32_to_bf16_kernel(const float* __restrict
   }
 }
 
+// H[r][c] = H[c][r] for c > r: the upper triangle from the lower one, 32 x 32 tiles through shared memory
+__global__ void mirror_lower_kernel(float* __restrict__ H, int64_t n) {
+  if (blockIdx.x < blockIdx.y) return;   // blockIdx.x: tile column of the destination, blockIdx.y: its tile row
+  __shared__ float tile[32][33];
+  const int64_t c0 = (int64_t)blockIdx.x * 32, r0 = (int64_t)blockIdx.y * 32;
+  // source tile: rows c0.., columns r0..
+  for (int j = threadIdx.y; j < 32; j += blockDim.y) {
+    const int64_t sr = c0 + j, sc = r0 + threadIdx.x;
+    tile[j][threadIdx.x] = (sr < n && sc < n) ? H[sr * n + sc] : 0.f;
+  }
+  __syncthreads();
+  for (int j = threadIdx.y; j < 32; j += blockDim.y) {
+    const int64_t dr = r0 + j, dc = c0 + threadIdx.x;
+    if (dr < n && dc < n && dc > dr) H[dr * n + dc] = tile[threadIdx.x][j];
+  }
+}
+
 inline int grid_for(int64_t n) {
   int64_t b = (n + NT - 1) / NT;
   return (int)(b < 1 ? 1 : (b > 148 * 16 ? 148 * 16 : b));
@@ -464,6 +481,12 @@ void launch_transpose_split(armor_ctx* c, const void* X, int x_dtype, int64_t ld
                                                        (float*)nullptr, ldt);
   else
     transpose_split_kernel<<<grid, dim3(32, 8), 0, s>>>(static_cast<const float*>(X), ldx, rows, cols, Thi, Tlo, ldt);
+  c->launches++;
+}
+
+void launch_mirror_lower(armor_ctx* c, float* H, int64_t n, cudaStream_t s) {
+  const unsigned t = (unsigned)((n + 31) / 32);
+  mirror_lower_kernel<<<dim3(t, t), dim3(32, 8), 0, s>>>(H, n);
   c->launches++;
 }
 
