@@ -86,9 +86,11 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   if (c) c->nbo_pad = (int)nbo_pad;
   TAKE(colpart, double*, (size_t)64 * cfg.d_in * sizeof(double));
   if (tc) {
+    TAKE(gemm_slabs, float*, (size_t)160 * 128 * 256 * sizeof(float));
+    if (c) c->gemm_slab_count = 160;
     TAKE(Xt_hi, float*, (size_t)cfg.d_in * GRAM_ROWS * sizeof(float));
     if (x3) TAKE(Xt_lo, float*, (size_t)cfg.d_in * GRAM_ROWS * sizeof(float)); else if (c) c->Xt_lo = nullptr;
-  } else if (c) { c->Xt_hi = nullptr; c->Xt_lo = nullptr; }
+  } else if (c) { c->Xt_hi = nullptr; c->Xt_lo = nullptr; c->gemm_slabs = nullptr; c->gemm_slab_count = 0; }
   const int64_t tiles = ((cfg.d_out + 127) / 128) * ((cfg.d_in + 127) / 128) + ((cfg.d_in + 127) / 128) * ((cfg.d_in + 127) / 128);
   const int64_t npart = tiles > ARMOR_DOT_BLOCKS ? tiles : ARMOR_DOT_BLOCKS;
   {

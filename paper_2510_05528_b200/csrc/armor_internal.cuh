@@ -59,6 +59,8 @@ struct armor_ctx {
   float *G, *GamA, *dA, *At, *C, *GamB, *Delta, *Hjj, *Kfull, *Ktmp, *Bt;
   float *alpha, *hdiag;
   float *Hq1, *Hq2;      // [d_in, d_in] scratch of the paper's step size (s_step BETA, full weighting)
+  float* gemm_slabs;     // 128 x 256 slabs of partial sums of the dense product's split tail tiles
+  int64_t gemm_slab_count;
   float* gpart;          // partial products of split contractions
   int64_t gpart_floats;
   // sparse-core update: per selected group z = delta^T B_j[rows of the group, :] and a = A_i[:, r]

@@ -36,6 +36,11 @@ struct Params {
   const float* d1; const float* d2;
   double* part1; double* part2;
   int32_t* status;
+  // Tail split: tiles [split_first, n_tiles_total) are cut into split_parts pieces along K, each piece a work
+  // item of its own that writes a 128 x 256 slab of partial sums; a second kernel adds the slabs.  This fills
+  // the last, partly empty wave of tiles.
+  int split_first, split_parts, n_items;
+  float* slabs;
 };
 
 // K-major operand tile, rows of 128 bytes, 128-byte swizzle: 8-row groups are 1024 bytes apart.
@@ -75,6 +80,20 @@ __device__ __forceinline__ void tile_coords(const Params& p, int tile, int& mt, 
     rem -= cnt;
   }
   mt = 2 * nt + rem;
+}
+
+// work item -> tile, and its range of k-tiles
+__device__ __forceinline__ void item_decode(const Params& p, int item, int kt_total, int& tile, int& part, int& kt_begin,
+                                            int& kt_end) {
+  if (item < p.split_first) {
+    tile = item; part = -1; kt_begin = 0; kt_end = kt_total;
+  } else {
+    const int idx = item - p.split_first;
+    tile = p.split_first + idx / p.split_parts;
+    part = idx % p.split_parts;
+    const int per = kt_total / p.split_parts;
+    kt_begin = part * per; kt_end = kt_begin + per;
+  }
 }
 
 template <int PASSES>
@@ -118,10 +137,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0; long long issued = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < p.n_tiles_total && ok; tile += gridDim.x) {
-        int mt, nt;
+      for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
+        int tile, part, kt_begin, kt_end, mt, nt;
+        item_decode(p, item, kt_total, tile, part, kt_begin, kt_end);
         tile_coords(p, tile, mt, nt);
-        for (int kt = 0; kt < kt_total; ++kt) {
+        for (int kt = kt_begin; kt < kt_end; ++kt) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abortp, p.status)) { ok = false; break; }
           const uint32_t fb = full0 + 8 * stage;
           mbar_expect_tx(fb, STAGE_BYTES);
@@ -153,14 +173,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
       int stage = 0; uint32_t phase = 0;
       int local = 0;   // (tile, K segment) items handled so far: selects the accumulator buffer
       bool ok = true;
-      for (int tile = blockIdx.x; tile < p.n_tiles_total && ok; tile += gridDim.x) {
-        for (int kt0 = 0; kt0 < kt_total && ok; kt0 += p.kt_seg, ++local) {
+      for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
+        int tile, part, kt_begin, kt_end;
+        item_decode(p, item, kt_total, tile, part, kt_begin, kt_end);
+        for (int kt0 = kt_begin; kt0 < kt_end && ok; kt0 += p.kt_seg, ++local) {
           const int as = local & 1;
           const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
           if (!mbar_wait(tempty0 + 8 * as, aphase ^ 1, abortp, p.status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t tacc = tmem_base + (uint32_t)(as * BN);
-          const int kt1 = min(kt_total, kt0 + p.kt_seg);
+          const int kt1 = min(kt_end, kt0 + p.kt_seg);
           for (int kt = kt0; kt < kt1; ++kt) {
             if (!mbar_wait(full0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
             tc_fence_after();
@@ -193,9 +215,46 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     int local = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < p.n_tiles_total && ok; tile += gridDim.x) {
-      int mt, nt;
+    for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
+      int tile, part, kt_begin, kt_end, mt, nt;
+      item_decode(p, item, kt_total, tile, part, kt_begin, kt_end);
       tile_coords(p, tile, mt, nt);
+      if (part >= 0) {
+        // a piece of a split tile: its partial sums go, plainly, to this item's slab
+        float* slab = p.slabs + ((int64_t)(tile - p.split_first) * p.split_parts + part) * (BM * BN);
+        float* tilebuf = reinterpret_cast<float*>(smem + (size_t)STAGES * STAGE_BYTES) + q * (32 * 33);
+        for (int kt0 = kt_begin; kt0 < kt_end && ok; kt0 += p.kt_seg, ++local) {
+          const int as = local & 1;
+          const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
+          if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
+          tc_fence_after();
+#pragma unroll 1
+          for (int ch = 0; ch < BN / 32; ++ch) {
+            uint32_t r[32];
+            tmem_ld32(tmem_base + (uint32_t)(as * BN + ch * 32) + ((uint32_t)(q * 32) << 16), r);
+#pragma unroll
+            for (int cidx = 0; cidx < 32; ++cidx) tilebuf[lane * 33 + cidx] = __uint_as_float(r[cidx]);
+            __syncwarp();
+            float* dst = slab + (int64_t)(q * 32) * BN + ch * 32 + lane;
+#pragma unroll 1
+            for (int r0 = 0; r0 < 32; r0 += RB) {
+              float x[RB], o[RB];
+#pragma unroll
+              for (int j = 0; j < RB; ++j) {
+                x[j] = tilebuf[(r0 + j) * 33 + lane];
+                o[j] = (kt0 > kt_begin) ? dst[(int64_t)(r0 + j) * BN] : 0.f;
+              }
+#pragma unroll
+              for (int j = 0; j < RB; ++j) dst[(int64_t)(r0 + j) * BN] = x[j] + o[j];
+            }
+            __syncwarp();
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(tempty0 + 8 * as);
+        }
+        continue;
+      }
       double dot1 = 0.0, dot2 = 0.0;
       for (int kt0 = 0; kt0 < kt_total && ok; kt0 += p.kt_seg, ++local) {
         const int as = local & 1;
@@ -274,6 +333,53 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
   }
 }
 
+// Adds the slabs of every split tile into C (+ what C held, if the product accumulates) and forms the tile's
+// share of the fused dot products.  Four CTAs per split tile (32 rows each); fixed order.
+__global__ void __launch_bounds__(256) tc_gemm_fixup_kernel(const Params p) {
+  const int tile = p.split_first + blockIdx.x / 4, qq = blockIdx.x % 4;
+  int mt, nt;
+  tile_coords(p, tile, mt, nt);
+  const float* slab0 = p.slabs + (int64_t)(blockIdx.x / 4) * p.split_parts * (BM * BN);
+  double d1 = 0.0, d2 = 0.0;
+  for (int e = threadIdx.x; e < 32 * BN / 4; e += 256) {
+    const int r = qq * 32 + e / (BN / 4), c4 = (e % (BN / 4)) * 4;
+    const int64_t grow = (int64_t)mt * BM + r, gcol = (int64_t)nt * BN + c4;
+    if (grow >= p.M || gcol >= p.N) continue;
+    float4 v = *reinterpret_cast<const float4*>(slab0 + (int64_t)r * BN + c4);
+    for (int k = 1; k < p.split_parts; ++k) {
+      const float4 w = *reinterpret_cast<const float4*>(slab0 + (int64_t)k * (BM * BN) + (int64_t)r * BN + c4);
+      v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
+    }
+    float* cp = p.C + grow * p.ldc + gcol;
+    if (p.accumulate) {
+      const float4 o = *reinterpret_cast<const float4*>(cp);
+      v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+    }
+    *reinterpret_cast<float4*>(cp) = v;
+    if (p.d1) {
+      const float4 w = *reinterpret_cast<const float4*>(p.d1 + grow * p.ldc + gcol);
+      d1 += (double)(v.x * w.x + v.y * w.y) + (double)(v.z * w.z + v.w * w.w);
+    }
+    if (p.d2) {
+      const float4 w = *reinterpret_cast<const float4*>(p.d2 + grow * p.ldc + gcol);
+      d2 += (double)(v.x * w.x + v.y * w.y) + (double)(v.z * w.z + v.w * w.w);
+    }
+  }
+  __shared__ double red1[8], red2[8];
+  for (int o = 16; o > 0; o >>= 1) {
+    d1 += __shfl_down_sync(0xffffffffu, d1, o);
+    d2 += __shfl_down_sync(0xffffffffu, d2, o);
+  }
+  if ((threadIdx.x & 31) == 0) { red1[threadIdx.x >> 5] = d1; red2[threadIdx.x >> 5] = d2; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t1 = 0.0, t2 = 0.0;
+    for (int w = 0; w < 8; ++w) { t1 += red1[w]; t2 += red2[w]; }
+    if (p.part1) p.part1[(int64_t)tile * 4 + qq] = t1;
+    if (p.part2) p.part2[(int64_t)tile * 4 + qq] = t2;
+  }
+}
+
 // ------------------------------------------------------------------ host side
 // [rows][K] fp32, leading dimension ld: box = BK x box_rows, 128-byte swizzle, zero fill out of bounds.
 bool make_map(CUtensorMap* map, const float* base, int64_t rows, int64_t K, int64_t ld, int box_rows) {
@@ -290,7 +396,7 @@ bool make_map(CUtensorMap* map, const float* base, int64_t rows, int64_t K, int6
 }
 
 template <int PASSES>
-armor_status launch_impl(armor_ctx* c, const TcGemm& g, const Params& p, cudaStream_t s) {
+armor_status launch_impl(armor_ctx* c, const TcGemm& g, Params p, cudaStream_t s) {
   CUtensorMap mA, mAlo, mB, mBlo;
   if (!make_map(&mA, g.A, g.M, g.K, g.lda, BM)) return ARMOR_ERR_CUDA;
   if (!make_map(&mB, g.B, g.N, g.K, g.ldb, BN)) return ARMOR_ERR_CUDA;
@@ -316,10 +422,31 @@ armor_status launch_impl(armor_ctx* c, const TcGemm& g, const Params& p, cudaStr
     if (cudaGetDevice(&dev) != cudaSuccess) return ARMOR_ERR_CUDA;
     if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ARMOR_ERR_CUDA;
   }
-  const int grid = p.n_tiles_total < n_sm ? p.n_tiles_total : n_sm;
+  // tail split: the tiles of the last, partly filled wave are cut along K so that their pieces fill the wave
+  p.split_first = p.n_tiles_total; p.split_parts = 1; p.n_items = p.n_tiles_total; p.slabs = c->gemm_slabs;
+  const int kt_total = (int)((p.K + BK - 1) / BK);
+  const int rem = p.n_tiles_total % n_sm;
+  if (c->gemm_slabs && !p.symmetric_lower && rem > 0 && p.ldc % 4 == 0 && p.N % 4 == 0) {
+    int parts = n_sm / rem;
+    if (parts > 4) parts = 4;
+    // a piece must be whole K segments (or lie inside one) so that issuer and epilogue agree on the segments
+    while (parts > 1 && (kt_total % parts || kt_total / parts < 8 ||
+                         ((kt_total / parts) % p.kt_seg && p.kt_seg < kt_total / parts)))
+      --parts;
+    if (parts > 1 && (int64_t)rem * parts <= c->gemm_slab_count) {
+      p.split_first = p.n_tiles_total - rem;
+      p.split_parts = parts;
+      p.n_items = p.split_first + rem * parts;
+    }
+  }
+  const int grid = p.n_items < n_sm ? p.n_items : n_sm;
   const bool timed = c->timing_on && c->timing_n < ARMOR_MAX_TIMED;
   if (timed) cudaEventRecord(c->ev_beg[c->timing_n], s);
   tc_gemm_kernel<PASSES><<<grid, NTHREADS, SMEM, s>>>(mA, mAlo, mB, mBlo, p);
+  if (p.split_parts > 1) {
+    tc_gemm_fixup_kernel<<<4 * (p.n_tiles_total - p.split_first), 256, 0, s>>>(p);
+    c->launches++;
+  }
   if (timed) {
     cudaEventRecord(c->ev_end[c->timing_n], s);
     c->timing_n++;
