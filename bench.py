@@ -94,6 +94,22 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(ms: float, device) -> float:
+    """The slowest rank's time: what a job of independent replicas takes.  Works on any initialised process
+    group (NCCL with a CUDA device, gloo with the CPU)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(n_iters: int, world: int, ms_per_step: float) -> float:
+    """Iterations per second of the whole job: every rank optimises its own layer (weak scaling)."""
+    return world * n_iters / (ms_per_step / 1e3)
+
+
 def dist_env():
     return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
 
@@ -252,13 +268,7 @@ def run_ours(args, cfg):
             fn()
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if use_dist:
-            import torch.distributed as dist
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), dev)
 
     for _ in range(args.warmup):
         step_resident()
@@ -336,7 +346,7 @@ def run_ours(args, cfg):
         return
     peaks, peak_kind = load_peaks()
     ms_step = ms_total / args.steps
-    value = world * lcfg.n_iters / (ms_step / 1e3)
+    value = whole_job_value(lcfg.n_iters, world, ms_step)
     e2e_value = world * lcfg.n_iters / (ms_e2e / args.steps / 1e3) if ms_e2e else None
     tf32_peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * TF32_OVER_BF16
     achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
