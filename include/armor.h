@@ -52,7 +52,8 @@ typedef enum {
 } armor_status;
 
 enum { ARMOR_H_FULL = 0, ARMOR_H_DIAG = 1 };
-enum { ARMOR_SELECT_L1_RANDOM = 0, ARMOR_SELECT_L1_GREEDY = 1 };
+/* Group selection of the sparse-core update (Section 3.3.2; the other three are the ablation of Appendix E.1) */
+enum { ARMOR_SELECT_L1_RANDOM = 0, ARMOR_SELECT_L1_GREEDY = 1, ARMOR_SELECT_UNIFORM_RANDOM = 2, ARMOR_SELECT_L2_RANDOM = 3 };
 enum { ARMOR_S_EXACT = 0, ARMOR_S_BETA = 1 };
 /* How the dense contractions (Gram, .H) are evaluated on the tensor cores:
  *   FP32X3 : operands split into tf32 high and low parts, three tcgen05 passes

@@ -35,7 +35,7 @@ from dataclasses import dataclass, field
 import numpy as np
 
 FULL, DIAG = 0, 1
-L1_RANDOM, L1_GREEDY = 0, 1
+L1_RANDOM, L1_GREEDY, UNIFORM_RANDOM, L2_RANDOM = 0, 1, 2, 3
 S_EXACT, S_BETA = 0, 1
 PH_A, PH_B, PH_S, PH_MASK = 1, 2, 4, 8
 PH_ALL = 15
@@ -347,12 +347,18 @@ def pinv_solve(K: np.ndarray, z: np.ndarray):
     return w, float(z @ w)
 
 
-def group_scores(Gamma: np.ndarray, m_group: int) -> np.ndarray:
+def group_scores(Gamma: np.ndarray, m_group: int, select_mode: int = L1_RANDOM) -> np.ndarray:
     """l_g = L1 norm of the core gradient over all m positions of the group
     (Section 3.3.2).  Reading: masked-out positions count; their gradient is
-    what signals a better mask."""
+    what signals a better mask.  The ablation of Appendix E.1 adds the L2 norm
+    (L2_RANDOM) and equal weights (UNIFORM_RANDOM)."""
     d_out, d_in = Gamma.shape
-    return np.abs(Gamma).reshape(d_out, d_in // m_group, m_group).sum(axis=2)
+    G = Gamma.reshape(d_out, d_in // m_group, m_group)
+    if select_mode == L2_RANDOM:
+        return np.sqrt((G * G).sum(axis=2))
+    if select_mode == UNIFORM_RANDOM:
+        return np.ones((d_out, d_in // m_group))
+    return np.abs(G).sum(axis=2)
 
 
 def mask_step(W, A, B, S, M, Hw, cfg: OracleConfig, t: int, info: IterInfo | None = None):
@@ -384,11 +390,11 @@ def mask_step(W, A, B, S, M, Hw, cfg: OracleConfig, t: int, info: IterInfo | Non
     alpha = np.einsum("bor,bor->br", A, A).reshape(d_out)          # ||A[:, r]||^2
     Kfull = np.stack([B[j] @ Hw[j * db:(j + 1) * db, j * db:(j + 1) * db] @ B[j].T
                       for j in range(nbi)])                        # [nbi, db, db]
-    score = group_scores(Gamma, m)                                 # [d_out, ng_row]
+    score = group_scores(Gamma, m, cfg.select_mode)                # [d_out, ng_row]
     score = np.where(alpha[:, None] > 0.0, score, 0.0)
     gidx = (np.arange(d_out, dtype=np.uint64)[:, None] * np.uint64(ng_row)
             + np.arange(ng_row, dtype=np.uint64)[None, :])
-    if cfg.select_mode == L1_RANDOM:
+    if cfg.select_mode in (L1_RANDOM, L2_RANDOM, UNIFORM_RANDOM):
         u = selection_uniform(cfg.seed, t, gidx, G_total)
         with np.errstate(divide="ignore"):
             key = np.where(score > 0.0, -np.log(u) / score, np.inf)

@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libarmor.so")
 
 H_FULL, H_DIAG = 0, 1
-SELECT_L1_RANDOM, SELECT_L1_GREEDY = 0, 1
+SELECT_L1_RANDOM, SELECT_L1_GREEDY, SELECT_UNIFORM_RANDOM, SELECT_L2_RANDOM = 0, 1, 2, 3
 S_EXACT, S_BETA = 0, 1
 PREC_FP32X3, PREC_TF32, PREC_SIMT = 0, 1, 2
 PHASE_A, PHASE_B, PHASE_S, PHASE_MASK = 1, 2, 4, 8

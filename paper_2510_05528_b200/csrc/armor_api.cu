@@ -25,8 +25,7 @@ armor_status check_config(const armor_config* cfg) {
   if (cfg->d_block > 256 || cfg->d_block % 4) return ARMOR_ERR_UNSUPPORTED;
   if (cfg->d_block > 128 && cfg->d_block % 32) return ARMOR_ERR_UNSUPPORTED;   // large blocks use the panel solver
   if (cfg->h_mode != ARMOR_H_FULL && cfg->h_mode != ARMOR_H_DIAG) return ARMOR_ERR_INVALID_ARG;
-  if (cfg->select_mode != ARMOR_SELECT_L1_RANDOM && cfg->select_mode != ARMOR_SELECT_L1_GREEDY)
-    return ARMOR_ERR_INVALID_ARG;
+  if (cfg->select_mode < ARMOR_SELECT_L1_RANDOM || cfg->select_mode > ARMOR_SELECT_L2_RANDOM) return ARMOR_ERR_INVALID_ARG;
   if (cfg->s_step != ARMOR_S_EXACT && cfg->s_step != ARMOR_S_BETA) return ARMOR_ERR_INVALID_ARG;
   if (cfg->precision < ARMOR_PREC_FP32X3 || cfg->precision > ARMOR_PREC_SIMT) return ARMOR_ERR_INVALID_ARG;
   if (cfg->precision != ARMOR_PREC_SIMT) {

@@ -132,7 +132,7 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
     const int rl = idx / gpb, cl = idx % gpb;
     const int64_t row = (int64_t)bi * db + rl;
     const int64_t cg = (int64_t)bj * gpb + cl;
-    float score = 0.f;
+    float score = 0.f, sq = 0.f;
 #pragma unroll
     for (int h = 0; h < MG / 4; ++h) {
       const float4 g4 = *reinterpret_cast<const float4*>(Gam + row * d_in + cg * MG + 4 * h);
@@ -140,12 +140,19 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
       score += fabsf(g4.y);
       score += fabsf(g4.z);
       score += fabsf(g4.w);
+      sq = fmaf(g4.x, g4.x, sq);
+      sq = fmaf(g4.y, g4.y, sq);
+      sq = fmaf(g4.z, g4.z, sq);
+      sq = fmaf(g4.w, g4.w, sq);
     }
+    // the ablation's weights (Appendix E.1): L2 norm of the group's gradient, or equal weights
+    if (select_mode == ARMOR_SELECT_L2_RANDOM) score = sqrtf(sq);
+    else if (select_mode == ARMOR_SELECT_UNIFORM_RANDOM) score = 1.f;
     if (!(alpha[row] > 0.f)) score = 0.f;
     const uint64_t g = (uint64_t)row * (uint64_t)ng_row + (uint64_t)cg;
     float key = INFINITY;
     if (score > 0.f) {
-      if (select_mode == ARMOR_SELECT_L1_RANDOM) {
+      if (select_mode != ARMOR_SELECT_L1_GREEDY) {
         const uint64_t bits = splitmix64(seed ^ splitmix64(t * n_groups_total + g));
         key = neg_log_uniform((uint32_t)(bits >> 40)) / score;
       } else {

@@ -203,6 +203,13 @@ def test_teacher_forced_greedy_selection(tiny_data):
     run_teacher_forced(TINY, W, H32, Bd.PREC_FP32X3, Bd.H_FULL, 5, select=Bd.SELECT_L1_GREEDY)
 
 
+@pytest.mark.parametrize("select", [Bd.SELECT_UNIFORM_RANDOM, Bd.SELECT_L2_RANDOM])
+def test_teacher_forced_ablation_selection_heuristics(select, tiny_data):
+    """Uniform-random and L2-random group selection (the paper's ablation of the selection heuristic)."""
+    W, X, H32 = tiny_data
+    run_teacher_forced(TINY, W, H32, Bd.PREC_FP32X3, Bd.H_FULL, 5, select=select)
+
+
 @pytest.mark.parametrize("h_mode", [Bd.H_FULL, Bd.H_DIAG])
 def test_teacher_forced_4_of_8_groups(h_mode, tiny_data):
     """The 4:8 pattern: top-4 of 8 at the initialisation, 70 masks with 4 x 4 solves per selected group."""

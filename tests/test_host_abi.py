@@ -43,6 +43,7 @@ def test_config_validation(lib):
         (Bd.make_config(1024, 1024, 512), 7),          # d_block > 256
         (Bd.make_config(576, 576, 144), 7),            # above 128 the block size must be a multiple of 32
         (Bd.make_config(256, 256, 32, h_mode=5), 1),
+        (Bd.make_config(256, 256, 32, select_mode=4), 1),
         (Bd.make_config(256, 256, 32, ridge=-1.0), 1),
         (Bd.make_config(0, 256, 32), 2),
         (Bd.make_config(192, 192, 32, precision=Bd.PREC_TF32), 7),   # tensor-core tiles need multiples of 128

@@ -520,6 +520,34 @@ def test_l1_random_selection_frequencies_follow_the_scores():
     assert np.all(i1.selected == i2.selected)
 
 
+@pytest.mark.parametrize("mode", [O.L2_RANDOM, O.UNIFORM_RANDOM])
+def test_ablation_selection_heuristics_follow_their_weights(mode):
+    """Appendix E.1: L2-random draws a group with probability proportional to the L2 norm of its gradient,
+    uniform-random with equal probability.  Chi-square over many iteration counters, as for L1-random."""
+    from scipy import stats
+    rng = np.random.default_rng(13)
+    db = 4
+    W = rng.standard_normal((4, 4)) * 0.02
+    X = rng.standard_normal((32, 4))
+    H = O.gram(X)
+    Hw = O.weighting(H, O.DIAG)
+    oc = O.OracleConfig(db, h_mode=O.DIAG, seed=321, select_mode=mode)
+    A, B, S, M = rand_state(W, H, oc, rng, scale=0.3)
+    Gam = O.core_gradient(W, A, B, S, Hw)
+    weight = np.sqrt((Gam.reshape(4, 1, 4) ** 2).sum(axis=2)).reshape(-1) if mode == O.L2_RANDOM else np.ones(4)
+    counts = np.zeros(4)
+    n = 4000
+    for t in range(n):
+        info = O.IterInfo()
+        O.mask_step(W, A, B, S, M, Hw, oc, t, info)
+        counts[int(info.selected[0, 0])] += 1
+    expected = n * weight / weight.sum()
+    assert np.sum((counts - expected) ** 2 / expected) < stats.chi2.ppf(0.999, df=3)
+    # the L1 and L2 weights differ on this input, so the two heuristics are distinguishable
+    l1 = np.abs(Gam).reshape(4, 1, 4).sum(axis=2).reshape(-1)
+    assert not np.allclose(l1 / l1.sum(), weight / weight.sum(), rtol=1e-2)
+
+
 def test_splitmix64_reference_values():
     # first outputs of the SplitMix64 generator seeded with 0 and with 1234567
     # (published test vectors of the algorithm: state += golden gamma, then mix)
