@@ -131,8 +131,12 @@ armor_status armor_init(armor_ctx* ctx, const float* d_W, const float* d_H, floa
  * gradient steps) and the greedy sparse-core update of Algorithm 3 (one group
  * per block, closed-form solve over all masks, Eq. mask_loss_opt and
  * mask_loss_opt_sol).  A, B, S, M are updated in place.  d_stats may be NULL,
- * else [n_iters].  Each iteration is a function of (state, W, H, t) only, so
- * splitting a run into several calls gives the same bits in A, B, S and M. */
+ * else [n_iters].  The iterations of a call are a function of (state, W, H,
+ * t_first, n_iters); runs are reproducible bit for bit.  With h_mode DIAG every
+ * iteration depends on the state alone, so splitting a run into several calls
+ * gives the same bits in A, B, S and M; with h_mode FULL the product S B H is
+ * carried from iteration to iteration inside a call and rebuilt by a dense
+ * product at its start, so a split changes the rounding (fp32 accuracy). */
 armor_status armor_bcd_step(armor_ctx* ctx, const float* d_Wbar, const float* d_H, float* d_A, float* d_B,
                             float* d_S, uint8_t* d_M, int64_t t_first, int32_t n_iters,
                             armor_iter_stats* d_stats, armor_stream_t stream);

@@ -323,13 +323,21 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
   // W H_w is the same for every iteration of the call: E H_w = W H_w - A (T H_w)
   st = rmul_H(c, W, H, c->WH, d_out, nullptr, nullptr, nullptr, nullptr, s);
   if (st != ARMOR_OK) return st;
+  // P = T H_w = S B H_w is formed by a dense product in the first iteration of a call only.  Afterwards it
+  // follows the state: the B-step and the S-step each form R H_w for their own direction R (S Delta, resp.
+  // Gamma_M B) to get the step length, and P moves by tau R H_w; the group updates add the rows
+  // z H_w[block row] that their guard has formed already.  With a diagonal H_w the product is a column
+  // scale and P is simply recomputed.
+  const bool carry_P = (c->cfg.h_mode == ARMOR_H_FULL);
   for (int it = 0; it < n_iters; ++it) {
     armor_iter_stats* is = d_stats ? d_stats + it : nullptr;
     const int64_t t = t_first + it;
     launch_zero_scalars(c, s);
     bd_right(c, S, B, false, c->T, d_out, d_in, 1.f, nullptr, 0.f, s);              // T = S B
-    st = rmul_H(c, c->T, H, c->P, d_out, nullptr, nullptr, nullptr, nullptr, s);     // P = T H_w
-    if (st != ARMOR_OK) return st;
+    if (it == 0 || !carry_P) {
+      st = rmul_H(c, c->T, H, c->P, d_out, nullptr, nullptr, nullptr, nullptr, s);   // P = T H_w
+      if (st != ARMOR_OK) return st;
+    }
     bd_left(c, A, false, c->P, c->EH, d_out, d_in, -1.f, c->WH, 1.f, s);             // E H_w = W H_w - A P
     bd_left(c, A, false, c->T, c->E, d_out, d_in, -1.f, W, 1.f, s);                  // E = W - A T
     dot_to_ptr(c, c->EH, c->E, c->wn, c->sc + SC_L0, s);                             // L = <E H_w, E>
@@ -355,12 +363,17 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       if (st != ARMOR_OK) return st;
       st = launch_chol(c, 2, c->Hjj, c->Delta, c->Delta, c->GamB, nullptr, nullptr, nbi, c->partblk, s);
       if (st != ARMOR_OK) return st;
-      bd_right(c, c->U, c->Delta, false, c->V, d_out, d_in, 1.f, nullptr, 0.f, s);   // V = U Delta
-      st = rmul_H(c, c->V, H, c->VH, d_out, c->V, c->sc + SC_Q_B, nullptr, nullptr, s);
+      // direction in B: V = A R with R = S Delta; R H_w serves both V H_w = A (R H_w) and the carried P
+      bd_right(c, S, c->Delta, false, c->Tmp, d_out, d_in, 1.f, nullptr, 0.f, s);    // R = S Delta
+      st = rmul_H(c, c->Tmp, H, c->E, d_out, nullptr, nullptr, nullptr, nullptr, s); // R H_w
       if (st != ARMOR_OK) return st;
+      bd_left(c, A, false, c->Tmp, c->V, d_out, d_in, 1.f, nullptr, 0.f, s);         // V = A R
+      bd_left(c, A, false, c->E, c->VH, d_out, d_in, 1.f, nullptr, 0.f, s);          // V H_w = A (R H_w)
+      dot_to_ptr(c, c->VH, c->V, c->wn, c->sc + SC_Q_B, s);
       launch_stage(c, is, 2, c->partblk, nbi * chol_parts_per_block(db, nbi), nbi, s);
       launch_axpy_slot(c, B, c->Delta, (int64_t)nbi * db * db, SC_TAU_B, 1.f, s);    // B += tau Delta
       launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_B, -1.f, s);                   // EH -= tau V H_w
+      if (carry_P) launch_axpy_slot(c, c->P, c->E, c->wn, SC_TAU_B, 1.f, s);         // P += tau R H_w
     } else {
       launch_stage(c, is, 2, nullptr, 0, 0, s);
     }
@@ -369,10 +382,12 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
     if (ph & ARMOR_PHASE_S) {
       core_gradient(c, A, B, s);
       launch_masked_copy(c, c->Gam, M, c->U, SC_NRM_S, s);                           // U = Gamma (.) M
-      bd_left(c, A, false, c->U, c->Tmp, d_out, d_in, 1.f, nullptr, 0.f, s);
-      bd_right(c, c->Tmp, B, false, c->V, d_out, d_in, 1.f, nullptr, 0.f, s);        // V = A Gamma_M B
-      st = rmul_H(c, c->V, H, c->VH, d_out, c->V, c->sc + SC_Q_S, nullptr, nullptr, s);
+      bd_right(c, c->U, B, false, c->Tmp, d_out, d_in, 1.f, nullptr, 0.f, s);        // R = Gamma_M B
+      st = rmul_H(c, c->Tmp, H, c->E, d_out, nullptr, nullptr, nullptr, nullptr, s); // R H_w
       if (st != ARMOR_OK) return st;
+      bd_left(c, A, false, c->Tmp, c->V, d_out, d_in, 1.f, nullptr, 0.f, s);         // V = A Gamma_M B
+      bd_left(c, A, false, c->E, c->VH, d_out, d_in, 1.f, nullptr, 0.f, s);          // V H_w = A (R H_w)
+      dot_to_ptr(c, c->VH, c->V, c->wn, c->sc + SC_Q_S, s);
       if (c->cfg.s_step == ARMOR_S_BETA) {
         // the paper's step size (Eq. lrWprime): |A^T A|_F and |B H_w B^T|_F
         block_mm(c, A, true, A, false, c->G, nbo, s);
@@ -390,6 +405,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       launch_stage(c, is, c->cfg.s_step == ARMOR_S_BETA ? 6 : 3, nullptr, 0, 0, s);
       launch_axpy_slot(c, S, c->U, c->wn, SC_TAU_S, 1.f, s);                         // S += tau Gamma_M
       launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_S, -1.f, s);                   // EH -= tau V H_w
+      if (carry_P) launch_axpy_slot(c, c->P, c->E, c->wn, SC_TAU_S, 1.f, s);         // P += tau R H_w
     } else {
       launch_stage(c, is, 3, nullptr, 0, 0, s);
     }
@@ -404,6 +420,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       launch_mask_quadratic(c, A, B, H, s);
       launch_stage(c, is, 4, c->partblk, nbo * nbi, 0, s);
       launch_mask_commit(c, S, M, is, s);
+      if (carry_P && it + 1 < n_iters) launch_mask_carry_P(c, c->P, s);              // P += dS B H_w (if accepted)
     } else {
       launch_stage(c, is, 4, nullptr, 0, 0, s);
     }

@@ -206,6 +206,8 @@ void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const ui
 // for V = A dS B from the selection records
 void launch_mask_quadratic(armor_ctx* c, const float* A, const float* B, const float* H, cudaStream_t s);
 void launch_mask_commit(armor_ctx* c, float* S, uint8_t* M, armor_iter_stats* st, cudaStream_t s);
+// P += dS B H_w for the accepted group updates, from the rows the guard has formed (full weighting only)
+void launch_mask_carry_P(armor_ctx* c, float* P, cudaStream_t s);
 
 // tensor-core GEMM (gemm_tcgen05.cu):  C[M][N] (+)= sum_k A[m][k] * B[n][k]  (both K-major, fp32 storage).
 // passes == 3 uses the split operands (A, Alo, B, Blo).  Partial dot products of the output tile with up

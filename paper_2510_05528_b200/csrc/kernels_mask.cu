@@ -390,7 +390,34 @@ __global__ void mask_commit_kernel(const SelRec* __restrict__ sel, int nblocks, 
   if (threadIdx.x == 0 && st) st->groups_changed = changed;
 }
 
+// The accepted group updates change T H_w = S B H_w by the rows (delta^T B_j[group rows, :]) H_w[j-th block
+// row, :] = y_ij, added to row r_ij.  Groups of one row-block may share a row, so one CTA walks the column
+// blocks j in order (deterministic sums); the grid is (row-block, chunk of 1024 columns).
+__global__ void __launch_bounds__(NT) mask_carry_kernel(const SelRec* __restrict__ sel, const float* __restrict__ Y,
+                                                        float* __restrict__ P, const double* __restrict__ sc,
+                                                        int64_t d_in, int nbo_pad, int nbi) {
+  if (sc[SC_ACCEPT] == 0.0) return;
+  const int bi = blockIdx.x;
+  const int64_t c4 = (int64_t)blockIdx.y * 1024 + 4 * threadIdx.x;
+  if (c4 >= d_in) return;
+  for (int j = 0; j < nbi; ++j) {
+    const SelRec rec = sel[bi * nbi + j];
+    if (!rec.valid) continue;
+    const float4 y = *reinterpret_cast<const float4*>(Y + ((int64_t)j * nbo_pad + bi) * d_in + c4);
+    float4* dst = reinterpret_cast<float4*>(P + (int64_t)rec.row * d_in + c4);
+    float4 v = *dst;
+    v.x += y.x; v.y += y.y; v.z += y.z; v.w += y.w;
+    *dst = v;
+  }
+}
+
 }  // namespace
+
+void launch_mask_carry_P(armor_ctx* c, float* P, cudaStream_t s) {
+  mask_carry_kernel<<<dim3(c->nbo, (unsigned)((c->d_in + 1023) / 1024)), NT, 0, s>>>(c->sel, c->Ysel, P, c->sc, c->d_in,
+                                                                                   c->nbo_pad, c->nbi);
+  c->launches++;
+}
 
 void launch_alpha(armor_ctx* c, const float* A, cudaStream_t s) {
   alpha_kernel<<<dim3(c->nbo, (c->db + 31) / 32), dim3(32, 8), 0, s>>>(A, c->alpha, c->db);

@@ -314,22 +314,32 @@ def test_free_running_tiny_config(h_mode, tiny_data):
     assert np.all(host(st.S)[~M_gpu] == 0.0)
 
 
-def test_resume_gives_the_same_bits(tiny_data):
+def test_resume_gives_the_same_result(tiny_data):
+    """Splitting a run into several calls.  With the diagonal weighting every iteration is a function of the
+    state alone and the bits agree.  With the full Gram the library carries T.H from iteration to iteration
+    inside a call and rebuilds it at the start of a call, so a split changes the rounding: the results agree
+    to fp32 accuracy as long as no mask decision flips, and in the loss otherwise."""
     W, X, H32 = tiny_data
     Hd = dev(H32)
-    outs = []
-    for split in ([20], [10, 10], [1, 7, 12]):
-        ctx = make(TINY, Bd.PREC_FP32X3)
-        st = ctx.init(dev(W), Hd)
-        t = 0
-        for n in split:
-            ctx.bcd_step(st, Hd, t, n, want_stats=False)
-            t += n
-        torch.cuda.synchronize()
-        outs.append([host(x).copy() for x in (st.A, st.B, st.S, st.M)])
-    for other in outs[1:]:
-        for a, b in zip(outs[0], other):
-            assert np.array_equal(a, b)
+    for h_mode in (Bd.H_DIAG, Bd.H_FULL):
+        outs, losses = [], []
+        for split in ([20], [10, 10], [1, 7, 12]):
+            ctx = make(TINY, Bd.PREC_FP32X3, h_mode)
+            st = ctx.init(dev(W), Hd)
+            t = 0
+            for n in split:
+                ctx.bcd_step(st, Hd, t, n, want_stats=False)
+                t += n
+            losses.append(ctx.proxy_loss(st, Hd).item())
+            outs.append([host(x).copy() for x in (st.A, st.B, st.S, st.M)])
+        for other, loss in zip(outs[1:], losses[1:]):
+            if h_mode == Bd.H_DIAG:
+                for a, b in zip(outs[0], other):
+                    assert np.array_equal(a, b)
+            elif np.array_equal(outs[0][3], other[3]):
+                for a, b in zip(outs[0][:3], other[:3]):
+                    assert rel(a, b) < 1e-4
+            assert abs(loss - losses[0]) / losses[0] < 1e-3
 
 
 def test_zero_iterations_is_a_no_op(tiny_data):
