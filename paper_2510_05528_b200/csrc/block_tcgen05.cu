@@ -31,11 +31,11 @@ using namespace tc;
 
 constexpr int TILE = 128, BK = 32;
 constexpr int NTHREADS = 320;
-constexpr int STAGES = 2;
+constexpr int STAGES = 3;
 constexpr int OP_BYTES = TILE * BK * 4;           // 16 KiB: one operand chunk
 constexpr int STAGE_BYTES = 4 * OP_BYTES;         // A hi, A lo, B hi, B lo
 constexpr uint32_t TMEM_COLS = 256;               // two accumulators of 128 columns
-constexpr int EPI_BYTES = 32 * TILE * 4;          // per epilogue warp: 32 rows x 128 columns as four swizzled boxes
+constexpr int EPI_BYTES = 32 * 64 * 4;            // per epilogue warp: 32 rows x 64 columns (half a tile row) as two swizzled boxes
 constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 4 * EPI_BYTES + 1024;
 
 struct OpCoord {
@@ -232,7 +232,7 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     int local = 0;
     uint32_t d_loads = 0;   // D slabs requested so far: parity of their barrier
     bool ok = true;
-    uint8_t* buf = smem + (size_t)STAGES * STAGE_BYTES + (size_t)q * EPI_BYTES;   // four 4 KiB boxes of 32 x 32
+    uint8_t* buf = smem + (size_t)STAGES * STAGE_BYTES + (size_t)q * EPI_BYTES;   // two 4 KiB boxes of 32 x 32
     const uint32_t buf_u32 = smem_u32(buf);
     const uint32_t dbar = dfull0 + 8 * q;
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++local) {
@@ -242,54 +242,61 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
       const int64_t row_base = p.r_b * b + p.r_s * ks + (int64_t)tm * TILE + q * 32;
       const int64_t col_tile = p.c_b * b + (int64_t)tn * TILE;
-      // boxes of this warp's slab that lie inside C (warp-uniform)
-      int n_box = 0;
-      if (row_base < p.c_rows && tm * TILE + q * 32 < p.m_valid)
-        for (int ch = 0; ch < 4; ++ch) n_box += (col_tile + 32 * ch < p.c_cols) ? 1 : 0;
-      if (lane == 0) {
-        tma_store_wait_read();                      // the previous item's stores have read the slab
-        if (p.D && n_box > 0) {
-          mbar_expect_tx(dbar, (uint32_t)n_box * 4096u);
-          for (int ch = 0; ch < n_box; ++ch)
-            tma_load_2d(buf_u32 + ch * 4096, &mapD, (int)(col_tile + 32 * ch), (int)row_base, dbar);
-        }
-      }
-      __syncwarp();
-      if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
-      tc_fence_after();
-      if (p.D && n_box > 0) {
-        if (!mbar_wait(dbar, d_loads & 1u, abortp, p.status)) { ok = false; break; }
-        ++d_loads;
-      }
+      // The warp's 32 x 128 slab goes through shared memory in two halves of 64 columns (two 32 x 32 boxes).
+      bool waited = false;
 #pragma unroll 1
-      for (int ch = 0; ch < TILE / 32; ++ch) {
-        uint32_t r[32];
-        tmem_ld32(tmem_base + (uint32_t)(as * TILE + ch * 32) + ((uint32_t)(q * 32) << 16), r);
-        if (ch >= n_box) continue;                  // warp-uniform
-        // lane = row of the box; 16-byte chunk c of the row sits at chunk c ^ (row % 8)  (128-byte swizzle)
-        uint8_t* rowp = buf + ch * 4096 + lane * 128;
-#pragma unroll
-        for (int cq = 0; cq < 8; ++cq) {
-          float4* cell = reinterpret_cast<float4*>(rowp + ((cq ^ (lane & 7)) << 4));
-          float4 v = make_float4(p.alpha * __uint_as_float(r[4 * cq]), p.alpha * __uint_as_float(r[4 * cq + 1]),
-                                 p.alpha * __uint_as_float(r[4 * cq + 2]), p.alpha * __uint_as_float(r[4 * cq + 3]));
-          if (p.D) {
-            const float4 d = *cell;
-            v.x = fmaf(p.beta, d.x, v.x); v.y = fmaf(p.beta, d.y, v.y);
-            v.z = fmaf(p.beta, d.z, v.z); v.w = fmaf(p.beta, d.w, v.w);
+      for (int hf = 0; hf < 2 && ok; ++hf) {
+        // boxes of this half that lie inside C (warp-uniform)
+        int n_box = 0;
+        if (row_base < p.c_rows && tm * TILE + q * 32 < p.m_valid)
+          for (int ch = 0; ch < 2; ++ch) n_box += (col_tile + 64 * hf + 32 * ch < p.c_cols) ? 1 : 0;
+        if (lane == 0) {
+          tma_store_wait_read();                    // the previous stores have read the staging boxes
+          if (p.D && n_box > 0) {
+            mbar_expect_tx(dbar, (uint32_t)n_box * 4096u);
+            for (int ch = 0; ch < n_box; ++ch)
+              tma_load_2d(buf_u32 + ch * 4096, &mapD, (int)(col_tile + 64 * hf + 32 * ch), (int)row_base, dbar);
           }
-          *cell = v;
         }
-      }
-      // accumulator buffer is free again
-      tc_fence_before();
-      fence_proxy_async();
-      __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(tempty0 + 8 * as);
-        for (int ch = 0; ch < n_box; ++ch)
-          tma_store_2d(&mapC, (int)(col_tile + 32 * ch), (int)row_base, buf_u32 + ch * 4096);
-        tma_store_commit();
+        __syncwarp();
+        if (!waited) {
+          if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
+          tc_fence_after();
+          waited = true;
+        }
+        if (p.D && n_box > 0) {
+          if (!mbar_wait(dbar, d_loads & 1u, abortp, p.status)) { ok = false; break; }
+          ++d_loads;
+        }
+#pragma unroll 1
+        for (int ch = 0; ch < 2; ++ch) {
+          uint32_t r[32];
+          tmem_ld32(tmem_base + (uint32_t)(as * TILE + hf * 64 + ch * 32) + ((uint32_t)(q * 32) << 16), r);
+          if (ch >= n_box) continue;                // warp-uniform
+          // lane = row of the box; 16-byte chunk c of the row sits at chunk c ^ (row % 8)  (128-byte swizzle)
+          uint8_t* rowp = buf + ch * 4096 + lane * 128;
+#pragma unroll
+          for (int cq = 0; cq < 8; ++cq) {
+            float4* cell = reinterpret_cast<float4*>(rowp + ((cq ^ (lane & 7)) << 4));
+            float4 v = make_float4(p.alpha * __uint_as_float(r[4 * cq]), p.alpha * __uint_as_float(r[4 * cq + 1]),
+                                   p.alpha * __uint_as_float(r[4 * cq + 2]), p.alpha * __uint_as_float(r[4 * cq + 3]));
+            if (p.D) {
+              const float4 d = *cell;
+              v.x = fmaf(p.beta, d.x, v.x); v.y = fmaf(p.beta, d.y, v.y);
+              v.z = fmaf(p.beta, d.z, v.z); v.w = fmaf(p.beta, d.w, v.w);
+            }
+            *cell = v;
+          }
+        }
+        if (hf == 1) tc_fence_before();             // all reads of the accumulator are done
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) {
+          if (hf == 1) mbar_arrive(tempty0 + 8 * as);   // accumulator buffer is free again
+          for (int ch = 0; ch < n_box; ++ch)
+            tma_store_2d(&mapC, (int)(col_tile + 64 * hf + 32 * ch), (int)row_base, buf_u32 + ch * 4096);
+          tma_store_commit();
+        }
       }
     }
     if (lane == 0) tma_store_wait_read();           // shared memory stays valid until the stores have read it
