@@ -149,8 +149,10 @@ armor_status armor_proxy_loss(armor_ctx* ctx, const float* d_Wbar, const float* 
 /* Deployment form (Section 3.1): y_t = A (S (B x_t)) for the rows of
  * x [n_tokens, d_in] -> y [n_tokens, d_out].  With d_r1, d_r2 non-NULL the
  * normalisation is undone: y_t = r2 (.) A S B (r1 (.) x_t).  xy_dtype:
- * ARMOR_DTYPE_F32, or ARMOR_DTYPE_BF16 for bf16 x and y (widened on the way in,
- * rounded once on the way out; the products run in the context's precision).
+ * ARMOR_DTYPE_F32, or ARMOR_DTYPE_BF16 for bf16 x and y: the deployment form, in
+ * which the core S and the wrapped activations B x are rounded to bf16 and
+ * multiplied on the bf16 tensor-core path with fp32 accumulation (the two thin
+ * wrapper products stay fp32-grade; y is rounded to bf16 once).
  * d_M is accepted for symmetry and may be NULL (S already carries the zeros). */
 armor_status armor_apply(armor_ctx* ctx, const float* d_A, const float* d_B, const float* d_S,
                          const uint8_t* d_M, const float* d_r1, const float* d_r2, const void* d_x,

@@ -461,7 +461,7 @@ armor_status armor_apply(armor_ctx* c, const float* A, const float* B, const flo
       }
     }
     bd_right(c, xc, B, true, c->T, n, d_in, 1.f, nullptr, 0.f, s);                   // z1 = x B^T
-    armor_status st = apply_core(c, c->T, S, c->E, n, s);                            // z2 = z1 S^T
+    armor_status st = apply_core(c, c->T, S, c->E, n, bf16, s);                      // z2 = z1 S^T
     if (st != ARMOR_OK) return st;
     bd_right(c, c->E, A, true, yc, n, d_out, 1.f, nullptr, 0.f, s);                  // y = z2 A^T
     if (bf16) launch_f32_to_bf16(c, yc, r2, static_cast<char*>(d_y) + (size_t)(t0 * d_out) * esz, n, d_out, s);

@@ -156,7 +156,7 @@ armor_status prepare_H(armor_ctx* c, const float* H, cudaStream_t s);
 armor_status gram_accumulate(armor_ctx* c, const void* X, int x_dtype, int64_t n_rows, int64_t ldx, float* H,
                              cudaStream_t s);
 // z2 [n, d_out] = z1 [n, d_in] * S^T
-armor_status apply_core(armor_ctx* c, const float* z1, const float* S, float* z2, int64_t n, cudaStream_t s);
+armor_status apply_core(armor_ctx* c, const float* z1, const float* S, float* z2, int64_t n, bool bf16, cudaStream_t s);
 
 // deterministic reductions (two stages, fixed order)
 void dot_to_ptr(armor_ctx* c, const float* x, const float* y, int64_t n, double* out, cudaStream_t s);
@@ -217,7 +217,7 @@ struct TcGemm {
   const float* B; const float* Blo; int64_t ldb;
   float* C; int64_t ldc;
   int64_t M, N, K;
-  int passes;            // 1 or 3
+  int passes;            // 1 or 3 tf32 passes on fp32 operands; 0: A and B are bf16 arrays (one kind::f16 pass)
   int64_t k_segment;     // K extent accumulated in tensor memory before it is folded into C (0: all of K)
   int accumulate;        // C += (read-modify-write) instead of C =
   int symmetric_lower;   // only the lower triangle (tiles with n0 <= m0, elements with column <= row) is computed (M == N)

@@ -102,8 +102,21 @@ armor_status gram_accumulate(armor_ctx* c, const void* Xv, int x_dtype, int64_t 
   return ARMOR_OK;
 }
 
-armor_status apply_core(armor_ctx* c, const float* z1, const float* S, float* z2, int64_t n, cudaStream_t s) {
+armor_status apply_core(armor_ctx* c, const float* z1, const float* S, float* z2, int64_t n, bool bf16, cudaStream_t s) {
   const int64_t d_in = c->d_in, d_out = c->d_out;
+  if (bf16 && c->cfg.precision != ARMOR_PREC_SIMT && d_out % 32 == 0 && d_in % 8 == 0) {
+    // bf16 deployment: the core and the wrapped activations are rounded to bf16 and multiplied on the bf16
+    // tensor-core path with fp32 accumulation
+    launch_f32_to_bf16(c, z1, nullptr, c->U, n, d_in, s);
+    launch_f32_to_bf16(c, S, nullptr, c->P, d_out, d_in, s);
+    TcGemm g{};
+    g.lda = d_in; g.ldb = d_in; g.ldc = d_out;
+    g.M = n; g.N = d_out; g.K = d_in;
+    g.C = z2;
+    g.A = c->U; g.B = c->P; g.passes = 0;
+    g.k_segment = 0;
+    return launch_tc_gemm(c, g, nullptr, s);
+  }
   if (c->cfg.precision == ARMOR_PREC_SIMT || (d_out % 32) || (d_in % 4)) {
     BGemm g{};
     g.A = z1; g.sAm = d_in; g.sAk = 1;

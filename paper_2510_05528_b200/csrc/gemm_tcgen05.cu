@@ -54,12 +54,12 @@ __device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t addr) {
   return d;
 }
 
-// kind::tf32, fp32 accumulate, both operands K-major, M = 128, N = 256.
-__device__ __forceinline__ uint32_t instr_desc_tf32() {
+// fp32 accumulate, both operands K-major, M = 128, N = 256; operands tf32 (kind::tf32) or bf16 (kind::f16).
+__device__ __forceinline__ uint32_t instr_desc(bool bf16) {
   uint32_t d = 0;
   d |= 1u << 4;                   // D format: F32
-  d |= 2u << 7;                   // A format: TF32
-  d |= 2u << 10;                  // B format: TF32
+  d |= (bf16 ? 1u : 2u) << 7;     // A format: BF16 / TF32
+  d |= (bf16 ? 1u : 2u) << 10;    // B format: BF16 / TF32
   d |= (uint32_t)(BN >> 3) << 17; // N
   d |= (uint32_t)(BM >> 4) << 24; // M
   return d;
@@ -112,7 +112,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]);
   const uint32_t tfull0 = smem_u32(&bars[2 * STAGES]), tempty0 = smem_u32(&bars[2 * STAGES + 2]);
-  const int kt_total = (int)((p.K + BK - 1) / BK);
+  constexpr int BKE = (PASSES == 0) ? 64 : 32;      // elements of K per 128-byte row: bf16 or fp32
+  const int kt_total = (int)((p.K + BKE - 1) / BKE);
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -146,12 +147,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
           const uint32_t fb = full0 + 8 * stage;
           mbar_expect_tx(fb, STAGE_BYTES);
           uint32_t dst = smem_u32(smem + (size_t)stage * STAGE_BYTES);
-          tma_load_2d(dst, &mapA, kt * BK, mt * BM, fb);
+          tma_load_2d(dst, &mapA, kt * BKE, mt * BM, fb);
           dst += A_BYTES;
-          if (PASSES == 3) { tma_load_2d(dst, &mapAlo, kt * BK, mt * BM, fb); dst += A_BYTES; }
-          tma_load_2d(dst, &mapB, kt * BK, nt * BN, fb);
+          if (PASSES == 3) { tma_load_2d(dst, &mapAlo, kt * BKE, mt * BM, fb); dst += A_BYTES; }
+          tma_load_2d(dst, &mapB, kt * BKE, nt * BN, fb);
           dst += B_BYTES;
-          if (PASSES == 3) tma_load_2d(dst, &mapBlo, kt * BK, nt * BN, fb);
+          if (PASSES == 3) tma_load_2d(dst, &mapBlo, kt * BKE, nt * BN, fb);
           ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -169,7 +170,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = instr_desc_tf32();
+      const uint32_t idesc = instr_desc(PASSES == 0);
       int stage = 0; uint32_t phase = 0;
       int local = 0;   // (tile, K segment) items handled so far: selects the accumulator buffer
       bool ok = true;
@@ -199,6 +200,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
                 umma_tf32(tacc, dal, dbm, idesc, acc);
                 umma_tf32(tacc, da, dbl, idesc, 1);
                 umma_tf32(tacc, da, dbm, idesc, 1);
+              } else if (PASSES == 0) {
+                umma_bf16(tacc, da, dbm, idesc, acc);
               } else {
                 umma_tf32(tacc, da, dbm, idesc, acc);
               }
@@ -382,14 +385,16 @@ __global__ void __launch_bounds__(256) tc_gemm_fixup_kernel(const Params p) {
 
 // ------------------------------------------------------------------ host side
 // [rows][K] fp32, leading dimension ld: box = BK x box_rows, 128-byte swizzle, zero fill out of bounds.
-bool make_map(CUtensorMap* map, const float* base, int64_t rows, int64_t K, int64_t ld, int box_rows) {
+bool make_map(CUtensorMap* map, const float* base, int64_t rows, int64_t K, int64_t ld, int box_rows,
+              bool bf16 = false) {
   PFN_cuTensorMapEncodeTiled_v12000 enc = get_encode();
   if (!enc) return false;
   cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(float)};
-  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * (bf16 ? 2 : 4)};
+  cuuint32_t box[2] = {(cuuint32_t)(bf16 ? 64 : BK), (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+  CUresult r = enc(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                   const_cast<float*>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
@@ -398,8 +403,8 @@ bool make_map(CUtensorMap* map, const float* base, int64_t rows, int64_t K, int6
 template <int PASSES>
 armor_status launch_impl(armor_ctx* c, const TcGemm& g, Params p, cudaStream_t s) {
   CUtensorMap mA, mAlo, mB, mBlo;
-  if (!make_map(&mA, g.A, g.M, g.K, g.lda, BM)) return ARMOR_ERR_CUDA;
-  if (!make_map(&mB, g.B, g.N, g.K, g.ldb, BN)) return ARMOR_ERR_CUDA;
+  if (!make_map(&mA, g.A, g.M, g.K, g.lda, BM, PASSES == 0)) return ARMOR_ERR_CUDA;
+  if (!make_map(&mB, g.B, g.N, g.K, g.ldb, BN, PASSES == 0)) return ARMOR_ERR_CUDA;
   if (PASSES == 3) {
     if (!make_map(&mAlo, g.Alo, g.M, g.K, g.lda, BM)) return ARMOR_ERR_CUDA;
     if (!make_map(&mBlo, g.Blo, g.N, g.K, g.ldb, BN)) return ARMOR_ERR_CUDA;
@@ -424,7 +429,7 @@ armor_status launch_impl(armor_ctx* c, const TcGemm& g, Params p, cudaStream_t s
   }
   // tail split: the tiles of the last, partly filled wave are cut along K so that their pieces fill the wave
   p.split_first = p.n_tiles_total; p.split_parts = 1; p.n_items = p.n_tiles_total; p.slabs = c->gemm_slabs;
-  const int kt_total = (int)((p.K + BK - 1) / BK);
+  const int kt_total = (int)((p.K + (PASSES == 0 ? 64 : BK) - 1) / (PASSES == 0 ? 64 : BK));
   const int rem = p.n_tiles_total % n_sm;
   if (c->gemm_slabs && !p.symmetric_lower && rem > 0 && p.ldc % 4 == 0 && p.N % 4 == 0) {
     int parts = n_sm / rem;
@@ -465,7 +470,7 @@ bool tc_gemm_shape_ok(int64_t M, int64_t N, int64_t K) {
 
 armor_status launch_tc_gemm(armor_ctx* c, const TcGemm& g, int* n_tiles, cudaStream_t s) {
   if (!tc_gemm_shape_ok(g.M, g.N, g.K)) return ARMOR_ERR_UNSUPPORTED;
-  if ((g.lda % 4) || (g.ldb % 4) || (g.ldc % 4)) return ARMOR_ERR_UNSUPPORTED;
+  if ((g.lda % (g.passes == 0 ? 8 : 4)) || (g.ldb % (g.passes == 0 ? 8 : 4)) || (g.ldc % 4)) return ARMOR_ERR_UNSUPPORTED;
   if (g.symmetric_lower && g.M != g.N) return ARMOR_ERR_INVALID_ARG;
   Params p{};
   p.C = g.C; p.ldc = g.ldc; p.M = g.M; p.N = g.N; p.K = g.K;
@@ -484,9 +489,11 @@ armor_status launch_tc_gemm(armor_ctx* c, const TcGemm& g, int* n_tiles, cudaStr
   p.accumulate = g.accumulate; p.symmetric_lower = g.symmetric_lower;
   p.d1 = g.d1; p.d2 = g.d2; p.part1 = g.part1; p.part2 = g.part2;
   p.status = c->status;
-  p.kt_seg = g.k_segment > 0 ? (int)((g.k_segment + BK - 1) / BK) : (int)((g.K + BK - 1) / BK);
+  const int bke = (g.passes == 0) ? 64 : BK;
+  p.kt_seg = g.k_segment > 0 ? (int)((g.k_segment + bke - 1) / bke) : (int)((g.K + bke - 1) / bke);
   if (p.kt_seg < 1) p.kt_seg = 1;
   if (n_tiles) *n_tiles = p.n_tiles_total;
   if (g.passes == 3) return launch_impl<3>(c, g, p, s);
+  if (g.passes == 0) return launch_impl<0>(c, g, p, s);
   return launch_impl<1>(c, g, p, s);
 }

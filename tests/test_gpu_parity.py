@@ -436,8 +436,9 @@ def test_apply_with_bf16_activations(mid_data):
         assert y.dtype == torch.bfloat16
         r1, r2 = (host(st.r1).astype(np.float64), host(st.r2).astype(np.float64)) if den else (None, None)
         yo = O.apply(A, B, S, xr, r1, r2)
-        # one rounding to bf16 (2^-9 relative per element) on the way out
-        assert rel(y.float().cpu().numpy(), yo) < 3e-3
+        # bf16 core, bf16 wrapped activations and one rounding of y: three roundings of 2^-9 relative half-width
+        # (rms 2^-9 / sqrt(3) each) give about 2e-3; fp32 accumulation adds nothing visible
+        assert rel(y.float().cpu().numpy(), yo) < 5e-3
 
 
 # ------------------------------------------------------------------------------------------ block products
