@@ -68,14 +68,12 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   TAKE(G, float*, ao);
   TAKE(GamA, float*, ao);
   TAKE(dA, float*, ao);
-  TAKE(At, float*, ao);
   TAKE(C, float*, bo);
   TAKE(GamB, float*, bo);
   TAKE(Delta, float*, bo);
   TAKE(Hjj, float*, bo);
   TAKE(Kfull, float*, bo);
   TAKE(Ktmp, float*, bo);
-  TAKE(Bt, float*, bo);
   TAKE(alpha, float*, (size_t)cfg.d_out * sizeof(float));
   TAKE(hdiag, float*, (size_t)cfg.d_in * sizeof(float));
   const int64_t nbo_pad = (nbo + 31) / 32 * 32;
@@ -346,7 +344,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
     // ---- A-step: A_i += Gamma_i (G_i + lam I)^-1 -------------------------------------------
     if (ph & ARMOR_PHASE_A) {
       rowblock_grams(c, c->P, c->EH, c->T, c->G, c->GamA, s);   // G_i = T_i H_w T_i^T, Gamma_i = E_i H_w T_i^T
-      st = launch_chol(c, 0, c->G, c->GamA, c->dA, nullptr, A, c->At, nbo, c->partblk, s);
+      st = launch_chol(c, 0, c->G, c->GamA, c->dA, nullptr, A, nbo, c->partblk, s);
       if (st != ARMOR_OK) return st;
       launch_stage(c, is, 1, c->partblk, nbo * chol_parts_per_block(db, nbo), nbo, s);
       bd_left(c, c->dA, false, c->P, c->EH, d_out, d_in, -1.f, c->EH, 1.f, s);       // EH -= dA P
@@ -359,9 +357,9 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       launch_zero_flags(c, s);
       bd_left(c, A, false, S, c->U, d_out, d_in, 1.f, nullptr, 0.f, s);              // U = A S
       colblock_grams(c, c->U, c->U, c->EH, c->C, c->GamB, s);   // C_j = U_j^T U_j, Gamma_j = U_j^T (E H_w)_j
-      st = launch_chol(c, 1, c->C, c->GamB, c->Delta, nullptr, nullptr, nullptr, nbi, nullptr, s);
+      st = launch_chol(c, 1, c->C, c->GamB, c->Delta, nullptr, nullptr, nbi, nullptr, s);
       if (st != ARMOR_OK) return st;
-      st = launch_chol(c, 2, c->Hjj, c->Delta, c->Delta, c->GamB, nullptr, nullptr, nbi, c->partblk, s);
+      st = launch_chol(c, 2, c->Hjj, c->Delta, c->Delta, c->GamB, nullptr, nbi, c->partblk, s);
       if (st != ARMOR_OK) return st;
       // direction in B: V = A R with R = S Delta; R H_w serves both V H_w = A (R H_w) and the carried P
       bd_right(c, S, c->Delta, false, c->Tmp, d_out, d_in, 1.f, nullptr, 0.f, s);    // R = S Delta

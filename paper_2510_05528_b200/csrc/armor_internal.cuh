@@ -56,7 +56,7 @@ struct armor_ctx {
   // low parts of the left operands / of H for the three-pass tensor-core mode
   float *Lo, *Hlo;
   // [nb, db, db] scratch
-  float *G, *GamA, *dA, *At, *C, *GamB, *Delta, *Hjj, *Kfull, *Ktmp, *Bt;
+  float *G, *GamA, *dA, *C, *GamB, *Delta, *Hjj, *Kfull, *Ktmp;
   float *alpha, *hdiag;
   float *Hq1, *Hq2;      // [d_in, d_in] scratch of the paper's step size (s_step BETA, full weighting)
   float* gemm_slabs;     // 128 x 256 slabs of partial sums of the dense product's split tail tiles
@@ -166,7 +166,6 @@ void reduce_partials_to(armor_ctx* c, const double* part, int n, double* out, cu
 void launch_colscale(armor_ctx* c, const float* in, const float* h, float* out, int64_t rows, int64_t cols,
                      cudaStream_t s);
 void launch_extract_hblocks(armor_ctx* c, const float* H, cudaStream_t s);   // hdiag, Hjj (per h_mode)
-void launch_transpose_blocks(armor_ctx* c, const float* in, float* out, int nb, cudaStream_t s);
 void launch_masked_copy(armor_ctx* c, const float* Gam, const uint8_t* M, float* out, int slot_norm,
                         cudaStream_t s);                                     // out = Gam (.) M, sc[slot] = ||out||^2
 void launch_axpy_slot(armor_ctx* c, float* y, const float* x, int64_t n, int slot, float sign,
@@ -190,13 +189,13 @@ void launch_f32_to_bf16(armor_ctx* c, const float* in, const float* colscale, vo
                         cudaStream_t s);
 
 // block solves (kernels_chol.cu)
-// mode 0: X = rhs (G + lam I)^-1, A += X, At = A^T, out = X, part[b] = exact decrease of block b
+// mode 0: X = rhs (G + lam I)^-1, A += X, out = X, part[b] = exact decrease of block b
 // mode 1: out = (G + lam I)^-1 rhs
 // mode 2: out = rhs (G + lam I)^-1, part[b] = <dotw, out>
 // partial sums written per block by launch_chol (modes 0 and 2)
 int chol_parts_per_block(int db, int nb);
 armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float* rhs, float* out, const float* dotw,
-                         float* A, float* At, int nb, double* part, cudaStream_t s);
+                         float* A, int nb, double* part, cudaStream_t s);
 
 // sparse-core update (kernels_mask.cu)
 void launch_alpha(armor_ctx* c, const float* A, cudaStream_t s);

@@ -8,22 +8,20 @@
 // Both operands are plain fp32 in global memory.  Either may be K-major (k contiguous) or MN-major (m or n
 // contiguous); tcgen05 reads both from swizzled shared memory (MN-major 32-bit operands in the 128-byte swizzle
 // with 32-byte atoms, which TMA writes directly), so no transposed copies are made.
-// fp32-grade accuracy comes from splitting every operand chunk, in shared memory, into a tf32-exact high part
-// and an fp32 low part and issuing three MMAs (lo*hi + hi*lo + hi*hi) into one fp32 accumulator.
+// fp32-grade accuracy comes from splitting every operand chunk, in shared memory, into a high part and an fp32
+// low part and issuing three MMAs (lo*hi + hi*lo + hi*hi) into one fp32 accumulator.  The tensor core reads the
+// top 19 bits of a 32-bit tf32 operand and ignores the rest, so the raw fp32 word serves as the high part and
+// only the low part x - trunc_tf32(x) has to be written (checked against a masked copy: same bits).
 //
 // Persistent kernel, 320 threads:
 //   warp 0    : TMA producer (raw fp32 chunks of 32 along K; MN-major chunks as four 32 x 32 boxes)
 //   warp 1    : MMA issuer   (tcgen05.mma kind::tf32, 128 x 128 x 8, two accumulators of 128 TMEM columns)
-//   warps 2-5 : splitter     (raw chunk -> high part in place, low part next to it, proxy fence)
+//   warps 2-5 : splitter     (raw chunk -> low part next to it, proxy fence)
 //   warps 6-9 : epilogue     (D tile prefetched by TMA into swizzled shared memory, tcgen05.ld, alpha / beta
 //                             in place, TMA store: no strided global access)
 // Every wait is bounded; a wait that runs out raises a status word and the CTA leaves through the common
 // exit that frees its tensor memory.
 #include "tc_common.cuh"
-
-// The tensor core reads the top 19 bits of a 32-bit tf32 operand and ignores the rest, so the raw fp32 word
-// serves as the high part and only the low part has to be written (checked against the masked form: same bits).
-int g_tc_raw_hi = 1;
 
 namespace {
 
@@ -33,7 +31,7 @@ constexpr int TILE = 128, BK = 32;
 constexpr int NTHREADS = 320;
 constexpr int STAGES = 3;
 constexpr int OP_BYTES = TILE * BK * 4;           // 16 KiB: one operand chunk
-constexpr int STAGE_BYTES = 4 * OP_BYTES;         // A hi, A lo, B hi, B lo
+constexpr int STAGE_BYTES = 4 * OP_BYTES;         // A raw (= high part), A low part, B raw, B low part
 constexpr uint32_t TMEM_COLS = 256;               // two accumulators of 128 columns
 constexpr int EPI_BYTES = 32 * 64 * 4;            // per epilogue warp: 32 rows x 64 columns (half a tile row) as two swizzled boxes
 constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 4 * EPI_BYTES + 1024;
@@ -57,7 +55,6 @@ struct BParams {
   float alpha, beta;
   int32_t* status;
   int batch_fastest;                // 1: consecutive work items are consecutive batches (neighbouring column blocks)
-  int raw_hi;                       // 1: the high part is the raw fp32 word (the tensor core reads its top 19 bits)
 };
 
 __device__ __forceinline__ void load_operand(uint32_t dst, const CUtensorMap* map, const OpCoord& o, int b, int t, int kc,
@@ -215,7 +212,6 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             h.y = __uint_as_float(__float_as_uint(v.y) & 0xffffe000u);
             h.z = __uint_as_float(__float_as_uint(v.z) & 0xffffe000u);
             h.w = __uint_as_float(__float_as_uint(v.w) & 0xffffe000u);
-            if (!p.raw_hi) hi[idx] = h;
             lo[idx] = make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w);
           }
         }
@@ -326,7 +322,6 @@ armor_status launch(armor_ctx* c, const HostOp& A, const HostOp& B, BParams p, c
   if (!make_map_2d(&mB, B.base, B.inner, B.outer, B.ld, 32, B.c.mn_major ? 32 : TILE, B.c.mn_major != 0)) return ARMOR_ERR_CUDA;
   p.a = A.c; p.b = B.c;
   p.status = c->status;
-  p.raw_hi = g_tc_raw_hi;
   static bool attr = false;
   if (!attr) {
     if (cudaFuncSetAttribute(tc_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)

@@ -6,8 +6,7 @@
 // The tensor-core accumulator adds with truncation, so a long run of same-sign terms drifts by about
 // (K / 8) * passes * 2^-24.  The GEMM therefore drains its accumulator into C every K_SEGMENT columns of
 // the contraction (the additions into C are ordinary round-to-nearest fp32 adds).
-static int64_t K_SEGMENT = 1024;
-extern "C" void armor_debug_set_k_segment(int64_t k) { K_SEGMENT = k; }
+static const int64_t K_SEGMENT = 1024;
 
 armor_status prepare_H(armor_ctx* c, const float* H, cudaStream_t s) {
   launch_extract_hblocks(c, H, s);

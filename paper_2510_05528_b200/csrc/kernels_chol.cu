@@ -45,7 +45,7 @@ __host__ __device__ inline size_t panel_floats(int db) {
 
 __global__ void __launch_bounds__(NT, 1)
 chol_blocked_kernel(int mode, const float* __restrict__ Gmat, const float* __restrict__ rhs, float* __restrict__ out,
-                    const float* __restrict__ dotw, float* __restrict__ A, float* __restrict__ At, float ridge, int db,
+                    const float* __restrict__ dotw, float* __restrict__ A, float ridge, int db,
                     int w, double* __restrict__ part, int32_t* __restrict__ failflag, int32_t* __restrict__ status) {
   extern __shared__ float smem[];
   const PanelMap pm{db};
@@ -409,7 +409,7 @@ chol_blocked_kernel(int mode, const float* __restrict__ Gmat, const float* __res
 // Unblocked variant for block sizes that are not a multiple of 32: thread i owns row i.
 __global__ void chol_kernel(int mode, const float* __restrict__ Gmat, const float* __restrict__ rhs,
                             float* __restrict__ out, const float* __restrict__ dotw, float* __restrict__ A,
-                            float* __restrict__ At, float ridge, int db, double* __restrict__ part,
+                            float ridge, int db, double* __restrict__ part,
                             int32_t* __restrict__ failflag, int32_t* __restrict__ status) {
   extern __shared__ float smem[];
   const int ld = db + 1;
@@ -481,7 +481,6 @@ __global__ void chol_kernel(int mode, const float* __restrict__ Gmat, const floa
     if (mode == 0) {
       const float a = A[off + e] + x;
       A[off + e] = a;
-      At[off + (int64_t)cidx * db + r] = a;
       out[off + e] = x;
       acc += (double)rhs[off + e] * (double)x + lam * (double)x * (double)x;
     } else {
@@ -518,7 +517,7 @@ int chol_parts_per_block(int db, int nb) {
 }
 
 armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float* rhs, float* out, const float* dotw,
-                         float* A, float* At, int nb, double* part, cudaStream_t s) {
+                         float* A, int nb, double* part, cudaStream_t s) {
   const int db = c->db;
   if (db % NB == 0) {
     const int slices = chol_parts_per_block(db, nb);
@@ -531,7 +530,7 @@ armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float*
         return ARMOR_ERR_CUDA;
       attr_bytes = smem;
     }
-    chol_blocked_kernel<<<dim3(nb, slices), NT, smem, s>>>(mode, Gmat, rhs, out, dotw, A, At, c->cfg.ridge, db, w,
+    chol_blocked_kernel<<<dim3(nb, slices), NT, smem, s>>>(mode, Gmat, rhs, out, dotw, A, c->cfg.ridge, db, w,
                                                           part, c->failflag, c->status);
     c->launches++;
     return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
@@ -544,7 +543,7 @@ armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float*
     attr_set = true;
   }
   const int nt = ((db + 31) / 32) * 32;
-  chol_kernel<<<nb, nt < 64 ? 64 : nt, smem, s>>>(mode, Gmat, rhs, out, dotw, A, At, c->cfg.ridge, db, part,
+  chol_kernel<<<nb, nt < 64 ? 64 : nt, smem, s>>>(mode, Gmat, rhs, out, dotw, A, c->cfg.ridge, db, part,
                                                  c->failflag, c->status);
   c->launches++;
   return ARMOR_OK;

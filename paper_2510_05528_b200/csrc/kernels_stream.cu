@@ -81,14 +81,6 @@ __global__ void extract_hblocks_kernel(const float* __restrict__ H, float* __res
   }
 }
 
-__global__ void transpose_blocks_kernel(const float* __restrict__ in, float* __restrict__ out, int db) {
-  const int64_t off = (int64_t)blockIdx.x * db * db;
-  for (int e = threadIdx.x; e < db * db; e += blockDim.x) {
-    int r = e / db, cc = e % db;
-    out[off + (int64_t)cc * db + r] = in[off + e];
-  }
-}
-
 // ---- Gamma_M = Gamma (.) M and its squared norm -------------------------------------------------
 // One float4 per thread step; a mask byte covers m_group / 4 consecutive float4 (q4 = 1 or 2).
 __global__ void __launch_bounds__(NT) masked_copy_kernel(const float4* __restrict__ gam, const uint8_t* __restrict__ M,
@@ -410,11 +402,6 @@ void launch_scale_rows_cols(armor_ctx* c, const float* in, const float* colscale
 
 void launch_extract_hblocks(armor_ctx* c, const float* H, cudaStream_t s) {
   extract_hblocks_kernel<<<c->nbi, NT, 0, s>>>(H, c->hdiag, c->Hjj, c->d_in, c->db, c->cfg.h_mode == ARMOR_H_DIAG);
-  c->launches++;
-}
-
-void launch_transpose_blocks(armor_ctx* c, const float* in, float* out, int nb, cudaStream_t s) {
-  transpose_blocks_kernel<<<nb, NT, 0, s>>>(in, out, c->db);
   c->launches++;
 }
 
