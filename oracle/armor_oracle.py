@@ -37,6 +37,7 @@ import numpy as np
 FULL, DIAG = 0, 1
 L1_RANDOM, L1_GREEDY, UNIFORM_RANDOM, L2_RANDOM = 0, 1, 2, 3
 S_EXACT, S_BETA = 0, 1
+AB_EXACT, AB_GD = 0, 1
 PH_A, PH_B, PH_S, PH_MASK = 1, 2, 4, 8
 PH_ALL = 15
 
@@ -49,6 +50,7 @@ class OracleConfig:
     h_mode: int = FULL
     select_mode: int = L1_RANDOM
     s_step: int = S_EXACT
+    ab_step: int = AB_EXACT
     ridge: float = 1e-6
     seed: int = 0
     phases: int = PH_ALL
@@ -58,6 +60,7 @@ class OracleConfig:
 class IterInfo:
     """What one iteration did (diagnostics; the margins feed the parity tests)."""
     loss: dict = field(default_factory=dict)       # loss after each sub-step
+    tau_A: float = 0.0
     tau_B: float = 0.0
     tau_S: float = 0.0
     chol_failed: int = 0
@@ -213,6 +216,52 @@ def a_step(W, A, B, S, Hw, cfg: OracleConfig):
             continue
         A[i] = A[i] + np.linalg.solve(Gr, Gam.T).T
     return A, failed
+
+
+def a_step_gd(W, A, B, S, Hw, cfg: OracleConfig):
+    """The paper's own A update (Algorithm 2): one gradient step A <- A - eta_A grad_A L with the step of
+    Eq. lrA, eta_A = 1 / beta_A, beta_A = 2 sum_{i,j} || T_ij D_j T_ij^T ||_F, T = (W' (.) M) B and D_j the
+    j-th block of the diagonal weighting.  grad_{A_i} L = -2 E_i D T_i^T = -2 Gamma_i (Appendix D.1), so the move
+    is Gamma_i / (beta_A / 2).  Defined for the diagonal weighting only, like the paper's loss."""
+    db = cfg.d_block
+    d = np.diag(Hw)
+    T = bd_right(S, B)
+    E = np.asarray(W, dtype=np.float64) - bd_left(A, T)
+    nbo, nbi = A.shape[0], B.shape[0]
+    half_beta = 0.0
+    for i in range(nbo):
+        for j in range(nbi):
+            Tij = T[i * db:(i + 1) * db, j * db:(j + 1) * db]
+            half_beta += np.linalg.norm((Tij * d[j * db:(j + 1) * db][None, :]) @ Tij.T)
+    tau = 1.0 / half_beta if half_beta > 0.0 else 0.0
+    A = A.copy()
+    for i in range(nbo):
+        r = slice(i * db, (i + 1) * db)
+        A[i] = A[i] + tau * ((E[r] * d[None, :]) @ T[r].T)
+    return A, tau
+
+
+def b_step_gd(W, A, B, S, Hw, cfg: OracleConfig):
+    """The paper's own B update: B <- B - eta_B grad_B L with Eq. lrB, eta_B = 1 / beta_B,
+    beta_B = 2 sum_{i,j} || U_ij^T U_ij ||_F || D_j ||_F, U = A (W' (.) M) (Reading: S'^T S' for the printed
+    S'^T S, as in the derivation above it).  grad_{B_j} L = -2 U_j^T (E D)_j = -2 Gamma_j (Appendix D.2)."""
+    db = cfg.d_block
+    d = np.diag(Hw)
+    U = bd_left(A, S)
+    E = np.asarray(W, dtype=np.float64) - bd_right(U, B)
+    nbo, nbi = A.shape[0], B.shape[0]
+    half_beta = 0.0
+    for j in range(nbi):
+        dn = np.linalg.norm(d[j * db:(j + 1) * db])
+        for i in range(nbo):
+            Uij = U[i * db:(i + 1) * db, j * db:(j + 1) * db]
+            half_beta += np.linalg.norm(Uij.T @ Uij) * dn
+    tau = 1.0 / half_beta if half_beta > 0.0 else 0.0
+    B = B.copy()
+    for j in range(nbi):
+        c = slice(j * db, (j + 1) * db)
+        B[j] = B[j] + tau * (U[:, c].T @ (E[:, c] * d[c][None, :]))
+    return B, tau
 
 
 def _is_spd(Mx: np.ndarray) -> bool:
@@ -478,14 +527,22 @@ def bcd_iteration(W, A, B, S, M, Hw, cfg: OracleConfig, t: int, want_loss: bool 
     info = IterInfo()
     if want_loss:
         info.loss["start"] = proxy_loss(W, A, B, S, Hw)
+    if cfg.ab_step == AB_GD and cfg.h_mode != DIAG:
+        raise ValueError("the paper's gradient steps for A and B are defined for the diagonal weighting")
     if cfg.phases & PH_A:
-        A, f = a_step(W, A, B, S, Hw, cfg)
-        info.chol_failed += f
+        if cfg.ab_step == AB_GD:
+            A, info.tau_A = a_step_gd(W, A, B, S, Hw, cfg)
+        else:
+            A, f = a_step(W, A, B, S, Hw, cfg)
+            info.chol_failed += f
         if want_loss:
             info.loss["A"] = proxy_loss(W, A, B, S, Hw)
     if cfg.phases & PH_B:
-        B, info.tau_B, f = b_step(W, A, B, S, Hw, cfg)
-        info.chol_failed += f
+        if cfg.ab_step == AB_GD:
+            B, info.tau_B = b_step_gd(W, A, B, S, Hw, cfg)
+        else:
+            B, info.tau_B, f = b_step(W, A, B, S, Hw, cfg)
+            info.chol_failed += f
         if want_loss:
             info.loss["B"] = proxy_loss(W, A, B, S, Hw)
     if cfg.phases & PH_S:

@@ -627,6 +627,73 @@ def test_theorem_1_with_4_of_8_groups():
     assert np.all(M.reshape(32, -1, 8).sum(axis=2) == 4) and np.all(S[~M] == 0)
 
 
+# ------------------------------------------------------------------ the paper's gradient steps (Algorithm 2)
+def _grad_fd(f, X, eps=1e-6):
+    g = np.zeros_like(X)
+    it = np.nditer(X, flags=["multi_index"])
+    for _ in it:
+        ix = it.multi_index
+        Xp, Xm = X.copy(), X.copy()
+        Xp[ix] += eps
+        Xm[ix] -= eps
+        g[ix] = (f(Xp) - f(Xm)) / (2 * eps)
+    return g
+
+
+def test_gradient_steps_follow_finite_differences_and_the_descent_lemma():
+    """A and B updates of Algorithm 2 with the steps of Eq. lrA / lrB: the move is -eta * gradient with the
+    gradient checked by central differences, beta bounds the change of the gradient between two points, and the
+    loss drops by at least ||grad||^2 / (2 beta) (descent lemma for a beta-smooth function)."""
+    cfg, W, X = tiny(d_out=8, d_in=12, db=4, n=60)
+    H = O.gram(X)
+    Hw = O.weighting(H, O.DIAG)
+    oc = O.OracleConfig(4, h_mode=O.DIAG, ab_step=O.AB_GD)
+    rng = np.random.default_rng(20)
+    A, B, S, M = rand_state(W, H, oc, rng, scale=0.3)
+    L0 = O.proxy_loss(W, A, B, S, Hw)
+    # ---- A
+    gA = _grad_fd(lambda Z: O.proxy_loss(W, Z, B, S, Hw), A)
+    A1, tauA = O.a_step_gd(W, A, B, S, Hw, oc)
+    assert np.allclose(A1 - A, -0.5 * tauA * gA, rtol=1e-5, atol=1e-9 * np.abs(gA).max())
+    betaA = 2.0 / tauA
+    A2 = A + 0.2 * rng.standard_normal(A.shape)
+    gA2 = _grad_fd(lambda Z: O.proxy_loss(W, Z, B, S, Hw), A2)
+    assert np.linalg.norm(gA - gA2) <= betaA * np.linalg.norm(A - A2) * (1 + 1e-6)
+    LA = O.proxy_loss(W, A1, B, S, Hw)
+    assert LA <= L0 - np.sum(gA * gA) / (2 * betaA) * (1 - 1e-6)
+    # ---- B, from the new A
+    gB = _grad_fd(lambda Z: O.proxy_loss(W, A1, Z, S, Hw), B)
+    B1, tauB = O.b_step_gd(W, A1, B, S, Hw, oc)
+    assert np.allclose(B1 - B, -0.5 * tauB * gB, rtol=1e-5, atol=1e-9 * np.abs(gB).max())
+    betaB = 2.0 / tauB
+    B2 = B + 0.2 * rng.standard_normal(B.shape)
+    gB2 = _grad_fd(lambda Z: O.proxy_loss(W, A1, Z, S, Hw), B2)
+    assert np.linalg.norm(gB - gB2) <= betaB * np.linalg.norm(B - B2) * (1 + 1e-6)
+    assert O.proxy_loss(W, A1, B1, S, Hw) <= LA - np.sum(gB * gB) / (2 * betaB) * (1 - 1e-6)
+
+
+def test_theorem_1_for_the_papers_literal_continuous_update():
+    """Algorithm 1 with Algorithm 2 as printed: gradient steps for A, B and W' with the 1/beta steps, diagonal
+    weighting.  Lemma 1 / Theorem 1: the loss never increases and never exceeds the initialisation's."""
+    cfg, W, X = tiny(d_out=32, d_in=32, db=8, n=128)
+    H = O.gram(X)
+    oc = O.OracleConfig(8, h_mode=O.DIAG, ab_step=O.AB_GD, s_step=O.S_BETA, seed=4)
+    Hw = O.weighting(H, O.DIAG)
+    L0 = O.proxy_loss(W, *O.init(W, H, oc)[:3], Hw)
+    (A, B, S, M), infos = O.run(W, H, oc, 12)
+    prev = L0
+    for info in infos:
+        seq = [info.loss[k] for k in ("start", "A", "B", "S", "mask")]
+        assert np.isclose(seq[0], prev, rtol=1e-12)
+        for a, b in zip(seq, seq[1:]):
+            assert b <= a * (1 + 1e-12)
+        assert info.tau_A > 0 and info.tau_B > 0
+        prev = seq[-1]
+    assert prev < L0
+    with pytest.raises(ValueError):
+        O.bcd_iteration(W, A, B, S, M, H, O.OracleConfig(8, h_mode=O.FULL, ab_step=O.AB_GD), 0)
+
+
 def test_resume_is_bitwise():
     cfg, W, X = tiny(d_out=16, d_in=16, db=8, n=64)
     H = O.gram(X)
