@@ -55,6 +55,9 @@ enum { ARMOR_H_FULL = 0, ARMOR_H_DIAG = 1 };
 /* Group selection of the sparse-core update (Section 3.3.2; the other three are the ablation of Appendix E.1) */
 enum { ARMOR_SELECT_L1_RANDOM = 0, ARMOR_SELECT_L1_GREEDY = 1, ARMOR_SELECT_UNIFORM_RANDOM = 2, ARMOR_SELECT_L2_RANDOM = 3 };
 enum { ARMOR_S_EXACT = 0, ARMOR_S_BETA = 1 };
+/* Wrapper updates: exact (proximal) block solves, or the paper's own gradient steps with the 1/beta steps of
+ * Eq. lrA and Eq. lrB (Algorithm 2; defined for the diagonal weighting, so ARMOR_AB_GD needs ARMOR_H_DIAG). */
+enum { ARMOR_AB_EXACT = 0, ARMOR_AB_GD = 1 };
 /* How the dense contractions (Gram, .H) are evaluated on the tensor cores:
  *   FP32X3 : operands split into tf32 high and low parts, three tcgen05 passes
  *            accumulated in fp32 -- fp32-grade results (the parity mode);
@@ -76,6 +79,7 @@ typedef struct {
   int32_t precision;   /* ARMOR_PREC_* */
   int32_t normalize;   /* 1: armor_init applies the NoWag normalisation */
   int32_t phases;      /* bitmask of ARMOR_PHASE_*; 0 means all four */
+  int32_t ab_step;     /* ARMOR_AB_* */
   float ridge;         /* relative proximal ridge of the block solves (1e-6) */
   uint64_t seed;       /* seed of the counter-based group selection */
 } armor_config;

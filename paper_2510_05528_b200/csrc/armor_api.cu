@@ -27,6 +27,8 @@ armor_status check_config(const armor_config* cfg) {
   if (cfg->h_mode != ARMOR_H_FULL && cfg->h_mode != ARMOR_H_DIAG) return ARMOR_ERR_INVALID_ARG;
   if (cfg->select_mode < ARMOR_SELECT_L1_RANDOM || cfg->select_mode > ARMOR_SELECT_L2_RANDOM) return ARMOR_ERR_INVALID_ARG;
   if (cfg->s_step != ARMOR_S_EXACT && cfg->s_step != ARMOR_S_BETA) return ARMOR_ERR_INVALID_ARG;
+  if (cfg->ab_step != ARMOR_AB_EXACT && cfg->ab_step != ARMOR_AB_GD) return ARMOR_ERR_INVALID_ARG;
+  if (cfg->ab_step == ARMOR_AB_GD && cfg->h_mode != ARMOR_H_DIAG) return ARMOR_ERR_UNSUPPORTED;
   if (cfg->precision < ARMOR_PREC_FP32X3 || cfg->precision > ARMOR_PREC_SIMT) return ARMOR_ERR_INVALID_ARG;
   if (cfg->precision != ARMOR_PREC_SIMT) {
     // the tensor-core GEMM works on whole 128 x 128 tiles with K in steps of 32
@@ -152,6 +154,20 @@ void colblock_grams(armor_ctx* c, const float* U, const float* Y, const float* Y
   g.M = db; g.N = db; g.K = (int)c->d_out; g.batch = 2 * c->nbi; g.alpha = 1.f;
   g.batch_inner = c->nbi; g.sAb2 = 0; g.sBb2 = Y2 - Y; g.sCb2 = Cm2 - Cm;
   g.ksplit = pick_ksplit(g.batch, (int64_t)((db + 127) / 128) * ((db + 127) / 128), g.K);
+  launch_bgemm(c, g, s);
+}
+// Z_(i,j) = X_ij Y_ij^T (by_rows) or X_ij^T Y_ij for every d_block x d_block tile (i, j) of two W-shaped
+// matrices: the terms of the paper's smoothness constants (Eq. lrA: T_ij D_j T_ij^T, Eq. lrB: U_ij^T U_ij).
+void tile_grams(armor_ctx* c, const float* X, const float* Y, bool by_rows, float* Z, cudaStream_t s) {
+  const int db = c->db;
+  const int64_t d_in = c->d_in;
+  BGemm g{};
+  g.A = X; g.B = Y;
+  if (by_rows) { g.sAm = d_in; g.sAk = 1; g.sBk = 1; g.sBn = d_in; }
+  else         { g.sAm = 1; g.sAk = d_in; g.sBk = d_in; g.sBn = 1; }
+  g.sAb = db; g.sAb2 = (int64_t)db * d_in; g.sBb = db; g.sBb2 = (int64_t)db * d_in;
+  g.C = Z; g.sCb = (int64_t)db * db; g.sCb2 = (int64_t)c->nbi * db * db; g.sCm = db; g.sCn = 1;
+  g.M = db; g.N = db; g.K = db; g.batch = c->nbo * c->nbi; g.batch_inner = c->nbi; g.alpha = 1.f;
   launch_bgemm(c, g, s);
 }
 void block_mm(armor_ctx* c, const float* X, bool tX, const float* Y, bool tY, float* Z, int nb, cudaStream_t s) {
@@ -344,9 +360,24 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
     // ---- A-step: A_i += Gamma_i (G_i + lam I)^-1 -------------------------------------------
     if (ph & ARMOR_PHASE_A) {
       rowblock_grams(c, c->P, c->EH, c->T, c->G, c->GamA, s);   // G_i = T_i H_w T_i^T, Gamma_i = E_i H_w T_i^T
-      st = launch_chol(c, 0, c->G, c->GamA, c->dA, nullptr, A, nbo, c->partblk, s);
-      if (st != ARMOR_OK) return st;
-      launch_stage(c, is, 1, c->partblk, nbo * chol_parts_per_block(db, nbo), nbo, s);
+      if (c->cfg.ab_step == ARMOR_AB_GD) {
+        // the paper's gradient step (Algorithm 2): A_i += Gamma_i / (beta_A / 2), beta_A / 2 = sum_ij |T_ij D_j T_ij^T|_F
+        // (Eq. lrA; P = T D with the diagonal weighting)
+        const int64_t na = (int64_t)nbo * db * db;
+        tile_grams(c, c->P, c->T, true, c->V, s);
+        launch_block_fro_sum(c, c->V, nbo * nbi, nullptr, c->sc + SC_HB_A, s);
+        dot_to_ptr(c, c->GamA, c->GamA, na, c->sc + SC_TMP0, s);                     // |Gamma|^2
+        block_mm(c, c->GamA, false, c->G, false, c->dA, nbo, s);                     // Gamma_i G_i
+        dot_to_ptr(c, c->dA, c->GamA, na, c->sc + SC_TMP1, s);                       // sum_i <Gamma_i G_i, Gamma_i>
+        launch_stage(c, is, 7, nullptr, 0, 0, s);
+        if (cudaMemsetAsync(c->dA, 0, (size_t)na * sizeof(float), s) != cudaSuccess) return ARMOR_ERR_CUDA;
+        launch_axpy_slot(c, c->dA, c->GamA, na, SC_TAU_A, 1.f, s);                   // dA = tau Gamma
+        launch_axpy_slot(c, A, c->GamA, na, SC_TAU_A, 1.f, s);                       // A += tau Gamma
+      } else {
+        st = launch_chol(c, 0, c->G, c->GamA, c->dA, nullptr, A, nbo, c->partblk, s);
+        if (st != ARMOR_OK) return st;
+        launch_stage(c, is, 1, c->partblk, nbo * chol_parts_per_block(db, nbo), nbo, s);
+      }
       bd_left(c, c->dA, false, c->P, c->EH, d_out, d_in, -1.f, c->EH, 1.f, s);       // EH -= dA P
     } else {
       launch_stage(c, is, 1, nullptr, 0, 0, s);
@@ -357,10 +388,22 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       launch_zero_flags(c, s);
       bd_left(c, A, false, S, c->U, d_out, d_in, 1.f, nullptr, 0.f, s);              // U = A S
       colblock_grams(c, c->U, c->U, c->EH, c->C, c->GamB, s);   // C_j = U_j^T U_j, Gamma_j = U_j^T (E H_w)_j
-      st = launch_chol(c, 1, c->C, c->GamB, c->Delta, nullptr, nullptr, nbi, nullptr, s);
-      if (st != ARMOR_OK) return st;
-      st = launch_chol(c, 2, c->Hjj, c->Delta, c->Delta, c->GamB, nullptr, nbi, c->partblk, s);
-      if (st != ARMOR_OK) return st;
+      const bool b_gd = (c->cfg.ab_step == ARMOR_AB_GD);
+      if (b_gd) {
+        // the paper's gradient step: the direction is Gamma itself, the step 1 / (beta_B / 2) with
+        // beta_B / 2 = sum_ij |U_ij^T U_ij|_F |D_j|_F  (Eq. lrB)
+        const int64_t nbl = (int64_t)nbi * db * db;
+        if (cudaMemcpyAsync(c->Delta, c->GamB, (size_t)nbl * sizeof(float), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+          return ARMOR_ERR_CUDA;
+        tile_grams(c, c->U, c->U, false, c->V, s);
+        launch_block_fro_sum(c, c->V, nbo * nbi, c->hdiag, c->sc + SC_HB_B, s);
+        dot_to_ptr(c, c->GamB, c->GamB, nbl, c->sc + SC_GD_B, s);                    // <Gamma, Delta>
+      } else {
+        st = launch_chol(c, 1, c->C, c->GamB, c->Delta, nullptr, nullptr, nbi, nullptr, s);
+        if (st != ARMOR_OK) return st;
+        st = launch_chol(c, 2, c->Hjj, c->Delta, c->Delta, c->GamB, nullptr, nbi, c->partblk, s);
+        if (st != ARMOR_OK) return st;
+      }
       // direction in B: V = A R with R = S Delta; R H_w serves both V H_w = A (R H_w) and the carried P
       bd_right(c, S, c->Delta, false, c->Tmp, d_out, d_in, 1.f, nullptr, 0.f, s);    // R = S Delta
       st = rmul_H(c, c->Tmp, H, c->E, d_out, nullptr, nullptr, nullptr, nullptr, s); // R H_w
@@ -368,7 +411,8 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       bd_left(c, A, false, c->Tmp, c->V, d_out, d_in, 1.f, nullptr, 0.f, s);         // V = A R
       bd_left(c, A, false, c->E, c->VH, d_out, d_in, 1.f, nullptr, 0.f, s);          // V H_w = A (R H_w)
       dot_to_ptr(c, c->VH, c->V, c->wn, c->sc + SC_Q_B, s);
-      launch_stage(c, is, 2, c->partblk, nbi * chol_parts_per_block(db, nbi), nbi, s);
+      if (b_gd) launch_stage(c, is, 8, nullptr, 0, 0, s);
+      else launch_stage(c, is, 2, c->partblk, nbi * chol_parts_per_block(db, nbi), nbi, s);
       launch_axpy_slot(c, B, c->Delta, (int64_t)nbi * db * db, SC_TAU_B, 1.f, s);    // B += tau Delta
       launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_B, -1.f, s);                   // EH -= tau V H_w
       if (carry_P) launch_axpy_slot(c, c->P, c->E, c->wn, SC_TAU_B, 1.f, s);         // P += tau R H_w

@@ -26,6 +26,9 @@ enum {
   SC_BETA_K,     // ||B H_w B^T||_F^2 (BETA step)
   SC_TMP0,
   SC_TMP1,
+  SC_TAU_A,      // step of the A gradient step (ab_step GD)
+  SC_HB_A,       // beta_A / 2 of Eq. lrA
+  SC_HB_B,       // beta_B / 2 of Eq. lrB
   SC_COUNT = 32
 };
 
@@ -173,6 +176,9 @@ void launch_axpy_slot(armor_ctx* c, float* y, const float* x, int64_t n, int slo
 void launch_init(armor_ctx* c, const float* W, const float* H, float* Wbar, float* r1, float* r2,
                  float* A, float* B, float* S, uint8_t* M, cudaStream_t s);
 void launch_zero_scalars(armor_ctx* c, cudaStream_t s);
+// part[b] = weight_b * || X_b ||_F for the nblk blocks of db x db floats in X; weight_b = 1, or the Euclidean
+// norm of hdiag over the (b % nbi)-th block of columns; out = sum of the parts (fixed order)
+void launch_block_fro_sum(armor_ctx* c, const float* X, int nblk, const float* hdiag, double* out, cudaStream_t s);
 void launch_zero_flags(armor_ctx* c, cudaStream_t s);
 // per-iteration bookkeeping on the device: stage 0 start, 1 after A, 2 after B, 3 after S, 4 mask accept
 void launch_stage(armor_ctx* c, armor_iter_stats* st, int stage, const double* part, int npart, int nflag,

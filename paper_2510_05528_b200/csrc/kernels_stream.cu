@@ -282,6 +282,19 @@ __global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const 
     sc[SC_ACCEPT] = acc ? 1.0 : 0.0;
     if (acc) sc[SC_LOSS] += dl;
     if (st) { st->delta_L_mask = dl; st->mask_accepted = acc ? 1 : 0; st->loss_mask = sc[SC_LOSS]; }
+  } else if (stage == 7) {   // A gradient step with the step of Eq. lrA: tau = 1 / (beta_A / 2)
+    const double hb = sc[SC_HB_A], nrm = sc[SC_TMP0], q = sc[SC_TMP1];
+    const double tau = (hb > 0.0) ? 1.0 / hb : 0.0;
+    sc[SC_TAU_A] = tau;
+    sc[SC_DEC_A] = 2.0 * tau * nrm - tau * tau * q;   // exact decrease of the quadratic in A along Gamma
+    sc[SC_LOSS] -= sc[SC_DEC_A];
+    if (st) st->loss_A = sc[SC_LOSS];
+  } else if (stage == 8) {   // B gradient step with the step of Eq. lrB
+    const double hb = sc[SC_HB_B], gd = sc[SC_GD_B], q = sc[SC_Q_B];
+    const double tau = (hb > 0.0) ? 1.0 / hb : 0.0;
+    sc[SC_TAU_B] = tau;
+    sc[SC_LOSS] -= 2.0 * tau * gd - tau * tau * q;
+    if (st) { st->loss_B = sc[SC_LOSS]; st->tau_B = (float)tau; }
   } else if (stage == 5) {  // phases skipped: carry the loss forward
     if (st) { st->loss_A = st->loss_B = st->loss_S = st->loss_mask = sc[SC_LOSS]; }
   }
@@ -362,6 +375,30 @@ __global__ void mirror_lower_kernel(float* __restrict__ H, int64_t n) {
     const int64_t dr = r0 + j, dc = c0 + threadIdx.x;
     if (dr < n && dc < n && dc > dr) H[dr * n + dc] = tile[threadIdx.x][j];
   }
+}
+
+// part[b] = weight * || X_b ||_F for block b of db x db floats (the terms of beta_A and beta_B, Eq. lrA / lrB)
+__global__ void __launch_bounds__(NT) block_fro_kernel(const float4* __restrict__ X, int n4_per_block,
+                                                       const float* __restrict__ hdiag, int db, int nbi,
+                                                       double* __restrict__ part) {
+  const float4* xb = X + (int64_t)blockIdx.x * n4_per_block;
+  double acc = 0.0;
+  for (int i = threadIdx.x; i < n4_per_block; i += NT) {
+    const float4 v = xb[i];
+    float s = v.x * v.x;
+    s = fmaf(v.y, v.y, s);
+    s = fmaf(v.z, v.z, s);
+    s = fmaf(v.w, v.w, s);
+    acc += (double)s;
+  }
+  acc = block_reduce_sum(acc);
+  double wsum = 0.0;
+  if (hdiag) {
+    const float* h = hdiag + (int64_t)(blockIdx.x % nbi) * db;
+    for (int k = threadIdx.x; k < db; k += NT) wsum += (double)h[k] * (double)h[k];
+    wsum = block_reduce_sum(wsum);
+  }
+  if (threadIdx.x == 0) part[blockIdx.x] = sqrt(acc) * (hdiag ? sqrt(wsum) : 1.0);
 }
 
 inline int grid_for(int64_t n) {
@@ -475,6 +512,12 @@ void launch_mirror_lower(armor_ctx* c, float* H, int64_t n, cudaStream_t s) {
   const unsigned t = (unsigned)((n + 31) / 32);
   mirror_lower_kernel<<<dim3(t, t), dim3(32, 8), 0, s>>>(H, n);
   c->launches++;
+}
+
+void launch_block_fro_sum(armor_ctx* c, const float* X, int nblk, const float* hdiag, double* out, cudaStream_t s) {
+  block_fro_kernel<<<nblk, NT, 0, s>>>((const float4*)X, c->db * c->db / 4, hdiag, c->db, c->nbi, c->quadpart);
+  reduce_final_kernel<<<1, NT, 0, s>>>(c->quadpart, nblk, out);
+  c->launches += 2;
 }
 
 void launch_bf16_to_f32(armor_ctx* c, const void* in, const float* colscale, float* out, int64_t rows, int64_t cols,

@@ -137,12 +137,12 @@ def test_proxy_loss_matches_oracle(prec, h_mode, mid_data):
 
 # ------------------------------------------------------------------------- teacher-forced steps
 def run_teacher_forced(cfg, W, H32, prec, h_mode, n_steps, select=Bd.SELECT_L1_RANDOM, n_keep=2, m_group=4,
-                       s_step=Bd.S_EXACT, tol_scale=1.0):
-    ctx = make(cfg, prec, h_mode, select_mode=select, n_keep=n_keep, m_group=m_group, s_step=s_step)
+                       s_step=Bd.S_EXACT, tol_scale=1.0, ab_step=Bd.AB_EXACT):
+    ctx = make(cfg, prec, h_mode, select_mode=select, n_keep=n_keep, m_group=m_group, s_step=s_step, ab_step=ab_step)
     Hd = dev(H32)
     st = ctx.init(dev(W), Hd)
     oc = O.OracleConfig(cfg.d_block, h_mode=h_mode, seed=cfg.seed, select_mode=select, n_keep=n_keep,
-                        m_group=m_group, s_step=s_step)
+                        m_group=m_group, s_step=s_step, ab_step=ab_step)
     Hq = H32.astype(np.float64)
     Hw = O.weighting(Hq, h_mode)
     Wn = W.astype(np.float64)
@@ -228,6 +228,17 @@ def test_teacher_forced_paper_step_size_for_the_core(tiny_data):
     W, X, H32 = tiny_data
     for h_mode in (Bd.H_FULL, Bd.H_DIAG):
         run_teacher_forced(TINY, W, H32, Bd.PREC_FP32X3, h_mode, 4, s_step=Bd.S_BETA)
+
+
+@pytest.mark.parametrize("cfg_name", ["tiny", "mid"])
+def test_teacher_forced_paper_literal_continuous_update(cfg_name, tiny_data, mid_data):
+    """Algorithm 2 as printed: gradient steps for A, B (Eq. lrA, Eq. lrB) and for the core (Eq. lrWprime) with
+    the diagonal weighting of the paper's loss."""
+    cfg = TINY if cfg_name == "tiny" else MID
+    W, X, H32 = tiny_data if cfg_name == "tiny" else mid_data
+    worst, _ = run_teacher_forced(cfg, W, H32, Bd.PREC_FP32X3, Bd.H_DIAG, 4, s_step=Bd.S_BETA, ab_step=Bd.AB_GD)
+    print(f"paper-literal update on {cfg_name}: worst rel err {worst}")
+    run_teacher_forced(cfg, W, H32, Bd.PREC_SIMT, Bd.H_DIAG, 2, ab_step=Bd.AB_GD)
 
 
 BIG_BLOCK = TINY.with_(name="db256", d_out=512, d_in=768, d_block=256, n_tokens=5000, chunk_rows=2048, seed=21)

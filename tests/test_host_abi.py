@@ -44,12 +44,15 @@ def test_config_validation(lib):
         (Bd.make_config(576, 576, 144), 7),            # above 128 the block size must be a multiple of 32
         (Bd.make_config(256, 256, 32, h_mode=5), 1),
         (Bd.make_config(256, 256, 32, select_mode=4), 1),
+        (Bd.make_config(256, 256, 32, ab_step=2), 1),
+        (Bd.make_config(256, 256, 32, ab_step=Bd.AB_GD), 7),          # the paper's gradient steps need the diagonal weighting
         (Bd.make_config(256, 256, 32, ridge=-1.0), 1),
         (Bd.make_config(0, 256, 32), 2),
         (Bd.make_config(192, 192, 32, precision=Bd.PREC_TF32), 7),   # tensor-core tiles need multiples of 128
     ]
     for good in (Bd.make_config(256, 256, 32, n_keep=4, m_group=8), Bd.make_config(512, 512, 256),
-                 Bd.make_config(256, 256, 32, s_step=Bd.S_BETA)):
+                 Bd.make_config(256, 256, 32, s_step=Bd.S_BETA),
+                 Bd.make_config(256, 256, 32, ab_step=Bd.AB_GD, h_mode=Bd.H_DIAG)):
         assert Bd.armor_workspace_bytes(good) > 0
     for cfg, code in cases:
         n = C.c_size_t(0)
