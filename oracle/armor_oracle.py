@@ -37,7 +37,7 @@ import numpy as np
 FULL, DIAG = 0, 1
 L1_RANDOM, L1_GREEDY, UNIFORM_RANDOM, L2_RANDOM = 0, 1, 2, 3
 S_EXACT, S_BETA = 0, 1
-AB_EXACT, AB_GD = 0, 1
+AB_EXACT, AB_GD, AB_ADAM = 0, 1, 2
 PH_A, PH_B, PH_S, PH_MASK = 1, 2, 4, 8
 PH_ALL = 15
 
@@ -51,6 +51,10 @@ class OracleConfig:
     select_mode: int = L1_RANDOM
     s_step: int = S_EXACT
     ab_step: int = AB_EXACT
+    adam_lr: float = 1e-4          # Appendix F
+    adam_beta1: float = 0.9        # Reading: the defaults of Kingma & Ba, which the paper cites without values
+    adam_beta2: float = 0.999
+    adam_eps: float = 1e-8
     ridge: float = 1e-6
     seed: int = 0
     phases: int = PH_ALL
@@ -520,7 +524,46 @@ def mask_step(W, A, B, S, M, Hw, cfg: OracleConfig, t: int, info: IterInfo | Non
 # --------------------------------------------------------------------------
 # O4  one BCD iteration and the outer loop (Algorithm 1)
 # --------------------------------------------------------------------------
-def bcd_iteration(W, A, B, S, M, Hw, cfg: OracleConfig, t: int, want_loss: bool = True):
+def adam_state(A, B, S):
+    """First and second moment estimates of Adam for A, B and W', all zero."""
+    return {k: np.zeros_like(x, dtype=np.float64) for k, x in
+            (("mA", A), ("vA", A), ("mB", B), ("vB", B), ("mS", S), ("vS", S))}
+
+
+def joint_gradients(W, A, B, S, M, Hw, cfg: OracleConfig):
+    """Gradients of the loss with respect to A, B and W' at one and the same point (Appendix D.1-D.3):
+    -2 E_i H_w T_i^T, -2 U_j^T (E H_w)_j and -2 (A^T E H_w B^T) (.) M."""
+    db = cfg.d_block
+    T = bd_right(S, B)
+    U = bd_left(A, S)
+    E = np.asarray(W, dtype=np.float64) - bd_left(A, T)
+    EH = E @ Hw
+    gA = np.stack([-2.0 * EH[i * db:(i + 1) * db] @ T[i * db:(i + 1) * db].T for i in range(A.shape[0])])
+    gB = np.stack([-2.0 * U[:, j * db:(j + 1) * db].T @ EH[:, j * db:(j + 1) * db] for j in range(B.shape[0])])
+    gS = -2.0 * bd_left(bd_T(A), bd_right(EH, bd_T(B))) * M
+    return gA, gB, gS
+
+
+def adam_joint_step(W, A, B, S, M, Hw, cfg: OracleConfig, state: dict, t_adam: int):
+    """What the paper runs in practice (Section 3.3.1): one Adam step (Kingma & Ba, Algorithm 1 with bias
+    correction) on A, B and W' together, from gradients taken at the same point.  t_adam counts from 1.
+    The state dict is updated in place."""
+    b1, b2, lr, eps = cfg.adam_beta1, cfg.adam_beta2, cfg.adam_lr, cfg.adam_eps
+    grads = dict(zip("ABS", joint_gradients(W, A, B, S, M, Hw, cfg)))
+    new = {}
+    for k, theta in (("A", A), ("B", B), ("S", S)):
+        g = grads[k]
+        m = state["m" + k] = b1 * state["m" + k] + (1.0 - b1) * g
+        v = state["v" + k] = b2 * state["v" + k] + (1.0 - b2) * g * g
+        mhat = m / (1.0 - b1 ** t_adam)
+        vhat = v / (1.0 - b2 ** t_adam)
+        new[k] = theta - lr * mhat / (np.sqrt(vhat) + eps)
+    # Reading: the core is W' (.) M, so an entry that the sparse-core update has masked out stays zero even while
+    # its first moment is still decaying; the moments themselves are left alone when a mask changes.
+    return new["A"], new["B"], new["S"] * M
+
+
+def bcd_iteration(W, A, B, S, M, Hw, cfg: OracleConfig, t: int, want_loss: bool = True, opt_state: dict | None = None):
     """A-step, then B-step with the new A, then S-step with the new A and B
     (the order of Algorithm 2 / Lemma 1), then the sparse-core update
     (Algorithm 3).  Every sub-step recomputes the residual from scratch."""
@@ -529,6 +572,18 @@ def bcd_iteration(W, A, B, S, M, Hw, cfg: OracleConfig, t: int, want_loss: bool 
         info.loss["start"] = proxy_loss(W, A, B, S, Hw)
     if cfg.ab_step == AB_GD and cfg.h_mode != DIAG:
         raise ValueError("the paper's gradient steps for A and B are defined for the diagonal weighting")
+    if cfg.ab_step == AB_ADAM:
+        # joint Adam replaces the three sequential sub-steps; then the sparse-core update as usual
+        if opt_state is None:
+            raise ValueError("joint Adam needs its moment estimates (adam_state)")
+        A, B, S = adam_joint_step(W, A, B, S, M, Hw, cfg, opt_state, t + 1)
+        if want_loss:
+            info.loss["A"] = info.loss["B"] = info.loss["S"] = proxy_loss(W, A, B, S, Hw)
+        if cfg.phases & PH_MASK:
+            S, M = mask_step(W, A, B, S, M, Hw, cfg, t, info)
+            if want_loss:
+                info.loss["mask"] = proxy_loss(W, A, B, S, Hw)
+        return A, B, S, M, info
     if cfg.phases & PH_A:
         if cfg.ab_step == AB_GD:
             A, info.tau_A = a_step_gd(W, A, B, S, Hw, cfg)
@@ -556,7 +611,8 @@ def bcd_iteration(W, A, B, S, M, Hw, cfg: OracleConfig, t: int, want_loss: bool 
     return A, B, S, M, info
 
 
-def run(W, H, cfg: OracleConfig, n_iters: int, t_first: int = 0, state=None, want_loss: bool = True):
+def run(W, H, cfg: OracleConfig, n_iters: int, t_first: int = 0, state=None, want_loss: bool = True,
+        opt_state: dict | None = None):
     """Algorithm 1 without the normalisation (apply normalize() first if wanted).
     Returns the final (A, B, S, M) and the per-iteration IterInfo list."""
     Hw = weighting(H, cfg.h_mode)
@@ -566,8 +622,10 @@ def run(W, H, cfg: OracleConfig, n_iters: int, t_first: int = 0, state=None, wan
     else:
         A, B, S, M = (np.array(x) for x in state)
     infos = []
+    if cfg.ab_step == AB_ADAM and opt_state is None:
+        opt_state = adam_state(A, B, S)
     for k in range(n_iters):
-        A, B, S, M, info = bcd_iteration(W, A, B, S, M, Hw, cfg, t_first + k, want_loss)
+        A, B, S, M, info = bcd_iteration(W, A, B, S, M, Hw, cfg, t_first + k, want_loss, opt_state)
         infos.append(info)
     return (A, B, S, M), infos
 

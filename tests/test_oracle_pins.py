@@ -694,6 +694,61 @@ def test_theorem_1_for_the_papers_literal_continuous_update():
         O.bcd_iteration(W, A, B, S, M, H, O.OracleConfig(8, h_mode=O.FULL, ab_step=O.AB_GD), 0)
 
 
+def test_joint_adam_step_properties():
+    """The joint Adam step (Section 3.3.1; Kingma & Ba, Algorithm 1), pinned by what the algorithm's definition
+    fixes: (1) with zero moments the bias-corrected first step moves every entry by lr * sign(gradient);
+    (2) the three gradients are taken at the same point (A's move follows the finite-difference gradient at
+    the OLD B and W'); (3) masked-out entries of W' never move; (4) a constant gradient keeps the step at lr;
+    (5) the second step follows the recurrences written out by hand for one entry."""
+    cfg, W, X = tiny(d_out=8, d_in=12, db=4, n=60)
+    H = O.gram(X)
+    Hw = O.weighting(H, O.FULL)
+    oc = O.OracleConfig(4, ab_step=O.AB_ADAM, adam_lr=1e-3, adam_eps=1e-30)
+    rng = np.random.default_rng(21)
+    A, B, S, M = rand_state(W, H, oc, rng, scale=0.3)
+    st = O.adam_state(A, B, S)
+    gA_fd = _grad_fd(lambda Z: O.proxy_loss(W, Z, B, S, Hw), A)
+    gB_fd = _grad_fd(lambda Z: O.proxy_loss(W, A, Z, S, Hw), B)
+    gS_fd = _grad_fd(lambda Z: O.proxy_loss(W, A, B, Z * M, Hw), S)
+    gA, gB, gS = O.joint_gradients(W, A, B, S, M, Hw, oc)
+    for g, fd in ((gA, gA_fd), (gB, gB_fd), (gS, gS_fd)):
+        assert np.allclose(g, fd, rtol=1e-5, atol=1e-8 * np.abs(fd).max())
+    A1, B1, S1 = O.adam_joint_step(W, A, B, S, M, Hw, oc, st, 1)
+    assert np.allclose(A1 - A, -1e-3 * np.sign(gA_fd), rtol=1e-9)
+    assert np.allclose(B1 - B, -1e-3 * np.sign(gB_fd), rtol=1e-9)
+    assert np.allclose((S1 - S)[M], -1e-3 * np.sign(gS_fd[M]), rtol=1e-9)
+    assert np.all((S1 - S)[~M] == 0.0) and np.all(S1[~M] == 0.0)
+    # second step: recurrences by hand for one entry of A
+    g1 = gA[0, 1, 2]
+    g2 = O.joint_gradients(W, A1, B1, S1, M, Hw, oc)[0][0, 1, 2]
+    A2, _, _ = O.adam_joint_step(W, A1, B1, S1, M, Hw, oc, st, 2)
+    m2 = 0.9 * (0.1 * g1) + 0.1 * g2
+    v2 = 0.999 * (0.001 * g1 * g1) + 0.001 * g2 * g2
+    step = 1e-3 * (m2 / (1 - 0.9 ** 2)) / np.sqrt(v2 / (1 - 0.999 ** 2))
+    assert np.isclose(A2[0, 1, 2], A1[0, 1, 2] - step, rtol=1e-12, atol=0.0)
+    # a constant gradient: the step stays lr (quadratic with A only, far from its minimum along a fixed sign)
+    oc_eps = O.OracleConfig(4, ab_step=O.AB_ADAM, adam_lr=1e-6, adam_eps=1e-30)
+    st2 = O.adam_state(A, B, S)
+    Ak, Bk, Sk = A, B, S
+    for t in range(1, 4):
+        An, Bn, Sn = O.adam_joint_step(W, Ak, Bk, Sk, M, Hw, oc_eps, st2, t)
+        assert np.allclose(np.abs(An - Ak), 1e-6, rtol=1e-3)     # gradients barely change over 1e-6 moves
+        Ak, Bk, Sk = An, Bn, Sn
+
+
+def test_joint_adam_run_lowers_the_loss_and_keeps_the_pattern():
+    cfg, W, X = tiny(d_out=32, d_in=32, db=8, n=128)
+    H = O.gram(X)
+    oc = O.OracleConfig(8, h_mode=O.DIAG, ab_step=O.AB_ADAM, adam_lr=1e-3, seed=5)
+    Hw = O.weighting(H, O.DIAG)
+    L0 = O.proxy_loss(W, *O.init(W, H, oc)[:3], Hw)
+    (A, B, S, M), infos = O.run(W, H, oc, 40)
+    assert infos[-1].loss["mask"] < 0.9 * L0
+    for info in infos:      # the sparse-core update itself never raises the loss (Lemma 2), whatever Adam did before
+        assert info.loss["mask"] <= info.loss["S"] * (1 + 1e-12)
+    assert np.all(M.reshape(32, -1, 4).sum(axis=2) == 2) and np.all(S[~M] == 0)
+
+
 def test_resume_is_bitwise():
     cfg, W, X = tiny(d_out=16, d_in=16, db=8, n=64)
     H = O.gram(X)
