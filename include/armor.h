@@ -57,7 +57,11 @@ enum { ARMOR_SELECT_L1_RANDOM = 0, ARMOR_SELECT_L1_GREEDY = 1, ARMOR_SELECT_UNIF
 enum { ARMOR_S_EXACT = 0, ARMOR_S_BETA = 1 };
 /* Wrapper updates: exact (proximal) block solves, or the paper's own gradient steps with the 1/beta steps of
  * Eq. lrA and Eq. lrB (Algorithm 2; defined for the diagonal weighting, so ARMOR_AB_GD needs ARMOR_H_DIAG). */
-enum { ARMOR_AB_EXACT = 0, ARMOR_AB_GD = 1 };
+enum { ARMOR_AB_EXACT = 0, ARMOR_AB_GD = 1, ARMOR_AB_ADAM = 2 };
+/* ARMOR_AB_ADAM: what the paper runs in practice (Section 3.3.1): one joint Adam step on A, B and W' per
+ * iteration in place of the three sequential updates (s_step is then ignored), followed by the sparse-core
+ * update.  The moment estimates live in the context's workspace; armor_init and a call with t_first == 0
+ * reset them, later calls on the same context continue them. */
 /* How the dense contractions (Gram, .H) are evaluated on the tensor cores:
  *   FP32X3 : operands split into tf32 high and low parts, three tcgen05 passes
  *            accumulated in fp32 -- fp32-grade results (the parity mode);
@@ -81,6 +85,10 @@ typedef struct {
   int32_t phases;      /* bitmask of ARMOR_PHASE_*; 0 means all four */
   int32_t ab_step;     /* ARMOR_AB_* */
   float ridge;         /* relative proximal ridge of the block solves (1e-6) */
+  float adam_lr;       /* ARMOR_AB_ADAM: step size (0: 1e-4, Appendix F of the paper) */
+  float adam_beta1;    /* moment decay rates and epsilon (0: 0.9, 0.999, 1e-8, the defaults of the Adam paper) */
+  float adam_beta2;
+  float adam_eps;
   uint64_t seed;       /* seed of the counter-based group selection */
 } armor_config;
 

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libarmor.so")
 H_FULL, H_DIAG = 0, 1
 SELECT_L1_RANDOM, SELECT_L1_GREEDY, SELECT_UNIFORM_RANDOM, SELECT_L2_RANDOM = 0, 1, 2, 3
 S_EXACT, S_BETA = 0, 1
-AB_EXACT, AB_GD = 0, 1
+AB_EXACT, AB_GD, AB_ADAM = 0, 1, 2
 PREC_FP32X3, PREC_TF32, PREC_SIMT = 0, 1, 2
 PHASE_A, PHASE_B, PHASE_S, PHASE_MASK = 1, 2, 4, 8
 DTYPE_F32, DTYPE_BF16 = 0, 1
@@ -40,7 +40,8 @@ class armor_config(C.Structure):
     _fields_ = [("d_out", C.c_int64), ("d_in", C.c_int64), ("d_block", C.c_int32), ("n_keep", C.c_int32),
                 ("m_group", C.c_int32), ("h_mode", C.c_int32), ("select_mode", C.c_int32),
                 ("s_step", C.c_int32), ("precision", C.c_int32), ("normalize", C.c_int32),
-                ("phases", C.c_int32), ("ab_step", C.c_int32), ("ridge", C.c_float), ("seed", C.c_uint64)]
+                ("phases", C.c_int32), ("ab_step", C.c_int32), ("ridge", C.c_float), ("adam_lr", C.c_float),
+                ("adam_beta1", C.c_float), ("adam_beta2", C.c_float), ("adam_eps", C.c_float), ("seed", C.c_uint64)]
 
 
 STATS_DTYPE = np.dtype([("loss_start", "<f8"), ("loss_A", "<f8"), ("loss_B", "<f8"), ("loss_S", "<f8"),
@@ -110,9 +111,9 @@ def _stream() -> C.c_void_p:
 
 def make_config(d_out, d_in, d_block, *, n_keep=2, m_group=4, h_mode=H_FULL, select_mode=SELECT_L1_RANDOM,
                 s_step=S_EXACT, precision=PREC_FP32X3, normalize=0, phases=0, ab_step=AB_EXACT, ridge=1e-6,
-                seed=0) -> armor_config:
+                adam_lr=0.0, adam_beta1=0.0, adam_beta2=0.0, adam_eps=0.0, seed=0) -> armor_config:
     return armor_config(d_out, d_in, d_block, n_keep, m_group, h_mode, select_mode, s_step, precision,
-                        int(normalize), phases, ab_step, ridge, seed)
+                        int(normalize), phases, ab_step, ridge, adam_lr, adam_beta1, adam_beta2, adam_eps, seed)
 
 
 # ---------------------------------------------------------------- C entry points, same names

@@ -27,7 +27,10 @@ armor_status check_config(const armor_config* cfg) {
   if (cfg->h_mode != ARMOR_H_FULL && cfg->h_mode != ARMOR_H_DIAG) return ARMOR_ERR_INVALID_ARG;
   if (cfg->select_mode < ARMOR_SELECT_L1_RANDOM || cfg->select_mode > ARMOR_SELECT_L2_RANDOM) return ARMOR_ERR_INVALID_ARG;
   if (cfg->s_step != ARMOR_S_EXACT && cfg->s_step != ARMOR_S_BETA) return ARMOR_ERR_INVALID_ARG;
-  if (cfg->ab_step != ARMOR_AB_EXACT && cfg->ab_step != ARMOR_AB_GD) return ARMOR_ERR_INVALID_ARG;
+  if (cfg->ab_step < ARMOR_AB_EXACT || cfg->ab_step > ARMOR_AB_ADAM) return ARMOR_ERR_INVALID_ARG;
+  if (cfg->adam_lr < 0.f || cfg->adam_beta1 < 0.f || cfg->adam_beta1 >= 1.f || cfg->adam_beta2 < 0.f ||
+      cfg->adam_beta2 >= 1.f || cfg->adam_eps < 0.f)
+    return ARMOR_ERR_INVALID_ARG;
   if (cfg->ab_step == ARMOR_AB_GD && cfg->h_mode != ARMOR_H_DIAG) return ARMOR_ERR_UNSUPPORTED;
   if (cfg->precision < ARMOR_PREC_FP32X3 || cfg->precision > ARMOR_PREC_SIMT) return ARMOR_ERR_INVALID_ARG;
   if (cfg->precision != ARMOR_PREC_SIMT) {
@@ -106,6 +109,11 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
     TAKE(Hq1, float*, hbytes);
     TAKE(Hq2, float*, hbytes);
   } else if (c) { c->Hq1 = nullptr; c->Hq2 = nullptr; }
+  if (cfg.ab_step == ARMOR_AB_ADAM) {
+    TAKE(mA, float*, ao); TAKE(vA, float*, ao);
+    TAKE(mB, float*, bo); TAKE(vB, float*, bo);
+    TAKE(mS, float*, wbytes); TAKE(vS, float*, wbytes);
+  } else if (c) { c->mA = c->vA = c->mB = c->vB = c->mS = c->vS = nullptr; }
   TAKE(sc, double*, SC_COUNT * sizeof(double));
   TAKE(partials, double*, (size_t)8 * npart * sizeof(double));
   const int64_t nbmax = nbo > nbi ? nbo : nbi;
@@ -180,6 +188,16 @@ void block_mm(armor_ctx* c, const float* X, bool tX, const float* Y, bool tY, fl
   launch_bgemm(c, g, s);
 }
 
+armor_status reset_adam(armor_ctx* c, cudaStream_t s) {
+  if (c->cfg.ab_step != ARMOR_AB_ADAM) return ARMOR_OK;
+  const size_t ao = (size_t)c->nbo * c->db * c->db * sizeof(float), bo = (size_t)c->nbi * c->db * c->db * sizeof(float);
+  const size_t wb = (size_t)c->wn * sizeof(float);
+  ARMOR_CUDA_OK(cudaMemsetAsync(c->mA, 0, ao, s)); ARMOR_CUDA_OK(cudaMemsetAsync(c->vA, 0, ao, s));
+  ARMOR_CUDA_OK(cudaMemsetAsync(c->mB, 0, bo, s)); ARMOR_CUDA_OK(cudaMemsetAsync(c->vB, 0, bo, s));
+  ARMOR_CUDA_OK(cudaMemsetAsync(c->mS, 0, wb, s)); ARMOR_CUDA_OK(cudaMemsetAsync(c->vS, 0, wb, s));
+  return ARMOR_OK;
+}
+
 armor_status core_gradient(armor_ctx* c, const float* A, const float* B, cudaStream_t s) {
   // Gamma = A^T (E H_w) B^T  (minus half of the gradient display of Appendix D.3)
   bd_left(c, A, true, c->EH, c->Tmp, c->d_out, c->d_in, 1.f, nullptr, 0.f, s);
@@ -188,9 +206,15 @@ armor_status core_gradient(armor_ctx* c, const float* A, const float* B, cudaStr
 }
 
 armor_status residual_and_loss(armor_ctx* c, const float* W, const float* H, const float* A, const float* B,
-                               const float* S, double* out, cudaStream_t s) {
+                               const float* S, double* out, cudaStream_t s, bool exact_products = false) {
+  // exact_products: the two wrapper products on the fp32 CUDA-core kernel, whose products with 0 and 1 are
+  // exact, so that E vanishes exactly where W = A S B term by term (identity wrappers at the initialisation);
+  // the three-pass tensor-core product carries 22 bits of each operand
+  const int saved = g_tc_blocks;
+  if (exact_products) g_tc_blocks = 0;
   bd_right(c, S, B, false, c->T, c->d_out, c->d_in, 1.f, nullptr, 0.f, s);      // T = S B
   bd_left(c, A, false, c->T, c->E, c->d_out, c->d_in, -1.f, W, 1.f, s);         // E = W - A T
+  g_tc_blocks = saved;
   return rmul_H(c, c->E, H, c->EH, c->d_out, c->E, out, nullptr, nullptr, s);   // EH = E H_w, L = <EH, E>
 }
 
@@ -311,6 +335,7 @@ armor_status armor_init(armor_ctx* c, const float* d_W, const float* d_H, float*
   if (!c || !d_W || !d_H || !d_Wbar || !d_A || !d_B || !d_S || !d_M) return ARMOR_ERR_INVALID_ARG;
   if (c->cfg.normalize && (!d_r1 || !d_r2)) return ARMOR_ERR_INVALID_ARG;
   launch_init(c, d_W, d_H, d_Wbar, d_r1, d_r2, d_A, d_B, d_S, d_M, cs(stream));
+  if (reset_adam(c, cs(stream)) != ARMOR_OK) return ARMOR_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
 }
 
@@ -335,18 +360,30 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
   armor_status st = prepare_H(c, H, s);
   if (st != ARMOR_OK) return st;
   // W H_w is the same for every iteration of the call: E H_w = W H_w - A (T H_w)
-  st = rmul_H(c, W, H, c->WH, d_out, nullptr, nullptr, nullptr, nullptr, s);
-  if (st != ARMOR_OK) return st;
+  if (c->cfg.ab_step != ARMOR_AB_ADAM) {
+    st = rmul_H(c, W, H, c->WH, d_out, nullptr, nullptr, nullptr, nullptr, s);
+    if (st != ARMOR_OK) return st;
+  }
   // P = T H_w = S B H_w is formed by a dense product in the first iteration of a call only.  Afterwards it
   // follows the state: the B-step and the S-step each form R H_w for their own direction R (S Delta, resp.
   // Gamma_M B) to get the step length, and P moves by tau R H_w; the group updates add the rows
   // z H_w[block row] that their guard has formed already.  With a diagonal H_w the product is a column
   // scale and P is simply recomputed.
-  const bool carry_P = (c->cfg.h_mode == ARMOR_H_FULL);
+  const bool adam = (c->cfg.ab_step == ARMOR_AB_ADAM);
+  const bool carry_P = (c->cfg.h_mode == ARMOR_H_FULL) && !adam;
+  if (adam && t_first == 0 && reset_adam(c, s) != ARMOR_OK) return ARMOR_ERR_CUDA;
   for (int it = 0; it < n_iters; ++it) {
     armor_iter_stats* is = d_stats ? d_stats + it : nullptr;
     const int64_t t = t_first + it;
     launch_zero_scalars(c, s);
+    if (adam) {
+      // Adam normalises every entry's move, so a gradient that is exactly zero (the kept entries of the core at
+      // the initialisation, where E vanishes on them) must come out as zero: E H_w is formed from E itself, not
+      // as the difference W H_w - A P
+      st = residual_and_loss(c, W, H, A, B, S, c->sc + SC_L0, s, true);
+      if (st != ARMOR_OK) return st;
+      launch_stage(c, is, 0, nullptr, 0, 0, s);
+    } else {
     bd_right(c, S, B, false, c->T, d_out, d_in, 1.f, nullptr, 0.f, s);              // T = S B
     if (it == 0 || !carry_P) {
       st = rmul_H(c, c->T, H, c->P, d_out, nullptr, nullptr, nullptr, nullptr, s);   // P = T H_w
@@ -356,9 +393,26 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
     bd_left(c, A, false, c->T, c->E, d_out, d_in, -1.f, W, 1.f, s);                  // E = W - A T
     dot_to_ptr(c, c->EH, c->E, c->wn, c->sc + SC_L0, s);                             // L = <E H_w, E>
     launch_stage(c, is, 0, nullptr, 0, 0, s);
+    }
+
+    if (adam) {
+      // ---- joint Adam step on A, B and the core from gradients at one point (Section 3.3.1) --------------
+      const int64_t na = (int64_t)nbo * db * db, nbl = (int64_t)nbi * db * db;
+      rowblock_grams(c, c->EH, c->EH, c->T, c->G, c->GamA, s);                       // Gamma^A_i = E_i H_w T_i^T
+      bd_left(c, A, false, S, c->U, d_out, d_in, 1.f, nullptr, 0.f, s);              // U = A S
+      colblock_grams(c, c->U, c->U, c->EH, c->C, c->GamB, s);                        // Gamma^B_j = U_j^T (E H_w)_j
+      core_gradient(c, A, B, s);                                                     // Gamma = A^T E H_w B^T
+      launch_adam(c, A, c->GamA, c->mA, c->vA, na, nullptr, t + 1, s);
+      launch_adam(c, B, c->GamB, c->mB, c->vB, nbl, nullptr, t + 1, s);
+      launch_adam(c, S, c->Gam, c->mS, c->vS, c->wn, M, t + 1, s);
+      // the new state: residual, E H_w and the loss afresh
+      st = residual_and_loss(c, W, H, A, B, S, c->sc + SC_L0, s, true);
+      if (st != ARMOR_OK) return st;
+      launch_stage(c, is, 9, nullptr, 0, 0, s);
+    }
 
     // ---- A-step: A_i += Gamma_i (G_i + lam I)^-1 -------------------------------------------
-    if (ph & ARMOR_PHASE_A) {
+    if (!adam && (ph & ARMOR_PHASE_A)) {
       rowblock_grams(c, c->P, c->EH, c->T, c->G, c->GamA, s);   // G_i = T_i H_w T_i^T, Gamma_i = E_i H_w T_i^T
       if (c->cfg.ab_step == ARMOR_AB_GD) {
         // the paper's gradient step (Algorithm 2): A_i += Gamma_i / (beta_A / 2), beta_A / 2 = sum_ij |T_ij D_j T_ij^T|_F
@@ -379,12 +433,12 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
         launch_stage(c, is, 1, c->partblk, nbo * chol_parts_per_block(db, nbo), nbo, s);
       }
       bd_left(c, c->dA, false, c->P, c->EH, d_out, d_in, -1.f, c->EH, 1.f, s);       // EH -= dA P
-    } else {
+    } else if (!adam) {
       launch_stage(c, is, 1, nullptr, 0, 0, s);
     }
 
     // ---- B-step: block-Newton directions, one exact step --------------------------------------
-    if (ph & ARMOR_PHASE_B) {
+    if (!adam && (ph & ARMOR_PHASE_B)) {
       launch_zero_flags(c, s);
       bd_left(c, A, false, S, c->U, d_out, d_in, 1.f, nullptr, 0.f, s);              // U = A S
       colblock_grams(c, c->U, c->U, c->EH, c->C, c->GamB, s);   // C_j = U_j^T U_j, Gamma_j = U_j^T (E H_w)_j
@@ -416,12 +470,12 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       launch_axpy_slot(c, B, c->Delta, (int64_t)nbi * db * db, SC_TAU_B, 1.f, s);    // B += tau Delta
       launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_B, -1.f, s);                   // EH -= tau V H_w
       if (carry_P) launch_axpy_slot(c, c->P, c->E, c->wn, SC_TAU_B, 1.f, s);         // P += tau R H_w
-    } else {
+    } else if (!adam) {
       launch_stage(c, is, 2, nullptr, 0, 0, s);
     }
 
     // ---- S-step: exact line search along Gamma (.) M ------------------------------------------
-    if (ph & ARMOR_PHASE_S) {
+    if (!adam && (ph & ARMOR_PHASE_S)) {
       core_gradient(c, A, B, s);
       launch_masked_copy(c, c->Gam, M, c->U, SC_NRM_S, s);                           // U = Gamma (.) M
       bd_right(c, c->U, B, false, c->Tmp, d_out, d_in, 1.f, nullptr, 0.f, s);        // R = Gamma_M B
@@ -448,7 +502,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       launch_axpy_slot(c, S, c->U, c->wn, SC_TAU_S, 1.f, s);                         // S += tau Gamma_M
       launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_S, -1.f, s);                   // EH -= tau V H_w
       if (carry_P) launch_axpy_slot(c, c->P, c->E, c->wn, SC_TAU_S, 1.f, s);         // P += tau R H_w
-    } else {
+    } else if (!adam) {
       launch_stage(c, is, 3, nullptr, 0, 0, s);
     }
 

@@ -61,6 +61,7 @@ struct armor_ctx {
   // [nb, db, db] scratch
   float *G, *GamA, *dA, *C, *GamB, *Delta, *Hjj, *Kfull, *Ktmp;
   float *alpha, *hdiag;
+  float *mA, *vA, *mB, *vB, *mS, *vS;   // Adam moment estimates (ab_step ADAM)
   float *Hq1, *Hq2;      // [d_in, d_in] scratch of the paper's step size (s_step BETA, full weighting)
   float* gemm_slabs;     // 128 x 256 slabs of partial sums of the dense product's split tail tiles
   int64_t gemm_slab_count;
@@ -176,6 +177,10 @@ void launch_axpy_slot(armor_ctx* c, float* y, const float* x, int64_t n, int slo
 void launch_init(armor_ctx* c, const float* W, const float* H, float* Wbar, float* r1, float* r2,
                  float* A, float* B, float* S, uint8_t* M, cudaStream_t s);
 void launch_zero_scalars(armor_ctx* c, cudaStream_t s);
+// One Adam step (Kingma & Ba, Algorithm 1) on n parameters with gradient g = -2 * gamma; step counts from 1.
+// M != nullptr: theta is the N:M core, one mask byte per m_group entries, masked-out entries stay zero.
+void launch_adam(armor_ctx* c, float* theta, const float* gamma, float* m, float* v, int64_t n, const uint8_t* M,
+                 int64_t step, cudaStream_t s);
 // part[b] = weight_b * || X_b ||_F for the nblk blocks of db x db floats in X; weight_b = 1, or the Euclidean
 // norm of hdiag over the (b % nbi)-th block of columns; out = sum of the parts (fixed order)
 void launch_block_fro_sum(armor_ctx* c, const float* X, int nblk, const float* hdiag, double* out, cudaStream_t s);

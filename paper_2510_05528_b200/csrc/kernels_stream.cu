@@ -295,6 +295,9 @@ __global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const 
     sc[SC_TAU_B] = tau;
     sc[SC_LOSS] -= 2.0 * tau * gd - tau * tau * q;
     if (st) { st->loss_B = sc[SC_LOSS]; st->tau_B = (float)tau; }
+  } else if (stage == 9) {   // joint Adam step: the loss was evaluated afresh from the new state
+    sc[SC_LOSS] = sc[SC_L0];
+    if (st) st->loss_A = st->loss_B = st->loss_S = sc[SC_LOSS];
   } else if (stage == 5) {  // phases skipped: carry the loss forward
     if (st) { st->loss_A = st->loss_B = st->loss_S = st->loss_mask = sc[SC_LOSS]; }
   }
@@ -399,6 +402,32 @@ __global__ void __launch_bounds__(NT) block_fro_kernel(const float4* __restrict_
     wsum = block_reduce_sum(wsum);
   }
   if (threadIdx.x == 0) part[blockIdx.x] = sqrt(acc) * (hdiag ? sqrt(wsum) : 1.0);
+}
+
+// ---- Adam (Kingma & Ba, Algorithm 1, with bias correction) ----------------------------------------------
+__global__ void __launch_bounds__(NT) adam_kernel(float4* __restrict__ theta, const float4* __restrict__ gamma,
+                                                  float4* __restrict__ m, float4* __restrict__ v, int64_t n4,
+                                                  const uint8_t* __restrict__ M, int q4, float lr, float b1, float b2,
+                                                  float eps, float inv_bc1, float inv_bc2) {
+  for (int64_t i = (int64_t)blockIdx.x * NT + threadIdx.x; i < n4; i += (int64_t)gridDim.x * NT) {
+    const float4 ga = gamma[i];
+    float4 mm = m[i], vv = v[i], th = theta[i];
+    unsigned keep = 0xFu;
+    if (M) keep = (q4 == 1) ? M[i] : ((unsigned)M[i >> 1] >> (4 * (int)(i & 1)));
+    const float g[4] = {-2.f * ga.x, -2.f * ga.y, -2.f * ga.z, -2.f * ga.w};
+    float mo[4] = {mm.x, mm.y, mm.z, mm.w}, vo[4] = {vv.x, vv.y, vv.z, vv.w}, t[4] = {th.x, th.y, th.z, th.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float gk = ((keep >> k) & 1u) ? g[k] : 0.f;      // the core's gradient is masked
+      mo[k] = fmaf(b1, mo[k], (1.f - b1) * gk);
+      vo[k] = fmaf(b2, vo[k], (1.f - b2) * gk * gk);
+      const float upd = lr * (mo[k] * inv_bc1) / (sqrtf(vo[k] * inv_bc2) + eps);
+      t[k] = ((keep >> k) & 1u) ? t[k] - upd : 0.f;
+    }
+    m[i] = make_float4(mo[0], mo[1], mo[2], mo[3]);
+    v[i] = make_float4(vo[0], vo[1], vo[2], vo[3]);
+    theta[i] = make_float4(t[0], t[1], t[2], t[3]);
+  }
 }
 
 inline int grid_for(int64_t n) {
@@ -518,6 +547,18 @@ void launch_block_fro_sum(armor_ctx* c, const float* X, int nblk, const float* h
   block_fro_kernel<<<nblk, NT, 0, s>>>((const float4*)X, c->db * c->db / 4, hdiag, c->db, c->nbi, c->quadpart);
   reduce_final_kernel<<<1, NT, 0, s>>>(c->quadpart, nblk, out);
   c->launches += 2;
+}
+
+void launch_adam(armor_ctx* c, float* theta, const float* gamma, float* m, float* v, int64_t n, const uint8_t* M,
+                 int64_t step, cudaStream_t s) {
+  const float lr = c->cfg.adam_lr > 0.f ? c->cfg.adam_lr : 1e-4f;
+  const float b1 = c->cfg.adam_beta1 > 0.f ? c->cfg.adam_beta1 : 0.9f;
+  const float b2 = c->cfg.adam_beta2 > 0.f ? c->cfg.adam_beta2 : 0.999f;
+  const float eps = c->cfg.adam_eps > 0.f ? c->cfg.adam_eps : 1e-8f;
+  const double bc1 = 1.0 - pow((double)b1, (double)step), bc2 = 1.0 - pow((double)b2, (double)step);
+  adam_kernel<<<grid_for(n / 4), NT, 0, s>>>((float4*)theta, (const float4*)gamma, (float4*)m, (float4*)v, n / 4, M,
+                                            c->cfg.m_group / 4, lr, b1, b2, eps, (float)(1.0 / bc1), (float)(1.0 / bc2));
+  c->launches++;
 }
 
 void launch_bf16_to_f32(armor_ctx* c, const void* in, const float* colscale, float* out, int64_t rows, int64_t cols,

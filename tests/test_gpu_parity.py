@@ -241,6 +241,59 @@ def test_teacher_forced_paper_literal_continuous_update(cfg_name, tiny_data, mid
     run_teacher_forced(cfg, W, H32, Bd.PREC_SIMT, Bd.H_DIAG, 2, ab_step=Bd.AB_GD)
 
 
+@pytest.mark.parametrize("h_mode", [Bd.H_DIAG, Bd.H_FULL])
+def test_joint_adam_iterations_follow_the_oracle(h_mode, mid_data):
+    """ab_step = ADAM: one joint Adam step on A, B and the core per iteration, then the sparse-core update.
+    Teacher-forced on the state (the moment estimates stay on each side and see the same gradients); compared
+    are the MOVES of the iteration, which are of size lr, not the parameters themselves."""
+    W, X, H32 = mid_data
+    cfg, lr = MID, 1e-4          # the paper's step size (Appendix F)
+    ctx = make(cfg, Bd.PREC_FP32X3, h_mode, ab_step=Bd.AB_ADAM, adam_lr=lr)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    oc = O.OracleConfig(cfg.d_block, h_mode=h_mode, seed=cfg.seed, ab_step=O.AB_ADAM, adam_lr=lr)
+    Hq = H32.astype(np.float64)
+    Hw = O.weighting(Hq, h_mode)
+    Wn = W.astype(np.float64)
+    A, B, S, M = O.init(Wn, Hq, oc)
+    opt = O.adam_state(A, B, S)
+    for t in range(4):
+        load_state(st, A, B, S, M)
+        A0, B0, S0 = (host(x).astype(np.float64) for x in (st.A, st.B, st.S))
+        sg = ctx.read_stats(ctx.bcd_step(st, Hd, t, 1))[0]
+        gA, gB, gS = O.joint_gradients(Wn, A, B, S, M, Hw, oc)
+        A1, B1, S1, M1, info = O.bcd_iteration(Wn, A, B, S, M, Hw, oc, t, opt_state=opt)
+
+        def moves_agree(new_gpu, old_gpu, new_or, old_or, g, what):
+            # Adam normalises every entry's move to about lr whatever the size of its gradient, so an entry whose
+            # gradient is at rounding level may move the other way in fp32: a floating-point sign decision.
+            # Compared are the entries with a gradient clear of that level; the others are counted.
+            if not (g != 0.0).any():       # e.g. the kept core entries at the initialisation: E vanishes on them
+                assert np.array_equal(new_gpu, old_gpu), what
+                return
+            clear = np.abs(g) > 1e-3 * np.sqrt(np.mean(g[g != 0.0] ** 2))
+            assert clear.mean() > 0.9 * (g != 0.0).mean(), what
+            assert rel((new_gpu - old_gpu)[clear], (new_or - old_or)[clear]) < 1e-2, what
+        moves_agree(host(st.A), A0, A1, A, gA, "A")
+        moves_agree(host(st.B), B0, B1, B, gB, "B")
+        assert abs(sg["loss_start"] - info.loss["start"]) / info.loss["start"] < 1e-3
+        assert abs(sg["loss_S"] - info.loss["S"]) / info.loss["S"] < 1e-3
+        diff = mask_block_diffs(host(st.M), M1, cfg.d_block)
+        assert diff <= excused_blocks(info, 1e-5)
+        if not diff and sg["mask_accepted"] == info.mask_accepted:
+            Mk = M & M1                                   # entries the sparse-core update did not re-solve:
+            ng_row = cfg.d_in // 4                        # it re-solves the values of every selected group
+            for g in info.selected[info.selected >= 0]:
+                Mk[g // ng_row, 4 * (g % ng_row):4 * (g % ng_row) + 4] = False
+            moves_agree(np.where(Mk, host(st.S), 0.0), np.where(Mk, S0, 0.0), np.where(Mk, S1, 0.0),
+                        np.where(Mk, S, 0.0), np.where(Mk, gS, 0.0), "S")
+            assert abs(sg["loss_mask"] - info.loss["mask"]) / info.loss["mask"] < 1e-3
+        A, B, S, M = A1, B1, S1, M1
+    Mg = O.unpack_mask(host(st.M))
+    assert np.all(host(st.S)[~Mg] == 0.0)
+    assert ctx.device_status()[:4] == [0, 0, 0, 0]
+
+
 BIG_BLOCK = TINY.with_(name="db256", d_out=512, d_in=768, d_block=256, n_tokens=5000, chunk_rows=2048, seed=21)
 
 
