@@ -141,6 +141,12 @@ def test_init_ties_keep_lower_index_and_pack_roundtrip():
     assert np.all(O.unpack_mask(O.pack_mask(Mr)) == Mr)
     _, _, _, M48 = O.init(rng.standard_normal((4, 16)), np.eye(16), O.OracleConfig(8, n_keep=4, m_group=8))
     assert np.all(M48.reshape(4, 2, 8).sum(axis=2) == 4)
+    for n_keep in (5, 6):     # the denser patterns of Section 4.4: the n largest |w| of every eight (H = I)
+        Wn = rng.standard_normal((4, 16))
+        _, _, _, Mn = O.init(Wn, np.eye(16), O.OracleConfig(8, n_keep=n_keep, m_group=8))
+        kept = np.sort(np.abs(Wn).reshape(4, 2, 8), axis=2)[:, :, 8 - n_keep:]
+        assert np.array_equal(np.sort(np.abs(Wn * Mn).reshape(4, 2, 8), axis=2)[:, :, 8 - n_keep:], kept)
+        assert np.all(Mn.reshape(4, 2, 8).sum(axis=2) == n_keep)
 
 
 # ------------------------------------------------------------------ A-step
@@ -347,17 +353,19 @@ def test_group_solve_matches_brute_force_least_squares(h_mode):
             assert np.isclose(Lfrozen - red / alpha, Lbest, rtol=1e-9, atol=1e-12 * L0)
 
 
+@pytest.mark.parametrize("n_keep", [4, 5, 6])
 @pytest.mark.parametrize("h_mode", [O.FULL, O.DIAG])
-def test_group_solve_4_of_8_matches_brute_force_least_squares(h_mode):
-    """The 4:8 pattern: for a group and each of the 70 masks the four free values fitted by generic least
-    squares on the full loss agree with the closed form, and the mask step's choice is the best of the 70."""
+def test_group_solve_n_of_8_matches_brute_force_least_squares(h_mode, n_keep):
+    """The 4:8, 5:8 and 6:8 patterns (Section 4.4): for a group and each of its 70 / 56 / 28 masks the free
+    values fitted by generic least squares on the full loss agree with the closed form, and the mask step's
+    choice is the best of all masks."""
     cfg, W, X = tiny(d_out=8, d_in=16, db=8, n=60)
     H = O.gram(X)
     Hw = O.weighting(H, h_mode)
     R = X.T if h_mode == O.FULL else np.diag(np.sqrt(np.diag(H)))
-    oc = O.OracleConfig(8, n_keep=4, m_group=8, h_mode=h_mode, select_mode=O.L1_GREEDY, phases=O.PH_MASK)
+    oc = O.OracleConfig(8, n_keep=n_keep, m_group=8, h_mode=h_mode, select_mode=O.L1_GREEDY, phases=O.PH_MASK)
     A, B, S, M = rand_state(W, H, oc, np.random.default_rng(12), scale=0.3)
-    assert np.all(M.reshape(8, -1, 8).sum(axis=2) == 4)
+    assert np.all(M.reshape(8, -1, 8).sum(axis=2) == n_keep)
     Ad, Bd = O.bd_dense(A), O.bd_dense(B)
     Gamma = O.core_gradient(W, A, B, S, Hw)
     r, c = 5, 1
@@ -370,8 +378,8 @@ def test_group_solve_4_of_8_matches_brute_force_least_squares(h_mode):
     alpha = a @ a
     Kc = Bd[cols] @ Hw @ Bd[cols].T
     z = Gamma[r, cols] + alpha * Kc @ S[r, cols]
-    combos = list(itertools.combinations(range(8), 4))
-    assert len(combos) == 70
+    combos = list(itertools.combinations(range(8), n_keep))
+    assert len(combos) == {4: 70, 5: 56, 6: 28}[n_keep]
     for keep in combos[::7] + [combos[-1]]:
         ix = np.array(keep)
         Dm = np.stack([(np.outer(a, Bd[cols[p]]) @ R).reshape(-1) for p in keep], axis=1)
@@ -384,7 +392,7 @@ def test_group_solve_4_of_8_matches_brute_force_least_squares(h_mode):
     info = O.IterInfo()
     L0 = O.proxy_loss(W, A, B, S, Hw)
     S1, M1 = O.mask_step(W, A, B, S, M, Hw, oc, 0, info)
-    assert np.all(M1.reshape(8, -1, 8).sum(axis=2) == 4) and np.all(S1[~M1] == 0.0)
+    assert np.all(M1.reshape(8, -1, 8).sum(axis=2) == n_keep) and np.all(S1[~M1] == 0.0)
     assert O.proxy_loss(W, A, B, S1, Hw) <= L0 * (1 + 1e-12)
     for j in range(2):
         g = int(info.selected[0, j])
@@ -610,10 +618,11 @@ def test_theorem_1_monotone_and_below_init(h_mode, select):
     assert np.all(M.reshape(32, -1, 4).sum(axis=2) == 2) and np.all(S[~M] == 0)
 
 
-def test_theorem_1_with_4_of_8_groups():
+@pytest.mark.parametrize("n_keep", [4, 5, 6])
+def test_theorem_1_with_n_of_8_groups(n_keep):
     cfg, W, X = tiny(d_out=32, d_in=32, db=8, n=128)
     H = O.gram(X)
-    oc = O.OracleConfig(8, n_keep=4, m_group=8, seed=3)
+    oc = O.OracleConfig(8, n_keep=n_keep, m_group=8, seed=3)
     L0 = O.proxy_loss(W, *O.init(W, H, oc)[:3], H)
     (A, B, S, M), infos = O.run(W, H, oc, 6)
     prev = L0
@@ -624,7 +633,7 @@ def test_theorem_1_with_4_of_8_groups():
             assert b <= a * (1 + 1e-10)
         prev = seq[-1]
     assert prev < L0
-    assert np.all(M.reshape(32, -1, 8).sum(axis=2) == 4) and np.all(S[~M] == 0)
+    assert np.all(M.reshape(32, -1, 8).sum(axis=2) == n_keep) and np.all(S[~M] == 0)
 
 
 # ------------------------------------------------------------------ the paper's gradient steps (Algorithm 2)
