@@ -24,7 +24,7 @@
  *   - A, B: [d/d_block, d_block, d_block] fp32.  S: [d_out, d_in] fp32 with
  *     zeros outside the mask.  M: one byte per group of m_group consecutive
  *     columns, uint8 [d_out, d_in/m_group]; bit p set <=> column m*c+p kept.
- *   - N:M patterns: 2:4 and 4:8 (Section 4.4 of the paper names both).
+ *   - N:M patterns: 2:4, and 4:8, 5:8, 6:8 (Section 4.4 of the paper names them).
  */
 #ifndef ARMOR_H
 #define ARMOR_H
@@ -74,7 +74,7 @@ enum { ARMOR_DTYPE_F32 = 0, ARMOR_DTYPE_BF16 = 1 };
 typedef struct {
   int64_t d_out, d_in;
   int32_t d_block;     /* divides d_out and d_in; multiple of m_group; at most 256 */
-  int32_t n_keep;      /* N of N:M: 2 (with m_group 4) or 4 (with m_group 8) */
+  int32_t n_keep;      /* N of N:M: 2 (with m_group 4) or 4, 5, 6 (with m_group 8; Section 4.4) */
   int32_t m_group;     /* M of N:M: 4 or 8 */
   int32_t h_mode;      /* ARMOR_H_* */
   int32_t select_mode; /* ARMOR_SELECT_* (Section 3.3.2 / Appendix E.1) */
@@ -107,7 +107,7 @@ typedef struct {
 
 /* Scratch size for a configuration.  Error: INVALID_ARG (null), SHAPE
  * (d_block does not divide the dims, m_group does not divide d_block),
- * UNSUPPORTED (N:M other than 2:4 and 4:8; d_block > 256, not a multiple of 4, or above 128 and not a
+ * UNSUPPORTED (N:M other than 2:4, 4:8, 5:8, 6:8; d_block > 256, not a multiple of 4, or above 128 and not a
  * multiple of 32; tensor-core precisions with full weighting need d_out and d_in multiples of 128). */
 armor_status armor_workspace_bytes(const armor_config* cfg, size_t* bytes);
 

@@ -21,7 +21,8 @@ armor_status check_config(const armor_config* cfg) {
   if (cfg->d_out <= 0 || cfg->d_in <= 0 || cfg->d_block <= 0) return ARMOR_ERR_SHAPE;
   if (cfg->m_group <= 0 || cfg->n_keep <= 0 || cfg->n_keep > cfg->m_group) return ARMOR_ERR_SHAPE;
   if (cfg->d_out % cfg->d_block || cfg->d_in % cfg->d_block || cfg->d_block % cfg->m_group) return ARMOR_ERR_SHAPE;
-  if (!((cfg->n_keep == 2 && cfg->m_group == 4) || (cfg->n_keep == 4 && cfg->m_group == 8))) return ARMOR_ERR_UNSUPPORTED;
+  if (!((cfg->n_keep == 2 && cfg->m_group == 4) || (cfg->m_group == 8 && cfg->n_keep >= 4 && cfg->n_keep <= 6)))
+    return ARMOR_ERR_UNSUPPORTED;   // 2:4, and the 4:8, 5:8, 6:8 patterns of Section 4.4
   if (cfg->d_block > 256 || cfg->d_block % 4) return ARMOR_ERR_UNSUPPORTED;
   if (cfg->d_block > 128 && cfg->d_block % 32) return ARMOR_ERR_UNSUPPORTED;   // large blocks use the panel solver
   if (cfg->h_mode != ARMOR_H_FULL && cfg->h_mode != ARMOR_H_DIAG) return ARMOR_ERR_INVALID_ARG;

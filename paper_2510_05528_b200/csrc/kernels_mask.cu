@@ -62,18 +62,21 @@ __device__ __forceinline__ void pinv2(double k11, double k12, double k22, double
   red = z1 * w1 + z2 * w2;
 }
 
-// n x n SPD solve (n <= 4) by unpivoted Cholesky; false if a pivot is not positive (that mask is skipped).
-__device__ __forceinline__ bool chol_small(int n, const double (&Kin)[4][4], const double (&z)[4], double (&w)[4],
+constexpr int NK_MAX = 6;   // largest number of kept positions per group (6:8)
+
+// n x n SPD solve (n <= NK_MAX) by unpivoted Cholesky; false if a pivot is not positive (that mask is skipped).
+__device__ __forceinline__ bool chol_small(int n, const double (&Kin)[NK_MAX][NK_MAX], const double (&z)[NK_MAX],
+                                           double (&w)[NK_MAX],
                                            double& red) {
-  double L[4][4];
+  double L[NK_MAX][NK_MAX];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < NK_MAX; ++i) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < NK_MAX; ++j) {
       if (i >= n || j > i) continue;
       double sacc = Kin[i][j];
 #pragma unroll
-      for (int p = 0; p < 4; ++p)
+      for (int p = 0; p < NK_MAX; ++p)
         if (p < j) sacc -= L[i][p] * L[j][p];
       if (i == j) {
         if (!(sacc > 0.0) || !isfinite(sacc)) return false;
@@ -83,33 +86,33 @@ __device__ __forceinline__ bool chol_small(int n, const double (&Kin)[4][4], con
       }
     }
   }
-  double y[4];
+  double y[NK_MAX];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < NK_MAX; ++i) {
     if (i >= n) continue;
     double sacc = z[i];
 #pragma unroll
-    for (int p = 0; p < 4; ++p)
+    for (int p = 0; p < NK_MAX; ++p)
       if (p < i) sacc -= L[i][p] * y[p];
     y[i] = sacc / L[i][i];
   }
 #pragma unroll
-  for (int i = 3; i >= 0; --i) {
+  for (int i = NK_MAX - 1; i >= 0; --i) {
     if (i >= n) continue;
     double sacc = y[i];
 #pragma unroll
-    for (int p = 0; p < 4; ++p)
+    for (int p = 0; p < NK_MAX; ++p)
       if (p > i && p < n) sacc -= L[p][i] * w[p];
     w[i] = sacc / L[i][i];
   }
   red = 0.0;
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
+  for (int i = 0; i < NK_MAX; ++i)
     if (i < n) red += z[i] * w[i];
   return true;
 }
 
-// One CTA per (i, j) block of the core, N:M groups with M = MG (4 or 8) and N = n_keep (<= 4).
+// One CTA per (i, j) block of the core, N:M groups with M = MG (4 or 8) and N = n_keep (<= NK_MAX).
 // Pass 1: every group of the block is scored, keyed and the arg-min found by warp shuffles.
 // Pass 2: thread b < 2^MG evaluates the mask with bit pattern b (if it keeps exactly n_keep positions);
 // the best one is found with the oracle's order: larger reduction first; among equal reductions the
@@ -212,32 +215,32 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
   }
   const unsigned cand = threadIdx.x;
   bool ok = cand < (1u << MG) && __popc(cand) == n_keep;
-  double red = 0.0, wv[4] = {0.0, 0.0, 0.0, 0.0};
-  int pos[4] = {0, 0, 0, 0};
+  double red = 0.0, wv[NK_MAX] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
+  int pos[NK_MAX] = {0, 0, 0, 0, 0, 0};
   if (ok) {
     int cnt = 0;
 #pragma unroll
     for (int p = 0; p < MG; ++p)
-      if ((cand >> p) & 1u) { if (cnt < 4) pos[cnt] = p; ++cnt; }
+      if ((cand >> p) & 1u) { if (cnt < NK_MAX) pos[cnt] = p; ++cnt; }
     if (n_keep == 2) {
       pinv2((double)Kj[(int64_t)(lc + pos[0]) * db + lc + pos[0]], (double)Kj[(int64_t)(lc + pos[0]) * db + lc + pos[1]],
             (double)Kj[(int64_t)(lc + pos[1]) * db + lc + pos[1]], z[pos[0]], z[pos[1]], wv[0], wv[1], red);
     } else {
-      double Ks[4][4], zs[4];
+      double Ks[NK_MAX][NK_MAX], zs[NK_MAX];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < NK_MAX; ++i) {
         zs[i] = 0.0;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) Ks[i][j] = 0.0;
+        for (int j = 0; j < NK_MAX; ++j) Ks[i][j] = 0.0;
       }
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < NK_MAX; ++i) {
         if (i >= n_keep) continue;
 #pragma unroll
         for (int p = 0; p < MG; ++p)
           if (p == pos[i]) zs[i] = z[p];
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
+        for (int j = 0; j < NK_MAX; ++j)
           if (j < n_keep) Ks[i][j] = (double)Kj[(int64_t)(lc + pos[i]) * db + lc + pos[j]];
       }
       ok = chol_small(n_keep, Ks, zs, wv, red);
@@ -291,7 +294,7 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
 #pragma unroll
   for (int p = 0; p < MG; ++p) rec.old_val[p] = (float)sg_old[p];
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
+  for (int i = 0; i < NK_MAX; ++i)
     if (i < n_keep) rec.new_val[pos[i]] = (float)(wv[i] / a_r);
   // <Gamma, dS> restricted to this group: this block's share of <E H_w, V>
   double ehv = 0.0;

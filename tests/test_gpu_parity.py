@@ -210,16 +210,19 @@ def test_teacher_forced_ablation_selection_heuristics(select, tiny_data):
     run_teacher_forced(TINY, W, H32, Bd.PREC_FP32X3, Bd.H_FULL, 5, select=select)
 
 
+@pytest.mark.parametrize("n_keep", [4, 5, 6])
 @pytest.mark.parametrize("h_mode", [Bd.H_FULL, Bd.H_DIAG])
-def test_teacher_forced_4_of_8_groups(h_mode, tiny_data):
-    """The 4:8 pattern: top-4 of 8 at the initialisation, 70 masks with 4 x 4 solves per selected group."""
+def test_teacher_forced_n_of_8_groups(h_mode, n_keep, tiny_data):
+    """The 4:8, 5:8 and 6:8 patterns (Section 4.4): top-n of 8 at the initialisation, all 70 / 56 / 28 masks
+    with n x n solves per selected group."""
     W, X, H32 = tiny_data
-    ctx = make(TINY, Bd.PREC_SIMT, h_mode, n_keep=4, m_group=8)
+    ctx = make(TINY, Bd.PREC_SIMT, h_mode, n_keep=n_keep, m_group=8)
     st = ctx.init(dev(W), dev(H32))
-    _, _, S0, M0 = O.init(W.astype(np.float64), H32.astype(np.float64), O.OracleConfig(TINY.d_block, n_keep=4, m_group=8))
+    _, _, S0, M0 = O.init(W.astype(np.float64), H32.astype(np.float64),
+                          O.OracleConfig(TINY.d_block, n_keep=n_keep, m_group=8))
     assert np.array_equal(host(st.M), O.pack_mask(M0, 8)) and np.array_equal(host(st.S), S0.astype(np.float32))
-    worst, n_excused = run_teacher_forced(TINY, W, H32, Bd.PREC_FP32X3, h_mode, 8, n_keep=4, m_group=8)
-    print(f"4:8 h_mode={h_mode}: worst rel err {worst}, groups differing under the margin: {n_excused}")
+    worst, n_excused = run_teacher_forced(TINY, W, H32, Bd.PREC_FP32X3, h_mode, 8, n_keep=n_keep, m_group=8)
+    print(f"{n_keep}:8 h_mode={h_mode}: worst rel err {worst}, groups differing under the margin: {n_excused}")
     assert n_excused <= 2
 
 

@@ -38,7 +38,8 @@ def test_config_validation(lib):
     cases = [
         (Bd.make_config(256, 250, 32), 2),             # d_block does not divide d_in
         (Bd.make_config(256, 256, 30), 2),             # ... nor d_out; not a multiple of m_group either
-        (Bd.make_config(256, 256, 32, n_keep=3, m_group=8), 7),      # only 2:4 and 4:8
+        (Bd.make_config(256, 256, 32, n_keep=3, m_group=8), 7),      # only 2:4 and 4:8, 5:8, 6:8
+        (Bd.make_config(256, 256, 32, n_keep=7, m_group=8), 7),
         (Bd.make_config(256, 256, 32, n_keep=2, m_group=8), 7),
         (Bd.make_config(1024, 1024, 512), 7),          # d_block > 256
         (Bd.make_config(576, 576, 144), 7),            # above 128 the block size must be a multiple of 32
@@ -51,7 +52,8 @@ def test_config_validation(lib):
         (Bd.make_config(0, 256, 32), 2),
         (Bd.make_config(192, 192, 32, precision=Bd.PREC_TF32), 7),   # tensor-core tiles need multiples of 128
     ]
-    for good in (Bd.make_config(256, 256, 32, n_keep=4, m_group=8), Bd.make_config(512, 512, 256),
+    for good in (Bd.make_config(256, 256, 32, n_keep=4, m_group=8), Bd.make_config(256, 256, 32, n_keep=5, m_group=8),
+                 Bd.make_config(256, 256, 32, n_keep=6, m_group=8), Bd.make_config(512, 512, 256),
                  Bd.make_config(256, 256, 32, s_step=Bd.S_BETA),
                  Bd.make_config(256, 256, 32, ab_step=Bd.AB_GD, h_mode=Bd.H_DIAG),
                  Bd.make_config(256, 256, 32, ab_step=Bd.AB_ADAM, adam_lr=1e-3)):
