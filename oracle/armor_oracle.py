@@ -58,6 +58,7 @@ class OracleConfig:
     ridge: float = 1e-6
     seed: int = 0
     phases: int = PH_ALL
+    mask_sweeps: int = 1         # sparse-core updates (Algorithm 3) per continuous update; the paper runs 1
 
 
 @dataclass
@@ -75,6 +76,7 @@ class IterInfo:
     select_margin: np.ndarray | None = None        # [nbo, nbi] relative margin of the selection
     mask_margin: np.ndarray | None = None          # [nbo, nbi] relative margin of the mask sweep
     new_mask: np.ndarray | None = None             # [nbo, nbi] chosen mask byte
+    sweeps: list = field(default_factory=list)     # one IterInfo per sparse-core update of the iteration
 
 
 # --------------------------------------------------------------------------
@@ -563,6 +565,29 @@ def adam_joint_step(W, A, B, S, M, Hw, cfg: OracleConfig, state: dict, t_adam: i
     return new["A"], new["B"], new["S"] * M
 
 
+def mask_phase(W, A, B, S, M, Hw, cfg: OracleConfig, t: int, info: IterInfo):
+    """The sparse-core update of iteration t: Algorithm 3 run cfg.mask_sweeps times in a row, each run from
+    the state the previous one left (fresh residual, fresh gradient, fresh selection).
+    Reading: the paper alternates one continuous and one sparse-core update; with mask_sweeps = K the loop is
+    the same alternation with the continuous update skipped on K-1 of every K turns, so run k of iteration t
+    draws its selection with the counter t*K + k (for K = 1 this is t).  Each run keeps Lemma 2's guarantee,
+    so the loss cannot rise across the phase.  The record sums the loss changes evaluated, the runs accepted
+    and the groups changed; the selection fields are those of the last run."""
+    K = cfg.mask_sweeps
+    info.mask_accepted, info.delta_L_mask, info.groups_changed = 0, 0.0, 0
+    for k in range(K):
+        sub = IterInfo()
+        S, M = mask_step(W, A, B, S, M, Hw, cfg, t * K + k, sub)
+        info.sweeps.append(sub)
+        info.mask_accepted += sub.mask_accepted
+        info.delta_L_mask += sub.delta_L_mask
+        info.groups_changed += sub.groups_changed
+    last = info.sweeps[-1]
+    info.selected, info.select_margin = last.selected, last.select_margin
+    info.mask_margin, info.new_mask = last.mask_margin, last.new_mask
+    return S, M
+
+
 def bcd_iteration(W, A, B, S, M, Hw, cfg: OracleConfig, t: int, want_loss: bool = True, opt_state: dict | None = None):
     """A-step, then B-step with the new A, then S-step with the new A and B
     (the order of Algorithm 2 / Lemma 1), then the sparse-core update
@@ -580,7 +605,7 @@ def bcd_iteration(W, A, B, S, M, Hw, cfg: OracleConfig, t: int, want_loss: bool 
         if want_loss:
             info.loss["A"] = info.loss["B"] = info.loss["S"] = proxy_loss(W, A, B, S, Hw)
         if cfg.phases & PH_MASK:
-            S, M = mask_step(W, A, B, S, M, Hw, cfg, t, info)
+            S, M = mask_phase(W, A, B, S, M, Hw, cfg, t, info)
             if want_loss:
                 info.loss["mask"] = proxy_loss(W, A, B, S, Hw)
         return A, B, S, M, info
@@ -605,7 +630,7 @@ def bcd_iteration(W, A, B, S, M, Hw, cfg: OracleConfig, t: int, want_loss: bool 
         if want_loss:
             info.loss["S"] = proxy_loss(W, A, B, S, Hw)
     if cfg.phases & PH_MASK:
-        S, M = mask_step(W, A, B, S, M, Hw, cfg, t, info)
+        S, M = mask_phase(W, A, B, S, M, Hw, cfg, t, info)
         if want_loss:
             info.loss["mask"] = proxy_loss(W, A, B, S, Hw)
     return A, B, S, M, info

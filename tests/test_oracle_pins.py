@@ -636,6 +636,50 @@ def test_theorem_1_with_n_of_8_groups(n_keep):
     assert np.all(M.reshape(32, -1, 8).sum(axis=2) == n_keep) and np.all(S[~M] == 0)
 
 
+@pytest.mark.parametrize("h_mode", [O.FULL, O.DIAG])
+def test_several_sparse_core_updates_per_iteration(h_mode):
+    """mask_sweeps = K: K runs of Algorithm 3 after one continuous update.  Pinned to the single-run step,
+    which has its own pins: the phase equals K mask-only iterations numbered t*K .. t*K+K-1 started from the
+    state after the continuous update; K = 1 is the plain iteration; the loss (evaluated from the activations,
+    not the Gram) never rises from run to run; the summed record matches the runs."""
+    cfg, W, X = tiny(d_out=32, d_in=32, db=8, n=128)
+    H = O.gram(X)
+    Hw = O.weighting(H, h_mode)
+    Xw = X if h_mode == O.FULL else np.diag(np.sqrt(np.diag(H)))
+    K, t = 3, 5
+    oc = O.OracleConfig(8, h_mode=h_mode, seed=6, mask_sweeps=K)
+    A, B, S, M = rand_state(W, H, oc, np.random.default_rng(3), scale=0.2)
+    A1, B1, S1, M1, info = O.bcd_iteration(W, A, B, S, M, Hw, oc, t)
+    # the same thing by hand: continuous update only, then K single runs with their own counters
+    cont = O.OracleConfig(8, h_mode=h_mode, seed=6, phases=O.PH_A | O.PH_B | O.PH_S)
+    only = O.OracleConfig(8, h_mode=h_mode, seed=6, phases=O.PH_MASK)
+    A2, B2, S2, M2, _ = O.bcd_iteration(W, A, B, S, M, Hw, cont, t)
+    losses = [loss_from_X(W, A2, B2, S2, Xw)]
+    changed = 0
+    for k in range(K):
+        _, _, S2, M2, sub = O.bcd_iteration(W, A2, B2, S2, M2, Hw, only, t * K + k)
+        losses.append(loss_from_X(W, A2, B2, S2, Xw))
+        changed += sub.groups_changed
+        assert np.array_equal(sub.selected, info.sweeps[k].selected)
+    assert np.array_equal(A1, A2) and np.array_equal(B1, B2) and np.array_equal(S1, S2) and np.array_equal(M1, M2)
+    for a, b in zip(losses, losses[1:]):
+        assert b <= a * (1 + 1e-10)
+    assert losses[-1] < losses[0]
+    assert len(info.sweeps) == K and info.groups_changed == changed > 0
+    assert info.mask_accepted == sum(x.mask_accepted for x in info.sweeps)
+    assert np.isclose(info.loss["mask"], losses[-1], rtol=1e-9)
+    accepted_change = sum(x.delta_L_mask for x in info.sweeps if x.mask_accepted)
+    assert np.isclose(losses[-1] - losses[0], accepted_change, rtol=1e-6, atol=1e-9 * losses[0])
+    # the runs of one iteration draw different groups (different counters), and K = 1 is the plain iteration
+    assert any(not np.array_equal(info.sweeps[0].selected, info.sweeps[k].selected) for k in range(1, K))
+    one = O.OracleConfig(8, h_mode=h_mode, seed=6, mask_sweeps=1)
+    plain = O.OracleConfig(8, h_mode=h_mode, seed=6)
+    r1 = O.bcd_iteration(W, A, B, S, M, Hw, one, t)
+    r0 = O.bcd_iteration(W, A, B, S, M, Hw, plain, t)
+    assert all(np.array_equal(x, y) for x, y in zip(r1[:4], r0[:4]))
+    assert np.all(M1.reshape(32, -1, 4).sum(axis=2) == 2) and np.all(S1[~M1] == 0)
+
+
 # ------------------------------------------------------------------ the paper's gradient steps (Algorithm 2)
 def _grad_fd(f, X, eps=1e-6):
     g = np.zeros_like(X)
