@@ -84,6 +84,9 @@ typedef struct {
   int32_t normalize;   /* 1: armor_init applies the NoWag normalisation */
   int32_t phases;      /* bitmask of ARMOR_PHASE_*; 0 means all four */
   int32_t ab_step;     /* ARMOR_AB_* */
+  int32_t mask_sweeps; /* sparse-core updates (Algorithm 3) per iteration, each from the state the previous one
+                          left, run k of iteration t drawing its groups with the counter t*K + k; 0 means 1,
+                          the paper's alternation; at most 64 */
   float ridge;         /* relative proximal ridge of the block solves (1e-6) */
   float adam_lr;       /* ARMOR_AB_ADAM: step size (0: 1e-4, Appendix F of the paper) */
   float adam_beta1;    /* moment decay rates and epsilon (0: 0.9, 0.999, 1e-8, the defaults of the Adam paper) */
@@ -97,10 +100,10 @@ typedef struct {
  * step; loss_start itself is evaluated from the residual. */
 typedef struct {
   double loss_start, loss_A, loss_B, loss_S, loss_mask;
-  double delta_L_mask;   /* exact loss change of the iteration's group updates */
+  double delta_L_mask;   /* exact loss change of the iteration's group updates (summed over the sweeps) */
   float tau_B, tau_S;    /* exact step lengths of the B-step and S-step */
-  int32_t groups_changed;/* groups whose mask changed (0 if rejected) */
-  int32_t mask_accepted; /* 1 if the group updates were kept */
+  int32_t groups_changed;/* groups whose mask changed, summed over the sweeps (rejected sweeps count 0) */
+  int32_t mask_accepted; /* sweeps whose group updates were kept (0 or 1 with one sweep) */
   int32_t chol_failed;   /* blocks skipped because a Cholesky pivot was <= 0 */
   int32_t reserved;
 } armor_iter_stats;

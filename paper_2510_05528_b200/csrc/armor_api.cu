@@ -29,6 +29,7 @@ armor_status check_config(const armor_config* cfg) {
   if (cfg->select_mode < ARMOR_SELECT_L1_RANDOM || cfg->select_mode > ARMOR_SELECT_L2_RANDOM) return ARMOR_ERR_INVALID_ARG;
   if (cfg->s_step != ARMOR_S_EXACT && cfg->s_step != ARMOR_S_BETA) return ARMOR_ERR_INVALID_ARG;
   if (cfg->ab_step < ARMOR_AB_EXACT || cfg->ab_step > ARMOR_AB_ADAM) return ARMOR_ERR_INVALID_ARG;
+  if (cfg->mask_sweeps < 0 || cfg->mask_sweeps > 64) return ARMOR_ERR_INVALID_ARG;
   if (cfg->adam_lr < 0.f || cfg->adam_beta1 < 0.f || cfg->adam_beta1 >= 1.f || cfg->adam_beta2 < 0.f ||
       cfg->adam_beta2 >= 1.f || cfg->adam_eps < 0.f)
     return ARMOR_ERR_INVALID_ARG;
@@ -371,6 +372,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
   // z H_w[block row] that their guard has formed already.  With a diagonal H_w the product is a column
   // scale and P is simply recomputed.
   const bool adam = (c->cfg.ab_step == ARMOR_AB_ADAM);
+  const int sweeps = c->cfg.mask_sweeps > 0 ? c->cfg.mask_sweeps : 1;
   const bool carry_P = (c->cfg.h_mode == ARMOR_H_FULL) && !adam;
   if (adam && t_first == 0 && reset_adam(c, s) != ARMOR_OK) return ARMOR_ERR_CUDA;
   for (int it = 0; it < n_iters; ++it) {
@@ -380,8 +382,8 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
     if (adam) {
       // Adam normalises every entry's move, so a gradient that is exactly zero (the kept entries of the core at
       // the initialisation, where E vanishes on them) must come out as zero: E H_w is formed from E itself, not
-      // as the difference W H_w - A P
-      st = residual_and_loss(c, W, H, A, B, S, c->sc + SC_L0, s, true);
+      // as the difference W H_w - A P, and at t = 0 (identity wrappers) with the exact fp32 products
+      st = residual_and_loss(c, W, H, A, B, S, c->sc + SC_L0, s, t == 0);
       if (st != ARMOR_OK) return st;
       launch_stage(c, is, 0, nullptr, 0, 0, s);
     } else {
@@ -407,7 +409,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       launch_adam(c, B, c->GamB, c->mB, c->vB, nbl, nullptr, t + 1, s);
       launch_adam(c, S, c->Gam, c->mS, c->vS, c->wn, M, t + 1, s);
       // the new state: residual, E H_w and the loss afresh
-      st = residual_and_loss(c, W, H, A, B, S, c->sc + SC_L0, s, true);
+      st = residual_and_loss(c, W, H, A, B, S, c->sc + SC_L0, s);
       if (st != ARMOR_OK) return st;
       launch_stage(c, is, 9, nullptr, 0, 0, s);
     }
@@ -507,16 +509,34 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       launch_stage(c, is, 3, nullptr, 0, 0, s);
     }
 
-    // ---- sparse-core update (Algorithm 3) -----------------------------------------------------
+    // ---- sparse-core update (Algorithm 3), mask_sweeps times ------------------------------------
     if (ph & ARMOR_PHASE_MASK) {
-      core_gradient(c, A, B, s);
       launch_alpha(c, A, s);
       block_mm(c, B, false, c->Hjj, false, c->Ktmp, nbi, s);                         // B_j H_jj
       block_mm(c, c->Ktmp, false, B, true, c->Kfull, nbi, s);                        // K_j = B_j H_jj B_j^T
-      launch_mask_select(c, c->Gam, S, M, t, s);
-      launch_mask_quadratic(c, A, B, H, s);
-      launch_stage(c, is, 4, c->partblk, nbo * nbi, 0, s);
-      launch_mask_commit(c, S, M, is, s);
+      for (int sw = 0; sw < sweeps; ++sw) {
+        if (sw > 0) {
+          // E H_w for the state the previous run left
+          if (adam) {
+            st = residual_and_loss(c, W, H, A, B, S, c->sc + SC_TMP0, s);
+            if (st != ARMOR_OK) return st;
+          } else {
+            if (carry_P) {
+              launch_mask_carry_P(c, c->P, s);                                       // P += dS B H_w (if accepted)
+            } else {
+              bd_right(c, S, B, false, c->T, d_out, d_in, 1.f, nullptr, 0.f, s);     // T = S B
+              st = rmul_H(c, c->T, H, c->P, d_out, nullptr, nullptr, nullptr, nullptr, s);
+              if (st != ARMOR_OK) return st;
+            }
+            bd_left(c, A, false, c->P, c->EH, d_out, d_in, -1.f, c->WH, 1.f, s);     // E H_w = W H_w - A P
+          }
+        }
+        core_gradient(c, A, B, s);
+        launch_mask_select(c, c->Gam, S, M, t * sweeps + sw, s);
+        launch_mask_quadratic(c, A, B, H, s);
+        launch_stage(c, is, 4, c->partblk, nbo * nbi, 0, s);
+        launch_mask_commit(c, S, M, is, s);
+      }
       if (carry_P && it + 1 < n_iters) launch_mask_carry_P(c, c->P, s);              // P += dS B H_w (if accepted)
     } else {
       launch_stage(c, is, 4, nullptr, 0, 0, s);

@@ -390,7 +390,7 @@ __global__ void mask_commit_kernel(const SelRec* __restrict__ sel, int nblocks, 
   }
   atomicAdd(&changed, mine);
   __syncthreads();
-  if (threadIdx.x == 0 && st) st->groups_changed = changed;
+  if (threadIdx.x == 0 && st) st->groups_changed += changed;   // summed over the sweeps of the iteration
 }
 
 // The accepted group updates change T H_w = S B H_w by the rows (delta^T B_j[group rows, :]) H_w[j-th block

@@ -281,7 +281,7 @@ __global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const 
     sc[SC_DL_M] = dl;
     sc[SC_ACCEPT] = acc ? 1.0 : 0.0;
     if (acc) sc[SC_LOSS] += dl;
-    if (st) { st->delta_L_mask = dl; st->mask_accepted = acc ? 1 : 0; st->loss_mask = sc[SC_LOSS]; }
+    if (st) { st->delta_L_mask += dl; st->mask_accepted += acc ? 1 : 0; st->loss_mask = sc[SC_LOSS]; }   // summed over the sweeps
   } else if (stage == 7) {   // A gradient step with the step of Eq. lrA: tau = 1 / (beta_A / 2)
     const double hb = sc[SC_HB_A], nrm = sc[SC_TMP0], q = sc[SC_TMP1];
     const double tau = (hb > 0.0) ? 1.0 / hb : 0.0;

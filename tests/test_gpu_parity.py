@@ -226,6 +226,55 @@ def test_teacher_forced_n_of_8_groups(h_mode, n_keep, tiny_data):
     assert n_excused <= 2
 
 
+@pytest.mark.parametrize("ab_step", [Bd.AB_EXACT, Bd.AB_ADAM], ids=["exact", "adam"])
+@pytest.mark.parametrize("h_mode", [Bd.H_FULL, Bd.H_DIAG])
+def test_several_sparse_core_updates_per_iteration(h_mode, ab_step, mid_data):
+    """mask_sweeps = 3: three runs of the sparse-core update per iteration, each from the state the previous one
+    left.  Teacher-forced; a decision under the margin in any run excuses its block for the whole iteration."""
+    W, X, H32 = mid_data
+    cfg, K = MID, 3
+    adam = dict(ab_step=Bd.AB_ADAM, adam_lr=1e-4) if ab_step == Bd.AB_ADAM else {}
+    ctx = make(cfg, Bd.PREC_FP32X3, h_mode, mask_sweeps=K, **adam)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    oc = O.OracleConfig(cfg.d_block, h_mode=h_mode, seed=cfg.seed, mask_sweeps=K,
+                        **({"ab_step": O.AB_ADAM, "adam_lr": 1e-4} if adam else {}))
+    Hq = H32.astype(np.float64)
+    Hw = O.weighting(Hq, h_mode)
+    Wn = W.astype(np.float64)
+    A, B, S, M = O.init(Wn, Hq, oc)
+    opt = O.adam_state(A, B, S) if adam else None
+    tol = TOL[Bd.PREC_FP32X3]
+    compared = 0
+    for t in range(3):
+        load_state(st, A, B, S, M)
+        sg = ctx.read_stats(ctx.bcd_step(st, Hd, t, 1))[0]
+        A, B, S, M, info = O.bcd_iteration(Wn, A, B, S, M, Hw, oc, t, opt_state=opt)
+        assert len(info.sweeps) == K
+        excused = set().union(*(excused_blocks(x, tol["margin"]) for x in info.sweeps))
+        marginal_guard = any(abs(x.delta_L_mask) <= tol["margin"] * info.loss["S"] for x in info.sweeps)
+        diff = mask_block_diffs(host(st.M), M, cfg.d_block)
+        if sg["mask_accepted"] != info.mask_accepted:
+            assert marginal_guard, "accept/reject differs although no guard was marginal"
+            continue
+        assert diff <= excused
+        if not diff:
+            compared += 1
+            assert sg["groups_changed"] == info.groups_changed
+            assert abs(sg["loss_mask"] - info.loss["mask"]) / info.loss["mask"] < 1e-3
+            # the change is a difference of fp32 quantities of the size of the loss: K runs, each good to a few
+            # 1e-9 of the loss (right after an Adam step from the initialisation the change itself is that small)
+            assert abs(sg["delta_L_mask"] - info.delta_L_mask) <= 1e-3 * abs(info.delta_L_mask) + 1e-8 * info.loss["start"]
+            if not adam:
+                assert rel(host(st.S), S) < tol["S"]
+        # the tracked loss equals a fresh evaluation of the state the sweeps left
+        assert abs(ctx.proxy_loss(st, Hd).item() - sg["loss_mask"]) / sg["loss_mask"] < 1e-4
+    assert compared >= 1
+    Mg = O.unpack_mask(host(st.M))
+    assert np.all(Mg.reshape(cfg.d_out, -1, 4).sum(axis=2) == 2) and np.all(host(st.S)[~Mg] == 0.0)
+    assert ctx.device_status()[:4] == [0, 0, 0, 0]
+
+
 def test_teacher_forced_paper_step_size_for_the_core(tiny_data):
     """s_step = BETA: the paper's 1/beta_W' step (Eq. lrWprime) instead of the exact line search."""
     W, X, H32 = tiny_data
