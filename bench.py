@@ -330,6 +330,32 @@ def run_ours(args, cfg):
                      "gemm_share_of_step": gms32 / ms32 if ms32 > 0 else None}
         del ctx32
 
+    # ---- the paper's own operating point and two neighbours, on the same W and H (context only, rank-local):
+    # diagonal weighting with the exact block solves; diagonal weighting with the joint Adam step (what the paper
+    # runs, for 20,000 iterations per layer); full weighting with four sparse-core updates per iteration
+    other_modes = None
+    if args.other_modes:
+        other_modes = {}
+        H.zero_()
+        ctx.gram(X_d, H)
+        for name, kw, iters in (("diag_exact", dict(h_mode=Bd.H_DIAG), lcfg.n_iters),
+                                ("diag_adam_lr1e-4", dict(h_mode=Bd.H_DIAG, ab_step=Bd.AB_ADAM), 10 * lcfg.n_iters),
+                                ("full_adam_lr1e-4", dict(h_mode=Bd.H_FULL, ab_step=Bd.AB_ADAM), lcfg.n_iters),
+                                ("full_exact_4_sweeps", dict(h_mode=Bd.H_FULL, mask_sweeps=4), lcfg.n_iters)):
+            cx = Bd.ArmorContext(lcfg.d_out, lcfg.d_in, lcfg.d_block, device=dev, precision=prec, seed=lcfg.seed, **kw)
+            sx = cx.init(W_d, H)
+            cx.bcd_step(sx, H, 0, 3, want_stats=False)          # warm-up
+            sx = cx.init(W_d, H)
+            l_init = float(cx.proxy_loss(sx, H).item())
+            ms_x, _ = t_phase(lambda: cx.bcd_step(sx, H, 0, iters, want_stats=False))
+            other_modes[name] = {"iterations": iters, "ms_per_iteration": ms_x / iters,
+                                 "iterations_per_s": iters / (ms_x / 1e3),
+                                 "loss_init": l_init, "loss_final": float(cx.proxy_loss(sx, H).item()),
+                                 "device_status": cx.device_status()[:4]}
+            if "adam" in name:
+                other_modes[name]["s_per_20000_iterations"] = 20000 * ms_x / iters / 1e3
+            del cx, sx
+
     # ---- end to end (host buffers)
     if args.no_e2e:
         ms_e2e = None
@@ -365,6 +391,7 @@ def run_ours(args, cfg):
                 "ms_per_step": ms_e2e / args.steps if ms_e2e else None},
         "gpu_launches": int(launches),
         "tf32_mode": tf32_mode,
+        "other_modes": other_modes,
         "clocks": clocks,
         "roofline": {"bound": "tensor", "kernel": "tc_gemm_kernel (tcgen05 tf32, Gram + dense .H contractions)",
                      "achieved": achieved, "peak": tf32_peak, "unit": "TFLOP/s", "frac": achieved / tf32_peak,
@@ -400,6 +427,9 @@ def main():
                     help="profiling aid: BCD iterations per step instead of the workload's")
     ap.add_argument("--no-e2e", action="store_true", help="profiling aid: skip the host-buffer leg")
     ap.add_argument("--no-tf32", action="store_true", help="skip the extra measurement of the one-pass tf32 mode")
+    ap.add_argument("--other-modes", action="store_true",
+                    help="also time the BCD loop with the diagonal weighting, the joint Adam step and several "
+                         "sparse-core updates per iteration (a few seconds more)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
