@@ -137,11 +137,12 @@ inline cudaStream_t cs(armor_stream_t s) { return reinterpret_cast<cudaStream_t>
 // per-block Gram-type products over a long contraction, two at a time (the second pair of operands is
 // addressed through the distance between workspace buffers)
 void rowblock_grams(armor_ctx* c, const float* P, const float* P2, const float* T, float* G, float* G2, cudaStream_t s) {
-  // G_i = P_i T_i^T, G2_i = P2_i T_i^T  (contraction over d_in), batch over row-blocks i
+  // G_i = P_i T_i^T, G2_i = P2_i T_i^T  (contraction over d_in), batch over row-blocks i; P == nullptr: G2 only
   const int db = c->db;
-  if (g_tc_blocks && tc_gram_ok(c) && tc_rowblock_gram(c, P, T, G, s) == ARMOR_OK &&
+  if (g_tc_blocks && tc_gram_ok(c) && (!P || tc_rowblock_gram(c, P, T, G, s) == ARMOR_OK) &&
       tc_rowblock_gram(c, P2, T, G2, s) == ARMOR_OK)
     return;
+  if (!P) { P = P2; G = G2; }   // fallback kernel: the same Gram twice into the same place
   BGemm g{};
   g.A = P; g.sAb = (int64_t)db * c->d_in; g.sAm = c->d_in; g.sAk = 1;
   g.B = T; g.sBb = (int64_t)db * c->d_in; g.sBk = 1; g.sBn = c->d_in;
@@ -152,11 +153,12 @@ void rowblock_grams(armor_ctx* c, const float* P, const float* P2, const float* 
   launch_bgemm(c, g, s);
 }
 void colblock_grams(armor_ctx* c, const float* U, const float* Y, const float* Y2, float* Cm, float* Cm2, cudaStream_t s) {
-  // C_j = U_j^T Y_j, C2_j = U_j^T Y2_j  (contraction over d_out), batch over column-blocks j
+  // C_j = U_j^T Y_j, C2_j = U_j^T Y2_j  (contraction over d_out), batch over column-blocks j; Y == nullptr: C2 only
   const int db = c->db;
-  if (g_tc_blocks && tc_gram_ok(c) && tc_colblock_gram(c, U, Y, Cm, s) == ARMOR_OK &&
+  if (g_tc_blocks && tc_gram_ok(c) && (!Y || tc_colblock_gram(c, U, Y, Cm, s) == ARMOR_OK) &&
       tc_colblock_gram(c, U, Y2, Cm2, s) == ARMOR_OK)
     return;
+  if (!Y) { Y = Y2; Cm = Cm2; }
   BGemm g{};
   g.A = U; g.sAb = db; g.sAm = 1; g.sAk = c->d_in;
   g.B = Y; g.sBb = db; g.sBk = c->d_in; g.sBn = 1;
@@ -401,9 +403,9 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
     if (adam) {
       // ---- joint Adam step on A, B and the core from gradients at one point (Section 3.3.1) --------------
       const int64_t na = (int64_t)nbo * db * db, nbl = (int64_t)nbi * db * db;
-      rowblock_grams(c, c->EH, c->EH, c->T, c->G, c->GamA, s);                       // Gamma^A_i = E_i H_w T_i^T
+      rowblock_grams(c, nullptr, c->EH, c->T, nullptr, c->GamA, s);                  // Gamma^A_i = E_i H_w T_i^T
       bd_left(c, A, false, S, c->U, d_out, d_in, 1.f, nullptr, 0.f, s);              // U = A S
-      colblock_grams(c, c->U, c->U, c->EH, c->C, c->GamB, s);                        // Gamma^B_j = U_j^T (E H_w)_j
+      colblock_grams(c, c->U, nullptr, c->EH, nullptr, c->GamB, s);                  // Gamma^B_j = U_j^T (E H_w)_j
       core_gradient(c, A, B, s);                                                     // Gamma = A^T E H_w B^T
       launch_adam(c, A, c->GamA, c->mA, c->vA, na, nullptr, t + 1, s);
       launch_adam(c, B, c->GamB, c->mB, c->vB, nbl, nullptr, t + 1, s);
