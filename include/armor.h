@@ -69,7 +69,7 @@ enum { ARMOR_AB_EXACT = 0, ARMOR_AB_GD = 1, ARMOR_AB_ADAM = 2 };
  *   SIMT   : fp32 CUDA-core reference path (slow; for debugging and checks). */
 enum { ARMOR_PREC_FP32X3 = 0, ARMOR_PREC_TF32 = 1, ARMOR_PREC_SIMT = 2 };
 enum { ARMOR_PHASE_A = 1, ARMOR_PHASE_B = 2, ARMOR_PHASE_S = 4, ARMOR_PHASE_MASK = 8 };
-enum { ARMOR_DTYPE_F32 = 0, ARMOR_DTYPE_BF16 = 1 };
+enum { ARMOR_DTYPE_F32 = 0, ARMOR_DTYPE_BF16 = 1, ARMOR_DTYPE_BF16_SPARSE = 2 };
 
 typedef struct {
   int64_t d_out, d_in;
@@ -168,14 +168,22 @@ armor_status armor_proxy_loss(armor_ctx* ctx, const float* d_Wbar, const float* 
  * which the core S and the wrapped activations B x are rounded to bf16 and
  * multiplied on the bf16 tensor-core path with fp32 accumulation (the two thin
  * wrapper products stay fp32-grade; y is rounded to bf16 once).
- * d_M is accepted for symmetry and may be NULL (S already carries the zeros). */
+ * ARMOR_DTYPE_BF16_SPARSE: the same bf16 x and y, with the core on the sparse
+ * tensor cores (the 2:4 speed-up the paper's inference measurements rely on,
+ * Section 4.3): S is packed to its kept values (bf16) and 2-bit positions taken
+ * from d_M on every call; needs the 2:4 pattern, d_M non-NULL and d_out, d_in
+ * multiples of 128, else UNSUPPORTED / INVALID_ARG.  A group of d_M with more
+ * than two kept positions is counted in device status word 4 and contributes
+ * its first two.  With the other two dtypes d_M may be NULL (S already carries
+ * the zeros). */
 armor_status armor_apply(armor_ctx* ctx, const float* d_A, const float* d_B, const float* d_S,
                          const uint8_t* d_M, const float* d_r1, const float* d_r2, const void* d_x,
                          void* d_y, int32_t xy_dtype, int64_t n_tokens, armor_stream_t stream);
 
 /* Copies up to n device status words to h_codes (host).  Word 0: number of
  * Cholesky failures since the context was created; word 1: first failing
- * block id + 1; word 2: bounded waits that gave up; word 3: last
+ * block id + 1; word 2: bounded waits that gave up; word 4: mask groups the sparse forward could
+ * not represent; word 3: last
  * armor_status recorded by a kernel.  The caller must have synchronised the
  * stream the context's work ran on.  (This call itself copies synchronously.) */
 armor_status armor_get_device_status(armor_ctx* ctx, int32_t* h_codes, int32_t n);

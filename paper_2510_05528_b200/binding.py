@@ -22,7 +22,7 @@ S_EXACT, S_BETA = 0, 1
 AB_EXACT, AB_GD, AB_ADAM = 0, 1, 2
 PREC_FP32X3, PREC_TF32, PREC_SIMT = 0, 1, 2
 PHASE_A, PHASE_B, PHASE_S, PHASE_MASK = 1, 2, 4, 8
-DTYPE_F32, DTYPE_BF16 = 0, 1
+DTYPE_F32, DTYPE_BF16, DTYPE_BF16_SPARSE = 0, 1, 2
 
 EXPORTS = ["armor_workspace_bytes", "armor_create", "armor_destroy", "armor_gram", "armor_init",
            "armor_bcd_step", "armor_proxy_loss", "armor_apply", "armor_get_device_status",
@@ -165,11 +165,15 @@ def armor_proxy_loss(ctx, Wbar, H, A, B, S, loss: torch.Tensor) -> None:
                                   _ptr(S, f, "S"), _ptr(loss, torch.float64, "loss"), _stream()), "armor_proxy_loss")
 
 
-def armor_apply(ctx, A, B, S, M, r1, r2, x, y) -> None:
+def armor_apply(ctx, A, B, S, M, r1, r2, x, y, sparse: bool = False) -> None:
     f = torch.float32
     if x.dtype != y.dtype or x.dtype not in (torch.float32, torch.bfloat16):
         raise ValueError("x and y must both be float32 or both be bfloat16")
     dt = DTYPE_BF16 if x.dtype == torch.bfloat16 else DTYPE_F32
+    if sparse:
+        if dt != DTYPE_BF16:
+            raise ValueError("the sparse tensor-core forward takes bf16 x and y")
+        dt = DTYPE_BF16_SPARSE
     _check(lib().armor_apply(ctx, _ptr(A, f, "A"), _ptr(B, f, "B"), _ptr(S, f, "S"), _ptr(M, torch.uint8, "M"),
                              _ptr(r1, f, "r1"), _ptr(r2, f, "r2"), _ptr(x, x.dtype, "x"), _ptr(y, y.dtype, "y"), dt,
                              x.shape[0], _stream()), "armor_apply")
@@ -292,10 +296,10 @@ class ArmorContext:
         armor_proxy_loss(self.ctx, st.Wbar, H, st.A, st.B, st.S, out)
         return out
 
-    def apply(self, st: LayerState, x: torch.Tensor, denormalize: bool = False) -> torch.Tensor:
+    def apply(self, st: LayerState, x: torch.Tensor, denormalize: bool = False, sparse: bool = False) -> torch.Tensor:
         y = torch.empty(x.shape[0], self.d_out, dtype=x.dtype, device=self.device)
         r1, r2 = (st.r1, st.r2) if denormalize else (None, None)
-        armor_apply(self.ctx, st.A, st.B, st.S, st.M, r1, r2, x, y)
+        armor_apply(self.ctx, st.A, st.B, st.S, st.M, r1, r2, x, y, sparse)
         return y
 
     def device_status(self) -> list[int]:

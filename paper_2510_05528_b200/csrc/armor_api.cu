@@ -550,14 +550,17 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
 armor_status armor_apply(armor_ctx* c, const float* A, const float* B, const float* S, const uint8_t* M,
                          const float* r1, const float* r2, const void* d_x, void* d_y, int32_t xy_dtype,
                          int64_t n_tokens, armor_stream_t stream) {
-  (void)M;
   if (!c || !A || !B || !S || n_tokens < 0) return ARMOR_ERR_INVALID_ARG;
   if (n_tokens == 0) return ARMOR_OK;
   if (!d_x || !d_y) return ARMOR_ERR_INVALID_ARG;
-  if (xy_dtype != ARMOR_DTYPE_F32 && xy_dtype != ARMOR_DTYPE_BF16) return ARMOR_ERR_UNSUPPORTED;
+  if (xy_dtype != ARMOR_DTYPE_F32 && xy_dtype != ARMOR_DTYPE_BF16 && xy_dtype != ARMOR_DTYPE_BF16_SPARSE)
+    return ARMOR_ERR_UNSUPPORTED;
+  const bool sparse = (xy_dtype == ARMOR_DTYPE_BF16_SPARSE);
+  if (sparse && !M) return ARMOR_ERR_INVALID_ARG;
+  if (sparse && !tc_sparse_ok(c)) return ARMOR_ERR_UNSUPPORTED;
   if ((r1 == nullptr) != (r2 == nullptr)) return ARMOR_ERR_INVALID_ARG;
   cudaStream_t s = cs(stream);
-  const bool bf16 = (xy_dtype == ARMOR_DTYPE_BF16);
+  const bool bf16 = (xy_dtype != ARMOR_DTYPE_F32);
   const size_t esz = bf16 ? 2 : 4;
   const int64_t d_out = c->d_out, d_in = c->d_in;
   const int64_t chunk = d_out < d_in ? d_out : d_in;   // z1 [chunk, d_in] and z2 [chunk, d_out] fit W-shaped scratch
@@ -580,7 +583,7 @@ armor_status armor_apply(armor_ctx* c, const float* A, const float* B, const flo
       }
     }
     bd_right(c, xc, B, true, c->T, n, d_in, 1.f, nullptr, 0.f, s);                   // z1 = x B^T
-    armor_status st = apply_core(c, c->T, S, c->E, n, bf16, s);                      // z2 = z1 S^T
+    armor_status st = apply_core(c, c->T, S, M, c->E, n, bf16, sparse, s);                      // z2 = z1 S^T
     if (st != ARMOR_OK) return st;
     bd_right(c, c->E, A, true, yc, n, d_out, 1.f, nullptr, 0.f, s);                  // y = z2 A^T
     if (bf16) launch_f32_to_bf16(c, yc, r2, static_cast<char*>(d_y) + (size_t)(t0 * d_out) * esz, n, d_out, s);

@@ -33,7 +33,7 @@ enum {
 };
 
 // status words in the device status buffer
-enum { ST_CHOL_FAILS = 0, ST_FIRST_FAIL = 1, ST_WAIT_TIMEOUTS = 2, ST_LAST_ERR = 3, ST_COUNT = 8 };
+enum { ST_CHOL_FAILS = 0, ST_FIRST_FAIL = 1, ST_WAIT_TIMEOUTS = 2, ST_LAST_ERR = 3, ST_SPARSE_BAD_GROUPS = 4, ST_COUNT = 8 };
 
 // One selected group per (i, j) block of the sparse core (Algorithm 3).
 struct SelRec {
@@ -160,7 +160,8 @@ armor_status prepare_H(armor_ctx* c, const float* H, cudaStream_t s);
 armor_status gram_accumulate(armor_ctx* c, const void* X, int x_dtype, int64_t n_rows, int64_t ldx, float* H,
                              cudaStream_t s);
 // z2 [n, d_out] = z1 [n, d_in] * S^T
-armor_status apply_core(armor_ctx* c, const float* z1, const float* S, float* z2, int64_t n, bool bf16, cudaStream_t s);
+armor_status apply_core(armor_ctx* c, const float* z1, const float* S, const uint8_t* M, float* z2, int64_t n, bool bf16,
+                        bool sparse, cudaStream_t s);
 
 // deterministic reductions (two stages, fixed order)
 void dot_to_ptr(armor_ctx* c, const float* x, const float* y, int64_t n, double* out, cudaStream_t s);
@@ -236,3 +237,9 @@ struct TcGemm {
 };
 armor_status launch_tc_gemm(armor_ctx* c, const TcGemm& g, int* n_tiles, cudaStream_t s);
 bool tc_gemm_shape_ok(int64_t M, int64_t N, int64_t K);
+// the 2:4 core on the sparse tensor cores (sparse_tcgen05.cu)
+bool tc_sparse_ok(const armor_ctx* c);
+size_t tc_sparse_values_bytes(const armor_ctx* c);
+void launch_compress_24(armor_ctx* c, const float* S, const uint8_t* M, void* Sc, void* E, cudaStream_t s);
+armor_status launch_tc_sparse(armor_ctx* c, const void* Sc, const void* E, const void* z1_bf16, float* z2, int64_t n,
+                              cudaStream_t s);

@@ -101,8 +101,17 @@ armor_status gram_accumulate(armor_ctx* c, const void* Xv, int x_dtype, int64_t 
   return ARMOR_OK;
 }
 
-armor_status apply_core(armor_ctx* c, const float* z1, const float* S, float* z2, int64_t n, bool bf16, cudaStream_t s) {
+armor_status apply_core(armor_ctx* c, const float* z1, const float* S, const uint8_t* M, float* z2, int64_t n, bool bf16,
+                        bool sparse, cudaStream_t s) {
   const int64_t d_in = c->d_in, d_out = c->d_out;
+  if (sparse) {
+    // bf16 deployment with the 2:4 core on the sparse tensor cores: kept values and positions from S and M
+    if (!bf16 || !M || !tc_sparse_ok(c)) return ARMOR_ERR_UNSUPPORTED;
+    char* buf = reinterpret_cast<char*>(c->P);                 // values: wn bytes, positions: wn / 8 bytes
+    launch_f32_to_bf16(c, z1, nullptr, c->U, n, d_in, s);
+    launch_compress_24(c, S, M, buf, buf + tc_sparse_values_bytes(c), s);
+    return launch_tc_sparse(c, buf, buf + tc_sparse_values_bytes(c), c->U, z2, n, s);
+  }
   if (bf16 && c->cfg.precision != ARMOR_PREC_SIMT && d_out % 32 == 0 && d_in % 8 == 0) {
     // bf16 deployment: the core and the wrapped activations are rounded to bf16 and multiplied on the bf16
     // tensor-core path with fp32 accumulation

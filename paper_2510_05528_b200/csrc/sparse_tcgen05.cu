@@ -1,0 +1,350 @@
+// The core product of the deployment form (Section 3.1: y = A (S (B x)), S the 2:4 sparse core) on the sparse
+// tensor cores of sm_100a:  Z2[t][m] = sum_k S[m][k] * Z1[t][k]  with S given as its kept values (two of every
+// four along k, bf16) plus the 2-bit positions of the kept values, Z1 bf16, fp32 accumulation and output.
+//
+// S is the A operand of tcgen05.mma.sp (kind::f16): each instruction multiplies a 128 x 32 slice of S, held in
+// shared memory as 128 x 16 kept values, by a 32 x 128 slice of Z1^T; the positions come from tensor memory.
+//
+// Layout of the positions (what the instruction reads, M = 128, 16-bit operands): one 32-bit tensor-memory column
+// per instruction; lane l = m0 + 8 k1 + 16 m2 (m0 < 8, k1 < 2, m2 < 8) holds, in its low half, the 16 bits of row
+// m0 + 16 m2 for the k-half k1 (16 consecutive k: four groups, four bits each, the lower kept position in bits
+// 0-1 and the higher one in bits 2-3 of the group's nibble) and, in its high half, the same for row m0 + 16 m2 + 8.
+// Consecutive instructions along k use consecutive columns; the instruction is given the even column of the pair
+// and the column's parity as the selector field of its descriptor.  compress_24_kernel writes the positions in
+// exactly this order, 128 lanes x 4 columns (16 bytes per lane) per 128 x 128 block of S, so that the kernel
+// moves them from global memory to tensor memory with one 16-byte load and one tcgen05.st per lane and stage.
+//
+// Kernel: persistent, one CTA per SM, 320 threads: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 epilogue
+// (transposing store: lanes are rows m of S, columns are tokens), warps 6-9 bring the positions into tensor
+// memory.  128 x 128 output tiles, 128 k per stage (16 KiB of kept values + 32 KiB of Z1), four stages, two
+// accumulator buffers.  Every wait is bounded.
+#include <cuda_bf16.h>
+
+#include "tc_common.cuh"
+
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128, BN = 128, BKL = 128;        // BKL: logical k per stage (64 kept values = 128 bytes per row)
+constexpr int NTHREADS = 320;
+constexpr int STAGES = 4;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr uint32_t META_COL0 = 256;                 // accumulators: columns 0-127 and 128-255
+constexpr int A_BYTES = BM * 64 * 2;                // 16 KiB
+constexpr int BH_BYTES = BN * 64 * 2;               // 16 KiB: one half (64 k) of the Z1 stage
+constexpr int STAGE_BYTES = A_BYTES + 2 * BH_BYTES; // 48 KiB
+
+struct SParams {
+  float* Z; int64_t ldz;        // [N tokens][ldz], written transposed
+  int64_t M, N, K;              // rows of S, tokens, logical k
+  int m_tiles, n_tiles, k_tiles;
+  const uint4* E;               // positions: [m_tiles][k_tiles][128 lanes] x 16 bytes
+  int32_t* status;
+};
+
+__device__ __forceinline__ uint64_t smem_desc_k(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;                           // 128-byte swizzle
+  return d;
+}
+
+// bf16 operands, fp32 accumulation, both K-major, sparse A; sel = parity of the position column
+__device__ __forceinline__ uint32_t instr_desc_sp(uint32_t sel) {
+  uint32_t d = sel & 3u;          // position selector
+  d |= 1u << 2;                   // A is 2:4 sparse
+  d |= 1u << 4;                   // D format: F32
+  d |= 1u << 7;                   // A format: BF16
+  d |= 1u << 10;                  // B format: BF16
+  d |= (uint32_t)(BN >> 3) << 17;
+  d |= (uint32_t)(BM >> 4) << 24;
+  return d;
+}
+
+__device__ __forceinline__ void umma_bf16_sp(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t tmem_e,
+                                             uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(tmem_e), "r"(idesc), "r"(acc)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_st4(uint32_t taddr, const uint4& v) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
+               ::"r"(taddr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+               : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+tc_sparse_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const SParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ __align__(8) uint64_t bars[3 * STAGES + 4];
+  __shared__ uint32_t tmem_base_holder;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]), mfull0 = smem_u32(&bars[2 * STAGES]);
+  const uint32_t tfull0 = smem_u32(&bars[3 * STAGES]), tempty0 = smem_u32(&bars[3 * STAGES + 2]);
+  const int n_tiles_total = p.m_tiles * p.n_tiles;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full0 + 8 * s, 1);
+      mbar_init(empty0 + 8 * s, 1);
+      mbar_init(mfull0 + 8 * s, 4);
+    }
+    for (int s = 0; s < 2; ++s) { mbar_init(tfull0 + 8 * s, 1); mbar_init(tempty0 + 8 * s, 4); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_holder;
+  volatile int* abortp = &abort_flag;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0; long long issued = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles_total && ok; tile += gridDim.x) {
+        const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+        for (int kt = 0; kt < p.k_tiles; ++kt) {
+          if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abortp, p.status)) { ok = false; break; }
+          const uint32_t fb = full0 + 8 * stage;
+          mbar_expect_tx(fb, STAGE_BYTES);
+          const uint32_t dst = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+          tma_load_2d(dst, &mapA, kt * 64, mt * BM, fb);                      // 64 kept values = 128 logical k
+          tma_load_2d(dst + A_BYTES, &mapB, kt * BKL, nt * BN, fb);
+          tma_load_2d(dst + A_BYTES + BH_BYTES, &mapB, kt * BKL + 64, nt * BN, fb);
+          ++issued;
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) {
+        for (int back = 1; back <= STAGES && back <= issued; ++back) {
+          int s = stage - back; uint32_t ph = phase;
+          if (s < 0) { s += STAGES; ph ^= 1; }
+          const long long t0 = clock64();
+          while (!mbar_try(full0 + 8 * s, ph) && clock64() - t0 < 20000000ll) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles_total && ok; tile += gridDim.x, ++local) {
+        const int as = local & 1;
+        const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
+        if (!mbar_wait(tempty0 + 8 * as, aphase ^ 1, abortp, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tacc = tmem_base + (uint32_t)(as * BN);
+        for (int kt = 0; kt < p.k_tiles; ++kt) {
+          if (!mbar_wait(full0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
+          if (!mbar_wait(mfull0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+          const uint32_t sb = sa + A_BYTES;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {                                        // 32 logical k per instruction
+            const uint64_t da = smem_desc_k(sa + j * 32);                      // 16 kept values = 32 bytes
+            const uint64_t dbm = smem_desc_k(sb + (j >> 1) * BH_BYTES + (j & 1) * 64);
+            const uint32_t ecol = tmem_base + META_COL0 + (uint32_t)(4 * stage + j);
+            umma_bf16_sp(tacc, da, dbm, ecol & ~1u, instr_desc_sp(ecol & 1u), (uint32_t)((kt > 0) | (j != 0)));
+          }
+          umma_commit(empty0 + 8 * stage);
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (ok) umma_commit(tfull0 + 8 * as);
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------------------ epilogue warps
+    const int q = warp & 3;
+    int local = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < n_tiles_total && ok; tile += gridDim.x, ++local) {
+      const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+      const int as = local & 1;
+      const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
+      if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
+      tc_fence_after();
+      const int64_t row = (int64_t)mt * BM + q * 32 + lane;                    // row of S = column of Z
+#pragma unroll 1
+      for (int ch = 0; ch < BN / 32; ++ch) {
+        uint32_t r[32];
+        tmem_ld32(tmem_base + (uint32_t)(as * BN + ch * 32) + ((uint32_t)(q * 32) << 16), r);
+        const int64_t tok0 = (int64_t)nt * BN + ch * 32;
+        if (row < p.M) {
+#pragma unroll
+          for (int cidx = 0; cidx < 32; ++cidx)
+            if (tok0 + cidx < p.N) p.Z[(tok0 + cidx) * p.ldz + row] = __uint_as_float(r[cidx]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty0 + 8 * as);
+    }
+  } else {
+    // ------------------------------------------------------------ positions: global -> tensor memory
+    const int q = warp & 3;
+    int stage = 0; uint32_t phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < n_tiles_total && ok; tile += gridDim.x) {
+      const int mt = tile % p.m_tiles;
+      const uint4* src = p.E + ((int64_t)mt * p.k_tiles) * 128 + q * 32 + lane;
+      for (int kt = 0; kt < p.k_tiles; ++kt) {
+        const uint4 v = __ldg(src + (int64_t)kt * 128);
+        if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abortp, p.status)) { ok = false; break; }
+        tc_fence_after();
+        tmem_st4(tmem_base + ((uint32_t)(q * 32) << 16) + META_COL0 + (uint32_t)(4 * stage), v);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(mfull0 + 8 * stage);
+        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// One thread per 32-bit word of positions: 2 rows x 16 k.  Writes the word and the eight pairs of kept values.
+// A group whose mask byte keeps fewer than two positions is padded with unkept positions (their values are
+// written as zeros); more than two kept positions cannot be represented: the first two are taken and the
+// status word counts the group.
+__global__ void __launch_bounds__(256)
+compress_24_kernel(const float* __restrict__ S, const uint8_t* __restrict__ Mk, __nv_bfloat16* __restrict__ Sc,
+                   uint32_t* __restrict__ E, int64_t d_out, int64_t d_in, int32_t* status) {
+  const int64_t k_tiles = d_in / 128;
+  const int64_t n_words = d_out * (d_in / 32);          // (d_out / 128) * k_tiles * 128 * 4
+  const int64_t w = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (w >= n_words) return;
+  const int k2 = (int)(w & 3), l = (int)((w >> 2) & 127);
+  const int64_t blk = w >> 9;
+  const int64_t kt = blk % k_tiles, mt = blk / k_tiles;
+  const int m0 = l & 7, k1 = (l >> 3) & 1, m2 = l >> 4;
+  const int64_t kbase = kt * 128 + k2 * 32 + k1 * 16;
+  uint32_t word = 0;
+  int bad = 0;
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int64_t row = mt * 128 + m0 + 16 * m2 + 8 * h;
+#pragma unroll
+    for (int qd = 0; qd < 4; ++qd) {
+      const int64_t g = kbase / 4 + qd;
+      const unsigned m = Mk[row * (d_in / 4) + g] & 15u;
+      const float4 v = *reinterpret_cast<const float4*>(S + row * d_in + 4 * g);
+      const float vals[4] = {v.x, v.y, v.z, v.w};
+      int i0 = -1, i1 = -1, cnt = 0;
+#pragma unroll
+      for (int pidx = 0; pidx < 4; ++pidx)
+        if ((m >> pidx) & 1u) { if (cnt == 0) i0 = pidx; else if (cnt == 1) i1 = pidx; ++cnt; }
+      if (cnt > 2) bad = 1;
+      if (cnt < 2) {                                   // pad with unkept positions, keeping i0 < i1
+        if (cnt == 0) { i0 = 0; i1 = 1; }
+        else if (i0 < 3) i1 = i0 + 1;
+        else { i1 = 3; i0 = 2; }
+      }
+      const float a = ((m >> i0) & 1u) ? vals[i0] : 0.f, b = ((m >> i1) & 1u) ? vals[i1] : 0.f;
+      __nv_bfloat162 pr;
+      pr.x = __float2bfloat16(a);
+      pr.y = __float2bfloat16(b);
+      *reinterpret_cast<__nv_bfloat162*>(Sc + row * (d_in / 2) + 2 * g) = pr;
+      word |= (uint32_t)(i0 | (i1 << 2)) << (16 * h + 4 * qd);
+    }
+  }
+  E[w] = word;
+  if (bad) atomicAdd(&status[ST_SPARSE_BAD_GROUPS], 1);
+}
+
+bool make_map_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t K, int64_t ld) {
+  PFN_cuTensorMapEncodeTiled_v12000 enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {64, 128};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool tc_sparse_ok(const armor_ctx* c) {
+  return c->cfg.n_keep == 2 && c->cfg.m_group == 4 && c->d_out % 128 == 0 && c->d_in % 128 == 0 &&
+         c->cfg.precision != ARMOR_PREC_SIMT;
+}
+
+size_t tc_sparse_values_bytes(const armor_ctx* c) { return (size_t)c->d_out * (size_t)c->d_in; }   // bf16, half the entries
+
+void launch_compress_24(armor_ctx* c, const float* S, const uint8_t* M, void* Sc, void* E, cudaStream_t s) {
+  const int64_t n_words = c->d_out * (c->d_in / 32);
+  compress_24_kernel<<<(unsigned)((n_words + 255) / 256), 256, 0, s>>>(S, M, static_cast<__nv_bfloat16*>(Sc),
+                                                                        static_cast<uint32_t*>(E), c->d_out, c->d_in,
+                                                                        c->status);
+  c->launches++;
+}
+
+// Z2[n][d_out] = Z1[n][d_in] * S^T with S given compressed (Sc, E); Z1 bf16.
+armor_status launch_tc_sparse(armor_ctx* c, const void* Sc, const void* E, const void* z1_bf16, float* z2, int64_t n,
+                              cudaStream_t s) {
+  if (!tc_sparse_ok(c) || n <= 0) return ARMOR_ERR_UNSUPPORTED;
+  CUtensorMap mA, mB;
+  if (!make_map_bf16(&mA, Sc, c->d_out, c->d_in / 2, c->d_in / 2)) return ARMOR_ERR_CUDA;
+  if (!make_map_bf16(&mB, z1_bf16, n, c->d_in, c->d_in)) return ARMOR_ERR_CUDA;
+  SParams p{};
+  p.Z = z2; p.ldz = c->d_out; p.M = c->d_out; p.N = n; p.K = c->d_in;
+  p.m_tiles = (int)(c->d_out / BM); p.n_tiles = (int)((n + BN - 1) / BN); p.k_tiles = (int)(c->d_in / BKL);
+  p.E = static_cast<const uint4*>(E);
+  p.status = c->status;
+  constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024;
+  static bool attr = false;
+  if (!attr) {
+    if (cudaFuncSetAttribute(tc_sparse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess)
+      return ARMOR_ERR_CUDA;
+    attr = true;
+  }
+  static int n_sm = 0;
+  if (!n_sm) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ARMOR_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ARMOR_ERR_CUDA;
+  }
+  const int tiles = p.m_tiles * p.n_tiles;
+  const int grid = tiles < n_sm ? tiles : n_sm;
+  const bool timed = c->timing_on && c->timing_n < ARMOR_MAX_TIMED;
+  if (timed) cudaEventRecord(c->ev_beg[c->timing_n], s);
+  tc_sparse_kernel<<<grid, NTHREADS, SMEM, s>>>(mA, mB, p);
+  if (timed) {
+    cudaEventRecord(c->ev_end[c->timing_n], s);
+    c->timing_n++;
+    c->timing_flops += 2.0 * (double)p.M * (double)p.N * (double)p.K;   // dense-equivalent
+  }
+  c->launches++;
+  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+}

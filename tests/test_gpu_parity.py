@@ -557,6 +557,61 @@ def test_apply_with_bf16_activations(mid_data):
         assert rel(y.float().cpu().numpy(), yo) < 5e-3
 
 
+def test_sparse_tensor_core_forward_is_exact_on_integers(mid_data):
+    """The 2:4 core on the sparse tensor cores: with identity wrappers, small-integer core values at random kept
+    positions (all six position pairs occur) and activations in {-1, 0, 1}, every product and sum is exact in
+    bf16 x bf16 -> fp32, so y must equal the integer result rounded once to bf16 -- any slip in the packing of
+    the kept values or of their positions shows as a wrong integer."""
+    W, X, H32 = mid_data
+    cfg = MID
+    ctx = make(cfg, Bd.PREC_FP32X3)
+    st = ctx.init(dev(W), dev(H32))
+    rng = np.random.default_rng(11)
+    ng = cfg.d_in // 4
+    pairs = np.array([[0, 1], [0, 2], [0, 3], [1, 2], [1, 3], [2, 3]])
+    pick = pairs[rng.integers(0, 6, size=(cfg.d_out, ng))]
+    M = np.zeros((cfg.d_out, ng, 4), dtype=bool)
+    np.put_along_axis(M, pick, True, axis=2)
+    M = M.reshape(cfg.d_out, cfg.d_in)
+    S = rng.integers(-3, 4, size=(cfg.d_out, cfg.d_in)).astype(np.float64) * M
+    nb_o, nb_i, db = cfg.d_out // cfg.d_block, cfg.d_in // cfg.d_block, cfg.d_block
+    load_state(st, np.tile(np.eye(db), (nb_o, 1, 1)), np.tile(np.eye(db), (nb_i, 1, 1)), S, M)
+    for n_tok in (300, 128, 1):
+        x = (rng.integers(-1, 2, size=(n_tok, cfg.d_in)) * (rng.random((n_tok, cfg.d_in)) < 0.15)).astype(np.float32)
+        xb = dev(x).to(torch.bfloat16)
+        y = ctx.apply(st, xb, sparse=True)
+        exact = torch.from_numpy(x.astype(np.float64) @ S.T).to(torch.bfloat16)
+        assert y.dtype == torch.bfloat16 and torch.equal(y.cpu(), exact), n_tok
+        assert torch.equal(ctx.apply(st, xb).cpu(), exact)            # the dense bf16 path on the same input
+    assert ctx.device_status()[:5] == [0, 0, 0, 0, 0]
+
+
+def test_sparse_tensor_core_forward_against_the_oracle(mid_data):
+    W, X, H32 = mid_data
+    ctx = make(MID, Bd.PREC_FP32X3, normalize=1)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    ctx.bcd_step(st, Hd, 0, 2, want_stats=False)
+    xb = dev(inputs.make_tokens(MID, 300)).to(torch.bfloat16)
+    A, B, S = (host(t).astype(np.float64) for t in (st.A, st.B, st.S))
+    xr = xb.float().cpu().numpy()
+    for den in (False, True):
+        y = ctx.apply(st, xb, denormalize=den, sparse=True)
+        r1, r2 = (host(st.r1).astype(np.float64), host(st.r2).astype(np.float64)) if den else (None, None)
+        yo = O.apply(A, B, S, xr, r1, r2)
+        assert rel(y.float().cpu().numpy(), yo) < 5e-3                # same roundings as the dense bf16 forward
+        # against the dense bf16 forward: the same rounded operands, only the order of the fp32 sums differs
+        yd = ctx.apply(st, xb, denormalize=den)
+        assert rel(y.float().cpu().numpy(), yd.float().cpu().numpy()) < 1e-3
+    with pytest.raises(ValueError):
+        ctx.apply(st, xb.float(), sparse=True)
+    ctx48 = make(MID, Bd.PREC_FP32X3, n_keep=4, m_group=8)
+    st48 = ctx48.init(dev(W), Hd)
+    with pytest.raises(RuntimeError):
+        ctx48.apply(st48, xb, sparse=True)                            # sparse tensor cores take 2:4 only
+    assert ctx.device_status()[:5] == [0, 0, 0, 0, 0]
+
+
 # ------------------------------------------------------------------------------------------ block products
 @pytest.mark.parametrize("db", [128, 256])
 @pytest.mark.parametrize("side,transpose", [(0, False), (0, True), (1, False), (1, True)])
