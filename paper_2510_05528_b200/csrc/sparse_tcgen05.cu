@@ -231,6 +231,223 @@ tc_sparse_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
   }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// The same product on pairs of CTAs (cta_group::2): a cluster of two CTAs works on a 256 x 256 output tile.
+// Each CTA holds 128 rows of S (kept values in shared memory, positions in its own tensor memory) and half of
+// the tile's tokens (128 rows of Z1); one instruction issued by the even CTA multiplies 256 x 32 of S by
+// 32 x 256 of Z1^T, every SM reading only half of Z1's tile from its shared memory.  Per SM and 128 k this
+// loads 16 KiB + 32 KiB for 128 x 256 outputs, half of what the one-CTA kernel above loads.
+//   full[s]   (even CTA): armed by the even CTA's producer for the bytes of both CTAs; both CTAs' TMA loads
+//             complete on it (cta_group::2 loads may signal the pair's other CTA)
+//   mfull[s]  (even CTA): 8 arrivals, one per position-loading warp of either CTA
+//   empty[s], tfull (both CTAs): tcgen05.commit multicast to the pair
+//   tempty    (even CTA): 8 arrivals, one per epilogue warp of either CTA
+// One accumulator buffer of 256 columns (the positions need tensor-memory columns too).
+constexpr int BN2 = 256;
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t cluster_bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(cluster_bar)
+      : "memory");
+}
+__device__ __forceinline__ void umma_bf16_sp_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t tmem_e,
+                                                  uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.sp.cta_group::2.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(tmem_e), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// arrives on the barrier at this shared-memory offset in both CTAs of the pair once the MMAs issued so far are done
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"((uint16_t)3)
+      : "memory");
+}
+__device__ __forceinline__ uint32_t instr_desc_sp_pair(uint32_t sel) {
+  uint32_t d = sel & 3u;
+  d |= 1u << 2;
+  d |= 1u << 4;
+  d |= 1u << 7;
+  d |= 1u << 10;
+  d |= (uint32_t)(BN2 >> 3) << 17;
+  d |= (uint32_t)(256 >> 4) << 24;
+  return d;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+tc_sparse_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const SParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ __align__(8) uint64_t bars[3 * STAGES + 2];
+  __shared__ uint32_t tmem_base_holder;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]), mfull0 = smem_u32(&bars[2 * STAGES]);
+  const uint32_t tfull = smem_u32(&bars[3 * STAGES]), tempty = smem_u32(&bars[3 * STAGES + 1]);
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int m_pairs = p.m_tiles >> 1;                       // 256-row tiles
+  const int n_tiles_total = m_pairs * p.n_tiles;            // p.n_tiles counts 256-token tiles here
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full0 + 8 * s, 1);
+      mbar_init(empty0 + 8 * s, 1);
+      mbar_init(mfull0 + 8 * s, 8);
+    }
+    mbar_init(tfull, 1);
+    mbar_init(tempty, 8);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                       // both CTAs' barriers exist before anyone signals them
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_holder;
+  volatile int* abortp = &abort_flag;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0; long long issued = 0;
+      bool ok = true;
+      for (int tile = pair; tile < n_tiles_total && ok; tile += n_pairs) {
+        const int mt = tile % m_pairs, nt = tile / m_pairs;
+        const int row0 = mt * 256 + (int)rank * 128, tok0 = nt * BN2 + (int)rank * 128;
+        for (int kt = 0; kt < p.k_tiles; ++kt) {
+          if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abortp, p.status)) { ok = false; break; }
+          if (rank == 0) mbar_expect_tx(full0 + 8 * stage, 2 * STAGE_BYTES);
+          const uint32_t fb = map_to_cta(full0 + 8 * stage, 0);
+          const uint32_t dst = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+          tma_load_2d_pair(dst, &mapA, kt * 64, row0, fb);
+          tma_load_2d_pair(dst + A_BYTES, &mapB, kt * BKL, tok0, fb);
+          tma_load_2d_pair(dst + A_BYTES + BH_BYTES, &mapB, kt * BKL + 64, tok0, fb);
+          ++issued;
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+      // tail: the MMAs that read the stages issued last have finished (their commits reach both CTAs), so
+      // nothing is in flight towards this CTA's shared memory when it leaves
+      for (int back = 1; back <= STAGES && back <= issued; ++back) {
+        int s = stage - back; uint32_t ph = phase;
+        if (s < 0) { s += STAGES; ph ^= 1; }
+        const long long t0 = clock64();
+        while (!mbar_try(empty0 + 8 * s, ph) && clock64() - t0 < (ok ? WAIT_CYCLES : 20000000ll)) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (even CTA only)
+    if (lane == 0 && rank == 0) {
+      int stage = 0; uint32_t phase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int tile = pair; tile < n_tiles_total && ok; tile += n_pairs, ++local) {
+        if (!mbar_wait(tempty, ((uint32_t)local & 1u) ^ 1u, abortp, p.status)) { ok = false; break; }
+        tc_fence_after();
+        for (int kt = 0; kt < p.k_tiles; ++kt) {
+          if (!mbar_wait(full0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
+          if (!mbar_wait(mfull0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+          const uint32_t sb = sa + A_BYTES;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint64_t da = smem_desc_k(sa + j * 32);
+            const uint64_t dbm = smem_desc_k(sb + (j >> 1) * BH_BYTES + (j & 1) * 64);
+            const uint32_t ecol = tmem_base + META_COL0 + (uint32_t)(4 * stage + j);
+            umma_bf16_sp_pair(tmem_base, da, dbm, ecol & ~1u, instr_desc_sp_pair(ecol & 1u), (uint32_t)((kt > 0) | (j != 0)));
+          }
+          umma_commit_pair(empty0 + 8 * stage);
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (ok) umma_commit_pair(tfull);
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------------------ epilogue warps (both CTAs)
+    const int q = warp & 3;
+    const uint32_t tempty_lead = map_to_cta(tempty, 0);
+    int local = 0;
+    bool ok = true;
+    for (int tile = pair; tile < n_tiles_total && ok; tile += n_pairs, ++local) {
+      const int mt = tile % m_pairs, nt = tile / m_pairs;
+      if (!mbar_wait(tfull, (uint32_t)local & 1u, abortp, p.status)) { ok = false; break; }
+      tc_fence_after();
+      const int64_t row = (int64_t)mt * 256 + rank * 128 + q * 32 + lane;
+#pragma unroll 1
+      for (int ch = 0; ch < BN2 / 32; ++ch) {
+        uint32_t r[32];
+        tmem_ld32(tmem_base + (uint32_t)(ch * 32) + ((uint32_t)(q * 32) << 16), r);
+        const int64_t tok0 = (int64_t)nt * BN2 + ch * 32;
+        if (row < p.M) {
+#pragma unroll
+          for (int cidx = 0; cidx < 32; ++cidx)
+            if (tok0 + cidx < p.N) p.Z[(tok0 + cidx) * p.ldz + row] = __uint_as_float(r[cidx]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(tempty_lead);
+    }
+  } else {
+    // ------------------------------------------------------------ positions: global -> tensor memory (both CTAs)
+    const int q = warp & 3;
+    int stage = 0; uint32_t phase = 0;
+    bool ok = true;
+    for (int tile = pair; tile < n_tiles_total && ok; tile += n_pairs) {
+      const int mt = tile % m_pairs;
+      const uint4* src = p.E + ((int64_t)(2 * mt + (int)rank) * p.k_tiles) * 128 + q * 32 + lane;
+      for (int kt = 0; kt < p.k_tiles; ++kt) {
+        const uint4 v = __ldg(src + (int64_t)kt * 128);
+        if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abortp, p.status)) { ok = false; break; }
+        tc_fence_after();
+        tmem_st4(tmem_base + ((uint32_t)(q * 32) << 16) + META_COL0 + (uint32_t)(4 * stage), v);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(map_to_cta(mfull0 + 8 * stage, 0));
+        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                       // neither CTA leaves while its partner may still signal it
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
 // One thread per 32-bit word of positions: 2 rows x 16 k.  Writes the word and the eight pairs of kept values.
 // A group whose mask byte keeps fewer than two positions is padded with unkept positions (their values are
 // written as zeros); more than two kept positions cannot be represented: the first two are taken and the
@@ -295,6 +512,8 @@ bool make_map_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t K, 
 
 }  // namespace
 
+int g_sparse_pairs = 1;   // 0: the one-CTA kernel only (tests compare the two)
+
 bool tc_sparse_ok(const armor_ctx* c) {
   return c->cfg.n_keep == 2 && c->cfg.m_group == 4 && c->d_out % 128 == 0 && c->d_in % 128 == 0 &&
          c->cfg.precision != ARMOR_PREC_SIMT;
@@ -335,11 +554,31 @@ armor_status launch_tc_sparse(armor_ctx* c, const void* Sc, const void* E, const
     if (cudaGetDevice(&dev) != cudaSuccess) return ARMOR_ERR_CUDA;
     if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ARMOR_ERR_CUDA;
   }
-  const int tiles = p.m_tiles * p.n_tiles;
-  const int grid = tiles < n_sm ? tiles : n_sm;
   const bool timed = c->timing_on && c->timing_n < ARMOR_MAX_TIMED;
   if (timed) cudaEventRecord(c->ev_beg[c->timing_n], s);
-  tc_sparse_kernel<<<grid, NTHREADS, SMEM, s>>>(mA, mB, p);
+  if (g_sparse_pairs && c->d_out % 256 == 0 && n_sm >= 2) {
+    static bool attr2 = false;
+    if (!attr2) {
+      if (cudaFuncSetAttribute(tc_sparse_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess)
+        return ARMOR_ERR_CUDA;
+      attr2 = true;
+    }
+    p.n_tiles = (int)((n + BN2 - 1) / BN2);
+    const int tiles = (p.m_tiles / 2) * p.n_tiles;
+    int pairs = n_sm / 2;
+    if (tiles < pairs) pairs = tiles;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(NTHREADS); cfg.dynamicSmemBytes = SMEM; cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, tc_sparse_pair_kernel, mA, mB, p) != cudaSuccess) return ARMOR_ERR_CUDA;
+  } else {
+    const int tiles = p.m_tiles * p.n_tiles;
+    const int grid = tiles < n_sm ? tiles : n_sm;
+    tc_sparse_kernel<<<grid, NTHREADS, SMEM, s>>>(mA, mB, p);
+  }
   if (timed) {
     cudaEventRecord(c->ev_end[c->timing_n], s);
     c->timing_n++;

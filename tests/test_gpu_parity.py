@@ -557,27 +557,28 @@ def test_apply_with_bf16_activations(mid_data):
         assert rel(y.float().cpu().numpy(), yo) < 5e-3
 
 
-def test_sparse_tensor_core_forward_is_exact_on_integers(mid_data):
+@pytest.mark.parametrize("d_out,d_in", [(384, 512), (512, 768), (1024, 256)],
+                         ids=["one-cta-kernel", "cta-pair-kernel", "cta-pair-kernel-4-row-tiles"])
+def test_sparse_tensor_core_forward_is_exact_on_integers(d_out, d_in):
     """The 2:4 core on the sparse tensor cores: with identity wrappers, small-integer core values at random kept
     positions (all six position pairs occur) and activations in {-1, 0, 1}, every product and sum is exact in
     bf16 x bf16 -> fp32, so y must equal the integer result rounded once to bf16 -- any slip in the packing of
-    the kept values or of their positions shows as a wrong integer."""
-    W, X, H32 = mid_data
-    cfg = MID
-    ctx = make(cfg, Bd.PREC_FP32X3)
-    st = ctx.init(dev(W), dev(H32))
-    rng = np.random.default_rng(11)
-    ng = cfg.d_in // 4
+    the kept values or of their positions shows as a wrong integer.  A row count that is a multiple of 256 runs
+    on pairs of CTAs (256 x 256 tiles), any other multiple of 128 on the one-CTA kernel."""
+    db = 128
+    rng = np.random.default_rng(11 + d_out)
+    ctx = Bd.ArmorContext(d_out, d_in, db, device=DEV, precision=Bd.PREC_FP32X3)
+    st = ctx.init(dev(rng.standard_normal((d_out, d_in))), torch.eye(d_in, device=DEV))
+    ng = d_in // 4
     pairs = np.array([[0, 1], [0, 2], [0, 3], [1, 2], [1, 3], [2, 3]])
-    pick = pairs[rng.integers(0, 6, size=(cfg.d_out, ng))]
-    M = np.zeros((cfg.d_out, ng, 4), dtype=bool)
+    pick = pairs[rng.integers(0, 6, size=(d_out, ng))]
+    M = np.zeros((d_out, ng, 4), dtype=bool)
     np.put_along_axis(M, pick, True, axis=2)
-    M = M.reshape(cfg.d_out, cfg.d_in)
-    S = rng.integers(-3, 4, size=(cfg.d_out, cfg.d_in)).astype(np.float64) * M
-    nb_o, nb_i, db = cfg.d_out // cfg.d_block, cfg.d_in // cfg.d_block, cfg.d_block
-    load_state(st, np.tile(np.eye(db), (nb_o, 1, 1)), np.tile(np.eye(db), (nb_i, 1, 1)), S, M)
-    for n_tok in (300, 128, 1):
-        x = (rng.integers(-1, 2, size=(n_tok, cfg.d_in)) * (rng.random((n_tok, cfg.d_in)) < 0.15)).astype(np.float32)
+    M = M.reshape(d_out, d_in)
+    S = rng.integers(-3, 4, size=(d_out, d_in)).astype(np.float64) * M
+    load_state(st, np.tile(np.eye(db), (d_out // db, 1, 1)), np.tile(np.eye(db), (d_in // db, 1, 1)), S, M)
+    for n_tok in (300, 256, 1, 700):
+        x = (rng.integers(-1, 2, size=(n_tok, d_in)) * (rng.random((n_tok, d_in)) < 0.15)).astype(np.float32)
         xb = dev(x).to(torch.bfloat16)
         y = ctx.apply(st, xb, sparse=True)
         exact = torch.from_numpy(x.astype(np.float64) @ S.T).to(torch.bfloat16)
