@@ -11,13 +11,16 @@
 // 0-1 and the higher one in bits 2-3 of the group's nibble) and, in its high half, the same for row m0 + 16 m2 + 8.
 // Consecutive instructions along k use consecutive columns; the instruction is given the even column of the pair
 // and the column's parity as the selector field of its descriptor.  compress_24_kernel writes the positions in
-// exactly this order, 128 lanes x 4 columns (16 bytes per lane) per 128 x 128 block of S, so that the kernel
-// moves them from global memory to tensor memory with one 16-byte load and one tcgen05.st per lane and stage.
+// exactly this order, 128 lanes x 4 columns (16 bytes per lane) per 128 x 128 block of S: 2 KiB that travel with
+// the stage's operands by TMA and go from shared to tensor memory with one tcgen05.cp (128 lanes x 128 bits)
+// issued by the MMA thread in front of the stage's four instructions -- the copy runs in the tensor-core pipe,
+// in order with the MMAs.  (Writing the positions with tcgen05.st from other warps was measured first: every
+// store waited about 1600 cycles behind the running MMAs and the kernel ran at a quarter of its rate.)
 //
-// Kernel: persistent, one CTA per SM, 320 threads: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 epilogue
-// (transposing store: lanes are rows m of S, columns are tokens), warps 6-9 bring the positions into tensor
-// memory.  128 x 128 output tiles, 128 k per stage (16 KiB of kept values + 32 KiB of Z1), four stages, two
-// accumulator buffers.  Every wait is bounded.
+// Kernel: persistent, one CTA per SM, 192 threads: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 epilogue
+// (transposing store: lanes are rows m of S, columns are tokens).  128 x 128 output tiles, 128 k per stage
+// (16 KiB of kept values + 32 KiB of Z1 + 2 KiB of positions), four stages, two accumulator buffers.  Every wait
+// is bounded.
 #include <cuda_bf16.h>
 
 #include "tc_common.cuh"
@@ -27,19 +30,19 @@ namespace {
 using namespace tc;
 
 constexpr int BM = 128, BN = 128, BKL = 128;        // BKL: logical k per stage (64 kept values = 128 bytes per row)
-constexpr int NTHREADS = 320;
+constexpr int NTHREADS = 192;
 constexpr int STAGES = 4;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t META_COL0 = 256;                 // accumulators: columns 0-127 and 128-255
 constexpr int A_BYTES = BM * 64 * 2;                // 16 KiB
 constexpr int BH_BYTES = BN * 64 * 2;               // 16 KiB: one half (64 k) of the Z1 stage
-constexpr int STAGE_BYTES = A_BYTES + 2 * BH_BYTES; // 48 KiB
+constexpr int E_BYTES = 128 * 16;                   // positions of one stage
+constexpr int STAGE_BYTES = A_BYTES + 2 * BH_BYTES + E_BYTES; // 50 KiB
 
 struct SParams {
   float* Z; int64_t ldz;        // [N tokens][ldz], written transposed
   int64_t M, N, K;              // rows of S, tokens, logical k
   int m_tiles, n_tiles, k_tiles;
-  const uint4* E;               // positions: [m_tiles][k_tiles][128 lanes] x 16 bytes
   int32_t* status;
 };
 
@@ -75,24 +78,47 @@ __device__ __forceinline__ void umma_bf16_sp(uint32_t tmem_d, uint64_t adesc, ui
       : "memory");
 }
 
-__device__ __forceinline__ void tmem_st4(uint32_t taddr, const uint4& v) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
-               ::"r"(taddr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
-               : "memory");
-  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+// Tile order: groups of GROUP_M row tiles of S; inside a group the row tile runs fastest, then the token tile.
+// The CTAs running at one time then share a few row tiles of S (read from DRAM once) and a band of token tiles
+// (Z1 stays in L2), instead of sweeping all of S for every token tile.
+constexpr int GROUP_M = 8;
+__device__ __forceinline__ void tile_to_mn(int tile, int m_tiles, int n_tiles, int& mt, int& nt) {
+  const int per_group = GROUP_M * n_tiles;
+  const int g = tile / per_group, r = tile - g * per_group;
+  const int gm = min(GROUP_M, m_tiles - g * GROUP_M);
+  mt = g * GROUP_M + r % gm;
+  nt = r / gm;
+}
+
+// 128 rows of 16 bytes, packed (8-row groups 128 bytes apart), no swizzle: the positions of one stage
+__device__ __forceinline__ uint64_t smem_desc_e(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(128 >> 4) << 16;
+  d |= (uint64_t)(128 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  return d;
+}
+// shared -> tensor memory, 128 lanes x 128 bits (four columns), in the tensor-core pipe
+__device__ __forceinline__ void tmem_cp_e(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::1.128x128b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tmem_cp_e_pair(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::2.128x128b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
 }
 
 __global__ void __launch_bounds__(NTHREADS, 1)
-tc_sparse_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const SParams p) {
+tc_sparse_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                 const __grid_constant__ CUtensorMap mapE, const SParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  __shared__ __align__(8) uint64_t bars[3 * STAGES + 4];
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 4];
   __shared__ uint32_t tmem_base_holder;
   __shared__ int abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]), mfull0 = smem_u32(&bars[2 * STAGES]);
-  const uint32_t tfull0 = smem_u32(&bars[3 * STAGES]), tempty0 = smem_u32(&bars[3 * STAGES + 2]);
+  const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]);
+  const uint32_t tfull0 = smem_u32(&bars[2 * STAGES]), tempty0 = smem_u32(&bars[2 * STAGES + 2]);
   const int n_tiles_total = p.m_tiles * p.n_tiles;
 
   if (threadIdx.x == 0) {
@@ -100,7 +126,6 @@ tc_sparse_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, 1);
-      mbar_init(mfull0 + 8 * s, 4);
     }
     for (int s = 0; s < 2; ++s) { mbar_init(tfull0 + 8 * s, 1); mbar_init(tempty0 + 8 * s, 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -123,7 +148,8 @@ tc_sparse_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
       int stage = 0; uint32_t phase = 0; long long issued = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles_total && ok; tile += gridDim.x) {
-        const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+        int mt, nt;
+        tile_to_mn(tile, p.m_tiles, p.n_tiles, mt, nt);
         for (int kt = 0; kt < p.k_tiles; ++kt) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abortp, p.status)) { ok = false; break; }
           const uint32_t fb = full0 + 8 * stage;
@@ -132,6 +158,7 @@ tc_sparse_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
           tma_load_2d(dst, &mapA, kt * 64, mt * BM, fb);                      // 64 kept values = 128 logical k
           tma_load_2d(dst + A_BYTES, &mapB, kt * BKL, nt * BN, fb);
           tma_load_2d(dst + A_BYTES + BH_BYTES, &mapB, kt * BKL + 64, nt * BN, fb);
+          tma_load_2d(dst + A_BYTES + 2 * BH_BYTES, &mapE, 0, (mt * p.k_tiles + kt) * 128, fb);
           ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -159,10 +186,10 @@ tc_sparse_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         const uint32_t tacc = tmem_base + (uint32_t)(as * BN);
         for (int kt = 0; kt < p.k_tiles; ++kt) {
           if (!mbar_wait(full0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
-          if (!mbar_wait(mfull0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
           const uint32_t sb = sa + A_BYTES;
+          tmem_cp_e(tmem_base + META_COL0 + (uint32_t)(4 * stage), smem_desc_e(sb + 2 * BH_BYTES));
 #pragma unroll
           for (int j = 0; j < 4; ++j) {                                        // 32 logical k per instruction
             const uint64_t da = smem_desc_k(sa + j * 32);                      // 16 kept values = 32 bytes
@@ -176,13 +203,14 @@ tc_sparse_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         if (ok) umma_commit(tfull0 + 8 * as);
       }
     }
-  } else if (warp < 6) {
+  } else {
     // ------------------------------------------------------------ epilogue warps
     const int q = warp & 3;
     int local = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < n_tiles_total && ok; tile += gridDim.x, ++local) {
-      const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+      int mt, nt;
+        tile_to_mn(tile, p.m_tiles, p.n_tiles, mt, nt);
       const int as = local & 1;
       const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
       if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
@@ -203,25 +231,6 @@ tc_sparse_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty0 + 8 * as);
     }
-  } else {
-    // ------------------------------------------------------------ positions: global -> tensor memory
-    const int q = warp & 3;
-    int stage = 0; uint32_t phase = 0;
-    bool ok = true;
-    for (int tile = blockIdx.x; tile < n_tiles_total && ok; tile += gridDim.x) {
-      const int mt = tile % p.m_tiles;
-      const uint4* src = p.E + ((int64_t)mt * p.k_tiles) * 128 + q * 32 + lane;
-      for (int kt = 0; kt < p.k_tiles; ++kt) {
-        const uint4 v = __ldg(src + (int64_t)kt * 128);
-        if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abortp, p.status)) { ok = false; break; }
-        tc_fence_after();
-        tmem_st4(tmem_base + ((uint32_t)(q * 32) << 16) + META_COL0 + (uint32_t)(4 * stage), v);
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(mfull0 + 8 * stage);
-        if (++stage == STAGES) { stage = 0; phase ^= 1; }
-      }
-    }
   }
   tc_fence_before();
   __syncthreads();
@@ -239,9 +248,9 @@ tc_sparse_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
 // loads 16 KiB + 32 KiB for 128 x 256 outputs, half of what the one-CTA kernel above loads.
 //   full[s]   (even CTA): armed by the even CTA's producer for the bytes of both CTAs; both CTAs' TMA loads
 //             complete on it (cta_group::2 loads may signal the pair's other CTA)
-//   mfull[s]  (even CTA): 8 arrivals, one per position-loading warp of either CTA
 //   empty[s], tfull (both CTAs): tcgen05.commit multicast to the pair
 //   tempty    (even CTA): 8 arrivals, one per epilogue warp of either CTA
+// The positions of both CTAs go from their shared to their tensor memory with one tcgen05.cp of the pair.
 // One accumulator buffer of 256 columns (the positions need tensor-memory columns too).
 constexpr int BN2 = 256;
 
@@ -297,17 +306,18 @@ __device__ __forceinline__ void cluster_sync_all() {
 }
 
 __global__ void __launch_bounds__(NTHREADS, 1)
-tc_sparse_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const SParams p) {
+tc_sparse_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                      const __grid_constant__ CUtensorMap mapE, const SParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  __shared__ __align__(8) uint64_t bars[3 * STAGES + 2];
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 2];
   __shared__ uint32_t tmem_base_holder;
   __shared__ int abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
-  const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]), mfull0 = smem_u32(&bars[2 * STAGES]);
-  const uint32_t tfull = smem_u32(&bars[3 * STAGES]), tempty = smem_u32(&bars[3 * STAGES + 1]);
+  const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]);
+  const uint32_t tfull = smem_u32(&bars[2 * STAGES]), tempty = smem_u32(&bars[2 * STAGES + 1]);
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   const int m_pairs = p.m_tiles >> 1;                       // 256-row tiles
   const int n_tiles_total = m_pairs * p.n_tiles;            // p.n_tiles counts 256-token tiles here
@@ -317,7 +327,6 @@ tc_sparse_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, 1);
-      mbar_init(mfull0 + 8 * s, 8);
     }
     mbar_init(tfull, 1);
     mbar_init(tempty, 8);
@@ -342,7 +351,8 @@ tc_sparse_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
       int stage = 0; uint32_t phase = 0; long long issued = 0;
       bool ok = true;
       for (int tile = pair; tile < n_tiles_total && ok; tile += n_pairs) {
-        const int mt = tile % m_pairs, nt = tile / m_pairs;
+        int mt, nt;
+        tile_to_mn(tile, m_pairs, p.n_tiles, mt, nt);
         const int row0 = mt * 256 + (int)rank * 128, tok0 = nt * BN2 + (int)rank * 128;
         for (int kt = 0; kt < p.k_tiles; ++kt) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abortp, p.status)) { ok = false; break; }
@@ -352,6 +362,7 @@ tc_sparse_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
           tma_load_2d_pair(dst, &mapA, kt * 64, row0, fb);
           tma_load_2d_pair(dst + A_BYTES, &mapB, kt * BKL, tok0, fb);
           tma_load_2d_pair(dst + A_BYTES + BH_BYTES, &mapB, kt * BKL + 64, tok0, fb);
+          tma_load_2d_pair(dst + A_BYTES + 2 * BH_BYTES, &mapE, 0, ((2 * mt + (int)rank) * p.k_tiles + kt) * 128, fb);
           ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -376,10 +387,10 @@ tc_sparse_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
         tc_fence_after();
         for (int kt = 0; kt < p.k_tiles; ++kt) {
           if (!mbar_wait(full0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
-          if (!mbar_wait(mfull0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
           const uint32_t sb = sa + A_BYTES;
+          tmem_cp_e_pair(tmem_base + META_COL0 + (uint32_t)(4 * stage), smem_desc_e(sb + 2 * BH_BYTES));
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const uint64_t da = smem_desc_k(sa + j * 32);
@@ -393,14 +404,15 @@ tc_sparse_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
         if (ok) umma_commit_pair(tfull);
       }
     }
-  } else if (warp < 6) {
+  } else {
     // ------------------------------------------------------------ epilogue warps (both CTAs)
     const int q = warp & 3;
     const uint32_t tempty_lead = map_to_cta(tempty, 0);
     int local = 0;
     bool ok = true;
     for (int tile = pair; tile < n_tiles_total && ok; tile += n_pairs, ++local) {
-      const int mt = tile % m_pairs, nt = tile / m_pairs;
+      int mt, nt;
+        tile_to_mn(tile, m_pairs, p.n_tiles, mt, nt);
       if (!mbar_wait(tfull, (uint32_t)local & 1u, abortp, p.status)) { ok = false; break; }
       tc_fence_after();
       const int64_t row = (int64_t)mt * 256 + rank * 128 + q * 32 + lane;
@@ -418,25 +430,6 @@ tc_sparse_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(tempty_lead);
-    }
-  } else {
-    // ------------------------------------------------------------ positions: global -> tensor memory (both CTAs)
-    const int q = warp & 3;
-    int stage = 0; uint32_t phase = 0;
-    bool ok = true;
-    for (int tile = pair; tile < n_tiles_total && ok; tile += n_pairs) {
-      const int mt = tile % m_pairs;
-      const uint4* src = p.E + ((int64_t)(2 * mt + (int)rank) * p.k_tiles) * 128 + q * 32 + lane;
-      for (int kt = 0; kt < p.k_tiles; ++kt) {
-        const uint4 v = __ldg(src + (int64_t)kt * 128);
-        if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abortp, p.status)) { ok = false; break; }
-        tc_fence_after();
-        tmem_st4(tmem_base + ((uint32_t)(q * 32) << 16) + META_COL0 + (uint32_t)(4 * stage), v);
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(map_to_cta(mfull0 + 8 * stage, 0));
-        if (++stage == STAGES) { stage = 0; phase ^= 1; }
-      }
     }
   }
   tc_fence_before();
@@ -510,6 +503,20 @@ bool make_map_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t K, 
   return r == CUDA_SUCCESS;
 }
 
+// positions: [rows of 16 bytes], box = 128 rows, no swizzle
+bool make_map_e(CUtensorMap* map, const void* base, int64_t rows) {
+  PFN_cuTensorMapEncodeTiled_v12000 enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t dims[2] = {4, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {16};
+  cuuint32_t box[2] = {4, 128};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 int g_sparse_pairs = 1;   // 0: the one-CTA kernel only (tests compare the two)
@@ -533,13 +540,13 @@ void launch_compress_24(armor_ctx* c, const float* S, const uint8_t* M, void* Sc
 armor_status launch_tc_sparse(armor_ctx* c, const void* Sc, const void* E, const void* z1_bf16, float* z2, int64_t n,
                               cudaStream_t s) {
   if (!tc_sparse_ok(c) || n <= 0) return ARMOR_ERR_UNSUPPORTED;
-  CUtensorMap mA, mB;
+  CUtensorMap mA, mB, mE;
   if (!make_map_bf16(&mA, Sc, c->d_out, c->d_in / 2, c->d_in / 2)) return ARMOR_ERR_CUDA;
   if (!make_map_bf16(&mB, z1_bf16, n, c->d_in, c->d_in)) return ARMOR_ERR_CUDA;
+  if (!make_map_e(&mE, E, (c->d_out / 128) * (c->d_in / 128) * 128)) return ARMOR_ERR_CUDA;
   SParams p{};
   p.Z = z2; p.ldz = c->d_out; p.M = c->d_out; p.N = n; p.K = c->d_in;
   p.m_tiles = (int)(c->d_out / BM); p.n_tiles = (int)((n + BN - 1) / BN); p.k_tiles = (int)(c->d_in / BKL);
-  p.E = static_cast<const uint4*>(E);
   p.status = c->status;
   constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024;
   static bool attr = false;
@@ -573,11 +580,11 @@ armor_status launch_tc_sparse(armor_ctx* c, const void* Sc, const void* E, const
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, tc_sparse_pair_kernel, mA, mB, p) != cudaSuccess) return ARMOR_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, tc_sparse_pair_kernel, mA, mB, mE, p) != cudaSuccess) return ARMOR_ERR_CUDA;
   } else {
     const int tiles = p.m_tiles * p.n_tiles;
     const int grid = tiles < n_sm ? tiles : n_sm;
-    tc_sparse_kernel<<<grid, NTHREADS, SMEM, s>>>(mA, mB, p);
+    tc_sparse_kernel<<<grid, NTHREADS, SMEM, s>>>(mA, mB, mE, p);
   }
   if (timed) {
     cudaEventRecord(c->ev_end[c->timing_n], s);
