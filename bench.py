@@ -356,6 +356,35 @@ def run_ours(args, cfg):
                 other_modes[name]["s_per_20000_iterations"] = 20000 * ms_x / iters / 1e3
             del cx, sx
 
+        # the deployment form on the same layer: fp32-grade, bf16 with the core dense, bf16 with the 2:4 core packed
+        # for the sparse tensor cores (packed once, and packed on every call)
+        cf = Bd.ArmorContext(lcfg.d_out, lcfg.d_in, lcfg.d_block, device=dev, precision=prec, seed=lcfg.seed)
+        sf = cf.init(W_d, H)
+        cf.bcd_step(sf, H, 0, 2, want_stats=False)
+        xb = xt_d.to(torch.bfloat16)
+        y32 = cf.apply(sf, xt_d)
+        fwd = {"tokens": APPLY_TOKENS}
+        variants = [("fp32", lambda: cf.apply(sf, xt_d)), ("bf16_dense_core", lambda: cf.apply(sf, xb))]
+        if lcfg.d_out % 128 == 0 and lcfg.d_in % 128 == 0:
+            packed = cf.pack_core(sf)
+            variants += [("bf16_sparse_core_packed_once", lambda: cf.apply_packed(sf, packed, xb)),
+                         ("bf16_sparse_core_packed_per_call", lambda: cf.apply(sf, xb, sparse=True))]
+        for name, fn in variants:
+            for _ in range(3):
+                yv = fn()
+            torch.cuda.synchronize()
+            Bd.armor_gemm_timing_enable(cf.ctx, True)
+            Bd.armor_gemm_timing(cf.ctx)
+            ms_f, _ = t_phase(lambda: [fn() for _ in range(10)])
+            n_c, ms_c, fl_c = Bd.armor_gemm_timing(cf.ctx)
+            Bd.armor_gemm_timing_enable(cf.ctx, False)
+            fwd[name] = {"ms_per_forward": ms_f / 10, "core_product_ms": ms_c / 10,
+                         "core_product_tflops_dense_equivalent": fl_c / (ms_c * 1e-3) / 1e12 if ms_c > 0 else None,
+                         "rel_diff_to_fp32": float(((yv.float() - y32).norm() / y32.norm()).item())}
+        fwd["device_status"] = cf.device_status()[:5]
+        other_modes["forward"] = fwd
+        del cf, sf
+
     # ---- end to end (host buffers)
     if args.no_e2e:
         ms_e2e = None

@@ -180,6 +180,22 @@ armor_status armor_apply(armor_ctx* ctx, const float* d_A, const float* d_B, con
                          const uint8_t* d_M, const float* d_r1, const float* d_r2, const void* d_x,
                          void* d_y, int32_t xy_dtype, int64_t n_tokens, armor_stream_t stream);
 
+/* The deployment form with the core packed once (Section 3.1; the paper's inference measurements, Section 4.3,
+ * use a 2:4 core in the hardware's compressed format).  armor_packed_core_bytes: size of the packed core,
+ * d_out*d_in bytes of kept values (bf16, two of every four, in order) followed by d_out*d_in/8 bytes of 2-bit
+ * positions in the order the sparse tensor cores read them (needs 2:4 and d_out, d_in multiples of 128, else
+ * UNSUPPORTED).  armor_pack_core: packs S with the kept positions of d_M into d_packed (device, caller-owned,
+ * 128-byte aligned); a group of d_M with more than two kept positions is counted in device status word 4.
+ * armor_apply_packed: y = A S B x for bf16 x [n_tokens, d_in] -> bf16 y [n_tokens, d_out] with the packed
+ * core on the sparse tensor cores (fp32 accumulation; the wrapper products as in armor_apply; d_r1, d_r2 as
+ * there).  Equal to armor_apply with ARMOR_DTYPE_BF16_SPARSE, which packs on every call. */
+armor_status armor_packed_core_bytes(const armor_config* cfg, size_t* out_bytes);
+armor_status armor_pack_core(armor_ctx* ctx, const float* d_S, const uint8_t* d_M, void* d_packed,
+                             armor_stream_t stream);
+armor_status armor_apply_packed(armor_ctx* ctx, const float* d_A, const float* d_B, const void* d_packed,
+                                const float* d_r1, const float* d_r2, const void* d_x, void* d_y,
+                                int64_t n_tokens, armor_stream_t stream);
+
 /* Copies up to n device status words to h_codes (host).  Word 0: number of
  * Cholesky failures since the context was created; word 1: first failing
  * block id + 1; word 2: bounded waits that gave up; word 4: mask groups the sparse forward could

@@ -547,20 +547,10 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
   return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
 }
 
-armor_status armor_apply(armor_ctx* c, const float* A, const float* B, const float* S, const uint8_t* M,
-                         const float* r1, const float* r2, const void* d_x, void* d_y, int32_t xy_dtype,
-                         int64_t n_tokens, armor_stream_t stream) {
-  if (!c || !A || !B || !S || n_tokens < 0) return ARMOR_ERR_INVALID_ARG;
-  if (n_tokens == 0) return ARMOR_OK;
-  if (!d_x || !d_y) return ARMOR_ERR_INVALID_ARG;
-  if (xy_dtype != ARMOR_DTYPE_F32 && xy_dtype != ARMOR_DTYPE_BF16 && xy_dtype != ARMOR_DTYPE_BF16_SPARSE)
-    return ARMOR_ERR_UNSUPPORTED;
-  const bool sparse = (xy_dtype == ARMOR_DTYPE_BF16_SPARSE);
-  if (sparse && !M) return ARMOR_ERR_INVALID_ARG;
-  if (sparse && !tc_sparse_ok(c)) return ARMOR_ERR_UNSUPPORTED;
-  if ((r1 == nullptr) != (r2 == nullptr)) return ARMOR_ERR_INVALID_ARG;
-  cudaStream_t s = cs(stream);
-  const bool bf16 = (xy_dtype != ARMOR_DTYPE_F32);
+// x -> y = A (S (B x)) in chunks of tokens; `packed` non-null: the core comes packed for the sparse tensor cores
+static armor_status apply_impl(armor_ctx* c, const float* A, const float* B, const float* S, const void* packed,
+                               const float* r1, const float* r2, const void* d_x, void* d_y, bool bf16, int64_t n_tokens,
+                               cudaStream_t s) {
   const size_t esz = bf16 ? 2 : 4;
   const int64_t d_out = c->d_out, d_in = c->d_in;
   const int64_t chunk = d_out < d_in ? d_out : d_in;   // z1 [chunk, d_in] and z2 [chunk, d_out] fit W-shaped scratch
@@ -583,13 +573,64 @@ armor_status armor_apply(armor_ctx* c, const float* A, const float* B, const flo
       }
     }
     bd_right(c, xc, B, true, c->T, n, d_in, 1.f, nullptr, 0.f, s);                   // z1 = x B^T
-    armor_status st = apply_core(c, c->T, S, M, c->E, n, bf16, sparse, s);                      // z2 = z1 S^T
+    armor_status st = apply_core(c, c->T, S, packed, c->E, n, bf16, s);              // z2 = z1 S^T
     if (st != ARMOR_OK) return st;
     bd_right(c, c->E, A, true, yc, n, d_out, 1.f, nullptr, 0.f, s);                  // y = z2 A^T
     if (bf16) launch_f32_to_bf16(c, yc, r2, static_cast<char*>(d_y) + (size_t)(t0 * d_out) * esz, n, d_out, s);
     else if (r2) launch_scale_rows_cols(c, yc, r2, nullptr, yc, n, d_out, s);
   }
   return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+}
+
+armor_status armor_apply(armor_ctx* c, const float* A, const float* B, const float* S, const uint8_t* M,
+                         const float* r1, const float* r2, const void* d_x, void* d_y, int32_t xy_dtype,
+                         int64_t n_tokens, armor_stream_t stream) {
+  if (!c || !A || !B || !S || n_tokens < 0) return ARMOR_ERR_INVALID_ARG;
+  if (n_tokens == 0) return ARMOR_OK;
+  if (!d_x || !d_y) return ARMOR_ERR_INVALID_ARG;
+  if (xy_dtype != ARMOR_DTYPE_F32 && xy_dtype != ARMOR_DTYPE_BF16 && xy_dtype != ARMOR_DTYPE_BF16_SPARSE)
+    return ARMOR_ERR_UNSUPPORTED;
+  const bool sparse = (xy_dtype == ARMOR_DTYPE_BF16_SPARSE);
+  if (sparse && !M) return ARMOR_ERR_INVALID_ARG;
+  if (sparse && !tc_sparse_ok(c)) return ARMOR_ERR_UNSUPPORTED;
+  if ((r1 == nullptr) != (r2 == nullptr)) return ARMOR_ERR_INVALID_ARG;
+  cudaStream_t s = cs(stream);
+  const void* packed = nullptr;
+  if (sparse) {
+    char* buf = reinterpret_cast<char*>(c->P);          // workspace: values wn bytes, positions wn / 8 bytes
+    launch_compress_24(c, S, M, buf, buf + tc_sparse_values_bytes(c), s);
+    packed = buf;
+  }
+  return apply_impl(c, A, B, S, packed, r1, r2, d_x, d_y, xy_dtype != ARMOR_DTYPE_F32, n_tokens, s);
+}
+
+armor_status armor_packed_core_bytes(const armor_config* cfg, size_t* out_bytes) {
+  if (!cfg || !out_bytes) return ARMOR_ERR_INVALID_ARG;
+  armor_status st = check_config(cfg);
+  if (st != ARMOR_OK) return st;
+  if (cfg->n_keep != 2 || cfg->m_group != 4 || cfg->d_out % 128 || cfg->d_in % 128) return ARMOR_ERR_UNSUPPORTED;
+  const size_t wn = (size_t)cfg->d_out * (size_t)cfg->d_in;
+  *out_bytes = wn + wn / 8;
+  return ARMOR_OK;
+}
+
+armor_status armor_pack_core(armor_ctx* c, const float* S, const uint8_t* M, void* d_packed, armor_stream_t stream) {
+  if (!c || !S || !M || !d_packed) return ARMOR_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(d_packed) % 128) return ARMOR_ERR_INVALID_ARG;
+  if (!tc_sparse_ok(c)) return ARMOR_ERR_UNSUPPORTED;
+  char* buf = static_cast<char*>(d_packed);
+  launch_compress_24(c, S, M, buf, buf + tc_sparse_values_bytes(c), cs(stream));
+  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+}
+
+armor_status armor_apply_packed(armor_ctx* c, const float* A, const float* B, const void* d_packed, const float* r1,
+                                const float* r2, const void* d_x, void* d_y, int64_t n_tokens, armor_stream_t stream) {
+  if (!c || !A || !B || !d_packed || n_tokens < 0) return ARMOR_ERR_INVALID_ARG;
+  if (n_tokens == 0) return ARMOR_OK;
+  if (!d_x || !d_y || reinterpret_cast<uintptr_t>(d_packed) % 128) return ARMOR_ERR_INVALID_ARG;
+  if (!tc_sparse_ok(c)) return ARMOR_ERR_UNSUPPORTED;
+  if ((r1 == nullptr) != (r2 == nullptr)) return ARMOR_ERR_INVALID_ARG;
+  return apply_impl(c, A, B, nullptr, d_packed, r1, r2, d_x, d_y, true, n_tokens, cs(stream));
 }
 
 }  // extern "C"

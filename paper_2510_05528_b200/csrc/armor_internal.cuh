@@ -160,8 +160,8 @@ armor_status prepare_H(armor_ctx* c, const float* H, cudaStream_t s);
 armor_status gram_accumulate(armor_ctx* c, const void* X, int x_dtype, int64_t n_rows, int64_t ldx, float* H,
                              cudaStream_t s);
 // z2 [n, d_out] = z1 [n, d_in] * S^T
-armor_status apply_core(armor_ctx* c, const float* z1, const float* S, const uint8_t* M, float* z2, int64_t n, bool bf16,
-                        bool sparse, cudaStream_t s);
+armor_status apply_core(armor_ctx* c, const float* z1, const float* S, const void* packed, float* z2, int64_t n,
+                        bool bf16, cudaStream_t s);
 
 // deterministic reductions (two stages, fixed order)
 void dot_to_ptr(armor_ctx* c, const float* x, const float* y, int64_t n, double* out, cudaStream_t s);

@@ -101,15 +101,14 @@ armor_status gram_accumulate(armor_ctx* c, const void* Xv, int x_dtype, int64_t 
   return ARMOR_OK;
 }
 
-armor_status apply_core(armor_ctx* c, const float* z1, const float* S, const uint8_t* M, float* z2, int64_t n, bool bf16,
-                        bool sparse, cudaStream_t s) {
+armor_status apply_core(armor_ctx* c, const float* z1, const float* S, const void* packed, float* z2, int64_t n,
+                        bool bf16, cudaStream_t s) {
   const int64_t d_in = c->d_in, d_out = c->d_out;
-  if (sparse) {
-    // bf16 deployment with the 2:4 core on the sparse tensor cores: kept values and positions from S and M
-    if (!bf16 || !M || !tc_sparse_ok(c)) return ARMOR_ERR_UNSUPPORTED;
-    char* buf = reinterpret_cast<char*>(c->P);                 // values: wn bytes, positions: wn / 8 bytes
+  if (packed) {
+    // bf16 deployment with the 2:4 core on the sparse tensor cores: kept values, then positions
+    if (!bf16 || !tc_sparse_ok(c)) return ARMOR_ERR_UNSUPPORTED;
+    const char* buf = static_cast<const char*>(packed);
     launch_f32_to_bf16(c, z1, nullptr, c->U, n, d_in, s);
-    launch_compress_24(c, S, M, buf, buf + tc_sparse_values_bytes(c), s);
     return launch_tc_sparse(c, buf, buf + tc_sparse_values_bytes(c), c->U, z2, n, s);
   }
   if (bf16 && c->cfg.precision != ARMOR_PREC_SIMT && d_out % 32 == 0 && d_in % 8 == 0) {

@@ -604,6 +604,10 @@ def test_sparse_tensor_core_forward_against_the_oracle(mid_data):
         # against the dense bf16 forward: the same rounded operands, only the order of the fp32 sums differs
         yd = ctx.apply(st, xb, denormalize=den)
         assert rel(y.float().cpu().numpy(), yd.float().cpu().numpy()) < 1e-3
+        # the core packed once, then applied: the same bits as packing on every call
+        packed = ctx.pack_core(st)
+        assert packed.numel() == MID.d_out * MID.d_in * 9 // 8
+        assert torch.equal(ctx.apply_packed(st, packed, xb, denormalize=den), y)
     with pytest.raises(ValueError):
         ctx.apply(st, xb.float(), sparse=True)
     ctx48 = make(MID, Bd.PREC_FP32X3, n_keep=4, m_group=8)
