@@ -572,10 +572,15 @@ static armor_status apply_impl(armor_ctx* c, const float* A, const float* B, con
         xc = c->Tmp;
       }
     }
+    // the bf16 forward rounds z1, S and y to 8 bits: its wrapper products take one tf32 pass (11 bits)
+    c->block_one_pass = bf16 ? 1 : 0;
     bd_right(c, xc, B, true, c->T, n, d_in, 1.f, nullptr, 0.f, s);                   // z1 = x B^T
+    c->block_one_pass = 0;
     armor_status st = apply_core(c, c->T, S, packed, c->E, n, bf16, s);              // z2 = z1 S^T
     if (st != ARMOR_OK) return st;
+    c->block_one_pass = bf16 ? 1 : 0;
     bd_right(c, c->E, A, true, yc, n, d_out, 1.f, nullptr, 0.f, s);                  // y = z2 A^T
+    c->block_one_pass = 0;
     if (bf16) launch_f32_to_bf16(c, yc, r2, static_cast<char*>(d_y) + (size_t)(t0 * d_out) * esz, n, d_out, s);
     else if (r2) launch_scale_rows_cols(c, yc, r2, nullptr, yc, n, d_out, s);
   }

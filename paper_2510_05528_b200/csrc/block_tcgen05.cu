@@ -55,6 +55,7 @@ struct BParams {
   float alpha, beta;
   int32_t* status;
   int batch_fastest;                // 1: consecutive work items are consecutive batches (neighbouring column blocks)
+  int one_pass;                     // 1: operands as they are, rounded to tf32 by the tensor core; no low parts
 };
 
 __device__ __forceinline__ void load_operand(uint32_t dst, const CUtensorMap* map, const OpCoord& o, int b, int t, int kc,
@@ -180,9 +181,13 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
           for (int k = 0; k < BK / 8; ++k) {
             const uint64_t da = operand_desc(sa, p.a.mn_major, k), dal = operand_desc(sa_lo, p.a.mn_major, k);
             const uint64_t dbm = operand_desc(sb, p.b.mn_major, k), dbl = operand_desc(sb_lo, p.b.mn_major, k);
-            umma_tf32(tacc, dal, dbm, idesc, (uint32_t)((kc > 0) | (k != 0)));
-            umma_tf32(tacc, da, dbl, idesc, 1);
-            umma_tf32(tacc, da, dbm, idesc, 1);
+            if (p.one_pass) {
+              umma_tf32(tacc, da, dbm, idesc, (uint32_t)((kc > 0) | (k != 0)));
+            } else {
+              umma_tf32(tacc, dal, dbm, idesc, (uint32_t)((kc > 0) | (k != 0)));
+              umma_tf32(tacc, da, dbl, idesc, 1);
+              umma_tf32(tacc, da, dbm, idesc, 1);
+            }
           }
           umma_commit(empty0 + 8 * stage);   // frees the stage once these MMAs have read it
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -200,7 +205,7 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         if (!mbar_wait(full0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
         float4* base = reinterpret_cast<float4*>(smem + (size_t)stage * STAGE_BYTES);
 #pragma unroll
-        for (int op = 0; op < 2; ++op) {
+        for (int op = 0; op < (p.one_pass ? 0 : 2); ++op) {
           float4* hi = base + op * (2 * OP_BYTES / 16);
           float4* lo = hi + OP_BYTES / 16;
 #pragma unroll
@@ -366,6 +371,7 @@ armor_status tc_bd_right(armor_ctx* c, const float* in, const float* Bblk, bool 
   p.alpha = alpha; p.beta = add ? beta : 0.f;
   p.n_split = 1; p.r_s = 0; p.m_valid = 1 << 30;
   p.batch_fastest = 1;   // neighbouring CTAs read neighbouring column blocks of the same rows
+  p.one_pass = c->block_one_pass;
   return launch(c, A, B, p, s);
 }
 
@@ -385,6 +391,7 @@ armor_status tc_bd_left(armor_ctx* c, const float* Ablk, bool transA, const floa
   p.m_tiles = db / TILE; p.n_tiles = (int)((cols + TILE - 1) / TILE); p.batch = nb; p.k_chunks = db / BK;
   p.alpha = alpha; p.beta = add ? beta : 0.f;
   p.n_split = 1; p.r_s = 0; p.m_valid = 1 << 30;
+  p.one_pass = c->block_one_pass;
   return launch(c, A, B, p, s);
 }
 
