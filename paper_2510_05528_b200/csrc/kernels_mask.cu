@@ -62,21 +62,20 @@ __device__ __forceinline__ void pinv2(double k11, double k12, double k22, double
   red = z1 * w1 + z2 * w2;
 }
 
-constexpr int NK_MAX = 6;   // largest number of kept positions per group (6:8)
-
-// n x n SPD solve (n <= NK_MAX) by unpivoted Cholesky; false if a pivot is not positive (that mask is skipped).
-__device__ __forceinline__ bool chol_small(int n, const double (&Kin)[NK_MAX][NK_MAX], const double (&z)[NK_MAX],
-                                           double (&w)[NK_MAX],
+// n x n SPD solve (n <= NKM) by unpivoted Cholesky; false if a pivot is not positive (that mask is skipped).
+template <int NKM>
+__device__ __forceinline__ bool chol_small(int n, const double (&Kin)[NKM][NKM], const double (&z)[NKM],
+                                           double (&w)[NKM],
                                            double& red) {
-  double L[NK_MAX][NK_MAX];
+  double L[NKM][NKM];
 #pragma unroll
-  for (int i = 0; i < NK_MAX; ++i) {
+  for (int i = 0; i < NKM; ++i) {
 #pragma unroll
-    for (int j = 0; j < NK_MAX; ++j) {
+    for (int j = 0; j < NKM; ++j) {
       if (i >= n || j > i) continue;
       double sacc = Kin[i][j];
 #pragma unroll
-      for (int p = 0; p < NK_MAX; ++p)
+      for (int p = 0; p < NKM; ++p)
         if (p < j) sacc -= L[i][p] * L[j][p];
       if (i == j) {
         if (!(sacc > 0.0) || !isfinite(sacc)) return false;
@@ -86,38 +85,38 @@ __device__ __forceinline__ bool chol_small(int n, const double (&Kin)[NK_MAX][NK
       }
     }
   }
-  double y[NK_MAX];
+  double y[NKM];
 #pragma unroll
-  for (int i = 0; i < NK_MAX; ++i) {
+  for (int i = 0; i < NKM; ++i) {
     if (i >= n) continue;
     double sacc = z[i];
 #pragma unroll
-    for (int p = 0; p < NK_MAX; ++p)
+    for (int p = 0; p < NKM; ++p)
       if (p < i) sacc -= L[i][p] * y[p];
     y[i] = sacc / L[i][i];
   }
 #pragma unroll
-  for (int i = NK_MAX - 1; i >= 0; --i) {
+  for (int i = NKM - 1; i >= 0; --i) {
     if (i >= n) continue;
     double sacc = y[i];
 #pragma unroll
-    for (int p = 0; p < NK_MAX; ++p)
+    for (int p = 0; p < NKM; ++p)
       if (p > i && p < n) sacc -= L[p][i] * w[p];
     w[i] = sacc / L[i][i];
   }
   red = 0.0;
 #pragma unroll
-  for (int i = 0; i < NK_MAX; ++i)
+  for (int i = 0; i < NKM; ++i)
     if (i < n) red += z[i] * w[i];
   return true;
 }
 
-// One CTA per (i, j) block of the core, N:M groups with M = MG (4 or 8) and N = n_keep (<= NK_MAX).
+// One CTA per (i, j) block of the core, N:M groups with M = MG (4 or 8) and N = n_keep (<= NKM: 4 for 2:4 and 4:8, 6 for 5:8 and 6:8).
 // Pass 1: every group of the block is scored, keyed and the arg-min found by warp shuffles.
 // Pass 2: thread b < 2^MG evaluates the mask with bit pattern b (if it keeps exactly n_keep positions);
 // the best one is found with the oracle's order: larger reduction first; among equal reductions the
 // incumbent, then the lexicographically first index tuple.
-template <int MG>
+template <int MG, int NKM>
 __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict__ Gam, const float* __restrict__ S,
                                                          const uint8_t* __restrict__ M, const float* __restrict__ alpha,
                                                          const float* __restrict__ Kfull, SelRec* __restrict__ sel,
@@ -215,35 +214,37 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
   }
   const unsigned cand = threadIdx.x;
   bool ok = cand < (1u << MG) && __popc(cand) == n_keep;
-  double red = 0.0, wv[NK_MAX] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
-  int pos[NK_MAX] = {0, 0, 0, 0, 0, 0};
+  double red = 0.0, wv[NKM];
+  int pos[NKM];
+#pragma unroll
+  for (int i = 0; i < NKM; ++i) { wv[i] = 0.0; pos[i] = 0; }
   if (ok) {
     int cnt = 0;
 #pragma unroll
     for (int p = 0; p < MG; ++p)
-      if ((cand >> p) & 1u) { if (cnt < NK_MAX) pos[cnt] = p; ++cnt; }
+      if ((cand >> p) & 1u) { if (cnt < NKM) pos[cnt] = p; ++cnt; }
     if (n_keep == 2) {
       pinv2((double)Kj[(int64_t)(lc + pos[0]) * db + lc + pos[0]], (double)Kj[(int64_t)(lc + pos[0]) * db + lc + pos[1]],
             (double)Kj[(int64_t)(lc + pos[1]) * db + lc + pos[1]], z[pos[0]], z[pos[1]], wv[0], wv[1], red);
     } else {
-      double Ks[NK_MAX][NK_MAX], zs[NK_MAX];
+      double Ks[NKM][NKM], zs[NKM];
 #pragma unroll
-      for (int i = 0; i < NK_MAX; ++i) {
+      for (int i = 0; i < NKM; ++i) {
         zs[i] = 0.0;
 #pragma unroll
-        for (int j = 0; j < NK_MAX; ++j) Ks[i][j] = 0.0;
+        for (int j = 0; j < NKM; ++j) Ks[i][j] = 0.0;
       }
 #pragma unroll
-      for (int i = 0; i < NK_MAX; ++i) {
+      for (int i = 0; i < NKM; ++i) {
         if (i >= n_keep) continue;
 #pragma unroll
         for (int p = 0; p < MG; ++p)
           if (p == pos[i]) zs[i] = z[p];
 #pragma unroll
-        for (int j = 0; j < NK_MAX; ++j)
+        for (int j = 0; j < NKM; ++j)
           if (j < n_keep) Ks[i][j] = (double)Kj[(int64_t)(lc + pos[i]) * db + lc + pos[j]];
       }
-      ok = chol_small(n_keep, Ks, zs, wv, red);
+      ok = chol_small<NKM>(n_keep, Ks, zs, wv, red);
     }
     red /= a_r;
   }
@@ -294,7 +295,7 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
 #pragma unroll
   for (int p = 0; p < MG; ++p) rec.old_val[p] = (float)sg_old[p];
 #pragma unroll
-  for (int i = 0; i < NK_MAX; ++i)
+  for (int i = 0; i < NKM; ++i)
     if (i < n_keep) rec.new_val[pos[i]] = (float)(wv[i] / a_r);
   // <Gamma, dS> restricted to this group: this block's share of <E H_w, V>
   double ehv = 0.0;
@@ -430,14 +431,12 @@ void launch_alpha(armor_ctx* c, const float* A, cudaStream_t s) {
 void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const uint8_t* M, int64_t t, cudaStream_t s) {
   const int mg = c->cfg.m_group;
   const uint64_t n_groups = (uint64_t)(c->d_out * (c->d_in / mg));
-  if (mg == 8)
-    mask_select_kernel<8><<<c->nbo * c->nbi, NT, 0, s>>>(Gam, S, M, c->alpha, c->Kfull, c->sel, c->partblk, c->d_in,
-                                                        c->db, c->nbi, c->cfg.n_keep, c->cfg.select_mode, c->cfg.seed,
-                                                        (uint64_t)t, n_groups);
-  else
-    mask_select_kernel<4><<<c->nbo * c->nbi, NT, 0, s>>>(Gam, S, M, c->alpha, c->Kfull, c->sel, c->partblk, c->d_in,
-                                                        c->db, c->nbi, c->cfg.n_keep, c->cfg.select_mode, c->cfg.seed,
-                                                        (uint64_t)t, n_groups);
+#define ARMOR_SELECT_ARGS Gam, S, M, c->alpha, c->Kfull, c->sel, c->partblk, c->d_in, c->db, c->nbi, c->cfg.n_keep, \
+                          c->cfg.select_mode, c->cfg.seed, (uint64_t)t, n_groups
+  if (mg == 8 && c->cfg.n_keep > 4) mask_select_kernel<8, 6><<<c->nbo * c->nbi, NT, 0, s>>>(ARMOR_SELECT_ARGS);
+  else if (mg == 8) mask_select_kernel<8, 4><<<c->nbo * c->nbi, NT, 0, s>>>(ARMOR_SELECT_ARGS);
+  else mask_select_kernel<4, 4><<<c->nbo * c->nbi, NT, 0, s>>>(ARMOR_SELECT_ARGS);
+#undef ARMOR_SELECT_ARGS
   c->launches++;
 }
 
