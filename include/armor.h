@@ -196,6 +196,22 @@ armor_status armor_apply_packed(armor_ctx* ctx, const float* d_A, const float* d
                                 const float* d_r1, const float* d_r2, const void* d_x, void* d_y,
                                 int64_t n_tokens, armor_stream_t stream);
 
+/* The whole layer packed for a bf16 forward that touches no fp32 intermediate (Section 3.1 and the last
+ * paragraph of Section 3.2: the normalisation's scales are folded into the wrappers).  The packed layer is the
+ * packed core of armor_pack_core followed by the blocks of B with their columns scaled by r1 and the blocks of A
+ * with their rows scaled by r2, both rounded to bf16 (d_r1 and d_r2 both NULL: no scales).
+ * armor_packed_layer_bytes gives its size (needs 2:4, d_out and d_in multiples of 128, d_block 128 or 256, else
+ * UNSUPPORTED); d_packed is caller-owned device memory, 128-byte aligned.
+ * armor_apply_layer: bf16 x [n_tokens, d_in] -> bf16 y [n_tokens, d_out] (both 16-byte aligned), three kernels
+ * per chunk of tokens: z1 = (r1 . x) B^T and y = r2 . (z2 A^T) as batched bf16 tensor-core products over the
+ * blocks, z2 = z1 S^T on the sparse tensor cores; fp32 accumulation, z1 and z2 rounded to bf16 in the
+ * context's workspace. */
+armor_status armor_packed_layer_bytes(const armor_config* cfg, size_t* out_bytes);
+armor_status armor_pack_layer(armor_ctx* ctx, const float* d_A, const float* d_B, const float* d_S, const uint8_t* d_M,
+                              const float* d_r1, const float* d_r2, void* d_packed, armor_stream_t stream);
+armor_status armor_apply_layer(armor_ctx* ctx, const void* d_packed, const void* d_x, void* d_y, int64_t n_tokens,
+                               armor_stream_t stream);
+
 /* Copies up to n device status words to h_codes (host).  Word 0: number of
  * Cholesky failures since the context was created; word 1: first failing
  * block id + 1; word 2: bounded waits that gave up; word 4: mask groups the sparse forward could

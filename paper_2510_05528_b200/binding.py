@@ -26,6 +26,7 @@ DTYPE_F32, DTYPE_BF16, DTYPE_BF16_SPARSE = 0, 1, 2
 
 EXPORTS = ["armor_workspace_bytes", "armor_create", "armor_destroy", "armor_gram", "armor_init",
            "armor_bcd_step", "armor_proxy_loss", "armor_apply", "armor_packed_core_bytes", "armor_pack_core", "armor_apply_packed",
+           "armor_packed_layer_bytes", "armor_pack_layer", "armor_apply_layer",
            "armor_get_device_status",
            "armor_status_string", "armor_launch_count", "armor_gemm_timing_enable", "armor_gemm_timing",
            "armor_normalize_noalloc", "armor_block_product"]
@@ -72,6 +73,9 @@ def lib() -> C.CDLL:
         L.armor_packed_core_bytes.argtypes = [C.POINTER(armor_config), C.POINTER(C.c_size_t)]
         L.armor_pack_core.argtypes = [vp, vp, vp, vp, vp]
         L.armor_apply_packed.argtypes = [vp] + [vp] * 7 + [i64, vp]
+        L.armor_packed_layer_bytes.argtypes = [C.POINTER(armor_config), C.POINTER(C.c_size_t)]
+        L.armor_pack_layer.argtypes = [vp] + [vp] * 7 + [vp]
+        L.armor_apply_layer.argtypes = [vp, vp, vp, vp, i64, vp]
         L.armor_get_device_status.argtypes = [vp, C.POINTER(i32), i32]
         L.armor_status_string.argtypes = [C.c_int]
         L.armor_status_string.restype = C.c_char_p
@@ -201,6 +205,26 @@ def armor_apply_packed(ctx, A, B, packed, r1, r2, x, y) -> None:
     _check(lib().armor_apply_packed(ctx, _ptr(A, f, "A"), _ptr(B, f, "B"), _ptr(packed, torch.uint8, "packed"),
                                     _ptr(r1, f, "r1"), _ptr(r2, f, "r2"), _ptr(x, x.dtype, "x"), _ptr(y, y.dtype, "y"),
                                     x.shape[0], _stream()), "armor_apply_packed")
+
+
+def armor_packed_layer_bytes(cfg: armor_config) -> int:
+    n = C.c_size_t(0)
+    _check(lib().armor_packed_layer_bytes(C.byref(cfg), C.byref(n)), "armor_packed_layer_bytes")
+    return int(n.value)
+
+
+def armor_pack_layer(ctx, A, B, S, M, r1, r2, packed) -> None:
+    f = torch.float32
+    _check(lib().armor_pack_layer(ctx, _ptr(A, f, "A"), _ptr(B, f, "B"), _ptr(S, f, "S"), _ptr(M, torch.uint8, "M"),
+                                  _ptr(r1, f, "r1"), _ptr(r2, f, "r2"), _ptr(packed, torch.uint8, "packed"), _stream()),
+           "armor_pack_layer")
+
+
+def armor_apply_layer(ctx, packed, x, y) -> None:
+    if x.dtype != torch.bfloat16 or y.dtype != torch.bfloat16:
+        raise ValueError("the packed layer takes bf16 x and y")
+    _check(lib().armor_apply_layer(ctx, _ptr(packed, torch.uint8, "packed"), _ptr(x, x.dtype, "x"), _ptr(y, y.dtype, "y"),
+                                   x.shape[0], _stream()), "armor_apply_layer")
 
 
 def armor_get_device_status(ctx, n: int = 8) -> list[int]:
@@ -336,6 +360,18 @@ class ArmorContext:
         y = torch.empty(x.shape[0], self.d_out, dtype=x.dtype, device=self.device)
         r1, r2 = (st.r1, st.r2) if denormalize else (None, None)
         armor_apply_packed(self.ctx, st.A, st.B, packed, r1, r2, x, y)
+        return y
+
+    def pack_layer(self, st: LayerState, denormalize: bool = False) -> torch.Tensor:
+        """Core and wrappers packed for the all-bf16 forward (the normalisation's scales folded into the wrappers)."""
+        packed = torch.empty(armor_packed_layer_bytes(self.cfg), dtype=torch.uint8, device=self.device)
+        r1, r2 = (st.r1, st.r2) if denormalize else (None, None)
+        armor_pack_layer(self.ctx, st.A, st.B, st.S, st.M, r1, r2, packed)
+        return packed
+
+    def apply_layer(self, packed: torch.Tensor, x: torch.Tensor) -> torch.Tensor:
+        y = torch.empty(x.shape[0], self.d_out, dtype=x.dtype, device=self.device)
+        armor_apply_layer(self.ctx, packed, x, y)
         return y
 
     def device_status(self) -> list[int]:

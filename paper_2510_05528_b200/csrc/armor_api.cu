@@ -638,4 +638,57 @@ armor_status armor_apply_packed(armor_ctx* c, const float* A, const float* B, co
   return apply_impl(c, A, B, nullptr, d_packed, r1, r2, d_x, d_y, true, n_tokens, cs(stream));
 }
 
+// ---- the whole layer packed for the bf16 forward: core values, core positions, B blocks, A blocks -------------
+static size_t layer_off_B(const armor_ctx* c) { return (size_t)c->wn + (size_t)c->wn / 8; }
+static size_t layer_off_A(const armor_ctx* c) { return layer_off_B(c) + (size_t)c->nbi * c->db * c->db * 2; }
+
+armor_status armor_packed_layer_bytes(const armor_config* cfg, size_t* out_bytes) {
+  if (!cfg || !out_bytes) return ARMOR_ERR_INVALID_ARG;
+  armor_status st = check_config(cfg);
+  if (st != ARMOR_OK) return st;
+  if (cfg->n_keep != 2 || cfg->m_group != 4 || cfg->d_out % 128 || cfg->d_in % 128 || cfg->d_block % 128)
+    return ARMOR_ERR_UNSUPPORTED;
+  const size_t wn = (size_t)cfg->d_out * (size_t)cfg->d_in;
+  *out_bytes = wn + wn / 8 + ((size_t)cfg->d_out + (size_t)cfg->d_in) * (size_t)cfg->d_block * 2;
+  return ARMOR_OK;
+}
+
+armor_status armor_pack_layer(armor_ctx* c, const float* A, const float* B, const float* S, const uint8_t* M,
+                              const float* r1, const float* r2, void* d_packed, armor_stream_t stream) {
+  if (!c || !A || !B || !S || !M || !d_packed) return ARMOR_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(d_packed) % 128 || (r1 == nullptr) != (r2 == nullptr)) return ARMOR_ERR_INVALID_ARG;
+  if (!tc_sparse_ok(c) || !fwd_block_ok(c)) return ARMOR_ERR_UNSUPPORTED;
+  cudaStream_t s = cs(stream);
+  char* buf = static_cast<char*>(d_packed);
+  launch_compress_24(c, S, M, buf, buf + tc_sparse_values_bytes(c), s);
+  launch_pack_blocks(c, B, nullptr, r1, buf + layer_off_B(c), c->nbi, s);   // B's columns carry r1
+  launch_pack_blocks(c, A, r2, nullptr, buf + layer_off_A(c), c->nbo, s);   // A's rows carry r2
+  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+}
+
+armor_status armor_apply_layer(armor_ctx* c, const void* d_packed, const void* d_x, void* d_y, int64_t n_tokens,
+                               armor_stream_t stream) {
+  if (!c || !d_packed || n_tokens < 0) return ARMOR_ERR_INVALID_ARG;
+  if (n_tokens == 0) return ARMOR_OK;
+  if (!d_x || !d_y || reinterpret_cast<uintptr_t>(d_packed) % 128) return ARMOR_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(d_x) % 16 || reinterpret_cast<uintptr_t>(d_y) % 16) return ARMOR_ERR_INVALID_ARG;
+  if (!tc_sparse_ok(c) || !fwd_block_ok(c)) return ARMOR_ERR_UNSUPPORTED;
+  cudaStream_t s = cs(stream);
+  const char* buf = static_cast<const char*>(d_packed);
+  const int64_t d_out = c->d_out, d_in = c->d_in;
+  const int64_t chunk = d_out < d_in ? d_out : d_in;   // bf16 z1 [chunk, d_in] and z2 [chunk, d_out] fit W-shaped scratch
+  for (int64_t t0 = 0; t0 < n_tokens; t0 += chunk) {
+    const int64_t n = (n_tokens - t0 < chunk) ? n_tokens - t0 : chunk;
+    const char* xc = static_cast<const char*>(d_x) + (size_t)(t0 * d_in) * 2;
+    char* yc = static_cast<char*>(d_y) + (size_t)(t0 * d_out) * 2;
+    armor_status st = launch_fwd_block(c, xc, buf + layer_off_B(c), c->T, n, d_in, s);        // z1 = (r1 . x) B^T
+    if (st != ARMOR_OK) return st;
+    st = launch_tc_sparse(c, buf, buf + tc_sparse_values_bytes(c), c->T, c->E, true, n, s);   // z2 = z1 S^T
+    if (st != ARMOR_OK) return st;
+    st = launch_fwd_block(c, c->E, buf + layer_off_A(c), yc, n, d_out, s);                    // y = r2 . (z2 A^T)
+    if (st != ARMOR_OK) return st;
+  }
+  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+}
+
 }  // extern "C"

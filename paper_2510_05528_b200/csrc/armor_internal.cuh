@@ -243,5 +243,11 @@ bool tc_gemm_shape_ok(int64_t M, int64_t N, int64_t K);
 bool tc_sparse_ok(const armor_ctx* c);
 size_t tc_sparse_values_bytes(const armor_ctx* c);
 void launch_compress_24(armor_ctx* c, const float* S, const uint8_t* M, void* Sc, void* E, cudaStream_t s);
-armor_status launch_tc_sparse(armor_ctx* c, const void* Sc, const void* E, const void* z1_bf16, float* z2, int64_t n,
+armor_status launch_tc_sparse(armor_ctx* c, const void* Sc, const void* E, const void* z1_bf16, void* z2, bool out_bf16,
+                              int64_t n, cudaStream_t s);
+// the wrapper products of the bf16 forward (fwd_tcgen05.cu)
+bool fwd_block_ok(const armor_ctx* c);
+void launch_pack_blocks(armor_ctx* c, const float* P, const float* rowscale, const float* colscale, void* Q, int nb,
+                        cudaStream_t s);
+armor_status launch_fwd_block(armor_ctx* c, const void* X, const void* Q, void* out, int64_t rows, int64_t d,
                               cudaStream_t s);

@@ -109,7 +109,7 @@ armor_status apply_core(armor_ctx* c, const float* z1, const float* S, const voi
     if (!bf16 || !tc_sparse_ok(c)) return ARMOR_ERR_UNSUPPORTED;
     const char* buf = static_cast<const char*>(packed);
     launch_f32_to_bf16(c, z1, nullptr, c->U, n, d_in, s);
-    return launch_tc_sparse(c, buf, buf + tc_sparse_values_bytes(c), c->U, z2, n, s);
+    return launch_tc_sparse(c, buf, buf + tc_sparse_values_bytes(c), c->U, z2, false, n, s);
   }
   if (bf16 && c->cfg.precision != ARMOR_PREC_SIMT && d_out % 32 == 0 && d_in % 8 == 0) {
     // bf16 deployment: the core and the wrapped activations are rounded to bf16 and multiplied on the bf16

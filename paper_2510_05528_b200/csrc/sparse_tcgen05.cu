@@ -41,6 +41,7 @@ constexpr int STAGE_BYTES = A_BYTES + 2 * BH_BYTES + E_BYTES; // 50 KiB
 
 struct SParams {
   float* Z; int64_t ldz;        // [N tokens][ldz], written transposed
+  __nv_bfloat16* Zb;            // non-null: the output is written as bf16 here instead
   int64_t M, N, K;              // rows of S, tokens, logical k
   int m_tiles, n_tiles, k_tiles;
   int32_t* status;
@@ -224,7 +225,10 @@ tc_sparse_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         if (row < p.M) {
 #pragma unroll
           for (int cidx = 0; cidx < 32; ++cidx)
-            if (tok0 + cidx < p.N) p.Z[(tok0 + cidx) * p.ldz + row] = __uint_as_float(r[cidx]);
+            if (tok0 + cidx < p.N) {
+              if (p.Zb) p.Zb[(tok0 + cidx) * p.ldz + row] = __float2bfloat16(__uint_as_float(r[cidx]));
+              else p.Z[(tok0 + cidx) * p.ldz + row] = __uint_as_float(r[cidx]);
+            }
         }
       }
       tc_fence_before();
@@ -424,7 +428,10 @@ tc_sparse_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
         if (row < p.M) {
 #pragma unroll
           for (int cidx = 0; cidx < 32; ++cidx)
-            if (tok0 + cidx < p.N) p.Z[(tok0 + cidx) * p.ldz + row] = __uint_as_float(r[cidx]);
+            if (tok0 + cidx < p.N) {
+              if (p.Zb) p.Zb[(tok0 + cidx) * p.ldz + row] = __float2bfloat16(__uint_as_float(r[cidx]));
+              else p.Z[(tok0 + cidx) * p.ldz + row] = __uint_as_float(r[cidx]);
+            }
         }
       }
       tc_fence_before();
@@ -536,16 +543,17 @@ void launch_compress_24(armor_ctx* c, const float* S, const uint8_t* M, void* Sc
   c->launches++;
 }
 
-// Z2[n][d_out] = Z1[n][d_in] * S^T with S given compressed (Sc, E); Z1 bf16.
-armor_status launch_tc_sparse(armor_ctx* c, const void* Sc, const void* E, const void* z1_bf16, float* z2, int64_t n,
-                              cudaStream_t s) {
+// Z2[n][d_out] = Z1[n][d_in] * S^T with S given compressed (Sc, E); Z1 bf16; Z2 fp32, or bf16 if out_bf16.
+armor_status launch_tc_sparse(armor_ctx* c, const void* Sc, const void* E, const void* z1_bf16, void* z2, bool out_bf16,
+                              int64_t n, cudaStream_t s) {
   if (!tc_sparse_ok(c) || n <= 0) return ARMOR_ERR_UNSUPPORTED;
   CUtensorMap mA, mB, mE;
   if (!make_map_bf16(&mA, Sc, c->d_out, c->d_in / 2, c->d_in / 2)) return ARMOR_ERR_CUDA;
   if (!make_map_bf16(&mB, z1_bf16, n, c->d_in, c->d_in)) return ARMOR_ERR_CUDA;
   if (!make_map_e(&mE, E, (c->d_out / 128) * (c->d_in / 128) * 128)) return ARMOR_ERR_CUDA;
   SParams p{};
-  p.Z = z2; p.ldz = c->d_out; p.M = c->d_out; p.N = n; p.K = c->d_in;
+  p.Z = out_bf16 ? nullptr : static_cast<float*>(z2); p.Zb = out_bf16 ? static_cast<__nv_bfloat16*>(z2) : nullptr;
+  p.ldz = c->d_out; p.M = c->d_out; p.N = n; p.K = c->d_in;
   p.m_tiles = (int)(c->d_out / BM); p.n_tiles = (int)((n + BN - 1) / BN); p.k_tiles = (int)(c->d_in / BKL);
   p.status = c->status;
   constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024;

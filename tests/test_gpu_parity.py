@@ -584,6 +584,9 @@ def test_sparse_tensor_core_forward_is_exact_on_integers(d_out, d_in):
         exact = torch.from_numpy(x.astype(np.float64) @ S.T).to(torch.bfloat16)
         assert y.dtype == torch.bfloat16 and torch.equal(y.cpu(), exact), n_tok
         assert torch.equal(ctx.apply(st, xb).cpu(), exact)            # the dense bf16 path on the same input
+        if n_tok == 300:                                              # the all-bf16 packed layer: exact as well
+            layer = ctx.pack_layer(st)
+            assert torch.equal(ctx.apply_layer(layer, xb).cpu(), exact)
     assert ctx.device_status()[:5] == [0, 0, 0, 0, 0]
 
 
@@ -608,6 +611,11 @@ def test_sparse_tensor_core_forward_against_the_oracle(mid_data):
         packed = ctx.pack_core(st)
         assert packed.numel() == MID.d_out * MID.d_in * 9 // 8
         assert torch.equal(ctx.apply_packed(st, packed, xb, denormalize=den), y)
+        # the whole layer packed, wrappers in bf16 with the scales folded in: two more roundings (B, A) and
+        # bf16 z2 instead of fp32; about sqrt(7) x 2^-9 / sqrt(3) = 3e-3 expected
+        layer = ctx.pack_layer(st, denormalize=den)
+        yl = ctx.apply_layer(layer, xb)
+        assert yl.dtype == torch.bfloat16 and rel(yl.float().cpu().numpy(), yo) < 8e-3
     with pytest.raises(ValueError):
         ctx.apply(st, xb.float(), sparse=True)
     ctx48 = make(MID, Bd.PREC_FP32X3, n_keep=4, m_group=8)
