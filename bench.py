@@ -369,6 +369,9 @@ def run_ours(args, cfg):
             packed = cf.pack_core(sf)
             variants += [("bf16_sparse_core_packed_once", lambda: cf.apply_packed(sf, packed, xb)),
                          ("bf16_sparse_core_packed_per_call", lambda: cf.apply(sf, xb, sparse=True))]
+            if lcfg.d_block % 128 == 0:
+                layer = cf.pack_layer(sf)
+                variants += [("bf16_packed_layer", lambda: cf.apply_layer(layer, xb))]
         for name, fn in variants:
             for _ in range(3):
                 yv = fn()

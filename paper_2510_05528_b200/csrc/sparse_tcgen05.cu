@@ -108,6 +108,33 @@ __device__ __forceinline__ void tmem_cp_e_pair(uint32_t taddr, uint64_t sdesc) {
   asm volatile("tcgen05.cp.cta_group::2.128x128b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
 }
 
+// Epilogue store of 32 tokens of one row of S per lane (the output is [token][row], so a warp's 32 rows are
+// contiguous for every token).  bf16: neighbouring lanes swap one value per pair of tokens so that every lane
+// stores two adjacent rows (4 bytes) of one token -- as many store instructions per element as in fp32.
+__device__ __forceinline__ void store_chunk(const SParams& p, const uint32_t (&r)[32], int64_t row, int64_t tok0, int lane) {
+  if (p.Zb == nullptr) {
+    if (row < p.M) {
+#pragma unroll
+      for (int cidx = 0; cidx < 32; ++cidx)
+        if (tok0 + cidx < p.N) p.Z[(tok0 + cidx) * p.ldz + row] = __uint_as_float(r[cidx]);
+    }
+    return;
+  }
+  const bool odd = lane & 1;
+  const int64_t row2 = row - (odd ? 1 : 0);                  // the even row of the lane pair (p.M is even)
+#pragma unroll
+  for (int cidx = 0; cidx < 32; cidx += 2) {
+    const uint32_t give = odd ? r[cidx] : r[cidx + 1];
+    const uint32_t got = __shfl_xor_sync(0xffffffffu, give, 1);
+    const float lo = __uint_as_float(odd ? got : r[cidx]), hi = __uint_as_float(odd ? r[cidx + 1] : got);
+    const int64_t tok = tok0 + cidx + (odd ? 1 : 0);
+    if (row2 < p.M && tok < p.N) {
+      const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+      *reinterpret_cast<__nv_bfloat162*>(p.Zb + tok * p.ldz + row2) = v;
+    }
+  }
+}
+
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_sparse_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                  const __grid_constant__ CUtensorMap mapE, const SParams p) {
@@ -222,14 +249,7 @@ tc_sparse_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         uint32_t r[32];
         tmem_ld32(tmem_base + (uint32_t)(as * BN + ch * 32) + ((uint32_t)(q * 32) << 16), r);
         const int64_t tok0 = (int64_t)nt * BN + ch * 32;
-        if (row < p.M) {
-#pragma unroll
-          for (int cidx = 0; cidx < 32; ++cidx)
-            if (tok0 + cidx < p.N) {
-              if (p.Zb) p.Zb[(tok0 + cidx) * p.ldz + row] = __float2bfloat16(__uint_as_float(r[cidx]));
-              else p.Z[(tok0 + cidx) * p.ldz + row] = __uint_as_float(r[cidx]);
-            }
-        }
+        store_chunk(p, r, row, tok0, lane);
       }
       tc_fence_before();
       __syncwarp();
@@ -425,14 +445,7 @@ tc_sparse_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
         uint32_t r[32];
         tmem_ld32(tmem_base + (uint32_t)(ch * 32) + ((uint32_t)(q * 32) << 16), r);
         const int64_t tok0 = (int64_t)nt * BN2 + ch * 32;
-        if (row < p.M) {
-#pragma unroll
-          for (int cidx = 0; cidx < 32; ++cidx)
-            if (tok0 + cidx < p.N) {
-              if (p.Zb) p.Zb[(tok0 + cidx) * p.ldz + row] = __float2bfloat16(__uint_as_float(r[cidx]));
-              else p.Z[(tok0 + cidx) * p.ldz + row] = __uint_as_float(r[cidx]);
-            }
-        }
+        store_chunk(p, r, row, tok0, lane);
       }
       tc_fence_before();
       __syncwarp();
