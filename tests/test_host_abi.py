@@ -67,6 +67,26 @@ def test_config_validation(lib):
     assert lib.armor_workspace_bytes(C.byref(ok), None) == 1
 
 
+def test_packed_sizes_and_their_limits(lib):
+    """Sizes of the packed core and of the packed layer: kept values (half the entries, bf16), positions (4 bits
+    per group of four), and for the layer the bf16 blocks of both wrappers; only 2:4 with 128-aligned shapes."""
+    cfg = Bd.make_config(512, 768, 128)
+    wn = 512 * 768
+    assert Bd.armor_packed_core_bytes(cfg) == wn + wn // 8
+    assert Bd.armor_packed_layer_bytes(cfg) == wn + wn // 8 + (512 + 768) * 128 * 2
+    n = C.c_size_t(0)
+    for bad in (Bd.make_config(512, 768, 128, n_keep=4, m_group=8),     # the sparse tensor cores take 2:4 only
+                Bd.make_config(512, 704, 64)):                          # d_in not a multiple of 128
+        assert lib.armor_packed_core_bytes(C.byref(bad), C.byref(n)) == 7
+        assert lib.armor_packed_layer_bytes(C.byref(bad), C.byref(n)) == 7
+    small_blocks = Bd.make_config(512, 768, 64)                         # the core packs, the bf16 wrappers need d_block 128 / 256
+    assert lib.armor_packed_core_bytes(C.byref(small_blocks), C.byref(n)) == 0
+    assert lib.armor_packed_layer_bytes(C.byref(small_blocks), C.byref(n)) == 7
+    assert lib.armor_packed_layer_bytes(None, C.byref(n)) == 1
+    assert lib.armor_pack_core(None, None, None, None, None) == 1
+    assert lib.armor_apply_layer(None, None, None, None, 4, None) == 1
+
+
 def test_create_rejects_bad_workspace(lib):
     cfg = Bd.make_config(256, 256, 32)
     ctx = C.c_void_p(0)
