@@ -11,7 +11,7 @@
 // last paragraph) and the layer forward built from this kernel and the sparse core product.
 //
 // Kernel: persistent, 192 threads: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 epilogue (accumulator ->
-// bf16 -> shared-memory turn -> 128-byte row segments).  Four stages of 32 KiB, two accumulator buffers.  Every
+// bf16 -> shared-memory turn -> 128-byte row segments).  Six stages of 32 KiB, two accumulator buffers.  Every
 // wait is bounded.
 #include <cuda_bf16.h>
 
@@ -23,7 +23,7 @@ using namespace tc;
 
 constexpr int BM = 128, BN = 128, BKE = 64;         // BKE bf16 = 128 bytes = one swizzle row
 constexpr int NTHREADS = 192;
-constexpr int STAGES = 4;
+constexpr int STAGES = 6;
 constexpr uint32_t TMEM_COLS = 256;                 // two accumulator buffers of BN columns
 constexpr int A_BYTES = BM * BKE * 2;               // 16 KiB
 constexpr int B_BYTES = BN * BKE * 2;               // 16 KiB
