@@ -10,9 +10,10 @@
 // Also here: the packing of the wrappers for this kernel (bf16, the normalisation's scales folded in, Section 3.2
 // last paragraph) and the layer forward built from this kernel and the sparse core product.
 //
-// Kernel: persistent, 192 threads: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 epilogue (accumulator ->
-// bf16 -> shared-memory turn -> 128-byte row segments).  Six stages of 32 KiB, two accumulator buffers.  Every
-// wait is bounded.
+// Kernel: persistent, 320 threads: warp 0 TMA producer, warp 1 MMA issuer, warps 2-9 epilogue (accumulator ->
+// bf16 -> shared-memory turn -> 128-byte row segments; warps 2-5 take the left 64 columns of the tile, warps 6-9
+// the right 64: with four warps the epilogue, not HBM, set the pace).  Five stages of 32 KiB, two accumulator
+// buffers.  Every wait is bounded.
 #include <cuda_bf16.h>
 
 #include "tc_common.cuh"
@@ -22,8 +23,8 @@ namespace {
 using namespace tc;
 
 constexpr int BM = 128, BN = 128, BKE = 64;         // BKE bf16 = 128 bytes = one swizzle row
-constexpr int NTHREADS = 192;
-constexpr int STAGES = 6;
+constexpr int NTHREADS = 320;
+constexpr int STAGES = 5;
 constexpr uint32_t TMEM_COLS = 256;                 // two accumulator buffers of BN columns
 constexpr int A_BYTES = BM * BKE * 2;               // 16 KiB
 constexpr int B_BYTES = BN * BKE * 2;               // 16 KiB
@@ -78,7 +79,7 @@ fwd_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(tfull0 + 8 * s, 1); mbar_init(tempty0 + 8 * s, 4); }
+    for (int s = 0; s < 2; ++s) { mbar_init(tfull0 + 8 * s, 1); mbar_init(tempty0 + 8 * s, 8); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -150,8 +151,9 @@ fwd_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
     }
   } else {
     // ------------------------------------------------------------ epilogue warps
-    const int q = warp & 3;
-    uint32_t* tilebuf = reinterpret_cast<uint32_t*>(smem + (size_t)STAGES * STAGE_BYTES) + q * (32 * 33);
+    const int q = warp & 3;                 // tensor-memory lane quarter this warp may read
+    const int half = (warp - 2) >> 2;       // which 64 columns of the tile
+    uint32_t* tilebuf = reinterpret_cast<uint32_t*>(smem + (size_t)STAGES * STAGE_BYTES) + (warp - 2) * (32 * 33);
     int local = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < n_tiles_total && ok; tile += gridDim.x, ++local) {
@@ -161,8 +163,8 @@ fwd_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
       if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
       tc_fence_after();
       const int64_t row_base = (int64_t)mt * BM + q * 32;
-#pragma unroll 1
-      for (int ch = 0; ch < BN / 64; ++ch) {
+      {
+        const int ch = half;
         // 64 columns of the lane's row -> 32 words of two bf16; the 32 x 32 words are turned through shared
         // memory so that one store instruction writes 128 contiguous bytes of one row
         uint32_t r0[32], r1[32];
@@ -250,7 +252,7 @@ armor_status launch_fwd_block(armor_ctx* c, const void* X, const void* Q, void* 
   p.out = static_cast<__nv_bfloat16*>(out); p.ldo = d; p.rows = rows; p.d = d; p.db = c->db;
   p.m_tiles = (int)((rows + BM - 1) / BM); p.n_tiles = (int)(d / BN); p.k_tiles = c->db / BKE;
   p.status = c->status;
-  constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024 + 4 * 32 * 33 * sizeof(uint32_t);
+  constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024 + 8 * 32 * 33 * sizeof(uint32_t);
   static bool attr = false;
   if (!attr) {
     if (cudaFuncSetAttribute(fwd_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess)
