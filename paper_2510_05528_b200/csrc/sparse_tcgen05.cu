@@ -31,7 +31,6 @@ using namespace tc;
 
 constexpr int BM = 128, BN = 128, BKL = 128;        // BKL: logical k per stage (64 kept values = 128 bytes per row)
 constexpr int NTHREADS = 192;
-constexpr int NTHREADS_PAIR = 320;                  // the pair kernel drains its accumulator with eight warps
 constexpr int STAGES = 4;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t META_COL0 = 256;                 // accumulators: columns 0-127 and 128-255
@@ -274,8 +273,7 @@ tc_sparse_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
 //   full[s]   (even CTA): armed by the even CTA's producer for the bytes of both CTAs; both CTAs' TMA loads
 //             complete on it (cta_group::2 loads may signal the pair's other CTA)
 //   empty[s], tfull (both CTAs): tcgen05.commit multicast to the pair
-//   tempty    (even CTA): 16 arrivals, one per epilogue warp of either CTA (eight warps per CTA: warps 2-5 drain
-//             the left 128 columns, warps 6-9 the right 128; the epilogue is exposed, see below)
+//   tempty    (even CTA): 8 arrivals, one per epilogue warp of either CTA
 // The positions of both CTAs go from their shared to their tensor memory with one tcgen05.cp of the pair.
 // One accumulator buffer of 256 columns (the positions need tensor-memory columns too).
 constexpr int BN2 = 256;
@@ -331,7 +329,7 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-__global__ void __launch_bounds__(NTHREADS_PAIR, 1)
+__global__ void __launch_bounds__(NTHREADS, 1)
 tc_sparse_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                       const __grid_constant__ CUtensorMap mapE, const SParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -355,7 +353,7 @@ tc_sparse_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
       mbar_init(empty0 + 8 * s, 1);
     }
     mbar_init(tfull, 1);
-    mbar_init(tempty, 16);
+    mbar_init(tempty, 8);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -443,7 +441,7 @@ tc_sparse_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_con
       tc_fence_after();
       const int64_t row = (int64_t)mt * 256 + rank * 128 + q * 32 + lane;
 #pragma unroll 1
-      for (int ch = 4 * ((warp - 2) >> 2); ch < 4 * ((warp - 2) >> 2) + 4; ++ch) {
+      for (int ch = 0; ch < BN2 / 32; ++ch) {
         uint32_t r[32];
         tmem_ld32(tmem_base + (uint32_t)(ch * 32) + ((uint32_t)(q * 32) << 16), r);
         const int64_t tok0 = (int64_t)nt * BN2 + ch * 32;
@@ -598,7 +596,7 @@ armor_status launch_tc_sparse(armor_ctx* c, const void* Sc, const void* E, const
     int pairs = n_sm / 2;
     if (tiles < pairs) pairs = tiles;
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(NTHREADS_PAIR); cfg.dynamicSmemBytes = SMEM; cfg.stream = s;
+    cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(NTHREADS); cfg.dynamicSmemBytes = SMEM; cfg.stream = s;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
