@@ -625,6 +625,26 @@ def test_sparse_tensor_core_forward_against_the_oracle(mid_data):
     assert ctx.device_status()[:5] == [0, 0, 0, 0, 0]
 
 
+def test_packed_layer_forward_with_d_block_256():
+    """The all-bf16 forward with 256 x 256 wrapper blocks (four k-tiles per block, two column tiles per block) and a
+    ragged token count, after two BCD iterations with the normalisation on: against the oracle's forward."""
+    W = inputs.make_weight(BIG_BLOCK)
+    X = inputs.make_activations(BIG_BLOCK)
+    H32 = O.gram(X).astype(np.float32)
+    ctx = make(BIG_BLOCK, Bd.PREC_FP32X3, normalize=1)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    ctx.bcd_step(st, Hd, 0, 2, want_stats=False)
+    xb = dev(inputs.make_tokens(BIG_BLOCK, 1000)).to(torch.bfloat16)     # two chunks of 512 tokens, the second ragged
+    A, B, S = (host(t).astype(np.float64) for t in (st.A, st.B, st.S))
+    r1, r2 = host(st.r1).astype(np.float64), host(st.r2).astype(np.float64)
+    yo = O.apply(A, B, S, xb.float().cpu().numpy(), r1, r2)
+    y = ctx.apply_layer(ctx.pack_layer(st, denormalize=True), xb)
+    assert y.shape == (1000, BIG_BLOCK.d_out) and rel(y.float().cpu().numpy(), yo) < 8e-3
+    assert rel(ctx.apply(st, xb, denormalize=True, sparse=True).float().cpu().numpy(), yo) < 5e-3
+    assert ctx.device_status()[:5] == [0, 0, 0, 0, 0]
+
+
 # ------------------------------------------------------------------------------------------ block products
 @pytest.mark.parametrize("db", [128, 256])
 @pytest.mark.parametrize("side,transpose", [(0, False), (0, True), (1, False), (1, True)])
