@@ -127,3 +127,42 @@ def test_full_iterations_properties(layer):
     assert stats["chol_failed"].sum() == 0
     assert all(0 <= g <= (CFG.d_out // CFG.d_block) * (CFG.d_in // CFG.d_block) for g in stats["groups_changed"])
     assert ctx.device_status()[:4] == [0, 0, 0, 0]
+
+
+def test_forward_at_full_size_on_sampled_outputs(layer):
+    """The deployment form at 4096 x 4096 with the token count bench.py applies (8192, two chunks), after three
+    iterations: sampled outputs y[t, r] = A[r-th row] (S (B x_t)) computed one by one in fp64 against the fp32
+    path, the bf16 path with the dense core, the packed 2:4 core on the sparse tensor cores and the all-bf16
+    packed layer."""
+    ctx, W, H = layer
+    st = ctx.init(dev(W), H)
+    ctx.bcd_step(st, H, 0, 3, want_stats=False)
+    x = inputs.make_tokens(CFG, 8192)
+    xd = dev(x)
+    xb = xd.to(torch.bfloat16)
+    A, B, S = (host(t).astype(np.float64) for t in (st.A, st.B, st.S))
+    db = CFG.d_block
+    rng = np.random.default_rng(3)
+    toks = rng.choice(8192, 12, replace=False)
+    rows = rng.choice(CFG.d_out, 12, replace=False)
+
+    def sampled(xs):
+        out = np.zeros((len(toks), len(rows)))
+        for a, t in enumerate(toks):
+            z1 = np.concatenate([B[j] @ xs[t, j * db:(j + 1) * db] for j in range(CFG.d_in // db)])
+            z2 = S @ z1
+            for b, r in enumerate(rows):
+                i, m = divmod(int(r), db)
+                out[a, b] = A[i][m] @ z2[i * db:(i + 1) * db]
+        return out
+    ref32 = sampled(x.astype(np.float64))
+    refbf = sampled(xb.float().cpu().numpy().astype(np.float64))
+    scale = np.sqrt(np.mean(ref32 ** 2))
+    pick = lambda y: y.float().cpu().numpy()[np.ix_(toks, rows)]
+    assert np.abs(pick(ctx.apply(st, xd)) - ref32).max() < 1e-4 * scale
+    packed, whole = ctx.pack_core(st), ctx.pack_layer(st)
+    for name, y, tol in (("dense bf16 core", ctx.apply(st, xb), 2e-2), ("sparse core", ctx.apply_packed(st, packed, xb), 2e-2),
+                         ("packed layer", ctx.apply_layer(whole, xb), 3e-2)):
+        assert y.shape == (8192, CFG.d_out) and y.dtype == torch.bfloat16
+        assert np.abs(pick(y) - refbf).max() < tol * scale, name     # a few bf16 roundings on single entries
+    assert ctx.device_status()[:5] == [0, 0, 0, 0, 0]
