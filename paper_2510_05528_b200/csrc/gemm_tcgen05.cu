@@ -79,14 +79,19 @@ __device__ __forceinline__ void tile_coords(const Params& p, int tile, int& mt, 
     nt = r / gm;
     return;
   }
-  // only tiles that hold an element with column <= row: m tile >= 2 * n tile
+  // only tiles that hold an element with column <= row: m tile >= 2 * n tile.  Same grouping: bands of GROUP_M
+  // m tiles, inside a band the n tile is the outer index and m runs fastest
   int rem = tile;
-  for (nt = 0; nt < p.n_tiles; ++nt) {
-    const int cnt = p.m_tiles - 2 * nt;
-    if (rem < cnt) break;
-    rem -= cnt;
+  for (int m0 = 0; m0 < p.m_tiles; m0 += GROUP_M) {
+    const int m1 = min(m0 + GROUP_M, p.m_tiles);
+    for (nt = 0; 2 * nt < m1 && nt < p.n_tiles; ++nt) {
+      const int lo = max(m0, 2 * nt);
+      const int cnt = m1 - lo;
+      if (rem < cnt) { mt = lo + rem; return; }
+      rem -= cnt;
+    }
   }
-  mt = 2 * nt + rem;
+  mt = 0; nt = 0;   // not reached: tile < number of tiles
 }
 
 // work item -> tile, and its range of k-tiles
