@@ -36,7 +36,7 @@ TF32_OVER_BF16 = 1.1 / 2.25
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes (read + write) of one dense 4096^3 launch of the tensor-core GEMM in FP32X3 mode, from the ncu
 # capture summarised in profiles/ncu_tc_gemm_4096x4096x4096_fp32x3.md (read 759.5 MB + write 156.1 MB)
-GEMM_DRAM_TRAFFIC_BYTES = 914.0e6
+GEMM_DRAM_TRAFFIC_BYTES = 812.6e6
 
 
 def load_peaks():
