@@ -588,6 +588,19 @@ def test_sparse_tensor_core_forward_is_exact_on_integers(d_out, d_in):
             layer = ctx.pack_layer(st)
             assert torch.equal(ctx.apply_layer(layer, xb).cpu(), exact)
     assert ctx.device_status()[:5] == [0, 0, 0, 0, 0]
+    # a mask byte that keeps three of four positions cannot be packed as 2:4: the packing takes the first two kept
+    # positions and counts the group in status word 4; a byte that keeps one position is padded with a zero
+    st.M[3, 5] = 0b0111
+    st.M[4, 6] = 0b0100
+    bad = ctx.pack_core(st)
+    assert ctx.device_status()[4] == 1
+    yb = ctx.apply_packed(st, bad, xb).float().cpu().numpy()
+    S2 = S.copy()
+    S2[3, 20:24] = S2[3, 20:24] * np.array([1.0, 1.0, 0.0, 0.0])   # group (3, 5): the first two kept positions survive
+    keep1 = np.zeros(4, dtype=bool); keep1[2] = True
+    S2[4, 24:28] = S2[4, 24:28] * keep1                       # group (4, 6): only position 2 survives
+    exact2 = torch.from_numpy(x.astype(np.float64) @ S2.T).to(torch.bfloat16).float().numpy()
+    assert np.array_equal(yb, exact2)
 
 
 def test_sparse_tensor_core_forward_against_the_oracle(mid_data):
@@ -641,6 +654,9 @@ def test_packed_layer_forward_with_d_block_256():
     yo = O.apply(A, B, S, xb.float().cpu().numpy(), r1, r2)
     y = ctx.apply_layer(ctx.pack_layer(st, denormalize=True), xb)
     assert y.shape == (1000, BIG_BLOCK.d_out) and rel(y.float().cpu().numpy(), yo) < 8e-3
+    layer = ctx.pack_layer(st, denormalize=True)
+    assert ctx.apply_layer(layer, xb[:0]).shape == (0, BIG_BLOCK.d_out)            # no tokens: nothing is launched
+    assert ctx.apply_packed(st, ctx.pack_core(st), xb[:0]).shape == (0, BIG_BLOCK.d_out)
     assert rel(ctx.apply(st, xb, denormalize=True, sparse=True).float().cpu().numpy(), yo) < 5e-3
     assert ctx.device_status()[:5] == [0, 0, 0, 0, 0]
 
