@@ -59,6 +59,7 @@ class OracleConfig:
     seed: int = 0
     phases: int = PH_ALL
     mask_sweeps: int = 1         # sparse-core updates (Algorithm 3) per continuous update; the paper runs 1
+    mask_groups: int = 1         # groups drawn per block in one sparse-core update; the paper draws 1
 
 
 @dataclass
@@ -77,6 +78,7 @@ class IterInfo:
     mask_margin: np.ndarray | None = None          # [nbo, nbi] relative margin of the mask sweep
     new_mask: np.ndarray | None = None             # [nbo, nbi] chosen mask byte
     sweeps: list = field(default_factory=list)     # one IterInfo per sparse-core update of the iteration
+    selected_all: np.ndarray | None = None         # [nbo, nbi, mask_groups] every group drawn, -1 where none
 
 
 # --------------------------------------------------------------------------
@@ -432,8 +434,14 @@ def mask_step(W, A, B, S, M, Hw, cfg: OracleConfig, t: int, info: IterInfo | Non
     Reading (full H_w): simultaneous updates in different column-blocks of one
     row-block interact, so all updates of the iteration are accepted only if
     the exact change of the loss, -2<E H_w, V> + tr(V H_w V^T) with
-    V = A dS B, is <= 0, and discarded together otherwise."""
+    V = A dS B, is <= 0, and discarded together otherwise.
+    Reading (mask_groups = k > 1, not in the paper): the k groups with the smallest race keys are drawn in every
+    block -- the exponential race then samples k groups without replacement with probability proportional to
+    the score -- and each is re-solved on its own from the state before the update, exactly as a single group
+    would be.  Groups of one block interact (they share columns of A or rows of B), so the test on the exact
+    joint change of the loss above applies with either weighting."""
     db, n, m = cfg.d_block, cfg.n_keep, cfg.m_group
+    kg = cfg.mask_groups
     d_out, d_in = S.shape
     nbo, nbi = d_out // db, d_in // db
     ng_row = d_in // m                      # groups per row
@@ -460,60 +468,71 @@ def mask_step(W, A, B, S, M, Hw, cfg: OracleConfig, t: int, info: IterInfo | Non
     dS = np.zeros_like(S)
     newM = M.copy()
     selected = -np.ones((nbo, nbi), dtype=np.int64)
+    selected_all = -np.ones((nbo, nbi, kg), dtype=np.int64)
     sel_margin = np.full((nbo, nbi), np.inf)
     msk_margin = np.full((nbo, nbi), np.inf)
     new_mask = np.zeros((nbo, nbi), dtype=np.int64)
+    def _solve_group(i, j, kk, p):
+        r = i * db + p // gpb
+        c = j * gpb + p % gpb           # group column index within the row
+        if kk == 0:
+            selected[i, j] = r * ng_row + c
+        selected_all[i, j, kk] = r * ng_row + c
+        cols = np.arange(m * c, m * c + m)
+        lc = m * (p % gpb)              # group's first row inside B_j
+        Kc = Kfull[j][lc:lc + m, lc:lc + m]
+        a_r = alpha[r]
+        s_g = S[r, cols]
+        z = Gamma[r, cols] + a_r * (Kc @ s_g)
+        inc = tuple(np.nonzero(M[r, cols])[0])
+        order = [inc] + [cb for cb in combos if cb != inc]
+        best = None
+        reds = []
+        for cb in order:
+            ix = np.array(cb)
+            sol = pinv_solve(Kc[np.ix_(ix, ix)], z[ix])
+            if sol is None:
+                continue
+            w, red = sol
+            red /= a_r
+            reds.append(red)
+            if best is None or red > best[0]:
+                best = (red, cb, w / a_r)
+        if best is None:
+            return
+        if len(reds) > 1:
+            rs = np.sort(np.array(reds))[::-1]
+            msk_margin[i, j] = min(msk_margin[i, j], (rs[0] - rs[1]) / max(abs(rs[0]), 1e-300))
+        red, cb, w = best
+        new_g = np.zeros(m)
+        new_g[list(cb)] = w
+        dS[r, cols] = new_g - s_g
+        newM[r, cols] = False
+        newM[r, m * c + np.array(cb)] = True
+        if kk == 0:
+            new_mask[i, j] = sum(1 << q for q in cb)
+
     for i in range(nbo):
         for j in range(nbi):
             kb = key[i * db:(i + 1) * db, j * gpb:(j + 1) * gpb]
             flat = kb.reshape(-1)           # row-major == ascending global group index
-            p = int(np.argmin(flat))        # first minimum: ties -> lowest g
-            if not np.isfinite(flat[p]):
+            picks = [int(q) for q in np.argsort(flat, kind="stable")[:kg] if np.isfinite(flat[q])]   # ties -> lowest g
+            if not picks:
                 continue
-            if flat.size > 1:
-                second = np.partition(flat, 1)[1]
-                if np.isfinite(second):
-                    sel_margin[i, j] = abs(second - flat[p]) / max(abs(second), 1e-300)
-            r = i * db + p // gpb
-            c = j * gpb + p % gpb           # group column index within the row
-            selected[i, j] = r * ng_row + c
-            cols = np.arange(m * c, m * c + m)
-            lc = m * (p % gpb)              # group's first row inside B_j
-            Kc = Kfull[j][lc:lc + m, lc:lc + m]
-            a_r = alpha[r]
-            s_g = S[r, cols]
-            z = Gamma[r, cols] + a_r * (Kc @ s_g)
-            inc = tuple(np.nonzero(M[r, cols])[0])
-            order = [inc] + [cb for cb in combos if cb != inc]
-            best = None
-            reds = []
-            for cb in order:
-                ix = np.array(cb)
-                sol = pinv_solve(Kc[np.ix_(ix, ix)], z[ix])
-                if sol is None:
-                    continue
-                w, red = sol
-                red /= a_r
-                reds.append(red)
-                if best is None or red > best[0]:
-                    best = (red, cb, w / a_r)
-            if best is None:
-                continue
-            if len(reds) > 1:
-                rs = np.sort(np.array(reds))[::-1]
-                msk_margin[i, j] = (rs[0] - rs[1]) / max(abs(rs[0]), 1e-300)
-            red, cb, w = best
-            new_g = np.zeros(m)
-            new_g[list(cb)] = w
-            dS[r, cols] = new_g - s_g
-            newM[r, cols] = False
-            newM[r, m * c + np.array(cb)] = True
-            new_mask[i, j] = sum(1 << q for q in cb)
+            if flat.size > len(picks) and len(picks) == kg:
+                # how close the draw was: the gap between the last key taken and the first one left out
+                srt = np.sort(flat)
+                last_in, first_out = srt[kg - 1], srt[kg]
+                if np.isfinite(first_out):
+                    sel_margin[i, j] = abs(first_out - last_in) / max(abs(first_out), 1e-300)
+            for kk, p in enumerate(picks):
+                _solve_group(i, j, kk, p)
     V = bd_right(bd_left(A, dS), B)
     dL = float(-2.0 * np.sum(EH * V) + np.sum((V @ Hw) * V))
     accepted = dL <= 0.0
     if info is not None:
         info.selected, info.select_margin = selected, sel_margin
+        info.selected_all = selected_all
         info.mask_margin, info.new_mask = msk_margin, new_mask
         info.delta_L_mask = dL
         info.mask_accepted = int(accepted)

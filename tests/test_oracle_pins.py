@@ -680,6 +680,77 @@ def test_several_sparse_core_updates_per_iteration(h_mode):
     assert np.all(M1.reshape(32, -1, 4).sum(axis=2) == 2) and np.all(S1[~M1] == 0)
 
 
+@pytest.mark.parametrize("h_mode", [O.FULL, O.DIAG])
+def test_several_groups_per_block_in_one_update(h_mode):
+    """mask_groups = k: the k smallest race keys of every block are drawn and each group is solved on its own.
+    Pinned to the single-group step (which has its own pins) and to the loss evaluated from the activations:
+    the drawn groups are the k best keys of the block (brute force over the keys of a greedy selection, whose
+    keys are the negated scores); each group's new values are what that group gets when it
+    is fitted alone by least squares; the reported change of the loss is the true one; a rejected update changes
+    nothing."""
+    cfg, W, X = tiny(d_out=32, d_in=32, db=16, n=128)
+    H = O.gram(X)
+    Hw = O.weighting(H, h_mode)
+    Xw = X if h_mode == O.FULL else np.diag(np.sqrt(np.diag(H)))
+    k = 3
+    oc = O.OracleConfig(16, h_mode=h_mode, seed=9, mask_groups=k, select_mode=O.L1_GREEDY, phases=O.PH_MASK)
+    A, B, S, M = rand_state(W, H, oc, np.random.default_rng(8), scale=0.2)
+    info = O.IterInfo()
+    S1, M1 = O.mask_step(W, A, B, S, M, Hw, oc, 4, info)
+    Gamma = O.core_gradient(W, A, B, S, Hw)
+    score = np.abs(Gamma).reshape(32, 8, 4).sum(axis=2)                     # L1 norm of every group's gradient
+    for i in range(2):
+        for j in range(2):
+            blk = score[16 * i:16 * i + 16, 4 * j:4 * j + 4]
+            best = np.argsort(-blk.reshape(-1), kind="stable")[:k]
+            want = sorted(int((16 * i + q // 4) * 8 + 4 * j + q % 4) for q in best)
+            assert sorted(int(g) for g in info.selected_all[i, j]) == want
+            assert info.selected[i, j] == info.selected_all[i, j, 0]
+    L0, L1 = loss_from_X(W, A, B, S, Xw), loss_from_X(W, A, B, S1, Xw)
+    if info.mask_accepted:
+        assert np.isclose(L1 - L0, info.delta_L_mask, rtol=1e-7, atol=1e-9 * L0) and L1 <= L0 * (1 + 1e-12)
+        # every drawn group carries the values that a least-squares fit of that group alone gives on the full loss,
+        # the other groups at their old values: checked on the third pick of block (1, 0)
+        g = int(info.selected_all[1, 0, 2])
+        r, c = divmod(g, 8)
+        cols = slice(4 * c, 4 * c + 4)
+        # solve that group alone by least squares on the full loss with the other groups at their old values
+        Ad, Bd_ = O.bd_dense(A), O.bd_dense(B)
+        S0 = S.copy(); S0[r, cols] = 0.0
+        dW = (W - Ad @ S0 @ Bd_) @ (X.T if h_mode == O.FULL else np.diag(np.sqrt(np.diag(H))))
+        keep = np.nonzero(M1[r, cols])[0]
+        R = X.T if h_mode == O.FULL else np.diag(np.sqrt(np.diag(H)))
+        Dm = np.stack([(np.outer(Ad[:, r], Bd_[4 * c + p_]) @ R).reshape(-1) for p_ in keep], axis=1)
+        sol, *_ = np.linalg.lstsq(Dm, dW.reshape(-1), rcond=None)
+        assert np.allclose(S1[r, cols][keep], sol, rtol=1e-6, atol=1e-10)
+    else:
+        assert np.array_equal(S1, S) and np.array_equal(M1, M)
+    assert np.all(M1.reshape(32, -1, 4).sum(axis=2) == 2) and np.all(S1[~M1] == 0.0)
+    # k = 1 is the plain step
+    a = O.mask_step(W, A, B, S, M, Hw, O.OracleConfig(16, h_mode=h_mode, seed=9, mask_groups=1, phases=O.PH_MASK), 4)
+    b = O.mask_step(W, A, B, S, M, Hw, O.OracleConfig(16, h_mode=h_mode, seed=9, phases=O.PH_MASK), 4)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+
+
+def test_theorem_1_with_several_groups_per_block():
+    cfg, W, X = tiny(d_out=32, d_in=32, db=8, n=128)
+    H = O.gram(X)
+    for h_mode in (O.FULL, O.DIAG):
+        Hw = O.weighting(H, h_mode)
+        oc = O.OracleConfig(8, h_mode=h_mode, seed=5, mask_groups=4)
+        L0 = O.proxy_loss(W, *O.init(W, H, oc)[:3], Hw)
+        (A, B, S, M), infos = O.run(W, H, oc, 6)
+        prev = L0
+        for info in infos:
+            seq = [info.loss[k_] for k_ in ("start", "A", "B", "S", "mask")]
+            assert np.isclose(seq[0], prev, rtol=1e-12)
+            for a, b in zip(seq, seq[1:]):
+                assert b <= a * (1 + 1e-10)
+            prev = seq[-1]
+        assert prev < L0 and sum(i.groups_changed for i in infos) > 0
+        assert np.all(M.reshape(32, -1, 4).sum(axis=2) == 2) and np.all(S[~M] == 0)
+
+
 # ------------------------------------------------------------------ the paper's gradient steps (Algorithm 2)
 def _grad_fd(f, X, eps=1e-6):
     g = np.zeros_like(X)
