@@ -87,6 +87,9 @@ typedef struct {
   int32_t mask_sweeps; /* sparse-core updates (Algorithm 3) per iteration, each from the state the previous one
                           left, run k of iteration t drawing its groups with the counter t*K + k; 0 means 1,
                           the paper's alternation; at most 64 */
+  int32_t mask_groups; /* groups drawn per block in one sparse-core update: the k smallest race keys, each solved on
+                          its own, all kept or dropped together by the exact joint change of the loss (either
+                          weighting); 0 means 1, the paper's single group; at most 8 */
   float ridge;         /* relative proximal ridge of the block solves (1e-6) */
   float adam_lr;       /* ARMOR_AB_ADAM: step size (0: 1e-4, Appendix F of the paper) */
   float adam_beta1;    /* moment decay rates and epsilon (0: 0.9, 0.999, 1e-8, the defaults of the Adam paper) */

@@ -42,7 +42,7 @@ class armor_config(C.Structure):
     _fields_ = [("d_out", C.c_int64), ("d_in", C.c_int64), ("d_block", C.c_int32), ("n_keep", C.c_int32),
                 ("m_group", C.c_int32), ("h_mode", C.c_int32), ("select_mode", C.c_int32),
                 ("s_step", C.c_int32), ("precision", C.c_int32), ("normalize", C.c_int32),
-                ("phases", C.c_int32), ("ab_step", C.c_int32), ("mask_sweeps", C.c_int32), ("ridge", C.c_float), ("adam_lr", C.c_float),
+                ("phases", C.c_int32), ("ab_step", C.c_int32), ("mask_sweeps", C.c_int32), ("mask_groups", C.c_int32), ("ridge", C.c_float), ("adam_lr", C.c_float),
                 ("adam_beta1", C.c_float), ("adam_beta2", C.c_float), ("adam_eps", C.c_float), ("seed", C.c_uint64)]
 
 
@@ -118,10 +118,10 @@ def _stream() -> C.c_void_p:
 
 
 def make_config(d_out, d_in, d_block, *, n_keep=2, m_group=4, h_mode=H_FULL, select_mode=SELECT_L1_RANDOM,
-                s_step=S_EXACT, precision=PREC_FP32X3, normalize=0, phases=0, ab_step=AB_EXACT, mask_sweeps=1, ridge=1e-6,
+                s_step=S_EXACT, precision=PREC_FP32X3, normalize=0, phases=0, ab_step=AB_EXACT, mask_sweeps=1, mask_groups=1, ridge=1e-6,
                 adam_lr=0.0, adam_beta1=0.0, adam_beta2=0.0, adam_eps=0.0, seed=0) -> armor_config:
     return armor_config(d_out, d_in, d_block, n_keep, m_group, h_mode, select_mode, s_step, precision,
-                        int(normalize), phases, ab_step, mask_sweeps, ridge, adam_lr, adam_beta1, adam_beta2, adam_eps, seed)
+                        int(normalize), phases, ab_step, mask_sweeps, mask_groups, ridge, adam_lr, adam_beta1, adam_beta2, adam_eps, seed)
 
 
 # ---------------------------------------------------------------- C entry points, same names

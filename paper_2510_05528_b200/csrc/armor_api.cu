@@ -30,6 +30,7 @@ armor_status check_config(const armor_config* cfg) {
   if (cfg->s_step != ARMOR_S_EXACT && cfg->s_step != ARMOR_S_BETA) return ARMOR_ERR_INVALID_ARG;
   if (cfg->ab_step < ARMOR_AB_EXACT || cfg->ab_step > ARMOR_AB_ADAM) return ARMOR_ERR_INVALID_ARG;
   if (cfg->mask_sweeps < 0 || cfg->mask_sweeps > 64) return ARMOR_ERR_INVALID_ARG;
+  if (cfg->mask_groups < 0 || cfg->mask_groups > 8) return ARMOR_ERR_INVALID_ARG;
   if (cfg->adam_lr < 0.f || cfg->adam_beta1 < 0.f || cfg->adam_beta1 >= 1.f || cfg->adam_beta2 < 0.f ||
       cfg->adam_beta2 >= 1.f || cfg->adam_eps < 0.f)
     return ARMOR_ERR_INVALID_ARG;
@@ -84,9 +85,10 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   TAKE(alpha, float*, (size_t)cfg.d_out * sizeof(float));
   TAKE(hdiag, float*, (size_t)cfg.d_in * sizeof(float));
   const int64_t nbo_pad = (nbo + 31) / 32 * 32;
-  TAKE(Zsel, float*, (size_t)nbo_pad * nbi * db * sizeof(float));
-  TAKE(Acol, float*, (size_t)nbo * nbi * db * sizeof(float));
-  TAKE(Ysel, float*, (size_t)nbo_pad * nbi * cfg.d_in * sizeof(float));
+  const int64_t kg = cfg.mask_groups > 0 ? cfg.mask_groups : 1;   // draws per block: every per-draw table grows by kg
+  TAKE(Zsel, float*, (size_t)nbo_pad * nbi * kg * db * sizeof(float));
+  TAKE(Acol, float*, (size_t)nbo * nbi * kg * db * sizeof(float));
+  TAKE(Ysel, float*, (size_t)nbo_pad * nbi * kg * cfg.d_in * sizeof(float));
   if (c) c->nbo_pad = (int)nbo_pad;
   TAKE(colpart, double*, (size_t)64 * cfg.d_in * sizeof(double));
   if (tc) {
@@ -119,10 +121,10 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   TAKE(sc, double*, SC_COUNT * sizeof(double));
   TAKE(partials, double*, (size_t)8 * npart * sizeof(double));
   const int64_t nbmax = nbo > nbi ? nbo : nbi;
-  TAKE(partblk, double*, (size_t)(4 * nbmax > nbo * nbi ? 4 * nbmax : nbo * nbi) * sizeof(double));
-  TAKE(quadpart, double*, (size_t)nbo * nbi * sizeof(double));
+  TAKE(partblk, double*, (size_t)(4 * nbmax > nbo * nbi * kg ? 4 * nbmax : nbo * nbi * kg) * sizeof(double));
+  TAKE(quadpart, double*, (size_t)nbo * nbi * kg * sizeof(double));
   TAKE(failflag, int32_t*, (size_t)nbmax * sizeof(int32_t));
-  TAKE(sel, SelRec*, (size_t)nbo * nbi * sizeof(SelRec));
+  TAKE(sel, SelRec*, (size_t)nbo * nbi * kg * sizeof(SelRec));
   TAKE(status, int32_t*, ST_COUNT * sizeof(int32_t));
 #undef TAKE
   if (c) {
@@ -265,6 +267,7 @@ armor_status armor_create(armor_ctx** out, const armor_config* cfg, void* d_work
   c->db = cfg->d_block; c->nbo = (int)(cfg->d_out / cfg->d_block); c->nbi = (int)(cfg->d_in / cfg->d_block);
   c->ws = static_cast<char*>(d_workspace); c->ws_bytes = bytes;
   c->launches = 0;
+  c->kg = cfg->mask_groups > 0 ? cfg->mask_groups : 1;
   c->h_cached = nullptr;
   c->timing_on = 0; c->timing_n = 0; c->ev_beg = nullptr; c->ev_end = nullptr; c->ev_created = 0; c->timing_flops = 0.0;
   carve(*cfg, c, c->ws);
@@ -536,7 +539,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
         core_gradient(c, A, B, s);
         launch_mask_select(c, c->Gam, S, M, t * sweeps + sw, s);
         launch_mask_quadratic(c, A, B, H, s);
-        launch_stage(c, is, 4, c->partblk, nbo * nbi, 0, s);
+        launch_stage(c, is, 4, c->partblk, nbo * nbi * c->kg, 0, s);
         launch_mask_commit(c, S, M, is, s);
       }
       if (carry_P && it + 1 < n_iters) launch_mask_carry_P(c, c->P, s);              // P += dS B H_w (if accepted)

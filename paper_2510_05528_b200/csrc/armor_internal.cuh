@@ -83,6 +83,7 @@ struct armor_ctx {
   SelRec* sel;        // [nbo * nbi]
   int32_t* status;    // [ST_COUNT]
   int64_t launches;
+  int kg;               // groups drawn per block in one sparse-core update (mask_groups, at least 1)
   int block_one_pass;   // 1: products with the wrappers take one tf32 pass (the bf16 forward, whose operands are
                         // rounded to 8 bits anyway); 0: three passes, fp32-grade
   // identity of the H whose low part is cached in Hlo

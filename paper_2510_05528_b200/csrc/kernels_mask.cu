@@ -122,12 +122,16 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
                                                          const float* __restrict__ Kfull, SelRec* __restrict__ sel,
                                                          double* __restrict__ part, int64_t d_in, int db, int nbi,
                                                          int n_keep, int select_mode, uint64_t seed, uint64_t t,
-                                                         uint64_t n_groups_total) {
-  const int blk = blockIdx.x;
-  const int bi = blk / nbi, bj = blk % nbi;
+                                                         uint64_t n_groups_total, int kg) {
+  const int bi = blockIdx.x / nbi, bj = blockIdx.x % nbi;
+  __shared__ uint64_t s_chosen[8];
   const int gpb = db / MG;                // groups per block row
   const int64_t ng_row = d_in / MG;       // groups per matrix row
   const int n_in_block = db * gpb;
+  // kg draws: the kg smallest keys of the block, one after the other; the record of draw kk of block (i, j) is
+  // entry (i, kk * nbi + j) of a [nbo][kg * nbi] table (kk * nbi + j acts as a column block of its own downstream)
+  for (int kk = 0; kk < kg; ++kk) {
+  const int blk = bi * (kg * nbi) + kk * nbi + bj;
   float best_key = INFINITY;
   uint64_t best_g = ~0ull;
   for (int idx = threadIdx.x; idx < n_in_block; idx += NT) {
@@ -152,6 +156,8 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
     else if (select_mode == ARMOR_SELECT_UNIFORM_RANDOM) score = 1.f;
     if (!(alpha[row] > 0.f)) score = 0.f;
     const uint64_t g = (uint64_t)row * (uint64_t)ng_row + (uint64_t)cg;
+    for (int q = 0; q < kk; ++q)
+      if (s_chosen[q] == g) score = 0.f;                    // drawn already
     float key = INFINITY;
     if (score > 0.f) {
       if (select_mode != ARMOR_SELECT_L1_GREEDY) {
@@ -184,16 +190,19 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
   __syncthreads();
   best_key = s_key;
   best_g = s_g;
-  if (!(best_key < INFINITY)) {
+  if (!(best_key < INFINITY)) {                               // nothing left to draw in this block (uniform)
     if (threadIdx.x == 0) {
       SelRec rec;
       rec.valid = 0; rec.row = 0; rec.cgrp = 0; rec.new_mask = 0; rec.old_mask = 0;
       for (int p = 0; p < 8; ++p) { rec.new_val[p] = 0.f; rec.old_val[p] = 0.f; }
-      sel[blk] = rec;
-      part[blk] = 0.0;
+      for (int k2 = kk; k2 < kg; ++k2) {
+        sel[bi * (kg * nbi) + k2 * nbi + bj] = rec;
+        part[bi * (kg * nbi) + k2 * nbi + bj] = 0.0;
+      }
     }
     return;
   }
+  if (threadIdx.x == 0) s_chosen[kk] = best_g;
 
   // ---- the selected group: z = Gamma_g + alpha K_c s_g, one candidate mask per thread
   const int64_t row = (int64_t)(best_g / (uint64_t)ng_row);
@@ -283,7 +292,7 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
     }
   }
   __syncthreads();
-  if (s_win == 0xffffffffu || cand != s_win) return;
+  if (s_win != 0xffffffffu && cand == s_win) {
   // the winning thread writes the record
   SelRec rec;
   rec.valid = 1;
@@ -304,6 +313,9 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
     ehv += (double)Gam[row * d_in + cg * MG + p] * ((double)rec.new_val[p] - (double)rec.old_val[p]);
   part[blk] = ehv;
   sel[blk] = rec;
+  }
+  __syncthreads();                                          // the shared scratch is reused by the next draw
+  }
 }
 
 // The group updates of one iteration change the core by dS (one group per (i, j) block) and the
@@ -314,9 +326,10 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
 // row, :], and mask_quad_kernel sums the pairs in a fixed order.
 __global__ void __launch_bounds__(NT) mask_vectors_kernel(const float* __restrict__ A, const float* __restrict__ B,
                                                           const SelRec* __restrict__ sel, float* __restrict__ Zsel,
-                                                          float* __restrict__ Acol, int db, int nbo_pad, int nbi, int mg) {
-  const int blk = blockIdx.x;
-  const int bi = blk / nbi, bj = blk % nbi;
+                                                          float* __restrict__ Acol, int db, int nbo_pad, int nbi, int mg,
+                                                          int nbv) {
+  const int blk = blockIdx.x;                  // (row block, virtual column block v = draw * nbi + column block)
+  const int bi = blk / nbv, v = blk % nbv, bj = v % nbi;
   const SelRec rec = sel[blk];
   for (int k = threadIdx.x; k < db; k += NT) {
     float a = 0.f, z = 0.f;
@@ -327,8 +340,8 @@ __global__ void __launch_bounds__(NT) mask_vectors_kernel(const float* __restric
       const float* Bj = B + (int64_t)bj * db * db;
       for (int p = 0; p < mg; ++p) z = fmaf(rec.new_val[p] - rec.old_val[p], Bj[(int64_t)(lc + p) * db + k], z);
     }
-    Acol[((int64_t)bi * nbi + bj) * db + k] = a;
-    Zsel[((int64_t)bj * nbo_pad + bi) * db + k] = z;
+    Acol[((int64_t)bi * nbv + v) * db + k] = a;
+    Zsel[((int64_t)v * nbo_pad + bi) * db + k] = z;
   }
 }
 
@@ -337,21 +350,23 @@ __global__ void __launch_bounds__(NT) mask_vectors_kernel(const float* __restric
 __global__ void __launch_bounds__(NT) mask_quad_kernel(const float* __restrict__ Zsel, const float* __restrict__ Acol,
                                                        const float* __restrict__ Y, const float* __restrict__ hdiag,
                                                        double* __restrict__ part, int64_t d_in, int db, int nbo_pad,
-                                                       int nbi) {
-  const int bi = blockIdx.x / nbi, j = blockIdx.x % nbi;
+                                                       int nbi, int nbv) {
+  const int bi = blockIdx.x / nbv, j = blockIdx.x % nbv;      // j, j2: virtual column blocks (draw * nbi + column block)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = NT / 32;
   double acc = 0.0;
-  const float* a1 = Acol + ((int64_t)bi * nbi + j) * db;
-  for (int j2 = Y ? warp : j + warp; j2 < (Y ? nbi : j + 1); j2 += nw) {
-    const float* a2 = Acol + ((int64_t)bi * nbi + j2) * db;
+  const float* a1 = Acol + ((int64_t)bi * nbv + j) * db;
+  const float* z1 = Zsel + ((int64_t)j * nbo_pad + bi) * db;
+  for (int j2 = warp; j2 < nbv; j2 += nw) {
+    if (!Y && (j2 % nbi) != (j % nbi)) continue;              // diagonal weighting: other column blocks do not interact
+    const float* a2 = Acol + ((int64_t)bi * nbv + j2) * db;
     const float* z2 = Zsel + ((int64_t)j2 * nbo_pad + bi) * db;
     float w = 0.f, m = 0.f;
     if (Y) {
-      const float* y = Y + ((int64_t)j * nbo_pad + bi) * d_in + (int64_t)j2 * db;
+      const float* y = Y + ((int64_t)j * nbo_pad + bi) * d_in + (int64_t)(j2 % nbi) * db;
       for (int k = lane; k < db; k += 32) { w = fmaf(a1[k], a2[k], w); m = fmaf(y[k], z2[k], m); }
     } else {
-      const float* h = hdiag + (int64_t)j * db;
-      for (int k = lane; k < db; k += 32) { w = fmaf(a1[k], a2[k], w); m = fmaf(z2[k] * h[k], z2[k], m); }
+      const float* h = hdiag + (int64_t)(j % nbi) * db;
+      for (int k = lane; k < db; k += 32) { w = fmaf(a1[k], a2[k], w); m = fmaf(z1[k] * h[k], z2[k], m); }
     }
     for (int o = 16; o > 0; o >>= 1) {
       w += __shfl_xor_sync(0xffffffffu, w, o);
@@ -399,13 +414,13 @@ __global__ void mask_commit_kernel(const SelRec* __restrict__ sel, int nblocks, 
 // blocks j in order (deterministic sums); the grid is (row-block, chunk of 1024 columns).
 __global__ void __launch_bounds__(NT) mask_carry_kernel(const SelRec* __restrict__ sel, const float* __restrict__ Y,
                                                         float* __restrict__ P, const double* __restrict__ sc,
-                                                        int64_t d_in, int nbo_pad, int nbi) {
+                                                        int64_t d_in, int nbo_pad, int nbv) {
   if (sc[SC_ACCEPT] == 0.0) return;
   const int bi = blockIdx.x;
   const int64_t c4 = (int64_t)blockIdx.y * 1024 + 4 * threadIdx.x;
   if (c4 >= d_in) return;
-  for (int j = 0; j < nbi; ++j) {
-    const SelRec rec = sel[bi * nbi + j];
+  for (int j = 0; j < nbv; ++j) {                            // virtual column blocks in order: deterministic sums
+    const SelRec rec = sel[bi * nbv + j];
     if (!rec.valid) continue;
     const float4 y = *reinterpret_cast<const float4*>(Y + ((int64_t)j * nbo_pad + bi) * d_in + c4);
     float4* dst = reinterpret_cast<float4*>(P + (int64_t)rec.row * d_in + c4);
@@ -419,7 +434,7 @@ __global__ void __launch_bounds__(NT) mask_carry_kernel(const SelRec* __restrict
 
 void launch_mask_carry_P(armor_ctx* c, float* P, cudaStream_t s) {
   mask_carry_kernel<<<dim3(c->nbo, (unsigned)((c->d_in + 1023) / 1024)), NT, 0, s>>>(c->sel, c->Ysel, P, c->sc, c->d_in,
-                                                                                   c->nbo_pad, c->nbi);
+                                                                                   c->nbo_pad, c->nbi * c->kg);
   c->launches++;
 }
 
@@ -432,7 +447,7 @@ void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const ui
   const int mg = c->cfg.m_group;
   const uint64_t n_groups = (uint64_t)(c->d_out * (c->d_in / mg));
 #define ARMOR_SELECT_ARGS Gam, S, M, c->alpha, c->Kfull, c->sel, c->partblk, c->d_in, c->db, c->nbi, c->cfg.n_keep, \
-                          c->cfg.select_mode, c->cfg.seed, (uint64_t)t, n_groups
+                          c->cfg.select_mode, c->cfg.seed, (uint64_t)t, n_groups, c->kg
   if (mg == 8 && c->cfg.n_keep > 4) mask_select_kernel<8, 6><<<c->nbo * c->nbi, NT, 0, s>>>(ARMOR_SELECT_ARGS);
   else if (mg == 8) mask_select_kernel<8, 4><<<c->nbo * c->nbi, NT, 0, s>>>(ARMOR_SELECT_ARGS);
   else mask_select_kernel<4, 4><<<c->nbo * c->nbi, NT, 0, s>>>(ARMOR_SELECT_ARGS);
@@ -441,29 +456,33 @@ void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const ui
 }
 
 void launch_mask_quadratic(armor_ctx* c, const float* A, const float* B, const float* H, cudaStream_t s) {
-  const int db = c->db, nbo = c->nbo, nbi = c->nbi, nbo_pad = c->nbo_pad;
-  mask_vectors_kernel<<<nbo * nbi, NT, 0, s>>>(A, B, c->sel, c->Zsel, c->Acol, db, nbo_pad, nbi, c->cfg.m_group);
+  const int db = c->db, nbo = c->nbo, nbi = c->nbi, nbo_pad = c->nbo_pad, kg = c->kg, nbv = nbi * kg;
+  mask_vectors_kernel<<<nbo * nbv, NT, 0, s>>>(A, B, c->sel, c->Zsel, c->Acol, db, nbo_pad, nbi, c->cfg.m_group, nbv);
   c->launches++;
   const float* Y = nullptr;
   if (c->cfg.h_mode == ARMOR_H_FULL) {
-    // y_ij = z_ij H[j-th block row, :], batched over j:  [nbo, db] x [db, d_in]
-    if (!(g_tc_blocks && tc_gram_ok(c) && tc_select_rows_times_H(c, c->Zsel, H, c->Ysel, nbo_pad, s) == ARMOR_OK)) {
-      BGemm g{};
-      g.A = c->Zsel; g.sAb = (int64_t)nbo_pad * db; g.sAm = db; g.sAk = 1;
-      g.B = H; g.sBb = (int64_t)db * c->d_in; g.sBk = c->d_in; g.sBn = 1;
-      g.C = c->Ysel; g.sCb = (int64_t)nbo_pad * c->d_in; g.sCm = c->d_in; g.sCn = 1;
-      g.M = nbo; g.N = (int)c->d_in; g.K = db; g.batch = nbi; g.alpha = 1.f;
-      launch_bgemm(c, g, s);
+    // y_v = z_v H[j-th block row, :], batched over the column blocks j, one launch per draw:  [nbo, db] x [db, d_in]
+    for (int kk = 0; kk < kg; ++kk) {
+      const float* Zk = c->Zsel + (int64_t)kk * nbi * nbo_pad * db;
+      float* Yk = c->Ysel + (int64_t)kk * nbi * nbo_pad * c->d_in;
+      if (!(g_tc_blocks && tc_gram_ok(c) && tc_select_rows_times_H(c, Zk, H, Yk, nbo_pad, s) == ARMOR_OK)) {
+        BGemm g{};
+        g.A = Zk; g.sAb = (int64_t)nbo_pad * db; g.sAm = db; g.sAk = 1;
+        g.B = H; g.sBb = (int64_t)db * c->d_in; g.sBk = c->d_in; g.sBn = 1;
+        g.C = Yk; g.sCb = (int64_t)nbo_pad * c->d_in; g.sCm = c->d_in; g.sCn = 1;
+        g.M = nbo; g.N = (int)c->d_in; g.K = db; g.batch = nbi; g.alpha = 1.f;
+        launch_bgemm(c, g, s);
+      }
     }
     Y = c->Ysel;
   }
   double* part = c->quadpart;
-  mask_quad_kernel<<<nbo * nbi, NT, 0, s>>>(c->Zsel, c->Acol, Y, c->hdiag, part, c->d_in, db, nbo_pad, nbi);
+  mask_quad_kernel<<<nbo * nbv, NT, 0, s>>>(c->Zsel, c->Acol, Y, c->hdiag, part, c->d_in, db, nbo_pad, nbi, nbv);
   c->launches++;
-  reduce_partials_to(c, part, nbo * nbi, c->sc + SC_Q_M, s);
+  reduce_partials_to(c, part, nbo * nbv, c->sc + SC_Q_M, s);
 }
 
 void launch_mask_commit(armor_ctx* c, float* S, uint8_t* M, armor_iter_stats* st, cudaStream_t s) {
-  mask_commit_kernel<<<1, 256, 0, s>>>(c->sel, c->nbo * c->nbi, S, M, c->d_in, c->cfg.m_group, c->sc, st);
+  mask_commit_kernel<<<1, 256, 0, s>>>(c->sel, c->nbo * c->nbi * c->kg, S, M, c->d_in, c->cfg.m_group, c->sc, st);
   c->launches++;
 }

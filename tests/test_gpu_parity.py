@@ -275,6 +275,46 @@ def test_several_sparse_core_updates_per_iteration(h_mode, ab_step, mid_data):
     assert ctx.device_status()[:4] == [0, 0, 0, 0]
 
 
+@pytest.mark.parametrize("cfg_name", ["tiny", "mid"])
+@pytest.mark.parametrize("h_mode", [Bd.H_FULL, Bd.H_DIAG])
+def test_several_groups_per_block_in_one_update(h_mode, cfg_name, tiny_data, mid_data):
+    """mask_groups = 3: the three smallest race keys of every block are drawn in one sparse-core update, each group
+    solved on its own, all kept or dropped by the exact joint change of the loss.  Teacher-forced."""
+    cfg, (W, X, H32) = (TINY, tiny_data) if cfg_name == "tiny" else (MID, mid_data)
+    k = 3
+    ctx = make(cfg, Bd.PREC_FP32X3, h_mode, mask_groups=k)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    oc = O.OracleConfig(cfg.d_block, h_mode=h_mode, seed=cfg.seed, mask_groups=k)
+    Hq = H32.astype(np.float64)
+    Hw = O.weighting(Hq, h_mode)
+    Wn = W.astype(np.float64)
+    A, B, S, M = O.init(Wn, Hq, oc)
+    tol = TOL[Bd.PREC_FP32X3]
+    compared = 0
+    for t in range(4):
+        load_state(st, A, B, S, M)
+        sg = ctx.read_stats(ctx.bcd_step(st, Hd, t, 1))[0]
+        A, B, S, M, info = O.bcd_iteration(Wn, A, B, S, M, Hw, oc, t)
+        assert rel(host(st.A), A) < tol["A"] and rel(host(st.B), B) < tol["B"]
+        diff = mask_block_diffs(host(st.M), M, cfg.d_block)
+        if sg["mask_accepted"] != info.mask_accepted:
+            assert abs(info.delta_L_mask) <= tol["margin"] * info.loss["S"]
+            continue
+        assert diff <= excused_blocks(info, tol["margin"])
+        if not diff:
+            compared += 1
+            assert rel(host(st.S), S) < tol["S"]
+            assert sg["groups_changed"] == info.groups_changed
+            assert abs(sg["delta_L_mask"] - info.delta_L_mask) <= 1e-3 * abs(info.delta_L_mask) + 1e-9 * info.loss["start"]
+            assert abs(sg["loss_mask"] - info.loss["mask"]) / info.loss["mask"] < 1e-3
+        assert abs(ctx.proxy_loss(st, Hd).item() - sg["loss_mask"]) / sg["loss_mask"] < 1e-4
+    assert compared >= 2
+    Mg = O.unpack_mask(host(st.M))
+    assert np.all(Mg.reshape(cfg.d_out, -1, 4).sum(axis=2) == 2) and np.all(host(st.S)[~Mg] == 0.0)
+    assert ctx.device_status()[:4] == [0, 0, 0, 0]
+
+
 def test_teacher_forced_paper_step_size_for_the_core(tiny_data):
     """s_step = BETA: the paper's 1/beta_W' step (Eq. lrWprime) instead of the exact line search."""
     W, X, H32 = tiny_data

@@ -48,6 +48,7 @@ def test_config_validation(lib):
         (Bd.make_config(256, 256, 32, ab_step=3), 1),
         (Bd.make_config(256, 256, 32, mask_sweeps=65), 1),
         (Bd.make_config(256, 256, 32, mask_sweeps=-1), 1),
+        (Bd.make_config(256, 256, 32, mask_groups=9), 1),
         (Bd.make_config(256, 256, 32, ab_step=Bd.AB_ADAM, adam_beta1=1.5), 1),
         (Bd.make_config(256, 256, 32, ab_step=Bd.AB_GD), 7),          # the paper's gradient steps need the diagonal weighting
         (Bd.make_config(256, 256, 32, ridge=-1.0), 1),
@@ -56,7 +57,7 @@ def test_config_validation(lib):
     ]
     for good in (Bd.make_config(256, 256, 32, n_keep=4, m_group=8), Bd.make_config(256, 256, 32, n_keep=5, m_group=8),
                  Bd.make_config(256, 256, 32, n_keep=6, m_group=8), Bd.make_config(512, 512, 256),
-                 Bd.make_config(256, 256, 32, s_step=Bd.S_BETA), Bd.make_config(256, 256, 32, mask_sweeps=8),
+                 Bd.make_config(256, 256, 32, s_step=Bd.S_BETA), Bd.make_config(256, 256, 32, mask_sweeps=8), Bd.make_config(256, 256, 32, mask_groups=4),
                  Bd.make_config(256, 256, 32, ab_step=Bd.AB_GD, h_mode=Bd.H_DIAG),
                  Bd.make_config(256, 256, 32, ab_step=Bd.AB_ADAM, adam_lr=1e-3)):
         assert Bd.armor_workspace_bytes(good) > 0
