@@ -383,7 +383,10 @@ def run_ours(args, cfg):
         for name, kw, iters in (("diag_exact", dict(h_mode=Bd.H_DIAG), lcfg.n_iters),
                                 ("diag_adam_lr1e-4", dict(h_mode=Bd.H_DIAG, ab_step=Bd.AB_ADAM), 10 * lcfg.n_iters),
                                 ("full_adam_lr1e-4", dict(h_mode=Bd.H_FULL, ab_step=Bd.AB_ADAM), lcfg.n_iters),
-                                ("full_exact_4_sweeps", dict(h_mode=Bd.H_FULL, mask_sweeps=4), lcfg.n_iters)):
+                                ("full_exact_4_sweeps", dict(h_mode=Bd.H_FULL, mask_sweeps=4), lcfg.n_iters),
+                                ("full_exact_4_groups", dict(h_mode=Bd.H_FULL, mask_groups=4), lcfg.n_iters),
+                                ("diag_adam_lr1e-4_8_groups", dict(h_mode=Bd.H_DIAG, ab_step=Bd.AB_ADAM, mask_groups=8),
+                                 10 * lcfg.n_iters)):
             cx = Bd.ArmorContext(lcfg.d_out, lcfg.d_in, lcfg.d_block, device=dev, precision=prec, seed=lcfg.seed, **kw)
             sx = cx.init(W_d, H)
             cx.bcd_step(sx, H, 0, 3, want_stats=False)          # warm-up
