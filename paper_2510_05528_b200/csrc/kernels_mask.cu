@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
                                                          int n_keep, int select_mode, uint64_t seed, uint64_t t,
                                                          uint64_t n_groups_total, int kg) {
   const int bi = blockIdx.x / nbi, bj = blockIdx.x % nbi;
-  __shared__ uint64_t s_chosen[8];
+  extern __shared__ float s_keys[];         // kg > 1: the keys of the block's groups, kept for the later draws
   const int gpb = db / MG;                // groups per block row
   const int64_t ng_row = d_in / MG;       // groups per matrix row
   const int n_in_block = db * gpb;
@@ -138,6 +138,12 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
     const int rl = idx / gpb, cl = idx % gpb;
     const int64_t row = (int64_t)bi * db + rl;
     const int64_t cg = (int64_t)bj * gpb + cl;
+    if (kk > 0) {                                           // later draws: keys from the first pass, drawn ones at +inf
+      const float key = s_keys[idx];
+      const uint64_t g = (uint64_t)row * (uint64_t)ng_row + (uint64_t)cg;
+      if (key < best_key || (key == best_key && g < best_g)) { best_key = key; best_g = g; }
+      continue;
+    }
     float score = 0.f, sq = 0.f;
 #pragma unroll
     for (int h = 0; h < MG / 4; ++h) {
@@ -156,8 +162,6 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
     else if (select_mode == ARMOR_SELECT_UNIFORM_RANDOM) score = 1.f;
     if (!(alpha[row] > 0.f)) score = 0.f;
     const uint64_t g = (uint64_t)row * (uint64_t)ng_row + (uint64_t)cg;
-    for (int q = 0; q < kk; ++q)
-      if (s_chosen[q] == g) score = 0.f;                    // drawn already
     float key = INFINITY;
     if (score > 0.f) {
       if (select_mode != ARMOR_SELECT_L1_GREEDY) {
@@ -167,6 +171,7 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
         key = -score;
       }
     }
+    if (kg > 1) s_keys[idx] = key;
     if (key < best_key || (key == best_key && g < best_g)) { best_key = key; best_g = g; }
   }
   // arg-min over the CTA; ties go to the lower group index
@@ -202,7 +207,10 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
     }
     return;
   }
-  if (threadIdx.x == 0) s_chosen[kk] = best_g;
+  if (threadIdx.x == 0 && kg > 1) {                         // out of the race for the later draws
+    const int rl0 = (int)(best_g / (uint64_t)ng_row) - bi * db, cl0 = (int)(best_g % (uint64_t)ng_row) - bj * gpb;
+    s_keys[rl0 * gpb + cl0] = INFINITY;
+  }
 
   // ---- the selected group: z = Gamma_g + alpha K_c s_g, one candidate mask per thread
   const int64_t row = (int64_t)(best_g / (uint64_t)ng_row);
@@ -448,9 +456,18 @@ void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const ui
   const uint64_t n_groups = (uint64_t)(c->d_out * (c->d_in / mg));
 #define ARMOR_SELECT_ARGS Gam, S, M, c->alpha, c->Kfull, c->sel, c->partblk, c->d_in, c->db, c->nbi, c->cfg.n_keep, \
                           c->cfg.select_mode, c->cfg.seed, (uint64_t)t, n_groups, c->kg
-  if (mg == 8 && c->cfg.n_keep > 4) mask_select_kernel<8, 6><<<c->nbo * c->nbi, NT, 0, s>>>(ARMOR_SELECT_ARGS);
-  else if (mg == 8) mask_select_kernel<8, 4><<<c->nbo * c->nbi, NT, 0, s>>>(ARMOR_SELECT_ARGS);
-  else mask_select_kernel<4, 4><<<c->nbo * c->nbi, NT, 0, s>>>(ARMOR_SELECT_ARGS);
+  // kg > 1: the block's keys stay in shared memory between the draws (up to 64 KiB: d_block 256, groups of four)
+  const size_t smem = c->kg > 1 ? (size_t)c->db * (c->db / mg) * sizeof(float) : 0;
+  if (mg == 8 && c->cfg.n_keep > 4) {
+    if (smem > 48 * 1024) cudaFuncSetAttribute(mask_select_kernel<8, 6>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    mask_select_kernel<8, 6><<<c->nbo * c->nbi, NT, smem, s>>>(ARMOR_SELECT_ARGS);
+  } else if (mg == 8) {
+    if (smem > 48 * 1024) cudaFuncSetAttribute(mask_select_kernel<8, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    mask_select_kernel<8, 4><<<c->nbo * c->nbi, NT, smem, s>>>(ARMOR_SELECT_ARGS);
+  } else {
+    if (smem > 48 * 1024) cudaFuncSetAttribute(mask_select_kernel<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    mask_select_kernel<4, 4><<<c->nbo * c->nbi, NT, smem, s>>>(ARMOR_SELECT_ARGS);
+  }
 #undef ARMOR_SELECT_ARGS
   c->launches++;
 }
