@@ -116,13 +116,14 @@ __device__ __forceinline__ bool chol_small(int n, const double (&Kin)[NKM][NKM],
 // Pass 2: thread b < 2^MG evaluates the mask with bit pattern b (if it keeps exactly n_keep positions);
 // the best one is found with the oracle's order: larger reduction first; among equal reductions the
 // incumbent, then the lexicographically first index tuple.
-template <int MG, int NKM>
+template <int MG, int NKM, bool MULTI>
 __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict__ Gam, const float* __restrict__ S,
                                                          const uint8_t* __restrict__ M, const float* __restrict__ alpha,
                                                          const float* __restrict__ Kfull, SelRec* __restrict__ sel,
                                                          double* __restrict__ part, int64_t d_in, int db, int nbi,
                                                          int n_keep, int select_mode, uint64_t seed, uint64_t t,
-                                                         uint64_t n_groups_total, int kg) {
+                                                         uint64_t n_groups_total, int kg_arg) {
+  const int kg = MULTI ? kg_arg : 1;                       // one draw: the loop and the key cache compile away
   const int bi = blockIdx.x / nbi, bj = blockIdx.x % nbi;
   extern __shared__ float s_keys[];         // kg > 1: the keys of the block's groups, kept for the later draws
   const int gpb = db / MG;                // groups per block row
@@ -138,7 +139,7 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
     const int rl = idx / gpb, cl = idx % gpb;
     const int64_t row = (int64_t)bi * db + rl;
     const int64_t cg = (int64_t)bj * gpb + cl;
-    if (kk > 0) {                                           // later draws: keys from the first pass, drawn ones at +inf
+    if (MULTI && kk > 0) {                                  // later draws: keys from the first pass, drawn ones at +inf
       const float key = s_keys[idx];
       const uint64_t g = (uint64_t)row * (uint64_t)ng_row + (uint64_t)cg;
       if (key < best_key || (key == best_key && g < best_g)) { best_key = key; best_g = g; }
@@ -171,7 +172,7 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
         key = -score;
       }
     }
-    if (kg > 1) s_keys[idx] = key;
+    if (MULTI) s_keys[idx] = key;
     if (key < best_key || (key == best_key && g < best_g)) { best_key = key; best_g = g; }
   }
   // arg-min over the CTA; ties go to the lower group index
@@ -207,7 +208,7 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
     }
     return;
   }
-  if (threadIdx.x == 0 && kg > 1) {                         // out of the race for the later draws
+  if (MULTI && threadIdx.x == 0) {                          // out of the race for the later draws
     const int rl0 = (int)(best_g / (uint64_t)ng_row) - bi * db, cl0 = (int)(best_g % (uint64_t)ng_row) - bj * gpb;
     s_keys[rl0 * gpb + cl0] = INFINITY;
   }
@@ -458,16 +459,17 @@ void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const ui
                           c->cfg.select_mode, c->cfg.seed, (uint64_t)t, n_groups, c->kg
   // kg > 1: the block's keys stay in shared memory between the draws (up to 64 KiB: d_block 256, groups of four)
   const size_t smem = c->kg > 1 ? (size_t)c->db * (c->db / mg) * sizeof(float) : 0;
-  if (mg == 8 && c->cfg.n_keep > 4) {
-    if (smem > 48 * 1024) cudaFuncSetAttribute(mask_select_kernel<8, 6>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    mask_select_kernel<8, 6><<<c->nbo * c->nbi, NT, smem, s>>>(ARMOR_SELECT_ARGS);
-  } else if (mg == 8) {
-    if (smem > 48 * 1024) cudaFuncSetAttribute(mask_select_kernel<8, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    mask_select_kernel<8, 4><<<c->nbo * c->nbi, NT, smem, s>>>(ARMOR_SELECT_ARGS);
-  } else {
-    if (smem > 48 * 1024) cudaFuncSetAttribute(mask_select_kernel<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    mask_select_kernel<4, 4><<<c->nbo * c->nbi, NT, smem, s>>>(ARMOR_SELECT_ARGS);
-  }
+#define ARMOR_SELECT_LAUNCH(MGV, NKV, MULTIV)                                                                           \
+  do {                                                                                                                  \
+    if (smem > 48 * 1024)                                                                                               \
+      cudaFuncSetAttribute(mask_select_kernel<MGV, NKV, MULTIV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+    mask_select_kernel<MGV, NKV, MULTIV><<<c->nbo * c->nbi, NT, smem, s>>>(ARMOR_SELECT_ARGS);                          \
+  } while (0)
+  const bool multi = c->kg > 1;
+  if (mg == 8 && c->cfg.n_keep > 4) { if (multi) ARMOR_SELECT_LAUNCH(8, 6, true); else ARMOR_SELECT_LAUNCH(8, 6, false); }
+  else if (mg == 8) { if (multi) ARMOR_SELECT_LAUNCH(8, 4, true); else ARMOR_SELECT_LAUNCH(8, 4, false); }
+  else { if (multi) ARMOR_SELECT_LAUNCH(4, 4, true); else ARMOR_SELECT_LAUNCH(4, 4, false); }
+#undef ARMOR_SELECT_LAUNCH
 #undef ARMOR_SELECT_ARGS
   c->launches++;
 }
