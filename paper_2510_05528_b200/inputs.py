@@ -140,3 +140,11 @@ def make_tokens(cfg: LayerConfig, n: int, stream: int = 77) -> np.ndarray:
     scales = torch.from_numpy(channel_scales(cfg))
     x = torch.randn(n, cfg.d_in, generator=_gen(cfg.seed, stream), dtype=torch.float32)
     return (x * scales).numpy()
+
+
+def coupled_blocks(nb: int, d_block: int, strength: float) -> np.ndarray:
+    """Wrapper blocks [nb, d_block, d_block] fp64 whose columns are nearly parallel: the identity plus
+    ``strength / sqrt(d_block)`` in every entry.  Test input for states in which the updates of different
+    groups of one row-block overlap strongly."""
+    eye = np.eye(d_block, dtype=np.float64)
+    return np.broadcast_to(eye + strength / np.sqrt(d_block), (nb, d_block, d_block)).copy()

@@ -572,28 +572,114 @@ def test_splitmix64_reference_values():
     assert u.min() > 0.0 and u.max() < 1.0 and abs(u.mean() - 0.5) < 0.05
 
 
-def test_guard_rejects_an_increase_and_keeps_the_state(monkeypatch):
-    """Plant interacting updates: with a guard the loss still never rises (FULL mode)."""
-    cfg, W, X = tiny(d_out=8, d_in=32, db=8, n=12)      # n < d_in: strongly coupled columns
+def overlapping_state(d_out=64, d_in=256, db=32, n=4, strength=0.3, seed=5):
+    """A state in which the group updates of one iteration interact strongly: four calibration tokens (H has
+    rank 4, so the columns of a residual row are tied together) and wrapper blocks A_i whose columns are
+    nearly parallel (every group of row-block i then removes nearly the same component of E_i X^T)."""
+    cfg, W, X = tiny(d_out=d_out, d_in=d_in, db=db, n=n, seed=seed)
     H = O.gram(X)
+    oc = O.OracleConfig(db, h_mode=O.FULL, seed=1, phases=O.PH_MASK)
+    A, B, S, M = O.init(W, H, oc)
+    A = inputs.coupled_blocks(d_out // db, db, strength)
+    return W, X, H, oc, (A, B, S, M)
+
+
+def rebuild_discarded_update(W, X, A, B, S, info, m=4):
+    """The update the oracle evaluated, rebuilt without its formulas: for every selected group (info.selected)
+    and the mask chosen for it (info.new_mask), the kept values by generic least squares on the loss written
+    from the activations, every other entry of S at its old value."""
+    Ad, Bd = O.bd_dense(A), O.bd_dense(B)
+    R = X.T
+    ng_row = W.shape[1] // m
+    S_new = S.copy()
+    for g, bits in zip(info.selected.reshape(-1), info.new_mask.reshape(-1)):
+        if g < 0:
+            continue
+        r, c = divmod(int(g), ng_row)
+        cols = np.arange(m * c, m * c + m)
+        keep = [p for p in range(m) if (int(bits) >> p) & 1]
+        S0 = S.copy()
+        S0[r, cols] = 0.0
+        target = ((W - Ad @ S0 @ Bd) @ R).reshape(-1)
+        Dm = np.stack([(np.outer(Ad[:, r], Bd[cols[p]]) @ R).reshape(-1) for p in keep], axis=1)
+        sol, *_ = np.linalg.lstsq(Dm, target, rcond=None)
+        S_new[r, cols] = 0.0
+        S_new[r, cols[keep]] = sol
+    return S_new
+
+
+def test_guard_rejects_an_increase_and_keeps_the_state():
+    """Full weighting: group updates that are each optimal on their own can raise the loss together.  On a
+    state built to make them overlap the update MUST be discarded: the reported change is positive and equals
+    the change of ||E X^T||_F^2 under the rebuilt update, each group alone would have lowered the loss
+    (Lemma 2 for a single group), and the state comes back untouched."""
+    W, X, H, oc, (A, B, S, M) = overlapping_state()
     Hw = O.weighting(H, O.FULL)
-    oc = O.OracleConfig(8, h_mode=O.FULL, seed=1)
-    rng = np.random.default_rng(13)
-    seen_reject = False
-    for trial in range(30):
-        A, B, S, M = rand_state(W, H, oc, rng, scale=0.5)
+    L0 = loss_from_X(W, A, B, S, X)
+    n_reject = 0
+    for t in range(3):
         info = O.IterInfo()
-        L0 = O.proxy_loss(W, A, B, S, Hw)
-        S1, M1 = O.mask_step(W, A, B, S, M, Hw, oc, trial, info)
-        L1 = O.proxy_loss(W, A, B, S1, Hw)
-        assert L1 <= L0 * (1 + 1e-12) + 1e-18
-        if info.mask_accepted:
-            assert np.isclose(L1 - L0, info.delta_L_mask, rtol=1e-6, atol=1e-12 * L0)
+        S1, M1 = O.mask_step(W, A, B, S, M, Hw, oc, t, info)
+        S_try = rebuild_discarded_update(W, X, A, B, S, info)
+        dL_true = loss_from_X(W, A, B, S_try, X) - L0
+        assert np.isclose(info.delta_L_mask, dL_true, rtol=1e-6, atol=1e-12 * L0)
+        if t < 2:                              # found by running the oracle: t = 0, 1 overshoot, t = 2 does not
+            assert dL_true > 1e-3 * L0 and info.mask_accepted == 0 and info.groups_changed == 0
+            assert S1 is S or np.array_equal(S1, S)
+            assert M1 is M or np.array_equal(M1, M)
+            n_reject += 1
+            # one group of the discarded update on its own: a decrease, as Lemma 2 says
+            g0 = int(info.selected[0, 0])
+            one = O.IterInfo()
+            one.selected = np.array([[g0]])
+            one.new_mask = info.new_mask[:1, :1]
+            S_one = rebuild_discarded_update(W, X, A, B, S, one)
+            assert loss_from_X(W, A, B, S_one, X) <= L0 * (1 + 1e-12)
         else:
-            seen_reject = True
-            assert info.delta_L_mask > 0 and np.all(S1 == S) and np.all(M1 == M)
-    # (a rejection is possible but not guaranteed on random data)
-    assert seen_reject in (True, False)
+            assert info.mask_accepted == 1 and dL_true < 0 and np.allclose(S1, S_try, rtol=1e-7, atol=1e-12)
+    assert n_reject == 2
+
+
+def test_rejected_update_leaves_the_iteration_where_it_was():
+    """Whole iterations around a rejection (sparse-core phase only): the loss after a discarded update is the
+    loss before it, bit for bit, the next iteration draws other groups, and accepted updates follow
+    rejected ones in the same run."""
+    W, X, H, oc, state = overlapping_state()
+    (A, B, S, M), infos = O.run(W, H, oc, 5, state=state)
+    acc = [i.mask_accepted for i in infos]
+    assert acc[:2] == [0, 0] and 1 in acc[2:]
+    assert infos[0].loss["mask"] == infos[0].loss["start"] == infos[1].loss["start"]
+    assert not np.array_equal(infos[0].selected, infos[1].selected)
+    prev = infos[0].loss["start"]
+    for i in infos:
+        assert i.loss["mask"] <= prev
+        assert (i.loss["mask"] < prev) == bool(i.mask_accepted and i.delta_L_mask < 0)
+        prev = i.loss["mask"]
+    assert np.isclose(prev, loss_from_X(W, A, B, S, X), rtol=1e-9)
+
+
+def test_guard_applies_to_several_groups_per_block_with_the_diagonal_weighting():
+    """With mask_groups > 1 groups of one block share columns of A or rows of B, so the joint test can fail
+    with the paper's diagonal weighting as well; with one group per block it never does (Lemma 2)."""
+    W, X, H, oc, (A, B, S, M) = overlapping_state(strength=1.0)
+    Hw = O.weighting(H, O.DIAG)
+    R = np.diag(np.sqrt(np.diag(H)))
+    one = O.OracleConfig(oc.d_block, h_mode=O.DIAG, seed=1)
+    many = O.OracleConfig(oc.d_block, h_mode=O.DIAG, seed=1, mask_groups=8)
+    L0 = O.proxy_loss(W, A, B, S, Hw)
+    seen = 0
+    for t in range(6):
+        i1, i8 = O.IterInfo(), O.IterInfo()
+        O.mask_step(W, A, B, S, M, Hw, one, t, i1)
+        assert i1.mask_accepted == 1 and i1.delta_L_mask <= 0
+        S8, M8 = O.mask_step(W, A, B, S, M, Hw, many, t, i8)
+        if not i8.mask_accepted:
+            seen += 1
+            assert i8.delta_L_mask > 0 and np.array_equal(S8, S) and np.array_equal(M8, M)
+        else:
+            E = W - O.bd_dense(A) @ S8 @ O.bd_dense(B)
+            assert np.isclose(np.linalg.norm(E @ R) ** 2 - L0, i8.delta_L_mask, rtol=1e-6, atol=1e-12 * L0)
+    assert seen >= 1
 
 
 # ------------------------------------------------------------------ whole iteration
