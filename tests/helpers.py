@@ -52,3 +52,54 @@ def excused_blocks(info, margin):
     """Blocks whose selection or mask decision was closer than the margin (several answers are valid)."""
     close = (info.select_margin <= margin) | (info.mask_margin <= margin)
     return {(int(i), int(j)) for i, j in zip(*np.nonzero(close))}
+
+
+def make(cfg, precision, h_mode=Bd.H_FULL, **kw):
+    return Bd.ArmorContext(cfg.d_out, cfg.d_in, cfg.d_block, device=DEV, precision=precision, h_mode=h_mode,
+                           seed=cfg.seed, **kw)
+
+
+def run_teacher_forced(cfg, W, H32, prec, h_mode, n_steps, select=Bd.SELECT_L1_RANDOM, n_keep=2, m_group=4,
+                       s_step=Bd.S_EXACT, tol_scale=1.0, ab_step=Bd.AB_EXACT):
+    ctx = make(cfg, prec, h_mode, select_mode=select, n_keep=n_keep, m_group=m_group, s_step=s_step, ab_step=ab_step)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    oc = O.OracleConfig(cfg.d_block, h_mode=h_mode, seed=cfg.seed, select_mode=select, n_keep=n_keep,
+                        m_group=m_group, s_step=s_step, ab_step=ab_step)
+    Hq = H32.astype(np.float64)
+    Hw = O.weighting(Hq, h_mode)
+    Wn = W.astype(np.float64)
+    A, B, S, M = O.init(Wn, Hq, oc)
+    tol = {k: v * tol_scale for k, v in TOL[prec].items()}
+    n_excused = 0
+    worst = dict(A=0.0, B=0.0, S=0.0, loss=0.0)
+    for t in range(n_steps):
+        load_state(st, A, B, S, M, m_group)        # the GPU starts every step from the oracle's state
+        stats = ctx.bcd_step(st, Hd, t, 1)
+        sg = ctx.read_stats(stats)[0]
+        A, B, S, M, info = O.bcd_iteration(Wn, A, B, S, M, Hw, oc, t)
+        worst["A"] = max(worst["A"], rel(host(st.A), A))
+        worst["B"] = max(worst["B"], rel(host(st.B), B))
+        for k_gpu, k_or in (("loss_start", "start"), ("loss_A", "A"), ("loss_B", "B"), ("loss_S", "S")):
+            worst["loss"] = max(worst["loss"], abs(sg[k_gpu] - info.loss[k_or]) / info.loss[k_or])
+        assert abs(sg["tau_B"] - info.tau_B) <= 10 * tol["B"] * abs(info.tau_B) + 1e-6
+        assert abs(sg["tau_S"] - info.tau_S) <= 10 * tol["S"] * abs(info.tau_S) + 1e-12
+        assert sg["chol_failed"] == info.chol_failed == 0
+        # masks: identical outside blocks whose decision margin is below the threshold
+        diff = mask_block_diffs(host(st.M), M, cfg.d_block, m_group)
+        excused = excused_blocks(info, tol["margin"])
+        guard_close = abs(info.delta_L_mask) <= tol["margin"] * info.loss["S"]
+        if sg["mask_accepted"] != info.mask_accepted:
+            assert guard_close, "accept/reject differs although the guard was not marginal"
+            n_excused += len(diff)
+            continue
+        assert diff <= excused, f"step {t}: masks differ in blocks {sorted(diff - excused)} with a clear margin"
+        n_excused += len(diff)
+        if not diff:
+            worst["S"] = max(worst["S"], rel(host(st.S), S))
+            assert sg["groups_changed"] == info.groups_changed
+            worst["loss"] = max(worst["loss"], abs(sg["loss_mask"] - info.loss["mask"]) / info.loss["mask"])
+    assert ctx.device_status()[:4] == [0, 0, 0, 0]
+    for k in worst:
+        assert worst[k] < tol[k], (k, worst)
+    return worst, n_excused

@@ -8,7 +8,8 @@ import torch
 from oracle import armor_oracle as O
 from paper_2510_05528_b200 import binding as Bd
 from paper_2510_05528_b200 import inputs
-from tests.helpers import DEV, TOL, dev, excused_blocks, host, load_state, mask_block_diffs, rel
+from tests.helpers import (DEV, TOL, dev, excused_blocks, host, load_state, make, mask_block_diffs, rel,
+                           run_teacher_forced)
 
 pytestmark = pytest.mark.gpu
 
@@ -16,11 +17,6 @@ TINY = inputs.CONFIGS["tiny"]
 MID = TINY.with_(name="mid", d_out=384, d_in=512, d_block=128, n_tokens=6000, chunk_rows=2048, seed=11)
 PRECS = [Bd.PREC_SIMT, Bd.PREC_FP32X3, Bd.PREC_TF32]
 PNAME = {Bd.PREC_SIMT: "simt", Bd.PREC_FP32X3: "fp32x3", Bd.PREC_TF32: "tf32"}
-
-
-def make(cfg, precision, h_mode=Bd.H_FULL, **kw):
-    return Bd.ArmorContext(cfg.d_out, cfg.d_in, cfg.d_block, device=DEV, precision=precision, h_mode=h_mode,
-                           seed=cfg.seed, **kw)
 
 
 @pytest.fixture(scope="module")
@@ -136,52 +132,6 @@ def test_proxy_loss_matches_oracle(prec, h_mode, mid_data):
 
 
 # ------------------------------------------------------------------------- teacher-forced steps
-def run_teacher_forced(cfg, W, H32, prec, h_mode, n_steps, select=Bd.SELECT_L1_RANDOM, n_keep=2, m_group=4,
-                       s_step=Bd.S_EXACT, tol_scale=1.0, ab_step=Bd.AB_EXACT):
-    ctx = make(cfg, prec, h_mode, select_mode=select, n_keep=n_keep, m_group=m_group, s_step=s_step, ab_step=ab_step)
-    Hd = dev(H32)
-    st = ctx.init(dev(W), Hd)
-    oc = O.OracleConfig(cfg.d_block, h_mode=h_mode, seed=cfg.seed, select_mode=select, n_keep=n_keep,
-                        m_group=m_group, s_step=s_step, ab_step=ab_step)
-    Hq = H32.astype(np.float64)
-    Hw = O.weighting(Hq, h_mode)
-    Wn = W.astype(np.float64)
-    A, B, S, M = O.init(Wn, Hq, oc)
-    tol = {k: v * tol_scale for k, v in TOL[prec].items()}
-    n_excused = 0
-    worst = dict(A=0.0, B=0.0, S=0.0, loss=0.0)
-    for t in range(n_steps):
-        load_state(st, A, B, S, M, m_group)        # the GPU starts every step from the oracle's state
-        stats = ctx.bcd_step(st, Hd, t, 1)
-        sg = ctx.read_stats(stats)[0]
-        A, B, S, M, info = O.bcd_iteration(Wn, A, B, S, M, Hw, oc, t)
-        worst["A"] = max(worst["A"], rel(host(st.A), A))
-        worst["B"] = max(worst["B"], rel(host(st.B), B))
-        for k_gpu, k_or in (("loss_start", "start"), ("loss_A", "A"), ("loss_B", "B"), ("loss_S", "S")):
-            worst["loss"] = max(worst["loss"], abs(sg[k_gpu] - info.loss[k_or]) / info.loss[k_or])
-        assert abs(sg["tau_B"] - info.tau_B) <= 10 * tol["B"] * abs(info.tau_B) + 1e-6
-        assert abs(sg["tau_S"] - info.tau_S) <= 10 * tol["S"] * abs(info.tau_S) + 1e-12
-        assert sg["chol_failed"] == info.chol_failed == 0
-        # masks: identical outside blocks whose decision margin is below the threshold
-        diff = mask_block_diffs(host(st.M), M, cfg.d_block, m_group)
-        excused = excused_blocks(info, tol["margin"])
-        guard_close = abs(info.delta_L_mask) <= tol["margin"] * info.loss["S"]
-        if sg["mask_accepted"] != info.mask_accepted:
-            assert guard_close, "accept/reject differs although the guard was not marginal"
-            n_excused += len(diff)
-            continue
-        assert diff <= excused, f"step {t}: masks differ in blocks {sorted(diff - excused)} with a clear margin"
-        n_excused += len(diff)
-        if not diff:
-            worst["S"] = max(worst["S"], rel(host(st.S), S))
-            assert sg["groups_changed"] == info.groups_changed
-            worst["loss"] = max(worst["loss"], abs(sg["loss_mask"] - info.loss["mask"]) / info.loss["mask"])
-    assert ctx.device_status()[:4] == [0, 0, 0, 0]
-    for k in worst:
-        assert worst[k] < tol[k], (k, worst)
-    return worst, n_excused
-
-
 @pytest.mark.parametrize("h_mode", [Bd.H_FULL, Bd.H_DIAG])
 @pytest.mark.parametrize("prec", [Bd.PREC_SIMT, Bd.PREC_FP32X3], ids=PNAME.get)
 def test_teacher_forced_all_20_steps_of_the_tiny_config(prec, h_mode, tiny_data):
@@ -725,4 +675,80 @@ def test_block_products_on_both_paths(db, side, transpose):
         out = dev(D)                                   # addend in place: out = 1.5 * product - 0.5 * out
         Bd.armor_block_product(ctx.ctx, side, transpose, Qd, Xd, out, alpha=1.5, add=out, beta=-0.5, path=path)
         assert rel(host(out), 1.5 * ref - 0.5 * D) < tol
+    assert ctx.device_status()[:4] == [0, 0, 0, 0]
+
+
+# ------------------------------------------------------------------ the guard's rejection (full weighting)
+def overlapping_case(d_out, d_in, db, strength, n=4, seed=5):
+    """Four calibration tokens and wrapper blocks with nearly parallel columns: the group updates of one
+    iteration overlap so strongly that their joint change of the loss is positive in some iterations."""
+    cfg = inputs.LayerConfig("overlap", d_out, d_in, db, n, 4, seed=seed, n_outlier=2, outlier_scale=20.0, chunk_rows=32)
+    W = inputs.make_weight(cfg)
+    H32 = O.gram(inputs.make_activations(cfg)).astype(np.float32)
+    oc = O.OracleConfig(db, h_mode=O.FULL, seed=1, phases=O.PH_MASK)
+    Hq = H32.astype(np.float64)
+    A, B, S, M = O.init(W.astype(np.float64), Hq, oc)
+    A = inputs.coupled_blocks(d_out // db, db, strength).astype(np.float32).astype(np.float64)
+    return cfg, W, H32, oc, (A, B, S, M)
+
+
+@pytest.mark.parametrize("shape,prec", [((64, 256, 32, 0.3), Bd.PREC_SIMT), ((256, 512, 128, 0.5), Bd.PREC_SIMT),
+                                        ((256, 512, 128, 0.5), Bd.PREC_FP32X3)],
+                         ids=["simt-32", "simt-128", "fp32x3-128"])
+def test_guard_rejection_matches_oracle_and_leaves_the_state_alone(shape, prec):
+    """Iterations in which the oracle discards the group updates (and the accepted ones between them), sparse-core
+    phase only, teacher-forced.  A rejected iteration must report mask_accepted 0, the oracle's positive loss
+    change, loss_mask == loss_S, and leave S and M bit for bit as loaded.  A second iteration inside the same
+    call must still follow the oracle: the product T H_w carried from one iteration to the next may advance only
+    by accepted updates."""
+    cfg, W, H32, oc, (A, B, S, M) = overlapping_case(*shape)
+    ctx = Bd.ArmorContext(cfg.d_out, cfg.d_in, cfg.d_block, device=DEV, precision=prec, h_mode=Bd.H_FULL, seed=1,
+                          phases=Bd.PHASE_MASK)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    Hq = H32.astype(np.float64)
+    Wn = W.astype(np.float64)
+    tol = TOL[prec]
+    seen = {0: 0, 1: 0}
+    second_after_reject = 0
+    for t in range(7):
+        A1, B1, S1, M1, i1 = O.bcd_iteration(Wn, A, B, S, M, Hq, oc, t)
+        A2, B2, S2, M2, i2 = O.bcd_iteration(Wn, A1, B1, S1, M1, Hq, oc, t + 1)
+        marginal = any(abs(i.delta_L_mask) <= 10 * tol["margin"] * i.loss["start"] for i in (i1, i2))
+        # --- one iteration per call
+        load_state(st, A, B, S, M)
+        S_before, M_before = host(st.S).copy(), host(st.M).copy()
+        sg = ctx.read_stats(ctx.bcd_step(st, Hd, t, 1))[0]
+        assert abs(sg["loss_start"] - i1.loss["start"]) / i1.loss["start"] < tol["loss"]
+        if not marginal:
+            assert sg["mask_accepted"] == i1.mask_accepted
+            assert abs(sg["delta_L_mask"] - i1.delta_L_mask) <= 1e-3 * abs(i1.delta_L_mask)
+            seen[i1.mask_accepted] += 1
+            if not i1.mask_accepted:
+                assert sg["delta_L_mask"] > 0 and sg["groups_changed"] == 0
+                assert sg["loss_mask"] == sg["loss_S"] == sg["loss_start"]
+                assert np.array_equal(host(st.S), S_before) and np.array_equal(host(st.M), M_before)
+            else:
+                diff = mask_block_diffs(host(st.M), M1, cfg.d_block)
+                assert diff <= excused_blocks(i1, tol["margin"])
+                if not diff:
+                    assert rel(host(st.S), S1) < tol["S"] and sg["groups_changed"] == i1.groups_changed
+                    assert abs(sg["loss_mask"] - i1.loss["mask"]) / i1.loss["mask"] < tol["loss"]
+        # --- two iterations in one call from the same state
+        load_state(st, A, B, S, M)
+        s2 = ctx.read_stats(ctx.bcd_step(st, Hd, t, 2))
+        if not marginal:
+            assert [int(x) for x in s2["mask_accepted"]] == [i1.mask_accepted, i2.mask_accepted]
+            diff = mask_block_diffs(host(st.M), M2, cfg.d_block)
+            if diff <= (excused_blocks(i1, tol["margin"]) | excused_blocks(i2, tol["margin"])) and not diff:
+                assert rel(host(st.S), S2) < tol["S"]
+                assert abs(s2["loss_start"][1] - i2.loss["start"]) / i2.loss["start"] < tol["loss"]
+                assert abs(s2["delta_L_mask"][1] - i2.delta_L_mask) <= 1e-3 * abs(i2.delta_L_mask)
+                assert abs(s2["loss_mask"][1] - i2.loss["mask"]) / i2.loss["mask"] < tol["loss"]
+                second_after_reject += (i1.mask_accepted == 0)
+            # the tracked loss is the loss of the state the call left
+            assert abs(ctx.proxy_loss(st, Hd).item() - s2["loss_mask"][1]) / s2["loss_mask"][1] < 1e-4
+        A, B, S, M = A1, B1, S1, M1
+    assert seen[0] >= 1 and seen[1] >= 1, seen
+    assert second_after_reject >= 1
     assert ctx.device_status()[:4] == [0, 0, 0, 0]
