@@ -66,8 +66,12 @@ enum { ARMOR_AB_EXACT = 0, ARMOR_AB_GD = 1, ARMOR_AB_ADAM = 2 };
  *   FP32X3 : operands split into tf32 high and low parts, three tcgen05 passes
  *            accumulated in fp32 -- fp32-grade results (the parity mode);
  *   TF32   : one pass, operands rounded to tf32 (10-bit mantissa);
- *   SIMT   : fp32 CUDA-core reference path (slow; for debugging and checks). */
-enum { ARMOR_PREC_FP32X3 = 0, ARMOR_PREC_TF32 = 1, ARMOR_PREC_SIMT = 2 };
+ *   SIMT   : fp32 CUDA-core reference path (slow; for debugging and checks);
+ *   FP16X3 : operands scaled by exact powers of two into the fp16 range and split into fp16 high and low
+ *            parts (22 significant bits, as two tf32 parts), three kind::f16 passes at twice the tf32 rate,
+ *            the accumulator rescaled in the epilogue -- fp32-grade results like FP32X3.  The products
+ *            with the block-diagonal wrappers are the same in both modes. */
+enum { ARMOR_PREC_FP32X3 = 0, ARMOR_PREC_TF32 = 1, ARMOR_PREC_SIMT = 2, ARMOR_PREC_FP16X3 = 3 };
 enum { ARMOR_PHASE_A = 1, ARMOR_PHASE_B = 2, ARMOR_PHASE_S = 4, ARMOR_PHASE_MASK = 8 };
 enum { ARMOR_DTYPE_F32 = 0, ARMOR_DTYPE_BF16 = 1, ARMOR_DTYPE_BF16_SPARSE = 2 };
 

@@ -20,7 +20,7 @@ H_FULL, H_DIAG = 0, 1
 SELECT_L1_RANDOM, SELECT_L1_GREEDY, SELECT_UNIFORM_RANDOM, SELECT_L2_RANDOM = 0, 1, 2, 3
 S_EXACT, S_BETA = 0, 1
 AB_EXACT, AB_GD, AB_ADAM = 0, 1, 2
-PREC_FP32X3, PREC_TF32, PREC_SIMT = 0, 1, 2
+PREC_FP32X3, PREC_TF32, PREC_SIMT, PREC_FP16X3 = 0, 1, 2, 3
 PHASE_A, PHASE_B, PHASE_S, PHASE_MASK = 1, 2, 4, 8
 DTYPE_F32, DTYPE_BF16, DTYPE_BF16_SPARSE = 0, 1, 2
 

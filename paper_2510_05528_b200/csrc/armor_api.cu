@@ -35,7 +35,7 @@ armor_status check_config(const armor_config* cfg) {
       cfg->adam_beta2 >= 1.f || cfg->adam_eps < 0.f)
     return ARMOR_ERR_INVALID_ARG;
   if (cfg->ab_step == ARMOR_AB_GD && cfg->h_mode != ARMOR_H_DIAG) return ARMOR_ERR_UNSUPPORTED;
-  if (cfg->precision < ARMOR_PREC_FP32X3 || cfg->precision > ARMOR_PREC_SIMT) return ARMOR_ERR_INVALID_ARG;
+  if (cfg->precision < ARMOR_PREC_FP32X3 || cfg->precision > ARMOR_PREC_FP16X3) return ARMOR_ERR_INVALID_ARG;
   if (cfg->precision != ARMOR_PREC_SIMT) {
     // the tensor-core GEMM works on whole 128 x 128 tiles with K in steps of 32
     if (cfg->h_mode == ARMOR_H_FULL && (cfg->d_out % 128 || cfg->d_in % 128)) return ARMOR_ERR_UNSUPPORTED;
@@ -54,7 +54,7 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   const size_t wbytes = (size_t)wn * sizeof(float);
   const size_t hbytes = (size_t)cfg.d_in * cfg.d_in * sizeof(float);
   const bool tc = cfg.precision != ARMOR_PREC_SIMT;
-  const bool x3 = cfg.precision == ARMOR_PREC_FP32X3;
+  const bool x3 = cfg.precision == ARMOR_PREC_FP32X3 || cfg.precision == ARMOR_PREC_FP16X3;   // split operands
 #define TAKE(field, type, bytes)                         \
   do {                                                   \
     size_t off_ = L.take(bytes);                         \
@@ -91,11 +91,20 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   TAKE(Ysel, float*, (size_t)nbo_pad * nbi * kg * cfg.d_in * sizeof(float));
   if (c) c->nbo_pad = (int)nbo_pad;
   TAKE(colpart, double*, (size_t)64 * cfg.d_in * sizeof(double));
+  {
+    const int64_t dmax = cfg.d_out > cfg.d_in ? cfg.d_out : cfg.d_in;
+    TAKE(hpow, float*, (size_t)cfg.d_in * sizeof(float));
+    TAKE(gscale, float*, (size_t)cfg.d_in * sizeof(float));
+    TAKE(gmax, unsigned*, (size_t)cfg.d_in * sizeof(unsigned));
+    TAKE(rowscale, float*, (size_t)dmax * sizeof(float));
+    TAKE(rowscale2, float*, (size_t)dmax * sizeof(float));
+  }
   if (tc) {
     TAKE(gemm_slabs, float*, (size_t)160 * 128 * 256 * sizeof(float));
     if (c) c->gemm_slab_count = 160;
     TAKE(Xt_hi, float*, (size_t)cfg.d_in * GRAM_ROWS * sizeof(float));
-    if (x3) TAKE(Xt_lo, float*, (size_t)cfg.d_in * GRAM_ROWS * sizeof(float)); else if (c) c->Xt_lo = nullptr;
+    // (the fp16 mode keeps both 16-bit parts of the staged chunk in Xt_hi)
+    if (cfg.precision == ARMOR_PREC_FP32X3) TAKE(Xt_lo, float*, (size_t)cfg.d_in * GRAM_ROWS * sizeof(float)); else if (c) c->Xt_lo = nullptr;
   } else if (c) { c->Xt_hi = nullptr; c->Xt_lo = nullptr; c->gemm_slabs = nullptr; c->gemm_slab_count = 0; }
   const int64_t tiles = ((cfg.d_out + 127) / 128) * ((cfg.d_in + 127) / 128) + ((cfg.d_in + 127) / 128) * ((cfg.d_in + 127) / 128);
   const int64_t npart = tiles > ARMOR_DOT_BLOCKS ? tiles : ARMOR_DOT_BLOCKS;

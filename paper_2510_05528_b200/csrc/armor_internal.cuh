@@ -70,6 +70,10 @@ struct armor_ctx {
   // sparse-core update: per selected group z = delta^T B_j[rows of the group, :] and a = A_i[:, r]
   float *Zsel, *Acol, *Ysel;  // [nbi][nbo_pad][db], [nbo][nbi][db], [nbi][nbo_pad][d_in]
   int nbo_pad;                // nbo rounded up to a multiple of 32
+  // three-pass fp16 mode: column scales derived from diag(H), per-row output scales of the two operands,
+  // per-channel maxima and output scales of a Gram chunk
+  float *hpow, *rowscale, *rowscale2, *gscale;
+  unsigned* gmax;
   // Gram staging (transposed, split chunk of X)
   float *Xt_hi, *Xt_lo;
   int64_t gram_rows;  // rows of X staged per pass
@@ -166,6 +170,14 @@ armor_status gram_accumulate(armor_ctx* c, const void* X, int x_dtype, int64_t n
 armor_status apply_core(armor_ctx* c, const float* z1, const float* S, const void* packed, float* z2, int64_t n,
                         bool bf16, cudaStream_t s);
 
+// operand preparation of the three-pass fp16 mode (split_f16.cu)
+void launch_f16_prepare_H(armor_ctx* c, const float* H, cudaStream_t s);   // hpow, scaled H as fp16 hi | lo in Hlo
+void launch_f16_split_rows(armor_ctx* c, const float* in, int64_t ld, int64_t rows, int64_t cols, const float* colscale,
+                           float post, void* hi, void* lo, float* out_scale, cudaStream_t s);
+float f16_H_post_scale();
+armor_status launch_f16_gram_stage(armor_ctx* c, const void* X, int x_dtype, int64_t ldx, int64_t rows, int64_t cols,
+                                   void* Thi, void* Tlo, int64_t ldt, cudaStream_t s);
+
 // deterministic reductions (two stages, fixed order)
 void dot_to_ptr(armor_ctx* c, const float* x, const float* y, int64_t n, double* out, cudaStream_t s);
 void reduce_partials_to(armor_ctx* c, const double* part, int n, double* out, cudaStream_t s);
@@ -227,11 +239,14 @@ void launch_mask_carry_P(armor_ctx* c, float* P, cudaStream_t s);
 // passes == 3 uses the split operands (A, Alo, B, Blo).  Partial dot products of the output tile with up
 // to two W-shaped tensors go to dot partial buffers.
 struct TcGemm {
-  const float* A; const float* Alo; int64_t lda;
-  const float* B; const float* Blo; int64_t ldb;
+  const void* A; const void* Alo; int64_t lda;   // fp32 arrays (passes 1, 3) or 16-bit arrays (passes 0, 6)
+  const void* B; const void* Blo; int64_t ldb;
   float* C; int64_t ldc;
   int64_t M, N, K;
-  int passes;            // 1 or 3 tf32 passes on fp32 operands; 0: A and B are bf16 arrays (one kind::f16 pass)
+  int passes;            // 1 or 3 tf32 passes on fp32 operands; 0: A and B are 16-bit arrays (one kind::f16 pass);
+                         // 6: 16-bit high and low parts, three kind::f16 passes
+  int fp16;              // passes 0 / 6: the 16-bit type is fp16 (1) or bf16 (0)
+  const float* row_scale; const float* col_scale;   // both or neither: C = acc * row_scale[m] * col_scale[n]
   int64_t k_segment;     // K extent accumulated in tensor memory before it is folded into C (0: all of K)
   int accumulate;        // C += (read-modify-write) instead of C =
   int symmetric_lower;   // only the lower triangle (tiles with n0 <= m0, elements with column <= row) is computed (M == N)

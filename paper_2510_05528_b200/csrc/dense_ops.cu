@@ -1,6 +1,9 @@
 // Dense contractions of the ARMOR iteration, dispatched by the configured precision:
 // right-multiplication by the weighting H_w, the calibration Gram, and the core product of the
-// deployment form.  SIMT = fp32 CUDA cores; TF32 / FP32X3 = tcgen05 tensor cores (1 or 3 passes).
+// deployment form.  SIMT = fp32 CUDA cores; TF32 / FP32X3 = tcgen05 tensor cores (1 or 3 tf32 passes);
+// FP16X3 = three fp16 passes on operands scaled into the fp16 range (split_f16.cu).
+#include <cuda_fp16.h>
+
 #include "armor_internal.cuh"
 
 // The tensor-core accumulator adds with truncation, so a long run of same-sign terms drifts by about
@@ -12,6 +15,8 @@ armor_status prepare_H(armor_ctx* c, const float* H, cudaStream_t s) {
   launch_extract_hblocks(c, H, s);
   if (c->cfg.h_mode == ARMOR_H_FULL && c->cfg.precision == ARMOR_PREC_FP32X3)
     launch_split_hilo(c, H, nullptr, c->Hlo, c->d_in * c->d_in, s);
+  if (c->cfg.h_mode == ARMOR_H_FULL && c->cfg.precision == ARMOR_PREC_FP16X3)
+    launch_f16_prepare_H(c, H, s);
   return ARMOR_OK;
 }
 
@@ -37,11 +42,18 @@ armor_status rmul_H(armor_ctx* c, const float* in, const float* H, float* out, i
       // 32-bit operand, so the operand itself serves as its high part and only the remainder is written.
       launch_split_hilo(c, in, nullptr, c->Lo, rows * d_in, s);
       g.A = in; g.Alo = c->Lo; g.B = H; g.Blo = c->Hlo; g.passes = 3;
+    } else if (c->cfg.precision == ARMOR_PREC_FP16X3) {
+      // in . H = rowscale . [(in d) rho] [H / (d d^T) 2^12] . d : both factors as fp16 high and low parts
+      __half* ahi = reinterpret_cast<__half*>(c->Lo);
+      __half* hhi = reinterpret_cast<__half*>(c->Hlo);
+      launch_f16_split_rows(c, in, d_in, rows, d_in, c->hpow, f16_H_post_scale(), ahi, ahi + rows * d_in, c->rowscale, s);
+      g.A = ahi; g.Alo = ahi + rows * d_in; g.B = hhi; g.Blo = hhi + d_in * d_in; g.passes = 6; g.fp16 = 1;
+      g.row_scale = c->rowscale; g.col_scale = c->hpow;
     } else {
       g.A = in; g.B = H; g.passes = 1;
     }
     g.d1 = d1; g.d2 = d2;
-    g.k_segment = (g.passes == 3) ? K_SEGMENT : 0;   // one-pass tf32 rounding (2^-11) dwarfs the accumulator drift
+    g.k_segment = (g.passes >= 3) ? K_SEGMENT : 0;   // one-pass tf32 rounding (2^-11) dwarfs the accumulator drift
     g.part1 = d1 ? c->partials : nullptr;
     g.part2 = d2 ? c->partials + 4 * c->npart : nullptr;
     int tiles = 0;
@@ -75,6 +87,33 @@ armor_status gram_accumulate(armor_ctx* c, const void* Xv, int x_dtype, int64_t 
       g.M = (int)d_in; g.N = (int)d_in; g.K = (int)n; g.batch = 1; g.alpha = 1.f; g.beta = 1.f;
       launch_bgemm(c, g, s);
     }
+    return ARMOR_OK;
+  }
+  if (c->cfg.precision == ARMOR_PREC_FP16X3) {
+    // every chunk is scaled per channel into the fp16 range; bf16 activations are then exact in one fp16 part
+    __half* thi = reinterpret_cast<__half*>(c->Xt_hi);
+    __half* tlo = thi + d_in * c->gram_rows;
+    const size_t esz = bf16 ? 2 : 4;
+    for (int64_t r0 = 0; r0 < n_rows; r0 += c->gram_rows) {
+      const int64_t n = n_rows - r0 < c->gram_rows ? n_rows - r0 : c->gram_rows;
+      const int64_t kpad = (n + 63) / 64 * 64;
+      armor_status st = launch_f16_gram_stage(c, static_cast<const char*>(Xv) + (size_t)(r0 * ldx) * esz, x_dtype, ldx, n,
+                                              d_in, thi, tlo, kpad, s);
+      if (st != ARMOR_OK) return st;
+      TcGemm g{};
+      g.A = thi; g.Alo = tlo; g.lda = kpad;
+      g.B = thi; g.Blo = tlo; g.ldb = kpad;
+      g.C = H; g.ldc = d_in;
+      g.M = d_in; g.N = d_in; g.K = kpad;
+      g.passes = bf16 ? 0 : 6; g.fp16 = 1;
+      g.row_scale = c->gscale; g.col_scale = c->gscale;
+      g.accumulate = 1;
+      g.symmetric_lower = 1;
+      g.k_segment = K_SEGMENT;
+      st = launch_tc_gemm(c, g, nullptr, s);
+      if (st != ARMOR_OK) return st;
+    }
+    launch_mirror_lower(c, H, d_in, s);
     return ARMOR_OK;
   }
   // bf16 values are exact in tf32: one tensor-core pass gives exact products
@@ -141,9 +180,17 @@ armor_status apply_core(armor_ctx* c, const float* z1, const float* S, const voi
     launch_split_hilo(c, z1, nullptr, c->Lo, n * d_in, s);
     launch_split_hilo(c, S, nullptr, c->U, c->wn, s);
     g.A = z1; g.Alo = c->Lo; g.B = S; g.Blo = c->U; g.passes = 3;
+  } else if (c->cfg.precision == ARMOR_PREC_FP16X3) {
+    // rows of z1 (tokens) and rows of S (outputs) each scaled by their own power of two
+    __half* ahi = reinterpret_cast<__half*>(c->Lo);
+    __half* shi = reinterpret_cast<__half*>(c->U);
+    launch_f16_split_rows(c, z1, d_in, n, d_in, nullptr, 1.f, ahi, ahi + n * d_in, c->rowscale, s);
+    launch_f16_split_rows(c, S, d_in, d_out, d_in, nullptr, 1.f, shi, shi + c->wn, c->rowscale2, s);
+    g.A = ahi; g.Alo = ahi + n * d_in; g.B = shi; g.Blo = shi + c->wn; g.passes = 6; g.fp16 = 1;
+    g.row_scale = c->rowscale; g.col_scale = c->rowscale2;
   } else {
     g.A = z1; g.B = S; g.passes = 1;
   }
-  g.k_segment = (g.passes == 3) ? K_SEGMENT : 0;
+  g.k_segment = (g.passes >= 3) ? K_SEGMENT : 0;
   return launch_tc_gemm(c, g, nullptr, s);
 }

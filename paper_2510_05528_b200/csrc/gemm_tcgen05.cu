@@ -12,6 +12,11 @@
 //                             product writes its lower triangle only, the caller mirrors it once at the end)
 // passes == 3: every operand is given as a tf32-exact high part and an fp32 low part; the three products
 // hi*hi, lo*hi, hi*lo are accumulated into the same fp32 accumulator (error-compensated tf32, fp32-grade).
+// passes == 6: the same three products on fp16 high and low parts (kind::f16, twice the tf32 issue rate, half
+// the operand bytes).  Two fp16 parts carry 22 significant bits like two tf32 parts, but only 5 exponent bits,
+// so the caller scales rows of the operands by powers of two into the fp16 range beforehand and the epilogue
+// multiplies the accumulator by the inverse scales (a per-row and a per-column vector): every scaling is
+// exact, the result is fp32-grade.
 // Every wait is bounded: a wait that runs out raises a status word and the CTA leaves through the common
 // exit that frees its tensor memory.
 #include "tc_common.cuh"
@@ -35,6 +40,8 @@ struct Params {
   int kt_seg;            // k-tiles accumulated in tensor memory before the epilogue folds them into C
   const float* d1; const float* d2;
   double* part1; double* part2;
+  const float* row_scale; const float* col_scale;   // optional powers of two the accumulator is multiplied by
+  int f16;               // 16-bit operands are fp16 (1) or bf16 (0)
   int32_t* status;
   // Tail split: tiles [split_first, n_tiles_total) are cut into split_parts pieces along K, each piece a work
   // item of its own that writes a 128 x 256 slab of partial sums; a second kernel adds the slabs.  This fills
@@ -54,12 +61,13 @@ __device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t addr) {
   return d;
 }
 
-// fp32 accumulate, both operands K-major, M = 128, N = 256; operands tf32 (kind::tf32) or bf16 (kind::f16).
-__device__ __forceinline__ uint32_t instr_desc(bool bf16) {
+// fp32 accumulate, both operands K-major, M = 128, N = 256; operand format 0: fp16, 1: bf16 (both kind::f16),
+// 2: tf32 (kind::tf32).
+__device__ __forceinline__ uint32_t instr_desc(uint32_t fmt) {
   uint32_t d = 0;
   d |= 1u << 4;                   // D format: F32
-  d |= (bf16 ? 1u : 2u) << 7;     // A format: BF16 / TF32
-  d |= (bf16 ? 1u : 2u) << 10;    // B format: BF16 / TF32
+  d |= fmt << 7;                  // A format
+  d |= fmt << 10;                 // B format
   d |= (uint32_t)(BN >> 3) << 17; // N
   d |= (uint32_t)(BM >> 4) << 24; // M
   return d;
@@ -112,8 +120,10 @@ template <int PASSES>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapAlo,
                const __grid_constant__ CUtensorMap mapB, const __grid_constant__ CUtensorMap mapBlo, const Params p) {
-  constexpr int STAGE_BYTES = (PASSES == 3 ? 2 : 1) * (A_BYTES + B_BYTES);
-  constexpr int STAGES = (PASSES == 3) ? 2 : 4;
+  constexpr bool SPLIT = (PASSES == 3 || PASSES == 6);   // operands come as high and low parts
+  constexpr bool H16 = (PASSES == 0 || PASSES == 6);     // 16-bit operands (kind::f16)
+  constexpr int STAGE_BYTES = (SPLIT ? 2 : 1) * (A_BYTES + B_BYTES);
+  constexpr int STAGES = SPLIT ? 2 : 4;
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment for the swizzled tiles
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -124,7 +134,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]);
   const uint32_t tfull0 = smem_u32(&bars[2 * STAGES]), tempty0 = smem_u32(&bars[2 * STAGES + 2]);
-  constexpr int BKE = (PASSES == 0) ? 64 : 32;      // elements of K per 128-byte row: bf16 or fp32
+  constexpr int BKE = H16 ? 64 : 32;                // elements of K per 128-byte row: 16-bit or fp32
   const int kt_total = (int)((p.K + BKE - 1) / BKE);
 
   if (threadIdx.x == 0) {
@@ -161,10 +171,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
           uint32_t dst = smem_u32(smem + (size_t)stage * STAGE_BYTES);
           tma_load_2d(dst, &mapA, kt * BKE, mt * BM, fb);
           dst += A_BYTES;
-          if (PASSES == 3) { tma_load_2d(dst, &mapAlo, kt * BKE, mt * BM, fb); dst += A_BYTES; }
+          if (SPLIT) { tma_load_2d(dst, &mapAlo, kt * BKE, mt * BM, fb); dst += A_BYTES; }
           tma_load_2d(dst, &mapB, kt * BKE, nt * BN, fb);
           dst += B_BYTES;
-          if (PASSES == 3) tma_load_2d(dst, &mapBlo, kt * BKE, nt * BN, fb);
+          if (SPLIT) tma_load_2d(dst, &mapBlo, kt * BKE, nt * BN, fb);
           ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -182,7 +192,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = instr_desc(PASSES == 0);
+      const uint32_t idesc = instr_desc(H16 ? (p.f16 ? 0u : 1u) : 2u);
       int stage = 0; uint32_t phase = 0;
       int local = 0;   // (tile, K segment) items handled so far: selects the accumulator buffer
       bool ok = true;
@@ -201,7 +211,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
             tc_fence_after();
             const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
             const uint32_t sa_lo = sa + A_BYTES;
-            const uint32_t sb = sa + (PASSES == 3 ? 2 : 1) * A_BYTES;
+            const uint32_t sb = sa + (SPLIT ? 2 : 1) * A_BYTES;
             const uint32_t sb_lo = sb + B_BYTES;
 #pragma unroll
             for (int k = 0; k < BK / 8; ++k) {
@@ -212,6 +222,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
                 umma_tf32(tacc, dal, dbm, idesc, acc);
                 umma_tf32(tacc, da, dbl, idesc, 1);
                 umma_tf32(tacc, da, dbm, idesc, 1);
+              } else if (PASSES == 6) {
+                const uint64_t dal = smem_desc_k_sw128(sa_lo + k * 32), dbl = smem_desc_k_sw128(sb_lo + k * 32);
+                umma_bf16(tacc, dal, dbm, idesc, acc);
+                umma_bf16(tacc, da, dbl, idesc, 1);
+                umma_bf16(tacc, da, dbm, idesc, 1);
               } else if (PASSES == 0) {
                 umma_bf16(tacc, da, dbm, idesc, acc);
               } else {
@@ -293,6 +308,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
           for (int cidx = 0; cidx < 32; ++cidx) tilebuf[lane * 33 + cidx] = __uint_as_float(r[cidx]);
           __syncwarp();
           const int64_t col = col0 + lane;
+          const float cscale = p.col_scale ? p.col_scale[col] : 1.f;
           float f1 = 0.f, f2 = 0.f;
 #pragma unroll 1
           for (int r0 = 0; r0 < 32; r0 += RB) {
@@ -303,6 +319,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
               const int64_t grow = row_base + r0 + j;
               keep[j] = grow < p.M && (!p.symmetric_lower || col <= grow);
               x[j] = tilebuf[(r0 + j) * 33 + lane];
+              if (p.row_scale) x[j] *= (grow < p.M ? p.row_scale[grow] : 1.f) * cscale;
               o[j] = (accum && keep[j]) ? p.C[grow * p.ldc + col] : 0.f;
             }
             if (last && p.d1) {
@@ -365,6 +382,11 @@ __global__ void __launch_bounds__(256) tc_gemm_fixup_kernel(const Params p) {
       const float4 w = *reinterpret_cast<const float4*>(slab0 + (int64_t)k * (BM * BN) + (int64_t)r * BN + c4);
       v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
     }
+    if (p.row_scale) {
+      const float rs = p.row_scale[grow];
+      const float4 cs = *reinterpret_cast<const float4*>(p.col_scale + gcol);
+      v.x *= rs * cs.x; v.y *= rs * cs.y; v.z *= rs * cs.z; v.w *= rs * cs.w;
+    }
     float* cp = p.C + grow * p.ldc + gcol;
     if (p.accumulate) {
       const float4 o = *reinterpret_cast<const float4*>(cp);
@@ -397,16 +419,17 @@ __global__ void __launch_bounds__(256) tc_gemm_fixup_kernel(const Params p) {
 
 // ------------------------------------------------------------------ host side
 // [rows][K] fp32, leading dimension ld: box = BK x box_rows, 128-byte swizzle, zero fill out of bounds.
-bool make_map(CUtensorMap* map, const float* base, int64_t rows, int64_t K, int64_t ld, int box_rows,
-              bool bf16 = false) {
+// bits16: 0 fp32 elements, 1 bf16, 2 fp16
+bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t K, int64_t ld, int box_rows, int bits16 = 0) {
   PFN_cuTensorMapEncodeTiled_v12000 enc = get_encode();
   if (!enc) return false;
   cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)ld * (bf16 ? 2 : 4)};
-  cuuint32_t box[2] = {(cuuint32_t)(bf16 ? 64 : BK), (cuuint32_t)box_rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * (bits16 ? 2 : 4)};
+  cuuint32_t box[2] = {(cuuint32_t)(bits16 ? 64 : BK), (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = enc(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
-                   const_cast<float*>(base), dims, strides, box, estr,
+  const CUtensorMapDataType dt = bits16 == 0 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                 : bits16 == 1 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+  CUresult r = enc(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
@@ -415,17 +438,20 @@ bool make_map(CUtensorMap* map, const float* base, int64_t rows, int64_t K, int6
 template <int PASSES>
 armor_status launch_impl(armor_ctx* c, const TcGemm& g, Params p, cudaStream_t s) {
   CUtensorMap mA, mAlo, mB, mBlo;
-  if (!make_map(&mA, g.A, g.M, g.K, g.lda, BM, PASSES == 0)) return ARMOR_ERR_CUDA;
-  if (!make_map(&mB, g.B, g.N, g.K, g.ldb, BN, PASSES == 0)) return ARMOR_ERR_CUDA;
-  if (PASSES == 3) {
-    if (!make_map(&mAlo, g.Alo, g.M, g.K, g.lda, BM)) return ARMOR_ERR_CUDA;
-    if (!make_map(&mBlo, g.Blo, g.N, g.K, g.ldb, BN)) return ARMOR_ERR_CUDA;
+  constexpr bool SPLIT = (PASSES == 3 || PASSES == 6);
+  constexpr bool H16 = (PASSES == 0 || PASSES == 6);
+  const int bits16 = H16 ? (g.fp16 ? 2 : 1) : 0;
+  if (!make_map(&mA, g.A, g.M, g.K, g.lda, BM, bits16)) return ARMOR_ERR_CUDA;
+  if (!make_map(&mB, g.B, g.N, g.K, g.ldb, BN, bits16)) return ARMOR_ERR_CUDA;
+  if (SPLIT) {
+    if (!make_map(&mAlo, g.Alo, g.M, g.K, g.lda, BM, bits16)) return ARMOR_ERR_CUDA;
+    if (!make_map(&mBlo, g.Blo, g.N, g.K, g.ldb, BN, bits16)) return ARMOR_ERR_CUDA;
   } else {
     mAlo = mA;
     mBlo = mB;
   }
-  constexpr int STAGE_BYTES = (PASSES == 3 ? 2 : 1) * (A_BYTES + B_BYTES);
-  constexpr int STAGES = (PASSES == 3) ? 2 : 4;
+  constexpr int STAGE_BYTES = (SPLIT ? 2 : 1) * (A_BYTES + B_BYTES);
+  constexpr int STAGES = SPLIT ? 2 : 4;
   constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024 + 4 * 32 * 33 * sizeof(float);
   static bool attr = false;
   if (!attr) {
@@ -441,7 +467,7 @@ armor_status launch_impl(armor_ctx* c, const TcGemm& g, Params p, cudaStream_t s
   }
   // tail split: the tiles of the last, partly filled wave are cut along K so that their pieces fill the wave
   p.split_first = p.n_tiles_total; p.split_parts = 1; p.n_items = p.n_tiles_total; p.slabs = c->gemm_slabs;
-  const int kt_total = (int)((p.K + (PASSES == 0 ? 64 : BK) - 1) / (PASSES == 0 ? 64 : BK));
+  const int kt_total = (int)((p.K + (H16 ? 64 : BK) - 1) / (H16 ? 64 : BK));
   const int rem = p.n_tiles_total % n_sm;
   if (c->gemm_slabs && !p.symmetric_lower && rem > 0 && p.ldc % 4 == 0 && p.N % 4 == 0) {
     int parts = n_sm / rem;
@@ -482,7 +508,9 @@ bool tc_gemm_shape_ok(int64_t M, int64_t N, int64_t K) {
 
 armor_status launch_tc_gemm(armor_ctx* c, const TcGemm& g, int* n_tiles, cudaStream_t s) {
   if (!tc_gemm_shape_ok(g.M, g.N, g.K)) return ARMOR_ERR_UNSUPPORTED;
-  if ((g.lda % (g.passes == 0 ? 8 : 4)) || (g.ldb % (g.passes == 0 ? 8 : 4)) || (g.ldc % 4)) return ARMOR_ERR_UNSUPPORTED;
+  const bool h16 = (g.passes == 0 || g.passes == 6);
+  if ((g.lda % (h16 ? 8 : 4)) || (g.ldb % (h16 ? 8 : 4)) || (g.ldc % 4)) return ARMOR_ERR_UNSUPPORTED;
+  if ((g.row_scale == nullptr) != (g.col_scale == nullptr)) return ARMOR_ERR_INVALID_ARG;
   if (g.symmetric_lower && g.M != g.N) return ARMOR_ERR_INVALID_ARG;
   Params p{};
   p.C = g.C; p.ldc = g.ldc; p.M = g.M; p.N = g.N; p.K = g.K;
@@ -500,12 +528,14 @@ armor_status launch_tc_gemm(armor_ctx* c, const TcGemm& g, int* n_tiles, cudaStr
   }
   p.accumulate = g.accumulate; p.symmetric_lower = g.symmetric_lower;
   p.d1 = g.d1; p.d2 = g.d2; p.part1 = g.part1; p.part2 = g.part2;
+  p.row_scale = g.row_scale; p.col_scale = g.col_scale; p.f16 = g.fp16;
   p.status = c->status;
-  const int bke = (g.passes == 0) ? 64 : BK;
+  const int bke = h16 ? 64 : BK;
   p.kt_seg = g.k_segment > 0 ? (int)((g.k_segment + bke - 1) / bke) : (int)((g.K + bke - 1) / bke);
   if (p.kt_seg < 1) p.kt_seg = 1;
   if (n_tiles) *n_tiles = p.n_tiles_total;
   if (g.passes == 3) return launch_impl<3>(c, g, p, s);
+  if (g.passes == 6) return launch_impl<6>(c, g, p, s);
   if (g.passes == 0) return launch_impl<0>(c, g, p, s);
   return launch_impl<1>(c, g, p, s);
 }

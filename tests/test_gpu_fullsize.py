@@ -30,10 +30,11 @@ def layer():
     return ctx, W, H
 
 
-def test_gram_full_token_count_on_sampled_entries():
+@pytest.mark.parametrize("prec", [Bd.PREC_FP32X3, Bd.PREC_FP16X3], ids=["fp32x3", "fp16x3"])
+def test_gram_full_token_count_on_sampled_entries(prec):
     """All 262,144 tokens through armor_gram; 96 sampled entries (diagonal, outlier rows, random pairs)
     recomputed in fp64 straight from the activations."""
-    ctx = Bd.ArmorContext(CFG.d_out, CFG.d_in, CFG.d_block, device=DEV, precision=Bd.PREC_FP32X3, seed=CFG.seed)
+    ctx = Bd.ArmorContext(CFG.d_out, CFG.d_in, CFG.d_block, device=DEV, precision=prec, seed=CFG.seed)
     H = ctx.new_gram()
     scales_np = inputs.channel_scales(CFG)
     scales = torch.from_numpy(scales_np)
@@ -108,15 +109,16 @@ def test_loss_and_first_iteration_blocks(layer):
     assert 0.5 < sgB["tau_B"] < 1.5 and sgB["loss_B"] < sgB["loss_start"]
 
 
-def test_three_teacher_forced_iterations_at_full_size(layer):
+@pytest.mark.parametrize("prec", [Bd.PREC_FP32X3, Bd.PREC_FP16X3], ids=["fp32x3", "fp16x3"])
+def test_three_teacher_forced_iterations_at_full_size(prec, layer):
     """Whole iterations at 4096 x 4096 in the mode the benchmark times, each started from the oracle's state:
     A, B, S, every tracked loss, both step lengths and the accept flag against the oracle; masks identical
     outside the blocks whose selection or mask decision was closer than the 1e-5 margin (their number is
     printed).  This is where the 1,024-block selection grid, the guard's thin product over 32 row-blocks, the
     carried product over 32 column-blocks and the tail-split dense product meet the oracle."""
     ctx, W, H = layer
-    worst, n_excused = run_teacher_forced(CFG, W, host(H), Bd.PREC_FP32X3, Bd.H_FULL, 3)
-    print(f"llama7b_attn fp32x3, 3 teacher-forced iterations: worst rel err {worst}; "
+    worst, n_excused = run_teacher_forced(CFG, W, host(H), prec, Bd.H_FULL, 3)
+    print(f"llama7b_attn precision {prec}, 3 teacher-forced iterations: worst rel err {worst}; "
           f"blocks differing under the margin: {n_excused} of {3 * 32 * 32}")
     assert n_excused <= 6
 

@@ -15,8 +15,8 @@ pytestmark = pytest.mark.gpu
 
 TINY = inputs.CONFIGS["tiny"]
 MID = TINY.with_(name="mid", d_out=384, d_in=512, d_block=128, n_tokens=6000, chunk_rows=2048, seed=11)
-PRECS = [Bd.PREC_SIMT, Bd.PREC_FP32X3, Bd.PREC_TF32]
-PNAME = {Bd.PREC_SIMT: "simt", Bd.PREC_FP32X3: "fp32x3", Bd.PREC_TF32: "tf32"}
+PRECS = [Bd.PREC_SIMT, Bd.PREC_FP32X3, Bd.PREC_TF32, Bd.PREC_FP16X3]
+PNAME = {Bd.PREC_SIMT: "simt", Bd.PREC_FP32X3: "fp32x3", Bd.PREC_TF32: "tf32", Bd.PREC_FP16X3: "fp16x3"}
 
 
 @pytest.fixture(scope="module")
@@ -133,7 +133,7 @@ def test_proxy_loss_matches_oracle(prec, h_mode, mid_data):
 
 # ------------------------------------------------------------------------- teacher-forced steps
 @pytest.mark.parametrize("h_mode", [Bd.H_FULL, Bd.H_DIAG])
-@pytest.mark.parametrize("prec", [Bd.PREC_SIMT, Bd.PREC_FP32X3], ids=PNAME.get)
+@pytest.mark.parametrize("prec", [Bd.PREC_SIMT, Bd.PREC_FP32X3, Bd.PREC_FP16X3], ids=PNAME.get)
 def test_teacher_forced_all_20_steps_of_the_tiny_config(prec, h_mode, tiny_data):
     W, X, H32 = tiny_data
     worst, n_excused = run_teacher_forced(TINY, W, H32, prec, h_mode, TINY.n_iters)
@@ -693,8 +693,8 @@ def overlapping_case(d_out, d_in, db, strength, n=4, seed=5):
 
 
 @pytest.mark.parametrize("shape,prec", [((64, 256, 32, 0.3), Bd.PREC_SIMT), ((256, 512, 128, 0.5), Bd.PREC_SIMT),
-                                        ((256, 512, 128, 0.5), Bd.PREC_FP32X3)],
-                         ids=["simt-32", "simt-128", "fp32x3-128"])
+                                        ((256, 512, 128, 0.5), Bd.PREC_FP32X3), ((256, 512, 128, 0.5), Bd.PREC_FP16X3)],
+                         ids=["simt-32", "simt-128", "fp32x3-128", "fp16x3-128"])
 def test_guard_rejection_matches_oracle_and_leaves_the_state_alone(shape, prec):
     """Iterations in which the oracle discards the group updates (and the accepted ones between them), sparse-core
     phase only, teacher-forced.  A rejected iteration must report mask_accepted 0, the oracle's positive loss
