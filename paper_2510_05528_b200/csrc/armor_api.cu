@@ -128,7 +128,7 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
     TAKE(mS, float*, wbytes); TAKE(vS, float*, wbytes);
   } else if (c) { c->mA = c->vA = c->mB = c->vB = c->mS = c->vS = nullptr; }
   TAKE(sc, double*, SC_COUNT * sizeof(double));
-  TAKE(partials, double*, (size_t)8 * npart * sizeof(double));
+  TAKE(partials, double*, (size_t)16 * npart * sizeof(double));
   const int64_t nbmax = nbo > nbi ? nbo : nbi;
   TAKE(partblk, double*, (size_t)(4 * nbmax > nbo * nbi * kg ? 4 * nbmax : nbo * nbi * kg) * sizeof(double));
   TAKE(quadpart, double*, (size_t)nbo * nbi * kg * sizeof(double));
@@ -150,9 +150,11 @@ inline cudaStream_t cs(armor_stream_t s) { return reinterpret_cast<cudaStream_t>
 void rowblock_grams(armor_ctx* c, const float* P, const float* P2, const float* T, float* G, float* G2, cudaStream_t s) {
   // G_i = P_i T_i^T, G2_i = P2_i T_i^T  (contraction over d_in), batch over row-blocks i; P == nullptr: G2 only
   const int db = c->db;
-  if (g_tc_blocks && tc_gram_ok(c) && (!P || tc_rowblock_gram(c, P, T, G, s) == ARMOR_OK) &&
-      tc_rowblock_gram(c, P2, T, G2, s) == ARMOR_OK)
-    return;
+  if (c->tc_blocks && tc_gram_ok(c)) {
+    armor_status st = P ? tc_rowblock_gram(c, P, T, G, s) : ARMOR_OK;
+    if (st == ARMOR_OK) st = tc_rowblock_gram(c, P2, T, G2, s);
+    if (tc_done(c, st)) return;
+  }
   if (!P) { P = P2; G = G2; }   // fallback kernel: the same Gram twice into the same place
   BGemm g{};
   g.A = P; g.sAb = (int64_t)db * c->d_in; g.sAm = c->d_in; g.sAk = 1;
@@ -166,9 +168,11 @@ void rowblock_grams(armor_ctx* c, const float* P, const float* P2, const float* 
 void colblock_grams(armor_ctx* c, const float* U, const float* Y, const float* Y2, float* Cm, float* Cm2, cudaStream_t s) {
   // C_j = U_j^T Y_j, C2_j = U_j^T Y2_j  (contraction over d_out), batch over column-blocks j; Y == nullptr: C2 only
   const int db = c->db;
-  if (g_tc_blocks && tc_gram_ok(c) && (!Y || tc_colblock_gram(c, U, Y, Cm, s) == ARMOR_OK) &&
-      tc_colblock_gram(c, U, Y2, Cm2, s) == ARMOR_OK)
-    return;
+  if (c->tc_blocks && tc_gram_ok(c)) {
+    armor_status st = Y ? tc_colblock_gram(c, U, Y, Cm, s) : ARMOR_OK;
+    if (st == ARMOR_OK) st = tc_colblock_gram(c, U, Y2, Cm2, s);
+    if (tc_done(c, st)) return;
+  }
   if (!Y) { Y = Y2; Cm = Cm2; }
   BGemm g{};
   g.A = U; g.sAb = db; g.sAm = 1; g.sAk = c->d_in;
@@ -225,11 +229,11 @@ armor_status residual_and_loss(armor_ctx* c, const float* W, const float* H, con
   // exact_products: the two wrapper products on the fp32 CUDA-core kernel, whose products with 0 and 1 are
   // exact, so that E vanishes exactly where W = A S B term by term (identity wrappers at the initialisation);
   // the three-pass tensor-core product carries 22 bits of each operand
-  const int saved = g_tc_blocks;
-  if (exact_products) g_tc_blocks = 0;
+  const int saved = c->tc_blocks;
+  if (exact_products) c->tc_blocks = 0;
   bd_right(c, S, B, false, c->T, c->d_out, c->d_in, 1.f, nullptr, 0.f, s);      // T = S B
   bd_left(c, A, false, c->T, c->E, c->d_out, c->d_in, -1.f, W, 1.f, s);         // E = W - A T
-  g_tc_blocks = saved;
+  c->tc_blocks = saved;
   return rmul_H(c, c->E, H, c->EH, c->d_out, c->E, out, nullptr, nullptr, s);   // EH = E H_w, L = <EH, E>
 }
 
@@ -276,6 +280,13 @@ armor_status armor_create(armor_ctx** out, const armor_config* cfg, void* d_work
   c->db = cfg->d_block; c->nbo = (int)(cfg->d_out / cfg->d_block); c->nbi = (int)(cfg->d_in / cfg->d_block);
   c->ws = static_cast<char*>(d_workspace); c->ws_bytes = bytes;
   c->launches = 0;
+  c->tc_blocks = 1;
+  c->host_err = ARMOR_OK;
+  if (cudaGetDevice(&c->device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess || c->n_sm < 1) {
+    delete c;
+    return ARMOR_ERR_CUDA;
+  }
   c->kg = cfg->mask_groups > 0 ? cfg->mask_groups : 1;
   c->h_cached = nullptr;
   c->timing_on = 0; c->timing_n = 0; c->ev_beg = nullptr; c->ev_end = nullptr; c->ev_created = 0; c->timing_flops = 0.0;
@@ -299,13 +310,14 @@ int64_t armor_launch_count(const armor_ctx* c) { return c ? c->launches : -1; }
 
 armor_status armor_gemm_timing_enable(armor_ctx* c, int32_t enable) {
   if (!c) return ARMOR_ERR_INVALID_ARG;
-  if (enable && !c->ev_beg) {
-    c->ev_beg = new (std::nothrow) cudaEvent_t[ARMOR_MAX_TIMED];
-    c->ev_end = new (std::nothrow) cudaEvent_t[ARMOR_MAX_TIMED];
+  if (enable && c->ev_created < ARMOR_MAX_TIMED) {
+    if (!c->ev_beg) c->ev_beg = new (std::nothrow) cudaEvent_t[ARMOR_MAX_TIMED];
+    if (!c->ev_end) c->ev_end = new (std::nothrow) cudaEvent_t[ARMOR_MAX_TIMED];
     if (!c->ev_beg || !c->ev_end) return ARMOR_ERR_INVALID_ARG;
-    for (int i = 0; i < ARMOR_MAX_TIMED; ++i) {
-      if (cudaEventCreate(&c->ev_beg[i]) != cudaSuccess || cudaEventCreate(&c->ev_end[i]) != cudaSuccess)
-        return ARMOR_ERR_CUDA;
+    // (an earlier call may have stopped part of the way: continue from the pairs that exist)
+    for (int i = c->ev_created; i < ARMOR_MAX_TIMED; ++i) {
+      if (cudaEventCreate(&c->ev_beg[i]) != cudaSuccess) return ARMOR_ERR_CUDA;
+      if (cudaEventCreate(&c->ev_end[i]) != cudaSuccess) { cudaEventDestroy(c->ev_beg[i]); return ARMOR_ERR_CUDA; }
       c->ev_created = i + 1;
     }
   }
@@ -352,7 +364,7 @@ armor_status armor_init(armor_ctx* c, const float* d_W, const float* d_H, float*
   if (c->cfg.normalize && (!d_r1 || !d_r2)) return ARMOR_ERR_INVALID_ARG;
   launch_init(c, d_W, d_H, d_Wbar, d_r1, d_r2, d_A, d_B, d_S, d_M, cs(stream));
   if (reset_adam(c, cs(stream)) != ARMOR_OK) return ARMOR_ERR_CUDA;
-  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+  return finish_call(c);
 }
 
 armor_status armor_proxy_loss(armor_ctx* c, const float* W, const float* H, const float* A, const float* B,
@@ -363,7 +375,7 @@ armor_status armor_proxy_loss(armor_ctx* c, const float* W, const float* H, cons
   if (st != ARMOR_OK) return st;
   st = residual_and_loss(c, W, H, A, B, S, d_loss, s);
   if (st != ARMOR_OK) return st;
-  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+  return finish_call(c);
 }
 
 armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float* A, float* B, float* S, uint8_t* M,
@@ -553,10 +565,10 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       }
       if (carry_P && it + 1 < n_iters) launch_mask_carry_P(c, c->P, s);              // P += dS B H_w (if accepted)
     } else {
-      launch_stage(c, is, 4, nullptr, 0, 0, s);
+      launch_stage(c, is, 5, nullptr, 0, 0, s);
     }
   }
-  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+  return finish_call(c);
 }
 
 // x -> y = A (S (B x)) in chunks of tokens; `packed` non-null: the core comes packed for the sparse tensor cores
@@ -596,7 +608,7 @@ static armor_status apply_impl(armor_ctx* c, const float* A, const float* B, con
     if (bf16) launch_f32_to_bf16(c, yc, r2, static_cast<char*>(d_y) + (size_t)(t0 * d_out) * esz, n, d_out, s);
     else if (r2) launch_scale_rows_cols(c, yc, r2, nullptr, yc, n, d_out, s);
   }
-  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+  return finish_call(c);
 }
 
 armor_status armor_apply(armor_ctx* c, const float* A, const float* B, const float* S, const uint8_t* M,
@@ -637,7 +649,7 @@ armor_status armor_pack_core(armor_ctx* c, const float* S, const uint8_t* M, voi
   if (!tc_sparse_ok(c)) return ARMOR_ERR_UNSUPPORTED;
   char* buf = static_cast<char*>(d_packed);
   launch_compress_24(c, S, M, buf, buf + tc_sparse_values_bytes(c), cs(stream));
-  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+  return finish_call(c);
 }
 
 armor_status armor_apply_packed(armor_ctx* c, const float* A, const float* B, const void* d_packed, const float* r1,
@@ -675,7 +687,7 @@ armor_status armor_pack_layer(armor_ctx* c, const float* A, const float* B, cons
   launch_compress_24(c, S, M, buf, buf + tc_sparse_values_bytes(c), s);
   launch_pack_blocks(c, B, nullptr, r1, buf + layer_off_B(c), c->nbi, s);   // B's columns carry r1
   launch_pack_blocks(c, A, r2, nullptr, buf + layer_off_A(c), c->nbo, s);   // A's rows carry r2
-  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+  return finish_call(c);
 }
 
 armor_status armor_apply_layer(armor_ctx* c, const void* d_packed, const void* d_x, void* d_y, int64_t n_tokens,
@@ -700,7 +712,7 @@ armor_status armor_apply_layer(armor_ctx* c, const void* d_packed, const void* d
     st = launch_fwd_block(c, c->E, buf + layer_off_A(c), yc, n, d_out, s);                    // y = r2 . (z2 A^T)
     if (st != ARMOR_OK) return st;
   }
-  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+  return finish_call(c);
 }
 
 }  // extern "C"

@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "armor.h"
 
 // ---------------------------------------------------------------- scalars
@@ -78,7 +80,7 @@ struct armor_ctx {
   float *Xt_hi, *Xt_lo;
   int64_t gram_rows;  // rows of X staged per pass
   double* sc;         // [SC_COUNT]
-  double* partials;   // [2][4 * npart] partial sums of the fused / streaming reductions
+  double* partials;   // [2][8 * npart] partial sums of the fused / streaming reductions
   int64_t npart;
   double* partblk;    // [max(4 * nbo, 4 * nbi, nbo * nbi)] per-block partial sums
   double* quadpart;   // [nbo * nbi] per-block terms of the group updates' quadratic form
@@ -87,6 +89,11 @@ struct armor_ctx {
   SelRec* sel;        // [nbo * nbi]
   int32_t* status;    // [ST_COUNT]
   int64_t launches;
+  int device;           // the device that was current at armor_create; every call must be issued with it current
+  int n_sm;             // its number of SMs
+  int tc_blocks;        // 1: block products and per-block Grams on the tensor cores where the shape allows;
+                        // 0: always the fp32 CUDA-core kernels (exact products with 0 and 1)
+  armor_status host_err;   // first launch failure inside the running call that no fallback covers
   int kg;               // groups drawn per block in one sparse-core update (mask_groups, at least 1)
   int block_one_pass;   // 1: products with the wrappers take one tf32 pass (the bf16 forward, whose operands are
                         // rounded to 8 bits anyway); 0: three passes, fp32-grade
@@ -156,7 +163,37 @@ bool tc_gram_ok(const armor_ctx* c);
 armor_status tc_rowblock_gram(armor_ctx* c, const float* P, const float* T, float* G, cudaStream_t s);
 armor_status tc_colblock_gram(armor_ctx* c, const float* U, const float* Y, float* Cm, cudaStream_t s);
 armor_status tc_select_rows_times_H(armor_ctx* c, const float* Z, const float* H, float* Y, int nbo_pad, cudaStream_t s);
-extern int g_tc_blocks;   // 1: block products and per-block Grams on the tensor cores where the shape allows
+// A tensor-core launch that is refused for its shape or alignment (UNSUPPORTED) is replaced by the CUDA-core
+// kernel; any other failure is an error of the call: it is recorded and the entry point returns it.
+inline bool tc_done(armor_ctx* c, armor_status st) {
+  if (st == ARMOR_OK) return true;
+  if (st == ARMOR_ERR_UNSUPPORTED) return false;
+  if (c->host_err == ARMOR_OK) c->host_err = st;
+  return true;
+}
+// what an entry point returns: the recorded launch failure, else the state of the runtime
+inline armor_status finish_call(armor_ctx* c) {
+  const armor_status st = c->host_err;
+  c->host_err = ARMOR_OK;
+  if (st != ARMOR_OK) return st;
+  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+}
+
+// Function attributes (the dynamic shared-memory limit) hold per device: one bit per device ordinal and call
+// site remembers where the attribute has been set.
+struct PerDeviceOnce {
+  std::atomic<unsigned long long> mask{0};
+  bool done(int dev) const { return dev >= 0 && dev < 64 && ((mask.load(std::memory_order_relaxed) >> dev) & 1ull); }
+  void set(int dev) { if (dev >= 0 && dev < 64) mask.fetch_or(1ull << dev, std::memory_order_relaxed); }
+};
+template <typename K>
+inline armor_status ensure_dynamic_smem(PerDeviceOnce& once, int device, K kernel, size_t bytes) {
+  if (once.done(device)) return ARMOR_OK;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
+    return ARMOR_ERR_CUDA;
+  once.set(device);
+  return ARMOR_OK;
+}
 
 // out = in * H_w (FULL: dense GEMM by cfg.precision; DIAG: column scale) with up to two
 // fused dot products <out, d1> -> sc[slot1], <out, d2> -> sc[slot2] (slot < 0: none).

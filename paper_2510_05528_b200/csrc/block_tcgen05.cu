@@ -327,18 +327,9 @@ armor_status launch(armor_ctx* c, const HostOp& A, const HostOp& B, BParams p, c
   if (!make_map_2d(&mB, B.base, B.inner, B.outer, B.ld, 32, B.c.mn_major ? 32 : TILE, B.c.mn_major != 0)) return ARMOR_ERR_CUDA;
   p.a = A.c; p.b = B.c;
   p.status = c->status;
-  static bool attr = false;
-  if (!attr) {
-    if (cudaFuncSetAttribute(tc_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)
-      return ARMOR_ERR_CUDA;
-    attr = true;
-  }
-  static int n_sm = 0;
-  if (!n_sm) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return ARMOR_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ARMOR_ERR_CUDA;
-  }
+  static PerDeviceOnce attr;
+  if (ensure_dynamic_smem(attr, c->device, tc_block_kernel, SMEM_BYTES) != ARMOR_OK) return ARMOR_ERR_CUDA;
+  const int n_sm = c->n_sm;
   const int n_items = p.batch * p.m_tiles * p.n_tiles * p.n_split;
   const int grid = n_items < n_sm ? n_items : n_sm;
   tc_block_kernel<<<grid, NTHREADS, SMEM_BYTES, s>>>(mA, mB, mC, mD, p);

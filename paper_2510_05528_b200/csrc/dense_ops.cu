@@ -7,8 +7,8 @@
 #include "armor_internal.cuh"
 
 // The tensor-core accumulator adds with truncation, so a long run of same-sign terms drifts by about
-// (K / 8) * passes * 2^-24.  The GEMM therefore drains its accumulator into C every K_SEGMENT columns of
-// the contraction (the additions into C are ordinary round-to-nearest fp32 adds).
+// (K / 8) * passes * 2^-24.  The GEMM therefore drains its accumulator every K_SEGMENT columns of the
+// contraction into running sums held by its epilogue warps (ordinary round-to-nearest fp32 adds).
 static const int64_t K_SEGMENT = 1024;
 
 armor_status prepare_H(armor_ctx* c, const float* H, cudaStream_t s) {
@@ -55,12 +55,12 @@ armor_status rmul_H(armor_ctx* c, const float* in, const float* H, float* out, i
     g.d1 = d1; g.d2 = d2;
     g.k_segment = (g.passes >= 3) ? K_SEGMENT : 0;   // one-pass tf32 rounding (2^-11) dwarfs the accumulator drift
     g.part1 = d1 ? c->partials : nullptr;
-    g.part2 = d2 ? c->partials + 4 * c->npart : nullptr;
+    g.part2 = d2 ? c->partials + 8 * c->npart : nullptr;
     int tiles = 0;
     armor_status st = launch_tc_gemm(c, g, &tiles, s);
     if (st != ARMOR_OK) return st;
-    if (d1) reduce_partials_to(c, c->partials, 4 * tiles, out1, s);
-    if (d2) reduce_partials_to(c, c->partials + 4 * c->npart, 4 * tiles, out2, s);
+    if (d1) reduce_partials_to(c, c->partials, 8 * tiles, out1, s);
+    if (d2) reduce_partials_to(c, c->partials + 8 * c->npart, 8 * tiles, out2, s);
     return ARMOR_OK;
   }
   if (d1) dot_to_ptr(c, out, d1, rows * d_in, out1, s);

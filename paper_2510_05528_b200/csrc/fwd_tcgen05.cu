@@ -253,18 +253,9 @@ armor_status launch_fwd_block(armor_ctx* c, const void* X, const void* Q, void* 
   p.m_tiles = (int)((rows + BM - 1) / BM); p.n_tiles = (int)(d / BN); p.k_tiles = c->db / BKE;
   p.status = c->status;
   constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024 + 8 * 32 * 33 * sizeof(uint32_t);
-  static bool attr = false;
-  if (!attr) {
-    if (cudaFuncSetAttribute(fwd_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess)
-      return ARMOR_ERR_CUDA;
-    attr = true;
-  }
-  static int n_sm = 0;
-  if (!n_sm) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return ARMOR_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ARMOR_ERR_CUDA;
-  }
+  static PerDeviceOnce attr;
+  if (ensure_dynamic_smem(attr, c->device, fwd_block_kernel, SMEM) != ARMOR_OK) return ARMOR_ERR_CUDA;
+  const int n_sm = c->n_sm;
   const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
   const int grid = tiles < n_sm ? (int)tiles : n_sm;
   fwd_block_kernel<<<grid, NTHREADS, SMEM, s>>>(mX, mQ, p);

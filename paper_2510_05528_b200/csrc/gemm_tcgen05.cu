@@ -8,8 +8,9 @@
 //   warp 0   : TMA producer  (cp.async.bulk.tensor.2d, 128-byte swizzle, mbarrier complete_tx)
 //   warp 1   : MMA issuer    (one thread issues tcgen05.mma kind::tf32, 128 x 256 x 8 per instruction,
 //                             accumulators in tensor memory, two accumulator buffers of 256 columns)
-//   warps 2-5: epilogue      (tcgen05.ld 32 lanes x 32 columns, fused C-update / dot products; a symmetric
-//                             product writes its lower triangle only, the caller mirrors it once at the end)
+//   warps 2-9: epilogue      (tcgen05.ld 32 lanes x 32 columns; the K segments of a tile are summed in registers,
+//                             then one fused C-update / dot products; a symmetric product writes its lower
+//                             triangle only, the caller mirrors it once at the end)
 // passes == 3: every operand is given as a tf32-exact high part and an fp32 low part; the three products
 // hi*hi, lo*hi, hi*lo are accumulated into the same fp32 accumulator (error-compensated tf32, fp32-grade).
 // passes == 6: the same three products on fp16 high and low parts (kind::f16, twice the tf32 issue rate, half
@@ -26,8 +27,10 @@ namespace {
 using namespace tc;
 
 constexpr int BM = 128, BN = 256, BK = 32;          // BK fp32 = 128 bytes = one swizzle row
-constexpr int NTHREADS = 192;
-constexpr int RB = 16;                              // rows of C an epilogue lane keeps in flight
+constexpr int NTHREADS = 320;                       // TMA warp, MMA warp, eight epilogue warps
+constexpr int RB = 8;                               // rows of C an epilogue lane keeps in flight
+constexpr int EPI_COLS = 128;                       // accumulator columns per epilogue warp
+constexpr int TB_LD = 17;                           // padded row length of an epilogue warp's 32 x 16 staging tile
 constexpr uint32_t TMEM_COLS = 512;                 // two accumulator buffers of BN columns
 constexpr int A_BYTES = BM * BK * 4;                // 16 KiB
 constexpr int B_BYTES = BN * BK * 4;                // 32 KiB
@@ -116,6 +119,59 @@ __device__ __forceinline__ void item_decode(const Params& p, int item, int kt_to
   }
 }
 
+// One epilogue warp's 32 rows x 128 columns of finished sums (lane = row) go out through shared memory, 16
+// columns at a time, so that every store instruction writes two rows of 64 contiguous bytes.  Optional:
+// power-of-two scales, C += (read-modify-write), lower triangle only, partial dot products with d1 / d2.
+__device__ __forceinline__ void write_out(const float (&acc)[EPI_COLS], float* tilebuf, int lane, float* C, int64_t ldc,
+                                          int64_t row_base, int64_t col_base, int64_t M, int64_t N, bool accum, bool sym,
+                                          const float* rs, const float* cs, const float* d1, const float* d2, int64_t ldd,
+                                          double& dot1, double& dot2) {
+  if (row_base >= M) return;                                  // warp-uniform
+  const int rr = lane >> 4, cc = lane & 15;
+#pragma unroll
+  for (int c16 = 0; c16 < EPI_COLS / 16; ++c16) {
+    const int64_t col0 = col_base + c16 * 16;
+    if (col0 >= N) continue;                                   // warp-uniform (N is a multiple of 32)
+    if (sym && col0 > row_base + 31) continue;                 // chunk lies above the diagonal
+#pragma unroll
+    for (int i = 0; i < 16; ++i) tilebuf[lane * TB_LD + i] = acc[c16 * 16 + i];
+    __syncwarp();
+    const int64_t col = col0 + cc;
+    const float cscale = cs ? cs[col] : 1.f;
+    float f1 = 0.f, f2 = 0.f;
+#pragma unroll 1
+    for (int r0 = 0; r0 < 32; r0 += 2 * RB) {
+      float x[RB], o[RB];
+      bool keep[RB];
+#pragma unroll
+      for (int j = 0; j < RB; ++j) {
+        const int r = r0 + 2 * j + rr;
+        const int64_t grow = row_base + r;
+        keep[j] = grow < M && (!sym || col <= grow);
+        x[j] = tilebuf[r * TB_LD + cc];
+        if (rs) x[j] *= (grow < M ? rs[grow] : 1.f) * cscale;
+        o[j] = (accum && keep[j]) ? C[grow * ldc + col] : 0.f;
+      }
+      if (d1) {
+#pragma unroll
+        for (int j = 0; j < RB; ++j)
+          if (keep[j]) f1 = fmaf(x[j] + o[j], d1[(row_base + r0 + 2 * j + rr) * ldd + col], f1);
+      }
+      if (d2) {
+#pragma unroll
+        for (int j = 0; j < RB; ++j)
+          if (keep[j]) f2 = fmaf(x[j] + o[j], d2[(row_base + r0 + 2 * j + rr) * ldd + col], f2);
+      }
+#pragma unroll
+      for (int j = 0; j < RB; ++j)
+        if (keep[j]) C[(row_base + r0 + 2 * j + rr) * ldc + col] = x[j] + o[j];
+    }
+    dot1 += (double)f1;
+    dot2 += (double)f2;
+    __syncwarp();
+  }
+}
+
 template <int PASSES>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapAlo,
@@ -140,7 +196,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(tfull0 + 8 * s, 1); mbar_init(tempty0 + 8 * s, 4); }
+    for (int s = 0; s < 2; ++s) { mbar_init(tfull0 + 8 * s, 1); mbar_init(tempty0 + 8 * s, 8); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -242,117 +298,57 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     }
   } else {
     // ------------------------------------------------------------ epilogue warps
-    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    // Eight warps: warp w reads TMEM lanes 32 (w % 4) .. and one half (128 columns) of the accumulator, one
+    // row per lane.  The K segments of a tile are summed in registers (ordinary round-to-nearest adds), so the
+    // accumulator buffer is handed back right after it has been read and C is touched once per tile.
+    const int q = warp & 3;
+    const int half = (warp - 2) >> 2;
+    float* tilebuf = reinterpret_cast<float*>(smem + (size_t)STAGES * STAGE_BYTES) + (warp - 2) * (32 * TB_LD);
     int local = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
       int tile, part, kt_begin, kt_end, mt, nt;
       item_decode(p, item, kt_total, tile, part, kt_begin, kt_end);
       tile_coords(p, tile, mt, nt);
-      if (part >= 0) {
-        // a piece of a split tile: its partial sums go, plainly, to this item's slab
-        float* slab = p.slabs + ((int64_t)(tile - p.split_first) * p.split_parts + part) * (BM * BN);
-        float* tilebuf = reinterpret_cast<float*>(smem + (size_t)STAGES * STAGE_BYTES) + q * (32 * 33);
-        for (int kt0 = kt_begin; kt0 < kt_end && ok; kt0 += p.kt_seg, ++local) {
-          const int as = local & 1;
-          const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
-          if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
-          tc_fence_after();
-#pragma unroll 1
-          for (int ch = 0; ch < BN / 32; ++ch) {
-            uint32_t r[32];
-            tmem_ld32(tmem_base + (uint32_t)(as * BN + ch * 32) + ((uint32_t)(q * 32) << 16), r);
+      float acc[EPI_COLS];
 #pragma unroll
-            for (int cidx = 0; cidx < 32; ++cidx) tilebuf[lane * 33 + cidx] = __uint_as_float(r[cidx]);
-            __syncwarp();
-            float* dst = slab + (int64_t)(q * 32) * BN + ch * 32 + lane;
-#pragma unroll 1
-            for (int r0 = 0; r0 < 32; r0 += RB) {
-              float x[RB], o[RB];
-#pragma unroll
-              for (int j = 0; j < RB; ++j) {
-                x[j] = tilebuf[(r0 + j) * 33 + lane];
-                o[j] = (kt0 > kt_begin) ? dst[(int64_t)(r0 + j) * BN] : 0.f;
-              }
-#pragma unroll
-              for (int j = 0; j < RB; ++j) dst[(int64_t)(r0 + j) * BN] = x[j] + o[j];
-            }
-            __syncwarp();
-          }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(tempty0 + 8 * as);
-        }
-        continue;
-      }
-      double dot1 = 0.0, dot2 = 0.0;
-      for (int kt0 = 0; kt0 < kt_total && ok; kt0 += p.kt_seg, ++local) {
+      for (int i = 0; i < EPI_COLS; ++i) acc[i] = 0.f;
+      for (int kt0 = kt_begin; kt0 < kt_end && ok; kt0 += p.kt_seg, ++local) {
         const int as = local & 1;
         const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
-        const bool accum = p.accumulate || kt0 > 0;           // later K segments add to what is in C
-        const bool last = kt0 + p.kt_seg >= kt_total;
         if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
         tc_fence_after();
-        // Each lane holds one row of a 32 x 32 chunk.  The chunk is turned through shared memory so that
-        // global memory sees whole 128-byte row segments (lanes = consecutive columns).
-        float* tilebuf = reinterpret_cast<float*>(smem + (size_t)STAGES * STAGE_BYTES) + q * (32 * 33);
-        const int64_t row_base = (int64_t)mt * BM + q * 32;
-#pragma unroll 1
-        for (int ch = 0; ch < BN / 32; ++ch) {
-          const int64_t col0 = (int64_t)nt * BN + ch * 32;
+#pragma unroll
+        for (int ch = 0; ch < EPI_COLS / 32; ++ch) {
           uint32_t r[32];
-          tmem_ld32(tmem_base + (uint32_t)(as * BN + ch * 32) + ((uint32_t)(q * 32) << 16), r);
-          if (col0 >= p.N || row_base >= p.M) continue;                       // warp-uniform
-          if (p.symmetric_lower && col0 > row_base + 31) continue;           // chunk lies above the diagonal
+          tmem_ld32(tmem_base + (uint32_t)(as * BN + half * EPI_COLS + ch * 32) + ((uint32_t)(q * 32) << 16), r);
 #pragma unroll
-          for (int cidx = 0; cidx < 32; ++cidx) tilebuf[lane * 33 + cidx] = __uint_as_float(r[cidx]);
-          __syncwarp();
-          const int64_t col = col0 + lane;
-          const float cscale = p.col_scale ? p.col_scale[col] : 1.f;
-          float f1 = 0.f, f2 = 0.f;
-#pragma unroll 1
-          for (int r0 = 0; r0 < 32; r0 += RB) {
-            float x[RB], o[RB];
-            bool keep[RB];
-#pragma unroll
-            for (int j = 0; j < RB; ++j) {
-              const int64_t grow = row_base + r0 + j;
-              keep[j] = grow < p.M && (!p.symmetric_lower || col <= grow);
-              x[j] = tilebuf[(r0 + j) * 33 + lane];
-              if (p.row_scale) x[j] *= (grow < p.M ? p.row_scale[grow] : 1.f) * cscale;
-              o[j] = (accum && keep[j]) ? p.C[grow * p.ldc + col] : 0.f;
-            }
-            if (last && p.d1) {
-#pragma unroll
-              for (int j = 0; j < RB; ++j)
-                if (keep[j]) f1 = fmaf(x[j] + o[j], p.d1[(row_base + r0 + j) * p.ldc + col], f1);
-            }
-            if (last && p.d2) {
-#pragma unroll
-              for (int j = 0; j < RB; ++j)
-                if (keep[j]) f2 = fmaf(x[j] + o[j], p.d2[(row_base + r0 + j) * p.ldc + col], f2);
-            }
-#pragma unroll
-            for (int j = 0; j < RB; ++j)
-              if (keep[j]) p.C[(row_base + r0 + j) * p.ldc + col] = x[j] + o[j];
-          }
-          dot1 += (double)f1;
-          dot2 += (double)f2;
-          __syncwarp();
+          for (int i = 0; i < 32; ++i) acc[ch * 32 + i] += __uint_as_float(r[i]);
         }
-        // accumulator buffer is free again
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(tempty0 + 8 * as);
       }
-      if (ok && (p.part1 || p.part2)) {
+      if (!ok) break;
+      if (part >= 0) {
+        // a piece of a split tile: its partial sums go, plainly, to this item's slab
+        float* slab = p.slabs + ((int64_t)(tile - p.split_first) * p.split_parts + part) * (BM * BN);
+        double u1 = 0.0, u2 = 0.0;
+        write_out(acc, tilebuf, lane, slab, BN, q * 32, half * EPI_COLS, BM, BN, false, false, nullptr, nullptr, nullptr,
+                  nullptr, 0, u1, u2);
+        continue;
+      }
+      double dot1 = 0.0, dot2 = 0.0;
+      write_out(acc, tilebuf, lane, p.C, p.ldc, (int64_t)mt * BM + q * 32, (int64_t)nt * BN + half * EPI_COLS, p.M, p.N,
+                p.accumulate != 0, p.symmetric_lower != 0, p.row_scale, p.col_scale, p.d1, p.d2, p.ldc, dot1, dot2);
+      if (p.part1 || p.part2) {
         for (int o = 16; o > 0; o >>= 1) {
           dot1 += __shfl_down_sync(0xffffffffu, dot1, o);
           dot2 += __shfl_down_sync(0xffffffffu, dot2, o);
         }
         if (lane == 0) {
-          if (p.part1) p.part1[(int64_t)tile * 4 + q] = dot1;
-          if (p.part2) p.part2[(int64_t)tile * 4 + q] = dot2;
+          if (p.part1) p.part1[(int64_t)tile * 8 + half * 4 + q] = dot1;
+          if (p.part2) p.part2[(int64_t)tile * 8 + half * 4 + q] = dot2;
         }
       }
     }
@@ -412,8 +408,9 @@ __global__ void __launch_bounds__(256) tc_gemm_fixup_kernel(const Params p) {
   if (threadIdx.x == 0) {
     double t1 = 0.0, t2 = 0.0;
     for (int w = 0; w < 8; ++w) { t1 += red1[w]; t2 += red2[w]; }
-    if (p.part1) p.part1[(int64_t)tile * 4 + qq] = t1;
-    if (p.part2) p.part2[(int64_t)tile * 4 + qq] = t2;
+    // eight slots per tile (the GEMM's eight epilogue warps); this kernel fills four and clears the rest
+    if (p.part1) { p.part1[(int64_t)tile * 8 + qq] = t1; p.part1[(int64_t)tile * 8 + 4 + qq] = 0.0; }
+    if (p.part2) { p.part2[(int64_t)tile * 8 + qq] = t2; p.part2[(int64_t)tile * 8 + 4 + qq] = 0.0; }
   }
 }
 
@@ -452,19 +449,10 @@ armor_status launch_impl(armor_ctx* c, const TcGemm& g, Params p, cudaStream_t s
   }
   constexpr int STAGE_BYTES = (SPLIT ? 2 : 1) * (A_BYTES + B_BYTES);
   constexpr int STAGES = SPLIT ? 2 : 4;
-  constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024 + 4 * 32 * 33 * sizeof(float);
-  static bool attr = false;
-  if (!attr) {
-    if (cudaFuncSetAttribute(tc_gemm_kernel<PASSES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess)
-      return ARMOR_ERR_CUDA;
-    attr = true;
-  }
-  static int n_sm = 0;
-  if (!n_sm) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return ARMOR_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ARMOR_ERR_CUDA;
-  }
+  constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024 + 8 * 32 * TB_LD * sizeof(float);
+  static PerDeviceOnce attr;
+  if (ensure_dynamic_smem(attr, c->device, tc_gemm_kernel<PASSES>, SMEM) != ARMOR_OK) return ARMOR_ERR_CUDA;
+  const int n_sm = c->n_sm;
   // tail split: the tiles of the last, partly filled wave are cut along K so that their pieces fill the wave
   p.split_first = p.n_tiles_total; p.split_parts = 1; p.n_items = p.n_tiles_total; p.slabs = c->gemm_slabs;
   const int kt_total = (int)((p.K + (H16 ? 64 : BK) - 1) / (H16 ? 64 : BK));

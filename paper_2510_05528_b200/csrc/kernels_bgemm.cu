@@ -301,13 +301,10 @@ void launch_bgemm(armor_ctx* c, const BGemm& g_in, cudaStream_t s) {
   c->launches++;
 }
 
-// 1: block-diagonal products on the tensor cores where the shape allows; 0: always the fp32 CUDA-core kernels
-int g_tc_blocks = 1;
-
 void bd_right(armor_ctx* c, const float* in, const float* Bblk, bool transB, float* out, int64_t rows,
               int64_t cols, float alpha, const float* add, float beta, cudaStream_t s) {
-  if (g_tc_blocks && tc_block_ok(c, rows, cols) &&
-      tc_bd_right(c, in, Bblk, transB, out, rows, cols, alpha, add, beta, s) == ARMOR_OK)
+  if (c->tc_blocks && tc_block_ok(c, rows, cols) &&
+      tc_done(c, tc_bd_right(c, in, Bblk, transB, out, rows, cols, alpha, add, beta, s)))
     return;
   const int db = c->db;
   BGemm g{};
@@ -323,8 +320,8 @@ void bd_right(armor_ctx* c, const float* in, const float* Bblk, bool transB, flo
 
 void bd_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, float* out, int64_t rows,
              int64_t cols, float alpha, const float* add, float beta, cudaStream_t s) {
-  if (g_tc_blocks && tc_block_ok(c, rows, cols) &&
-      tc_bd_left(c, Ablk, transA, in, out, rows, cols, alpha, add, beta, s) == ARMOR_OK)
+  if (c->tc_blocks && tc_block_ok(c, rows, cols) &&
+      tc_done(c, tc_bd_left(c, Ablk, transA, in, out, rows, cols, alpha, add, beta, s)))
     return;
   const int db = c->db;
   BGemm g{};
@@ -346,10 +343,10 @@ extern "C" armor_status armor_block_product(armor_ctx* c, int32_t side, int32_t 
   if (cols % 4 || (side == 0 ? cols : rows) % c->db) return ARMOR_ERR_SHAPE;
   if (path == 1 && !tc_block_ok(c, rows, cols)) return ARMOR_ERR_UNSUPPORTED;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-  const int saved = g_tc_blocks;
-  g_tc_blocks = (path != 0);
+  const int saved = c->tc_blocks;
+  c->tc_blocks = (path != 0);
   if (side == 1) bd_left(c, d_blocks, transpose != 0, d_in, d_out, rows, cols, alpha, d_add, beta, s);
   else bd_right(c, d_in, d_blocks, transpose != 0, d_out, rows, cols, alpha, d_add, beta, s);
-  g_tc_blocks = saved;
-  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+  c->tc_blocks = saved;
+  return finish_call(c);
 }

@@ -523,12 +523,13 @@ armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float*
     const int slices = chol_parts_per_block(db, nb);
     const int w = db / slices;
     const size_t smem = (panel_floats(db) + (size_t)db * (w + 1)) * sizeof(float);
-    static size_t attr_bytes = 0;
-    if (smem > attr_bytes) {
+    static size_t attr_bytes[64] = {};   // per device: the limit set so far
+    const int dv = (c->device >= 0 && c->device < 64) ? c->device : 0;
+    if (smem > attr_bytes[dv] || c->device != dv) {
       if (cudaFuncSetAttribute(chol_blocked_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
           cudaSuccess)
         return ARMOR_ERR_CUDA;
-      attr_bytes = smem;
+      attr_bytes[dv] = smem;
     }
     chol_blocked_kernel<<<dim3(nb, slices), NT, smem, s>>>(mode, Gmat, rhs, out, dotw, A, c->cfg.ridge, db, w,
                                                           part, c->failflag, c->status);
@@ -536,15 +537,11 @@ armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float*
     return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
   }
   const size_t smem = 2 * (size_t)db * (db + 1) * sizeof(float);
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 128 * 129 * 4) != cudaSuccess)
-      return ARMOR_ERR_CUDA;
-    attr_set = true;
-  }
+  static PerDeviceOnce attr_set;
+  if (ensure_dynamic_smem(attr_set, c->device, chol_kernel, 2 * 128 * 129 * 4) != ARMOR_OK) return ARMOR_ERR_CUDA;
   const int nt = ((db + 31) / 32) * 32;
   chol_kernel<<<nb, nt < 64 ? 64 : nt, smem, s>>>(mode, Gmat, rhs, out, dotw, A, c->cfg.ridge, db, part,
                                                  c->failflag, c->status);
   c->launches++;
-  return ARMOR_OK;
+  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
 }

@@ -484,7 +484,7 @@ void launch_mask_quadratic(armor_ctx* c, const float* A, const float* B, const f
     for (int kk = 0; kk < kg; ++kk) {
       const float* Zk = c->Zsel + (int64_t)kk * nbi * nbo_pad * db;
       float* Yk = c->Ysel + (int64_t)kk * nbi * nbo_pad * c->d_in;
-      if (!(g_tc_blocks && tc_gram_ok(c) && tc_select_rows_times_H(c, Zk, H, Yk, nbo_pad, s) == ARMOR_OK)) {
+      if (!(c->tc_blocks && tc_gram_ok(c) && tc_done(c, tc_select_rows_times_H(c, Zk, H, Yk, nbo_pad, s)))) {
         BGemm g{};
         g.A = Zk; g.sAb = (int64_t)nbo_pad * db; g.sAm = db; g.sAk = 1;
         g.B = H; g.sBb = (int64_t)db * c->d_in; g.sBk = c->d_in; g.sBn = 1;

@@ -230,7 +230,7 @@ __device__ __forceinline__ int warp_count_flags(const int32_t* __restrict__ f, i
   return v;
 }
 
-// stage 0: start, 1: after A, 2: after B, 3 / 6: after S, 4: mask accept.  One warp.
+// stage 0: start, 1: after A, 2: after B, 3 / 6: after S, 4: mask accept, 5: mask phase off.  One warp.
 __global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const int32_t* failflag, int nflag,
                              const double* partA, int nA, int32_t* status) {
   double psum = 0.0;
@@ -298,8 +298,10 @@ __global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const 
   } else if (stage == 9) {   // joint Adam step: the loss was evaluated afresh from the new state
     sc[SC_LOSS] = sc[SC_L0];
     if (st) st->loss_A = st->loss_B = st->loss_S = sc[SC_LOSS];
-  } else if (stage == 5) {  // phases skipped: carry the loss forward
-    if (st) { st->loss_A = st->loss_B = st->loss_S = st->loss_mask = sc[SC_LOSS]; }
+  } else if (stage == 5) {  // sparse-core update switched off: nothing was evaluated, nothing accepted
+    sc[SC_ACCEPT] = 0.0;
+    sc[SC_DL_M] = 0.0;
+    if (st) st->loss_mask = sc[SC_LOSS];
   }
 }
 

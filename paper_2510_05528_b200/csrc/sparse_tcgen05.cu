@@ -570,27 +570,14 @@ armor_status launch_tc_sparse(armor_ctx* c, const void* Sc, const void* E, const
   p.m_tiles = (int)(c->d_out / BM); p.n_tiles = (int)((n + BN - 1) / BN); p.k_tiles = (int)(c->d_in / BKL);
   p.status = c->status;
   constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024;
-  static bool attr = false;
-  if (!attr) {
-    if (cudaFuncSetAttribute(tc_sparse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess)
-      return ARMOR_ERR_CUDA;
-    attr = true;
-  }
-  static int n_sm = 0;
-  if (!n_sm) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return ARMOR_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ARMOR_ERR_CUDA;
-  }
+  static PerDeviceOnce attr;
+  if (ensure_dynamic_smem(attr, c->device, tc_sparse_kernel, SMEM) != ARMOR_OK) return ARMOR_ERR_CUDA;
+  const int n_sm = c->n_sm;
   const bool timed = c->timing_on && c->timing_n < ARMOR_MAX_TIMED;
   if (timed) cudaEventRecord(c->ev_beg[c->timing_n], s);
   if (g_sparse_pairs && c->d_out % 256 == 0 && n_sm >= 2) {
-    static bool attr2 = false;
-    if (!attr2) {
-      if (cudaFuncSetAttribute(tc_sparse_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess)
-        return ARMOR_ERR_CUDA;
-      attr2 = true;
-    }
+      static PerDeviceOnce attr2;
+    if (ensure_dynamic_smem(attr2, c->device, tc_sparse_pair_kernel, SMEM) != ARMOR_OK) return ARMOR_ERR_CUDA;
     p.n_tiles = (int)((n + BN2 - 1) / BN2);
     const int tiles = (p.m_tiles / 2) * p.n_tiles;
     int pairs = n_sm / 2;
