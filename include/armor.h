@@ -219,15 +219,30 @@ armor_status armor_pack_layer(armor_ctx* ctx, const float* d_A, const float* d_B
 armor_status armor_apply_layer(armor_ctx* ctx, const void* d_packed, const void* d_x, void* d_y, int64_t n_tokens,
                                armor_stream_t stream);
 
-/* Copies up to n device status words to h_codes (host).  Word 0: number of
- * Cholesky failures since the context was created; word 1: first failing
- * block id + 1; word 2: bounded waits that gave up; word 4: mask groups the sparse forward could
- * not represent; word 3: last
- * armor_status recorded by a kernel.  The caller must have synchronised the
- * stream the context's work ran on.  (This call itself copies synchronously.) */
+/* Copies up to n (at most 16) device status words to h_codes (host).
+ *   word 0: Cholesky failures since the context was created; word 1: first failing block id + 1;
+ *   word 2: bounded waits that gave up; word 3: last armor_status recorded by a kernel;
+ *   word 4: mask groups the sparse forward could not represent;
+ *   words 5-9, written by the input screening that armor_init and armor_bcd_step run first:
+ *     5: NaN / Inf entries seen in W, 6: NaN / Inf entries seen in H, 7: negative diagonal entries of H
+ *     (all three cumulative), 8: zero diagonal entries of H in the last screened call (legal: a channel
+ *     without weight), 9: 1 if the last screened call met any of 5-7.  Such a call withholds every update:
+ *     A, B, S and M come back bit for bit as they went in (armor_init still writes its outputs), word 3 reads
+ *     ARMOR_ERR_INVALID_ARG, and the next call with clean inputs runs normally.
+ * The caller must have synchronised the stream the context's work ran on.  (This call itself copies
+ * synchronously.) */
 armor_status armor_get_device_status(armor_ctx* ctx, int32_t* h_codes, int32_t n);
 
 const char* armor_status_string(armor_status s);
+
+/* Self-test of the bounded waits (no counterpart in the paper): every wait of the tensor-core kernels on an
+ * mbarrier gives up after a cycle budget, raises status word 2, records ARMOR_ERR_TIMEOUT in word 3 and lets the
+ * kernel end normally.  This call runs one warp that waits, with a limit of limit_cycles (1 .. 2e9) clock
+ * cycles, on a barrier nothing arrives on, and writes d_result[0] = 0 (the wait gave up; 1 would mean it was
+ * satisfied) and d_result[1] = 1 (the abort flag the other roles of a kernel watch).  d_result: two int32 on
+ * the device.  The context stays usable. */
+armor_status armor_selftest_wait_timeout(armor_ctx* ctx, int64_t limit_cycles, int32_t* d_result,
+                                         armor_stream_t stream);
 
 /* Number of kernel launches the context has enqueued so far (host counter). */
 int64_t armor_launch_count(const armor_ctx* ctx);

@@ -29,7 +29,7 @@ EXPORTS = ["armor_workspace_bytes", "armor_create", "armor_destroy", "armor_gram
            "armor_packed_layer_bytes", "armor_pack_layer", "armor_apply_layer",
            "armor_get_device_status",
            "armor_status_string", "armor_launch_count", "armor_gemm_timing_enable", "armor_gemm_timing",
-           "armor_normalize_noalloc", "armor_block_product"]
+           "armor_normalize_noalloc", "armor_block_product", "armor_selftest_wait_timeout"]
 
 
 class ArmorError(RuntimeError):
@@ -85,6 +85,7 @@ def lib() -> C.CDLL:
         L.armor_block_product.argtypes = [vp, i32, i32, vp, vp, vp, i64, i64, C.c_float, vp, C.c_float, i32, vp]
         L.armor_gemm_timing_enable.argtypes = [vp, i32]
         L.armor_gemm_timing.argtypes = [vp, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
+        L.armor_selftest_wait_timeout.argtypes = [vp, i64, vp, vp]
         for name in EXPORTS:
             if name not in ("armor_status_string", "armor_launch_count"):
                 getattr(L, name).restype = C.c_int
@@ -227,10 +228,15 @@ def armor_apply_layer(ctx, packed, x, y) -> None:
                                    x.shape[0], _stream()), "armor_apply_layer")
 
 
-def armor_get_device_status(ctx, n: int = 8) -> list[int]:
+def armor_get_device_status(ctx, n: int = 16) -> list[int]:
     buf = (C.c_int32 * n)()
     _check(lib().armor_get_device_status(ctx, buf, n), "armor_get_device_status")
     return list(buf)
+
+
+def armor_selftest_wait_timeout(ctx, limit_cycles: int, result: torch.Tensor) -> None:
+    _check(lib().armor_selftest_wait_timeout(ctx, int(limit_cycles), _ptr(result, torch.int32, "result"), _stream()),
+           "armor_selftest_wait_timeout")
 
 
 def armor_launch_count(ctx) -> int:

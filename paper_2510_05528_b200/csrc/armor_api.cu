@@ -135,6 +135,7 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   TAKE(failflag, int32_t*, (size_t)nbmax * sizeof(int32_t));
   TAKE(sel, SelRec*, (size_t)nbo * nbi * kg * sizeof(SelRec));
   TAKE(status, int32_t*, ST_COUNT * sizeof(int32_t));
+  TAKE(screen, int32_t*, 4 * sizeof(int32_t));
 #undef TAKE
   if (c) {
     c->npart = npart;
@@ -362,6 +363,7 @@ armor_status armor_init(armor_ctx* c, const float* d_W, const float* d_H, float*
                         float* d_A, float* d_B, float* d_S, uint8_t* d_M, armor_stream_t stream) {
   if (!c || !d_W || !d_H || !d_Wbar || !d_A || !d_B || !d_S || !d_M) return ARMOR_ERR_INVALID_ARG;
   if (c->cfg.normalize && (!d_r1 || !d_r2)) return ARMOR_ERR_INVALID_ARG;
+  if (launch_screen_inputs(c, d_W, d_H, cs(stream)) != ARMOR_OK) return ARMOR_ERR_CUDA;
   launch_init(c, d_W, d_H, d_Wbar, d_r1, d_r2, d_A, d_B, d_S, d_M, cs(stream));
   if (reset_adam(c, cs(stream)) != ARMOR_OK) return ARMOR_ERR_CUDA;
   return finish_call(c);
@@ -385,6 +387,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
   const int db = c->db, nbo = c->nbo, nbi = c->nbi;
   const int64_t d_out = c->d_out, d_in = c->d_in;
   const int ph = c->cfg.phases;
+  if (launch_screen_inputs(c, W, H, s) != ARMOR_OK) return ARMOR_ERR_CUDA;
   armor_status st = prepare_H(c, H, s);
   if (st != ARMOR_OK) return st;
   // W H_w is the same for every iteration of the call: E H_w = W H_w - A (T H_w)

@@ -35,7 +35,15 @@ enum {
 };
 
 // status words in the device status buffer
-enum { ST_CHOL_FAILS = 0, ST_FIRST_FAIL = 1, ST_WAIT_TIMEOUTS = 2, ST_LAST_ERR = 3, ST_SPARSE_BAD_GROUPS = 4, ST_COUNT = 8 };
+enum {
+  ST_CHOL_FAILS = 0, ST_FIRST_FAIL = 1, ST_WAIT_TIMEOUTS = 2, ST_LAST_ERR = 3, ST_SPARSE_BAD_GROUPS = 4,
+  ST_NONFINITE_W = 5,    // NaN / Inf entries seen in W by the input screening (cumulative)
+  ST_NONFINITE_H = 6,    // NaN / Inf entries seen in H
+  ST_NEG_DIAG_H = 7,     // negative diagonal entries of H (H cannot be a Gram matrix)
+  ST_DEAD_CHANNELS = 8,  // zero diagonal entries of H in the last screened call (legal: the channel carries no weight)
+  ST_POISON = 9,         // 1 while the last screened call had unusable inputs: its updates were all withheld
+  ST_COUNT = 16
+};
 
 // One selected group per (i, j) block of the sparse core (Algorithm 3).
 struct SelRec {
@@ -88,6 +96,7 @@ struct armor_ctx {
   int32_t* failflag;  // [max(nbo, nbi)]
   SelRec* sel;        // [nbo * nbi]
   int32_t* status;    // [ST_COUNT]
+  int32_t* screen;    // [4] per-call counters of the input screening
   int64_t launches;
   int device;           // the device that was current at armor_create; every call must be issued with it current
   int n_sm;             // its number of SMs
@@ -230,6 +239,9 @@ void launch_axpy_slot(armor_ctx* c, float* y, const float* x, int64_t n, int slo
 void launch_init(armor_ctx* c, const float* W, const float* H, float* Wbar, float* r1, float* r2,
                  float* A, float* B, float* S, uint8_t* M, cudaStream_t s);
 void launch_zero_scalars(armor_ctx* c, cudaStream_t s);
+// Input screening at the top of a call: counts non-finite entries of W and H and negative / zero diagonal
+// entries of H into the status words and sets or clears ST_POISON for the call.
+armor_status launch_screen_inputs(armor_ctx* c, const float* W, const float* H, cudaStream_t s);
 // One Adam step (Kingma & Ba, Algorithm 1) on n parameters with gradient g = -2 * gamma; step counts from 1.
 // M != nullptr: theta is the N:M core, one mask byte per m_group entries, masked-out entries stay zero.
 void launch_adam(armor_ctx* c, float* theta, const float* gamma, float* m, float* v, int64_t n, const uint8_t* M,

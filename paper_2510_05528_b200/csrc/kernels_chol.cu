@@ -234,6 +234,7 @@ chol_blocked_kernel(int mode, const float* __restrict__ Gmat, const float* __res
   }
   __syncthreads();
   const bool fail = (s_fail != 0);
+  const bool hold = (mode == 0) && status[ST_POISON] != 0;   // unusable inputs: the A-step is withheld (X = 0)
 
   if (!fail) {
     const int wq = w / 4;          // column c of tile column tc: tc + wq * j  (conflict-free shared-memory rows)
@@ -357,13 +358,13 @@ chol_blocked_kernel(int mode, const float* __restrict__ Gmat, const float* __res
         if (right) {
           const int vid = e / q4, r4 = (e % q4) * 4;
           gidx[u] = (int64_t)(v0 + vid) * db + r4;
-          if (!fail) x[u] = make_float4(Rs[r4 * ldr + vid], Rs[(r4 + 1) * ldr + vid], Rs[(r4 + 2) * ldr + vid],
-                                        Rs[(r4 + 3) * ldr + vid]);
+          if (!fail && !hold) x[u] = make_float4(Rs[r4 * ldr + vid], Rs[(r4 + 1) * ldr + vid], Rs[(r4 + 2) * ldr + vid],
+                                                 Rs[(r4 + 3) * ldr + vid]);
         } else {
           const int r = e / (w / 4), vid4 = (e % (w / 4)) * 4;
           gidx[u] = (int64_t)r * db + v0 + vid4;
-          if (!fail) x[u] = make_float4(Rs[r * ldr + vid4], Rs[r * ldr + vid4 + 1], Rs[r * ldr + vid4 + 2],
-                                        Rs[r * ldr + vid4 + 3]);
+          if (!fail && !hold) x[u] = make_float4(Rs[r * ldr + vid4], Rs[r * ldr + vid4 + 1], Rs[r * ldr + vid4 + 2],
+                                                 Rs[r * ldr + vid4 + 3]);
         }
         if (mode == 0) {
           aold[u] = *reinterpret_cast<const float4*>(A + off + gidx[u]);
@@ -456,6 +457,7 @@ __global__ void chol_kernel(int mode, const float* __restrict__ Gmat, const floa
     __syncthreads();
   }
   const bool fail = (s_fail != 0);
+  const bool hold = (mode == 0) && status[ST_POISON] != 0;   // unusable inputs: the A-step is withheld (X = 0)
 
   double acc = 0.0;
   if (!fail) {
@@ -477,7 +479,7 @@ __global__ void chol_kernel(int mode, const float* __restrict__ Gmat, const floa
   for (int e = tid; e < db * db; e += nt) {
     const int r = e / db, cidx = e % db;
     float x = 0.f;
-    if (!fail) x = right ? Rs[cidx * ld + r] : Rs[r * ld + cidx];
+    if (!fail && !hold) x = right ? Rs[cidx * ld + r] : Rs[r * ld + cidx];
     if (mode == 0) {
       const float a = A[off + e] + x;
       A[off + e] = a;

@@ -110,6 +110,7 @@ __global__ void __launch_bounds__(NT) axpy_slot_kernel(float4* __restrict__ y, c
                                                        int64_t n4, const double* __restrict__ sc, int slot,
                                                        float sign) {
   const float a = sign * (float)sc[slot];
+  if (a == 0.f) return;                 // a zero step (also what withheld updates look like): y stays bit for bit
   for (int64_t i = (int64_t)blockIdx.x * NT + threadIdx.x; i < n4; i += (int64_t)gridDim.x * NT) {
     float4 u = y[i], v = x[i];
     y[i] = make_float4(fmaf(a, v.x, u.x), fmaf(a, v.y, u.y), fmaf(a, v.z, u.z), fmaf(a, v.w, u.w));
@@ -238,6 +239,7 @@ __global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const 
   if (stage == 1 || stage == 2 || stage == 4) psum = warp_sum_f64(partA, nA);
   if (stage == 1 || stage == 2) nf = warp_count_flags(failflag, nflag);
   if (threadIdx.x != 0) return;
+  const bool poisoned = status[ST_POISON] != 0;   // unusable inputs: every step length is zero, nothing is accepted
   if (stage == 0) {
     sc[SC_LOSS] = sc[SC_L0];
     if (st) {
@@ -259,7 +261,7 @@ __global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const 
     const double gd = psum;
     sc[SC_GD_B] = gd;
     const double q = sc[SC_Q_B];
-    const double tau = (q > 0.0) ? gd / q : 0.0;
+    const double tau = (q > 0.0 && !poisoned) ? gd / q : 0.0;
     sc[SC_TAU_B] = tau;
     sc[SC_LOSS] -= 2.0 * tau * gd - tau * tau * q;
     if (st) { st->loss_B = sc[SC_LOSS]; st->tau_B = (float)tau; st->chol_failed += nf; }
@@ -271,27 +273,28 @@ __global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const 
       const double bh = sqrt(sc[SC_BETA_A]) * sqrt(sc[SC_BETA_K]);
       tau = (bh > 0.0) ? 1.0 / bh : 0.0;
     }
+    if (poisoned) tau = 0.0;
     sc[SC_TAU_S] = tau;
     sc[SC_LOSS] -= 2.0 * tau * nrm - tau * tau * q;
     if (st) { st->loss_S = sc[SC_LOSS]; st->tau_S = (float)tau; }
   } else if (stage == 4) {
     sc[SC_EHV_M] = psum;   // <Gamma, dS> = <E H_w, V>, one term per block
     const double dl = -2.0 * sc[SC_EHV_M] + sc[SC_Q_M];
-    const bool acc = (dl <= 0.0);
+    const bool acc = (dl <= 0.0) && !poisoned;
     sc[SC_DL_M] = dl;
     sc[SC_ACCEPT] = acc ? 1.0 : 0.0;
     if (acc) sc[SC_LOSS] += dl;
     if (st) { st->delta_L_mask += dl; st->mask_accepted += acc ? 1 : 0; st->loss_mask = sc[SC_LOSS]; }   // summed over the sweeps
   } else if (stage == 7) {   // A gradient step with the step of Eq. lrA: tau = 1 / (beta_A / 2)
     const double hb = sc[SC_HB_A], nrm = sc[SC_TMP0], q = sc[SC_TMP1];
-    const double tau = (hb > 0.0) ? 1.0 / hb : 0.0;
+    const double tau = (hb > 0.0 && !poisoned) ? 1.0 / hb : 0.0;
     sc[SC_TAU_A] = tau;
     sc[SC_DEC_A] = 2.0 * tau * nrm - tau * tau * q;   // exact decrease of the quadratic in A along Gamma
     sc[SC_LOSS] -= sc[SC_DEC_A];
     if (st) st->loss_A = sc[SC_LOSS];
   } else if (stage == 8) {   // B gradient step with the step of Eq. lrB
     const double hb = sc[SC_HB_B], gd = sc[SC_GD_B], q = sc[SC_Q_B];
-    const double tau = (hb > 0.0) ? 1.0 / hb : 0.0;
+    const double tau = (hb > 0.0 && !poisoned) ? 1.0 / hb : 0.0;
     sc[SC_TAU_B] = tau;
     sc[SC_LOSS] -= 2.0 * tau * gd - tau * tau * q;
     if (st) { st->loss_B = sc[SC_LOSS]; st->tau_B = (float)tau; }
@@ -303,6 +306,44 @@ __global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const 
     sc[SC_DL_M] = 0.0;
     if (st) st->loss_mask = sc[SC_LOSS];
   }
+}
+
+// ---- input screening -----------------------------------------------------------------------------
+__device__ __forceinline__ int bad4(const float4 v) {
+  return (isfinite(v.x) ? 0 : 1) + (isfinite(v.y) ? 0 : 1) + (isfinite(v.z) ? 0 : 1) + (isfinite(v.w) ? 0 : 1);
+}
+__global__ void __launch_bounds__(NT) screen_count_kernel(const float4* __restrict__ W, int64_t wn4,
+                                                          const float4* __restrict__ H, int64_t hn4,
+                                                          const float* __restrict__ Hs, int64_t d_in,
+                                                          int32_t* __restrict__ scr) {
+  int bw = 0, bh = 0, neg = 0, zero = 0;
+  const int64_t stride = (int64_t)gridDim.x * NT, i0 = (int64_t)blockIdx.x * NT + threadIdx.x;
+  for (int64_t i = i0; i < wn4; i += stride) bw += bad4(W[i]);
+  for (int64_t i = i0; i < hn4; i += stride) bh += bad4(H[i]);
+  for (int64_t i = i0; i < d_in; i += stride) {
+    const float d = Hs[i * d_in + i];
+    neg += (d < 0.f) ? 1 : 0;
+    zero += (d == 0.f) ? 1 : 0;
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    bw += __shfl_xor_sync(0xffffffffu, bw, o); bh += __shfl_xor_sync(0xffffffffu, bh, o);
+    neg += __shfl_xor_sync(0xffffffffu, neg, o); zero += __shfl_xor_sync(0xffffffffu, zero, o);
+  }
+  if ((threadIdx.x & 31) == 0) {        // integer sums: the order does not matter
+    if (bw) atomicAdd(&scr[0], bw);
+    if (bh) atomicAdd(&scr[1], bh);
+    if (neg) atomicAdd(&scr[2], neg);
+    if (zero) atomicAdd(&scr[3], zero);
+  }
+}
+__global__ void screen_final_kernel(const int32_t* __restrict__ scr, int32_t* __restrict__ status) {
+  status[ST_NONFINITE_W] += scr[0];
+  status[ST_NONFINITE_H] += scr[1];
+  status[ST_NEG_DIAG_H] += scr[2];
+  status[ST_DEAD_CHANNELS] = scr[3];
+  const bool bad = scr[0] || scr[1] || scr[2];
+  status[ST_POISON] = bad ? 1 : 0;
+  if (bad) status[ST_LAST_ERR] = ARMOR_ERR_INVALID_ARG;
 }
 
 // ---- operand split for the three-pass tensor-core mode ------------------------------------------
@@ -410,7 +451,9 @@ __global__ void __launch_bounds__(NT) block_fro_kernel(const float4* __restrict_
 __global__ void __launch_bounds__(NT) adam_kernel(float4* __restrict__ theta, const float4* __restrict__ gamma,
                                                   float4* __restrict__ m, float4* __restrict__ v, int64_t n4,
                                                   const uint8_t* __restrict__ M, int q4, float lr, float b1, float b2,
-                                                  float eps, float inv_bc1, float inv_bc2) {
+                                                  float eps, float inv_bc1, float inv_bc2,
+                                                  const int32_t* __restrict__ status) {
+  if (status[ST_POISON] != 0) return;   // unusable inputs: parameters and moments stay as they are
   for (int64_t i = (int64_t)blockIdx.x * NT + threadIdx.x; i < n4; i += (int64_t)gridDim.x * NT) {
     const float4 ga = gamma[i];
     float4 mm = m[i], vv = v[i], th = theta[i];
@@ -511,6 +554,17 @@ void launch_init(armor_ctx* c, const float* W, const float* H, float* Wbar, floa
   c->launches += 3;
 }
 
+armor_status launch_screen_inputs(armor_ctx* c, const float* W, const float* H, cudaStream_t s) {
+  if (cudaMemsetAsync(c->screen, 0, 4 * sizeof(int32_t), s) != cudaSuccess) return ARMOR_ERR_CUDA;
+  const int64_t wn4 = c->wn / 4, hn4 = c->d_in * c->d_in / 4;
+  screen_count_kernel<<<grid_for(wn4 > hn4 ? wn4 : hn4), NT, 0, s>>>(reinterpret_cast<const float4*>(W), wn4,
+                                                                     reinterpret_cast<const float4*>(H), hn4, H, c->d_in,
+                                                                     c->screen);
+  screen_final_kernel<<<1, 1, 0, s>>>(c->screen, c->status);
+  c->launches += 2;
+  return ARMOR_OK;
+}
+
 void launch_zero_scalars(armor_ctx* c, cudaStream_t s) {
   const int nflag = c->nbo > c->nbi ? c->nbo : c->nbi;
   zero_scalars_kernel<<<1, NT, 0, s>>>(c->sc, c->failflag, nflag);
@@ -559,7 +613,8 @@ void launch_adam(armor_ctx* c, float* theta, const float* gamma, float* m, float
   const float eps = c->cfg.adam_eps > 0.f ? c->cfg.adam_eps : 1e-8f;
   const double bc1 = 1.0 - pow((double)b1, (double)step), bc2 = 1.0 - pow((double)b2, (double)step);
   adam_kernel<<<grid_for(n / 4), NT, 0, s>>>((float4*)theta, (const float4*)gamma, (float4*)m, (float4*)v, n / 4, M,
-                                            c->cfg.m_group / 4, lr, b1, b2, eps, (float)(1.0 / bc1), (float)(1.0 / bc2));
+                                            c->cfg.m_group / 4, lr, b1, b2, eps, (float)(1.0 / bc1), (float)(1.0 / bc2),
+                                            c->status);
   c->launches++;
 }
 

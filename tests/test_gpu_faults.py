@@ -1,0 +1,119 @@
+"""Failure detection without a GPU fault: a bounded wait that is made to run out, and inputs the method cannot
+use (NaN / Inf in W or H, a negative diagonal entry of H) or can use but should report (a dead channel).  Every
+case is produced on the host; the device only ever sees ordinary launches."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import armor_oracle as O
+from paper_2510_05528_b200 import binding as Bd
+from paper_2510_05528_b200 import inputs
+from tests.helpers import DEV, TOL, dev, host, load_state, make, rel
+
+pytestmark = pytest.mark.gpu
+
+TINY = inputs.CONFIGS["tiny"]
+MID = TINY.with_(name="mid", d_out=384, d_in=512, d_block=128, n_tokens=6000, chunk_rows=2048, seed=11)
+ST_TIMEOUTS, ST_LAST, ST_BAD_W, ST_BAD_H, ST_NEG, ST_DEAD, ST_POISON = 2, 3, 5, 6, 7, 8, 9
+ERR_INVALID_ARG, ERR_TIMEOUT = 1, 6
+
+
+def data(cfg):
+    W = inputs.make_weight(cfg)
+    X = inputs.make_activations(cfg)
+    return W, X, O.gram(X).astype(np.float32)
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    W, X, H32 = data(MID)
+    ctx = make(MID, Bd.PREC_FP16X3)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    before = ctx.proxy_loss(st, Hd).item()
+    res = torch.full((2,), -1, dtype=torch.int32, device=DEV)
+    Bd.armor_selftest_wait_timeout(ctx.ctx, 200_000, res)          # about 0.1 ms of spinning
+    status = ctx.device_status()
+    assert res.tolist() == [0, 1]                                  # gave up; the abort flag is up
+    assert status[ST_TIMEOUTS] == 1 and status[ST_LAST] == ERR_TIMEOUT
+    Bd.armor_selftest_wait_timeout(ctx.ctx, 1000, res)
+    assert ctx.device_status()[ST_TIMEOUTS] == 2
+    # the tensor-core kernels (which share the wait routine and the status words) still run and agree
+    assert ctx.proxy_loss(st, Hd).item() == before
+    sg = ctx.read_stats(ctx.bcd_step(st, Hd, 0, 1))[0]
+    assert sg["loss_mask"] < sg["loss_start"] and ctx.device_status()[ST_TIMEOUTS] == 2
+    with pytest.raises(Bd.ArmorError):
+        Bd.armor_selftest_wait_timeout(ctx.ctx, 0, res)
+
+
+@pytest.mark.parametrize("cfg,prec", [(TINY, Bd.PREC_SIMT), (MID, Bd.PREC_FP16X3), (MID, Bd.PREC_FP32X3)],
+                         ids=["tiny-simt", "mid-fp16x3", "mid-fp32x3"])
+def test_unusable_inputs_are_counted_and_every_update_is_withheld(cfg, prec):
+    W, X, H32 = data(cfg)
+    ctx = make(cfg, prec)
+    Hd, Wd = dev(H32), dev(W)
+    st = ctx.init(Wd, Hd)
+    ctx.bcd_step(st, Hd, 0, 1, want_stats=False)                   # a state away from the initialisation
+    keep = [host(t).copy() for t in (st.A, st.B, st.S, st.M)]
+    assert ctx.device_status()[ST_BAD_W:ST_POISON + 1] == [0, 0, 0, 0, 0]
+
+    def unchanged():
+        return all(np.array_equal(host(t), k) for t, k in zip((st.A, st.B, st.S, st.M), keep))
+
+    # one NaN in W
+    Wbad = W.copy(); Wbad[3, 7] = np.nan
+    st.Wbar.copy_(dev(Wbad))
+    sg = ctx.read_stats(ctx.bcd_step(st, Hd, 1, 2))
+    s = ctx.device_status()
+    assert unchanged() and s[ST_BAD_W] == 1 and s[ST_POISON] == 1 and s[ST_LAST] == ERR_INVALID_ARG
+    assert int(sg["mask_accepted"].sum()) == 0 and int(sg["groups_changed"].sum()) == 0
+    assert float(sg["tau_B"].max()) == 0.0 and float(sg["tau_S"].max()) == 0.0
+    st.Wbar.copy_(Wd)
+    # Inf in H (two entries: the matrix is symmetric)
+    Hbad = H32.copy(); Hbad[5, 9] = Hbad[9, 5] = np.inf
+    ctx.bcd_step(st, dev(Hbad), 1, 1, want_stats=False)
+    s = ctx.device_status()
+    assert unchanged() and s[ST_BAD_H] == 2 and s[ST_BAD_W] == 1 and s[ST_POISON] == 1
+    # a negative diagonal entry: not a Gram matrix
+    Hneg = H32.copy(); Hneg[11, 11] = -Hneg[11, 11]
+    ctx.bcd_step(st, dev(Hneg), 1, 1, want_stats=False)
+    s = ctx.device_status()
+    assert unchanged() and s[ST_NEG] == 1 and s[ST_POISON] == 1
+    # clean inputs again: the same context carries on and follows the oracle
+    A, B, S = (k.astype(np.float64) for k in keep[:3])
+    M = O.unpack_mask(keep[3])
+    oc = O.OracleConfig(cfg.d_block, seed=cfg.seed)
+    A1, B1, S1, M1, info = O.bcd_iteration(W.astype(np.float64), A, B, S, M, H32.astype(np.float64), oc, 1)
+    sg = ctx.read_stats(ctx.bcd_step(st, Hd, 1, 1))[0]
+    s = ctx.device_status()
+    assert s[ST_POISON] == 0 and s[ST_BAD_W] == 1 and s[ST_BAD_H] == 2 and s[ST_NEG] == 1
+    tol = TOL[prec]
+    assert rel(host(st.A), A1) < tol["A"] and rel(host(st.B), B1) < tol["B"]
+    assert abs(sg["loss_S"] - info.loss["S"]) / info.loss["S"] < tol["loss"]
+    # armor_init screens its inputs as well
+    ctx.init(dev(Wbad), Hd)
+    assert ctx.device_status()[ST_BAD_W] == 2
+
+
+def test_a_dead_channel_is_reported_and_handled():
+    """A channel that is zero on every calibration token: row and column of H vanish.  Legal input (the channel
+    carries no weight): counted in its status word, no block solve fails, and the iteration follows the oracle."""
+    cfg = MID
+    W = inputs.make_weight(cfg)
+    X = inputs.make_activations(cfg).copy()
+    X[:, 37] = 0.0
+    H32 = O.gram(X).astype(np.float32)
+    ctx = make(cfg, Bd.PREC_FP16X3)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    oc = O.OracleConfig(cfg.d_block, seed=cfg.seed)
+    Wn, Hq = W.astype(np.float64), H32.astype(np.float64)
+    A, B, S, M = O.init(Wn, Hq, oc)
+    assert np.array_equal(host(st.M), O.pack_mask(M))
+    sg = ctx.read_stats(ctx.bcd_step(st, Hd, 0, 1))[0]
+    A, B, S, M, info = O.bcd_iteration(Wn, A, B, S, M, Hq, oc, 0)
+    s = ctx.device_status()
+    assert s[ST_DEAD] == 1 and s[ST_POISON] == 0 and s[0] == 0 and sg["chol_failed"] == info.chol_failed == 0
+    tol = TOL[Bd.PREC_FP16X3]
+    assert rel(host(st.A), A) < tol["A"] and rel(host(st.B), B) < tol["B"]
+    for k_gpu, k_or in (("loss_start", "start"), ("loss_A", "A"), ("loss_B", "B"), ("loss_S", "S")):
+        assert abs(sg[k_gpu] - info.loss[k_or]) / info.loss[k_or] < tol["loss"]
