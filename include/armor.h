@@ -104,7 +104,9 @@ typedef struct {
 
 /* One record per BCD iteration, written on the device.  The losses after the
  * sub-steps follow from loss_start by the exact decrease of each quadratic
- * step; loss_start itself is evaluated from the residual. */
+ * step.  loss_start is evaluated from the residual in the first iteration of a
+ * call and every 64 iterations after it (and in every iteration with
+ * ARMOR_AB_ADAM); in between it is the previous iteration's loss_mask. */
 typedef struct {
   double loss_start, loss_A, loss_B, loss_S, loss_mask;
   double delta_L_mask;   /* exact loss change of the iteration's group updates (summed over the sweeps) */

@@ -5,6 +5,7 @@
 
 namespace {
 
+constexpr int LOSS_REFRESH = 64;      // iterations of a call between two evaluations of the loss from the residual
 constexpr int64_t GRAM_ROWS = 16384;  // rows of X staged (transposed, split) per tensor-core Gram pass
 
 struct Layout {
@@ -407,7 +408,11 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
   for (int it = 0; it < n_iters; ++it) {
     armor_iter_stats* is = d_stats ? d_stats + it : nullptr;
     const int64_t t = t_first + it;
-    launch_zero_scalars(c, s);
+    // The loss at the start of an iteration is evaluated from the residual in the first iteration of a call and
+    // every LOSS_REFRESH iterations after it; in between it is the loss the previous iteration ended with, which
+    // follows from the evaluated one by the exact decreases of the quadratic sub-steps.
+    const bool fresh_loss = adam || (it % LOSS_REFRESH == 0);
+    launch_zero_scalars(c, !fresh_loss, s);
     if (adam) {
       // Adam normalises every entry's move, so a gradient that is exactly zero (the kept entries of the core at
       // the initialisation, where E vanishes on them) must come out as zero: E H_w is formed from E itself, not
@@ -422,8 +427,10 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       if (st != ARMOR_OK) return st;
     }
     bd_left(c, A, false, c->P, c->EH, d_out, d_in, -1.f, c->WH, 1.f, s);             // E H_w = W H_w - A P
-    bd_left(c, A, false, c->T, c->E, d_out, d_in, -1.f, W, 1.f, s);                  // E = W - A T
-    dot_to_ptr(c, c->EH, c->E, c->wn, c->sc + SC_L0, s);                             // L = <E H_w, E>
+    if (fresh_loss) {
+      bd_left(c, A, false, c->T, c->E, d_out, d_in, -1.f, W, 1.f, s);                // E = W - A T
+      dot_to_ptr(c, c->EH, c->E, c->wn, c->sc + SC_L0, s);                           // L = <E H_w, E>
+    }
     launch_stage(c, is, 0, nullptr, 0, 0, s);
     }
 

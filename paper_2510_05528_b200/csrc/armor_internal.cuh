@@ -238,7 +238,7 @@ void launch_axpy_slot(armor_ctx* c, float* y, const float* x, int64_t n, int slo
                       cudaStream_t s);                                       // y += sign * sc[slot] * x
 void launch_init(armor_ctx* c, const float* W, const float* H, float* Wbar, float* r1, float* r2,
                  float* A, float* B, float* S, uint8_t* M, cudaStream_t s);
-void launch_zero_scalars(armor_ctx* c, cudaStream_t s);
+void launch_zero_scalars(armor_ctx* c, bool carry_loss, cudaStream_t s);
 // Input screening at the top of a call: counts non-finite entries of W and H and negative / zero diagonal
 // entries of H into the status words and sets or clears ST_POISON for the call.
 armor_status launch_screen_inputs(armor_ctx* c, const float* W, const float* H, cudaStream_t s);

@@ -114,7 +114,7 @@ __device__ __forceinline__ bool chol_small(int n, const double (&Kin)[NKM][NKM],
 // One CTA per (i, j) block of the core, N:M groups with M = MG (4 or 8) and N = n_keep (<= NKM: 4 for 2:4 and 4:8, 6 for 5:8 and 6:8).
 // Pass 1: every group of the block is scored, keyed and the arg-min found by warp shuffles.
 // Pass 2: thread b < 2^MG evaluates the mask with bit pattern b (if it keeps exactly n_keep positions);
-// the best one is found with the oracle's order: larger reduction first; among equal reductions the
+// the best one is found in this order: larger reduction first; among equal reductions the
 // incumbent, then the lexicographically first index tuple.
 template <int MG, int NKM, bool MULTI>
 __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict__ Gam, const float* __restrict__ S,
@@ -135,45 +135,81 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
   const int blk = bi * (kg * nbi) + kk * nbi + bj;
   float best_key = INFINITY;
   uint64_t best_g = ~0ull;
-  for (int idx = threadIdx.x; idx < n_in_block; idx += NT) {
-    const int rl = idx / gpb, cl = idx % gpb;
-    const int64_t row = (int64_t)bi * db + rl;
-    const int64_t cg = (int64_t)bj * gpb + cl;
-    if (MULTI && kk > 0) {                                  // later draws: keys from the first pass, drawn ones at +inf
+  if (MULTI && kk > 0) {
+    // later draws: keys from the first pass, drawn ones at +inf
+    for (int idx = threadIdx.x; idx < n_in_block; idx += NT) {
+      const int rl = idx / gpb, cl = idx % gpb;
       const float key = s_keys[idx];
-      const uint64_t g = (uint64_t)row * (uint64_t)ng_row + (uint64_t)cg;
+      const uint64_t g = (uint64_t)((int64_t)bi * db + rl) * (uint64_t)ng_row + (uint64_t)((int64_t)bj * gpb + cl);
       if (key < best_key || (key == best_key && g < best_g)) { best_key = key; best_g = g; }
-      continue;
     }
-    float score = 0.f, sq = 0.f;
+  } else {
+    // Four groups per thread and step: the loads are issued together, then scores and hashes.  With a single
+    // draw most logarithms are skipped: -ln(u) >= 1 - u, so a group whose (1 - u) / score already reaches the
+    // thread's best key cannot win (the bound is tight exactly where winners live, u next to 1).  A thread
+    // meets its groups in ascending order, so a tie never replaces an earlier group either.
+    constexpr int U = 4;
+    for (int base = threadIdx.x; base < n_in_block; base += U * NT) {
+      float4 g4[U][MG / 4];
+      float al[U];
 #pragma unroll
-    for (int h = 0; h < MG / 4; ++h) {
-      const float4 g4 = *reinterpret_cast<const float4*>(Gam + row * d_in + cg * MG + 4 * h);
-      score += fabsf(g4.x);
-      score += fabsf(g4.y);
-      score += fabsf(g4.z);
-      score += fabsf(g4.w);
-      sq = fmaf(g4.x, g4.x, sq);
-      sq = fmaf(g4.y, g4.y, sq);
-      sq = fmaf(g4.z, g4.z, sq);
-      sq = fmaf(g4.w, g4.w, sq);
-    }
-    // the ablation's weights (Appendix E.1): L2 norm of the group's gradient, or equal weights
-    if (select_mode == ARMOR_SELECT_L2_RANDOM) score = sqrtf(sq);
-    else if (select_mode == ARMOR_SELECT_UNIFORM_RANDOM) score = 1.f;
-    if (!(alpha[row] > 0.f)) score = 0.f;
-    const uint64_t g = (uint64_t)row * (uint64_t)ng_row + (uint64_t)cg;
-    float key = INFINITY;
-    if (score > 0.f) {
-      if (select_mode != ARMOR_SELECT_L1_GREEDY) {
-        const uint64_t bits = splitmix64(seed ^ splitmix64(t * n_groups_total + g));
-        key = neg_log_uniform((uint32_t)(bits >> 40)) / score;
-      } else {
-        key = -score;
+      for (int u = 0; u < U; ++u) {
+        const int idx = base + u * NT;
+        al[u] = 0.f;
+#pragma unroll
+        for (int h = 0; h < MG / 4; ++h) g4[u][h] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (idx < n_in_block) {
+          const int rl = idx / gpb, cl = idx % gpb;
+          const int64_t row = (int64_t)bi * db + rl;
+          const int64_t cg = (int64_t)bj * gpb + cl;
+          al[u] = alpha[row];
+#pragma unroll
+          for (int h = 0; h < MG / 4; ++h)
+            g4[u][h] = *reinterpret_cast<const float4*>(Gam + row * d_in + cg * MG + 4 * h);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int idx = base + u * NT;
+        if (idx >= n_in_block) continue;
+        const int rl = idx / gpb, cl = idx % gpb;
+        const int64_t row = (int64_t)bi * db + rl;
+        const int64_t cg = (int64_t)bj * gpb + cl;
+        float score = 0.f, sq = 0.f;
+#pragma unroll
+        for (int h = 0; h < MG / 4; ++h) {
+          score += fabsf(g4[u][h].x);
+          score += fabsf(g4[u][h].y);
+          score += fabsf(g4[u][h].z);
+          score += fabsf(g4[u][h].w);
+          sq = fmaf(g4[u][h].x, g4[u][h].x, sq);
+          sq = fmaf(g4[u][h].y, g4[u][h].y, sq);
+          sq = fmaf(g4[u][h].z, g4[u][h].z, sq);
+          sq = fmaf(g4[u][h].w, g4[u][h].w, sq);
+        }
+        // the ablation's weights (Appendix E.1): L2 norm of the group's gradient, or equal weights
+        if (select_mode == ARMOR_SELECT_L2_RANDOM) score = sqrtf(sq);
+        else if (select_mode == ARMOR_SELECT_UNIFORM_RANDOM) score = 1.f;
+        if (!(al[u] > 0.f)) score = 0.f;
+        const uint64_t g = (uint64_t)row * (uint64_t)ng_row + (uint64_t)cg;
+        float key = INFINITY;
+        if (score > 0.f) {
+          if (select_mode != ARMOR_SELECT_L1_GREEDY) {
+            const uint64_t bits = splitmix64(seed ^ splitmix64(t * n_groups_total + g));
+            const uint32_t k24 = (uint32_t)(bits >> 40);
+            // 1 - u = (2^24 - k24 - 1/2) 2^-24, exact in fp32; the factor 1 - 1e-5 covers the few ulp by which the
+            // computed key can fall below (1 - u) / score
+            const float one_minus_u = (float)(2u * ((1u << 24) - k24) - 1u) * 2.98023223876953125e-8f;
+            if (MULTI || !(one_minus_u * 0.99999f >= best_key * score))
+              key = neg_log_uniform(k24) / score;
+          } else {
+            key = -score;
+          }
+        }
+        if (MULTI) s_keys[idx] = key;
+        if (key < best_key || (key == best_key && g < best_g)) { best_key = key; best_g = g; }
       }
     }
-    if (MULTI) s_keys[idx] = key;
-    if (key < best_key || (key == best_key && g < best_g)) { best_key = key; best_g = g; }
   }
   // arg-min over the CTA; ties go to the lower group index
   for (int o = 16; o > 0; o >>= 1) {

@@ -212,8 +212,11 @@ __global__ void copy_kernel(const float4* __restrict__ in, float4* __restrict__ 
 }
 
 // ---- scalars and per-iteration bookkeeping ------------------------------------------------------
-__global__ void zero_scalars_kernel(double* sc, int32_t* failflag, int nflag) {
-  for (int i = threadIdx.x; i < SC_COUNT; i += blockDim.x) sc[i] = 0.0;
+// carry_loss: the running loss of the previous iteration becomes this iteration's starting loss
+__global__ void zero_scalars_kernel(double* sc, int32_t* failflag, int nflag, int carry_loss) {
+  const double carried = sc[SC_LOSS];
+  __syncthreads();
+  for (int i = threadIdx.x; i < SC_COUNT; i += blockDim.x) sc[i] = (carry_loss && i == SC_L0) ? carried : 0.0;
   for (int i = threadIdx.x; i < nflag; i += blockDim.x) failflag[i] = 0;
 }
 
@@ -565,9 +568,9 @@ armor_status launch_screen_inputs(armor_ctx* c, const float* W, const float* H, 
   return ARMOR_OK;
 }
 
-void launch_zero_scalars(armor_ctx* c, cudaStream_t s) {
+void launch_zero_scalars(armor_ctx* c, bool carry_loss, cudaStream_t s) {
   const int nflag = c->nbo > c->nbi ? c->nbo : c->nbi;
-  zero_scalars_kernel<<<1, NT, 0, s>>>(c->sc, c->failflag, nflag);
+  zero_scalars_kernel<<<1, NT, 0, s>>>(c->sc, c->failflag, nflag, carry_loss ? 1 : 0);
   c->launches++;
 }
 
