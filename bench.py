@@ -167,6 +167,25 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+def kernel_table_rows(raw, peaks):
+    """Per kernel class: launches, device time, algorithmic work per second and its fraction of the bound that
+    applies (HBM copy bandwidth for the streaming classes, nothing for the classes of small kernels)."""
+    rows = {}
+    total = sum(ms for _, ms, _ in raw.values())
+    for name, (n, ms, work) in raw.items():
+        if n == 0:
+            continue
+        row = {"launches": n, "total_ms": ms, "avg_us": 1e3 * ms / n, "share": ms / total if total else None}
+        if work > 0 and ms > 0:
+            if name in ("gemm", "cholesky"):
+                row["tflops"] = work / (ms * 1e-3) / 1e12
+            else:
+                row["gb_per_s"] = work / (ms * 1e-3) / 1e9
+                row["frac_of_hbm_peak"] = row["gb_per_s"] / peaks["hbm_gbs"]
+        rows[name] = row
+    return rows
+
+
 def workload_config(cfg, precision):
     return {"workload": f"{cfg.name}: W {cfg.d_out}x{cfg.d_in} fp32, d_block {cfg.d_block}, 2:4, {cfg.n_tokens} calibration "
                         f"tokens, {cfg.n_iters} BCD iterations, h_mode FULL, apply on {APPLY_TOKENS} tokens",
@@ -344,6 +363,18 @@ def run_ours(args, cfg):
     ms_apply, _ = t_phase(lambda: ctx.apply(st, xt_d))
     srec = ctx.read_stats(stats)
 
+    # ---- every kernel class of one more step, each launch bracketed by events on its stream (the brackets cost
+    # about a microsecond per launch, so this step is not part of the headline)
+    kernel_table = None
+    if args.kernel_table:
+        Bd.armor_kernel_timing_enable(ctx.ctx, 2)
+        Bd.armor_kernel_timing(ctx.ctx)
+        step_resident()
+        torch.cuda.synchronize()
+        raw = Bd.armor_kernel_timing(ctx.ctx)
+        Bd.armor_kernel_timing_enable(ctx.ctx, 0)
+        kernel_table = kernel_table_rows(raw, load_peaks()[0])
+
     # ---- the one-pass tf32 mode on the same workload (context only; not the headline: its parity tolerance
     # is looser, see tests/helpers.py)
     tf32_mode = None
@@ -478,6 +509,7 @@ def run_ours(args, cfg):
                 "pipelined_note": "same copies, but the tokens of step k+1 are uploaded while step k iterates; the first "
                                   "of the timed steps uploads its own under its Gram"},
         "gpu_launches": int(launches),
+        "kernel_table": kernel_table,
         "tf32_mode": tf32_mode,
         "other_modes": other_modes,
         "clocks": clocks,
@@ -515,6 +547,9 @@ def main():
                     help="profiling aid: BCD iterations per step instead of the workload's")
     ap.add_argument("--no-e2e", action="store_true", help="profiling aid: skip the host-buffer leg")
     ap.add_argument("--no-tf32", action="store_true", help="skip the extra measurement of the one-pass tf32 mode")
+    ap.add_argument("--kernel-table", action="store_true",
+                    help="also run one step with every launch bracketed by events and report time, algorithmic "
+                         "bytes per second and the fraction of the HBM roofline per kernel class")
     ap.add_argument("--other-modes", action="store_true",
                     help="also time the BCD loop with the diagonal weighting, the joint Adam step and several "
                          "sparse-core updates per iteration (a few seconds more)")

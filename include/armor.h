@@ -260,6 +260,35 @@ int64_t armor_launch_count(const armor_ctx* ctx);
 armor_status armor_gemm_timing_enable(armor_ctx* ctx, int32_t enable);
 armor_status armor_gemm_timing(armor_ctx* ctx, int64_t* n_launches, double* total_ms, double* total_flops);
 
+/* The same measurement aid for every kernel class (no counterpart in the paper).  Level 0: off; 1: the dense
+ * tensor-core products only (what armor_gemm_timing_enable(ctx, 1) sets); 2: every launch of the context is
+ * bracketed by a pair of events on its stream (at most 8192 launches are recorded between two reads; the pairs
+ * cost about a microsecond each, so time a step as a whole with level 0 or 1).
+ * armor_kernel_timing waits for the recorded events and returns, for the classes 0 .. n_classes - 1, the number
+ * of launches, their summed device time in ms and their summed algorithmic work: flops for ARMOR_KC_GEMM
+ * (single-pass, 2 M N K; M (N + 128) K for the lower-triangle Gram) and ARMOR_KC_CHOLESKY, bytes that must cross
+ * HBM for all others (0 for classes of small kernels).  It clears the record. */
+enum {
+  ARMOR_KC_GEMM = 0,           /* dense tensor-core products: Gram, .H, the forward's core */
+  ARMOR_KC_BLOCK_PRODUCT = 1,  /* products of a W-shaped matrix with the block-diagonal wrappers: 8 B / element, 12 with an addend */
+  ARMOR_KC_BLOCK_GRAM = 2,     /* per-block Gram matrices over d_in or d_out: two W-shaped operands read */
+  ARMOR_KC_CHOLESKY = 3,       /* per-block factorisation and two triangular solves: (7/3) d_block^3 flops per block */
+  ARMOR_KC_AXPY = 4,           /* y += a x on W-shaped arrays (12 B / element), column scale, Adam update */
+  ARMOR_KC_DOT = 5,            /* dot products of W-shaped arrays: 8 B / element */
+  ARMOR_KC_MASKED_COPY = 6,    /* Gamma (.) M with its squared norm */
+  ARMOR_KC_MASK_SELECT = 7,    /* scoring, selection and mask sweep: one read of Gamma, 4 B / element */
+  ARMOR_KC_MASK_GUARD = 8,     /* the other kernels of the sparse-core update (vectors, thin product with H, commit, carry) */
+  ARMOR_KC_OPERAND_SPLIT = 9,  /* high / low parts of a dense product's operands: 8 B / element */
+  ARMOR_KC_GRAM_STAGING = 10,  /* channel maxima, transposition and split of a chunk of activations */
+  ARMOR_KC_INIT = 11,          /* normalisation, initial masks and core, input screening */
+  ARMOR_KC_SMALL = 12,         /* reductions, bookkeeping, small block products */
+  ARMOR_KC_FORWARD = 13,       /* conversions, packing and wrapper products of the deployment form */
+  ARMOR_KC_COUNT = 14
+};
+armor_status armor_kernel_timing_enable(armor_ctx* ctx, int32_t level);
+armor_status armor_kernel_timing(armor_ctx* ctx, int32_t n_classes, int64_t* launches, double* total_ms,
+                                 double* total_work);
+
 /* One product with a block-diagonal wrapper (Section 3.1: A and B are applied as batched d_block x d_block
  * products), exposed for tests and measurements; armor_bcd_step and armor_apply are built from it.
  *   side 0: d_out[:, j-th block] = alpha * d_in[:, j-th block] * Q_j (+ beta * d_add[:, j-th block])

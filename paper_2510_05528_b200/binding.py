@@ -29,7 +29,8 @@ EXPORTS = ["armor_workspace_bytes", "armor_create", "armor_destroy", "armor_gram
            "armor_packed_layer_bytes", "armor_pack_layer", "armor_apply_layer",
            "armor_get_device_status",
            "armor_status_string", "armor_launch_count", "armor_gemm_timing_enable", "armor_gemm_timing",
-           "armor_normalize_noalloc", "armor_block_product", "armor_selftest_wait_timeout"]
+           "armor_normalize_noalloc", "armor_block_product", "armor_selftest_wait_timeout", "armor_kernel_timing_enable",
+           "armor_kernel_timing"]
 
 
 class ArmorError(RuntimeError):
@@ -85,6 +86,8 @@ def lib() -> C.CDLL:
         L.armor_block_product.argtypes = [vp, i32, i32, vp, vp, vp, i64, i64, C.c_float, vp, C.c_float, i32, vp]
         L.armor_gemm_timing_enable.argtypes = [vp, i32]
         L.armor_gemm_timing.argtypes = [vp, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
+        L.armor_kernel_timing_enable.argtypes = [vp, i32]
+        L.armor_kernel_timing.argtypes = [vp, i32, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.armor_selftest_wait_timeout.argtypes = [vp, i64, vp, vp]
         for name in EXPORTS:
             if name not in ("armor_status_string", "armor_launch_count"):
@@ -264,6 +267,22 @@ def armor_block_product(ctx, side: int, transpose: bool, blocks, x, out, alpha=1
 
 def armor_gemm_timing_enable(ctx, enable: bool) -> None:
     _check(lib().armor_gemm_timing_enable(ctx, int(bool(enable))), "armor_gemm_timing_enable")
+
+
+KERNEL_CLASSES = ["gemm", "block_product", "block_gram", "cholesky", "axpy", "dot", "masked_copy", "mask_select",
+                  "mask_guard", "operand_split", "gram_staging", "init", "small", "forward"]
+
+
+def armor_kernel_timing_enable(ctx, level: int) -> None:
+    _check(lib().armor_kernel_timing_enable(ctx, int(level)), "armor_kernel_timing_enable")
+
+
+def armor_kernel_timing(ctx) -> dict:
+    """{class name: (launches, total ms, total work)} since the last read; clears the record."""
+    n = len(KERNEL_CLASSES)
+    cnt, ms, work = (C.c_int64 * n)(), (C.c_double * n)(), (C.c_double * n)()
+    _check(lib().armor_kernel_timing(ctx, n, cnt, ms, work), "armor_kernel_timing")
+    return {name: (int(cnt[k]), float(ms[k]), float(work[k])) for k, name in enumerate(KERNEL_CLASSES)}
 
 
 def armor_gemm_timing(ctx) -> tuple[int, float, float]:

@@ -135,6 +135,8 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   TAKE(quadpart, double*, (size_t)nbo * nbi * kg * sizeof(double));
   TAKE(failflag, int32_t*, (size_t)nbmax * sizeof(int32_t));
   TAKE(sel, SelRec*, (size_t)nbo * nbi * kg * sizeof(SelRec));
+  TAKE(tab_key, float*, (size_t)nbo * nbi * sizeof(float));
+  TAKE(tab_g, unsigned long long*, (size_t)nbo * nbi * sizeof(unsigned long long));
   TAKE(status, int32_t*, ST_COUNT * sizeof(int32_t));
   TAKE(screen, int32_t*, 4 * sizeof(int32_t));
 #undef TAKE
@@ -291,7 +293,8 @@ armor_status armor_create(armor_ctx** out, const armor_config* cfg, void* d_work
   }
   c->kg = cfg->mask_groups > 0 ? cfg->mask_groups : 1;
   c->h_cached = nullptr;
-  c->timing_on = 0; c->timing_n = 0; c->ev_beg = nullptr; c->ev_end = nullptr; c->ev_created = 0; c->timing_flops = 0.0;
+  c->timing_on = 0; c->timing_n = 0; c->ev_beg = nullptr; c->ev_end = nullptr; c->ev_cls = nullptr; c->ev_work = nullptr;
+  c->ev_created = 0;
   carve(*cfg, c, c->ws);
   if (cudaMemset(c->status, 0, ST_COUNT * sizeof(int32_t)) != cudaSuccess) { delete c; return ARMOR_ERR_CUDA; }
   if (cudaMemset(c->sc, 0, SC_COUNT * sizeof(double)) != cudaSuccess) { delete c; return ARMOR_ERR_CUDA; }
@@ -304,18 +307,22 @@ armor_status armor_destroy(armor_ctx* c) {
   for (int i = 0; i < c->ev_created; ++i) { cudaEventDestroy(c->ev_beg[i]); cudaEventDestroy(c->ev_end[i]); }
   delete[] c->ev_beg;
   delete[] c->ev_end;
+  delete[] c->ev_cls;
+  delete[] c->ev_work;
   delete c;
   return ARMOR_OK;
 }
 
 int64_t armor_launch_count(const armor_ctx* c) { return c ? c->launches : -1; }
 
-armor_status armor_gemm_timing_enable(armor_ctx* c, int32_t enable) {
-  if (!c) return ARMOR_ERR_INVALID_ARG;
-  if (enable && c->ev_created < ARMOR_MAX_TIMED) {
+armor_status armor_kernel_timing_enable(armor_ctx* c, int32_t level) {
+  if (!c || level < 0 || level > 2) return ARMOR_ERR_INVALID_ARG;
+  if (level && c->ev_created < ARMOR_MAX_TIMED) {
     if (!c->ev_beg) c->ev_beg = new (std::nothrow) cudaEvent_t[ARMOR_MAX_TIMED];
     if (!c->ev_end) c->ev_end = new (std::nothrow) cudaEvent_t[ARMOR_MAX_TIMED];
-    if (!c->ev_beg || !c->ev_end) return ARMOR_ERR_INVALID_ARG;
+    if (!c->ev_cls) c->ev_cls = new (std::nothrow) int32_t[ARMOR_MAX_TIMED];
+    if (!c->ev_work) c->ev_work = new (std::nothrow) double[ARMOR_MAX_TIMED];
+    if (!c->ev_beg || !c->ev_end || !c->ev_cls || !c->ev_work) return ARMOR_ERR_INVALID_ARG;
     // (an earlier call may have stopped part of the way: continue from the pairs that exist)
     for (int i = c->ev_created; i < ARMOR_MAX_TIMED; ++i) {
       if (cudaEventCreate(&c->ev_beg[i]) != cudaSuccess) return ARMOR_ERR_CUDA;
@@ -323,25 +330,32 @@ armor_status armor_gemm_timing_enable(armor_ctx* c, int32_t enable) {
       c->ev_created = i + 1;
     }
   }
-  c->timing_on = enable ? 1 : 0;
+  c->timing_on = level;
   return ARMOR_OK;
 }
 
-armor_status armor_gemm_timing(armor_ctx* c, int64_t* n_launches, double* total_ms, double* total_flops) {
-  if (!c || !n_launches || !total_ms || !total_flops) return ARMOR_ERR_INVALID_ARG;
-  double ms = 0.0;
+armor_status armor_kernel_timing(armor_ctx* c, int32_t n_classes, int64_t* launches, double* total_ms, double* total_work) {
+  if (!c || !launches || !total_ms || !total_work || n_classes < 1) return ARMOR_ERR_INVALID_ARG;
+  for (int k = 0; k < n_classes; ++k) { launches[k] = 0; total_ms[k] = 0.0; total_work[k] = 0.0; }
   for (int i = 0; i < c->timing_n; ++i) {
     ARMOR_CUDA_OK(cudaEventSynchronize(c->ev_end[i]));
     float t = 0.f;
     ARMOR_CUDA_OK(cudaEventElapsedTime(&t, c->ev_beg[i], c->ev_end[i]));
-    ms += (double)t;
+    const int k = c->ev_cls[i];
+    if (k < 0 || k >= n_classes) continue;
+    launches[k] += 1;
+    total_ms[k] += (double)t;
+    total_work[k] += c->ev_work[i];
   }
-  *n_launches = c->timing_n;
-  *total_ms = ms;
-  *total_flops = c->timing_flops;
   c->timing_n = 0;
-  c->timing_flops = 0.0;
   return ARMOR_OK;
+}
+
+armor_status armor_gemm_timing_enable(armor_ctx* c, int32_t enable) { return armor_kernel_timing_enable(c, enable ? 1 : 0); }
+
+armor_status armor_gemm_timing(armor_ctx* c, int64_t* n_launches, double* total_ms, double* total_flops) {
+  if (!c || !n_launches || !total_ms || !total_flops) return ARMOR_ERR_INVALID_ARG;
+  return armor_kernel_timing(c, 1, n_launches, total_ms, total_flops);
 }
 
 armor_status armor_get_device_status(armor_ctx* c, int32_t* h_codes, int32_t n) {

@@ -95,6 +95,8 @@ struct armor_ctx {
   double* colpart;    // [64][d_in] column partial sums of the normalisation
   int32_t* failflag;  // [max(nbo, nbi)]
   SelRec* sel;        // [nbo * nbi]
+  float* tab_key;     // [nbo * nbi] winning race key of every block (single draw)
+  unsigned long long* tab_g;   // its global group index
   int32_t* status;    // [ST_COUNT]
   int32_t* screen;    // [4] per-call counters of the input screening
   int64_t launches;
@@ -108,15 +110,31 @@ struct armor_ctx {
                         // rounded to 8 bits anyway); 0: three passes, fp32-grade
   // identity of the H whose low part is cached in Hlo
   const float* h_cached;
-  // optional event timing of the tensor-core GEMM launches
+  // optional event timing of the launches: 0 off, 1 the dense tensor-core products only, 2 every kernel class
   int timing_on;
   int timing_n;              // launches recorded
   cudaEvent_t* ev_beg;       // [ARMOR_MAX_TIMED]
   cudaEvent_t* ev_end;
+  int32_t* ev_cls;           // kernel class of the recorded launch (ARMOR_KC_*)
+  double* ev_work;           // its algorithmic work: flops (dense products, Cholesky) or bytes (everything else)
   int ev_created;
-  double timing_flops;
 };
-static const int ARMOR_MAX_TIMED = 4096;
+static const int ARMOR_MAX_TIMED = 8192;
+
+// Brackets the launches made during its lifetime with a pair of events on the launching stream when timing is on.
+struct KTimer {
+  armor_ctx* c; cudaStream_t s; int slot;
+  KTimer(armor_ctx* c_, int cls, double work, cudaStream_t s_) : c(c_), s(s_), slot(-1) {
+    if (!c->timing_on || (c->timing_on == 1 && cls != ARMOR_KC_GEMM) || c->timing_n >= c->ev_created) return;
+    slot = c->timing_n++;
+    c->ev_cls[slot] = cls;
+    c->ev_work[slot] = work;
+    cudaEventRecord(c->ev_beg[slot], s);
+  }
+  ~KTimer() { if (slot >= 0) cudaEventRecord(c->ev_end[slot], s); }
+  KTimer(const KTimer&) = delete;
+  KTimer& operator=(const KTimer&) = delete;
+};
 
 #define ARMOR_CUDA_OK(expr)                                  \
   do {                                                       \

@@ -315,7 +315,7 @@ struct HostOp {
   OpCoord c;
 };
 
-armor_status launch(armor_ctx* c, const HostOp& A, const HostOp& B, BParams p, cudaStream_t s) {
+armor_status launch(armor_ctx* c, const HostOp& A, const HostOp& B, BParams p, int kclass, double kbytes, cudaStream_t s) {
   CUtensorMap mA, mB, mC, mD;
   if (!make_map_2d(&mC, p.C, p.c_cols, p.c_rows, p.ldc, 32, 32)) return ARMOR_ERR_CUDA;
   if (p.D) {
@@ -332,6 +332,7 @@ armor_status launch(armor_ctx* c, const HostOp& A, const HostOp& B, BParams p, c
   const int n_sm = c->n_sm;
   const int n_items = p.batch * p.m_tiles * p.n_tiles * p.n_split;
   const int grid = n_items < n_sm ? n_items : n_sm;
+  KTimer kt(c, kclass, kbytes, s);
   tc_block_kernel<<<grid, NTHREADS, SMEM_BYTES, s>>>(mA, mB, mC, mD, p);
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
@@ -363,7 +364,7 @@ armor_status tc_bd_right(armor_ctx* c, const float* in, const float* Bblk, bool 
   p.n_split = 1; p.r_s = 0; p.m_valid = 1 << 30;
   p.batch_fastest = 1;   // neighbouring CTAs read neighbouring column blocks of the same rows
   p.one_pass = c->block_one_pass;
-  return launch(c, A, B, p, s);
+  return launch(c, A, B, p, ARMOR_KC_BLOCK_PRODUCT, (add ? 12.0 : 8.0) * (double)rows * (double)cols, s);
 }
 
 // out[i-th block, :] = alpha * P_i * in[i-th block, :] (+ beta * add[i-th block, :]),  P_i = Ablk[i] or its transpose
@@ -383,7 +384,7 @@ armor_status tc_bd_left(armor_ctx* c, const float* Ablk, bool transA, const floa
   p.alpha = alpha; p.beta = add ? beta : 0.f;
   p.n_split = 1; p.r_s = 0; p.m_valid = 1 << 30;
   p.one_pass = c->block_one_pass;
-  return launch(c, A, B, p, s);
+  return launch(c, A, B, p, ARMOR_KC_BLOCK_PRODUCT, (add ? 12.0 : 8.0) * (double)rows * (double)cols, s);
 }
 
 namespace {
@@ -422,8 +423,10 @@ armor_status gram_launch(armor_ctx* c, const HostOp& A, const HostOp& B, float* 
   p.r_b = db; p.c_b = 0; p.r_s = (int64_t)nb * db;
   p.m_tiles = db / TILE; p.n_tiles = db / TILE; p.batch = nb; p.k_chunks = (int)(chunks / ks); p.n_split = ks;
   p.alpha = 1.f; p.beta = 0.f; p.m_valid = 1 << 30;
-  armor_status st = launch(c, A, B, p, s);
+  // two W-shaped operands are read once each
+  armor_status st = launch(c, A, B, p, ARMOR_KC_BLOCK_GRAM, 8.0 * (double)c->wn, s);
   if (st != ARMOR_OK || ks == 1) return st;
+  KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
   int64_t blocks = (slab / 4 + 255) / 256;
   if (blocks > 148 * 8) blocks = 148 * 8;
   sum_slabs_kernel<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(c->gpart), slab / 4, ks,
@@ -470,5 +473,6 @@ armor_status tc_select_rows_times_H(armor_ctx* c, const float* Z, const float* H
   p.m_tiles = (c->nbo + TILE - 1) / TILE; p.n_tiles = (int)((c->d_in + TILE - 1) / TILE); p.batch = c->nbi;
   p.k_chunks = db / BK; p.n_split = 1; p.m_valid = c->nbo;
   p.alpha = 1.f; p.beta = 0.f;
-  return launch(c, A, B, p, s);
+  // reads H once, plus the thin operands
+  return launch(c, A, B, p, ARMOR_KC_MASK_GUARD, 4.0 * (double)c->d_in * (double)c->d_in, s);
 }

@@ -236,6 +236,7 @@ void launch_pack_blocks(armor_ctx* c, const float* P, const float* rowscale, con
   const int64_t n = (int64_t)nb * c->db * c->db;
   int64_t blocks = (n + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
+  KTimer kt(c, ARMOR_KC_FORWARD, 0.0, s);
   pack_blocks_kernel<<<(unsigned)blocks, 256, 0, s>>>(P, rowscale, colscale, static_cast<__nv_bfloat16*>(Q), n, c->db);
   c->launches++;
 }
@@ -258,6 +259,7 @@ armor_status launch_fwd_block(armor_ctx* c, const void* X, const void* Q, void* 
   const int n_sm = c->n_sm;
   const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
   const int grid = tiles < n_sm ? (int)tiles : n_sm;
+  KTimer kt(c, ARMOR_KC_FORWARD, 4.0 * (double)rows * (double)d, s);
   fwd_block_kernel<<<grid, NTHREADS, SMEM, s>>>(mX, mQ, p);
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;

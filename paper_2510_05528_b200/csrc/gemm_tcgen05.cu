@@ -471,18 +471,14 @@ armor_status launch_impl(armor_ctx* c, const TcGemm& g, Params p, cudaStream_t s
     }
   }
   const int grid = p.n_items < n_sm ? p.n_items : n_sm;
-  const bool timed = c->timing_on && c->timing_n < ARMOR_MAX_TIMED;
-  if (timed) cudaEventRecord(c->ev_beg[c->timing_n], s);
-  tc_gemm_kernel<PASSES><<<grid, NTHREADS, SMEM, s>>>(mA, mAlo, mB, mBlo, p);
-  if (p.split_parts > 1) {
-    tc_gemm_fixup_kernel<<<4 * (p.n_tiles_total - p.split_first), 256, 0, s>>>(p);
-    c->launches++;
-  }
-  if (timed) {
-    cudaEventRecord(c->ev_end[c->timing_n], s);
-    c->timing_n++;
-    c->timing_flops += p.symmetric_lower ? (double)p.M * (double)(p.N + BM) * (double)p.K
-                                         : 2.0 * (double)p.M * (double)p.N * (double)p.K;
+  {
+    KTimer kt(c, ARMOR_KC_GEMM, p.symmetric_lower ? (double)p.M * (double)(p.N + BM) * (double)p.K
+                                                  : 2.0 * (double)p.M * (double)p.N * (double)p.K, s);
+    tc_gemm_kernel<PASSES><<<grid, NTHREADS, SMEM, s>>>(mA, mAlo, mB, mBlo, p);
+    if (p.split_parts > 1) {
+      tc_gemm_fixup_kernel<<<4 * (p.n_tiles_total - p.split_first), 256, 0, s>>>(p);
+      c->launches++;
+    }
   }
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;

@@ -273,6 +273,7 @@ bool tile_kernel_ok(const BGemm& g, bool& a_kfast, bool& b_nfast) {
 }  // namespace
 
 void launch_bgemm(armor_ctx* c, const BGemm& g_in, cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);   // CUDA-core products: small block systems, or every product of a SIMT run
   BGemm g = g_in;
   if (g.M <= 0 || g.N <= 0 || g.batch <= 0) return;
   if (g.ksplit > 1 && (g.D || !c->gpart || (int64_t)g.ksplit * g.batch * g.M * g.N > c->gpart_floats)) g.ksplit = 1;

@@ -521,6 +521,7 @@ int chol_parts_per_block(int db, int nb) {
 armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float* rhs, float* out, const float* dotw,
                          float* A, int nb, double* part, cudaStream_t s) {
   const int db = c->db;
+  KTimer kt(c, ARMOR_KC_CHOLESKY, (double)nb * (7.0 / 3.0) * (double)db * (double)db * (double)db, s);   // flops
   if (db % NB == 0) {
     const int slices = chol_parts_per_block(db, nb);
     const int w = db / slices;

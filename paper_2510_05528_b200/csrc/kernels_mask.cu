@@ -116,13 +116,19 @@ __device__ __forceinline__ bool chol_small(int n, const double (&Kin)[NKM][NKM],
 // Pass 2: thread b < 2^MG evaluates the mask with bit pattern b (if it keeps exactly n_keep positions);
 // the best one is found in this order: larger reduction first; among equal reductions the
 // incumbent, then the lexicographically first index tuple.
-template <int MG, int NKM, bool MULTI>
+// PHASE 0: both passes in one launch (several draws per block).  A single draw runs as two launches, so that the
+// streaming pass keeps few registers and the per-block solves, which are chains of dependent loads, all run
+// side by side: PHASE 1 is pass 1 alone (the block's winner goes to best_key / best_g), PHASE 2 is pass 2
+// alone (one warp per block for groups of four, 256 threads for groups of eight).
+template <int MG, int NKM, bool MULTI, int PHASE>
 __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict__ Gam, const float* __restrict__ S,
                                                          const uint8_t* __restrict__ M, const float* __restrict__ alpha,
                                                          const float* __restrict__ Kfull, SelRec* __restrict__ sel,
                                                          double* __restrict__ part, int64_t d_in, int db, int nbi,
                                                          int n_keep, int select_mode, uint64_t seed, uint64_t t,
-                                                         uint64_t n_groups_total, int kg_arg) {
+                                                         uint64_t n_groups_total, int kg_arg,
+                                                         float* __restrict__ tab_key,
+                                                         unsigned long long* __restrict__ tab_g) {
   const int kg = MULTI ? kg_arg : 1;                       // one draw: the loop and the key cache compile away
   const int bi = blockIdx.x / nbi, bj = blockIdx.x % nbi;
   extern __shared__ float s_keys[];         // kg > 1: the keys of the block's groups, kept for the later draws
@@ -135,6 +141,10 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
   const int blk = bi * (kg * nbi) + kk * nbi + bj;
   float best_key = INFINITY;
   uint64_t best_g = ~0ull;
+  if (PHASE == 2) {
+    best_key = tab_key[blk];
+    best_g = tab_g[blk];
+  } else {
   if (MULTI && kk > 0) {
     // later draws: keys from the first pass, drawn ones at +inf
     for (int idx = threadIdx.x; idx < n_in_block; idx += NT) {
@@ -144,70 +154,90 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
       if (key < best_key || (key == best_key && g < best_g)) { best_key = key; best_g = g; }
     }
   } else {
-    // Four groups per thread and step: the loads are issued together, then scores and hashes.  With a single
-    // draw most logarithms are skipped: -ln(u) >= 1 - u, so a group whose (1 - u) / score already reaches the
-    // thread's best key cannot win (the bound is tight exactly where winners live, u next to 1).  A thread
-    // meets its groups in ascending order, so a tie never replaces an earlier group either.
+    // A thread keeps one group column of the block and walks down its rows, NT / gpb rows apart (threads beyond
+    // the last whole row of groups idle), so the group index, the hash counter and the addresses advance by
+    // additions.  Four groups per thread and step: the loads are issued together, then scores and hashes.
+    // With a single draw most logarithms are skipped: -ln(u) >= 1 - u, so a group whose (1 - u) / score
+    // exceeds the best key its warp has seen cannot win (the bound is tight exactly where winners live, u next
+    // to 1; the warp-wide bound, refreshed after every step, makes whole warps skip the logarithm, which a
+    // per-thread bound would not: among 32 lanes one almost always passes its own).
     constexpr int U = 4;
-    for (int base = threadIdx.x; base < n_in_block; base += U * NT) {
-      float4 g4[U][MG / 4];
-      float al[U];
+    const int rstep = NT / gpb;                                  // rows of the block covered per step (gpb <= 64)
+    const int cl = (int)threadIdx.x % gpb, rl0 = (int)threadIdx.x / gpb;
+    {
+      const bool lane_on = rl0 < rstep;
+      float wbound = INFINITY;                                   // warp-uniform: the smallest key any lane holds
+      const int n_steps = (db + U * rstep - 1) / (U * rstep);    // the same for every lane: the shuffles below need all 32
+      const int64_t row0 = (int64_t)bi * db + (lane_on ? rl0 : 0);
+      const int64_t cg = (int64_t)bj * gpb + cl;
+      const float* gp = Gam + row0 * d_in + cg * MG;
+      const float* ap = alpha + row0;
+      uint64_t g = (uint64_t)row0 * (uint64_t)ng_row + (uint64_t)cg;
+      uint64_t ctr = t * n_groups_total + g;
+      const uint64_t gstep = (uint64_t)rstep * (uint64_t)ng_row;
+      const int64_t pstep = (int64_t)rstep * d_in;
+      for (int step = 0, rl = rl0; step < n_steps; ++step, rl += U * rstep) {
+        float4 g4[U][MG / 4];
+        float al[U];
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int idx = base + u * NT;
-        al[u] = 0.f;
+        for (int u = 0; u < U; ++u) {
+          al[u] = 0.f;
 #pragma unroll
-        for (int h = 0; h < MG / 4; ++h) g4[u][h] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (idx < n_in_block) {
-          const int rl = idx / gpb, cl = idx % gpb;
-          const int64_t row = (int64_t)bi * db + rl;
-          const int64_t cg = (int64_t)bj * gpb + cl;
-          al[u] = alpha[row];
+          for (int h = 0; h < MG / 4; ++h) g4[u][h] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (lane_on && rl + u * rstep < db) {
+            al[u] = ap[u * rstep];
 #pragma unroll
-          for (int h = 0; h < MG / 4; ++h)
-            g4[u][h] = *reinterpret_cast<const float4*>(Gam + row * d_in + cg * MG + 4 * h);
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int idx = base + u * NT;
-        if (idx >= n_in_block) continue;
-        const int rl = idx / gpb, cl = idx % gpb;
-        const int64_t row = (int64_t)bi * db + rl;
-        const int64_t cg = (int64_t)bj * gpb + cl;
-        float score = 0.f, sq = 0.f;
-#pragma unroll
-        for (int h = 0; h < MG / 4; ++h) {
-          score += fabsf(g4[u][h].x);
-          score += fabsf(g4[u][h].y);
-          score += fabsf(g4[u][h].z);
-          score += fabsf(g4[u][h].w);
-          sq = fmaf(g4[u][h].x, g4[u][h].x, sq);
-          sq = fmaf(g4[u][h].y, g4[u][h].y, sq);
-          sq = fmaf(g4[u][h].z, g4[u][h].z, sq);
-          sq = fmaf(g4[u][h].w, g4[u][h].w, sq);
-        }
-        // the ablation's weights (Appendix E.1): L2 norm of the group's gradient, or equal weights
-        if (select_mode == ARMOR_SELECT_L2_RANDOM) score = sqrtf(sq);
-        else if (select_mode == ARMOR_SELECT_UNIFORM_RANDOM) score = 1.f;
-        if (!(al[u] > 0.f)) score = 0.f;
-        const uint64_t g = (uint64_t)row * (uint64_t)ng_row + (uint64_t)cg;
-        float key = INFINITY;
-        if (score > 0.f) {
-          if (select_mode != ARMOR_SELECT_L1_GREEDY) {
-            const uint64_t bits = splitmix64(seed ^ splitmix64(t * n_groups_total + g));
-            const uint32_t k24 = (uint32_t)(bits >> 40);
-            // 1 - u = (2^24 - k24 - 1/2) 2^-24, exact in fp32; the factor 1 - 1e-5 covers the few ulp by which the
-            // computed key can fall below (1 - u) / score
-            const float one_minus_u = (float)(2u * ((1u << 24) - k24) - 1u) * 2.98023223876953125e-8f;
-            if (MULTI || !(one_minus_u * 0.99999f >= best_key * score))
-              key = neg_log_uniform(k24) / score;
-          } else {
-            key = -score;
+            for (int h = 0; h < MG / 4; ++h) g4[u][h] = *reinterpret_cast<const float4*>(gp + u * pstep + 4 * h);
           }
         }
-        if (MULTI) s_keys[idx] = key;
-        if (key < best_key || (key == best_key && g < best_g)) { best_key = key; best_g = g; }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          if (lane_on && rl + u * rstep < db) {
+            float score = 0.f, sq = 0.f;
+#pragma unroll
+            for (int h = 0; h < MG / 4; ++h) {
+              score += fabsf(g4[u][h].x);
+              score += fabsf(g4[u][h].y);
+              score += fabsf(g4[u][h].z);
+              score += fabsf(g4[u][h].w);
+              if (select_mode == ARMOR_SELECT_L2_RANDOM) {
+                sq = fmaf(g4[u][h].x, g4[u][h].x, sq);
+                sq = fmaf(g4[u][h].y, g4[u][h].y, sq);
+                sq = fmaf(g4[u][h].z, g4[u][h].z, sq);
+                sq = fmaf(g4[u][h].w, g4[u][h].w, sq);
+              }
+            }
+            // the ablation's weights (Appendix E.1): L2 norm of the group's gradient, or equal weights
+            if (select_mode == ARMOR_SELECT_L2_RANDOM) score = sqrtf(sq);
+            else if (select_mode == ARMOR_SELECT_UNIFORM_RANDOM) score = 1.f;
+            if (!(al[u] > 0.f)) score = 0.f;
+            const uint64_t gu = g + (uint64_t)u * gstep;
+            float key = INFINITY;
+            if (score > 0.f) {
+              if (select_mode != ARMOR_SELECT_L1_GREEDY) {
+                const uint64_t bits = splitmix64(seed ^ splitmix64(ctr + (uint64_t)u * gstep));
+                const uint32_t k24 = (uint32_t)(bits >> 40);
+                // 1 - u = (2^24 - k24 - 1/2) 2^-24, exact in fp32; the factor 1 - 1e-5 covers the few ulp by
+                // which the computed key can fall below (1 - u) / score
+                const float one_minus_u = (float)(2u * ((1u << 24) - k24) - 1u) * 2.98023223876953125e-8f;
+                if (MULTI || !(one_minus_u * 0.99999f >= wbound * score))
+                  key = neg_log_uniform(k24) / score;
+              } else {
+                key = -score;
+              }
+              if (key < best_key || (key == best_key && gu < best_g)) { best_key = key; best_g = gu; }
+            }
+            if (MULTI) s_keys[(rl + u * rstep) * gpb + cl] = key;
+          }
+        }
+        gp += U * pstep;
+        ap += U * rstep;
+        g += U * gstep;
+        ctr += U * gstep;
+        if (!MULTI) {
+          wbound = best_key;
+          for (int o = 16; o > 0; o >>= 1) wbound = fminf(wbound, __shfl_xor_sync(0xffffffffu, wbound, o));
+        }
       }
     }
   }
@@ -232,6 +262,11 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
   __syncthreads();
   best_key = s_key;
   best_g = s_g;
+  if (PHASE == 1) {
+    if (threadIdx.x == 0) { tab_key[blk] = best_key; tab_g[blk] = best_g; }
+    return;
+  }
+  }
   if (!(best_key < INFINITY)) {                               // nothing left to draw in this block (uniform)
     if (threadIdx.x == 0) {
       SelRec rec;
@@ -322,7 +357,7 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
   if ((threadIdx.x & 31) == 0) { sred[threadIdx.x >> 5] = b_red; stie[threadIdx.x >> 5] = b_tie; scand[threadIdx.x >> 5] = b_cand; }
   __syncthreads();
   if (threadIdx.x == 0) {
-    for (int w = 1; w < NT / 32; ++w) {
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) {
       const bool take = (scand[w] != 0xffffffffu) &&
                         (b_cand == 0xffffffffu || sred[w] > b_red || (sred[w] == b_red && stie[w] > b_tie));
       if (take) { b_red = sred[w]; b_tie = stie[w]; b_cand = scand[w]; }
@@ -478,12 +513,14 @@ __global__ void __launch_bounds__(NT) mask_carry_kernel(const SelRec* __restrict
 }  // namespace
 
 void launch_mask_carry_P(armor_ctx* c, float* P, cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_MASK_GUARD, 0.0, s);
   mask_carry_kernel<<<dim3(c->nbo, (unsigned)((c->d_in + 1023) / 1024)), NT, 0, s>>>(c->sel, c->Ysel, P, c->sc, c->d_in,
                                                                                    c->nbo_pad, c->nbi * c->kg);
   c->launches++;
 }
 
 void launch_alpha(armor_ctx* c, const float* A, cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_MASK_GUARD, 0.0, s);
   alpha_kernel<<<dim3(c->nbo, (c->db + 31) / 32), dim3(32, 8), 0, s>>>(A, c->alpha, c->db);
   c->launches++;
 }
@@ -492,16 +529,24 @@ void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const ui
   const int mg = c->cfg.m_group;
   const uint64_t n_groups = (uint64_t)(c->d_out * (c->d_in / mg));
 #define ARMOR_SELECT_ARGS Gam, S, M, c->alpha, c->Kfull, c->sel, c->partblk, c->d_in, c->db, c->nbi, c->cfg.n_keep, \
-                          c->cfg.select_mode, c->cfg.seed, (uint64_t)t, n_groups, c->kg
+                          c->cfg.select_mode, c->cfg.seed, (uint64_t)t, n_groups, c->kg, c->tab_key, c->tab_g
   // kg > 1: the block's keys stay in shared memory between the draws (up to 64 KiB: d_block 256, groups of four)
   const size_t smem = c->kg > 1 ? (size_t)c->db * (c->db / mg) * sizeof(float) : 0;
 #define ARMOR_SELECT_LAUNCH(MGV, NKV, MULTIV)                                                                           \
   do {                                                                                                                  \
-    if (smem > 48 * 1024)                                                                                               \
-      cudaFuncSetAttribute(mask_select_kernel<MGV, NKV, MULTIV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
-    mask_select_kernel<MGV, NKV, MULTIV><<<c->nbo * c->nbi, NT, smem, s>>>(ARMOR_SELECT_ARGS);                          \
+    if (MULTIV) {                                                                                                       \
+      if (smem > 48 * 1024)                                                                                             \
+        cudaFuncSetAttribute(mask_select_kernel<MGV, NKV, MULTIV, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
+                             (int)smem);                                                                                \
+      mask_select_kernel<MGV, NKV, MULTIV, 0><<<c->nbo * c->nbi, NT, smem, s>>>(ARMOR_SELECT_ARGS);                     \
+    } else {                                                                                                            \
+      mask_select_kernel<MGV, NKV, false, 1><<<c->nbo * c->nbi, NT, 0, s>>>(ARMOR_SELECT_ARGS);                         \
+      mask_select_kernel<MGV, NKV, false, 2><<<c->nbo * c->nbi, MGV == 4 ? 32 : NT, 0, s>>>(ARMOR_SELECT_ARGS);         \
+      c->launches++;                                                                                                    \
+    }                                                                                                                   \
   } while (0)
   const bool multi = c->kg > 1;
+  KTimer kt(c, ARMOR_KC_MASK_SELECT, 4.0 * (double)c->wn, s);   // one read of the core gradient
   if (mg == 8 && c->cfg.n_keep > 4) { if (multi) ARMOR_SELECT_LAUNCH(8, 6, true); else ARMOR_SELECT_LAUNCH(8, 6, false); }
   else if (mg == 8) { if (multi) ARMOR_SELECT_LAUNCH(8, 4, true); else ARMOR_SELECT_LAUNCH(8, 4, false); }
   else { if (multi) ARMOR_SELECT_LAUNCH(4, 4, true); else ARMOR_SELECT_LAUNCH(4, 4, false); }
@@ -512,7 +557,10 @@ void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const ui
 
 void launch_mask_quadratic(armor_ctx* c, const float* A, const float* B, const float* H, cudaStream_t s) {
   const int db = c->db, nbo = c->nbo, nbi = c->nbi, nbo_pad = c->nbo_pad, kg = c->kg, nbv = nbi * kg;
-  mask_vectors_kernel<<<nbo * nbv, NT, 0, s>>>(A, B, c->sel, c->Zsel, c->Acol, db, nbo_pad, nbi, c->cfg.m_group, nbv);
+  {
+    KTimer kt(c, ARMOR_KC_MASK_GUARD, 0.0, s);
+    mask_vectors_kernel<<<nbo * nbv, NT, 0, s>>>(A, B, c->sel, c->Zsel, c->Acol, db, nbo_pad, nbi, c->cfg.m_group, nbv);
+  }
   c->launches++;
   const float* Y = nullptr;
   if (c->cfg.h_mode == ARMOR_H_FULL) {
@@ -532,12 +580,16 @@ void launch_mask_quadratic(armor_ctx* c, const float* A, const float* B, const f
     Y = c->Ysel;
   }
   double* part = c->quadpart;
-  mask_quad_kernel<<<nbo * nbv, NT, 0, s>>>(c->Zsel, c->Acol, Y, c->hdiag, part, c->d_in, db, nbo_pad, nbi, nbv);
+  {
+    KTimer kt(c, ARMOR_KC_MASK_GUARD, 0.0, s);
+    mask_quad_kernel<<<nbo * nbv, NT, 0, s>>>(c->Zsel, c->Acol, Y, c->hdiag, part, c->d_in, db, nbo_pad, nbi, nbv);
+  }
   c->launches++;
   reduce_partials_to(c, part, nbo * nbv, c->sc + SC_Q_M, s);
 }
 
 void launch_mask_commit(armor_ctx* c, float* S, uint8_t* M, armor_iter_stats* st, cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_MASK_GUARD, 0.0, s);
   mask_commit_kernel<<<1, 256, 0, s>>>(c->sel, c->nbo * c->nbi * c->kg, S, M, c->d_in, c->cfg.m_group, c->sc, st);
   c->launches++;
 }

@@ -486,12 +486,14 @@ inline int grid_for(int64_t n) {
 }  // namespace
 
 void dot_to_ptr(armor_ctx* c, const float* x, const float* y, int64_t n, double* out, cudaStream_t s) {
+  KTimer kt(c, n >= (1 << 22) ? ARMOR_KC_DOT : ARMOR_KC_SMALL, 8.0 * (double)n, s);
   dot_partial_kernel<<<ARMOR_DOT_BLOCKS, NT, 0, s>>>((const float4*)x, (const float4*)y, n / 4, c->partials);
   reduce_final_kernel<<<1, NT, 0, s>>>(c->partials, ARMOR_DOT_BLOCKS, out);
   c->launches += 2;
 }
 
 void reduce_partials_to(armor_ctx* c, const double* part, int n, double* out, cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
   reduce_final_kernel<<<1, NT, 0, s>>>(part, n, out);
   c->launches++;
 }
@@ -503,6 +505,7 @@ void launch_zero_flags(armor_ctx* c, cudaStream_t s) {
 
 void launch_colscale(armor_ctx* c, const float* in, const float* h, float* out, int64_t rows, int64_t cols,
                      cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_AXPY, 8.0 * (double)rows * (double)cols, s);
   colscale_kernel<<<grid_for(rows * cols / 4), NT, 0, s>>>((const float4*)in, (const float4*)h, (float4*)out,
                                                           rows * cols / 4, (int)(cols / 4));
   c->launches++;
@@ -510,16 +513,19 @@ void launch_colscale(armor_ctx* c, const float* in, const float* h, float* out, 
 
 void launch_scale_rows_cols(armor_ctx* c, const float* in, const float* colscale, const float* rowscale, float* out,
                             int64_t rows, int64_t cols, cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_FORWARD, 8.0 * (double)rows * (double)cols, s);
   rowcolscale_kernel<<<grid_for(rows * cols), NT, 0, s>>>(in, colscale, rowscale, out, rows, cols);
   c->launches++;
 }
 
 void launch_extract_hblocks(armor_ctx* c, const float* H, cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
   extract_hblocks_kernel<<<c->nbi, NT, 0, s>>>(H, c->hdiag, c->Hjj, c->d_in, c->db, c->cfg.h_mode == ARMOR_H_DIAG);
   c->launches++;
 }
 
 void launch_masked_copy(armor_ctx* c, const float* Gam, const uint8_t* M, float* out, int slot_norm, cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_MASKED_COPY, (8.0 + 1.0 / c->cfg.m_group) * (double)c->wn, s);
   masked_copy_kernel<<<ARMOR_DOT_BLOCKS, NT, 0, s>>>((const float4*)Gam, M, (float4*)out, c->wn / 4,
                                                     c->cfg.m_group / 4, c->partials);
   reduce_final_kernel<<<1, NT, 0, s>>>(c->partials, ARMOR_DOT_BLOCKS, c->sc + slot_norm);
@@ -527,6 +533,7 @@ void launch_masked_copy(armor_ctx* c, const float* Gam, const uint8_t* M, float*
 }
 
 void launch_axpy_slot(armor_ctx* c, float* y, const float* x, int64_t n, int slot, float sign, cudaStream_t s) {
+  KTimer kt(c, n >= (1 << 22) ? ARMOR_KC_AXPY : ARMOR_KC_SMALL, 12.0 * (double)n, s);
   axpy_slot_kernel<<<grid_for(n / 4), NT, 0, s>>>((float4*)y, (const float4*)x, n / 4, c->sc, slot, sign);
   c->launches++;
 }
@@ -534,6 +541,9 @@ void launch_axpy_slot(armor_ctx* c, float* y, const float* x, int64_t n, int slo
 void launch_init(armor_ctx* c, const float* W, const float* H, float* Wbar, float* r1, float* r2, float* A, float* B,
                  float* S, uint8_t* M, cudaStream_t s) {
   const int64_t rows = c->d_out, cols = c->d_in;
+  // W read (twice more with the normalisation), Wbar, S and the mask bytes written
+  KTimer kt(c, ARMOR_KC_INIT, (double)c->wn * (c->cfg.normalize ? 20.0 : 12.0 + (Wbar != W ? 4.0 : 0.0)) +
+                                  (double)c->wn / c->cfg.m_group, s);
   if (c->cfg.normalize) {
     double* part = c->colpart;
     dim3 g1((unsigned)((cols + NT - 1) / NT), COLSUM_CHUNKS);
@@ -560,6 +570,7 @@ void launch_init(armor_ctx* c, const float* W, const float* H, float* Wbar, floa
 armor_status launch_screen_inputs(armor_ctx* c, const float* W, const float* H, cudaStream_t s) {
   if (cudaMemsetAsync(c->screen, 0, 4 * sizeof(int32_t), s) != cudaSuccess) return ARMOR_ERR_CUDA;
   const int64_t wn4 = c->wn / 4, hn4 = c->d_in * c->d_in / 4;
+  KTimer kt(c, ARMOR_KC_INIT, 4.0 * ((double)c->wn + (double)c->d_in * (double)c->d_in), s);
   screen_count_kernel<<<grid_for(wn4 > hn4 ? wn4 : hn4), NT, 0, s>>>(reinterpret_cast<const float4*>(W), wn4,
                                                                      reinterpret_cast<const float4*>(H), hn4, H, c->d_in,
                                                                      c->screen);
@@ -570,17 +581,20 @@ armor_status launch_screen_inputs(armor_ctx* c, const float* W, const float* H, 
 
 void launch_zero_scalars(armor_ctx* c, bool carry_loss, cudaStream_t s) {
   const int nflag = c->nbo > c->nbi ? c->nbo : c->nbi;
+  KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
   zero_scalars_kernel<<<1, NT, 0, s>>>(c->sc, c->failflag, nflag, carry_loss ? 1 : 0);
   c->launches++;
 }
 
 void launch_stage(armor_ctx* c, armor_iter_stats* st, int stage, const double* part, int npart, int nflag,
                   cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
   stage_kernel<<<1, 32, 0, s>>>(c->sc, st, stage, c->failflag, nflag, part, npart, c->status);
   c->launches++;
 }
 
 void launch_split_hilo(armor_ctx* c, const float* in, float* hi, float* lo, int64_t n, cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_OPERAND_SPLIT, 8.0 * (double)n, s);
   split_hilo_kernel<<<grid_for(n / 4), NT, 0, s>>>((const float4*)in, (float4*)hi, (float4*)lo, n / 4);
   c->launches++;
 }
@@ -588,6 +602,7 @@ void launch_split_hilo(armor_ctx* c, const float* in, float* hi, float* lo, int6
 void launch_transpose_split(armor_ctx* c, const void* X, int x_dtype, int64_t ldx, int64_t rows, int64_t cols,
                             float* Thi, float* Tlo, int64_t ldt, cudaStream_t s) {
   dim3 grid((unsigned)((cols + 31) / 32), (unsigned)((ldt + 31) / 32));
+  KTimer kt(c, ARMOR_KC_GRAM_STAGING, (double)rows * (double)cols * (x_dtype == ARMOR_DTYPE_BF16 ? 6.0 : (Tlo ? 12.0 : 8.0)), s);
   if (x_dtype == ARMOR_DTYPE_BF16)
     transpose_split_kernel<<<grid, dim3(32, 8), 0, s>>>(static_cast<const __nv_bfloat16*>(X), ldx, rows, cols, Thi,
                                                        (float*)nullptr, ldt);
@@ -598,11 +613,13 @@ void launch_transpose_split(armor_ctx* c, const void* X, int x_dtype, int64_t ld
 
 void launch_mirror_lower(armor_ctx* c, float* H, int64_t n, cudaStream_t s) {
   const unsigned t = (unsigned)((n + 31) / 32);
+  KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
   mirror_lower_kernel<<<dim3(t, t), dim3(32, 8), 0, s>>>(H, n);
   c->launches++;
 }
 
 void launch_block_fro_sum(armor_ctx* c, const float* X, int nblk, const float* hdiag, double* out, cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
   block_fro_kernel<<<nblk, NT, 0, s>>>((const float4*)X, c->db * c->db / 4, hdiag, c->db, c->nbi, c->quadpart);
   reduce_final_kernel<<<1, NT, 0, s>>>(c->quadpart, nblk, out);
   c->launches += 2;
@@ -615,6 +632,7 @@ void launch_adam(armor_ctx* c, float* theta, const float* gamma, float* m, float
   const float b2 = c->cfg.adam_beta2 > 0.f ? c->cfg.adam_beta2 : 0.999f;
   const float eps = c->cfg.adam_eps > 0.f ? c->cfg.adam_eps : 1e-8f;
   const double bc1 = 1.0 - pow((double)b1, (double)step), bc2 = 1.0 - pow((double)b2, (double)step);
+  KTimer kt(c, n >= (1 << 22) ? ARMOR_KC_AXPY : ARMOR_KC_SMALL, 28.0 * (double)n, s);
   adam_kernel<<<grid_for(n / 4), NT, 0, s>>>((float4*)theta, (const float4*)gamma, (float4*)m, (float4*)v, n / 4, M,
                                             c->cfg.m_group / 4, lr, b1, b2, eps, (float)(1.0 / bc1), (float)(1.0 / bc2),
                                             c->status);
@@ -623,6 +641,7 @@ void launch_adam(armor_ctx* c, float* theta, const float* gamma, float* m, float
 
 void launch_bf16_to_f32(armor_ctx* c, const void* in, const float* colscale, float* out, int64_t rows, int64_t cols,
                         cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_FORWARD, 6.0 * (double)rows * (double)cols, s);
   bf16_to_f32_kernel<<<grid_for(rows * cols), NT, 0, s>>>(static_cast<const __nv_bfloat16*>(in), colscale, out,
                                                          rows * cols, cols);
   c->launches++;
@@ -630,6 +649,7 @@ void launch_bf16_to_f32(armor_ctx* c, const void* in, const float* colscale, flo
 
 void launch_f32_to_bf16(armor_ctx* c, const float* in, const float* colscale, void* out, int64_t rows, int64_t cols,
                         cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_FORWARD, 6.0 * (double)rows * (double)cols, s);
   f32_to_bf16_kernel<<<grid_for(rows * cols), NT, 0, s>>>(in, colscale, static_cast<__nv_bfloat16*>(out), rows * cols,
                                                          cols);
   c->launches++;

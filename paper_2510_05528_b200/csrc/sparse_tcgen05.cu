@@ -550,6 +550,7 @@ size_t tc_sparse_values_bytes(const armor_ctx* c) { return (size_t)c->d_out * (s
 
 void launch_compress_24(armor_ctx* c, const float* S, const uint8_t* M, void* Sc, void* E, cudaStream_t s) {
   const int64_t n_words = c->d_out * (c->d_in / 32);
+  KTimer kt(c, ARMOR_KC_FORWARD, (double)c->wn * 5.125, s);
   compress_24_kernel<<<(unsigned)((n_words + 255) / 256), 256, 0, s>>>(S, M, static_cast<__nv_bfloat16*>(Sc),
                                                                         static_cast<uint32_t*>(E), c->d_out, c->d_in,
                                                                         c->status);
@@ -573,8 +574,7 @@ armor_status launch_tc_sparse(armor_ctx* c, const void* Sc, const void* E, const
   static PerDeviceOnce attr;
   if (ensure_dynamic_smem(attr, c->device, tc_sparse_kernel, SMEM) != ARMOR_OK) return ARMOR_ERR_CUDA;
   const int n_sm = c->n_sm;
-  const bool timed = c->timing_on && c->timing_n < ARMOR_MAX_TIMED;
-  if (timed) cudaEventRecord(c->ev_beg[c->timing_n], s);
+  KTimer kt(c, ARMOR_KC_GEMM, 2.0 * (double)p.M * (double)p.N * (double)p.K, s);   // dense-equivalent flops
   if (g_sparse_pairs && c->d_out % 256 == 0 && n_sm >= 2) {
       static PerDeviceOnce attr2;
     if (ensure_dynamic_smem(attr2, c->device, tc_sparse_pair_kernel, SMEM) != ARMOR_OK) return ARMOR_ERR_CUDA;
@@ -593,11 +593,6 @@ armor_status launch_tc_sparse(armor_ctx* c, const void* Sc, const void* E, const
     const int tiles = p.m_tiles * p.n_tiles;
     const int grid = tiles < n_sm ? tiles : n_sm;
     tc_sparse_kernel<<<grid, NTHREADS, SMEM, s>>>(mA, mB, mE, p);
-  }
-  if (timed) {
-    cudaEventRecord(c->ev_end[c->timing_n], s);
-    c->timing_n++;
-    c->timing_flops += 2.0 * (double)p.M * (double)p.N * (double)p.K;   // dense-equivalent
   }
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;

@@ -180,6 +180,7 @@ inline unsigned grid_for(int64_t n) {
 
 void launch_f16_prepare_H(armor_ctx* c, const float* H, cudaStream_t s) {
   const int64_t n = c->d_in;
+  KTimer kt(c, ARMOR_KC_OPERAND_SPLIT, 8.0 * (double)n * (double)n, s);
   hpow_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(c->hdiag, c->hpow, n);
   __half* hi = reinterpret_cast<__half*>(c->Hlo);
   split_H_kernel<<<grid_for(n * n / 4), NT, 0, s>>>(reinterpret_cast<const float4*>(H), c->hpow,
@@ -189,6 +190,7 @@ void launch_f16_prepare_H(armor_ctx* c, const float* H, cudaStream_t s) {
 
 void launch_f16_split_rows(armor_ctx* c, const float* in, int64_t ld, int64_t rows, int64_t cols, const float* colscale,
                            float post, void* hi, void* lo, float* out_scale, cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_OPERAND_SPLIT, 8.0 * (double)rows * (double)cols, s);
   split_rows_kernel<<<(unsigned)rows, NT, 0, s>>>(in, ld, cols, colscale, post, static_cast<__half2*>(hi),
                                                   static_cast<__half2*>(lo), out_scale);
   c->launches++;
@@ -199,6 +201,8 @@ float f16_H_post_scale() { return 1.f / (float)(1 << H_SHIFT); }
 armor_status launch_f16_gram_stage(armor_ctx* c, const void* X, int x_dtype, int64_t ldx, int64_t rows, int64_t cols,
                                    void* Thi, void* Tlo, int64_t ldt, cudaStream_t s) {
   if (cudaMemsetAsync(c->gmax, 0, (size_t)cols * sizeof(unsigned), s) != cudaSuccess) return ARMOR_ERR_CUDA;
+  // one read for the maxima, one read and one 16-bit write per part for the staged chunk
+  KTimer kt(c, ARMOR_KC_GRAM_STAGING, (double)rows * (double)cols * (x_dtype == ARMOR_DTYPE_BF16 ? 6.0 : 12.0), s);
   const dim3 g1((unsigned)((cols + NT - 1) / NT), (unsigned)((rows + 255) / 256));
   const dim3 g2((unsigned)((cols + 31) / 32), (unsigned)((ldt + 31) / 32));
   if (x_dtype == ARMOR_DTYPE_BF16) {
