@@ -27,13 +27,24 @@ __global__ void __launch_bounds__(NT) dot_partial_kernel(const float4* __restric
                                                          const float4* __restrict__ y, int64_t n4,
                                                          double* __restrict__ part) {
   double acc = 0.0;
-  for (int64_t i = (int64_t)blockIdx.x * NT + threadIdx.x; i < n4; i += (int64_t)gridDim.x * NT) {
-    float4 a = x[i], b = y[i];
-    float s = a.x * b.x;
-    s = fmaf(a.y, b.y, s);
-    s = fmaf(a.z, b.z, s);
-    s = fmaf(a.w, b.w, s);
-    acc += (double)s;
+  const int64_t stride = (int64_t)gridDim.x * NT;
+  // four independent pairs of loads in flight per thread; the order of the additions is fixed by the grid
+  for (int64_t i0 = (int64_t)blockIdx.x * NT + threadIdx.x; i0 < n4; i0 += 4 * stride) {
+    float4 a[4], b[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int64_t i = i0 + u * stride;
+      a[u] = b[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (i < n4) { a[u] = x[i]; b[u] = y[i]; }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      float s = a[u].x * b[u].x;
+      s = fmaf(a[u].y, b[u].y, s);
+      s = fmaf(a[u].z, b[u].z, s);
+      s = fmaf(a[u].w, b[u].w, s);
+      acc += (double)s;
+    }
   }
   acc = block_reduce_sum(acc);
   if (threadIdx.x == 0) part[blockIdx.x] = acc;

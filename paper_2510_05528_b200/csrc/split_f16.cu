@@ -147,27 +147,40 @@ __global__ void gram_scale_kernel(const unsigned* __restrict__ umax, float* __re
 }
 
 // X [rows, cols] (ld ldx) -> Thi/Tlo [cols, ldt] fp16: transposed, column c scaled by 2^e_c, split.  bf16 input
-// has 8 significant bits: it is exact in one fp16 part, Tlo is then not written.
+// has 8 significant bits: it is exact in one fp16 part, Tlo is then not written.  Tiles of 64 tokens x 64
+// channels: rows of 64 channels are read 128 bytes per warp instruction, and every channel's 64 tokens are written
+// as 32 pairs (128 bytes per warp instruction).  ldt is a multiple of 64; tokens beyond `rows` are written as zeros.
 template <typename TIn>
-__global__ void transpose_split_f16_kernel(const TIn* __restrict__ X, int64_t ldx, int64_t rows, int64_t cols,
-                                           const unsigned* __restrict__ umax, __half* __restrict__ Thi,
-                                           __half* __restrict__ Tlo, int64_t ldt) {
-  __shared__ float tile[32][33];
-  const int64_t c0 = (int64_t)blockIdx.x * 32, r0 = (int64_t)blockIdx.y * 32;
-  for (int j = threadIdx.y; j < 32; j += blockDim.y) {
-    const int64_t r = r0 + j, cidx = c0 + threadIdx.x;
-    tile[j][threadIdx.x] = (r < rows && cidx < cols) ? to_f32(X[r * ldx + cidx]) : 0.f;
+__global__ void __launch_bounds__(256) transpose_split_f16_kernel(const TIn* __restrict__ X, int64_t ldx, int64_t rows,
+                                                                  int64_t cols, const unsigned* __restrict__ umax,
+                                                                  __half* __restrict__ Thi, __half* __restrict__ Tlo,
+                                                                  int64_t ldt) {
+  __shared__ float tile[64][65];
+  const int64_t c0 = (int64_t)blockIdx.x * 64, r0 = (int64_t)blockIdx.y * 64;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int rr = w + 8 * i;
+    const int64_t r = r0 + rr;
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+      const int64_t cidx = c0 + lane + 32 * hf;
+      tile[rr][lane + 32 * hf] = (r < rows && cidx < cols) ? to_f32(X[r * ldx + cidx]) : 0.f;
+    }
   }
   __syncthreads();
-  for (int j = threadIdx.y; j < 32; j += blockDim.y) {
-    const int64_t cidx = c0 + j, r = r0 + threadIdx.x;
-    if (cidx < cols && r < ldt) {
-      const int e = scale_exp(__uint_as_float(umax[cidx]));
-      __half h, l;
-      split2(scalbnf(tile[threadIdx.x][j], e), h, l);
-      Thi[cidx * ldt + r] = h;
-      if (Tlo) Tlo[cidx * ldt + r] = l;
-    }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int ch = w + 8 * j;
+    const int64_t cidx = c0 + ch;
+    if (cidx >= cols) continue;
+    const int e = scale_exp(__uint_as_float(umax[cidx]));
+    __half h0, l0, h1, l1;
+    split2(scalbnf(tile[2 * lane][ch], e), h0, l0);
+    split2(scalbnf(tile[2 * lane + 1][ch], e), h1, l1);
+    const int64_t o = cidx * ldt + r0 + 2 * lane;             // even: ldt and r0 are multiples of 64
+    *reinterpret_cast<__half2*>(Thi + o) = __halves2half2(h0, h1);
+    if (Tlo) *reinterpret_cast<__half2*>(Tlo + o) = __halves2half2(l0, l1);
   }
 }
 
@@ -204,16 +217,16 @@ armor_status launch_f16_gram_stage(armor_ctx* c, const void* X, int x_dtype, int
   // one read for the maxima, one read and one 16-bit write per part for the staged chunk
   KTimer kt(c, ARMOR_KC_GRAM_STAGING, (double)rows * (double)cols * (x_dtype == ARMOR_DTYPE_BF16 ? 6.0 : 12.0), s);
   const dim3 g1((unsigned)((cols + NT - 1) / NT), (unsigned)((rows + 255) / 256));
-  const dim3 g2((unsigned)((cols + 31) / 32), (unsigned)((ldt + 31) / 32));
+  const dim3 g2((unsigned)((cols + 63) / 64), (unsigned)(ldt / 64));
   if (x_dtype == ARMOR_DTYPE_BF16) {
     const __nv_bfloat16* Xb = static_cast<const __nv_bfloat16*>(X);
     colabsmax_kernel<<<g1, NT, 0, s>>>(Xb, ldx, rows, cols, c->gmax);
-    transpose_split_f16_kernel<<<g2, dim3(32, 8), 0, s>>>(Xb, ldx, rows, cols, c->gmax, static_cast<__half*>(Thi),
+    transpose_split_f16_kernel<<<g2, 256, 0, s>>>(Xb, ldx, rows, cols, c->gmax, static_cast<__half*>(Thi),
                                                          (__half*)nullptr, ldt);
   } else {
     const float* Xf = static_cast<const float*>(X);
     colabsmax_kernel<<<g1, NT, 0, s>>>(Xf, ldx, rows, cols, c->gmax);
-    transpose_split_f16_kernel<<<g2, dim3(32, 8), 0, s>>>(Xf, ldx, rows, cols, c->gmax, static_cast<__half*>(Thi),
+    transpose_split_f16_kernel<<<g2, 256, 0, s>>>(Xf, ldx, rows, cols, c->gmax, static_cast<__half*>(Thi),
                                                          static_cast<__half*>(Tlo), ldt);
   }
   gram_scale_kernel<<<(unsigned)((cols + 255) / 256), 256, 0, s>>>(c->gmax, c->gscale, cols);
