@@ -651,6 +651,55 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------- long runs
+def run_long(args, cfg):
+    """Thousands of iterations in ONE armor_bcd_step call per mode (the regime of the paper's schedule): the
+    loss the library tracks through the call against the loss evaluated afresh from the final state, which shows
+    what the quantities carried from iteration to iteration (T H_w, the running loss) have drifted by."""
+    from paper_2510_05528_b200 import binding as Bd
+    from paper_2510_05528_b200 import build as armor_build
+    armor_build.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    prec = {"fp32x3": Bd.PREC_FP32X3, "tf32": Bd.PREC_TF32, "fp16x3": Bd.PREC_FP16X3}[args.precision]
+    n = args.long_run
+    W_d = torch.from_numpy(inputs.make_weight(cfg)).to(dev)
+    base = Bd.ArmorContext(cfg.d_out, cfg.d_in, cfg.d_block, device=dev, precision=prec, seed=cfg.seed)
+    H = base.new_gram()
+    scales = torch.from_numpy(inputs.channel_scales(cfg))
+    for i in range(inputs.n_chunks(cfg)):
+        base.gram(inputs.activation_chunk(cfg, i, scales).to(dev), H)
+    del base
+    out = {}
+    for name, kw in (("full_exact", dict(h_mode=Bd.H_FULL)),
+                     ("diag_adam_lr1e-4", dict(h_mode=Bd.H_DIAG, ab_step=Bd.AB_ADAM))):
+        ctx = Bd.ArmorContext(cfg.d_out, cfg.d_in, cfg.d_block, device=dev, precision=prec, seed=cfg.seed, **kw)
+        st = ctx.init(W_d, H)
+        l_init = float(ctx.proxy_loss(st, H).item())
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        stats = ctx.bcd_step(st, H, 0, n)
+        e1.record()
+        torch.cuda.synchronize()
+        sr = ctx.read_stats(stats)
+        fresh = float(ctx.proxy_loss(st, H).item())
+        tracked = float(sr["loss_mask"][-1])
+        seq = np.concatenate([[l_init], sr["loss_mask"]])
+        Mb = st.M.cpu().numpy()
+        out[name] = {"iterations": n, "ms_per_iteration": e0.elapsed_time(e1) / n, "seconds": e0.elapsed_time(e1) / 1e3,
+                     "loss_init": l_init, "loss_after_100": float(sr["loss_mask"][min(99, n - 1)]),
+                     "loss_tracked_final": tracked, "loss_evaluated_final": fresh,
+                     "tracked_minus_evaluated_rel": (tracked - fresh) / fresh,
+                     "largest_rise_between_iterations_rel": float(np.max(np.diff(seq) / seq[:-1])),
+                     "mask_steps_accepted": int(sr["mask_accepted"].sum()), "groups_changed": int(sr["groups_changed"].sum()),
+                     "chol_failed": int(sr["chol_failed"].sum()),
+                     "valid_2_of_4": bool(np.all(np.unpackbits(Mb[:, :, None], axis=2)[:, :, 4:].sum(axis=2) == 2)),
+                     "device_status": ctx.device_status()[:10]}
+        del ctx, st
+    print(json.dumps({"long_run": out, "config": workload_config(cfg), "precision": args.precision}), flush=True)
+
+
 # ------------------------------------------------------------------------------------- whole layers
 # Sets of matrices that share their calibration activations.  (matrix name, inputs.CONFIGS entry, seed offset of W)
 LAYER_SETS = {
@@ -800,6 +849,9 @@ def main():
                     help="one matrix (inputs.CONFIGS) or a whole set of matrices sharing activations: " + ", ".join(sorted(LAYER_SETS)))
     ap.add_argument("--nm", default="2:4", choices=["2:4", "4:8", "5:8", "6:8"], help="sparsity pattern of the core")
     ap.add_argument("--apply-tokens", type=int, default=0, help="token batch of the forward (default 8192)")
+    ap.add_argument("--long-run", type=int, default=0,
+                    help="instead of the benchmark: this many iterations in one call, with the full weighting and exact "
+                         "solves and with the diagonal weighting and joint Adam; prints tracked and re-evaluated losses")
     ap.add_argument("--precision", default="fp16x3", choices=["fp16x3", "fp32x3", "tf32"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tokens", type=int, default=0,
@@ -840,7 +892,9 @@ def main():
         cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
                "--master-addr", "127.0.0.1", "--master-port", "29511", os.path.abspath(__file__)] + sys.argv[1:]
         raise SystemExit(subprocess.call(cmd))
-    if args.impl == "reference":
+    if args.long_run > 0:
+        run_long(args, cfg)
+    elif args.impl == "reference":
         run_reference(args, cfg)
     else:
         run_ours(args, cfg)
