@@ -122,7 +122,7 @@ def _stream() -> C.c_void_p:
 
 
 def make_config(d_out, d_in, d_block, *, n_keep=2, m_group=4, h_mode=H_FULL, select_mode=SELECT_L1_RANDOM,
-                s_step=S_EXACT, precision=PREC_FP32X3, normalize=0, phases=0, ab_step=AB_EXACT, mask_sweeps=1, mask_groups=1, ridge=1e-6,
+                s_step=S_EXACT, precision=PREC_FP16X3, normalize=0, phases=0, ab_step=AB_EXACT, mask_sweeps=1, mask_groups=1, ridge=1e-6,
                 adam_lr=0.0, adam_beta1=0.0, adam_beta2=0.0, adam_eps=0.0, seed=0) -> armor_config:
     return armor_config(d_out, d_in, d_block, n_keep, m_group, h_mode, select_mode, s_step, precision,
                         int(normalize), phases, ab_step, mask_sweeps, mask_groups, ridge, adam_lr, adam_beta1, adam_beta2, adam_eps, seed)
