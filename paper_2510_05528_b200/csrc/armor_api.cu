@@ -426,7 +426,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
     // every LOSS_REFRESH iterations after it; in between it is the loss the previous iteration ended with, which
     // follows from the evaluated one by the exact decreases of the quadratic sub-steps.
     const bool fresh_loss = adam || (it % LOSS_REFRESH == 0);
-    launch_zero_scalars(c, !fresh_loss, s);
+    launch_zero_scalars(c, !fresh_loss, is, s);      // with a carried loss this also opens the iteration's record
     if (adam) {
       // Adam normalises every entry's move, so a gradient that is exactly zero (the kept entries of the core at
       // the initialisation, where E vanishes on them) must come out as zero: E H_w is formed from E itself, not
@@ -443,9 +443,9 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
     bd_left(c, A, false, c->P, c->EH, d_out, d_in, -1.f, c->WH, 1.f, s);             // E H_w = W H_w - A P
     if (fresh_loss) {
       bd_left(c, A, false, c->T, c->E, d_out, d_in, -1.f, W, 1.f, s);                // E = W - A T
-      dot_to_ptr(c, c->EH, c->E, c->wn, c->sc + SC_L0, s);                           // L = <E H_w, E>
+      dot_partials(c, c->EH, c->E, c->wn, c->partials, s);                           // L = <E H_w, E>
+      launch_stage(c, is, 0, nullptr, 0, 0, s, c->partials, ARMOR_DOT_BLOCKS, SC_L0);
     }
-    launch_stage(c, is, 0, nullptr, 0, 0, s);
     }
 
     if (adam) {
@@ -517,9 +517,10 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       if (st != ARMOR_OK) return st;
       bd_left(c, A, false, c->Tmp, c->V, d_out, d_in, 1.f, nullptr, 0.f, s);         // V = A R
       bd_left(c, A, false, c->E, c->VH, d_out, d_in, 1.f, nullptr, 0.f, s);          // V H_w = A (R H_w)
-      dot_to_ptr(c, c->VH, c->V, c->wn, c->sc + SC_Q_B, s);
-      if (b_gd) launch_stage(c, is, 8, nullptr, 0, 0, s);
-      else launch_stage(c, is, 2, c->partblk, nbi * chol_parts_per_block(db, nbi), nbi, s);
+      dot_partials(c, c->VH, c->V, c->wn, c->partials, s);                           // q = <V H_w, V>, summed by the stage
+      if (b_gd) launch_stage(c, is, 8, nullptr, 0, 0, s, c->partials, ARMOR_DOT_BLOCKS, SC_Q_B);
+      else launch_stage(c, is, 2, c->partblk, nbi * chol_parts_per_block(db, nbi), nbi, s, c->partials, ARMOR_DOT_BLOCKS,
+                        SC_Q_B);
       launch_axpy_slot(c, B, c->Delta, (int64_t)nbi * db * db, SC_TAU_B, 1.f, s);    // B += tau Delta
       launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_B, -1.f, s);                   // EH -= tau V H_w
       if (carry_P) launch_axpy_slot(c, c->P, c->E, c->wn, SC_TAU_B, 1.f, s);         // P += tau R H_w
@@ -530,15 +531,19 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
     // ---- S-step: exact line search along Gamma (.) M ------------------------------------------
     if (!adam && (ph & ARMOR_PHASE_S)) {
       core_gradient(c, A, B, s);
-      launch_masked_copy(c, c->Gam, M, c->U, SC_NRM_S, s);                           // U = Gamma (.) M
+      double* nrm_part = c->partials + 8 * c->npart;                                 // kept until the stage below
+      launch_masked_copy(c, c->Gam, M, c->U, nrm_part, s);                           // U = Gamma (.) M, |U|^2
       bd_right(c, c->U, B, false, c->Tmp, d_out, d_in, 1.f, nullptr, 0.f, s);        // R = Gamma_M B
       st = rmul_H(c, c->Tmp, H, c->E, d_out, nullptr, nullptr, nullptr, nullptr, s); // R H_w
       if (st != ARMOR_OK) return st;
       bd_left(c, A, false, c->Tmp, c->V, d_out, d_in, 1.f, nullptr, 0.f, s);         // V = A Gamma_M B
       bd_left(c, A, false, c->E, c->VH, d_out, d_in, 1.f, nullptr, 0.f, s);          // V H_w = A (R H_w)
-      dot_to_ptr(c, c->VH, c->V, c->wn, c->sc + SC_Q_S, s);
-      if (c->cfg.s_step == ARMOR_S_BETA) {
-        // the paper's step size (Eq. lrWprime): |A^T A|_F and |B H_w B^T|_F
+      dot_partials(c, c->VH, c->V, c->wn, c->partials, s);                           // q = <V H_w, V>
+      const bool beta_step = (c->cfg.s_step == ARMOR_S_BETA);
+      if (beta_step) {
+        // the paper's step size (Eq. lrWprime): |A^T A|_F and |B H_w B^T|_F  (these dot products reuse the
+        // partial-sum buffer, so q is summed first)
+        reduce_partials_to(c, c->partials, ARMOR_DOT_BLOCKS, c->sc + SC_Q_S, s);
         block_mm(c, A, true, A, false, c->G, nbo, s);
         dot_to_ptr(c, c->G, c->G, (int64_t)nbo * db * db, c->sc + SC_BETA_A, s);
         if (c->cfg.h_mode == ARMOR_H_FULL) {
@@ -551,7 +556,8 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
           dot_to_ptr(c, c->Kfull, c->Kfull, (int64_t)nbi * db * db, c->sc + SC_BETA_K, s);
         }
       }
-      launch_stage(c, is, c->cfg.s_step == ARMOR_S_BETA ? 6 : 3, nullptr, 0, 0, s);
+      launch_stage(c, is, beta_step ? 6 : 3, nullptr, 0, 0, s, beta_step ? nullptr : c->partials, ARMOR_DOT_BLOCKS, SC_Q_S,
+                   nrm_part, ARMOR_DOT_BLOCKS, SC_NRM_S);
       launch_axpy_slot(c, S, c->U, c->wn, SC_TAU_S, 1.f, s);                         // S += tau Gamma_M
       launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_S, -1.f, s);                   // EH -= tau V H_w
       if (carry_P) launch_axpy_slot(c, c->P, c->E, c->wn, SC_TAU_S, 1.f, s);         // P += tau R H_w
@@ -561,9 +567,8 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
 
     // ---- sparse-core update (Algorithm 3), mask_sweeps times ------------------------------------
     if (ph & ARMOR_PHASE_MASK) {
-      launch_alpha(c, A, s);
       block_mm(c, B, false, c->Hjj, false, c->Ktmp, nbi, s);                         // B_j H_jj
-      block_mm(c, c->Ktmp, false, B, true, c->Kfull, nbi, s);                        // K_j = B_j H_jj B_j^T
+      launch_mask_prep(c, A, B, c->Ktmp, s);               // alpha_r and the m x m diagonal blocks of K_j = B_j H_jj B_j^T
       for (int sw = 0; sw < sweeps; ++sw) {
         if (sw > 0) {
           // E H_w for the state the previous run left
@@ -584,7 +589,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
         core_gradient(c, A, B, s);
         launch_mask_select(c, c->Gam, S, M, t * sweeps + sw, s);
         launch_mask_quadratic(c, A, B, H, s);
-        launch_stage(c, is, 4, c->partblk, nbo * nbi * c->kg, 0, s);
+        launch_stage(c, is, 4, c->partblk, nbo * nbi * c->kg, 0, s, c->quadpart, nbo * nbi * c->kg, SC_Q_M);
         launch_mask_commit(c, S, M, is, s);
       }
       if (carry_P && it + 1 < n_iters) launch_mask_carry_P(c, c->P, s);              // P += dS B H_w (if accepted)

@@ -244,19 +244,20 @@ armor_status launch_f16_gram_stage(armor_ctx* c, const void* X, int x_dtype, int
 
 // deterministic reductions (two stages, fixed order)
 void dot_to_ptr(armor_ctx* c, const float* x, const float* y, int64_t n, double* out, cudaStream_t s);
+void dot_partials(armor_ctx* c, const float* x, const float* y, int64_t n, double* part, cudaStream_t s);
 void reduce_partials_to(armor_ctx* c, const double* part, int n, double* out, cudaStream_t s);
 
 // streaming kernels (kernels_stream.cu)
 void launch_colscale(armor_ctx* c, const float* in, const float* h, float* out, int64_t rows, int64_t cols,
                      cudaStream_t s);
 void launch_extract_hblocks(armor_ctx* c, const float* H, cudaStream_t s);   // hdiag, Hjj (per h_mode)
-void launch_masked_copy(armor_ctx* c, const float* Gam, const uint8_t* M, float* out, int slot_norm,
-                        cudaStream_t s);                                     // out = Gam (.) M, sc[slot] = ||out||^2
+void launch_masked_copy(armor_ctx* c, const float* Gam, const uint8_t* M, float* out, double* part,
+                        cudaStream_t s);              // out = Gam (.) M; ARMOR_DOT_BLOCKS partial sums of ||out||^2
 void launch_axpy_slot(armor_ctx* c, float* y, const float* x, int64_t n, int slot, float sign,
                       cudaStream_t s);                                       // y += sign * sc[slot] * x
 void launch_init(armor_ctx* c, const float* W, const float* H, float* Wbar, float* r1, float* r2,
                  float* A, float* B, float* S, uint8_t* M, cudaStream_t s);
-void launch_zero_scalars(armor_ctx* c, bool carry_loss, cudaStream_t s);
+void launch_zero_scalars(armor_ctx* c, bool carry_loss, armor_iter_stats* st, cudaStream_t s);
 // Input screening at the top of a call: counts non-finite entries of W and H and negative / zero diagonal
 // entries of H into the status words and sets or clears ST_POISON for the call.
 armor_status launch_screen_inputs(armor_ctx* c, const float* W, const float* H, cudaStream_t s);
@@ -269,8 +270,10 @@ void launch_adam(armor_ctx* c, float* theta, const float* gamma, float* m, float
 void launch_block_fro_sum(armor_ctx* c, const float* X, int nblk, const float* hdiag, double* out, cudaStream_t s);
 void launch_zero_flags(armor_ctx* c, cudaStream_t s);
 // per-iteration bookkeeping on the device: stage 0 start, 1 after A, 2 after B, 3 after S, 4 mask accept
+// (p1, n1, slot1), (p2, n2, slot2): partial sums the stage first adds up into sc[slot] (a preceding dot product)
 void launch_stage(armor_ctx* c, armor_iter_stats* st, int stage, const double* part, int npart, int nflag,
-                  cudaStream_t s);
+                  cudaStream_t s, const double* p1 = nullptr, int n1 = 0, int slot1 = 0, const double* p2 = nullptr,
+                  int n2 = 0, int slot2 = 0);
 void launch_scale_rows_cols(armor_ctx* c, const float* in, const float* colscale, const float* rowscale,
                             float* out, int64_t rows, int64_t cols, cudaStream_t s);
 void launch_split_hilo(armor_ctx* c, const float* in, float* hi, float* lo, int64_t n, cudaStream_t s);
@@ -293,10 +296,12 @@ armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float*
 
 // sparse-core update (kernels_mask.cu)
 void launch_alpha(armor_ctx* c, const float* A, cudaStream_t s);
+// alpha and the m x m diagonal blocks of K_j = Y_j B_j^T (Y = B_j H_jj, [nbi, db, db]) in one launch
+void launch_mask_prep(armor_ctx* c, const float* A, const float* B, const float* Y, cudaStream_t s);
 void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const uint8_t* M, int64_t t,
                         cudaStream_t s);
-// exact loss change of the iteration's group updates without a dense product: fills sc[SC_Q_M] = tr(V H_w V^T)
-// for V = A dS B from the selection records
+// exact loss change of the iteration's group updates without a dense product: fills quadpart with the per-block
+// terms of tr(V H_w V^T), V = A dS B, from the selection records (the stage kernel adds them into sc[SC_Q_M])
 void launch_mask_quadratic(armor_ctx* c, const float* A, const float* B, const float* H, cudaStream_t s);
 void launch_mask_commit(armor_ctx* c, float* S, uint8_t* M, armor_iter_stats* st, cudaStream_t s);
 // P += dS B H_w for the accepted group updates, from the rows the guard has formed (full weighting only)

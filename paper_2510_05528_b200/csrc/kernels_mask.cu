@@ -525,6 +525,79 @@ void launch_alpha(armor_ctx* c, const float* A, cudaStream_t s) {
   c->launches++;
 }
 
+// alpha (column norms of the blocks of A) and the m x m diagonal blocks of K_j = (B_j H_jj) B_j^T, the only entries
+// of K_j the group solves read (Appendix B.1: B' D B'^T for the m rows of one group), in one launch.
+// Y = B_j H_jj comes from a block product.  CTAs [0, n_kc): one warp per group, lane l takes columns l, l + 32, ..;
+// the remaining CTAs compute alpha.
+template <int MG>
+__global__ void __launch_bounds__(NT) mask_prep_kernel(const float* __restrict__ A, const float* __restrict__ B,
+                                                       const float* __restrict__ Y, float* __restrict__ Kfull,
+                                                       float* __restrict__ alpha, int db, int nbi, int n_kc) {
+  if ((int)blockIdx.x < n_kc) {
+    const int gpb = db / MG;
+    const int wg = blockIdx.x * (NT / 32) + (threadIdx.x >> 5);       // (column block, group)
+    const int lane = threadIdx.x & 31;
+    if (wg >= nbi * gpb) return;
+    const int j = wg / gpb, lc = (wg % gpb) * MG;
+    const float* Yj = Y + (int64_t)j * db * db;
+    const float* Bj = B + (int64_t)j * db * db;
+    float acc[MG][MG];
+#pragma unroll
+    for (int p = 0; p < MG; ++p)
+#pragma unroll
+      for (int q = 0; q < MG; ++q) acc[p][q] = 0.f;
+    for (int k = lane; k < db; k += 32) {
+      float y[MG], b[MG];
+#pragma unroll
+      for (int p = 0; p < MG; ++p) { y[p] = Yj[(int64_t)(lc + p) * db + k]; b[p] = Bj[(int64_t)(lc + p) * db + k]; }
+#pragma unroll
+      for (int p = 0; p < MG; ++p)
+#pragma unroll
+        for (int q = 0; q < MG; ++q) acc[p][q] = fmaf(y[p], b[q], acc[p][q]);
+    }
+#pragma unroll
+    for (int p = 0; p < MG; ++p)
+#pragma unroll
+      for (int q = 0; q < MG; ++q) {
+        float v = acc[p][q];
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) Kfull[(int64_t)j * db * db + (int64_t)(lc + p) * db + (lc + q)] = v;
+      }
+    return;
+  }
+  // alpha[r] = || A_i[:, r] ||^2: 256 threads = 32 columns x 8 row slices
+  const int ab = blockIdx.x - n_kc;
+  const int per = (db + 31) / 32;
+  const int i = ab / per;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int r = (ab % per) * 32 + tx;
+  const float* Ai = A + (int64_t)i * db * db;
+  double acc = 0.0;
+  if (r < db)
+    for (int o = ty; o < db; o += 8) {
+      const double v = Ai[(int64_t)o * db + r];
+      acc += v * v;
+    }
+  __shared__ double part[8][33];
+  part[ty][tx] = acc;
+  __syncthreads();
+  if (ty == 0 && r < db) {
+    double t = 0.0;
+    for (int k = 0; k < 8; ++k) t += part[k][tx];
+    alpha[i * db + r] = (float)t;
+  }
+}
+
+void launch_mask_prep(armor_ctx* c, const float* A, const float* B, const float* Y, cudaStream_t s) {
+  const int db = c->db, mg = c->cfg.m_group;
+  const int n_kc = (c->nbi * (db / mg) + NT / 32 - 1) / (NT / 32);
+  const int n_al = c->nbo * ((db + 31) / 32);
+  KTimer kt(c, ARMOR_KC_MASK_GUARD, 0.0, s);
+  if (mg == 8) mask_prep_kernel<8><<<n_kc + n_al, NT, 0, s>>>(A, B, Y, c->Kfull, c->alpha, db, c->nbi, n_kc);
+  else mask_prep_kernel<4><<<n_kc + n_al, NT, 0, s>>>(A, B, Y, c->Kfull, c->alpha, db, c->nbi, n_kc);
+  c->launches++;
+}
+
 void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const uint8_t* M, int64_t t, cudaStream_t s) {
   const int mg = c->cfg.m_group;
   const uint64_t n_groups = (uint64_t)(c->d_out * (c->d_in / mg));
@@ -585,7 +658,7 @@ void launch_mask_quadratic(armor_ctx* c, const float* A, const float* B, const f
     mask_quad_kernel<<<nbo * nbv, NT, 0, s>>>(c->Zsel, c->Acol, Y, c->hdiag, part, c->d_in, db, nbo_pad, nbi, nbv);
   }
   c->launches++;
-  reduce_partials_to(c, part, nbo * nbv, c->sc + SC_Q_M, s);
+  // (the caller's stage kernel adds the nbo * nbv terms up into sc[SC_Q_M])
 }
 
 void launch_mask_commit(armor_ctx* c, float* S, uint8_t* M, armor_iter_stats* st, cudaStream_t s) {

@@ -223,12 +223,26 @@ __global__ void copy_kernel(const float4* __restrict__ in, float4* __restrict__ 
 }
 
 // ---- scalars and per-iteration bookkeeping ------------------------------------------------------
-// carry_loss: the running loss of the previous iteration becomes this iteration's starting loss
-__global__ void zero_scalars_kernel(double* sc, int32_t* failflag, int nflag, int carry_loss) {
+__device__ __forceinline__ void start_record(armor_iter_stats* st, double loss) {
+  st->loss_start = loss;
+  st->chol_failed = 0;
+  st->groups_changed = 0;
+  st->mask_accepted = 0;
+  st->delta_L_mask = 0.0;
+  st->tau_B = 0.f;
+  st->tau_S = 0.f;
+  st->reserved = 0;
+}
+
+// carry_loss: the running loss of the previous iteration becomes this iteration's starting loss, and the
+// iteration's record is opened here (no loss evaluation follows)
+__global__ void zero_scalars_kernel(double* sc, int32_t* failflag, int nflag, int carry_loss, armor_iter_stats* st) {
   const double carried = sc[SC_LOSS];
   __syncthreads();
-  for (int i = threadIdx.x; i < SC_COUNT; i += blockDim.x) sc[i] = (carry_loss && i == SC_L0) ? carried : 0.0;
+  for (int i = threadIdx.x; i < SC_COUNT; i += blockDim.x)
+    sc[i] = (carry_loss && (i == SC_L0 || i == SC_LOSS)) ? carried : 0.0;
   for (int i = threadIdx.x; i < nflag; i += blockDim.x) failflag[i] = 0;
+  if (carry_loss && st && threadIdx.x == 0) start_record(st, carried);
 }
 
 // Fixed-order sums by one warp: lane l adds entries l, l + 32, ...; then a shuffle tree.  All lanes get the sum.
@@ -246,8 +260,14 @@ __device__ __forceinline__ int warp_count_flags(const int32_t* __restrict__ f, i
 }
 
 // stage 0: start, 1: after A, 2: after B, 3 / 6: after S, 4: mask accept, 5: mask phase off.  One warp.
+// Up to two arrays of partial sums (p1, p2) are first added, in a fixed order, into the scalars slot1 / slot2: the
+// reductions of the dot products that precede the stage need no launch of their own.
 __global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const int32_t* failflag, int nflag,
-                             const double* partA, int nA, int32_t* status) {
+                             const double* partA, int nA, int32_t* status, const double* p1, int n1, int slot1,
+                             const double* p2, int n2, int slot2) {
+  if (p1) { const double v = warp_sum_f64(p1, n1); if (threadIdx.x == 0) sc[slot1] = v; }
+  if (p2) { const double v = warp_sum_f64(p2, n2); if (threadIdx.x == 0) sc[slot2] = v; }
+  __syncwarp();
   double psum = 0.0;
   int nf = 0;
   if (stage == 1 || stage == 2 || stage == 4) psum = warp_sum_f64(partA, nA);
@@ -256,16 +276,7 @@ __global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const 
   const bool poisoned = status[ST_POISON] != 0;   // unusable inputs: every step length is zero, nothing is accepted
   if (stage == 0) {
     sc[SC_LOSS] = sc[SC_L0];
-    if (st) {
-      st->loss_start = sc[SC_L0];
-      st->chol_failed = 0;
-      st->groups_changed = 0;
-      st->mask_accepted = 0;
-      st->delta_L_mask = 0.0;
-      st->tau_B = 0.f;
-      st->tau_S = 0.f;
-      st->reserved = 0;
-    }
+    if (st) start_record(st, sc[SC_L0]);
   } else if (stage == 1) {
     sc[SC_DEC_A] = psum;
     sc[SC_LOSS] -= psum;
@@ -503,6 +514,13 @@ void dot_to_ptr(armor_ctx* c, const float* x, const float* y, int64_t n, double*
   c->launches += 2;
 }
 
+// partial sums of <x, y> only (ARMOR_DOT_BLOCKS entries at `part`); the consumer adds them up
+void dot_partials(armor_ctx* c, const float* x, const float* y, int64_t n, double* part, cudaStream_t s) {
+  KTimer kt(c, n >= (1 << 22) ? ARMOR_KC_DOT : ARMOR_KC_SMALL, 8.0 * (double)n, s);
+  dot_partial_kernel<<<ARMOR_DOT_BLOCKS, NT, 0, s>>>((const float4*)x, (const float4*)y, n / 4, part);
+  c->launches++;
+}
+
 void reduce_partials_to(armor_ctx* c, const double* part, int n, double* out, cudaStream_t s) {
   KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
   reduce_final_kernel<<<1, NT, 0, s>>>(part, n, out);
@@ -535,12 +553,11 @@ void launch_extract_hblocks(armor_ctx* c, const float* H, cudaStream_t s) {
   c->launches++;
 }
 
-void launch_masked_copy(armor_ctx* c, const float* Gam, const uint8_t* M, float* out, int slot_norm, cudaStream_t s) {
+void launch_masked_copy(armor_ctx* c, const float* Gam, const uint8_t* M, float* out, double* part, cudaStream_t s) {
   KTimer kt(c, ARMOR_KC_MASKED_COPY, (8.0 + 1.0 / c->cfg.m_group) * (double)c->wn, s);
   masked_copy_kernel<<<ARMOR_DOT_BLOCKS, NT, 0, s>>>((const float4*)Gam, M, (float4*)out, c->wn / 4,
-                                                    c->cfg.m_group / 4, c->partials);
-  reduce_final_kernel<<<1, NT, 0, s>>>(c->partials, ARMOR_DOT_BLOCKS, c->sc + slot_norm);
-  c->launches += 2;
+                                                    c->cfg.m_group / 4, part);
+  c->launches++;
 }
 
 void launch_axpy_slot(armor_ctx* c, float* y, const float* x, int64_t n, int slot, float sign, cudaStream_t s) {
@@ -590,17 +607,18 @@ armor_status launch_screen_inputs(armor_ctx* c, const float* W, const float* H, 
   return ARMOR_OK;
 }
 
-void launch_zero_scalars(armor_ctx* c, bool carry_loss, cudaStream_t s) {
+void launch_zero_scalars(armor_ctx* c, bool carry_loss, armor_iter_stats* st, cudaStream_t s) {
   const int nflag = c->nbo > c->nbi ? c->nbo : c->nbi;
   KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
-  zero_scalars_kernel<<<1, NT, 0, s>>>(c->sc, c->failflag, nflag, carry_loss ? 1 : 0);
+  zero_scalars_kernel<<<1, NT, 0, s>>>(c->sc, c->failflag, nflag, carry_loss ? 1 : 0, st);
   c->launches++;
 }
 
 void launch_stage(armor_ctx* c, armor_iter_stats* st, int stage, const double* part, int npart, int nflag,
-                  cudaStream_t s) {
+                  cudaStream_t s, const double* p1, int n1, int slot1, const double* p2, int n2, int slot2) {
   KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
-  stage_kernel<<<1, 32, 0, s>>>(c->sc, st, stage, c->failflag, nflag, part, npart, c->status);
+  stage_kernel<<<1, 32, 0, s>>>(c->sc, st, stage, c->failflag, nflag, part, npart, c->status, p1, n1, slot1, p2, n2,
+                               slot2);
   c->launches++;
 }
 
