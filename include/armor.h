@@ -7,7 +7,7 @@
  * sparse core S = W' (.) M  (Section 3.1 of the paper).  The library minimises
  * the layer-wise proxy loss  L = tr(E H_w E^T),  E = W - A S B,  where
  * H_w = diag(X^T X) is the paper's weighting (Eq. proxy_loss, Section 3.2) and
- * H_w = X^T X is the full-Gram generalisation this build is timed on.
+ * H_w = X^T X is the full-Gram generalisation (the mode the benchmark times).
  *
  * Conventions for every call
  *   - All d_* pointers are DEVICE pointers owned by the caller; tensors are

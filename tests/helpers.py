@@ -8,7 +8,7 @@ from paper_2510_05528_b200 import binding as Bd
 DEV = "cuda:0"
 
 # Tolerances (relative Frobenius error against the fp64 oracle):
-#   fp32-grade modes (SIMT, FP32X3): the 1e-3 of the benchmark spec;
+#   fp32-grade modes (SIMT, FP32X3): 1e-3, the bound this library is specified to (fp32 results against fp64);
 #   FP16X3 carries the same 22 operand bits as FP32X3 (exact power-of-two scaling, two fp16 parts): same bars;
 #   TF32 (one tensor-core pass, operands rounded to 10 mantissa bits, relative rounding 2^-11 = 4.9e-4
 #   per operand): GEMM outputs carry ~1e-3, the block solves pass that on to A and B with a small
