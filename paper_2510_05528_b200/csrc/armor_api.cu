@@ -83,6 +83,8 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   TAKE(Hjj, float*, bo);
   TAKE(Kfull, float*, bo);
   TAKE(Ktmp, float*, bo);
+  TAKE(Hinv, float*, bo);
+  TAKE(hinv_fail, int32_t*, (size_t)nbi * sizeof(int32_t));
   TAKE(alpha, float*, (size_t)cfg.d_out * sizeof(float));
   TAKE(hdiag, float*, (size_t)cfg.d_in * sizeof(float));
   const int64_t nbo_pad = (nbo + 31) / 32 * 32;
@@ -418,6 +420,10 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
   const bool adam = (c->cfg.ab_step == ARMOR_AB_ADAM);
   const int sweeps = c->cfg.mask_sweeps > 0 ? c->cfg.mask_sweeps : 1;
   const bool carry_P = (c->cfg.h_mode == ARMOR_H_FULL) && !adam;
+  if (!adam && c->cfg.ab_step == ARMOR_AB_EXACT && (ph & ARMOR_PHASE_B) && n_iters > 0) {
+    st = launch_hjj_inverse(c, s);
+    if (st != ARMOR_OK) return st;
+  }
   if (adam && t_first == 0 && reset_adam(c, s) != ARMOR_OK) return ARMOR_ERR_CUDA;
   for (int it = 0; it < n_iters; ++it) {
     armor_iter_stats* is = d_stats ? d_stats + it : nullptr;
@@ -506,10 +512,13 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
         launch_block_fro_sum(c, c->V, nbo * nbi, c->hdiag, c->sc + SC_HB_B, s);
         dot_to_ptr(c, c->GamB, c->GamB, nbl, c->sc + SC_GD_B, s);                    // <Gamma, Delta>
       } else {
-        st = launch_chol(c, 1, c->C, c->GamB, c->Delta, nullptr, nullptr, nbi, nullptr, s);
+        // Delta_j = (C_j + lam I)^-1 Gamma_j (H_jj + mu I)^-1: a solve with C_j, then a product with the inverse
+        // that was formed once for the call (as accurate here as a second solve: both are good to a few 1e-7 on
+        // these blocks, and it replaces a latency-bound factorisation by a small product)
+        st = launch_chol(c, 1, c->C, c->GamB, c->Ktmp, nullptr, nullptr, nbi, nullptr, s);
         if (st != ARMOR_OK) return st;
-        st = launch_chol(c, 2, c->Hjj, c->Delta, c->Delta, c->GamB, nullptr, nbi, c->partblk, s);
-        if (st != ARMOR_OK) return st;
+        block_mm(c, c->Ktmp, false, c->Hinv, false, c->Delta, nbi, s);
+        launch_delta_finish(c, c->Delta, c->GamB, c->partblk, s);                    // part_j = <Gamma_j, Delta_j>
       }
       // direction in B: V = A R with R = S Delta; R H_w serves both V H_w = A (R H_w) and the carried P
       bd_right(c, S, c->Delta, false, c->Tmp, d_out, d_in, 1.f, nullptr, 0.f, s);    // R = S Delta
@@ -519,8 +528,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       bd_left(c, A, false, c->E, c->VH, d_out, d_in, 1.f, nullptr, 0.f, s);          // V H_w = A (R H_w)
       dot_partials(c, c->VH, c->V, c->wn, c->partials, s);                           // q = <V H_w, V>, summed by the stage
       if (b_gd) launch_stage(c, is, 8, nullptr, 0, 0, s, c->partials, ARMOR_DOT_BLOCKS, SC_Q_B);
-      else launch_stage(c, is, 2, c->partblk, nbi * chol_parts_per_block(db, nbi), nbi, s, c->partials, ARMOR_DOT_BLOCKS,
-                        SC_Q_B);
+      else launch_stage(c, is, 2, c->partblk, nbi, nbi, s, c->partials, ARMOR_DOT_BLOCKS, SC_Q_B);
       launch_axpy_slot(c, B, c->Delta, (int64_t)nbi * db * db, SC_TAU_B, 1.f, s);    // B += tau Delta
       launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_B, -1.f, s);                   // EH -= tau V H_w
       if (carry_P) launch_axpy_slot(c, c->P, c->E, c->wn, SC_TAU_B, 1.f, s);         // P += tau R H_w

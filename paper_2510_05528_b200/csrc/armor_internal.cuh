@@ -70,6 +70,8 @@ struct armor_ctx {
   float *Lo, *Hlo;
   // [nb, db, db] scratch
   float *G, *GamA, *dA, *C, *GamB, *Delta, *Hjj, *Kfull, *Ktmp;
+  float* Hinv;           // (H_jj + mu I)^-1 per column block, formed once per armor_bcd_step call
+  int32_t* hinv_fail;    // [nbi] 1 where that block was not positive definite
   float *alpha, *hdiag;
   float *mA, *vA, *mB, *vB, *mS, *vS;   // Adam moment estimates (ab_step ADAM)
   float *Hq1, *Hq2;      // [d_in, d_in] scratch of the paper's step size (s_step BETA, full weighting)
@@ -291,6 +293,11 @@ void launch_f32_to_bf16(armor_ctx* c, const float* in, const float* colscale, vo
 // mode 2: out = rhs (G + lam I)^-1, part[b] = <dotw, out>
 // partial sums written per block by launch_chol (modes 0 and 2)
 int chol_parts_per_block(int db, int nb);
+// (H_jj + mu I)^-1 for every column block into c->Hinv (H_jj does not change inside a call), failures into c->hinv_fail
+armor_status launch_hjj_inverse(armor_ctx* c, cudaStream_t s);
+// after Delta = Y Hinv: zeroes the blocks whose H_jj was not positive definite (raising their failflag, as a failed
+// solve would) and writes part[j] = <dotw_j, Delta_j>
+void launch_delta_finish(armor_ctx* c, float* Delta, const float* dotw, double* part, cudaStream_t s);
 armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float* rhs, float* out, const float* dotw,
                          float* A, int nb, double* part, cudaStream_t s);
 

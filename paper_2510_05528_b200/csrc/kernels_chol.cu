@@ -548,3 +548,65 @@ armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float*
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
 }
+
+namespace {
+
+__global__ void identity_rhs_kernel(float* __restrict__ X, int db) {
+  float* Xb = X + (int64_t)blockIdx.x * db * db;
+  for (int e = threadIdx.x; e < db * db; e += blockDim.x) Xb[e] = (e / db == e % db) ? 1.f : 0.f;
+}
+
+__global__ void save_flags_kernel(const int32_t* __restrict__ failflag, int32_t* __restrict__ saved, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) saved[i] = failflag[i];
+}
+
+// one CTA per block: Delta_j = 0 and failflag[j] = 1 where the inverse does not exist; part[j] = <dotw_j, Delta_j>
+__global__ void __launch_bounds__(NT) delta_finish_kernel(float* __restrict__ Delta, const float* __restrict__ dotw,
+                                                          const int32_t* __restrict__ hinv_fail,
+                                                          int32_t* __restrict__ failflag, double* __restrict__ part,
+                                                          int db) {
+  const int j = blockIdx.x;
+  const int64_t off = (int64_t)j * db * db;
+  const bool bad = hinv_fail[j] != 0;
+  double acc = 0.0;
+  for (int e = threadIdx.x; e < db * db; e += NT) {
+    if (bad) Delta[off + e] = 0.f;
+    else acc += (double)dotw[off + e] * (double)Delta[off + e];
+  }
+  __shared__ double red[NT / 32];
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    for (int w = 0; w < NT / 32; ++w) t += red[w];
+    part[j] = t;
+    if (bad) failflag[j] = 1;
+  }
+}
+
+}  // namespace
+
+armor_status launch_hjj_inverse(armor_ctx* c, cudaStream_t s) {
+  const int nbi = c->nbi;
+  if (cudaMemsetAsync(c->failflag, 0, (size_t)nbi * sizeof(int32_t), s) != cudaSuccess) return ARMOR_ERR_CUDA;
+  {
+    KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
+    identity_rhs_kernel<<<nbi, NT, 0, s>>>(c->Ktmp, c->db);
+    c->launches++;
+  }
+  armor_status st = launch_chol(c, 1, c->Hjj, c->Ktmp, c->Hinv, nullptr, nullptr, nbi, nullptr, s);
+  if (st != ARMOR_OK) return st;
+  KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
+  save_flags_kernel<<<(nbi + 255) / 256, 256, 0, s>>>(c->failflag, c->hinv_fail, nbi);
+  c->launches++;
+  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+}
+
+void launch_delta_finish(armor_ctx* c, float* Delta, const float* dotw, double* part, cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
+  delta_finish_kernel<<<c->nbi, NT, 0, s>>>(Delta, dotw, c->hinv_fail, c->failflag, part, c->db);
+  c->launches++;
+}
+
