@@ -117,3 +117,37 @@ def test_a_dead_channel_is_reported_and_handled():
     assert rel(host(st.A), A) < tol["A"] and rel(host(st.B), B) < tol["B"]
     for k_gpu, k_or in (("loss_start", "start"), ("loss_A", "A"), ("loss_B", "B"), ("loss_S", "S")):
         assert abs(sg[k_gpu] - info.loss[k_or]) / info.loss[k_or] < tol["loss"]
+
+
+@pytest.mark.parametrize("prec", [Bd.PREC_SIMT, Bd.PREC_FP16X3], ids=["simt", "fp16x3"])
+def test_a_diagonal_block_of_H_that_is_not_positive_definite_is_skipped(prec):
+    """H with a positive diagonal but an indefinite diagonal block (one off-diagonal pair pushed beyond the
+    Cauchy-Schwarz bound): the screening lets it pass, the B-step finds (H_jj + mu I) not positive definite, leaves
+    that block of B where it was, counts the failure in every iteration, and moves the other blocks like the
+    oracle (B-step alone; its per-call inverse of H_jj is the object under test)."""
+    cfg = MID
+    W, X, H32 = data(cfg)
+    db = cfg.d_block
+    j, a, b = 2, 2 * db + 5, 2 * db + 40
+    H32 = H32.copy()
+    H32[a, b] = H32[b, a] = 1.5 * np.sqrt(H32[a, a] * H32[b, b])
+    ctx = make(cfg, prec, phases=Bd.PHASE_B)
+    Hd = dev(H32)
+    st = ctx.init(dev(W), Hd)
+    oc = O.OracleConfig(db, seed=cfg.seed, phases=O.PH_B)
+    Wn, Hq = W.astype(np.float64), H32.astype(np.float64)
+    A, B, S, M = O.init(Wn, Hq, oc)
+    rng = np.random.default_rng(5)
+    A = (A + 0.05 * rng.standard_normal(A.shape)).astype(np.float32).astype(np.float64)
+    B = (B + 0.05 * rng.standard_normal(B.shape)).astype(np.float32).astype(np.float64)
+    load_state(st, A, B, S, M)
+    sg = ctx.read_stats(ctx.bcd_step(st, Hd, 0, 2))
+    s = ctx.device_status()
+    assert [int(x) for x in sg["chol_failed"]] == [1, 1] and s[0] == 2 and s[1] == j + 1 and s[ST_POISON] == 0
+    assert np.array_equal(host(st.B)[j], B[j].astype(np.float32))              # the failing block did not move
+    B1, tau1, failed1 = O.b_step(Wn, A, B, S, Hq, oc)
+    B2, tau2, failed2 = O.b_step(Wn, A, B1, S, Hq, oc)
+    assert failed1 == failed2 == 1
+    tol = TOL[prec]
+    assert abs(sg["tau_B"][0] - tau1) <= 10 * tol["B"] * abs(tau1) and abs(sg["tau_B"][1] - tau2) <= 10 * tol["B"] * abs(tau2)
+    assert rel(host(st.B), B2) < tol["B"]
