@@ -141,6 +141,7 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
   TAKE(tab_g, unsigned long long*, (size_t)nbo * nbi * sizeof(unsigned long long));
   TAKE(status, int32_t*, ST_COUNT * sizeof(int32_t));
   TAKE(screen, int32_t*, 4 * sizeof(int32_t));
+  TAKE(it_dev, int64_t*, sizeof(int64_t));
 #undef TAKE
   if (c) {
     c->npart = npart;
@@ -293,6 +294,9 @@ armor_status armor_create(armor_ctx** out, const armor_config* cfg, void* d_work
     delete c;
     return ARMOR_ERR_CUDA;
   }
+  c->use_graphs = 1;
+  c->cap_stream = nullptr;
+  if (cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking) != cudaSuccess) c->cap_stream = nullptr;
   c->kg = cfg->mask_groups > 0 ? cfg->mask_groups : 1;
   c->h_cached = nullptr;
   c->timing_on = 0; c->timing_n = 0; c->ev_beg = nullptr; c->ev_end = nullptr; c->ev_cls = nullptr; c->ev_work = nullptr;
@@ -311,6 +315,7 @@ armor_status armor_destroy(armor_ctx* c) {
   delete[] c->ev_end;
   delete[] c->ev_cls;
   delete[] c->ev_work;
+  if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
   delete c;
   return ARMOR_OK;
 }
@@ -350,6 +355,12 @@ armor_status armor_kernel_timing(armor_ctx* c, int32_t n_classes, int64_t* launc
     total_work[k] += c->ev_work[i];
   }
   c->timing_n = 0;
+  return ARMOR_OK;
+}
+
+armor_status armor_use_graphs(armor_ctx* c, int32_t enable) {
+  if (!c) return ARMOR_ERR_INVALID_ARG;
+  c->use_graphs = enable ? 1 : 0;
   return ARMOR_OK;
 }
 
@@ -425,24 +436,28 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
     if (st != ARMOR_OK) return st;
   }
   if (adam && t_first == 0 && reset_adam(c, s) != ARMOR_OK) return ARMOR_ERR_CUDA;
-  for (int it = 0; it < n_iters; ++it) {
-    armor_iter_stats* is = d_stats ? d_stats + it : nullptr;
-    const int64_t t = t_first + it;
-    // The loss at the start of an iteration is evaluated from the residual in the first iteration of a call and
-    // every LOSS_REFRESH iterations after it; in between it is the loss the previous iteration ended with, which
-    // follows from the evaluated one by the exact decreases of the quadratic sub-steps.
-    const bool fresh_loss = adam || (it % LOSS_REFRESH == 0);
+  // One iteration, enqueued on stream s.  Which iteration it is reaches the kernels through the device counter
+  // c->it_dev (record d_stats[it], selection counter, Adam's step number), so that the same sequence of launches
+  // serves every iteration but the first of a call and can be replayed from a CUDA graph.
+  //   first:      the first iteration of the call (T H_w is formed by a dense product);
+  //   fresh_loss: the loss at the start is evaluated from the residual (first iteration, every LOSS_REFRESH-th, and
+  //               always with Adam); otherwise it is the loss the previous iteration ended with, which follows from
+  //               the evaluated one by the exact decreases of the quadratic sub-steps;
+  //   t_zero:     iteration 0 of the whole run (Adam: exact products, see below).
+  armor_iter_stats* const is = d_stats;   // base of the records; the kernels add the device counter
+  auto body = [&](bool first, bool fresh_loss, bool t_zero, cudaStream_t s) -> armor_status {
+    armor_status st = ARMOR_OK;
     launch_zero_scalars(c, !fresh_loss, is, s);      // with a carried loss this also opens the iteration's record
     if (adam) {
       // Adam normalises every entry's move, so a gradient that is exactly zero (the kept entries of the core at
       // the initialisation, where E vanishes on them) must come out as zero: E H_w is formed from E itself, not
       // as the difference W H_w - A P, and at t = 0 (identity wrappers) with the exact fp32 products
-      st = residual_and_loss(c, W, H, A, B, S, c->sc + SC_L0, s, t == 0);
+      st = residual_and_loss(c, W, H, A, B, S, c->sc + SC_L0, s, t_zero);
       if (st != ARMOR_OK) return st;
       launch_stage(c, is, 0, nullptr, 0, 0, s);
     } else {
     bd_right(c, S, B, false, c->T, d_out, d_in, 1.f, nullptr, 0.f, s);              // T = S B
-    if (it == 0 || !carry_P) {
+    if (first || !carry_P) {
       st = rmul_H(c, c->T, H, c->P, d_out, nullptr, nullptr, nullptr, nullptr, s);   // P = T H_w
       if (st != ARMOR_OK) return st;
     }
@@ -461,9 +476,9 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       bd_left(c, A, false, S, c->U, d_out, d_in, 1.f, nullptr, 0.f, s);              // U = A S
       colblock_grams(c, c->U, nullptr, c->EH, nullptr, c->GamB, s);                  // Gamma^B_j = U_j^T (E H_w)_j
       core_gradient(c, A, B, s);                                                     // Gamma = A^T E H_w B^T
-      launch_adam(c, A, c->GamA, c->mA, c->vA, na, nullptr, t + 1, s);
-      launch_adam(c, B, c->GamB, c->mB, c->vB, nbl, nullptr, t + 1, s);
-      launch_adam(c, S, c->Gam, c->mS, c->vS, c->wn, M, t + 1, s);
+      launch_adam(c, A, c->GamA, c->mA, c->vA, na, nullptr, t_first + 1, s);      // step number: t_first + 1 + counter
+      launch_adam(c, B, c->GamB, c->mB, c->vB, nbl, nullptr, t_first + 1, s);
+      launch_adam(c, S, c->Gam, c->mS, c->vS, c->wn, M, t_first + 1, s);
       // the new state: residual, E H_w and the loss afresh
       st = residual_and_loss(c, W, H, A, B, S, c->sc + SC_L0, s);
       if (st != ARMOR_OK) return st;
@@ -595,16 +610,65 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
           }
         }
         core_gradient(c, A, B, s);
-        launch_mask_select(c, c->Gam, S, M, t * sweeps + sw, s);
+        launch_mask_select(c, c->Gam, S, M, (uint64_t)(t_first * sweeps + sw), (uint64_t)sweeps, s);   // counter (t_first + it) K + k
         launch_mask_quadratic(c, A, B, H, s);
         launch_stage(c, is, 4, c->partblk, nbo * nbi * c->kg, 0, s, c->quadpart, nbo * nbi * c->kg, SC_Q_M);
         launch_mask_commit(c, S, M, is, s);
       }
-      if (carry_P && it + 1 < n_iters) launch_mask_carry_P(c, c->P, s);              // P += dS B H_w (if accepted)
+      if (carry_P) launch_mask_carry_P(c, c->P, s);                                  // P += dS B H_w (if accepted)
     } else {
       launch_stage(c, is, 5, nullptr, 0, 0, s);
     }
+    launch_advance_iteration(c, s);
+    return ARMOR_OK;
+  };
+
+  if (cudaMemsetAsync(c->it_dev, 0, sizeof(int64_t), s) != cudaSuccess) return ARMOR_ERR_CUDA;
+  // Iterations other than the first of the call (and the ones that re-evaluate the loss) enqueue the same launches:
+  // they are captured once, on a stream of the context's own, and replayed from a CUDA graph on the caller's stream
+  // (the gaps between the 50-odd small launches of an iteration are 3 - 4 % of its time otherwise).
+  auto is_generic = [&](int it) { return it > 0 && t_first + it != 0 && (adam || it % LOSS_REFRESH != 0); };
+  int n_generic = 0;
+  for (int it = 0; it < n_iters; ++it) n_generic += is_generic(it) ? 1 : 0;
+  bool use_graph = c->use_graphs && c->cap_stream && c->timing_on == 0 && n_generic >= 3;
+  if (use_graph) {
+    cudaStreamCaptureStatus cst = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(s, &cst) != cudaSuccess || cst != cudaStreamCaptureStatusNone) use_graph = false;
   }
+  cudaGraphExec_t exec = nullptr;
+  int64_t body_launches = 0;
+  armor_status result = ARMOR_OK;
+  for (int it = 0; it < n_iters && result == ARMOR_OK; ++it) {
+    if (use_graph && is_generic(it)) {
+      if (!exec) {
+        const int64_t l0 = c->launches;
+        cudaGraph_t graph = nullptr;
+        armor_status bst = ARMOR_ERR_CUDA;
+        if (cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+          bst = body(false, adam, false, c->cap_stream);
+          if (cudaStreamEndCapture(c->cap_stream, &graph) != cudaSuccess) bst = ARMOR_ERR_CUDA;
+        }
+        if (bst == ARMOR_OK && c->host_err == ARMOR_OK && graph && cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess) {
+          body_launches = c->launches - l0;
+        } else {
+          exec = nullptr;
+          use_graph = false;              // this call goes on with direct launches
+          c->host_err = ARMOR_OK;
+          (void)cudaGetLastError();
+        }
+        if (graph) cudaGraphDestroy(graph);
+        c->launches = l0;
+      }
+      if (exec) {
+        if (cudaGraphLaunch(exec, s) != cudaSuccess) result = ARMOR_ERR_CUDA;
+        c->launches += body_launches;
+        continue;
+      }
+    }
+    result = body(it == 0, adam || (it % LOSS_REFRESH == 0), t_first + it == 0, s);
+  }
+  if (exec) cudaGraphExecDestroy(exec);   // a graph still executing is released when it has finished
+  if (result != ARMOR_OK) { c->host_err = ARMOR_OK; return result; }
   return finish_call(c);
 }
 

@@ -101,6 +101,9 @@ struct armor_ctx {
   unsigned long long* tab_g;   // its global group index
   int32_t* status;    // [ST_COUNT]
   int32_t* screen;    // [4] per-call counters of the input screening
+  int64_t* it_dev;    // iteration index inside the running armor_bcd_step call (advanced by the last kernel of an iteration)
+  int use_graphs;     // 1: repeated iterations of a call are replayed from a CUDA graph
+  cudaStream_t cap_stream;   // the context's own stream, used only to capture that graph
   int64_t launches;
   int device;           // the device that was current at armor_create; every call must be issued with it current
   int n_sm;             // its number of SMs
@@ -259,14 +262,16 @@ void launch_axpy_slot(armor_ctx* c, float* y, const float* x, int64_t n, int slo
                       cudaStream_t s);                                       // y += sign * sc[slot] * x
 void launch_init(armor_ctx* c, const float* W, const float* H, float* Wbar, float* r1, float* r2,
                  float* A, float* B, float* S, uint8_t* M, cudaStream_t s);
+// st: base of the iteration records (the kernels add c->it_dev), or null
 void launch_zero_scalars(armor_ctx* c, bool carry_loss, armor_iter_stats* st, cudaStream_t s);
+void launch_advance_iteration(armor_ctx* c, cudaStream_t s);   // ++*c->it_dev
 // Input screening at the top of a call: counts non-finite entries of W and H and negative / zero diagonal
 // entries of H into the status words and sets or clears ST_POISON for the call.
 armor_status launch_screen_inputs(armor_ctx* c, const float* W, const float* H, cudaStream_t s);
 // One Adam step (Kingma & Ba, Algorithm 1) on n parameters with gradient g = -2 * gamma; step counts from 1.
 // M != nullptr: theta is the N:M core, one mask byte per m_group entries, masked-out entries stay zero.
 void launch_adam(armor_ctx* c, float* theta, const float* gamma, float* m, float* v, int64_t n, const uint8_t* M,
-                 int64_t step, cudaStream_t s);
+                 int64_t step_base, cudaStream_t s);   // step = step_base + *c->it_dev
 // part[b] = weight_b * || X_b ||_F for the nblk blocks of db x db floats in X; weight_b = 1, or the Euclidean
 // norm of hdiag over the (b % nbi)-th block of columns; out = sum of the parts (fixed order)
 void launch_block_fro_sum(armor_ctx* c, const float* X, int nblk, const float* hdiag, double* out, cudaStream_t s);
@@ -305,7 +310,8 @@ armor_status launch_chol(armor_ctx* c, int mode, const float* Gmat, const float*
 void launch_alpha(armor_ctx* c, const float* A, cudaStream_t s);
 // alpha and the m x m diagonal blocks of K_j = Y_j B_j^T (Y = B_j H_jj, [nbi, db, db]) in one launch
 void launch_mask_prep(armor_ctx* c, const float* A, const float* B, const float* Y, cudaStream_t s);
-void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const uint8_t* M, int64_t t,
+// selection counter t = t_base + t_mul * (*c->it_dev)
+void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const uint8_t* M, uint64_t t_base, uint64_t t_mul,
                         cudaStream_t s);
 // exact loss change of the iteration's group updates without a dense product: fills quadpart with the per-block
 // terms of tr(V H_w V^T), V = A dS B, from the selection records (the stage kernel adds them into sc[SC_Q_M])

@@ -125,10 +125,12 @@ __global__ void __launch_bounds__(NT) mask_select_kernel(const float* __restrict
                                                          const uint8_t* __restrict__ M, const float* __restrict__ alpha,
                                                          const float* __restrict__ Kfull, SelRec* __restrict__ sel,
                                                          double* __restrict__ part, int64_t d_in, int db, int nbi,
-                                                         int n_keep, int select_mode, uint64_t seed, uint64_t t,
+                                                         int n_keep, int select_mode, uint64_t seed, uint64_t t_base,
+                                                         uint64_t t_mul, const int64_t* __restrict__ it_dev,
                                                          uint64_t n_groups_total, int kg_arg,
                                                          float* __restrict__ tab_key,
                                                          unsigned long long* __restrict__ tab_g) {
+  const uint64_t t = t_base + t_mul * (uint64_t)(*it_dev);   // selection counter of this run of Algorithm 3
   const int kg = MULTI ? kg_arg : 1;                       // one draw: the loop and the key cache compile away
   const int bi = blockIdx.x / nbi, bj = blockIdx.x % nbi;
   extern __shared__ float s_keys[];         // kg > 1: the keys of the block's groups, kept for the later draws
@@ -466,7 +468,8 @@ __global__ void __launch_bounds__(NT) mask_quad_kernel(const float* __restrict__
 
 __global__ void mask_commit_kernel(const SelRec* __restrict__ sel, int nblocks, float* __restrict__ S,
                                    uint8_t* __restrict__ M, int64_t d_in, int mg, const double* __restrict__ sc,
-                                   armor_iter_stats* st) {
+                                   armor_iter_stats* st_base, const int64_t* __restrict__ it_dev) {
+  armor_iter_stats* st = st_base ? st_base + *it_dev : nullptr;
   __shared__ int changed;
   if (threadIdx.x == 0) changed = 0;
   __syncthreads();
@@ -598,11 +601,12 @@ void launch_mask_prep(armor_ctx* c, const float* A, const float* B, const float*
   c->launches++;
 }
 
-void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const uint8_t* M, int64_t t, cudaStream_t s) {
+void launch_mask_select(armor_ctx* c, const float* Gam, const float* S, const uint8_t* M, uint64_t t_base, uint64_t t_mul,
+                        cudaStream_t s) {
   const int mg = c->cfg.m_group;
   const uint64_t n_groups = (uint64_t)(c->d_out * (c->d_in / mg));
 #define ARMOR_SELECT_ARGS Gam, S, M, c->alpha, c->Kfull, c->sel, c->partblk, c->d_in, c->db, c->nbi, c->cfg.n_keep, \
-                          c->cfg.select_mode, c->cfg.seed, (uint64_t)t, n_groups, c->kg, c->tab_key, c->tab_g
+                          c->cfg.select_mode, c->cfg.seed, t_base, t_mul, c->it_dev, n_groups, c->kg, c->tab_key, c->tab_g
   // kg > 1: the block's keys stay in shared memory between the draws (up to 64 KiB: d_block 256, groups of four)
   const size_t smem = c->kg > 1 ? (size_t)c->db * (c->db / mg) * sizeof(float) : 0;
 #define ARMOR_SELECT_LAUNCH(MGV, NKV, MULTIV)                                                                           \
@@ -663,6 +667,7 @@ void launch_mask_quadratic(armor_ctx* c, const float* A, const float* B, const f
 
 void launch_mask_commit(armor_ctx* c, float* S, uint8_t* M, armor_iter_stats* st, cudaStream_t s) {
   KTimer kt(c, ARMOR_KC_MASK_GUARD, 0.0, s);
-  mask_commit_kernel<<<1, 256, 0, s>>>(c->sel, c->nbo * c->nbi * c->kg, S, M, c->d_in, c->cfg.m_group, c->sc, st);
+  mask_commit_kernel<<<1, 256, 0, s>>>(c->sel, c->nbo * c->nbi * c->kg, S, M, c->d_in, c->cfg.m_group, c->sc, st,
+                                       c->it_dev);
   c->launches++;
 }

@@ -236,7 +236,9 @@ __device__ __forceinline__ void start_record(armor_iter_stats* st, double loss) 
 
 // carry_loss: the running loss of the previous iteration becomes this iteration's starting loss, and the
 // iteration's record is opened here (no loss evaluation follows)
-__global__ void zero_scalars_kernel(double* sc, int32_t* failflag, int nflag, int carry_loss, armor_iter_stats* st) {
+__global__ void zero_scalars_kernel(double* sc, int32_t* failflag, int nflag, int carry_loss, armor_iter_stats* st_base,
+                                    const int64_t* __restrict__ it_dev) {
+  armor_iter_stats* st = st_base ? st_base + *it_dev : nullptr;
   const double carried = sc[SC_LOSS];
   __syncthreads();
   for (int i = threadIdx.x; i < SC_COUNT; i += blockDim.x)
@@ -262,9 +264,13 @@ __device__ __forceinline__ int warp_count_flags(const int32_t* __restrict__ f, i
 // stage 0: start, 1: after A, 2: after B, 3 / 6: after S, 4: mask accept, 5: mask phase off.  One warp.
 // Up to two arrays of partial sums (p1, p2) are first added, in a fixed order, into the scalars slot1 / slot2: the
 // reductions of the dot products that precede the stage need no launch of their own.
-__global__ void stage_kernel(double* sc, armor_iter_stats* st, int stage, const int32_t* failflag, int nflag,
+__global__ void advance_iteration_kernel(int64_t* it_dev) { *it_dev += 1; }
+
+__global__ void stage_kernel(double* sc, armor_iter_stats* st_base, const int64_t* __restrict__ it_dev, int stage,
+                             const int32_t* failflag, int nflag,
                              const double* partA, int nA, int32_t* status, const double* p1, int n1, int slot1,
                              const double* p2, int n2, int slot2) {
+  armor_iter_stats* st = st_base ? st_base + *it_dev : nullptr;
   if (p1) { const double v = warp_sum_f64(p1, n1); if (threadIdx.x == 0) sc[slot1] = v; }
   if (p2) { const double v = warp_sum_f64(p2, n2); if (threadIdx.x == 0) sc[slot2] = v; }
   __syncwarp();
@@ -476,9 +482,18 @@ __global__ void __launch_bounds__(NT) block_fro_kernel(const float4* __restrict_
 __global__ void __launch_bounds__(NT) adam_kernel(float4* __restrict__ theta, const float4* __restrict__ gamma,
                                                   float4* __restrict__ m, float4* __restrict__ v, int64_t n4,
                                                   const uint8_t* __restrict__ M, int q4, float lr, float b1, float b2,
-                                                  float eps, float inv_bc1, float inv_bc2,
+                                                  float eps, int64_t step_base, const int64_t* __restrict__ it_dev,
                                                   const int32_t* __restrict__ status) {
   if (status[ST_POISON] != 0) return;   // unusable inputs: parameters and moments stay as they are
+  // bias corrections 1 / (1 - beta^step), step = step_base + the iteration counter: once per block
+  __shared__ float s_bc[2];
+  if (threadIdx.x == 0) {
+    const double step = (double)(step_base + *it_dev);
+    s_bc[0] = (float)(1.0 / (1.0 - pow((double)b1, step)));
+    s_bc[1] = (float)(1.0 / (1.0 - pow((double)b2, step)));
+  }
+  __syncthreads();
+  const float inv_bc1 = s_bc[0], inv_bc2 = s_bc[1];
   for (int64_t i = (int64_t)blockIdx.x * NT + threadIdx.x; i < n4; i += (int64_t)gridDim.x * NT) {
     const float4 ga = gamma[i];
     float4 mm = m[i], vv = v[i], th = theta[i];
@@ -610,15 +625,21 @@ armor_status launch_screen_inputs(armor_ctx* c, const float* W, const float* H, 
 void launch_zero_scalars(armor_ctx* c, bool carry_loss, armor_iter_stats* st, cudaStream_t s) {
   const int nflag = c->nbo > c->nbi ? c->nbo : c->nbi;
   KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
-  zero_scalars_kernel<<<1, NT, 0, s>>>(c->sc, c->failflag, nflag, carry_loss ? 1 : 0, st);
+  zero_scalars_kernel<<<1, NT, 0, s>>>(c->sc, c->failflag, nflag, carry_loss ? 1 : 0, st, c->it_dev);
+  c->launches++;
+}
+
+void launch_advance_iteration(armor_ctx* c, cudaStream_t s) {
+  KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
+  advance_iteration_kernel<<<1, 1, 0, s>>>(c->it_dev);
   c->launches++;
 }
 
 void launch_stage(armor_ctx* c, armor_iter_stats* st, int stage, const double* part, int npart, int nflag,
                   cudaStream_t s, const double* p1, int n1, int slot1, const double* p2, int n2, int slot2) {
   KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
-  stage_kernel<<<1, 32, 0, s>>>(c->sc, st, stage, c->failflag, nflag, part, npart, c->status, p1, n1, slot1, p2, n2,
-                               slot2);
+  stage_kernel<<<1, 32, 0, s>>>(c->sc, st, c->it_dev, stage, c->failflag, nflag, part, npart, c->status, p1, n1, slot1,
+                               p2, n2, slot2);
   c->launches++;
 }
 
@@ -655,16 +676,14 @@ void launch_block_fro_sum(armor_ctx* c, const float* X, int nblk, const float* h
 }
 
 void launch_adam(armor_ctx* c, float* theta, const float* gamma, float* m, float* v, int64_t n, const uint8_t* M,
-                 int64_t step, cudaStream_t s) {
+                 int64_t step_base, cudaStream_t s) {
   const float lr = c->cfg.adam_lr > 0.f ? c->cfg.adam_lr : 1e-4f;
   const float b1 = c->cfg.adam_beta1 > 0.f ? c->cfg.adam_beta1 : 0.9f;
   const float b2 = c->cfg.adam_beta2 > 0.f ? c->cfg.adam_beta2 : 0.999f;
   const float eps = c->cfg.adam_eps > 0.f ? c->cfg.adam_eps : 1e-8f;
-  const double bc1 = 1.0 - pow((double)b1, (double)step), bc2 = 1.0 - pow((double)b2, (double)step);
   KTimer kt(c, n >= (1 << 22) ? ARMOR_KC_AXPY : ARMOR_KC_SMALL, 28.0 * (double)n, s);
   adam_kernel<<<grid_for(n / 4), NT, 0, s>>>((float4*)theta, (const float4*)gamma, (float4*)m, (float4*)v, n / 4, M,
-                                            c->cfg.m_group / 4, lr, b1, b2, eps, (float)(1.0 / bc1), (float)(1.0 / bc2),
-                                            c->status);
+                                            c->cfg.m_group / 4, lr, b1, b2, eps, step_base, c->it_dev, c->status);
   c->launches++;
 }
 
