@@ -231,6 +231,9 @@ armor_status armor_apply_layer(armor_ctx* ctx, const void* d_packed, const void*
  *     without weight), 9: 1 if the last screened call met any of 5-7.  Such a call withholds every update:
  *     A, B, S and M come back bit for bit as they went in (armor_init still writes its outputs), word 3 reads
  *     ARMOR_ERR_INVALID_ARG, and the next call with clean inputs runs normally.
+ *   word 10 (ARMOR_PREC_FP16X3): entries of H that, after the scaling by its diagonal, lie beyond the fp16 range and
+ *     were clamped (cumulative).  A positive semidefinite H has none; a non-zero count means the products with H
+ *     were not those of the H that was passed.
  * The caller must have synchronised the stream the context's work ran on.  (This call itself copies
  * synchronously.) */
 armor_status armor_get_device_status(armor_ctx* ctx, int32_t* h_codes, int32_t n);

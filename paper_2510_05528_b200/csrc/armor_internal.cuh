@@ -42,6 +42,7 @@ enum {
   ST_NEG_DIAG_H = 7,     // negative diagonal entries of H (H cannot be a Gram matrix)
   ST_DEAD_CHANNELS = 8,  // zero diagonal entries of H in the last screened call (legal: the channel carries no weight)
   ST_POISON = 9,         // 1 while the last screened call had unusable inputs: its updates were all withheld
+  ST_H_RANGE = 10,       // entries of the scaled H beyond the fp16 range (FP16X3; H not positive semidefinite): clamped
   ST_COUNT = 16
 };
 

@@ -23,7 +23,9 @@ constexpr int NT = 256;
 constexpr int TARGET_EXP = 15;   // frexp exponent of the scaled maximum: values in [2^14, 2^15)
 constexpr int H_SHIFT = 12;      // H / (d d^T) has entries below 4; times 2^12 they stay below 2^14
 
-__device__ __forceinline__ float clamp_f16(float v) { return fminf(fmaxf(v, -65504.f), 65504.f); }
+// Finite values beyond the fp16 range are clamped (after the scalings above this happens only to an H that is not
+// positive semidefinite); NaN and Inf pass through, so that unusable inputs stay visible in the result.
+__device__ __forceinline__ float clamp_f16(float v) { return isfinite(v) ? fminf(fmaxf(v, -65504.f), 65504.f) : v; }
 
 __device__ __forceinline__ void split2(float v, __half& hi, __half& lo) {
   v = clamp_f16(v);
@@ -69,18 +71,23 @@ __global__ void hpow_kernel(const float* __restrict__ hdiag, float* __restrict__
 
 // Hhi + Hlo = H_kn / (d_k d_n) * 2^H_SHIFT, four columns per thread
 __global__ void __launch_bounds__(NT) split_H_kernel(const float4* __restrict__ H, const float* __restrict__ hpow,
-                                                     __half2* __restrict__ hi, __half2* __restrict__ lo, int64_t n) {
+                                                     __half2* __restrict__ hi, __half2* __restrict__ lo, int64_t n,
+                                                     int32_t* __restrict__ status) {
   const int64_t n4 = n / 4;
   for (int64_t i = (int64_t)blockIdx.x * NT + threadIdx.x; i < n * n4; i += (int64_t)gridDim.x * NT) {
     const int64_t k = i / n4, c4 = (i % n4) * 4;
     const float rk = scalbnf(1.f / hpow[k], H_SHIFT);     // reciprocal of a power of two: exact
     const float4 v = H[i];
     const float4 d = *reinterpret_cast<const float4*>(hpow + c4);
+    const float x0 = v.x * rk / d.x, x1 = v.y * rk / d.y, x2 = v.z * rk / d.z, x3 = v.w * rk / d.w;
+    const int over = (fabsf(x0) > 65504.f && isfinite(x0)) + (fabsf(x1) > 65504.f && isfinite(x1)) +
+                     (fabsf(x2) > 65504.f && isfinite(x2)) + (fabsf(x3) > 65504.f && isfinite(x3));
+    if (over) atomicAdd(&status[ST_H_RANGE], over);
     __half h0, h1, h2, h3, l0, l1, l2, l3;
-    split2(v.x * rk / d.x, h0, l0);
-    split2(v.y * rk / d.y, h1, l1);
-    split2(v.z * rk / d.z, h2, l2);
-    split2(v.w * rk / d.w, h3, l3);
+    split2(x0, h0, l0);
+    split2(x1, h1, l1);
+    split2(x2, h2, l2);
+    split2(x3, h3, l3);
     hi[2 * i] = __halves2half2(h0, h1); hi[2 * i + 1] = __halves2half2(h2, h3);
     lo[2 * i] = __halves2half2(l0, l1); lo[2 * i + 1] = __halves2half2(l2, l3);
   }
@@ -197,7 +204,7 @@ void launch_f16_prepare_H(armor_ctx* c, const float* H, cudaStream_t s) {
   hpow_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(c->hdiag, c->hpow, n);
   __half* hi = reinterpret_cast<__half*>(c->Hlo);
   split_H_kernel<<<grid_for(n * n / 4), NT, 0, s>>>(reinterpret_cast<const float4*>(H), c->hpow,
-                                                    reinterpret_cast<__half2*>(hi), reinterpret_cast<__half2*>(hi + n * n), n);
+                                                    reinterpret_cast<__half2*>(hi), reinterpret_cast<__half2*>(hi + n * n), n, c->status);
   c->launches += 2;
 }
 

@@ -151,3 +151,27 @@ def test_a_diagonal_block_of_H_that_is_not_positive_definite_is_skipped(prec):
     tol = TOL[prec]
     assert abs(sg["tau_B"][0] - tau1) <= 10 * tol["B"] * abs(tau1) and abs(sg["tau_B"][1] - tau2) <= 10 * tol["B"] * abs(tau2)
     assert rel(host(st.B), B2) < tol["B"]
+
+
+def test_fp16_mode_reports_an_H_outside_its_range_and_passes_nan_activations_on():
+    """The three-pass fp16 mode scales H by its diagonal; a positive semidefinite H then fits the fp16 range.  An
+    entry far beyond the Cauchy-Schwarz bound does not: it is clamped and counted in status word 10.  A NaN in the
+    activations must reach the Gram (and from there the screening), not be swallowed by the clamping."""
+    cfg = MID
+    W, X, H32 = data(cfg)
+    ctx = make(cfg, Bd.PREC_FP16X3)
+    H_bad = H32.copy()
+    a, b = 7, 300
+    H_bad[a, b] = H_bad[b, a] = 100.0 * np.sqrt(H32[a, a] * H32[b, b])
+    Hd = dev(H_bad)
+    st = ctx.init(dev(W), Hd)
+    ctx.proxy_loss(st, Hd)
+    assert ctx.device_status()[10] == 2
+    Xn = X.copy()
+    Xn[17, 5] = np.nan
+    H = ctx.new_gram()
+    ctx.gram(dev(Xn), H)
+    Hh = host(H)
+    assert np.isnan(Hh[5, 5]) and np.isnan(Hh[5, 9]) and np.isnan(Hh[9, 5]) and np.isfinite(Hh[9, 9])
+    ctx.init(dev(W), H)
+    assert ctx.device_status()[ST_BAD_H] >= 2 * cfg.d_in - 1
