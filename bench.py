@@ -447,9 +447,9 @@ def run_ours(args, cfg):
     Bd.armor_gemm_timing_enable(ctx.ctx, False)
     status = ctx.device_status()
 
-    # ---- the same steps once more without the events around the GEMM launches: the library then replays the
-    # repeated iterations of a call from a CUDA graph (events cannot be replayed, so the headline region above,
-    # which carries them for the roofline, runs with direct launches)
+    # ---- the same steps once more without the events around the GEMM launches: the library then replays each
+    # repeated iteration of a call from ONE CUDA graph (the headline region above carries the events for the roofline,
+    # so there the iteration is replayed in pieces, with the dense products launched directly between their events)
     for _ in range(2):
         step_resident()
     ms_graph = timed(step_resident, args.steps)
@@ -632,8 +632,9 @@ def run_ours(args, cfg):
         "gpu_launches": int(launches),
         "graph_replay": {"value": whole_job_value(lcfg.n_iters, world, ms_graph / args.steps), "unit": UNIT,
                          "ms_per_step": ms_graph / args.steps,
-                         "note": "the same timed steps without events around the GEMM launches; armor_bcd_step then "
-                                 "replays iterations 2..n of a call from a CUDA graph"},
+                         "note": "the same timed steps without events around the GEMM launches: armor_bcd_step then "
+                                 "replays iterations 2..n of a call from one CUDA graph each (in the headline region "
+                                 "from graph pieces between the directly launched, event-bracketed GEMMs)"},
         "kernel_table": kernel_table,
         "tf32_mode": tf32_mode,
         "other_modes": other_modes,

@@ -293,9 +293,11 @@ armor_status armor_kernel_timing_enable(armor_ctx* ctx, int32_t level);
 /* armor_bcd_step replays the iterations of a call that enqueue identical launches (all but the first, and the
  * every-64th that re-evaluates the loss) from a CUDA graph, captured once per call on a stream of the context's
  * own and launched on the caller's stream; which iteration runs reaches the kernels through a device counter.
- * On by default; it is skipped when the caller's stream is itself being captured, when launch timing is on, for
- * calls of fewer than four iterations, and after any failure to capture (the call then continues with direct
- * launches).  Results are identical either way.  enable = 0 switches it off for the context.  (No counterpart
+ * On by default; it is skipped when the caller's stream is itself being captured, when every launch is being timed
+ * (armor_kernel_timing_enable level 2), for calls of fewer than four iterations, and after any failure to capture
+ * (the call then continues with direct launches).  While only the dense products are timed (level 1), the iteration
+ * is captured in pieces that end at each dense product with H; the replay alternates the pieces with those products,
+ * launched directly between their events.  Results are identical in every case.  enable = 0 switches it off for the context.  (No counterpart
  * in the paper.) */
 armor_status armor_use_graphs(armor_ctx* ctx, int32_t enable);
 armor_status armor_kernel_timing(armor_ctx* ctx, int32_t n_classes, int64_t* launches, double* total_ms,

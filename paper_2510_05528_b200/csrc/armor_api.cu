@@ -295,6 +295,7 @@ armor_status armor_create(armor_ctx** out, const armor_config* cfg, void* d_work
     return ARMOR_ERR_CUDA;
   }
   c->use_graphs = 1;
+  c->cap_split = 0; c->cap_n = 0; c->cap_failed = 0;
   c->cap_stream = nullptr;
   if (cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking) != cudaSuccess) c->cap_stream = nullptr;
   c->kg = cfg->mask_groups > 0 ? cfg->mask_groups : 1;
@@ -630,44 +631,64 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
   auto is_generic = [&](int it) { return it > 0 && t_first + it != 0 && (adam || it % LOSS_REFRESH != 0); };
   int n_generic = 0;
   for (int it = 0; it < n_iters; ++it) n_generic += is_generic(it) ? 1 : 0;
-  bool use_graph = c->use_graphs && c->cap_stream && c->timing_on == 0 && n_generic >= 3;
+  // With events around the dense products (timing level 1) the iteration is captured in pieces around them and the
+  // products themselves are launched directly; with every launch timed (level 2) nothing is captured.
+  bool use_graph = c->use_graphs && c->cap_stream && c->timing_on <= 1 && n_generic >= 3;
+  const bool split = c->timing_on == 1 && c->cfg.h_mode == ARMOR_H_FULL;
   if (use_graph) {
     cudaStreamCaptureStatus cst = cudaStreamCaptureStatusNone;
     if (cudaStreamIsCapturing(s, &cst) != cudaSuccess || cst != cudaStreamCaptureStatusNone) use_graph = false;
   }
-  cudaGraphExec_t exec = nullptr;
+  cudaGraphExec_t exec[ARMOR_MAX_PIECES] = {};
+  int n_pieces = 0;                 // graph pieces; piece k < n_pieces - 1 is followed by the remembered product k
   int64_t body_launches = 0;
   armor_status result = ARMOR_OK;
   for (int it = 0; it < n_iters && result == ARMOR_OK; ++it) {
     if (use_graph && is_generic(it)) {
-      if (!exec) {
+      if (n_pieces == 0) {
         const int64_t l0 = c->launches;
-        cudaGraph_t graph = nullptr;
         armor_status bst = ARMOR_ERR_CUDA;
+        c->cap_n = 0; c->cap_failed = 0;
+        for (int k = 0; k < ARMOR_MAX_PIECES; ++k) c->cap_graph[k] = nullptr;
         if (cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+          c->cap_split = split ? 1 : 0;
           bst = body(false, adam, false, c->cap_stream);
-          if (cudaStreamEndCapture(c->cap_stream, &graph) != cudaSuccess) bst = ARMOR_ERR_CUDA;
+          c->cap_split = 0;
+          if (cudaStreamEndCapture(c->cap_stream, &c->cap_graph[c->cap_n]) != cudaSuccess || c->cap_failed) bst = ARMOR_ERR_CUDA;
         }
-        if (bst == ARMOR_OK && c->host_err == ARMOR_OK && graph && cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess) {
+        bool ok = (bst == ARMOR_OK && c->host_err == ARMOR_OK);
+        for (int k = 0; ok && k <= c->cap_n; ++k)
+          ok = c->cap_graph[k] && cudaGraphInstantiate(&exec[k], c->cap_graph[k], 0) == cudaSuccess;
+        if (ok) {
+          n_pieces = c->cap_n + 1;
           body_launches = c->launches - l0;
         } else {
-          exec = nullptr;
+          for (int k = 0; k < ARMOR_MAX_PIECES; ++k)
+            if (exec[k]) { cudaGraphExecDestroy(exec[k]); exec[k] = nullptr; }
           use_graph = false;              // this call goes on with direct launches
           c->host_err = ARMOR_OK;
           (void)cudaGetLastError();
         }
-        if (graph) cudaGraphDestroy(graph);
+        for (int k = 0; k < ARMOR_MAX_PIECES; ++k)
+          if (c->cap_graph[k]) { cudaGraphDestroy(c->cap_graph[k]); c->cap_graph[k] = nullptr; }
         c->launches = l0;
       }
-      if (exec) {
-        if (cudaGraphLaunch(exec, s) != cudaSuccess) result = ARMOR_ERR_CUDA;
+      if (n_pieces > 0) {
+        for (int k = 0; k < n_pieces && result == ARMOR_OK; ++k) {
+          if (cudaGraphLaunch(exec[k], s) != cudaSuccess) result = ARMOR_ERR_CUDA;
+          if (k + 1 < n_pieces && result == ARMOR_OK) {
+            const armor_ctx::RmulCall& r = c->cap_call[k];
+            result = rmul_H(c, r.in, r.H, r.out, r.rows, r.d1, r.out1, r.d2, r.out2, s);
+          }
+        }
         c->launches += body_launches;
         continue;
       }
     }
     result = body(it == 0, adam || (it % LOSS_REFRESH == 0), t_first + it == 0, s);
   }
-  if (exec) cudaGraphExecDestroy(exec);   // a graph still executing is released when it has finished
+  for (int k = 0; k < ARMOR_MAX_PIECES; ++k)
+    if (exec[k]) cudaGraphExecDestroy(exec[k]);   // a graph still executing is released when it has finished
   if (result != ARMOR_OK) { c->host_err = ARMOR_OK; return result; }
   return finish_call(c);
 }

@@ -46,6 +46,8 @@ enum {
   ST_COUNT = 16
 };
 
+static const int ARMOR_MAX_PIECES = 16;   // graph pieces of one iteration when it is captured around its dense products
+
 // One selected group per (i, j) block of the sparse core (Algorithm 3).
 struct SelRec {
   int32_t valid;      // 0: nothing selected in this block
@@ -105,6 +107,15 @@ struct armor_ctx {
   int64_t* it_dev;    // iteration index inside the running armor_bcd_step call (advanced by the last kernel of an iteration)
   int use_graphs;     // 1: repeated iterations of a call are replayed from a CUDA graph
   cudaStream_t cap_stream;   // the context's own stream, used only to capture that graph
+  // Capture in pieces (while the dense products are being timed with events, which a graph cannot replay): every
+  // dense product with H closes the piece being captured, is remembered with its arguments and opens the next
+  // piece; the replay alternates graph pieces and directly launched products.
+  int cap_split;             // 1 while such a capture runs
+  int cap_n;                 // pieces closed so far (= products remembered)
+  int cap_failed;            // too many pieces or a failed capture call: the iteration is enqueued directly instead
+  cudaGraph_t cap_graph[ARMOR_MAX_PIECES];
+  struct RmulCall { const float* in; const float* H; float* out; int64_t rows; const float* d1; double* out1;
+                    const float* d2; double* out2; } cap_call[ARMOR_MAX_PIECES];
   int64_t launches;
   int device;           // the device that was current at armor_create; every call must be issued with it current
   int n_sm;             // its number of SMs

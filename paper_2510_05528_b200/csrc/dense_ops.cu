@@ -23,6 +23,18 @@ armor_status prepare_H(armor_ctx* c, const float* H, cudaStream_t s) {
 armor_status rmul_H(armor_ctx* c, const float* in, const float* H, float* out, int64_t rows, const float* d1,
                     double* out1, const float* d2, double* out2, cudaStream_t s) {
   const int64_t d_in = c->d_in;
+  if (c->cap_split && c->cfg.h_mode == ARMOR_H_FULL) {
+    // capture in pieces: close the piece, remember this product, open the next piece (s is the capturing stream)
+    if (c->cap_failed) return ARMOR_OK;
+    if (c->cap_n >= ARMOR_MAX_PIECES - 1 || cudaStreamEndCapture(s, &c->cap_graph[c->cap_n]) != cudaSuccess) {
+      c->cap_failed = 1;
+      return ARMOR_OK;
+    }
+    c->cap_call[c->cap_n] = {in, H, out, rows, d1, out1, d2, out2};
+    ++c->cap_n;
+    if (cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) != cudaSuccess) c->cap_failed = 1;
+    return ARMOR_OK;
+  }
   if (c->cfg.h_mode == ARMOR_H_DIAG) {
     launch_colscale(c, in, c->hdiag, out, rows, d_in, s);
   } else if (c->cfg.precision == ARMOR_PREC_SIMT) {

@@ -70,3 +70,35 @@ def test_a_captured_call_and_timing_fall_back_to_direct_launches():
     t = Bd.armor_kernel_timing(ctx2.ctx)
     assert np.array_equal(host(st2.S), ref)
     assert t["gemm"][0] >= 2 * 6 and t["block_product"][0] > 0 and t["cholesky"][0] == 2 * 6 + 1
+
+
+@pytest.mark.parametrize("mode", ["full-exact", "full-adam", "full-2-sweeps", "diag-exact"])
+def test_replay_in_pieces_around_timed_products_is_bit_identical(mode):
+    """With events around the dense products only, the iteration is replayed as graph pieces with the products launched
+    directly between them: same results as direct launches, and every product of every iteration is timed."""
+    cfg = MID
+    W = inputs.make_weight(cfg)
+    H32 = O.gram(inputs.make_activations(cfg)).astype(np.float32)
+    Hd, Wd = dev(H32), dev(W)
+    out = {}
+    for graphs in (False, True):
+        ctx = make(cfg, Bd.PREC_FP16X3, **MODES[mode])
+        Bd.armor_use_graphs(ctx.ctx, graphs)
+        Bd.armor_kernel_timing_enable(ctx.ctx, 1)
+        st = ctx.init(Wd, Hd)
+        n0 = ctx.launch_count()
+        stats_a = ctx.read_stats(ctx.bcd_step(st, Hd, 0, 9)).copy()
+        stats_b = ctx.read_stats(ctx.bcd_step(st, Hd, 9, 5)).copy()
+        torch.cuda.synchronize()
+        t = Bd.armor_kernel_timing(ctx.ctx)
+        out[graphs] = (host(st.A).copy(), host(st.B).copy(), host(st.S).copy(), host(st.M).copy(), stats_a, stats_b,
+                       ctx.launch_count() - n0, ctx.device_status()[:4], t["gemm"][0])
+    d, g = out[False], out[True]
+    for x, y in zip(d[:4], g[:4]):
+        assert np.array_equal(x, y)
+    for sa, sb in ((d[4], g[4]), (d[5], g[5])):
+        assert sa.tobytes() == sb.tobytes()
+    assert d[6] == g[6] and d[8] == g[8]
+    if MODES[mode]["h_mode"] == Bd.H_FULL:
+        assert g[8] >= 2 * 14
+    assert d[7] == g[7] == [0, 0, 0, 0]
