@@ -311,7 +311,9 @@ armor_status armor_kernel_timing(armor_ctx* ctx, int32_t n_classes, int64_t* lau
  * d_add (may be NULL; may equal d_out) are [rows, cols] fp32; d_in must not overlap d_out.  path 0: fp32
  * CUDA-core kernel; path 1: tensor-core kernel (tcgen05, operands split in shared memory into tf32 high and
  * low parts, three passes; needs d_block a multiple of 128 and a tensor-core precision, else UNSUPPORTED);
- * any other value: what the library itself would use.  Errors: INVALID_ARG, SHAPE (the blocked dimension is
+ * path 2: the same arithmetic with the wrapper block held in tensor memory as the M-side operand and two tiles per
+ * instruction (d_block = 128 only, else UNSUPPORTED; same bits as path 1);
+ * any other value: what the library itself would use (path 1 where it applies).  Errors: INVALID_ARG, SHAPE (the blocked dimension is
  * not a multiple of d_block, or cols is not a multiple of 4). */
 armor_status armor_block_product(armor_ctx* ctx, int32_t side, int32_t transpose, const float* d_blocks,
                                  const float* d_in, float* d_out, int64_t rows, int64_t cols, float alpha,

@@ -119,7 +119,9 @@ struct armor_ctx {
   int64_t launches;
   int device;           // the device that was current at armor_create; every call must be issued with it current
   int n_sm;             // its number of SMs
-  int tc_blocks;        // 1: block products and per-block Grams on the tensor cores where the shape allows;
+  int tc_blocks;        // 1, 2: block products and per-block Grams on the tensor cores where the shape allows
+                        // (2: with d_block = 128 the products keep the wrapper block in tensor memory; measured
+                        // equal to 1 at 4096 x 4096, so 1 is the default);
                         // 0: always the fp32 CUDA-core kernels (exact products with 0 and 1)
   armor_status host_err;   // first launch failure inside the running call that no fallback covers
   int kg;               // groups drawn per block in one sparse-core update (mask_groups, at least 1)
@@ -201,6 +203,13 @@ armor_status tc_bd_right(armor_ctx* c, const float* in, const float* Bblk, bool 
                          int64_t cols, float alpha, const float* add, float beta, cudaStream_t s);
 armor_status tc_bd_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, float* out, int64_t rows,
                         int64_t cols, float alpha, const float* add, float beta, cudaStream_t s);
+
+// the same with the wrapper block held in tensor memory (blockres_tcgen05.cu); d_block = 128
+bool tc_blockres_ok(const armor_ctx* c);
+armor_status tc_blockres_right(armor_ctx* c, const float* in, const float* Bblk, bool transB, float* out, int64_t rows,
+                               int64_t cols, float alpha, const float* add, float beta, cudaStream_t s);
+armor_status tc_blockres_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, float* out, int64_t rows,
+                              int64_t cols, float alpha, const float* add, float beta, cudaStream_t s);
 
 // per-block Grams over a long contraction on the tensor cores
 bool tc_gram_ok(const armor_ctx* c);

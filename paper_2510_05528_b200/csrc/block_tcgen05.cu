@@ -92,6 +92,16 @@ __device__ __forceinline__ uint64_t operand_desc(uint32_t base, int mn_major, in
   return mn_major ? smem_desc_mn_sw128_32b(base + kstep * 1024, 4096, 512) : smem_desc_sw128(base + kstep * 32, 16, 1024);
 }
 
+// tcgen05.mma with the accumulate flag set (the constant predicate costs no instruction)
+__device__ __forceinline__ void umma_tf32_acc(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, 1, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc)
+      : "memory");
+}
+
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                 const __grid_constant__ CUtensorMap mapC, const __grid_constant__ CUtensorMap mapD, const BParams p) {
@@ -163,6 +173,10 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc = instr_desc_tf32_mn(TILE, TILE, p.a.mn_major, p.b.mn_major);
+      const uint64_t da0 = operand_desc(smem_u32(smem), p.a.mn_major, 0);
+      const uint64_t db0 = operand_desc(smem_u32(smem) + 2 * OP_BYTES, p.b.mn_major, 0);
+      const uint64_t kinc_a = p.a.mn_major ? (1024u >> 4) : (32u >> 4);   // one k-step of 8 in the address field
+      const uint64_t kinc_b = p.b.mn_major ? (1024u >> 4) : (32u >> 4);
       int stage = 0; uint32_t phase = 0;
       int local = 0;
       bool ok = true;
@@ -175,18 +189,26 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         for (int kc = 0; kc < p.k_chunks; ++kc) {
           if (!mbar_wait(split0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
-          const uint32_t sa_lo = sa + OP_BYTES, sb = sa + 2 * OP_BYTES, sb_lo = sa + 3 * OP_BYTES;
+          // One thread issues every MMA, so the instructions around each tcgen05.mma bound the rate (a descriptor
+          // built from scratch per MMA costs more than the MMA takes to execute): the descriptors of stage 0 are
+          // formed once and only their address field moves.
+          const uint64_t so = (uint64_t)(uint32_t)(stage * (STAGE_BYTES >> 4));
+          const uint64_t da = da0 + so, dal = da + (OP_BYTES >> 4);
+          const uint64_t dbm = db0 + so, dbl = dbm + (OP_BYTES >> 4);
+          const uint32_t first = (uint32_t)(kc > 0);
+          if (p.one_pass) {
+            umma_tf32(tacc, da, dbm, idesc, first);
 #pragma unroll
-          for (int k = 0; k < BK / 8; ++k) {
-            const uint64_t da = operand_desc(sa, p.a.mn_major, k), dal = operand_desc(sa_lo, p.a.mn_major, k);
-            const uint64_t dbm = operand_desc(sb, p.b.mn_major, k), dbl = operand_desc(sb_lo, p.b.mn_major, k);
-            if (p.one_pass) {
-              umma_tf32(tacc, da, dbm, idesc, (uint32_t)((kc > 0) | (k != 0)));
-            } else {
-              umma_tf32(tacc, dal, dbm, idesc, (uint32_t)((kc > 0) | (k != 0)));
-              umma_tf32(tacc, da, dbl, idesc, 1);
-              umma_tf32(tacc, da, dbm, idesc, 1);
+            for (int k = 1; k < BK / 8; ++k) umma_tf32_acc(tacc, da + k * kinc_a, dbm + k * kinc_b, idesc);
+          } else {
+            umma_tf32(tacc, dal, dbm, idesc, first);
+            umma_tf32_acc(tacc, da, dbl, idesc);
+            umma_tf32_acc(tacc, da, dbm, idesc);
+#pragma unroll
+            for (int k = 1; k < BK / 8; ++k) {
+              umma_tf32_acc(tacc, dal + k * kinc_a, dbm + k * kinc_b, idesc);
+              umma_tf32_acc(tacc, da + k * kinc_a, dbl + k * kinc_b, idesc);
+              umma_tf32_acc(tacc, da + k * kinc_a, dbm + k * kinc_b, idesc);
             }
           }
           umma_commit(empty0 + 8 * stage);   // frees the stage once these MMAs have read it
@@ -349,6 +371,7 @@ bool tc_block_ok(const armor_ctx* c, int64_t rows, int64_t cols) {
 // out[:, j-th block] = alpha * in[:, j-th block] * Q_j (+ beta * add[:, j-th block]),  Q_j = Bblk[j] or its transpose
 armor_status tc_bd_right(armor_ctx* c, const float* in, const float* Bblk, bool transB, float* out, int64_t rows,
                          int64_t cols, float alpha, const float* add, float beta, cudaStream_t s) {
+  if (c->tc_blocks >= 2 && tc_blockres_ok(c)) return tc_blockres_right(c, in, Bblk, transB, out, rows, cols, alpha, add, beta, s);
   const int db = c->db;
   const int nb = (int)(cols / db);
   if (!ptr_ok(in) || !ptr_ok(Bblk) || !ptr_ok(out)) return ARMOR_ERR_UNSUPPORTED;
@@ -370,6 +393,7 @@ armor_status tc_bd_right(armor_ctx* c, const float* in, const float* Bblk, bool 
 // out[i-th block, :] = alpha * P_i * in[i-th block, :] (+ beta * add[i-th block, :]),  P_i = Ablk[i] or its transpose
 armor_status tc_bd_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, float* out, int64_t rows,
                         int64_t cols, float alpha, const float* add, float beta, cudaStream_t s) {
+  if (c->tc_blocks >= 2 && tc_blockres_ok(c)) return tc_blockres_left(c, Ablk, transA, in, out, rows, cols, alpha, add, beta, s);
   const int db = c->db;
   const int nb = (int)(rows / db);
   if (!ptr_ok(in) || !ptr_ok(Ablk) || !ptr_ok(out)) return ARMOR_ERR_UNSUPPORTED;

@@ -64,6 +64,17 @@ __device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t addr) {
   return d;
 }
 
+// tcgen05.mma with the accumulate flag set (the constant predicate costs no instruction)
+template <bool F16>
+__device__ __forceinline__ void umma_acc(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+  if (F16)
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 1, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc) : "memory");
+  else
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 1, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc) : "memory");
+}
+
 // fp32 accumulate, both operands K-major, M = 128, N = 256; operand format 0: fp16, 1: bf16 (both kind::f16),
 // 2: tf32 (kind::tf32).
 __device__ __forceinline__ uint32_t instr_desc(uint32_t fmt) {
@@ -249,6 +260,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc = instr_desc(H16 ? (p.f16 ? 0u : 1u) : 2u);
+      const uint64_t d0 = smem_desc_k_sw128(smem_u32(smem));
       int stage = 0; uint32_t phase = 0;
       int local = 0;   // (tile, K segment) items handled so far: selects the accumulator buffer
       bool ok = true;
@@ -265,29 +277,35 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
           for (int kt = kt0; kt < kt1; ++kt) {
             if (!mbar_wait(full0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
-            const uint32_t sa_lo = sa + A_BYTES;
-            const uint32_t sb = sa + (SPLIT ? 2 : 1) * A_BYTES;
-            const uint32_t sb_lo = sb + B_BYTES;
+            // One thread issues every MMA: the descriptors of stage 0 are formed once and only their address field
+            // moves, and every MMA but a tile's first carries a constant accumulate flag, so that the instructions
+            // around a tcgen05.mma stay well below the time it takes to execute.
+            const uint64_t da = d0 + (uint64_t)(uint32_t)(stage * (STAGE_BYTES >> 4));
+            const uint64_t dal = da + (A_BYTES >> 4);
+            const uint64_t dbm = da + (((SPLIT ? 2 : 1) * A_BYTES) >> 4);
+            const uint64_t dbl = dbm + (B_BYTES >> 4);
+            const uint32_t acc = (uint32_t)(kt > kt0);
+            if (PASSES == 3) {
+              umma_tf32(tacc, dal, dbm, idesc, acc);
+              umma_acc<false>(tacc, da, dbl, idesc);
+              umma_acc<false>(tacc, da, dbm, idesc);
+            } else if (PASSES == 6) {
+              umma_bf16(tacc, dal, dbm, idesc, acc);
+              umma_acc<true>(tacc, da, dbl, idesc);
+              umma_acc<true>(tacc, da, dbm, idesc);
+            } else if (PASSES == 0) {
+              umma_bf16(tacc, da, dbm, idesc, acc);
+            } else {
+              umma_tf32(tacc, da, dbm, idesc, acc);
+            }
 #pragma unroll
-            for (int k = 0; k < BK / 8; ++k) {
-              const uint64_t da = smem_desc_k_sw128(sa + k * 32), dbm = smem_desc_k_sw128(sb + k * 32);
-              const uint32_t acc = (uint32_t)((kt > kt0) | (k != 0));
-              if (PASSES == 3) {
-                const uint64_t dal = smem_desc_k_sw128(sa_lo + k * 32), dbl = smem_desc_k_sw128(sb_lo + k * 32);
-                umma_tf32(tacc, dal, dbm, idesc, acc);
-                umma_tf32(tacc, da, dbl, idesc, 1);
-                umma_tf32(tacc, da, dbm, idesc, 1);
-              } else if (PASSES == 6) {
-                const uint64_t dal = smem_desc_k_sw128(sa_lo + k * 32), dbl = smem_desc_k_sw128(sb_lo + k * 32);
-                umma_bf16(tacc, dal, dbm, idesc, acc);
-                umma_bf16(tacc, da, dbl, idesc, 1);
-                umma_bf16(tacc, da, dbm, idesc, 1);
-              } else if (PASSES == 0) {
-                umma_bf16(tacc, da, dbm, idesc, acc);
-              } else {
-                umma_tf32(tacc, da, dbm, idesc, acc);
+            for (int k = 1; k < BK / 8; ++k) {
+              const uint64_t ko = (uint64_t)(k * (32 >> 4));   // 8 fp32 (16 halves) of K: 32 bytes along the row
+              if (SPLIT) {
+                umma_acc<H16>(tacc, dal + ko, dbm + ko, idesc);
+                umma_acc<H16>(tacc, da + ko, dbl + ko, idesc);
               }
+              umma_acc<H16>(tacc, da + ko, dbm + ko, idesc);
             }
             umma_commit(empty0 + 8 * stage);   // frees the stage once these MMAs have read it
             if (++stage == STAGES) { stage = 0; phase ^= 1; }

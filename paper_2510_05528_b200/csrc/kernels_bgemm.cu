@@ -342,10 +342,11 @@ extern "C" armor_status armor_block_product(armor_ctx* c, int32_t side, int32_t 
   if (!c || !d_blocks || !d_in || !d_out || rows <= 0 || cols <= 0) return ARMOR_ERR_INVALID_ARG;
   if (side != 0 && side != 1) return ARMOR_ERR_INVALID_ARG;
   if (cols % 4 || (side == 0 ? cols : rows) % c->db) return ARMOR_ERR_SHAPE;
-  if (path == 1 && !tc_block_ok(c, rows, cols)) return ARMOR_ERR_UNSUPPORTED;
+  if ((path == 1 || path == 2) && !tc_block_ok(c, rows, cols)) return ARMOR_ERR_UNSUPPORTED;
+  if (path == 2 && !tc_blockres_ok(c)) return ARMOR_ERR_UNSUPPORTED;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   const int saved = c->tc_blocks;
-  c->tc_blocks = (path != 0);
+  c->tc_blocks = (path == 0 || path == 1 || path == 2) ? path : saved;
   if (side == 1) bd_left(c, d_blocks, transpose != 0, d_in, d_out, rows, cols, alpha, d_add, beta, s);
   else bd_right(c, d_in, d_blocks, transpose != 0, d_out, rows, cols, alpha, d_add, beta, s);
   c->tc_blocks = saved;

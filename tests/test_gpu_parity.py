@@ -668,13 +668,49 @@ def test_block_products_on_both_paths(db, side, transpose):
     Qe = np.ascontiguousarray(np.transpose(Q, (0, 2, 1))) if transpose else Q
     ref = O.bd_left(Qe, X) if side == 1 else O.bd_right(X, Qe)
     Qd, Xd = dev(Q), dev(X)
-    for path, tol in ((0, 2e-6), (1, 1e-5)):
+    for path, tol in ((0, 2e-6), (1, 1e-5)) + (((2, 1e-5),) if db == 128 else ()):
         out = torch.full((rows, cols), 7.0, device=DEV)
         Bd.armor_block_product(ctx.ctx, side, transpose, Qd, Xd, out, path=path)
         assert rel(host(out), ref) < tol
         out = dev(D)                                   # addend in place: out = 1.5 * product - 0.5 * out
         Bd.armor_block_product(ctx.ctx, side, transpose, Qd, Xd, out, alpha=1.5, add=out, beta=-0.5, path=path)
         assert rel(host(out), 1.5 * ref - 0.5 * D) < tol
+    if db != 128:
+        with pytest.raises(Bd.ArmorError):             # the wrapper-in-tensor-memory kernel is for d_block 128
+            Bd.armor_block_product(ctx.ctx, side, transpose, Qd, Xd, out, path=2)
+    assert ctx.device_status()[:4] == [0, 0, 0, 0]
+
+
+@pytest.mark.parametrize("many_blocks", [False, True], ids=["few-blocks", "many-blocks"])
+@pytest.mark.parametrize("side,transpose", [(0, False), (0, True), (1, False), (1, True)])
+def test_block_product_with_the_wrapper_in_tensor_memory(side, transpose, many_blocks):
+    """The kernel that keeps the wrapper block in tensor memory and takes two tiles per instruction.  Few blocks: several
+    CTAs share a wrapper block, each works through pairs of tiles and a single one; many blocks: contiguous ranges
+    of tiles, so that CTAs change their wrapper block on the way.  Ragged in the free dimension.  Same bits as the
+    streaming tensor-core kernel (the same MMAs in the same order), and the oracle's product within the fp32 bound."""
+    rng = np.random.default_rng(40 + 2 * side + int(transpose))
+    db = 128
+    if many_blocks:
+        rows, cols = (10240, 672) if side == 1 else (600, 10240)
+    else:
+        rows, cols = (1024, 8224) if side == 1 else (5000, 1280)
+    ctx = Bd.ArmorContext(1024, 1280, db, device=DEV, precision=Bd.PREC_FP16X3)
+    nb = (rows if side == 1 else cols) // db
+    Q = rng.standard_normal((nb, db, db)) * np.exp(rng.uniform(-3, 3, (nb, 1, 1)))
+    X = rng.standard_normal((rows, cols))
+    D = rng.standard_normal((rows, cols))
+    Qe = np.ascontiguousarray(np.transpose(Q, (0, 2, 1))) if transpose else Q
+    ref = O.bd_left(Qe, X) if side == 1 else O.bd_right(X, Qe)
+    Qd, Xd = dev(Q), dev(X)
+    outs = {}
+    for path in (1, 2):
+        a = torch.full((rows, cols), 7.0, device=DEV)
+        Bd.armor_block_product(ctx.ctx, side, transpose, Qd, Xd, a, path=path)
+        b = dev(D)
+        Bd.armor_block_product(ctx.ctx, side, transpose, Qd, Xd, b, alpha=-1.0, add=b, beta=1.0, path=path)
+        outs[path] = (host(a), host(b))
+    assert rel(outs[2][0], ref) < 1e-5 and rel(outs[2][1], D - ref) < 1e-5
+    assert np.array_equal(outs[1][0], outs[2][0]) and np.array_equal(outs[1][1], outs[2][1])
     assert ctx.device_status()[:4] == [0, 0, 0, 0]
 
 
