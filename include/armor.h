@@ -319,6 +319,17 @@ armor_status armor_block_product(armor_ctx* ctx, int32_t side, int32_t transpose
                                  const float* d_in, float* d_out, int64_t rows, int64_t cols, float alpha,
                                  const float* d_add, float beta, int32_t path, armor_stream_t stream);
 
+/* The pair of products behind the step length of a line search (Section 3.2: the exact step along a direction
+ * V needs tr(V H_w V^T) = <V H_w, V> with V = A R and V H_w = A (R H_w)):
+ *   d_out = Q d_in2 per block row (side 1 above, alpha 1, no addend) and *d_dot = <Q d_in1, Q d_in2>,
+ * Q = d_blocks [d_out / d_block, d_block, d_block]; d_in1, d_in2, d_out are [d_out, d_in] of the context (device
+ * fp32, d_out distinct from both inputs), d_dot one device double.  path 1: one fused tensor-core launch in which
+ * Q d_in1 only exists as an accumulator (needs d_block a multiple of 128 and a tensor-core precision, else
+ * UNSUPPORTED); path 0: two CUDA-core products and a dot product; any other value: what the library itself uses.
+ * The sum is formed in a fixed order (deterministic).  Exposed for tests and measurements. */
+armor_status armor_block_product_dual(armor_ctx* ctx, const float* d_blocks, const float* d_in1, const float* d_in2,
+                                      float* d_out, double* d_dot, int32_t path, armor_stream_t stream);
+
 /* The paper has no counterpart to this entry point; it exists for deployment reasons only.
  *
  * armor_normalize_noalloc computes the same row/column normalisation that armor_init applies when

@@ -29,7 +29,7 @@ EXPORTS = ["armor_workspace_bytes", "armor_create", "armor_destroy", "armor_gram
            "armor_packed_layer_bytes", "armor_pack_layer", "armor_apply_layer",
            "armor_get_device_status",
            "armor_status_string", "armor_launch_count", "armor_gemm_timing_enable", "armor_gemm_timing",
-           "armor_normalize_noalloc", "armor_block_product", "armor_selftest_wait_timeout", "armor_kernel_timing_enable", "armor_use_graphs",
+           "armor_normalize_noalloc", "armor_block_product", "armor_block_product_dual", "armor_selftest_wait_timeout", "armor_kernel_timing_enable", "armor_use_graphs",
            "armor_kernel_timing"]
 
 
@@ -84,6 +84,7 @@ def lib() -> C.CDLL:
         L.armor_launch_count.restype = i64
         L.armor_normalize_noalloc.argtypes = [vp, i64, i64, vp, vp, vp, vp]
         L.armor_block_product.argtypes = [vp, i32, i32, vp, vp, vp, i64, i64, C.c_float, vp, C.c_float, i32, vp]
+        L.armor_block_product_dual.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp]
         L.armor_gemm_timing_enable.argtypes = [vp, i32]
         L.armor_gemm_timing.argtypes = [vp, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.armor_kernel_timing_enable.argtypes = [vp, i32]
@@ -264,6 +265,16 @@ def armor_block_product(ctx, side: int, transpose: bool, blocks, x, out, alpha=1
     _check(lib().armor_block_product(ctx, int(side), int(bool(transpose)), _ptr(blocks, f, "blocks"), _ptr(x, f, "x"),
                                      _ptr(out, f, "out"), x.shape[0], x.shape[1], float(alpha), _ptr(add, f, "add"),
                                      float(beta), int(path), _stream()), "armor_block_product")
+
+
+def armor_block_product_dual(ctx, blocks, x1, x2, out, path=-1) -> float:
+    """out = Q . x2 per block row; returns <Q . x1, Q . x2> (see armor.h)."""
+    f = torch.float32
+    dot = torch.zeros(1, dtype=torch.float64, device=out.device)
+    _check(lib().armor_block_product_dual(ctx, _ptr(blocks, f, "blocks"), _ptr(x1, f, "x1"), _ptr(x2, f, "x2"),
+                                          _ptr(out, f, "out"), _ptr(dot, torch.float64, "dot"), int(path), _stream()),
+           "armor_block_product_dual")
+    return float(dot.item())
 
 
 def armor_gemm_timing_enable(ctx, enable: bool) -> None:

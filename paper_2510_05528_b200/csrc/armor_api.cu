@@ -540,11 +540,11 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       bd_right(c, S, c->Delta, false, c->Tmp, d_out, d_in, 1.f, nullptr, 0.f, s);    // R = S Delta
       st = rmul_H(c, c->Tmp, H, c->E, d_out, nullptr, nullptr, nullptr, nullptr, s); // R H_w
       if (st != ARMOR_OK) return st;
-      bd_left(c, A, false, c->Tmp, c->V, d_out, d_in, 1.f, nullptr, 0.f, s);         // V = A R
-      bd_left(c, A, false, c->E, c->VH, d_out, d_in, 1.f, nullptr, 0.f, s);          // V H_w = A (R H_w)
-      dot_partials(c, c->VH, c->V, c->wn, c->partials, s);                           // q = <V H_w, V>, summed by the stage
-      if (b_gd) launch_stage(c, is, 8, nullptr, 0, 0, s, c->partials, ARMOR_DOT_BLOCKS, SC_Q_B);
-      else launch_stage(c, is, 2, c->partblk, nbi, nbi, s, c->partials, ARMOR_DOT_BLOCKS, SC_Q_B);
+      // V H_w = A (R H_w) and q = <V H_w, V> with V = A R (summed by the stage; V itself is needed nowhere else)
+      int nq = 0;
+      bd_left_dual(c, A, c->Tmp, c->E, c->V, c->VH, d_out, d_in, c->partials, &nq, s);
+      if (b_gd) launch_stage(c, is, 8, nullptr, 0, 0, s, c->partials, nq, SC_Q_B);
+      else launch_stage(c, is, 2, c->partblk, nbi, nbi, s, c->partials, nq, SC_Q_B);
       launch_axpy_slot(c, B, c->Delta, (int64_t)nbi * db * db, SC_TAU_B, 1.f, s);    // B += tau Delta
       launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_B, -1.f, s);                   // EH -= tau V H_w
       if (carry_P) launch_axpy_slot(c, c->P, c->E, c->wn, SC_TAU_B, 1.f, s);         // P += tau R H_w
@@ -560,14 +560,14 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       bd_right(c, c->U, B, false, c->Tmp, d_out, d_in, 1.f, nullptr, 0.f, s);        // R = Gamma_M B
       st = rmul_H(c, c->Tmp, H, c->E, d_out, nullptr, nullptr, nullptr, nullptr, s); // R H_w
       if (st != ARMOR_OK) return st;
-      bd_left(c, A, false, c->Tmp, c->V, d_out, d_in, 1.f, nullptr, 0.f, s);         // V = A Gamma_M B
-      bd_left(c, A, false, c->E, c->VH, d_out, d_in, 1.f, nullptr, 0.f, s);          // V H_w = A (R H_w)
-      dot_partials(c, c->VH, c->V, c->wn, c->partials, s);                           // q = <V H_w, V>
+      // V H_w = A (R H_w) and q = <V H_w, V> with V = A Gamma_M B
+      int nq = 0;
+      bd_left_dual(c, A, c->Tmp, c->E, c->V, c->VH, d_out, d_in, c->partials, &nq, s);
       const bool beta_step = (c->cfg.s_step == ARMOR_S_BETA);
       if (beta_step) {
         // the paper's step size (Eq. lrWprime): |A^T A|_F and |B H_w B^T|_F  (these dot products reuse the
         // partial-sum buffer, so q is summed first)
-        reduce_partials_to(c, c->partials, ARMOR_DOT_BLOCKS, c->sc + SC_Q_S, s);
+        reduce_partials_to(c, c->partials, nq, c->sc + SC_Q_S, s);
         block_mm(c, A, true, A, false, c->G, nbo, s);
         dot_to_ptr(c, c->G, c->G, (int64_t)nbo * db * db, c->sc + SC_BETA_A, s);
         if (c->cfg.h_mode == ARMOR_H_FULL) {
@@ -580,7 +580,7 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
           dot_to_ptr(c, c->Kfull, c->Kfull, (int64_t)nbi * db * db, c->sc + SC_BETA_K, s);
         }
       }
-      launch_stage(c, is, beta_step ? 6 : 3, nullptr, 0, 0, s, beta_step ? nullptr : c->partials, ARMOR_DOT_BLOCKS, SC_Q_S,
+      launch_stage(c, is, beta_step ? 6 : 3, nullptr, 0, 0, s, beta_step ? nullptr : c->partials, nq, SC_Q_S,
                    nrm_part, ARMOR_DOT_BLOCKS, SC_NRM_S);
       launch_axpy_slot(c, S, c->U, c->wn, SC_TAU_S, 1.f, s);                         // S += tau Gamma_M
       launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_S, -1.f, s);                   // EH -= tau V H_w

@@ -19,6 +19,10 @@
 //   warps 2-5 : splitter     (raw chunk -> low part next to it, proxy fence)
 //   warps 6-9 : epilogue     (D tile prefetched by TMA into swizzled shared memory, tcgen05.ld, alpha / beta
 //                             in place, TMA store: no strided global access)
+// Dual mode: two inputs share the wrapper, A.X1 and A.X2 of a tile go through the pipeline back to back into
+// two accumulators, and the epilogue stores alpha * A.X2 only and writes partial sums of <A.X1, A.X2> (the
+// quadratic form of a line search needs the first product only inside that dot product, so it never
+// reaches HBM).
 // Every wait is bounded; a wait that runs out raises a status word and the CTA leaves through the common
 // exit that frees its tensor memory.
 #include "tc_common.cuh"
@@ -32,7 +36,7 @@ constexpr int NTHREADS = 320;
 constexpr int STAGES = 3;
 constexpr int OP_BYTES = TILE * BK * 4;           // 16 KiB: one operand chunk
 constexpr int STAGE_BYTES = 4 * OP_BYTES;         // A raw (= high part), A low part, B raw, B low part
-constexpr uint32_t TMEM_COLS = 256;               // two accumulators of 128 columns
+constexpr uint32_t TMEM_COLS = 512;               // four accumulators of 128 columns (two in use outside the dual mode)
 constexpr int EPI_BYTES = 32 * 64 * 4;            // per epilogue warp: 32 rows x 64 columns (half a tile row) as two swizzled boxes
 constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 4 * EPI_BYTES + 1024;
 
@@ -56,6 +60,8 @@ struct BParams {
   int32_t* status;
   int batch_fastest;                // 1: consecutive work items are consecutive batches (neighbouring column blocks)
   int one_pass;                     // 1: operands as they are, rounded to tf32 by the tensor core; no low parts
+  int dual;                         // 1: two B operands per tile (mapB, mapB2); C = alpha * A.B2, dot_part = <A.B1, A.B2>
+  double* dot_part;                 // dual: 4 partial sums per tile (one per epilogue warp), in tile order
 };
 
 __device__ __forceinline__ void load_operand(uint32_t dst, const CUtensorMap* map, const OpCoord& o, int b, int t, int kc,
@@ -104,18 +110,21 @@ __device__ __forceinline__ void umma_tf32_acc(uint32_t tmem_d, uint64_t adesc, u
 
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
-                const __grid_constant__ CUtensorMap mapC, const __grid_constant__ CUtensorMap mapD, const BParams p) {
+                const __grid_constant__ CUtensorMap mapB2, const __grid_constant__ CUtensorMap mapC,
+                const __grid_constant__ CUtensorMap mapD, const BParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  __shared__ __align__(8) uint64_t bars[3 * STAGES + 8];
+  __shared__ __align__(8) uint64_t bars[3 * STAGES + 12];
   __shared__ uint32_t tmem_base_holder;
   __shared__ int abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t full0 = smem_u32(&bars[0]), split0 = smem_u32(&bars[STAGES]), empty0 = smem_u32(&bars[2 * STAGES]);
-  const uint32_t tfull0 = smem_u32(&bars[3 * STAGES]), tempty0 = smem_u32(&bars[3 * STAGES + 2]);
-  const uint32_t dfull0 = smem_u32(&bars[3 * STAGES + 4]);
-  const int n_items = p.batch * p.m_tiles * p.n_tiles * p.n_split;
+  const uint32_t tfull0 = smem_u32(&bars[3 * STAGES]), tempty0 = smem_u32(&bars[3 * STAGES + 4]);
+  const uint32_t dfull0 = smem_u32(&bars[3 * STAGES + 8]);
+  const int n_items = p.batch * p.m_tiles * p.n_tiles * p.n_split;   // tiles (x slabs of the contraction)
+  const int n_sub = p.dual ? 2 : 1;                                  // passes through the pipeline per tile
+  const int acc_mask = p.dual ? 3 : 1, acc_shift = p.dual ? 2 : 1;   // accumulators in rotation
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -124,7 +133,7 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       mbar_init(split0 + 8 * s, 4);
       mbar_init(empty0 + 8 * s, 1);
     }
-    for (int s = 0; s < 2; ++s) { mbar_init(tfull0 + 8 * s, 1); mbar_init(tempty0 + 8 * s, 4); }
+    for (int s = 0; s < 4; ++s) { mbar_init(tfull0 + 8 * s, 1); mbar_init(tempty0 + 8 * s, 4); }
     for (int s = 0; s < 4; ++s) mbar_init(dfull0 + 8 * s, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -148,13 +157,14 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
         int tn, tm, b, ks;
         item_decode(p, item, tn, tm, b, ks);
+        for (int sub = 0; sub < n_sub && ok; ++sub)
         for (int kc = 0; kc < p.k_chunks; ++kc) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abortp, p.status)) { ok = false; break; }
           const uint32_t fb = full0 + 8 * stage;
           mbar_expect_tx(fb, 2 * OP_BYTES);
           const uint32_t dst = smem_u32(smem + (size_t)stage * STAGE_BYTES);
           load_operand(dst, &mapA, p.a, b, tm, ks * p.k_chunks + kc, fb);
-          load_operand(dst + 2 * OP_BYTES, &mapB, p.b, b, tn, ks * p.k_chunks + kc, fb);
+          load_operand(dst + 2 * OP_BYTES, sub ? &mapB2 : &mapB, p.b, b, tn, ks * p.k_chunks + kc, fb);
           ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -180,9 +190,10 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       int stage = 0; uint32_t phase = 0;
       int local = 0;
       bool ok = true;
-      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++local) {
-        const int as = local & 1;
-        const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x)
+      for (int sub = 0; sub < n_sub && ok; ++sub, ++local) {
+        const int as = local & acc_mask;
+        const uint32_t aphase = (uint32_t)(local >> acc_shift) & 1u;
         if (!mbar_wait(tempty0 + 8 * as, aphase ^ 1, abortp, p.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tacc = tmem_base + (uint32_t)(as * TILE);
@@ -223,7 +234,7 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     int stage = 0; uint32_t phase = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-      for (int kc = 0; kc < p.k_chunks; ++kc) {
+      for (int kc = 0; kc < n_sub * p.k_chunks; ++kc) {
         if (!mbar_wait(full0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
         float4* base = reinterpret_cast<float4*>(smem + (size_t)stage * STAGE_BYTES);
 #pragma unroll
@@ -261,10 +272,61 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++local) {
       int tn, tm, b, ks;
       item_decode(p, item, tn, tm, b, ks);
-      const int as = local & 1;
+      const int as = p.dual ? ((2 * local) & 3) : (local & 1);          // dual: accumulators as (A.B1) and as + 1 (A.B2)
       const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
       const int64_t row_base = p.r_b * b + p.r_s * ks + (int64_t)tm * TILE + q * 32;
       const int64_t col_tile = p.c_b * b + (int64_t)tn * TILE;
+      if (p.dual) {
+        // C = alpha * (A.B2); partial sum of <A.B1, A.B2> over this warp's 32 x 128 slab (rows or columns past the
+        // end of the operands were read as zeros and add nothing)
+        double dot = 0.0;
+#pragma unroll 1
+        for (int hf = 0; hf < 2 && ok; ++hf) {
+          int n_box = 0;
+          if (row_base < p.c_rows && tm * TILE + q * 32 < p.m_valid)
+            for (int ch = 0; ch < 2; ++ch) n_box += (col_tile + 64 * hf + 32 * ch < p.c_cols) ? 1 : 0;
+          if (lane == 0) tma_store_wait_read();       // the previous stores have read the staging boxes
+          __syncwarp();
+          if (hf == 0) {
+            if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
+            if (!mbar_wait(tfull0 + 8 * (as + 1), aphase, abortp, p.status)) { ok = false; break; }
+            tc_fence_after();
+          }
+#pragma unroll 1
+          for (int ch = 0; ch < 2; ++ch) {
+            uint32_t r1[32], r2[32];
+            const uint32_t col = (uint32_t)(hf * 64 + ch * 32) + ((uint32_t)(q * 32) << 16);
+            tmem_ld32(tmem_base + (uint32_t)(as * TILE) + col, r1);
+            tmem_ld32(tmem_base + (uint32_t)((as + 1) * TILE) + col, r2);
+            float part = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) part = fmaf(__uint_as_float(r1[i]), __uint_as_float(r2[i]), part);
+            dot += (double)part;
+            if (ch >= n_box) continue;                // warp-uniform
+            uint8_t* rowp = buf + ch * 4096 + lane * 128;
+#pragma unroll
+            for (int cq = 0; cq < 8; ++cq) {
+              float4* cell = reinterpret_cast<float4*>(rowp + ((cq ^ (lane & 7)) << 4));
+              *cell = make_float4(p.alpha * __uint_as_float(r2[4 * cq]), p.alpha * __uint_as_float(r2[4 * cq + 1]),
+                                  p.alpha * __uint_as_float(r2[4 * cq + 2]), p.alpha * __uint_as_float(r2[4 * cq + 3]));
+            }
+          }
+          if (hf == 1) tc_fence_before();             // all reads of the accumulators are done
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            if (hf == 1) { mbar_arrive(tempty0 + 8 * as); mbar_arrive(tempty0 + 8 * (as + 1)); }
+            for (int ch = 0; ch < n_box; ++ch)
+              tma_store_2d(&mapC, (int)(col_tile + 64 * hf + 32 * ch), (int)row_base, buf_u32 + ch * 4096);
+            tma_store_commit();
+          }
+        }
+        // lanes in a fixed order
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        if (ok && lane == 0) p.dot_part[(size_t)item * 4 + q] = dot;
+        continue;
+      }
       // The warp's 32 x 128 slab goes through shared memory in two halves of 64 columns (two 32 x 32 boxes).
       bool waited = false;
 #pragma unroll 1
@@ -337,8 +399,9 @@ struct HostOp {
   OpCoord c;
 };
 
-armor_status launch(armor_ctx* c, const HostOp& A, const HostOp& B, BParams p, int kclass, double kbytes, cudaStream_t s) {
-  CUtensorMap mA, mB, mC, mD;
+armor_status launch(armor_ctx* c, const HostOp& A, const HostOp& B, BParams p, int kclass, double kbytes, cudaStream_t s,
+                    const float* B2 = nullptr) {
+  CUtensorMap mA, mB, mB2, mC, mD;
   if (!make_map_2d(&mC, p.C, p.c_cols, p.c_rows, p.ldc, 32, 32)) return ARMOR_ERR_CUDA;
   if (p.D) {
     if (!make_map_2d(&mD, p.D, p.c_cols, p.c_rows, p.ldd, 32, 32)) return ARMOR_ERR_CUDA;
@@ -347,6 +410,11 @@ armor_status launch(armor_ctx* c, const HostOp& A, const HostOp& B, BParams p, i
   }
   if (!make_map_2d(&mA, A.base, A.inner, A.outer, A.ld, 32, A.c.mn_major ? 32 : TILE, A.c.mn_major != 0)) return ARMOR_ERR_CUDA;
   if (!make_map_2d(&mB, B.base, B.inner, B.outer, B.ld, 32, B.c.mn_major ? 32 : TILE, B.c.mn_major != 0)) return ARMOR_ERR_CUDA;
+  if (B2) {
+    if (!make_map_2d(&mB2, B2, B.inner, B.outer, B.ld, 32, B.c.mn_major ? 32 : TILE, B.c.mn_major != 0)) return ARMOR_ERR_CUDA;
+  } else {
+    mB2 = mB;
+  }
   p.a = A.c; p.b = B.c;
   p.status = c->status;
   static PerDeviceOnce attr;
@@ -355,7 +423,7 @@ armor_status launch(armor_ctx* c, const HostOp& A, const HostOp& B, BParams p, i
   const int n_items = p.batch * p.m_tiles * p.n_tiles * p.n_split;
   const int grid = n_items < n_sm ? n_items : n_sm;
   KTimer kt(c, kclass, kbytes, s);
-  tc_block_kernel<<<grid, NTHREADS, SMEM_BYTES, s>>>(mA, mB, mC, mD, p);
+  tc_block_kernel<<<grid, NTHREADS, SMEM_BYTES, s>>>(mA, mB, mB2, mC, mD, p);
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
 }
@@ -409,6 +477,30 @@ armor_status tc_bd_left(armor_ctx* c, const float* Ablk, bool transA, const floa
   p.n_split = 1; p.r_s = 0; p.m_valid = 1 << 30;
   p.one_pass = c->block_one_pass;
   return launch(c, A, B, p, ARMOR_KC_BLOCK_PRODUCT, (add ? 12.0 : 8.0) * (double)rows * (double)cols, s);
+}
+
+// out[i-th block, :] = P_i * in2[i-th block, :] and 4 partial sums per 128 x 128 tile of <P_i * in1, P_i * in2> at part
+// (tile order, then the four 32-row slabs of the tile); returns the number of partial sums through n_part
+armor_status tc_bd_left_dual(armor_ctx* c, const float* Ablk, bool transA, const float* in1, const float* in2, float* out,
+                             int64_t rows, int64_t cols, double* part, int* n_part, cudaStream_t s) {
+  const int db = c->db;
+  const int nb = (int)(rows / db);
+  if (!ptr_ok(in1) || !ptr_ok(in2) || !ptr_ok(Ablk) || !ptr_ok(out)) return ARMOR_ERR_UNSUPPORTED;
+  HostOp A{Ablk, db, (int64_t)nb * db, db, {}};
+  if (transA) A.c = {1, 0, TILE, 0, db, 0, BK};
+  else        A.c = {0, 0, 0, BK, db, TILE, 0};
+  HostOp B{in1, cols, rows, cols, {1, 0, TILE, 0, db, 0, BK}};
+  BParams p{};
+  p.C = out; p.D = nullptr; p.ldc = cols; p.ldd = cols; p.c_rows = rows; p.c_cols = cols;
+  p.r_b = db; p.c_b = 0;
+  p.m_tiles = db / TILE; p.n_tiles = (int)((cols + TILE - 1) / TILE); p.batch = nb; p.k_chunks = db / BK;
+  p.alpha = 1.f; p.beta = 0.f;
+  p.n_split = 1; p.r_s = 0; p.m_valid = 1 << 30;
+  p.one_pass = c->block_one_pass;
+  p.dual = 1; p.dot_part = part;
+  *n_part = 4 * p.batch * p.m_tiles * p.n_tiles;
+  // two W-shaped reads, one W-shaped write
+  return launch(c, A, B, p, ARMOR_KC_BLOCK_PRODUCT, 12.0 * (double)rows * (double)cols, s, in2);
 }
 
 namespace {

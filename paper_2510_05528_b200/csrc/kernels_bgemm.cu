@@ -336,6 +336,32 @@ void bd_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, floa
   launch_bgemm(c, g, s);
 }
 
+void bd_left_dual(armor_ctx* c, const float* Ablk, const float* in1, const float* in2, float* tmp, float* out,
+                  int64_t rows, int64_t cols, double* part, int* n_part, cudaStream_t s) {
+  if (c->tc_blocks && tc_block_ok(c, rows, cols) &&
+      tc_done(c, tc_bd_left_dual(c, Ablk, false, in1, in2, out, rows, cols, part, n_part, s)))
+    return;
+  bd_left(c, Ablk, false, in1, tmp, rows, cols, 1.f, nullptr, 0.f, s);
+  bd_left(c, Ablk, false, in2, out, rows, cols, 1.f, nullptr, 0.f, s);
+  dot_partials(c, out, tmp, rows * cols, part, s);
+  *n_part = ARMOR_DOT_BLOCKS;
+}
+
+extern "C" armor_status armor_block_product_dual(armor_ctx* c, const float* d_blocks, const float* d_in1,
+                                                 const float* d_in2, float* d_out, double* d_dot, int32_t path,
+                                                 armor_stream_t stream) {
+  if (!c || !d_blocks || !d_in1 || !d_in2 || !d_out || !d_dot) return ARMOR_ERR_INVALID_ARG;
+  if (path == 1 && !tc_block_ok(c, c->d_out, c->d_in)) return ARMOR_ERR_UNSUPPORTED;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  const int saved = c->tc_blocks;
+  c->tc_blocks = (path == 0 || path == 1) ? path : saved;
+  int nq = 0;
+  bd_left_dual(c, d_blocks, d_in1, d_in2, c->V, d_out, c->d_out, c->d_in, c->partials, &nq, s);
+  reduce_partials_to(c, c->partials, nq, d_dot, s);
+  c->tc_blocks = saved;
+  return finish_call(c);
+}
+
 extern "C" armor_status armor_block_product(armor_ctx* c, int32_t side, int32_t transpose, const float* d_blocks,
                                             const float* d_in, float* d_out, int64_t rows, int64_t cols, float alpha,
                                             const float* d_add, float beta, int32_t path, armor_stream_t stream) {

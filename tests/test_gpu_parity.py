@@ -714,6 +714,30 @@ def test_block_product_with_the_wrapper_in_tensor_memory(side, transpose, many_b
     assert ctx.device_status()[:4] == [0, 0, 0, 0]
 
 
+@pytest.mark.parametrize("db,shape", [(128, (1024, 1536)), (256, (512, 768)), (128, (4096, 4096))],
+                         ids=["128", "256", "4096"])
+def test_dual_block_product(db, shape):
+    """out = Q x2 and <Q x1, Q x2> in one launch (the first product exists as an accumulator only), against the oracle's
+    products and a float64 dot product; the CUDA-core path (two products and a dot) likewise."""
+    rng = np.random.default_rng(db + shape[1])
+    rows, cols = shape
+    ctx = Bd.ArmorContext(rows, cols, db, device=DEV, precision=Bd.PREC_FP16X3)
+    Q = rng.standard_normal((rows // db, db, db)) / np.sqrt(db)
+    X1 = rng.standard_normal((rows, cols))
+    X2 = X1 * 0.5 + rng.standard_normal((rows, cols))          # correlated: the dot product is far from zero
+    V1, V2 = O.bd_left(Q, X1), O.bd_left(Q, X2)
+    ref = float(np.sum(V1 * V2))
+    Qd, X1d, X2d = dev(Q), dev(X1), dev(X2)
+    for path, tol in ((0, 2e-6), (1, 1e-5)):
+        out = torch.full((rows, cols), 7.0, device=DEV)
+        dot = Bd.armor_block_product_dual(ctx.ctx, Qd, X1d, X2d, out, path=path)
+        assert rel(host(out), V2) < tol
+        assert abs(dot - ref) < 2e-6 * float(np.sqrt(np.sum(V1 * V1) * np.sum(V2 * V2)))
+        again = Bd.armor_block_product_dual(ctx.ctx, Qd, X1d, X2d, out, path=path)
+        assert again == dot                                    # fixed order of the partial sums
+    assert ctx.device_status()[:4] == [0, 0, 0, 0]
+
+
 # ------------------------------------------------------------------ the guard's rejection (full weighting)
 def overlapping_case(d_out, d_in, db, strength, n=4, seed=5):
     """Four calibration tokens and wrapper blocks with nearly parallel columns: the group updates of one
