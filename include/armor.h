@@ -325,7 +325,9 @@ armor_status armor_block_product(armor_ctx* ctx, int32_t side, int32_t transpose
  * Q = d_blocks [d_out / d_block, d_block, d_block]; d_in1, d_in2, d_out are [d_out, d_in] of the context (device
  * fp32, d_out distinct from both inputs), d_dot one device double.  path 1: one fused tensor-core launch in which
  * Q d_in1 only exists as an accumulator (needs d_block a multiple of 128 and a tensor-core precision, else
- * UNSUPPORTED); path 0: two CUDA-core products and a dot product; any other value: what the library itself uses.
+ * UNSUPPORTED); path 2: the same with Q in tensor memory and both inputs of a tile in one instruction (d_block = 128
+ * only); path 0: two CUDA-core products and a dot product; any other value: what the library itself uses (path 2
+ * where it applies, else path 1).
  * The sum is formed in a fixed order (deterministic).  Exposed for tests and measurements. */
 armor_status armor_block_product_dual(armor_ctx* ctx, const float* d_blocks, const float* d_in1, const float* d_in2,
                                       float* d_out, double* d_dot, int32_t path, armor_stream_t stream);

@@ -287,7 +287,7 @@ armor_status armor_create(armor_ctx** out, const armor_config* cfg, void* d_work
   c->db = cfg->d_block; c->nbo = (int)(cfg->d_out / cfg->d_block); c->nbi = (int)(cfg->d_in / cfg->d_block);
   c->ws = static_cast<char*>(d_workspace); c->ws_bytes = bytes;
   c->launches = 0;
-  c->tc_blocks = 1;
+  c->tc_blocks = 3;
   c->host_err = ARMOR_OK;
   if (cudaGetDevice(&c->device) != cudaSuccess ||
       cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess || c->n_sm < 1) {

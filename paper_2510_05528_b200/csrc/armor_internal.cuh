@@ -119,9 +119,11 @@ struct armor_ctx {
   int64_t launches;
   int device;           // the device that was current at armor_create; every call must be issued with it current
   int n_sm;             // its number of SMs
-  int tc_blocks;        // 1, 2: block products and per-block Grams on the tensor cores where the shape allows
-                        // (2: with d_block = 128 the products keep the wrapper block in tensor memory; measured
-                        // equal to 1 at 4096 x 4096, so 1 is the default);
+  int tc_blocks;        // 1, 2, 3: block products and per-block Grams on the tensor cores where the shape allows.
+                        // 1: the streaming kernel for every product; 2: with d_block = 128 the kernel that keeps the
+                        // wrapper block in tensor memory for every product; 3 (default): that kernel for the dual
+                        // product, where it halves the shared-memory traffic, and the streaming kernel elsewhere
+                        // (the two measure equal on single products at 4096 x 4096);
                         // 0: always the fp32 CUDA-core kernels (exact products with 0 and 1)
   armor_status host_err;   // first launch failure inside the running call that no fallback covers
   int kg;               // groups drawn per block in one sparse-core update (mask_groups, at least 1)
@@ -218,6 +220,9 @@ armor_status tc_blockres_right(armor_ctx* c, const float* in, const float* Bblk,
                                int64_t cols, float alpha, const float* add, float beta, cudaStream_t s);
 armor_status tc_blockres_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, float* out, int64_t rows,
                               int64_t cols, float alpha, const float* add, float beta, cudaStream_t s);
+
+armor_status tc_blockres_left_dual(armor_ctx* c, const float* Ablk, const float* in1, const float* in2, float* out,
+                                   int64_t rows, int64_t cols, double* part, int* n_part, cudaStream_t s);
 
 // per-block Grams over a long contraction on the tensor cores
 bool tc_gram_ok(const armor_ctx* c);

@@ -439,7 +439,7 @@ bool tc_block_ok(const armor_ctx* c, int64_t rows, int64_t cols) {
 // out[:, j-th block] = alpha * in[:, j-th block] * Q_j (+ beta * add[:, j-th block]),  Q_j = Bblk[j] or its transpose
 armor_status tc_bd_right(armor_ctx* c, const float* in, const float* Bblk, bool transB, float* out, int64_t rows,
                          int64_t cols, float alpha, const float* add, float beta, cudaStream_t s) {
-  if (c->tc_blocks >= 2 && tc_blockres_ok(c)) return tc_blockres_right(c, in, Bblk, transB, out, rows, cols, alpha, add, beta, s);
+  if (c->tc_blocks == 2 && tc_blockres_ok(c)) return tc_blockres_right(c, in, Bblk, transB, out, rows, cols, alpha, add, beta, s);
   const int db = c->db;
   const int nb = (int)(cols / db);
   if (!ptr_ok(in) || !ptr_ok(Bblk) || !ptr_ok(out)) return ARMOR_ERR_UNSUPPORTED;
@@ -461,7 +461,7 @@ armor_status tc_bd_right(armor_ctx* c, const float* in, const float* Bblk, bool 
 // out[i-th block, :] = alpha * P_i * in[i-th block, :] (+ beta * add[i-th block, :]),  P_i = Ablk[i] or its transpose
 armor_status tc_bd_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, float* out, int64_t rows,
                         int64_t cols, float alpha, const float* add, float beta, cudaStream_t s) {
-  if (c->tc_blocks >= 2 && tc_blockres_ok(c)) return tc_blockres_left(c, Ablk, transA, in, out, rows, cols, alpha, add, beta, s);
+  if (c->tc_blocks == 2 && tc_blockres_ok(c)) return tc_blockres_left(c, Ablk, transA, in, out, rows, cols, alpha, add, beta, s);
   const int db = c->db;
   const int nb = (int)(rows / db);
   if (!ptr_ok(in) || !ptr_ok(Ablk) || !ptr_ok(out)) return ARMOR_ERR_UNSUPPORTED;
@@ -483,6 +483,10 @@ armor_status tc_bd_left(armor_ctx* c, const float* Ablk, bool transA, const floa
 // (tile order, then the four 32-row slabs of the tile); returns the number of partial sums through n_part
 armor_status tc_bd_left_dual(armor_ctx* c, const float* Ablk, bool transA, const float* in1, const float* in2, float* out,
                              int64_t rows, int64_t cols, double* part, int* n_part, cudaStream_t s) {
+  // with d_block = 128 the kernel that keeps the wrapper block in tensor memory takes both inputs of a tile in one
+  // instruction (half the shared-memory traffic of two passes through the streaming kernel)
+  if (c->tc_blocks != 1 && !transA && tc_blockres_ok(c))
+    return tc_blockres_left_dual(c, Ablk, in1, in2, out, rows, cols, part, n_part, s);
   const int db = c->db;
   const int nb = (int)(rows / db);
   if (!ptr_ok(in1) || !ptr_ok(in2) || !ptr_ok(Ablk) || !ptr_ok(out)) return ARMOR_ERR_UNSUPPORTED;

@@ -67,16 +67,19 @@ struct RParams {
   float alpha, beta;
   int32_t* status;
   int one_pass;
+  int dual;                         // 1 (left only): the two halves of an instruction are the same tile of two inputs
+                                    // (mapX, mapX2); out = alpha * Q.X2, dot_part = <Q.X1, Q.X2>
+  double* dot_part;                 // dual: 8 partial sums per tile (one per epilogue warp), in tile order
 };
 
 // One or two neighbouring tiles of one wrapper block.
 struct Unit { int b, t, nt; };
-__device__ __forceinline__ bool next_unit(int& item, int i1, int tiles, Unit& u) {
+__device__ __forceinline__ bool next_unit(int& item, int i1, int tiles, int dual, Unit& u) {
   if (item >= i1) return false;
   u.b = item / tiles;
   u.t = item - u.b * tiles;
-  u.nt = (u.t + 1 < tiles && item + 1 < i1) ? 2 : 1;
-  item += u.nt;
+  u.nt = (dual || (u.t + 1 < tiles && item + 1 < i1)) ? 2 : 1;
+  item += dual ? 1 : u.nt;
   return true;
 }
 
@@ -116,7 +119,8 @@ __device__ __forceinline__ uint64_t x_desc(uint32_t base, int mn_major, int kste
 }
 
 __global__ void __launch_bounds__(NTHREADS, 1)
-tc_blockres_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapQ,
+tc_blockres_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapX2,
+                   const __grid_constant__ CUtensorMap mapQ,
                    const __grid_constant__ CUtensorMap mapC, const __grid_constant__ CUtensorMap mapD, const RParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -169,7 +173,7 @@ tc_blockres_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
       bool ok = true;
       int cur_b = -1;
       Unit u;
-      for (int item = i0; ok && next_unit(item, i1, p.tiles, u);) {
+      for (int item = i0; ok && next_unit(item, i1, p.tiles, p.dual, u);) {
         if (u.b != cur_b) {
           // the wrapper block: two pieces of 64 columns, each two boxes of 128 rows x 32 columns
           for (int piece = 0; piece < 2; ++piece) {
@@ -191,13 +195,15 @@ tc_blockres_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
           mbar_expect_tx(fb, (uint32_t)(u.nt * OP_BYTES));
           const uint32_t dst = smem_u32(smem + (size_t)stage * STAGE_BYTES);
           for (int j = 0; j < u.nt; ++j) {
-            const int x = p.x.x_b * u.b + p.x.x_t * (u.t + j) + p.x.x_k * kc;
-            const int y = p.x.y_b * u.b + p.x.y_t * (u.t + j) + p.x.y_k * kc;
+            const int tj = p.dual ? u.t : u.t + j;                      // dual: the same tile of the second input
+            const CUtensorMap* mx = (p.dual && j) ? &mapX2 : &mapX;
+            const int x = p.x.x_b * u.b + p.x.x_t * tj + p.x.x_k * kc;
+            const int y = p.x.y_b * u.b + p.x.y_t * tj + p.x.y_k * kc;
             if (p.x.mn_major) {
 #pragma unroll
-              for (int q = 0; q < 4; ++q) tma_load_2d(dst + (j * 4 + q) * 4096, &mapX, x + 32 * q, y, fb);
+              for (int q = 0; q < 4; ++q) tma_load_2d(dst + (j * 4 + q) * 4096, mx, x + 32 * q, y, fb);
             } else {
-              tma_load_2d(dst + j * OP_BYTES, &mapX, x, y, fb);
+              tma_load_2d(dst + j * OP_BYTES, mx, x, y, fb);
             }
           }
           ++issued;
@@ -228,7 +234,7 @@ tc_blockres_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
       uint32_t local = 0, w_loads = 0;          // units issued, wrapper blocks waited for
       bool ok = true;
       Unit u;
-      for (int item = i0; ok && next_unit(item, i1, p.tiles, u); ++local) {
+      for (int item = i0; ok && next_unit(item, i1, p.tiles, p.dual, u); ++local) {
         if (u.b != cur_b) {
           if (!mbar_wait(wfull, w_loads & 1u, abortp, p.status)) { ok = false; break; }
           ++w_loads;
@@ -298,7 +304,7 @@ tc_blockres_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
     uint32_t w_loads = 0;
     bool ok = true;
     Unit u;
-    for (int item = i0; ok && next_unit(item, i1, p.tiles, u);) {
+    for (int item = i0; ok && next_unit(item, i1, p.tiles, p.dual, u);) {
       if (u.b != cur_b) {
         // The block arrives as two pieces, each a stage holding two boxes of 128 rows x 32 columns (rows of 128
         // bytes, 128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r % 8)); box g of the block covers
@@ -408,7 +414,52 @@ tc_blockres_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
     const uint32_t buf_u32 = smem_u32(buf);
     const uint32_t dbar = dfull0 + 8 * e;
     Unit u;
-    for (int item = i0; ok && next_unit(item, i1, p.tiles, u); ++local) {
+    for (int item = i0; ok && next_unit(item, i1, p.tiles, p.dual, u); ++local) {
+      if (p.dual) {
+        // Accumulator columns 0..127 hold Q.X1 and 128..255 hold Q.X2 of the same tile.  Warp (q, h) takes rows
+        // 32 q .. and columns 64 h .. of the tile: both products of its two boxes, their dot product, and the store
+        // of alpha * Q.X2.
+        const int64_t row0 = (int64_t)TILE * u.b + 32 * q, col0 = (int64_t)TILE * u.t + 64 * h;
+        int n_box = 0;
+        for (int ch = 0; ch < 2; ++ch) n_box += (col0 + 32 * ch < p.c_cols && row0 < p.c_rows) ? 1 : 0;
+        if (lane == 0) tma_store_wait_read();        // the previous stores have read the staging boxes
+        __syncwarp();
+        if (!__all_sync(0xffffffffu, mbar_wait(tfull, local & 1u, abortp, p.status))) { ok = false; break; }
+        tc_fence_after();
+        double dot = 0.0;
+#pragma unroll 1
+        for (int ch = 0; ch < 2; ++ch) {
+          uint32_t r1[32], r2[32];
+          const uint32_t col = (uint32_t)(64 * h + 32 * ch) + ((uint32_t)(q * 32) << 16);
+          tmem_ld32(tmem_base + col, r1);
+          tmem_ld32(tmem_base + (uint32_t)TILE + col, r2);
+          float part = 0.f;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) part = fmaf(__uint_as_float(r1[i]), __uint_as_float(r2[i]), part);
+          dot += (double)part;
+          if (ch >= n_box) continue;                 // warp-uniform
+          uint8_t* rowp = buf + ch * 4096 + lane * 128;
+#pragma unroll
+          for (int cq = 0; cq < 8; ++cq) {
+            float4* cell = reinterpret_cast<float4*>(rowp + ((cq ^ (lane & 7)) << 4));
+            *cell = make_float4(p.alpha * __uint_as_float(r2[4 * cq]), p.alpha * __uint_as_float(r2[4 * cq + 1]),
+                                p.alpha * __uint_as_float(r2[4 * cq + 2]), p.alpha * __uint_as_float(r2[4 * cq + 3]));
+          }
+        }
+        tc_fence_before();                           // all reads of the accumulator are done
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(tempty);
+          for (int ch = 0; ch < n_box; ++ch)
+            tma_store_2d(&mapC, (int)(col0 + 32 * ch), (int)row0, buf_u32 + ch * 4096);
+          tma_store_commit();
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        if (lane == 0) p.dot_part[((size_t)u.b * p.tiles + u.t) * 8 + e] = dot;
+        continue;
+      }
       if (h >= u.nt) {
         // a single tile: nothing to store, but the accumulator's hand-over is counted per warp
         if (!__all_sync(0xffffffffu, mbar_wait(tfull, local & 1u, abortp, p.status))) { ok = false; break; }
@@ -528,8 +579,8 @@ tc_blockres_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
 }
 
 armor_status launch(armor_ctx* c, const float* X, const float* Q, int64_t rows, int64_t cols, RParams p, float* out,
-                    cudaStream_t s) {
-  CUtensorMap mX, mQ, mC, mD;
+                    cudaStream_t s, const float* X2 = nullptr) {
+  CUtensorMap mX, mX2, mQ, mC, mD;
   if (!make_map_2d(&mQ, Q, TILE, (int64_t)p.batch * TILE, TILE, 32, TILE)) return ARMOR_ERR_CUDA;
   if (!make_map_2d(&mC, out, cols, rows, cols, 32, 32)) return ARMOR_ERR_CUDA;
   if (p.D) {
@@ -538,6 +589,11 @@ armor_status launch(armor_ctx* c, const float* X, const float* Q, int64_t rows, 
     mD = mC;
   }
   if (!make_map_2d(&mX, X, cols, rows, cols, 32, p.x.mn_major ? 32 : TILE, p.x.mn_major != 0)) return ARMOR_ERR_CUDA;
+  if (X2) {
+    if (!make_map_2d(&mX2, X2, cols, rows, cols, 32, p.x.mn_major ? 32 : TILE, p.x.mn_major != 0)) return ARMOR_ERR_CUDA;
+  } else {
+    mX2 = mX;
+  }
   p.c_rows = rows; p.c_cols = cols;
   p.status = c->status;
   p.one_pass = c->block_one_pass;
@@ -545,8 +601,8 @@ armor_status launch(armor_ctx* c, const float* X, const float* Q, int64_t rows, 
   if (ensure_dynamic_smem(attr, c->device, tc_blockres_kernel, SMEM_BYTES) != ARMOR_OK) return ARMOR_ERR_CUDA;
   const int64_t n_items = (int64_t)p.batch * p.tiles;
   const int grid = (int)(n_items < c->n_sm ? n_items : c->n_sm);
-  KTimer kt(c, ARMOR_KC_BLOCK_PRODUCT, (p.D ? 12.0 : 8.0) * (double)rows * (double)cols, s);
-  tc_blockres_kernel<<<grid, NTHREADS, SMEM_BYTES, s>>>(mX, mQ, mC, mD, p);
+  KTimer kt(c, ARMOR_KC_BLOCK_PRODUCT, ((p.D || p.dual) ? 12.0 : 8.0) * (double)rows * (double)cols, s);
+  tc_blockres_kernel<<<grid, NTHREADS, SMEM_BYTES, s>>>(mX, mX2, mQ, mC, mD, p);
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
 }
@@ -579,4 +635,19 @@ armor_status tc_blockres_left(armor_ctx* c, const float* Ablk, bool transA, cons
   p.D = add; p.alpha = alpha; p.beta = add ? beta : 0.f;
   p.batch = (int)(rows / TILE); p.tiles = (int)((cols + TILE - 1) / TILE);
   return launch(c, in, Ablk, rows, cols, p, out, s);
+}
+
+// out[i-th block, :] = P_i * in2[i-th block, :] and 8 partial sums per 128 x 128 tile of <P_i * in1, P_i * in2> at part
+// (tile order, then the eight 32 x 64 pieces of the tile); the number of partial sums comes back through n_part
+armor_status tc_blockres_left_dual(armor_ctx* c, const float* Ablk, const float* in1, const float* in2, float* out,
+                                   int64_t rows, int64_t cols, double* part, int* n_part, cudaStream_t s) {
+  if (!ptr_ok(in1) || !ptr_ok(in2) || !ptr_ok(Ablk) || !ptr_ok(out)) return ARMOR_ERR_UNSUPPORTED;
+  RParams p{};
+  p.x = {1, 0, TILE, 0, TILE, 0, BK};
+  p.col_read = 0; p.right = 0;
+  p.D = nullptr; p.alpha = 1.f; p.beta = 0.f;
+  p.batch = (int)(rows / TILE); p.tiles = (int)((cols + TILE - 1) / TILE);
+  p.dual = 1; p.dot_part = part;
+  *n_part = 8 * p.batch * p.tiles;
+  return launch(c, in1, Ablk, rows, cols, p, out, s, in2);
 }

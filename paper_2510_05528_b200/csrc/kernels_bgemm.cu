@@ -351,10 +351,11 @@ extern "C" armor_status armor_block_product_dual(armor_ctx* c, const float* d_bl
                                                  const float* d_in2, float* d_out, double* d_dot, int32_t path,
                                                  armor_stream_t stream) {
   if (!c || !d_blocks || !d_in1 || !d_in2 || !d_out || !d_dot) return ARMOR_ERR_INVALID_ARG;
-  if (path == 1 && !tc_block_ok(c, c->d_out, c->d_in)) return ARMOR_ERR_UNSUPPORTED;
+  if ((path == 1 || path == 2) && !tc_block_ok(c, c->d_out, c->d_in)) return ARMOR_ERR_UNSUPPORTED;
+  if (path == 2 && !tc_blockres_ok(c)) return ARMOR_ERR_UNSUPPORTED;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   const int saved = c->tc_blocks;
-  c->tc_blocks = (path == 0 || path == 1) ? path : saved;
+  c->tc_blocks = (path == 0 || path == 1 || path == 2) ? path : saved;
   int nq = 0;
   bd_left_dual(c, d_blocks, d_in1, d_in2, c->V, d_out, c->d_out, c->d_in, c->partials, &nq, s);
   reduce_partials_to(c, c->partials, nq, d_dot, s);

@@ -728,7 +728,7 @@ def test_dual_block_product(db, shape):
     V1, V2 = O.bd_left(Q, X1), O.bd_left(Q, X2)
     ref = float(np.sum(V1 * V2))
     Qd, X1d, X2d = dev(Q), dev(X1), dev(X2)
-    for path, tol in ((0, 2e-6), (1, 1e-5)):
+    for path, tol in ((0, 2e-6), (1, 1e-5)) + (((2, 1e-5),) if db == 128 else ()):
         out = torch.full((rows, cols), 7.0, device=DEV)
         dot = Bd.armor_block_product_dual(ctx.ctx, Qd, X1d, X2d, out, path=path)
         assert rel(host(out), V2) < tol
