@@ -319,6 +319,18 @@ armor_status armor_block_product(armor_ctx* ctx, int32_t side, int32_t transpose
                                  const float* d_in, float* d_out, int64_t rows, int64_t cols, float alpha,
                                  const float* d_add, float beta, int32_t path, armor_stream_t stream);
 
+/* A product with both wrappers (Section 3.1; the gradient of the core, Gamma = A^T (E H_w) B^T, is one):
+ *   d_out[i-th block row, j-th block column] = alpha * Lop_i * d_in[i, j] * Rop_j,
+ * Lop_i = d_left[i] or, if transpose_left != 0, its transpose; Rop_j likewise from d_right.  d_left is
+ * [d_out / d_block, d_block, d_block], d_right [d_in / d_block, d_block, d_block], d_in and d_out [d_out, d_in] of the
+ * context (device fp32, distinct).  path 3: one fused tensor-core launch in which Lop_i d_in[i, j] stays in tensor
+ * memory (d_block = 128 and a tensor-core precision, else UNSUPPORTED); paths 0, 1, 2: the two one-sided products
+ * on the kernel armor_block_product names; any other value: what the library itself uses (path 3 where it applies).
+ * Paths 1, 2 and 3 give the same bits.  Exposed for tests and measurements. */
+armor_status armor_block_product_two_sided(armor_ctx* ctx, const float* d_left, int32_t transpose_left, const float* d_in,
+                                           const float* d_right, int32_t transpose_right, float* d_out, float alpha,
+                                           int32_t path, armor_stream_t stream);
+
 /* The pair of products behind the step length of a line search (Section 3.2: the exact step along a direction
  * V needs tr(V H_w V^T) = <V H_w, V> with V = A R and V H_w = A (R H_w)):
  *   d_out = Q d_in2 per block row (side 1 above, alpha 1, no addend) and *d_dot = <Q d_in1, Q d_in2>,

@@ -29,7 +29,7 @@ EXPORTS = ["armor_workspace_bytes", "armor_create", "armor_destroy", "armor_gram
            "armor_packed_layer_bytes", "armor_pack_layer", "armor_apply_layer",
            "armor_get_device_status",
            "armor_status_string", "armor_launch_count", "armor_gemm_timing_enable", "armor_gemm_timing",
-           "armor_normalize_noalloc", "armor_block_product", "armor_block_product_dual", "armor_selftest_wait_timeout", "armor_kernel_timing_enable", "armor_use_graphs",
+           "armor_normalize_noalloc", "armor_block_product", "armor_block_product_dual", "armor_block_product_two_sided", "armor_selftest_wait_timeout", "armor_kernel_timing_enable", "armor_use_graphs",
            "armor_kernel_timing"]
 
 
@@ -85,6 +85,7 @@ def lib() -> C.CDLL:
         L.armor_normalize_noalloc.argtypes = [vp, i64, i64, vp, vp, vp, vp]
         L.armor_block_product.argtypes = [vp, i32, i32, vp, vp, vp, i64, i64, C.c_float, vp, C.c_float, i32, vp]
         L.armor_block_product_dual.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp]
+        L.armor_block_product_two_sided.argtypes = [vp, vp, i32, vp, vp, i32, vp, C.c_float, i32, vp]
         L.armor_gemm_timing_enable.argtypes = [vp, i32]
         L.armor_gemm_timing.argtypes = [vp, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.armor_kernel_timing_enable.argtypes = [vp, i32]
@@ -265,6 +266,15 @@ def armor_block_product(ctx, side: int, transpose: bool, blocks, x, out, alpha=1
     _check(lib().armor_block_product(ctx, int(side), int(bool(transpose)), _ptr(blocks, f, "blocks"), _ptr(x, f, "x"),
                                      _ptr(out, f, "out"), x.shape[0], x.shape[1], float(alpha), _ptr(add, f, "add"),
                                      float(beta), int(path), _stream()), "armor_block_product")
+
+
+def armor_block_product_two_sided(ctx, left, transpose_left: bool, x, right, transpose_right: bool, out, alpha=1.0,
+                                  path=-1) -> None:
+    """out = alpha * Lop . x . Rop with both block-diagonal wrappers (see armor.h)."""
+    f = torch.float32
+    _check(lib().armor_block_product_two_sided(ctx, _ptr(left, f, "left"), int(bool(transpose_left)), _ptr(x, f, "x"),
+                                               _ptr(right, f, "right"), int(bool(transpose_right)), _ptr(out, f, "out"),
+                                               float(alpha), int(path), _stream()), "armor_block_product_two_sided")
 
 
 def armor_block_product_dual(ctx, blocks, x1, x2, out, path=-1) -> float:

@@ -14,7 +14,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libarmor.so")
 SOURCES = ["armor_api.cu", "block_tcgen05.cu", "dense_ops.cu", "gemm_tcgen05.cu", "kernels_bgemm.cu", "kernels_chol.cu",
            "kernels_mask.cu", "kernels_stream.cu", "noalloc_normalize.cu", "sparse_tcgen05.cu", "fwd_tcgen05.cu",
-           "split_f16.cu", "selftest.cu", "blockres_tcgen05.cu"]
+           "split_f16.cu", "selftest.cu", "blockres_tcgen05.cu", "block2_tcgen05.cu"]
 
 
 def _nvcc() -> str:

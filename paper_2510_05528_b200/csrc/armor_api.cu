@@ -226,8 +226,7 @@ armor_status reset_adam(armor_ctx* c, cudaStream_t s) {
 
 armor_status core_gradient(armor_ctx* c, const float* A, const float* B, cudaStream_t s) {
   // Gamma = A^T (E H_w) B^T  (minus half of the gradient display of Appendix D.3)
-  bd_left(c, A, true, c->EH, c->Tmp, c->d_out, c->d_in, 1.f, nullptr, 0.f, s);
-  bd_right(c, c->Tmp, B, true, c->Gam, c->d_out, c->d_in, 1.f, nullptr, 0.f, s);
+  bd_two_sided(c, A, true, c->EH, B, true, c->Tmp, c->Gam, c->d_out, c->d_in, 1.f, s);
   return ARMOR_OK;
 }
 

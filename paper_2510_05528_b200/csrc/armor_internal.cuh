@@ -198,6 +198,11 @@ void bd_right(armor_ctx* c, const float* in, const float* Bblk, bool transB, flo
               int64_t cols, float alpha, const float* add, float beta, cudaStream_t s);
 void bd_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, float* out, int64_t rows,
              int64_t cols, float alpha, const float* add, float beta, cudaStream_t s);
+// out = alpha * Lop X Rop with both wrappers (Lop_i = Lblk[i] or its transpose, Rop_j likewise): one fused launch on
+// the tensor cores where the shape allows (d_block 128; the intermediate stays in tensor memory), else the two
+// one-sided products through tmp
+void bd_two_sided(armor_ctx* c, const float* Lblk, bool transL, const float* X, const float* Rblk, bool transR, float* tmp,
+                  float* out, int64_t rows, int64_t cols, float alpha, cudaStream_t s);
 // out = Ablk in2 and partial sums of <Ablk in1, Ablk in2> at part, *n_part of them (the consumer adds them up): one
 // fused launch on the tensor cores (Ablk in1 never reaches memory), else two products (the first into tmp) and a dot
 void bd_left_dual(armor_ctx* c, const float* Ablk, const float* in1, const float* in2, float* tmp, float* out,
@@ -213,6 +218,11 @@ armor_status tc_bd_left(armor_ctx* c, const float* Ablk, bool transA, const floa
 // out = P in2 per block row, with the partial sums of <P in1, P in2> (four per 128 x 128 tile) at part
 armor_status tc_bd_left_dual(armor_ctx* c, const float* Ablk, bool transA, const float* in1, const float* in2, float* out,
                              int64_t rows, int64_t cols, double* part, int* n_part, cudaStream_t s);
+
+// both wrappers in one launch (block2_tcgen05.cu); d_block = 128
+bool tc_block2_ok(const armor_ctx* c, int64_t rows, int64_t cols);
+armor_status tc_two_sided(armor_ctx* c, const float* Lblk, bool transL, const float* X, const float* Rblk, bool transR,
+                          float* out, int64_t rows, int64_t cols, float alpha, cudaStream_t s);
 
 // the same with the wrapper block held in tensor memory (blockres_tcgen05.cu); d_block = 128
 bool tc_blockres_ok(const armor_ctx* c);

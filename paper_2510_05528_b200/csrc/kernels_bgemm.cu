@@ -336,6 +336,15 @@ void bd_left(armor_ctx* c, const float* Ablk, bool transA, const float* in, floa
   launch_bgemm(c, g, s);
 }
 
+void bd_two_sided(armor_ctx* c, const float* Lblk, bool transL, const float* X, const float* Rblk, bool transR, float* tmp,
+                  float* out, int64_t rows, int64_t cols, float alpha, cudaStream_t s) {
+  if (c->tc_blocks == 3 && tc_block2_ok(c, rows, cols) &&
+      tc_done(c, tc_two_sided(c, Lblk, transL, X, Rblk, transR, out, rows, cols, alpha, s)))
+    return;
+  bd_left(c, Lblk, transL, X, tmp, rows, cols, 1.f, nullptr, 0.f, s);
+  bd_right(c, tmp, Rblk, transR, out, rows, cols, alpha, nullptr, 0.f, s);
+}
+
 void bd_left_dual(armor_ctx* c, const float* Ablk, const float* in1, const float* in2, float* tmp, float* out,
                   int64_t rows, int64_t cols, double* part, int* n_part, cudaStream_t s) {
   if (c->tc_blocks && tc_block_ok(c, rows, cols) &&
@@ -345,6 +354,21 @@ void bd_left_dual(armor_ctx* c, const float* Ablk, const float* in1, const float
   bd_left(c, Ablk, false, in2, out, rows, cols, 1.f, nullptr, 0.f, s);
   dot_partials(c, out, tmp, rows * cols, part, s);
   *n_part = ARMOR_DOT_BLOCKS;
+}
+
+extern "C" armor_status armor_block_product_two_sided(armor_ctx* c, const float* d_left, int32_t transpose_left,
+                                                      const float* d_in, const float* d_right, int32_t transpose_right,
+                                                      float* d_out, float alpha, int32_t path, armor_stream_t stream) {
+  if (!c || !d_left || !d_in || !d_right || !d_out) return ARMOR_ERR_INVALID_ARG;
+  if (path == 3 && !tc_block2_ok(c, c->d_out, c->d_in)) return ARMOR_ERR_UNSUPPORTED;
+  if ((path == 1 || path == 2) && !tc_block_ok(c, c->d_out, c->d_in)) return ARMOR_ERR_UNSUPPORTED;
+  if (path == 2 && !tc_blockres_ok(c)) return ARMOR_ERR_UNSUPPORTED;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  const int saved = c->tc_blocks;
+  c->tc_blocks = (path >= 0 && path <= 3) ? path : saved;
+  bd_two_sided(c, d_left, transpose_left != 0, d_in, d_right, transpose_right != 0, c->Tmp, d_out, c->d_out, c->d_in, alpha, s);
+  c->tc_blocks = saved;
+  return finish_call(c);
 }
 
 extern "C" armor_status armor_block_product_dual(armor_ctx* c, const float* d_blocks, const float* d_in1,

@@ -738,6 +738,32 @@ def test_dual_block_product(db, shape):
     assert ctx.device_status()[:4] == [0, 0, 0, 0]
 
 
+@pytest.mark.parametrize("tl,tr", [(False, False), (False, True), (True, False), (True, True)])
+@pytest.mark.parametrize("shape", [(512, 768), (2048, 2560)], ids=["small", "several-tiles-per-cta"])
+def test_two_sided_block_product(shape, tl, tr):
+    """out = alpha * Lop x Rop in one launch, the intermediate in tensor memory: the oracle's two products within the
+    fp32 bound, and the bits of the two one-sided tensor-core launches (same MMAs, same fp32 intermediate)."""
+    rng = np.random.default_rng(7 + 2 * int(tl) + int(tr) + shape[0])
+    rows, cols = shape
+    db = 128
+    ctx = Bd.ArmorContext(rows, cols, db, device=DEV, precision=Bd.PREC_FP16X3)
+    L = rng.standard_normal((rows // db, db, db)) * np.exp(rng.uniform(-2, 2, (rows // db, 1, 1)))
+    Rw = rng.standard_normal((cols // db, db, db)) / np.sqrt(db)
+    X = rng.standard_normal((rows, cols))
+    Le = np.ascontiguousarray(np.transpose(L, (0, 2, 1))) if tl else L
+    Re = np.ascontiguousarray(np.transpose(Rw, (0, 2, 1))) if tr else Rw
+    ref = -0.75 * O.bd_right(O.bd_left(Le, X), Re)
+    Ld, Rd, Xd = dev(L), dev(Rw), dev(X)
+    outs = {}
+    for path in (0, 1, 3):
+        out = torch.full((rows, cols), 7.0, device=DEV)
+        Bd.armor_block_product_two_sided(ctx.ctx, Ld, tl, Xd, Rd, tr, out, alpha=-0.75, path=path)
+        outs[path] = host(out)
+        assert rel(outs[path], ref) < (2e-6 if path == 0 else 1e-5)
+    assert np.array_equal(outs[1], outs[3])
+    assert ctx.device_status()[:4] == [0, 0, 0, 0]
+
+
 # ------------------------------------------------------------------ the guard's rejection (full weighting)
 def overlapping_case(d_out, d_in, db, strength, n=4, seed=5):
     """Four calibration tokens and wrapper blocks with nearly parallel columns: the group updates of one
