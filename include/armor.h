@@ -300,6 +300,11 @@ armor_status armor_kernel_timing_enable(armor_ctx* ctx, int32_t level);
  * launched directly between their events.  Results are identical in every case.  enable = 0 switches it off for the context.  (No counterpart
  * in the paper.) */
 armor_status armor_use_graphs(armor_ctx* ctx, int32_t enable);
+/* The A-step needs G_i = P_i T_i^T and Gamma_i = (E H_w)_i T_i^T, the B-step C_j = U_j^T U_j and Gamma_j = U_j^T (E H_w)_j
+ * (Section 3.2): per step the two per-block Grams share an operand.  On the tensor cores they run as ONE launch that
+ * reads every shared chunk once (on by default; the column-block pair needs d_block = 128); enable = 0 runs them as
+ * two launches.  Same MMAs per accumulator in the same order: the results are identical.  For tests and measurements. */
+armor_status armor_fuse_grams(armor_ctx* ctx, int32_t enable);
 armor_status armor_kernel_timing(armor_ctx* ctx, int32_t n_classes, int64_t* launches, double* total_ms,
                                  double* total_work);
 

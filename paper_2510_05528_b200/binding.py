@@ -29,7 +29,7 @@ EXPORTS = ["armor_workspace_bytes", "armor_create", "armor_destroy", "armor_gram
            "armor_packed_layer_bytes", "armor_pack_layer", "armor_apply_layer",
            "armor_get_device_status",
            "armor_status_string", "armor_launch_count", "armor_gemm_timing_enable", "armor_gemm_timing",
-           "armor_normalize_noalloc", "armor_block_product", "armor_block_product_dual", "armor_block_product_two_sided", "armor_selftest_wait_timeout", "armor_kernel_timing_enable", "armor_use_graphs",
+           "armor_normalize_noalloc", "armor_block_product", "armor_block_product_dual", "armor_block_product_two_sided", "armor_selftest_wait_timeout", "armor_kernel_timing_enable", "armor_use_graphs", "armor_fuse_grams",
            "armor_kernel_timing"]
 
 
@@ -90,6 +90,7 @@ def lib() -> C.CDLL:
         L.armor_gemm_timing.argtypes = [vp, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.armor_kernel_timing_enable.argtypes = [vp, i32]
         L.armor_use_graphs.argtypes = [vp, i32]
+        L.armor_fuse_grams.argtypes = [vp, i32]
         L.armor_kernel_timing.argtypes = [vp, i32, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.armor_selftest_wait_timeout.argtypes = [vp, i64, vp, vp]
         for name in EXPORTS:
@@ -293,6 +294,10 @@ def armor_gemm_timing_enable(ctx, enable: bool) -> None:
 
 KERNEL_CLASSES = ["gemm", "block_product", "block_gram", "cholesky", "axpy", "dot", "masked_copy", "mask_select",
                   "mask_guard", "operand_split", "gram_staging", "init", "small", "forward"]
+
+
+def armor_fuse_grams(ctx, enable: bool) -> None:
+    _check(lib().armor_fuse_grams(ctx, 1 if enable else 0), "armor_fuse_grams")
 
 
 def armor_use_graphs(ctx, enable: bool) -> None:

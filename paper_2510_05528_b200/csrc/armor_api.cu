@@ -158,6 +158,7 @@ void rowblock_grams(armor_ctx* c, const float* P, const float* P2, const float* 
   // G_i = P_i T_i^T, G2_i = P2_i T_i^T  (contraction over d_in), batch over row-blocks i; P == nullptr: G2 only
   const int db = c->db;
   if (c->tc_blocks && tc_gram_ok(c)) {
+    if (P && c->gram_pairs && tc_done(c, tc_rowblock_gram_pair(c, P, P2, T, G, G2, s))) return;
     armor_status st = P ? tc_rowblock_gram(c, P, T, G, s) : ARMOR_OK;
     if (st == ARMOR_OK) st = tc_rowblock_gram(c, P2, T, G2, s);
     if (tc_done(c, st)) return;
@@ -176,6 +177,7 @@ void colblock_grams(armor_ctx* c, const float* U, const float* Y, const float* Y
   // C_j = U_j^T Y_j, C2_j = U_j^T Y2_j  (contraction over d_out), batch over column-blocks j; Y == nullptr: C2 only
   const int db = c->db;
   if (c->tc_blocks && tc_gram_ok(c)) {
+    if (Y == U && c->gram_pairs && tc_done(c, tc_colblock_gram_self_pair(c, U, Y2, Cm, Cm2, s))) return;
     armor_status st = Y ? tc_colblock_gram(c, U, Y, Cm, s) : ARMOR_OK;
     if (st == ARMOR_OK) st = tc_colblock_gram(c, U, Y2, Cm2, s);
     if (tc_done(c, st)) return;
@@ -287,6 +289,7 @@ armor_status armor_create(armor_ctx** out, const armor_config* cfg, void* d_work
   c->ws = static_cast<char*>(d_workspace); c->ws_bytes = bytes;
   c->launches = 0;
   c->tc_blocks = 3;
+  c->gram_pairs = 1;
   c->host_err = ARMOR_OK;
   if (cudaGetDevice(&c->device) != cudaSuccess ||
       cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess || c->n_sm < 1) {
@@ -361,6 +364,12 @@ armor_status armor_kernel_timing(armor_ctx* c, int32_t n_classes, int64_t* launc
 armor_status armor_use_graphs(armor_ctx* c, int32_t enable) {
   if (!c) return ARMOR_ERR_INVALID_ARG;
   c->use_graphs = enable ? 1 : 0;
+  return ARMOR_OK;
+}
+
+armor_status armor_fuse_grams(armor_ctx* c, int32_t enable) {
+  if (!c) return ARMOR_ERR_INVALID_ARG;
+  c->gram_pairs = enable ? 1 : 0;
   return ARMOR_OK;
 }
 

@@ -125,6 +125,7 @@ struct armor_ctx {
                         // product, where it halves the shared-memory traffic, and the streaming kernel elsewhere
                         // (the two measure equal on single products at 4096 x 4096);
                         // 0: always the fp32 CUDA-core kernels (exact products with 0 and 1)
+  int gram_pairs;       // 1: the two per-block Grams of a step in one launch (shared operand read once)
   armor_status host_err;   // first launch failure inside the running call that no fallback covers
   int kg;               // groups drawn per block in one sparse-core update (mask_groups, at least 1)
   int block_one_pass;   // 1: products with the wrappers take one tf32 pass (the bf16 forward, whose operands are
@@ -238,6 +239,10 @@ armor_status tc_blockres_left_dual(armor_ctx* c, const float* Ablk, const float*
 bool tc_gram_ok(const armor_ctx* c);
 armor_status tc_rowblock_gram(armor_ctx* c, const float* P, const float* T, float* G, cudaStream_t s);
 armor_status tc_colblock_gram(armor_ctx* c, const float* U, const float* Y, float* Cm, cudaStream_t s);
+// two Grams with a shared operand in one launch (the shared chunks are read once)
+armor_status tc_rowblock_gram_pair(armor_ctx* c, const float* P, const float* P2, const float* T, float* G, float* G2,
+                                   cudaStream_t s);
+armor_status tc_colblock_gram_self_pair(armor_ctx* c, const float* U, const float* Y, float* Cm, float* Cm2, cudaStream_t s);
 armor_status tc_select_rows_times_H(armor_ctx* c, const float* Z, const float* H, float* Y, int nbo_pad, cudaStream_t s);
 // A tensor-core launch that is refused for its shape or alignment (UNSUPPORTED) is replaced by the CUDA-core
 // kernel; any other failure is an error of the call: it is recorded and the entry point returns it.

@@ -33,12 +33,18 @@ using namespace tc;
 
 constexpr int TILE = 128, BK = 32;
 constexpr int NTHREADS = 320;
-constexpr int STAGES = 3;
 constexpr int OP_BYTES = TILE * BK * 4;           // 16 KiB: one operand chunk
-constexpr int STAGE_BYTES = 4 * OP_BYTES;         // A raw (= high part), A low part, B raw, B low part
+// A stage holds SLOTS operand chunks, each as its raw words (= high part) followed by its low part: the M-side and the
+// N-side chunk, and in the pair mode with a shared N side a second M-side chunk.
+template <int SLOTS> struct Geo {
+  static constexpr int STAGES = SLOTS == 3 ? 2 : 3;
+  static constexpr int STAGE_BYTES = 2 * SLOTS * OP_BYTES;
+};
 constexpr uint32_t TMEM_COLS = 512;               // four accumulators of 128 columns (two in use outside the dual mode)
 constexpr int EPI_BYTES = 32 * 64 * 4;            // per epilogue warp: 32 rows x 64 columns (half a tile row) as two swizzled boxes
-constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 4 * EPI_BYTES + 1024;
+template <int SLOTS> constexpr size_t smem_bytes() {
+  return (size_t)Geo<SLOTS>::STAGES * Geo<SLOTS>::STAGE_BYTES + 4 * EPI_BYTES + 1024;
+}
 
 struct OpCoord {
   int mn_major;                     // 0: K-major, 1: MN-major
@@ -60,6 +66,10 @@ struct BParams {
   int32_t* status;
   int batch_fastest;                // 1: consecutive work items are consecutive batches (neighbouring column blocks)
   int one_pass;                     // 1: operands as they are, rounded to tf32 by the tensor core; no low parts
+  int pair;                         // two products per tile into two accumulators from the SAME stages, both stored (C
+                                    // and, through mapD, C2).  1: a second M-side operand (mapB2, addressed like A):
+                                    // C = A.B, C2 = A2.B;  2: the M-side chunk also serves as N side: C = A.A^T-like
+                                    // (the operand with itself), C2 = A.B
   int dual;                         // 1: two B operands per tile (mapB, mapB2); C = alpha * A.B2, dot_part = <A.B1, A.B2>
   double* dot_part;                 // dual: 4 partial sums per tile (one per epilogue warp), in tile order
 };
@@ -108,10 +118,12 @@ __device__ __forceinline__ void umma_tf32_acc(uint32_t tmem_d, uint64_t adesc, u
       : "memory");
 }
 
+template <int SLOTS>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                 const __grid_constant__ CUtensorMap mapB2, const __grid_constant__ CUtensorMap mapC,
                 const __grid_constant__ CUtensorMap mapD, const BParams p) {
+  constexpr int STAGES = Geo<SLOTS>::STAGES, STAGE_BYTES = Geo<SLOTS>::STAGE_BYTES;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ __align__(8) uint64_t bars[3 * STAGES + 12];
@@ -124,7 +136,7 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
   const uint32_t dfull0 = smem_u32(&bars[3 * STAGES + 8]);
   const int n_items = p.batch * p.m_tiles * p.n_tiles * p.n_split;   // tiles (x slabs of the contraction)
   const int n_sub = p.dual ? 2 : 1;                                  // passes through the pipeline per tile
-  const int acc_mask = p.dual ? 3 : 1, acc_shift = p.dual ? 2 : 1;   // accumulators in rotation
+  const int n_acc = (p.dual || p.pair) ? 2 : 1;                      // accumulators per tile
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -161,10 +173,11 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         for (int kc = 0; kc < p.k_chunks; ++kc) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abortp, p.status)) { ok = false; break; }
           const uint32_t fb = full0 + 8 * stage;
-          mbar_expect_tx(fb, 2 * OP_BYTES);
+          mbar_expect_tx(fb, SLOTS * OP_BYTES);
           const uint32_t dst = smem_u32(smem + (size_t)stage * STAGE_BYTES);
           load_operand(dst, &mapA, p.a, b, tm, ks * p.k_chunks + kc, fb);
           load_operand(dst + 2 * OP_BYTES, sub ? &mapB2 : &mapB, p.b, b, tn, ks * p.k_chunks + kc, fb);
+          if (SLOTS == 3) load_operand(dst + 4 * OP_BYTES, &mapB2, p.a, b, tm, ks * p.k_chunks + kc, fb);
           ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -187,14 +200,17 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       const uint64_t db0 = operand_desc(smem_u32(smem) + 2 * OP_BYTES, p.b.mn_major, 0);
       const uint64_t kinc_a = p.a.mn_major ? (1024u >> 4) : (32u >> 4);   // one k-step of 8 in the address field
       const uint64_t kinc_b = p.b.mn_major ? (1024u >> 4) : (32u >> 4);
+      const uint32_t idesc_self = instr_desc_tf32_mn(TILE, TILE, p.a.mn_major, p.a.mn_major);   // pair 2: A chunk on both sides
       int stage = 0; uint32_t phase = 0;
       int local = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x)
       for (int sub = 0; sub < n_sub && ok; ++sub, ++local) {
-        const int as = local & acc_mask;
-        const uint32_t aphase = (uint32_t)(local >> acc_shift) & 1u;
+        // accumulators rotate: two of them, or (dual, pair) four, of which a tile takes two
+        const int as = p.pair ? ((2 * local) & 3) : (local & (2 * n_acc - 1));
+        const uint32_t aphase = (uint32_t)(local >> (p.pair ? 1 : n_acc)) & 1u;
         if (!mbar_wait(tempty0 + 8 * as, aphase ^ 1, abortp, p.status)) { ok = false; break; }
+        if (p.pair && !mbar_wait(tempty0 + 8 * (as + 1), aphase ^ 1, abortp, p.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tacc = tmem_base + (uint32_t)(as * TILE);
         for (int kc = 0; kc < p.k_chunks; ++kc) {
@@ -207,7 +223,28 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
           const uint64_t da = da0 + so, dal = da + (OP_BYTES >> 4);
           const uint64_t dbm = db0 + so, dbl = dbm + (OP_BYTES >> 4);
           const uint32_t first = (uint32_t)(kc > 0);
-          if (p.one_pass) {
+          if (p.pair) {
+            // two products from the same stage.  Accumulator 0: pair 1 A.B, pair 2 the M-side chunk with itself as N
+            // side; accumulator 1: pair 1 A2.B (third slot), pair 2 A.B.  Per accumulator the order of the one-product
+            // kernel (low part of the M side first).
+            const uint32_t tacc1 = tacc + (uint32_t)TILE;
+            const uint64_t m1 = (p.pair == 1) ? da + (4 * OP_BYTES >> 4) : da, m1l = m1 + (OP_BYTES >> 4);   // M side of accumulator 1
+            const uint64_t n0 = (p.pair == 1) ? dbm : da, n0l = n0 + (OP_BYTES >> 4);                       // N side of accumulator 0
+            const uint64_t kinc_n0 = (p.pair == 1) ? kinc_b : kinc_a;
+            const uint32_t id0 = (p.pair == 1) ? idesc : idesc_self;
+#pragma unroll
+            for (int k = 0; k < BK / 8; ++k) {
+              if (k == 0) umma_tf32(tacc, dal, n0, id0, first); else umma_tf32_acc(tacc, dal + k * kinc_a, n0 + k * kinc_n0, id0);
+              umma_tf32_acc(tacc, da + k * kinc_a, n0l + k * kinc_n0, id0);
+              umma_tf32_acc(tacc, da + k * kinc_a, n0 + k * kinc_n0, id0);
+            }
+#pragma unroll
+            for (int k = 0; k < BK / 8; ++k) {
+              if (k == 0) umma_tf32(tacc1, m1l, dbm, idesc, first); else umma_tf32_acc(tacc1, m1l + k * kinc_a, dbm + k * kinc_b, idesc);
+              umma_tf32_acc(tacc1, m1 + k * kinc_a, dbl + k * kinc_b, idesc);
+              umma_tf32_acc(tacc1, m1 + k * kinc_a, dbm + k * kinc_b, idesc);
+            }
+          } else if (p.one_pass) {
             umma_tf32(tacc, da, dbm, idesc, first);
 #pragma unroll
             for (int k = 1; k < BK / 8; ++k) umma_tf32_acc(tacc, da + k * kinc_a, dbm + k * kinc_b, idesc);
@@ -225,7 +262,10 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
           umma_commit(empty0 + 8 * stage);   // frees the stage once these MMAs have read it
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
-        if (ok) umma_commit(tfull0 + 8 * as);
+        if (ok) {
+          umma_commit(tfull0 + 8 * as);
+          if (p.pair) umma_commit(tfull0 + 8 * (as + 1));
+        }
       }
     }
   } else if (warp < 6) {
@@ -238,7 +278,7 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         if (!mbar_wait(full0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
         float4* base = reinterpret_cast<float4*>(smem + (size_t)stage * STAGE_BYTES);
 #pragma unroll
-        for (int op = 0; op < (p.one_pass ? 0 : 2); ++op) {
+        for (int op = 0; op < (p.one_pass ? 0 : SLOTS); ++op) {
           float4* hi = base + op * (2 * OP_BYTES / 16);
           float4* lo = hi + OP_BYTES / 16;
 #pragma unroll
@@ -272,10 +312,52 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++local) {
       int tn, tm, b, ks;
       item_decode(p, item, tn, tm, b, ks);
-      const int as = p.dual ? ((2 * local) & 3) : (local & 1);          // dual: accumulators as (A.B1) and as + 1 (A.B2)
+      const int as = (p.dual || p.pair) ? ((2 * local) & 3) : (local & 1);   // dual, pair: accumulators as and as + 1
       const uint32_t aphase = (uint32_t)(local >> 1) & 1u;
       const int64_t row_base = p.r_b * b + p.r_s * ks + (int64_t)tm * TILE + q * 32;
       const int64_t col_tile = p.c_b * b + (int64_t)tn * TILE;
+      if (p.pair) {
+        // both accumulators are stored: as through mapC, as + 1 through mapD (the second output)
+        bool got = false;
+#pragma unroll 1
+        for (int part = 0; part < 4 && ok; ++part) {
+          const int which = part >> 1, hf = part & 1;
+          int n_box = 0;
+          if (row_base < p.c_rows && tm * TILE + q * 32 < p.m_valid)
+            for (int ch = 0; ch < 2; ++ch) n_box += (col_tile + 64 * hf + 32 * ch < p.c_cols) ? 1 : 0;
+          if (lane == 0) tma_store_wait_read();       // the previous stores have read the staging boxes
+          __syncwarp();
+          if (!got) {
+            if (!mbar_wait(tfull0 + 8 * as, aphase, abortp, p.status)) { ok = false; break; }
+            if (!mbar_wait(tfull0 + 8 * (as + 1), aphase, abortp, p.status)) { ok = false; break; }
+            tc_fence_after();
+            got = true;
+          }
+#pragma unroll 1
+          for (int ch = 0; ch < 2; ++ch) {
+            uint32_t r[32];
+            tmem_ld32(tmem_base + (uint32_t)((as + which) * TILE + hf * 64 + ch * 32) + ((uint32_t)(q * 32) << 16), r);
+            if (ch >= n_box) continue;                // warp-uniform
+            uint8_t* rowp = buf + ch * 4096 + lane * 128;
+#pragma unroll
+            for (int cq = 0; cq < 8; ++cq) {
+              float4* cell = reinterpret_cast<float4*>(rowp + ((cq ^ (lane & 7)) << 4));
+              *cell = make_float4(p.alpha * __uint_as_float(r[4 * cq]), p.alpha * __uint_as_float(r[4 * cq + 1]),
+                                  p.alpha * __uint_as_float(r[4 * cq + 2]), p.alpha * __uint_as_float(r[4 * cq + 3]));
+            }
+          }
+          if (part == 3) tc_fence_before();           // all reads of the accumulators are done
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            if (part == 3) { mbar_arrive(tempty0 + 8 * as); mbar_arrive(tempty0 + 8 * (as + 1)); }
+            for (int ch = 0; ch < n_box; ++ch)
+              tma_store_2d(which ? &mapD : &mapC, (int)(col_tile + 64 * hf + 32 * ch), (int)row_base, buf_u32 + ch * 4096);
+            tma_store_commit();
+          }
+        }
+        continue;
+      }
       if (p.dual) {
         // C = alpha * (A.B2); partial sum of <A.B1, A.B2> over this warp's 32 x 128 slab (rows or columns past the
         // end of the operands were read as zeros and add nothing)
@@ -399,31 +481,39 @@ struct HostOp {
   OpCoord c;
 };
 
+// B2: the second N-side operand (dual) or the second M-side operand (pair 1); C2: the second output (pair)
 armor_status launch(armor_ctx* c, const HostOp& A, const HostOp& B, BParams p, int kclass, double kbytes, cudaStream_t s,
-                    const float* B2 = nullptr) {
+                    const float* B2 = nullptr, float* C2 = nullptr) {
   CUtensorMap mA, mB, mB2, mC, mD;
   if (!make_map_2d(&mC, p.C, p.c_cols, p.c_rows, p.ldc, 32, 32)) return ARMOR_ERR_CUDA;
-  if (p.D) {
+  if (p.pair) {
+    if (!C2 || p.D) return ARMOR_ERR_INVALID_ARG;
+    if (!make_map_2d(&mD, C2, p.c_cols, p.c_rows, p.ldc, 32, 32)) return ARMOR_ERR_CUDA;
+  } else if (p.D) {
     if (!make_map_2d(&mD, p.D, p.c_cols, p.c_rows, p.ldd, 32, 32)) return ARMOR_ERR_CUDA;
   } else {
     mD = mC;
   }
   if (!make_map_2d(&mA, A.base, A.inner, A.outer, A.ld, 32, A.c.mn_major ? 32 : TILE, A.c.mn_major != 0)) return ARMOR_ERR_CUDA;
   if (!make_map_2d(&mB, B.base, B.inner, B.outer, B.ld, 32, B.c.mn_major ? 32 : TILE, B.c.mn_major != 0)) return ARMOR_ERR_CUDA;
-  if (B2) {
+  if (B2 && p.pair == 1) {
+    if (!make_map_2d(&mB2, B2, A.inner, A.outer, A.ld, 32, A.c.mn_major ? 32 : TILE, A.c.mn_major != 0)) return ARMOR_ERR_CUDA;
+  } else if (B2) {
     if (!make_map_2d(&mB2, B2, B.inner, B.outer, B.ld, 32, B.c.mn_major ? 32 : TILE, B.c.mn_major != 0)) return ARMOR_ERR_CUDA;
   } else {
     mB2 = mB;
   }
   p.a = A.c; p.b = B.c;
   p.status = c->status;
-  static PerDeviceOnce attr;
-  if (ensure_dynamic_smem(attr, c->device, tc_block_kernel, SMEM_BYTES) != ARMOR_OK) return ARMOR_ERR_CUDA;
+  static PerDeviceOnce attr2, attr3;
+  if (ensure_dynamic_smem(attr2, c->device, tc_block_kernel<2>, smem_bytes<2>()) != ARMOR_OK) return ARMOR_ERR_CUDA;
+  if (ensure_dynamic_smem(attr3, c->device, tc_block_kernel<3>, smem_bytes<3>()) != ARMOR_OK) return ARMOR_ERR_CUDA;
   const int n_sm = c->n_sm;
   const int n_items = p.batch * p.m_tiles * p.n_tiles * p.n_split;
   const int grid = n_items < n_sm ? n_items : n_sm;
   KTimer kt(c, kclass, kbytes, s);
-  tc_block_kernel<<<grid, NTHREADS, SMEM_BYTES, s>>>(mA, mB, mB2, mC, mD, p);
+  if (p.pair == 1) tc_block_kernel<3><<<grid, NTHREADS, smem_bytes<3>(), s>>>(mA, mB, mB2, mC, mD, p);
+  else tc_block_kernel<2><<<grid, NTHREADS, smem_bytes<2>(), s>>>(mA, mB, mB2, mC, mD, p);
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
 }
@@ -555,6 +645,38 @@ armor_status gram_launch(armor_ctx* c, const HostOp& A, const HostOp& B, float* 
   return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
 }
 
+// Two Grams in one launch from the same stages.  pair 1: G = A.B, G2 = A2.B (A2 addressed like A); pair 2: G = A with
+// itself, G2 = A.B.  Every shared chunk is read once.
+armor_status gram_pair_launch(armor_ctx* c, const HostOp& A, const HostOp& B, const float* A2, int pair, float* G, float* G2,
+                              int nb, int64_t K, cudaStream_t s) {
+  const int db = c->db;
+  const int64_t chunks = K / BK;
+  const int tiles = (db / TILE) * (db / TILE);
+  int ks = pick_split((int64_t)nb * tiles, chunks);
+  const int64_t slab = (int64_t)nb * db * db;
+  if (ks > 1 && (!c->gpart || 2 * ks * slab > c->gpart_floats)) ks = 1;
+  BParams p{};
+  p.C = ks > 1 ? c->gpart : G; p.D = nullptr; p.ldc = db; p.ldd = db;
+  float* C2 = ks > 1 ? c->gpart + ks * slab : G2;
+  p.c_rows = (int64_t)ks * nb * db; p.c_cols = db;
+  p.r_b = db; p.c_b = 0; p.r_s = (int64_t)nb * db;
+  p.m_tiles = db / TILE; p.n_tiles = db / TILE; p.batch = nb; p.k_chunks = (int)(chunks / ks); p.n_split = ks;
+  p.alpha = 1.f; p.beta = 0.f; p.m_valid = 1 << 30;
+  p.pair = pair;
+  // three (pair 1) or two (pair 2) W-shaped operands are read once each
+  armor_status st = launch(c, A, B, p, ARMOR_KC_BLOCK_GRAM, (pair == 1 ? 12.0 : 8.0) * (double)c->wn, s, A2, C2);
+  if (st != ARMOR_OK || ks == 1) return st;
+  KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
+  int64_t blocks = (slab / 4 + 255) / 256;
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  sum_slabs_kernel<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(c->gpart), slab / 4, ks,
+                                                   reinterpret_cast<float4*>(G));
+  sum_slabs_kernel<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(c->gpart + ks * slab), slab / 4, ks,
+                                                   reinterpret_cast<float4*>(G2));
+  c->launches += 2;
+  return cudaGetLastError() == cudaSuccess ? ARMOR_OK : ARMOR_ERR_CUDA;
+}
+
 }  // namespace
 
 bool tc_gram_ok(const armor_ctx* c) {
@@ -577,6 +699,27 @@ armor_status tc_colblock_gram(armor_ctx* c, const float* U, const float* Y, floa
   HostOp A{U, c->d_in, c->d_out, c->d_in, {1, db, TILE, 0, 0, 0, BK}};   // Aop[m][k] = U[k][j*db + m]: M-major
   HostOp B{Y, c->d_in, c->d_out, c->d_in, {1, db, TILE, 0, 0, 0, BK}};
   return gram_launch(c, A, B, Cm, c->nbi, c->d_out, s);
+}
+
+// G_i = P_i T_i^T and G2_i = P2_i T_i^T in one launch (T read once)
+armor_status tc_rowblock_gram_pair(armor_ctx* c, const float* P, const float* P2, const float* T, float* G, float* G2,
+                                   cudaStream_t s) {
+  const int db = c->db;
+  if (!ptr_ok(P) || !ptr_ok(P2) || !ptr_ok(T) || !ptr_ok(G) || !ptr_ok(G2)) return ARMOR_ERR_UNSUPPORTED;
+  HostOp A{P, c->d_in, c->d_out, c->d_in, {0, 0, 0, BK, db, TILE, 0}};
+  HostOp B{T, c->d_in, c->d_out, c->d_in, {0, 0, 0, BK, db, TILE, 0}};
+  return gram_pair_launch(c, A, B, P2, 1, G, G2, c->nbo, c->d_in, s);
+}
+
+// C_j = U_j^T U_j and C2_j = U_j^T Y_j in one launch (U and Y read once each); d_block = 128 (one tile per block: the
+// chunk of U that is the M side of a tile is also its N side)
+armor_status tc_colblock_gram_self_pair(armor_ctx* c, const float* U, const float* Y, float* Cm, float* Cm2, cudaStream_t s) {
+  const int db = c->db;
+  if (db != TILE) return ARMOR_ERR_UNSUPPORTED;
+  if (!ptr_ok(U) || !ptr_ok(Y) || !ptr_ok(Cm) || !ptr_ok(Cm2)) return ARMOR_ERR_UNSUPPORTED;
+  HostOp A{U, c->d_in, c->d_out, c->d_in, {1, db, TILE, 0, 0, 0, BK}};
+  HostOp B{Y, c->d_in, c->d_out, c->d_in, {1, db, TILE, 0, 0, 0, BK}};
+  return gram_pair_launch(c, A, B, nullptr, 2, Cm, Cm2, c->nbi, c->d_out, s);
 }
 
 // Y[j][i][:] = Z[j][i][:] * H[j-th block row, :]  for i < nbo: per column-block j a thin [nbo, d_block] x

@@ -102,3 +102,29 @@ def test_replay_in_pieces_around_timed_products_is_bit_identical(mode):
     if MODES[mode]["h_mode"] == Bd.H_FULL:
         assert g[8] >= 2 * 14
     assert d[7] == g[7] == [0, 0, 0, 0]
+
+
+@pytest.mark.parametrize("cfg", [MID, MID.with_(name="mid256", d_block=256, d_out=512)], ids=["d_block-128", "d_block-256"])
+@pytest.mark.parametrize("mode", ["full-exact", "diag-exact", "full-adam"])
+def test_fused_gram_pairs_are_bit_identical_to_separate_launches(cfg, mode):
+    """The two per-block Grams of the A-step (shared T) and of the B-step (U with itself and with E H) in one launch each:
+    every accumulator sees the same MMAs in the same order, so whole runs agree bit for bit."""
+    W = inputs.make_weight(cfg)
+    H32 = O.gram(inputs.make_activations(cfg)).astype(np.float32)
+    Hd, Wd = dev(H32), dev(W)
+    out = {}
+    for fused in (False, True):
+        ctx = make(cfg, Bd.PREC_FP16X3, **MODES[mode])
+        Bd.armor_fuse_grams(ctx.ctx, fused)
+        st = ctx.init(Wd, Hd)
+        n0 = ctx.launch_count()
+        stats = ctx.read_stats(ctx.bcd_step(st, Hd, 0, 6)).copy()
+        out[fused] = (host(st.A).copy(), host(st.B).copy(), host(st.S).copy(), host(st.M).copy(), stats,
+                      ctx.launch_count() - n0, ctx.device_status()[:4])
+    d, g = out[False], out[True]
+    for x, y in zip(d[:4], g[:4]):
+        assert np.array_equal(x, y)
+    assert d[4].tobytes() == g[4].tobytes()
+    if mode != "full-adam":
+        assert g[5] < d[5]                       # fewer launches
+    assert d[6] == g[6] == [0, 0, 0, 0]
