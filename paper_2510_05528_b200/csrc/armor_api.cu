@@ -240,6 +240,15 @@ armor_status residual_and_loss(armor_ctx* c, const float* W, const float* H, con
   const int saved = c->tc_blocks;
   if (exact_products) c->tc_blocks = 0;
   bd_right(c, S, B, false, c->T, c->d_out, c->d_in, 1.f, nullptr, 0.f, s);      // T = S B
+  if (c->cfg.h_mode == ARMOR_H_DIAG && c->tc_blocks && tc_block_ok(c, c->d_out, c->d_in)) {
+    // diagonal weighting: E = W - A T, E H_w = E diag(h) and L = <E H_w, E> in one pass
+    int nq = 0;
+    if (tc_done(c, tc_bd_left_residual(c, A, c->T, W, c->hdiag, c->E, c->EH, c->d_out, c->d_in, c->partials, &nq, s))) {
+      c->tc_blocks = saved;
+      reduce_partials_to(c, c->partials, nq, out, s);
+      return ARMOR_OK;
+    }
+  }
   bd_left(c, A, false, c->T, c->E, c->d_out, c->d_in, -1.f, W, 1.f, s);         // E = W - A T
   c->tc_blocks = saved;
   return rmul_H(c, c->E, H, c->EH, c->d_out, c->E, out, nullptr, nullptr, s);   // EH = E H_w, L = <EH, E>

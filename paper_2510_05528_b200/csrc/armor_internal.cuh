@@ -225,6 +225,10 @@ bool tc_block2_ok(const armor_ctx* c, int64_t rows, int64_t cols);
 armor_status tc_two_sided(armor_ctx* c, const float* Lblk, bool transL, const float* X, const float* Rblk, bool transR,
                           float* out, int64_t rows, int64_t cols, float alpha, cudaStream_t s);
 
+// E = add - Ablk in, EH = E diag(colw), partial sums of <E, EH> at part: one launch
+armor_status tc_bd_left_residual(armor_ctx* c, const float* Ablk, const float* in, const float* add, const float* colw,
+                                 float* E, float* EH, int64_t rows, int64_t cols, double* part, int* n_part, cudaStream_t s);
+
 // the same with the wrapper block held in tensor memory (blockres_tcgen05.cu); d_block = 128
 bool tc_blockres_ok(const armor_ctx* c);
 armor_status tc_blockres_right(armor_ctx* c, const float* in, const float* Bblk, bool transB, float* out, int64_t rows,

@@ -71,7 +71,10 @@ struct BParams {
                                     // C = A.B, C2 = A2.B;  2: the M-side chunk also serves as N side: C = A.A^T-like
                                     // (the operand with itself), C2 = A.B
   int dual;                         // 1: two B operands per tile (mapB, mapB2); C = alpha * A.B2, dot_part = <A.B1, A.B2>
-  double* dot_part;                 // dual: 4 partial sums per tile (one per epilogue warp), in tile order
+  double* dot_part;                 // dual, colw: 4 partial sums per tile (one per epilogue warp), in tile order
+  const float* colw;                // not null: a second output C2 (through mapB2) = C scaled per column by colw, and
+                                    // dot_part = sum of C * C2 (the residual, its weighted form and the loss of the
+                                    // diagonal weighting, Eq. 2 with H_w = diag(h), in one pass)
 };
 
 __device__ __forceinline__ void load_operand(uint32_t dst, const CUtensorMap* map, const OpCoord& o, int b, int t, int kc,
@@ -411,6 +414,7 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       }
       // The warp's 32 x 128 slab goes through shared memory in two halves of 64 columns (two 32 x 32 boxes).
       bool waited = false;
+      double wdot = 0.0;
 #pragma unroll 1
       for (int hf = 0; hf < 2 && ok; ++hf) {
         // boxes of this half that lie inside C (warp-uniform)
@@ -464,6 +468,38 @@ tc_block_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             tma_store_2d(&mapC, (int)(col_tile + 64 * hf + 32 * ch), (int)row_base, buf_u32 + ch * 4096);
           tma_store_commit();
         }
+        if (p.colw) {
+          // the boxes still hold C: once the store has read them they become C2 = C * colw[column]
+          if (lane == 0) tma_store_wait_read();
+          __syncwarp();
+          float part = 0.f;
+          for (int ch = 0; ch < n_box; ++ch) {
+            const float4* w4 = reinterpret_cast<const float4*>(p.colw + col_tile + 64 * hf + 32 * ch);
+            uint8_t* rowp = buf + ch * 4096 + lane * 128;
+#pragma unroll
+            for (int cq = 0; cq < 8; ++cq) {
+              float4* cell = reinterpret_cast<float4*>(rowp + ((cq ^ (lane & 7)) << 4));
+              const float4 v = *cell, w = __ldg(w4 + cq);
+              const float4 e = make_float4(v.x * w.x, v.y * w.y, v.z * w.z, v.w * w.w);
+              part = fmaf(v.x, e.x, part); part = fmaf(v.y, e.y, part); part = fmaf(v.z, e.z, part); part = fmaf(v.w, e.w, part);
+              *cell = e;
+            }
+          }
+          wdot += (double)part;
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            for (int ch = 0; ch < n_box; ++ch)
+              tma_store_2d(&mapB2, (int)(col_tile + 64 * hf + 32 * ch), (int)row_base, buf_u32 + ch * 4096);
+            tma_store_commit();
+          }
+        }
+      }
+      if (p.colw) {
+        // lanes in a fixed order
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) wdot += __shfl_xor_sync(0xffffffffu, wdot, o);
+        if (ok && lane == 0) p.dot_part[(size_t)item * 4 + q] = wdot;
       }
     }
     if (lane == 0) tma_store_wait_read();           // shared memory stays valid until the stores have read it
@@ -496,7 +532,11 @@ armor_status launch(armor_ctx* c, const HostOp& A, const HostOp& B, BParams p, i
   }
   if (!make_map_2d(&mA, A.base, A.inner, A.outer, A.ld, 32, A.c.mn_major ? 32 : TILE, A.c.mn_major != 0)) return ARMOR_ERR_CUDA;
   if (!make_map_2d(&mB, B.base, B.inner, B.outer, B.ld, 32, B.c.mn_major ? 32 : TILE, B.c.mn_major != 0)) return ARMOR_ERR_CUDA;
-  if (B2 && p.pair == 1) {
+  if (p.colw) {
+    // the second output has the geometry of C
+    if (!C2 || p.pair || p.dual) return ARMOR_ERR_INVALID_ARG;
+    if (!make_map_2d(&mB2, C2, p.c_cols, p.c_rows, p.ldc, 32, 32)) return ARMOR_ERR_CUDA;
+  } else if (B2 && p.pair == 1) {
     if (!make_map_2d(&mB2, B2, A.inner, A.outer, A.ld, 32, A.c.mn_major ? 32 : TILE, A.c.mn_major != 0)) return ARMOR_ERR_CUDA;
   } else if (B2) {
     if (!make_map_2d(&mB2, B2, B.inner, B.outer, B.ld, 32, B.c.mn_major ? 32 : TILE, B.c.mn_major != 0)) return ARMOR_ERR_CUDA;
@@ -595,6 +635,28 @@ armor_status tc_bd_left_dual(armor_ctx* c, const float* Ablk, bool transA, const
   *n_part = 4 * p.batch * p.m_tiles * p.n_tiles;
   // two W-shaped reads, one W-shaped write
   return launch(c, A, B, p, ARMOR_KC_BLOCK_PRODUCT, 12.0 * (double)rows * (double)cols, s, in2);
+}
+
+// E = add - P_i * in per block row, EH = E scaled per column by colw, and 4 partial sums per 128 x 128 tile of <E, EH> at
+// part (the residual E = W - A T, E diag(h) and the proxy loss of the diagonal weighting in one pass)
+armor_status tc_bd_left_residual(armor_ctx* c, const float* Ablk, const float* in, const float* add, const float* colw,
+                                 float* E, float* EH, int64_t rows, int64_t cols, double* part, int* n_part, cudaStream_t s) {
+  const int db = c->db;
+  const int nb = (int)(rows / db);
+  if (!ptr_ok(in) || !ptr_ok(Ablk) || !ptr_ok(add) || !ptr_ok(colw) || !ptr_ok(E) || !ptr_ok(EH) || cols % TILE) return ARMOR_ERR_UNSUPPORTED;
+  HostOp A{Ablk, db, (int64_t)nb * db, db, {0, 0, 0, BK, db, TILE, 0}};
+  HostOp B{in, cols, rows, cols, {1, 0, TILE, 0, db, 0, BK}};
+  BParams p{};
+  p.C = E; p.D = add; p.ldc = cols; p.ldd = cols; p.c_rows = rows; p.c_cols = cols;
+  p.r_b = db; p.c_b = 0;
+  p.m_tiles = db / TILE; p.n_tiles = (int)(cols / TILE); p.batch = nb; p.k_chunks = db / BK;
+  p.alpha = -1.f; p.beta = 1.f;
+  p.n_split = 1; p.r_s = 0; p.m_valid = 1 << 30;
+  p.one_pass = c->block_one_pass;
+  p.colw = colw; p.dot_part = part;
+  *n_part = 4 * p.batch * p.m_tiles * p.n_tiles;
+  // two W-shaped reads (in, add), two writes
+  return launch(c, A, B, p, ARMOR_KC_BLOCK_PRODUCT, 16.0 * (double)rows * (double)cols, s, nullptr, EH);
 }
 
 namespace {
