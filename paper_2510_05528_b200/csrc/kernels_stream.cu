@@ -249,8 +249,17 @@ __global__ void zero_scalars_kernel(double* sc, int32_t* failflag, int nflag, in
 
 // Fixed-order sums by one warp: lane l adds entries l, l + 32, ...; then a shuffle tree.  All lanes get the sum.
 __device__ __forceinline__ double warp_sum_f64(const double* __restrict__ p, int n) {
+  // (eight loads in flight per lane; the additions keep their order)
   double v = 0.0;
-  for (int i = threadIdx.x; i < n; i += 32) v += p[i];
+  int i = threadIdx.x;
+  for (; i + 7 * 32 < n; i += 8 * 32) {
+    double t[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) t[u] = p[i + 32 * u];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v += t[u];
+  }
+  for (; i < n; i += 32) v += p[i];
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
 }
