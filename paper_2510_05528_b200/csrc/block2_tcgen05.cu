@@ -45,43 +45,7 @@ struct P2Params {
   int32_t* status;
 };
 
-__device__ __forceinline__ void umma_acc(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, 1, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc)
-      : "memory");
-}
-// A from tensor memory
-__device__ __forceinline__ void umma_ta(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(acc)
-      : "memory");
-}
-__device__ __forceinline__ void umma_ta_acc(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, 1, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc)
-      : "memory");
-}
 
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
-        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
-        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
 
 // chunk kc of a 128 x 128 block operand whose rows start at row0 of the [*, 128] array behind map: K-major as one
 // box of 128 rows x 32 columns, MN-major as four boxes of 32 x 32 (rows 32 kc .., columns 32 q ..)
@@ -196,13 +160,13 @@ tc_block2_kernel(const __grid_constant__ CUtensorMap mapL, const __grid_constant
           const uint64_t so = (uint64_t)(uint32_t)(stage * (STAGE_BYTES >> 4));
           const uint64_t da = da0 + so, dal = da + (OP_BYTES >> 4), dx = dx0 + so, dxl = dx + (OP_BYTES >> 4);
           umma_tf32(d1, dal, dx, idesc1, (uint32_t)(kc > 0));
-          umma_acc(d1, da, dxl, idesc1);
-          umma_acc(d1, da, dx, idesc1);
+          umma_tf32_acc(d1, da, dxl, idesc1);
+          umma_tf32_acc(d1, da, dx, idesc1);
 #pragma unroll
           for (int k = 1; k < BK / 8; ++k) {
-            umma_acc(d1, dal + k * kinc_a, dx + k * kinc_x, idesc1);
-            umma_acc(d1, da + k * kinc_a, dxl + k * kinc_x, idesc1);
-            umma_acc(d1, da + k * kinc_a, dx + k * kinc_x, idesc1);
+            umma_tf32_acc(d1, dal + k * kinc_a, dx + k * kinc_x, idesc1);
+            umma_tf32_acc(d1, da + k * kinc_a, dxl + k * kinc_x, idesc1);
+            umma_tf32_acc(d1, da + k * kinc_a, dx + k * kinc_x, idesc1);
           }
           umma_commit(empty0 + 8 * stage);
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -221,14 +185,14 @@ tc_block2_kernel(const __grid_constant__ CUtensorMap mapL, const __grid_constant
           tc_fence_after();
           const uint64_t dr = dr0 + (uint64_t)(uint32_t)(stage * (STAGE_BYTES >> 4)), drl = dr + (OP_BYTES >> 4);
           const uint32_t a_hi = d1 + (uint32_t)(kc * BK), a_lo = d1lo + (uint32_t)(kc * BK);
-          umma_ta(d2, a_lo, dr, idesc2, (uint32_t)(kc > 0));
-          umma_ta_acc(d2, a_hi, drl, idesc2);
-          umma_ta_acc(d2, a_hi, dr, idesc2);
+          umma_tf32_ta(d2, a_lo, dr, idesc2, (uint32_t)(kc > 0));
+          umma_tf32_ta_acc(d2, a_hi, drl, idesc2);
+          umma_tf32_ta_acc(d2, a_hi, dr, idesc2);
 #pragma unroll
           for (int k = 1; k < BK / 8; ++k) {
-            umma_ta_acc(d2, a_lo + 8 * k, dr + k * kinc_r, idesc2);
-            umma_ta_acc(d2, a_hi + 8 * k, drl + k * kinc_r, idesc2);
-            umma_ta_acc(d2, a_hi + 8 * k, dr + k * kinc_r, idesc2);
+            umma_tf32_ta_acc(d2, a_lo + 8 * k, dr + k * kinc_r, idesc2);
+            umma_tf32_ta_acc(d2, a_hi + 8 * k, drl + k * kinc_r, idesc2);
+            umma_tf32_ta_acc(d2, a_hi + 8 * k, dr + k * kinc_r, idesc2);
           }
           umma_commit(empty0 + 8 * stage);
           if (++stage == STAGES) { stage = 0; phase ^= 1; }

@@ -111,15 +111,6 @@ __device__ __forceinline__ uint64_t operand_desc(uint32_t base, int mn_major, in
   return mn_major ? smem_desc_mn_sw128_32b(base + kstep * 1024, 4096, 512) : smem_desc_sw128(base + kstep * 32, 16, 1024);
 }
 
-// tcgen05.mma with the accumulate flag set (the constant predicate costs no instruction)
-__device__ __forceinline__ void umma_tf32_acc(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, 1, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc)
-      : "memory");
-}
 
 template <int SLOTS>
 __global__ void __launch_bounds__(NTHREADS, 1)
