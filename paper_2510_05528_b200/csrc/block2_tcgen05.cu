@@ -12,12 +12,17 @@
 // same fp32 value, so the result has the same bits.
 //
 // Persistent kernel, 448 threads:
-//   warp 0       : TMA producer.  Per tile four chunks (32 along k) of Lop_i and X_ij, then four chunks (32 along l) of Rop_j
-//   warp 1       : MMA issuer: product 1 into D1, wait for the split, product 2 (A from tensor memory) into D2[t % 2]
+//   warp 0       : TMA producer.  Per tile four chunks (32 along k) of Lop_i and X_ij (product 1) and four chunks (32
+//                  along l) of Rop_j (product 2)
+//   warp 1       : MMA issuer: product 1 into D1[t % 2]; product 2 (A from tensor memory) into D2
 //   warps 2-5    : low parts of the chunks in shared memory
 //   warps 6-9    : epilogue of D2 (alpha, swizzled staging, TMA store)
 //   warps 10-13  : split of D1 in tensor memory
-// Tensor memory: D1 0..127, low part of D1 128..255, D2 256..383 and 384..511.
+// The products are software-pipelined: product 1 of tile t + 1 is issued BEFORE product 2 of tile t
+// (P1(0), P1(1), P2(0), P1(2), P2(1), ...), so that the tensor pipe works on the next tile while four warps split this
+// tile's intermediate, and the epilogue drains D2 while product 1 of the tile after next runs.  The producer and the
+// splitter walk their chunks in the same order.
+// Tensor memory: D1 0..127 and 128..255 (alternating), low part of D1 256..383, D2 384..511.
 // Every wait is bounded; a wait that runs out raises a status word and the CTA leaves through the common exit that
 // frees its tensor memory.
 #include "tc_common.cuh"
@@ -32,7 +37,7 @@ constexpr int STAGES = 3;
 constexpr int OP_BYTES = TILE * BK * 4;           // 16 KiB: one operand chunk
 constexpr int STAGE_BYTES = 4 * OP_BYTES;         // M side raw, M side low part, N side raw, N side low part
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t T_D1 = 0, T_D1LO = 128, T_D2 = 256;
+constexpr uint32_t T_D1 = 0, T_D1LO = 256, T_D2 = 384;
 constexpr int EPI_BYTES = 32 * 64 * 4;            // per epilogue warp: two swizzled 32 x 32 boxes
 constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 4 * EPI_BYTES + 1024;
 
@@ -59,6 +64,15 @@ __device__ __forceinline__ void load_block_chunk(uint32_t dst, const CUtensorMap
   }
 }
 
+// Step o of a CTA's schedule over its n tiles: P1(0), then (P1(t + 1), P2(t)) for t = 0 .. n - 2, then P2(n - 1).
+__device__ __forceinline__ void schedule_step(int o, int n, bool& second, int& t) {
+  if (o == 0) { second = false; t = 0; return; }
+  const int m = o - 1;
+  if (m == 2 * n - 2) { second = true; t = n - 1; return; }
+  second = (m & 1) != 0;
+  t = second ? (m >> 1) : (m >> 1) + 1;
+}
+
 __device__ __forceinline__ uint64_t op_desc(uint32_t base, int mn) {
   return mn ? smem_desc_mn_sw128_32b(base, 4096, 512) : smem_desc_sw128(base, 16, 1024);
 }
@@ -68,15 +82,16 @@ tc_block2_kernel(const __grid_constant__ CUtensorMap mapL, const __grid_constant
                  const __grid_constant__ CUtensorMap mapR, const __grid_constant__ CUtensorMap mapC, const P2Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  __shared__ __align__(8) uint64_t bars[3 * STAGES + 6];
+  __shared__ __align__(8) uint64_t bars[3 * STAGES + 5];
   __shared__ uint32_t tmem_base_holder;
   __shared__ int abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t full0 = smem_u32(&bars[0]), split0 = smem_u32(&bars[STAGES]), empty0 = smem_u32(&bars[2 * STAGES]);
-  const uint32_t d1full = smem_u32(&bars[3 * STAGES]), convdone = d1full + 8;
-  const uint32_t d2full0 = d1full + 16, d2empty0 = d1full + 32;
+  const uint32_t d1full0 = smem_u32(&bars[3 * STAGES]), convdone = d1full0 + 16;
+  const uint32_t d2full = d1full0 + 24, d2empty = d1full0 + 32;
   const int n_items = p.nbi * p.nbj;
+  const int n_local = (int)blockIdx.x < n_items ? (n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;   // this CTA's tiles
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -85,9 +100,11 @@ tc_block2_kernel(const __grid_constant__ CUtensorMap mapL, const __grid_constant
       mbar_init(split0 + 8 * s, 4);
       mbar_init(empty0 + 8 * s, 1);
     }
-    mbar_init(d1full, 1);
+    mbar_init(d1full0, 1);
+    mbar_init(d1full0 + 8, 1);
     mbar_init(convdone, 4);
-    for (int s = 0; s < 2; ++s) { mbar_init(d2full0 + 8 * s, 1); mbar_init(d2empty0 + 8 * s, 4); }
+    mbar_init(d2full, 1);
+    mbar_init(d2empty, 4);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -107,21 +124,24 @@ tc_block2_kernel(const __grid_constant__ CUtensorMap mapL, const __grid_constant
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0; long long issued = 0;
       bool ok = true;
-      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+      for (int o = 0; o < 2 * n_local && ok; ++o) {
+        bool second; int t;
+        schedule_step(o, n_local, second, t);
+        const int item = (int)blockIdx.x + t * (int)gridDim.x;
         const int i = item / p.nbj, j = item - i * p.nbj;
-        for (int c8 = 0; c8 < 8; ++c8) {
+        for (int kc = 0; kc < 4; ++kc) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abortp, p.status)) { ok = false; break; }
           const uint32_t fb = full0 + 8 * stage;
           const uint32_t dst = smem_u32(smem + (size_t)stage * STAGE_BYTES);
-          if (c8 < 4) {
+          if (!second) {
             // product 1: Lop_i[:, 32 kc ..] and X_ij[32 kc .., :]
             mbar_expect_tx(fb, 2 * OP_BYTES);
-            load_block_chunk(dst, &mapL, p.l_mn, TILE * i, 0, c8, fb);
-            load_block_chunk(dst + 2 * OP_BYTES, &mapX, 1, TILE * i, TILE * j, c8, fb);
+            load_block_chunk(dst, &mapL, p.l_mn, TILE * i, 0, kc, fb);
+            load_block_chunk(dst + 2 * OP_BYTES, &mapX, 1, TILE * i, TILE * j, kc, fb);
           } else {
             // product 2: Rop_j[32 kc .., :]
             mbar_expect_tx(fb, OP_BYTES);
-            load_block_chunk(dst + 2 * OP_BYTES, &mapR, p.r_mn, TILE * j, 0, c8 - 4, fb);
+            load_block_chunk(dst + 2 * OP_BYTES, &mapR, p.r_mn, TILE * j, 0, kc, fb);
           }
           ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -148,57 +168,61 @@ tc_block2_kernel(const __grid_constant__ CUtensorMap mapL, const __grid_constant
       const uint64_t dr0 = op_desc(smem_u32(smem) + 2 * OP_BYTES, p.r_mn);
       const uint64_t kinc_a = p.l_mn ? (1024u >> 4) : (32u >> 4), kinc_x = 1024u >> 4;
       const uint64_t kinc_r = p.r_mn ? (1024u >> 4) : (32u >> 4);
-      const uint32_t d1 = tmem_base + T_D1, d1lo = tmem_base + T_D1LO;
+      const uint32_t d1lo = tmem_base + T_D1LO, d2 = tmem_base + T_D2;
       int stage = 0; uint32_t phase = 0;
-      uint32_t local = 0;
       bool ok = true;
-      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++local) {
-        // ---- product 1: D1 = Lop_i X_ij  (low part of Lop first, as in the one-sided kernel)
-        for (int kc = 0; kc < 4; ++kc) {
-          if (!mbar_wait(split0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
-          tc_fence_after();
-          const uint64_t so = (uint64_t)(uint32_t)(stage * (STAGE_BYTES >> 4));
-          const uint64_t da = da0 + so, dal = da + (OP_BYTES >> 4), dx = dx0 + so, dxl = dx + (OP_BYTES >> 4);
-          umma_tf32(d1, dal, dx, idesc1, (uint32_t)(kc > 0));
-          umma_tf32_acc(d1, da, dxl, idesc1);
-          umma_tf32_acc(d1, da, dx, idesc1);
+      for (int o = 0; o < 2 * n_local && ok; ++o) {
+        bool second; int t;
+        schedule_step(o, n_local, second, t);
+        const uint32_t d1 = tmem_base + T_D1 + (uint32_t)((t & 1) * TILE);
+        if (!second) {
+          // ---- product 1 of tile t: D1[t % 2] = Lop_i X_ij  (low part of Lop first, as in the one-sided kernel).  The
+          // buffer was last read by product 2 of tile t - 2, which precedes this point in the pipe's order.
+          for (int kc = 0; kc < 4; ++kc) {
+            if (!mbar_wait(split0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
+            tc_fence_after();
+            const uint64_t so = (uint64_t)(uint32_t)(stage * (STAGE_BYTES >> 4));
+            const uint64_t da = da0 + so, dal = da + (OP_BYTES >> 4), dx = dx0 + so, dxl = dx + (OP_BYTES >> 4);
+            umma_tf32(d1, dal, dx, idesc1, (uint32_t)(kc > 0));
+            umma_tf32_acc(d1, da, dxl, idesc1);
+            umma_tf32_acc(d1, da, dx, idesc1);
 #pragma unroll
-          for (int k = 1; k < BK / 8; ++k) {
-            umma_tf32_acc(d1, dal + k * kinc_a, dx + k * kinc_x, idesc1);
-            umma_tf32_acc(d1, da + k * kinc_a, dxl + k * kinc_x, idesc1);
-            umma_tf32_acc(d1, da + k * kinc_a, dx + k * kinc_x, idesc1);
+            for (int k = 1; k < BK / 8; ++k) {
+              umma_tf32_acc(d1, dal + k * kinc_a, dx + k * kinc_x, idesc1);
+              umma_tf32_acc(d1, da + k * kinc_a, dxl + k * kinc_x, idesc1);
+              umma_tf32_acc(d1, da + k * kinc_a, dx + k * kinc_x, idesc1);
+            }
+            umma_commit(empty0 + 8 * stage);
+            if (++stage == STAGES) { stage = 0; phase ^= 1; }
           }
-          umma_commit(empty0 + 8 * stage);
-          if (++stage == STAGES) { stage = 0; phase ^= 1; }
-        }
-        if (!ok) break;
-        umma_commit(d1full);
-        // ---- D1 is split by warps 10-13; D2[as] has been drained by the epilogue of two tiles ago
-        const uint32_t as = local & 1u;
-        if (!mbar_wait(convdone, local & 1u, abortp, p.status)) { ok = false; break; }
-        if (!mbar_wait(d2empty0 + 8 * as, ((local >> 1) & 1u) ^ 1u, abortp, p.status)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t d2 = tmem_base + T_D2 + as * (uint32_t)TILE;
-        // ---- product 2: D2 = D1 Rop_j, D1 from tensor memory (its low part first: the M side of this product)
-        for (int kc = 0; kc < 4; ++kc) {
-          if (!mbar_wait(split0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
+          if (!ok) break;
+          umma_commit(d1full0 + 8 * (t & 1));
+        } else {
+          // ---- product 2 of tile t: D2 = D1[t % 2] Rop_j, D1 from tensor memory (its low part first: the M side of this
+          // product).  Warps 10-13 have split D1; the epilogue has drained D2 of tile t - 1.
+          if (!mbar_wait(convdone, (uint32_t)t & 1u, abortp, p.status)) { ok = false; break; }
+          if (t > 0 && !mbar_wait(d2empty, (uint32_t)(t - 1) & 1u, abortp, p.status)) { ok = false; break; }
           tc_fence_after();
-          const uint64_t dr = dr0 + (uint64_t)(uint32_t)(stage * (STAGE_BYTES >> 4)), drl = dr + (OP_BYTES >> 4);
-          const uint32_t a_hi = d1 + (uint32_t)(kc * BK), a_lo = d1lo + (uint32_t)(kc * BK);
-          umma_tf32_ta(d2, a_lo, dr, idesc2, (uint32_t)(kc > 0));
-          umma_tf32_ta_acc(d2, a_hi, drl, idesc2);
-          umma_tf32_ta_acc(d2, a_hi, dr, idesc2);
+          for (int kc = 0; kc < 4; ++kc) {
+            if (!mbar_wait(split0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
+            tc_fence_after();
+            const uint64_t dr = dr0 + (uint64_t)(uint32_t)(stage * (STAGE_BYTES >> 4)), drl = dr + (OP_BYTES >> 4);
+            const uint32_t a_hi = d1 + (uint32_t)(kc * BK), a_lo = d1lo + (uint32_t)(kc * BK);
+            umma_tf32_ta(d2, a_lo, dr, idesc2, (uint32_t)(kc > 0));
+            umma_tf32_ta_acc(d2, a_hi, drl, idesc2);
+            umma_tf32_ta_acc(d2, a_hi, dr, idesc2);
 #pragma unroll
-          for (int k = 1; k < BK / 8; ++k) {
-            umma_tf32_ta_acc(d2, a_lo + 8 * k, dr + k * kinc_r, idesc2);
-            umma_tf32_ta_acc(d2, a_hi + 8 * k, drl + k * kinc_r, idesc2);
-            umma_tf32_ta_acc(d2, a_hi + 8 * k, dr + k * kinc_r, idesc2);
+            for (int k = 1; k < BK / 8; ++k) {
+              umma_tf32_ta_acc(d2, a_lo + 8 * k, dr + k * kinc_r, idesc2);
+              umma_tf32_ta_acc(d2, a_hi + 8 * k, drl + k * kinc_r, idesc2);
+              umma_tf32_ta_acc(d2, a_hi + 8 * k, dr + k * kinc_r, idesc2);
+            }
+            umma_commit(empty0 + 8 * stage);
+            if (++stage == STAGES) { stage = 0; phase ^= 1; }
           }
-          umma_commit(empty0 + 8 * stage);
-          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+          if (!ok) break;
+          umma_commit(d2full);      // D2 is complete; the low part of D1 may be overwritten
         }
-        if (!ok) break;
-        umma_commit(d2full0 + 8 * as);
       }
     }
   } else if (warp < 6) {
@@ -206,13 +230,15 @@ tc_block2_kernel(const __grid_constant__ CUtensorMap mapL, const __grid_constant
     const int t = threadIdx.x - 64;   // 0..127
     int stage = 0; uint32_t phase = 0;
     bool ok = true;
-    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-      for (int c8 = 0; c8 < 8; ++c8) {
+    for (int o = 0; o < 2 * n_local && ok; ++o) {
+      bool second; int tt;
+      schedule_step(o, n_local, second, tt);
+      for (int kc = 0; kc < 4; ++kc) {
         if (!mbar_wait(full0 + 8 * stage, phase, abortp, p.status)) { ok = false; break; }
         float4* base = reinterpret_cast<float4*>(smem + (size_t)stage * STAGE_BYTES);
 #pragma unroll
         for (int op = 0; op < 2; ++op) {
-          if (op == 0 && c8 >= 4) continue;       // product 2 has no M-side chunk in shared memory
+          if (op == 0 && second) continue;        // product 2 has no M-side chunk in shared memory
           float4* hi = base + op * (2 * OP_BYTES / 16);
           float4* lo = hi + OP_BYTES / 16;
 #pragma unroll
@@ -243,7 +269,6 @@ tc_block2_kernel(const __grid_constant__ CUtensorMap mapL, const __grid_constant
     const uint32_t buf_u32 = smem_u32(buf);
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++local) {
       const int i = item / p.nbj, j = item - i * p.nbj;
-      const uint32_t as = local & 1u;
       const int64_t row_base = (int64_t)TILE * i + q * 32;
       const int64_t col_tile = (int64_t)TILE * j;
       // The warp's 32 x 128 slab goes through shared memory in two halves of 64 columns (two 32 x 32 boxes).
@@ -252,13 +277,13 @@ tc_block2_kernel(const __grid_constant__ CUtensorMap mapL, const __grid_constant
         if (lane == 0) tma_store_wait_read();        // the previous stores have read the staging boxes
         __syncwarp();
         if (hf == 0) {
-          if (!__all_sync(0xffffffffu, mbar_wait(d2full0 + 8 * as, (local >> 1) & 1u, abortp, p.status))) { ok = false; break; }
+          if (!__all_sync(0xffffffffu, mbar_wait(d2full, local & 1u, abortp, p.status))) { ok = false; break; }
           tc_fence_after();
         }
 #pragma unroll 1
         for (int ch = 0; ch < 2; ++ch) {
           uint32_t r[32];
-          tmem_ld32(tmem_base + T_D2 + as * (uint32_t)TILE + (uint32_t)(hf * 64 + ch * 32) + ((uint32_t)(q * 32) << 16), r);
+          tmem_ld32(tmem_base + T_D2 + (uint32_t)(hf * 64 + ch * 32) + ((uint32_t)(q * 32) << 16), r);
           // lane = row of the box; 16-byte chunk c of the row sits at chunk c ^ (row % 8)  (128-byte swizzle)
           uint8_t* rowp = buf + ch * 4096 + lane * 128;
 #pragma unroll
@@ -272,7 +297,7 @@ tc_block2_kernel(const __grid_constant__ CUtensorMap mapL, const __grid_constant
         fence_proxy_async();
         __syncwarp();
         if (lane == 0) {
-          if (hf == 1) mbar_arrive(d2empty0 + 8 * as);
+          if (hf == 1) mbar_arrive(d2empty);
           for (int ch = 0; ch < 2; ++ch)
             tma_store_2d(&mapC, (int)(col_tile + 64 * hf + 32 * ch), (int)row_base, buf_u32 + ch * 4096);
           tma_store_commit();
@@ -287,12 +312,14 @@ tc_block2_kernel(const __grid_constant__ CUtensorMap mapL, const __grid_constant
     uint32_t local = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++local) {
-      if (!__all_sync(0xffffffffu, mbar_wait(d1full, local & 1u, abortp, p.status))) { ok = false; break; }
+      // product 1 of this tile has finished, and product 2 of the tile before has read the low part that is overwritten now
+      if (!__all_sync(0xffffffffu, mbar_wait(d1full0 + 8 * (local & 1u), (local >> 1) & 1u, abortp, p.status))) { ok = false; break; }
+      if (local > 0 && !__all_sync(0xffffffffu, mbar_wait(d2full, (local - 1) & 1u, abortp, p.status))) { ok = false; break; }
       tc_fence_after();
 #pragma unroll 1
       for (int g = 0; g < 4; ++g) {
         uint32_t r[32];
-        tmem_ld32(tmem_base + T_D1 + (uint32_t)(32 * g) + lane_sel, r);
+        tmem_ld32(tmem_base + T_D1 + (uint32_t)((local & 1u) * TILE + 32 * g) + lane_sel, r);
 #pragma unroll
         for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) - __uint_as_float(r[e] & 0xffffe000u));
         tmem_st32(tmem_base + T_D1LO + (uint32_t)(32 * g) + lane_sel, r);
