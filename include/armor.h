@@ -125,7 +125,8 @@ armor_status armor_workspace_bytes(const armor_config* cfg, size_t* bytes);
 
 /* Creates a context over caller-owned device scratch (256-byte aligned, at
  * least armor_workspace_bytes).  The context holds the configuration and the
- * carve-up of the workspace only.  Must be called with the device current. */
+ * carve-up of the workspace only, plus two non-blocking streams and a few events of its own (graph capture of the
+ * iterations, staging of the Gram).  Must be called with the device current. */
 armor_status armor_create(armor_ctx** ctx, const armor_config* cfg, void* d_workspace, size_t bytes);
 armor_status armor_destroy(armor_ctx* ctx);
 
@@ -134,7 +135,10 @@ armor_status armor_destroy(armor_ctx* ctx);
  * dimension ldx (elements).  The caller zeroes d_H before the first chunk.
  * x_dtype: ARMOR_DTYPE_F32 or ARMOR_DTYPE_BF16 (bf16 values are exact tensor-core
  * operands, so their Gram needs one pass in every tensor-core precision; not
- * available with ARMOR_PREC_SIMT).  n_rows == 0 is a no-op. */
+ * available with ARMOR_PREC_SIMT).  n_rows == 0 is a no-op.  A chunk is worked through in pieces of 16,384 rows
+ * (transposed, scaled and split into a staging buffer, then contracted); with ARMOR_PREC_FP16X3 a call of several
+ * pieces stages piece p + 1 on a stream of the context's own while piece p is contracted on `stream` (the result does
+ * not depend on it; the call returns with all of its work ordered before later work on `stream`, as always). */
 armor_status armor_gram(armor_ctx* ctx, const void* d_X, int32_t x_dtype, int64_t n_rows, int64_t ldx,
                         float* d_H, armor_stream_t stream);
 

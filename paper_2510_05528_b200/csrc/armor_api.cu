@@ -98,6 +98,7 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
     const int64_t dmax = cfg.d_out > cfg.d_in ? cfg.d_out : cfg.d_in;
     TAKE(hpow, float*, (size_t)cfg.d_in * sizeof(float));
     TAKE(gscale, float*, (size_t)cfg.d_in * sizeof(float));
+    TAKE(gscale2, float*, (size_t)cfg.d_in * sizeof(float));
     TAKE(gmax, unsigned*, (size_t)cfg.d_in * sizeof(unsigned));
     TAKE(rowscale, float*, (size_t)dmax * sizeof(float));
     TAKE(rowscale2, float*, (size_t)dmax * sizeof(float));
@@ -108,7 +109,8 @@ size_t carve(const armor_config& cfg, armor_ctx* c, char* base) {
     TAKE(Xt_hi, float*, (size_t)cfg.d_in * GRAM_ROWS * sizeof(float));
     // (the fp16 mode keeps both 16-bit parts of the staged chunk in Xt_hi)
     if (cfg.precision == ARMOR_PREC_FP32X3) TAKE(Xt_lo, float*, (size_t)cfg.d_in * GRAM_ROWS * sizeof(float)); else if (c) c->Xt_lo = nullptr;
-  } else if (c) { c->Xt_hi = nullptr; c->Xt_lo = nullptr; c->gemm_slabs = nullptr; c->gemm_slab_count = 0; }
+    if (cfg.precision == ARMOR_PREC_FP16X3) TAKE(Xt_hi2, float*, (size_t)cfg.d_in * GRAM_ROWS * sizeof(float)); else if (c) c->Xt_hi2 = nullptr;
+  } else if (c) { c->Xt_hi = nullptr; c->Xt_lo = nullptr; c->Xt_hi2 = nullptr; c->gemm_slabs = nullptr; c->gemm_slab_count = 0; }
   const int64_t tiles = ((cfg.d_out + 127) / 128) * ((cfg.d_in + 127) / 128) + ((cfg.d_in + 127) / 128) * ((cfg.d_in + 127) / 128);
   const int64_t npart = tiles > ARMOR_DOT_BLOCKS ? tiles : ARMOR_DOT_BLOCKS;
   {
@@ -309,6 +311,18 @@ armor_status armor_create(armor_ctx** out, const armor_config* cfg, void* d_work
   c->cap_split = 0; c->cap_n = 0; c->cap_failed = 0;
   c->cap_stream = nullptr;
   if (cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking) != cudaSuccess) c->cap_stream = nullptr;
+  // a second stream of the context's own and five events: the Gram stages chunk p + 1 there while chunk p is contracted
+  c->side_stream = nullptr;
+  c->ev_fork = nullptr;
+  for (int k = 0; k < 2; ++k) { c->ev_staged[k] = nullptr; c->ev_used[k] = nullptr; }
+  {
+    bool ok = cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
+    for (int k = 0; k < 2 && ok; ++k)
+      ok = cudaEventCreateWithFlags(&c->ev_staged[k], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&c->ev_used[k], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok && c->side_stream) { cudaStreamDestroy(c->side_stream); c->side_stream = nullptr; }   // the Gram then runs in one stream
+  }
   c->kg = cfg->mask_groups > 0 ? cfg->mask_groups : 1;
   c->h_cached = nullptr;
   c->timing_on = 0; c->timing_n = 0; c->ev_beg = nullptr; c->ev_end = nullptr; c->ev_cls = nullptr; c->ev_work = nullptr;
@@ -328,6 +342,12 @@ armor_status armor_destroy(armor_ctx* c) {
   delete[] c->ev_cls;
   delete[] c->ev_work;
   if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
+  if (c->side_stream) cudaStreamDestroy(c->side_stream);
+  if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  for (int k = 0; k < 2; ++k) {
+    if (c->ev_staged[k]) cudaEventDestroy(c->ev_staged[k]);
+    if (c->ev_used[k]) cudaEventDestroy(c->ev_used[k]);
+  }
   delete c;
   return ARMOR_OK;
 }

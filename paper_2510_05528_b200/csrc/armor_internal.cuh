@@ -88,9 +88,13 @@ struct armor_ctx {
   // three-pass fp16 mode: column scales derived from diag(H), per-row output scales of the two operands,
   // per-channel maxima and output scales of a Gram chunk
   float *hpow, *rowscale, *rowscale2, *gscale;
+  float* gscale2;       // output scales of the chunk staged in Xt_hi2
   unsigned* gmax;
   // Gram staging (transposed, split chunk of X)
   float *Xt_hi, *Xt_lo;
+  float* Xt_hi2;        // second staging buffer (FP16X3): chunk p + 1 is staged on side_stream while chunk p is contracted
+  cudaStream_t side_stream;
+  cudaEvent_t ev_fork, ev_staged[2], ev_used[2];
   int64_t gram_rows;  // rows of X staged per pass
   double* sc;         // [SC_COUNT]
   double* partials;   // [2][8 * npart] partial sums of the fused / streaming reductions
@@ -298,7 +302,7 @@ void launch_f16_split_rows(armor_ctx* c, const float* in, int64_t ld, int64_t ro
                            float post, void* hi, void* lo, float* out_scale, cudaStream_t s);
 float f16_H_post_scale();
 armor_status launch_f16_gram_stage(armor_ctx* c, const void* X, int x_dtype, int64_t ldx, int64_t rows, int64_t cols,
-                                   void* Thi, void* Tlo, int64_t ldt, cudaStream_t s);
+                                   void* Thi, void* Tlo, int64_t ldt, float* gscale, cudaStream_t s);
 
 // deterministic reductions (two stages, fixed order)
 void dot_to_ptr(armor_ctx* c, const float* x, const float* y, int64_t n, double* out, cudaStream_t s);

@@ -103,27 +103,51 @@ armor_status gram_accumulate(armor_ctx* c, const void* Xv, int x_dtype, int64_t 
   }
   if (c->cfg.precision == ARMOR_PREC_FP16X3) {
     // every chunk is scaled per channel into the fp16 range; bf16 activations are then exact in one fp16 part
-    __half* thi = reinterpret_cast<__half*>(c->Xt_hi);
-    __half* tlo = thi + d_in * c->gram_rows;
     const size_t esz = bf16 ? 2 : 4;
-    for (int64_t r0 = 0; r0 < n_rows; r0 += c->gram_rows) {
+    // A call of several chunks stages chunk p + 1 (HBM bound) on the context's side stream while the tensor cores
+    // contract chunk p on the caller's stream: two staging buffers with their scales, an event per hand-over.  The
+    // contractions stay in the caller's stream in chunk order, so H is the same bit for bit.
+    const int64_t n_chunks = (n_rows + c->gram_rows - 1) / c->gram_rows;
+    bool overlap = n_chunks > 1 && c->side_stream && c->Xt_hi2 && c->timing_on < 2;
+    if (overlap) {
+      cudaStreamCaptureStatus cst = cudaStreamCaptureStatusNone;
+      if (cudaStreamIsCapturing(s, &cst) != cudaSuccess || cst != cudaStreamCaptureStatusNone) overlap = false;
+    }
+    if (overlap) {
+      // the side stream starts where the caller's stream is now: the inputs are ready and both buffers are free
+      if (cudaEventRecord(c->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(c->side_stream, c->ev_fork, 0) != cudaSuccess)
+        return ARMOR_ERR_CUDA;
+    }
+    int64_t p = 0;
+    for (int64_t r0 = 0; r0 < n_rows; r0 += c->gram_rows, ++p) {
+      const int b = overlap ? (int)(p & 1) : 0;
+      __half* thi = reinterpret_cast<__half*>(b ? c->Xt_hi2 : c->Xt_hi);
+      __half* tlo = thi + d_in * c->gram_rows;
+      float* gscale = b ? c->gscale2 : c->gscale;
+      cudaStream_t ss = overlap ? c->side_stream : s;
       const int64_t n = n_rows - r0 < c->gram_rows ? n_rows - r0 : c->gram_rows;
       const int64_t kpad = (n + 63) / 64 * 64;
+      // buffer b was last read by the contraction of chunk p - 2
+      if (overlap && p >= 2 && cudaStreamWaitEvent(ss, c->ev_used[b], 0) != cudaSuccess) return ARMOR_ERR_CUDA;
       armor_status st = launch_f16_gram_stage(c, static_cast<const char*>(Xv) + (size_t)(r0 * ldx) * esz, x_dtype, ldx, n,
-                                              d_in, thi, tlo, kpad, s);
+                                              d_in, thi, tlo, kpad, gscale, ss);
       if (st != ARMOR_OK) return st;
+      if (overlap && (cudaEventRecord(c->ev_staged[b], ss) != cudaSuccess ||
+                      cudaStreamWaitEvent(s, c->ev_staged[b], 0) != cudaSuccess))
+        return ARMOR_ERR_CUDA;
       TcGemm g{};
       g.A = thi; g.Alo = tlo; g.lda = kpad;
       g.B = thi; g.Blo = tlo; g.ldb = kpad;
       g.C = H; g.ldc = d_in;
       g.M = d_in; g.N = d_in; g.K = kpad;
       g.passes = bf16 ? 0 : 6; g.fp16 = 1;
-      g.row_scale = c->gscale; g.col_scale = c->gscale;
+      g.row_scale = gscale; g.col_scale = gscale;
       g.accumulate = 1;
       g.symmetric_lower = 1;
       g.k_segment = K_SEGMENT;
       st = launch_tc_gemm(c, g, nullptr, s);
       if (st != ARMOR_OK) return st;
+      if (overlap && cudaEventRecord(c->ev_used[b], s) != cudaSuccess) return ARMOR_ERR_CUDA;
     }
     launch_mirror_lower(c, H, d_in, s);
     return ARMOR_OK;

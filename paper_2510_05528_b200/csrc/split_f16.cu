@@ -219,7 +219,7 @@ void launch_f16_split_rows(armor_ctx* c, const float* in, int64_t ld, int64_t ro
 float f16_H_post_scale() { return 1.f / (float)(1 << H_SHIFT); }
 
 armor_status launch_f16_gram_stage(armor_ctx* c, const void* X, int x_dtype, int64_t ldx, int64_t rows, int64_t cols,
-                                   void* Thi, void* Tlo, int64_t ldt, cudaStream_t s) {
+                                   void* Thi, void* Tlo, int64_t ldt, float* gscale, cudaStream_t s) {
   if (cudaMemsetAsync(c->gmax, 0, (size_t)cols * sizeof(unsigned), s) != cudaSuccess) return ARMOR_ERR_CUDA;
   // one read for the maxima, one read and one 16-bit write per part for the staged chunk
   KTimer kt(c, ARMOR_KC_GRAM_STAGING, (double)rows * (double)cols * (x_dtype == ARMOR_DTYPE_BF16 ? 6.0 : 12.0), s);
@@ -236,7 +236,7 @@ armor_status launch_f16_gram_stage(armor_ctx* c, const void* X, int x_dtype, int
     transpose_split_f16_kernel<<<g2, 256, 0, s>>>(Xf, ldx, rows, cols, c->gmax, static_cast<__half*>(Thi),
                                                          static_cast<__half*>(Tlo), ldt);
   }
-  gram_scale_kernel<<<(unsigned)((cols + 255) / 256), 256, 0, s>>>(c->gmax, c->gscale, cols);
+  gram_scale_kernel<<<(unsigned)((cols + 255) / 256), 256, 0, s>>>(c->gmax, gscale, cols);
   c->launches += 3;
   return ARMOR_OK;
 }

@@ -128,3 +128,23 @@ def test_fused_gram_pairs_are_bit_identical_to_separate_launches(cfg, mode):
     if mode != "full-adam":
         assert g[5] < d[5]                       # fewer launches
     assert d[6] == g[6] == [0, 0, 0, 0]
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["fp32", "bf16"])
+def test_gram_with_overlapped_staging_matches_chunk_by_chunk_calls(dtype):
+    """One armor_gram call over several staging chunks stages chunk p + 1 on the context's side stream while chunk p is
+    contracted; the contractions keep their order, so H equals, bit for bit, the H of one call per chunk (which runs in
+    one stream), and both agree with the fp64 Gram."""
+    d_in, rows, chunk = 512, 3 * 16384 + 1000, 16384            # four staging chunks, the last one ragged
+    g = torch.Generator(device=DEV); g.manual_seed(5)
+    X = (torch.randn(rows, d_in, device=DEV, generator=g) * torch.exp(torch.randn(d_in, device=DEV, generator=g))).to(dtype)
+    ctx = Bd.ArmorContext(256, d_in, 128, device=DEV, precision=Bd.PREC_FP16X3)
+    H1 = ctx.new_gram(); ctx.gram(X, H1)
+    H2 = ctx.new_gram()
+    for lo in range(0, rows, chunk):
+        ctx.gram(X[lo: lo + chunk], H2)
+    torch.cuda.synchronize()
+    assert torch.equal(H1, H2)
+    ref = O.gram(X.float().cpu().numpy())
+    assert np.linalg.norm(host(H1) - ref) <= 2e-5 * np.linalg.norm(ref)
+    assert ctx.device_status()[:4] == [0, 0, 0, 0]
