@@ -583,8 +583,8 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       if (b_gd) launch_stage(c, is, 8, nullptr, 0, 0, s, c->partials, nq, SC_Q_B);
       else launch_stage(c, is, 2, c->partblk, nbi, nbi, s, c->partials, nq, SC_Q_B);
       launch_axpy_slot(c, B, c->Delta, (int64_t)nbi * db * db, SC_TAU_B, 1.f, s);    // B += tau Delta
-      launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_B, -1.f, s);                   // EH -= tau V H_w
-      if (carry_P) launch_axpy_slot(c, c->P, c->E, c->wn, SC_TAU_B, 1.f, s);         // P += tau R H_w
+      // EH -= tau V H_w and, where T H_w is carried, P += tau R H_w: one launch
+      launch_axpy_multi(c, c->EH, c->VH, -1.f, carry_P ? c->P : nullptr, c->E, 1.f, nullptr, nullptr, 0.f, c->wn, SC_TAU_B, s);
     } else if (!adam) {
       launch_stage(c, is, 2, nullptr, 0, 0, s);
     }
@@ -619,9 +619,8 @@ armor_status armor_bcd_step(armor_ctx* c, const float* W, const float* H, float*
       }
       launch_stage(c, is, beta_step ? 6 : 3, nullptr, 0, 0, s, beta_step ? nullptr : c->partials, nq, SC_Q_S,
                    nrm_part, ARMOR_DOT_BLOCKS, SC_NRM_S);
-      launch_axpy_slot(c, S, c->U, c->wn, SC_TAU_S, 1.f, s);                         // S += tau Gamma_M
-      launch_axpy_slot(c, c->EH, c->VH, c->wn, SC_TAU_S, -1.f, s);                   // EH -= tau V H_w
-      if (carry_P) launch_axpy_slot(c, c->P, c->E, c->wn, SC_TAU_S, 1.f, s);         // P += tau R H_w
+      // S += tau Gamma_M, EH -= tau V H_w and, where T H_w is carried, P += tau R H_w: one launch
+      launch_axpy_multi(c, S, c->U, 1.f, c->EH, c->VH, -1.f, carry_P ? c->P : nullptr, c->E, 1.f, c->wn, SC_TAU_S, s);
     } else if (!adam) {
       launch_stage(c, is, 3, nullptr, 0, 0, s);
     }

@@ -316,7 +316,9 @@ void launch_extract_hblocks(armor_ctx* c, const float* H, cudaStream_t s);   // 
 void launch_masked_copy(armor_ctx* c, const float* Gam, const uint8_t* M, float* out, double* part,
                         cudaStream_t s);              // out = Gam (.) M; ARMOR_DOT_BLOCKS partial sums of ||out||^2
 void launch_axpy_slot(armor_ctx* c, float* y, const float* x, int64_t n, int slot, float sign,
-                      cudaStream_t s);                                       // y += sign * sc[slot] * x
+                      cudaStream_t s);
+void launch_axpy_multi(armor_ctx* c, float* y0, const float* x0, float s0, float* y1, const float* x1, float s1, float* y2,
+                       const float* x2, float s2, int64_t n, int slot, cudaStream_t s);                                       // y += sign * sc[slot] * x
 void launch_init(armor_ctx* c, const float* W, const float* H, float* Wbar, float* r1, float* r2,
                  float* A, float* B, float* S, uint8_t* M, cudaStream_t s);
 // st: base of the iteration records (the kernels add c->it_dev), or null

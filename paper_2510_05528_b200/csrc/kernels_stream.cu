@@ -128,6 +128,24 @@ __global__ void __launch_bounds__(NT) axpy_slot_kernel(float4* __restrict__ y, c
   }
 }
 
+// the same for up to three arrays of one length that move by the same step: one launch
+struct AxpyTerm { float4* y; const float4* x; float sign; };
+__global__ void __launch_bounds__(NT) axpy_multi_slot_kernel(AxpyTerm t0, AxpyTerm t1, AxpyTerm t2, int n_terms, int64_t n4,
+                                                             const double* __restrict__ sc, int slot) {
+  const float a = (float)sc[slot];
+  if (a == 0.f) return;
+  const AxpyTerm t[3] = {t0, t1, t2};
+  for (int64_t i = (int64_t)blockIdx.x * NT + threadIdx.x; i < n4; i += (int64_t)gridDim.x * NT) {
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+      if (k >= n_terms) break;
+      const float ak = t[k].sign * a;
+      const float4 u = t[k].y[i], v = t[k].x[i];
+      t[k].y[i] = make_float4(fmaf(ak, v.x, u.x), fmaf(ak, v.y, u.y), fmaf(ak, v.z, u.z), fmaf(ak, v.w, u.w));
+    }
+  }
+}
+
 // ---- normalisation (Section 3.2): r1 = column norms, r2 = row norms of W / r1 -------------------
 constexpr int COLSUM_CHUNKS = 64;
 __global__ void __launch_bounds__(NT) colsumsq_partial_kernel(const float* __restrict__ W, int64_t rows, int64_t cols,
@@ -587,6 +605,21 @@ void launch_masked_copy(armor_ctx* c, const float* Gam, const uint8_t* M, float*
 void launch_axpy_slot(armor_ctx* c, float* y, const float* x, int64_t n, int slot, float sign, cudaStream_t s) {
   KTimer kt(c, n >= (1 << 22) ? ARMOR_KC_AXPY : ARMOR_KC_SMALL, 12.0 * (double)n, s);
   axpy_slot_kernel<<<grid_for(n / 4), NT, 0, s>>>((float4*)y, (const float4*)x, n / 4, c->sc, slot, sign);
+  c->launches++;
+}
+
+// y_k += sign_k * sc[slot] * x_k for up to three pairs of length n (a pair with y == nullptr is skipped)
+void launch_axpy_multi(armor_ctx* c, float* y0, const float* x0, float s0, float* y1, const float* x1, float s1, float* y2,
+                       const float* x2, float s2, int64_t n, int slot, cudaStream_t s) {
+  AxpyTerm t[3];
+  int k = 0;
+  if (y0) t[k++] = {(float4*)y0, (const float4*)x0, s0};
+  if (y1) t[k++] = {(float4*)y1, (const float4*)x1, s1};
+  if (y2) t[k++] = {(float4*)y2, (const float4*)x2, s2};
+  if (k == 0) return;
+  for (int j = k; j < 3; ++j) t[j] = t[0];
+  KTimer kt(c, n >= (1 << 22) ? ARMOR_KC_AXPY : ARMOR_KC_SMALL, 12.0 * (double)n * k, s);
+  axpy_multi_slot_kernel<<<grid_for(n / 4), NT, 0, s>>>(t[0], t[1], t[2], k, n / 4, c->sc, slot);
   c->launches++;
 }
 
