@@ -502,14 +502,51 @@ __global__ void __launch_bounds__(NT) mask_carry_kernel(const SelRec* __restrict
   const int bi = blockIdx.x;
   const int64_t c4 = (int64_t)blockIdx.y * 1024 + 4 * threadIdx.x;
   if (c4 >= d_in) return;
-  for (int j = 0; j < nbv; ++j) {                            // virtual column blocks in order: deterministic sums
-    const SelRec rec = sel[bi * nbv + j];
-    if (!rec.valid) continue;
-    const float4 y = *reinterpret_cast<const float4*>(Y + ((int64_t)j * nbo_pad + bi) * d_in + c4);
-    float4* dst = reinterpret_cast<float4*>(P + (int64_t)rec.row * d_in + c4);
-    float4 v = *dst;
-    v.x += y.x; v.y += y.y; v.z += y.z; v.w += y.w;
-    *dst = v;
+  // Virtual column blocks in order, eight at a time.  The eight rows are almost always distinct: then their loads are
+  // independent and issued together (a chain of 32 dependent read-modify-writes was the whole cost of this kernel);
+  // a batch in which two groups share a row is walked one by one, so that every element of P sees its additions in
+  // the order of the column blocks (deterministic sums).
+  for (int j0 = 0; j0 < nbv; j0 += 8) {
+    int row[8];
+    bool val[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      val[u] = false; row[u] = 0;
+      if (j0 + u < nbv) {
+        const SelRec* rec = sel + (bi * nbv + j0 + u);
+        val[u] = rec->valid != 0;
+        row[u] = rec->row;
+      }
+    }
+    bool shared_row = false;
+#pragma unroll
+    for (int u = 1; u < 8; ++u)
+#pragma unroll
+      for (int w = 0; w < u; ++w) shared_row |= val[u] && val[w] && row[u] == row[w];
+    if (!shared_row) {
+      float4 y[8], v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (val[u]) {
+          y[u] = *reinterpret_cast<const float4*>(Y + ((int64_t)(j0 + u) * nbo_pad + bi) * d_in + c4);
+          v[u] = *reinterpret_cast<const float4*>(P + (int64_t)row[u] * d_in + c4);
+        }
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (val[u]) {
+          v[u].x += y[u].x; v[u].y += y[u].y; v[u].z += y[u].z; v[u].w += y[u].w;
+          *reinterpret_cast<float4*>(P + (int64_t)row[u] * d_in + c4) = v[u];
+        }
+    } else {
+      for (int u = 0; u < 8; ++u) {
+        if (!val[u]) continue;
+        const float4 y = *reinterpret_cast<const float4*>(Y + ((int64_t)(j0 + u) * nbo_pad + bi) * d_in + c4);
+        float4* dst = reinterpret_cast<float4*>(P + (int64_t)row[u] * d_in + c4);
+        float4 v = *dst;
+        v.x += y.x; v.y += y.y; v.z += y.z; v.w += y.w;
+        *dst = v;
+      }
+    }
   }
 }
 
