@@ -265,30 +265,42 @@ __global__ void zero_scalars_kernel(double* sc, int32_t* failflag, int nflag, in
   if (carry_loss && st && threadIdx.x == 0) start_record(st, carried);
 }
 
-// Fixed-order sums by one warp: lane l adds entries l, l + 32, ...; then a shuffle tree.  All lanes get the sum.
-__device__ __forceinline__ double warp_sum_f64(const double* __restrict__ p, int n) {
-  // (eight loads in flight per lane; the additions keep their order)
+// Fixed-order sums by the CTA of the bookkeeping kernel (STAGE_NT threads): thread t adds entries t, t + STAGE_NT, ...
+// (eight loads in flight), a shuffle tree per warp, then the warps in order.  All threads get the sum.  The line
+// searches hand over thousands of partial sums (four or eight per tile); one warp took 14 us over them.
+constexpr int STAGE_NT = 256;
+__device__ __forceinline__ double stage_sum_f64(const double* __restrict__ p, int n, double* scratch) {
   double v = 0.0;
   int i = threadIdx.x;
-  for (; i + 7 * 32 < n; i += 8 * 32) {
+  for (; i + 7 * STAGE_NT < n; i += 8 * STAGE_NT) {
     double t[8];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) t[u] = p[i + 32 * u];
+    for (int u = 0; u < 8; ++u) t[u] = p[i + STAGE_NT * u];
 #pragma unroll
     for (int u = 0; u < 8; ++u) v += t[u];
   }
-  for (; i < n; i += 32) v += p[i];
+  for (; i < n; i += STAGE_NT) v += p[i];
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
+  if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+  __syncthreads();
+  double t = 0.0;
+  for (int w = 0; w < STAGE_NT / 32; ++w) t += scratch[w];
+  __syncthreads();
+  return t;
 }
-__device__ __forceinline__ int warp_count_flags(const int32_t* __restrict__ f, int n) {
+__device__ __forceinline__ int stage_count_flags(const int32_t* __restrict__ f, int n, double* scratch) {
   int v = 0;
-  for (int i = threadIdx.x; i < n; i += 32) v += f[i] ? 1 : 0;
+  for (int i = threadIdx.x; i < n; i += STAGE_NT) v += f[i] ? 1 : 0;
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
+  if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = (double)v;
+  __syncthreads();
+  int t = 0;
+  for (int w = 0; w < STAGE_NT / 32; ++w) t += (int)scratch[w];
+  __syncthreads();
+  return t;
 }
 
-// stage 0: start, 1: after A, 2: after B, 3 / 6: after S, 4: mask accept, 5: mask phase off.  One warp.
+// stage 0: start, 1: after A, 2: after B, 3 / 6: after S, 4: mask accept, 5: mask phase off.  One CTA of STAGE_NT threads.
 // Up to two arrays of partial sums (p1, p2) are first added, in a fixed order, into the scalars slot1 / slot2: the
 // reductions of the dot products that precede the stage need no launch of their own.
 __global__ void advance_iteration_kernel(int64_t* it_dev) { *it_dev += 1; }
@@ -298,13 +310,13 @@ __global__ void stage_kernel(double* sc, armor_iter_stats* st_base, const int64_
                              const double* partA, int nA, int32_t* status, const double* p1, int n1, int slot1,
                              const double* p2, int n2, int slot2) {
   armor_iter_stats* st = st_base ? st_base + *it_dev : nullptr;
-  if (p1) { const double v = warp_sum_f64(p1, n1); if (threadIdx.x == 0) sc[slot1] = v; }
-  if (p2) { const double v = warp_sum_f64(p2, n2); if (threadIdx.x == 0) sc[slot2] = v; }
-  __syncwarp();
+  __shared__ double scratch[STAGE_NT / 32];
+  if (p1) { const double v = stage_sum_f64(p1, n1, scratch); if (threadIdx.x == 0) sc[slot1] = v; }
+  if (p2) { const double v = stage_sum_f64(p2, n2, scratch); if (threadIdx.x == 0) sc[slot2] = v; }
   double psum = 0.0;
   int nf = 0;
-  if (stage == 1 || stage == 2 || stage == 4) psum = warp_sum_f64(partA, nA);
-  if (stage == 1 || stage == 2) nf = warp_count_flags(failflag, nflag);
+  if (stage == 1 || stage == 2 || stage == 4) psum = stage_sum_f64(partA, nA, scratch);
+  if (stage == 1 || stage == 2) nf = stage_count_flags(failflag, nflag, scratch);
   if (threadIdx.x != 0) return;
   const bool poisoned = status[ST_POISON] != 0;   // unusable inputs: every step length is zero, nothing is accepted
   if (stage == 0) {
@@ -680,7 +692,7 @@ void launch_advance_iteration(armor_ctx* c, cudaStream_t s) {
 void launch_stage(armor_ctx* c, armor_iter_stats* st, int stage, const double* part, int npart, int nflag,
                   cudaStream_t s, const double* p1, int n1, int slot1, const double* p2, int n2, int slot2) {
   KTimer kt(c, ARMOR_KC_SMALL, 0.0, s);
-  stage_kernel<<<1, 32, 0, s>>>(c->sc, st, c->it_dev, stage, c->failflag, nflag, part, npart, c->status, p1, n1, slot1,
+  stage_kernel<<<1, STAGE_NT, 0, s>>>(c->sc, st, c->it_dev, stage, c->failflag, nflag, part, npart, c->status, p1, n1, slot1,
                                p2, n2, slot2);
   c->launches++;
 }
